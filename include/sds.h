@@ -1,0 +1,200 @@
+/*
+ * sds.h - C ABI of libsds: speculative sampling for diffusion chains on one GPU.
+ *
+ * The library runs, for B independent chains, the draft-then-verify window of
+ * "Accelerated Diffusion Models via Speculative Sampling" (arxiv 2501.05370):
+ *   - target chain: Gaussian transitions N(m^q_k(y), sigma_k^2 I)                  (Eq. 3)
+ *   - frozen-target drafter: same transition with the denoiser output frozen       (Eq. 6 and the
+ *     "Efficient frozen draft strategy" paragraph of Appendix B)
+ *   - window loop: draft L steps, one batched target pass, sequential accept       (Algorithms 1, 4)
+ *   - accept test and adjusted law: reflection maximal coupling                    (Algorithm 3)
+ *   - Langevin variant: same loop with m = x - gamma grad E, sigma = sqrt(2 gamma) (Algorithm 5)
+ *
+ * Every transition mean is affine in (state, denoiser output): m_k(y, D) = a_k*y + c_k*D.
+ * The caller supplies a_k, c_k, sigma_k (k = 0..K-1 is the transition Y_k -> Y_{k+1}) and a denoiser.
+ *
+ * Conventions
+ *   - "dev" pointers are device pointers on the current CUDA device, "host" pointers are host
+ *     pointers. All are owned by the caller; the library neither frees nor allocates device memory.
+ *     Its only device storage is the workspace the caller binds (size from sds_workspace_bytes).
+ *   - Host arrays of sds_schedule are copied at sds_create. Device arrays named in sds_denoiser
+ *     must stay valid until sds_destroy.
+ *   - All work is enqueued on the stream given to sds_bind. Calls return after enqueueing except
+ *     sds_bind, sds_advance with a non-NULL n_active, sds_sample_all(_host), and sds_get with a host
+ *     destination, which wait for the stream.
+ *   - Every call returns SDS_OK (0) or a negative code; nothing throws across the boundary.
+ *     sds_last_cuda_error gives the CUDA error behind SDS_ECUDA.
+ *   - A context is used by one host thread at a time. Contexts are independent.
+ *   - Random numbers: Philox-4x32-10, counter (q, k, b_lo, stream + 256*b_hi), key = seed, where
+ *     q = element index / 4, k = transition index, b = global chain id (chain_id_offset + local
+ *     index). Stream 0 = draft noise, 1 = accept uniform, 2 = initial state. Results of a chain
+ *     therefore do not depend on which other chains share the context.
+ */
+#ifndef SDS_H_
+#define SDS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes ---- */
+#define SDS_OK            0
+#define SDS_EINVAL       (-1)   /* NULL pointer, B<=0, d<=0, L not in [1,32], non-finite schedule, sigma_k<=0 */
+#define SDS_ESTATE       (-2)   /* call order other than bind -> reset -> (draft -> verify_window -> advance)* */
+#define SDS_ENOMEM       (-3)   /* workspace too small or misaligned */
+#define SDS_EUNSUPPORTED (-4)   /* unknown denoiser kind / dtype / drafter mode, shape the kernels cannot take */
+#define SDS_ECUDA        (-5)   /* a CUDA call failed; see sds_last_cuda_error */
+#define SDS_ETIMEOUT     (-6)   /* a bounded device-side wait gave up */
+#define SDS_ENONFINITE   (-7)   /* some chain produced a non-finite log-ratio and was frozen; others valid */
+#define SDS_ECALLBACK    (-8)   /* the user denoiser callback returned non-zero */
+
+/* ---- denoiser kinds, dtypes, drafter modes, sds_get selectors ---- */
+#define SDS_DEN_GMM       1     /* closed-form Gaussian-mixture posterior mean / energy gradient */
+#define SDS_DEN_MLP       2     /* bf16 MLP with per-step embedding rows */
+#define SDS_DEN_CALLBACK  3     /* user function on device buffers */
+
+#define SDS_F32           0
+#define SDS_BF16          1
+
+#define SDS_FROZEN_PREV   0     /* drafter reuses the newest target output on the accepted path (no extra call) */
+
+#define SDS_GET_X         1     /* float  [nrows, d]  drafted states fed to the target (row r = rowoff[s]+j-1) */
+#define SDS_GET_TAIL      2     /* float  [B, d]      last drafted state of each chain's window */
+#define SDS_GET_DQ        3     /* float  [nrows, d]  target denoiser outputs, same rows as X */
+#define SDS_GET_DC        4     /* float  [B, d]      carried (frozen) denoiser output */
+#define SDS_GET_Y         5     /* float  [B, d]      current state Y_n */
+#define SDS_GET_N         6     /* int32  [B]         current index n_b */
+#define SDS_GET_ACT       7     /* int32  [B]         active chain ids, first n_active entries valid */
+#define SDS_GET_ROWOFF    8     /* int32  [B+1]       first row of each active slot; [n_active] = nrows */
+#define SDS_GET_S1        9     /* double [B, L]      |Delta|^2 per (chain, position) of the last verify */
+#define SDS_GET_S2        10    /* double [B, L]      Delta . Z */
+#define SDS_GET_ELL       11    /* float  [B, L]      log acceptance ratio */
+#define SDS_GET_LOGU      12    /* float  [B, L]      log of the accept uniform */
+#define SDS_GET_ACCMASK   13    /* uint32 [B]         bit j-1 set = position j accepted */
+#define SDS_GET_JSTAR     14    /* int32  [B]         first rejected position, Lt+1 if none */
+#define SDS_GET_NFE_CALLS 15    /* int32  [B]         sequential batched target calls the chain took part in */
+#define SDS_GET_NFE_ROWS  16    /* int32  [B]         target rows evaluated for the chain */
+#define SDS_GET_CTL       17    /* int32  [8]         n_active, nrows, windows done, error word, frozen chains, ... */
+#define SDS_GET_ROWK      18    /* int32  [nrows]     transition index of each row */
+
+typedef struct sds_ctx sds_ctx;   /* opaque, owned by the library */
+
+/* Transition schedule, caller-owned host arrays copied at create.
+ * mean_k(y, D) = a[k]*y + c[k]*D, std sigma[k] > 0 shared by target and drafter (the method needs
+ * equal covariances: Section 3.3 and the appendix on unequal variances).
+ * tcond: [K, tcond_dim] per-step scalars handed to the denoiser (GMM: 4 per step, see below). */
+typedef struct {
+  int32_t K;
+  const float* a;
+  const float* c;
+  const float* sigma;
+  const float* tcond;
+  int32_t tcond_dim;
+} sds_schedule;
+
+/* User denoiser: rows of x_dev [rows, d] (float, dense) at transition indices k_dev [rows] ->
+ * out_dev [rows, d]. Must enqueue on `stream` (a cudaStream_t) and return 0. */
+typedef int (*sds_denoise_fn)(void* user, const float* x_dev, const int32_t* k_dev, int64_t rows,
+                              int32_t d, float* out_dev, void* stream);
+
+/* Exactly one kind is used.
+ * GMM (mixture of ncomp isotropic Gaussians sharing one std): with tcond[k] = (A, Bq, C, E)
+ *     r = softmax_c( logw[c] + A * <x, mu_c> + Bq * |mu_c|^2 ),   D(x, k) = C * sum_c r_c mu_c + E * x.
+ *   Posterior mean E[x0 | x_t] of a variance-preserving forward process and the energy gradient of
+ *   the mixture both have this form (binding helpers compute the four scalars).
+ *   means_dev: [ncomp, d] float (SDS_F32) or bf16 (SDS_BF16; then <x,mu> and the mixing sum run on
+ *   tensor cores with x and r rounded to bf16). logw_dev: [ncomp] float.
+ * MLP: nlayer linear layers dims[0]=d -> ... -> dims[nlayer]=d.
+ *   h_l = SiLU(W_l h_{l-1} + bias_l + temb_l[k]) for l < nlayer, output = W_nlayer h + bias (float).
+ *   W_dev[l]: [dims[l+1], dims[l]] bf16 row-major; bias_dev[l]: [dims[l+1]] float;
+ *   temb_dev[l]: [K, dims[l+1]] bf16 (NULL for the last layer). Every dims[] a multiple of 128. */
+typedef struct {
+  int32_t kind;
+  int32_t ncomp;
+  const void* means_dev;
+  const float* logw_dev;
+  int32_t means_dtype;
+  int32_t nlayer;
+  const void* const* W_dev;
+  const float* const* bias_dev;
+  const void* const* temb_dev;
+  const int32_t* dims;
+  sds_denoise_fn fn;
+  void* user;
+} sds_denoiser;
+
+/* Bytes of device workspace sds_bind needs for this problem (256-byte aligned base required). */
+int sds_workspace_bytes(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_t d,
+                        int32_t L, size_t* bytes);
+
+/* Create a context for B chains of dimension d with window L (Algorithm 4's inputs L, K, p, q).
+ * Validates and copies the schedule. No device work. */
+int sds_create(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_t d, int32_t L,
+               sds_ctx** out);
+
+/* Attach workspace, stream (cudaStream_t, may be NULL for the default stream), seed, drafter mode
+ * and the global id of local chain 0. Uploads the schedule into the workspace and waits for it. */
+int sds_bind(sds_ctx* ctx, void* workspace_dev, size_t bytes, void* cuda_stream, uint64_t seed,
+             int32_t drafter_mode, int64_t chain_id_offset);
+
+/* Start all chains: Y_0 ~ N(0, I) from stream 2, n = 0, carried output D(Y_0, 0) (the one initial
+ * target call of the efficient frozen drafter), counters cleared, all chains active. */
+int sds_reset(sds_ctx* ctx);
+
+/* Draft: for every active chain, X[r0] = Y_n and, for j = 1..Lt (Lt = min(L, K-n)),
+ * W_j = a_k W_{j-1} + c_k D_c + sigma_k xi_{b,k}, k = n+j-1 (Algorithm 4, draft loop; Eq. 6). */
+int sds_draft(sds_ctx* ctx);
+
+/* Batched target pass on the drafted rows, then per position Delta = (m^p - m^q)/sigma,
+ * Z = (W_j - m^p)/sigma, log ratio = -|Delta|^2/2 - Delta.Z, accept iff log U <= log ratio,
+ * first rejection per chain, and the reflected state m^q + sigma (Z - 2 (Delta.Z/|Delta|^2) Delta)
+ * written over the rejected draft (Algorithm 4, verification loop; Algorithm 3). */
+int sds_verify_window(sds_ctx* ctx);
+
+/* n <- n + adv with adv = min(first rejection, Lt); Y <- W_adv; carried output <- target output of
+ * row adv; counters; rebuild the dense list of chains with n < K (Algorithm 4, "Set n <- k").
+ * n_active (host, may be NULL): if given, waits for the stream and stores the number of active chains. */
+int sds_advance(sds_ctx* ctx, int64_t* n_active);
+
+/* reset, then windows until no chain is active; copies Y_K to out_dev [B, d] and the counters to
+ * nfe_calls_dev / nfe_rows_dev [B] (either may be NULL). Waits for the stream.
+ * Small float mixtures run as one persistent kernel, one warp per chain, same results. */
+int sds_sample_all(sds_ctx* ctx, float* out_dev, int32_t* nfe_calls_dev, int32_t* nfe_rows_dev);
+
+/* Same with host buffers: copies the mixture parameters means_host [ncomp, d] / logw_host [ncomp]
+ * (float; NULL = keep what is on the device) to the device arrays named at create, runs
+ * sds_sample_all, copies the results to host memory. All copies are on the bound stream. */
+int sds_sample_all_host(sds_ctx* ctx, const float* means_host, const float* logw_host,
+                        float* out_host, int32_t* nfe_calls_host, int32_t* nfe_rows_host);
+
+/* Copy an internal array (selector above) to dst; dst_is_host != 0 waits for the stream. */
+int sds_get(sds_ctx* ctx, int32_t what, void* dst, size_t bytes, int32_t dst_is_host);
+
+/* Teacher forcing / resume: overwrite state Y [B,d], indices n [B], carried output Dc [B,d]
+ * (device pointers; any may be NULL = keep) and rebuild the active list. */
+int sds_set_state(sds_ctx* ctx, const float* Y_dev, const int32_t* n_dev, const float* Dc_dev);
+
+/* Stand-alone target pass (kernel-level parity and timing): the context's denoiser on
+ * x_dev [rows, d] at steps k_dev [rows] -> out_dev [rows, d]; rows <= B*L. */
+int sds_denoise(sds_ctx* ctx, const float* x_dev, const int32_t* k_dev, int64_t rows, float* out_dev);
+
+/* Philox normals / uniforms exactly as the path draws them (parity of the generator):
+ * out_dev [nb, d] = normals(seed, stream, chain b0+i, step k); u_dev [nb] = uniform(seed, b0+i, k). */
+int sds_rng_normals(uint64_t seed, int32_t stream_id, int64_t b0, int64_t nb, int32_t k, int32_t d,
+                    float* out_dev, void* cuda_stream);
+int sds_rng_uniforms(uint64_t seed, int64_t b0, int64_t nb, int32_t k, float* u_dev, void* cuda_stream);
+
+/* Number of kernels this context has launched since create (for launch accounting). */
+int64_t sds_launch_count(const sds_ctx* ctx);
+
+const char* sds_strerror(int code);
+int sds_last_cuda_error(const sds_ctx* ctx);
+void sds_destroy(sds_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SDS_H_ */

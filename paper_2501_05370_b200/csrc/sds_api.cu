@@ -1,0 +1,504 @@
+// C ABI of libsds (see include/sds.h): context, workspace carving, call-order checks and the
+// host loop of sds_sample_all. All device work is in the kernels this file launches.
+#include "../../include/sds.h"
+
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "sds_device.cuh"
+#include "sds_internal.h"
+
+using namespace sds;
+
+namespace {
+
+enum State { kCreated = 0, kBound, kReady, kDrafted, kVerified };
+
+constexpr size_t kAlign = 256;
+constexpr size_t kNone = (size_t)-1;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct Carve {
+  size_t off = 0;
+  size_t take(size_t bytes) {
+    const size_t o = off;
+    off = align_up(off + bytes);
+    return o;
+  }
+};
+
+// byte offsets of every workspace region
+struct Layout {
+  size_t a, c, sigma, tcond;
+  size_t Y, Dc, T, X, Dq, Xb;
+  size_t n, act, rowoff, rowk, ctl;
+  size_t S1, S2, ell, logU, accmask, jstar, nfe_calls, nfe_rows;
+  size_t musq;
+  size_t total;
+};
+
+}  // namespace
+
+struct sds_ctx {
+  int64_t B = 0;
+  int32_t d = 0, L = 0, K = 0;
+  std::vector<float> a, c, sigma, tcond;
+  int32_t tcond_dim = 0;
+  sds_denoiser den{};
+  Layout lay{};
+  char* ws = nullptr;
+  size_t ws_bytes = 0;
+  cudaStream_t stream = nullptr;
+  uint64_t seed = 0;
+  int64_t chain_off = 0;
+  int32_t mode = SDS_FROZEN_PREV;
+  State state = kCreated;
+  int ub = 0;                       // host upper bound on active chains
+  int last_cuda = 0;
+  int64_t launches = 0;
+  int32_t* h_pin = nullptr;         // pinned host words for the window loop
+  cudaEvent_t ev[2] = {nullptr, nullptr};
+  bool musq_ready = false;
+};
+
+namespace {
+
+bool wants_bf16_rows(const sds_denoiser& den) {
+  return den.kind == SDS_DEN_MLP || (den.kind == SDS_DEN_GMM && den.means_dtype == SDS_BF16);
+}
+
+void make_layout(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_t d, int32_t L, Layout* out) {
+  Carve cv;
+  Layout l{};
+  const size_t K = (size_t)sch->K, rows = (size_t)B * L, Bd = (size_t)B * d;
+  l.a = cv.take(K * 4);
+  l.c = cv.take(K * 4);
+  l.sigma = cv.take(K * 4);
+  l.tcond = cv.take(K * (size_t)(sch->tcond_dim > 0 ? sch->tcond_dim : 1) * 4);
+  l.Y = cv.take(Bd * 4);
+  l.Dc = cv.take(Bd * 4);
+  l.T = cv.take(Bd * 4);
+  l.X = cv.take(rows * d * 4);
+  l.Dq = cv.take(rows * d * 4);
+  l.Xb = wants_bf16_rows(*den) ? cv.take(rows * d * 2) : kNone;
+  l.n = cv.take((size_t)B * 4);
+  l.act = cv.take((size_t)B * 4);
+  l.rowoff = cv.take((size_t)(B + 1) * 4);
+  l.rowk = cv.take(rows * 4);
+  l.ctl = cv.take(kCtlWords * 4);
+  l.S1 = cv.take(rows * 8);
+  l.S2 = cv.take(rows * 8);
+  l.ell = cv.take(rows * 4);
+  l.logU = cv.take(rows * 4);
+  l.accmask = cv.take((size_t)B * 4);
+  l.jstar = cv.take((size_t)B * 4);
+  l.nfe_calls = cv.take((size_t)B * 4);
+  l.nfe_rows = cv.take((size_t)B * 4);
+  l.musq = (den->kind == SDS_DEN_GMM) ? cv.take((size_t)den->ncomp * 4) : kNone;
+  l.total = cv.off;
+  *out = l;
+}
+
+int validate(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_t d, int32_t L) {
+  if (!sch || !den) return SDS_EINVAL;
+  if (B <= 0 || d <= 0 || L < 1 || L > kMaxL || sch->K <= 0) return SDS_EINVAL;
+  if (B * (int64_t)L > ((int64_t)1 << 30) || B > ((int64_t)1 << 30)) return SDS_EINVAL;
+  if (!sch->a || !sch->c || !sch->sigma) return SDS_EINVAL;
+  for (int k = 0; k < sch->K; ++k) {
+    if (!std::isfinite(sch->a[k]) || !std::isfinite(sch->c[k]) || !std::isfinite(sch->sigma[k])) return SDS_EINVAL;
+    if (!(sch->sigma[k] > 0.f)) return SDS_EINVAL;
+  }
+  switch (den->kind) {
+    case SDS_DEN_GMM:
+      if (den->ncomp <= 0 || !den->means_dev || !den->logw_dev) return SDS_EINVAL;
+      if (!sch->tcond || sch->tcond_dim != 4) return SDS_EINVAL;
+      if (den->means_dtype != SDS_F32) return SDS_EUNSUPPORTED;
+      break;
+    case SDS_DEN_CALLBACK:
+      if (!den->fn) return SDS_EINVAL;
+      break;
+    case SDS_DEN_MLP:
+      return SDS_EUNSUPPORTED;
+    default:
+      return SDS_EUNSUPPORTED;
+  }
+  return SDS_OK;
+}
+
+template <class T>
+T* at(sds_ctx* c, size_t off) { return off == kNone ? nullptr : reinterpret_cast<T*>(c->ws + off); }
+
+WinArgs win_args(sds_ctx* c) {
+  WinArgs A{};
+  A.B = (int)c->B; A.d = c->d; A.L = c->L; A.K = c->K;
+  A.seed = c->seed; A.chain_off = (uint64_t)c->chain_off;
+  A.a = at<float>(c, c->lay.a); A.c = at<float>(c, c->lay.c); A.sigma = at<float>(c, c->lay.sigma);
+  A.Y = at<float>(c, c->lay.Y); A.Dc = at<float>(c, c->lay.Dc); A.T = at<float>(c, c->lay.T);
+  A.X = at<float>(c, c->lay.X); A.Dq = at<float>(c, c->lay.Dq); A.Xb = at<uint16_t>(c, c->lay.Xb);
+  A.n = at<int>(c, c->lay.n); A.act = at<int>(c, c->lay.act); A.rowoff = at<int>(c, c->lay.rowoff);
+  A.rowk = at<int>(c, c->lay.rowk); A.ctl = at<int>(c, c->lay.ctl);
+  A.S1 = at<double>(c, c->lay.S1); A.S2 = at<double>(c, c->lay.S2);
+  A.ell = at<float>(c, c->lay.ell); A.logU = at<float>(c, c->lay.logU);
+  A.accmask = at<uint32_t>(c, c->lay.accmask); A.jstar = at<int>(c, c->lay.jstar);
+  A.nfe_calls = at<int>(c, c->lay.nfe_calls); A.nfe_rows = at<int>(c, c->lay.nfe_rows);
+  return A;
+}
+
+GmmArgs gmm_args(sds_ctx* c) {
+  GmmArgs G{};
+  G.d = c->d; G.ncomp = c->den.ncomp; G.K = c->K;
+  G.tcond = at<float>(c, c->lay.tcond);
+  G.means = static_cast<const float*>(c->den.means_dev);
+  G.logw = c->den.logw_dev;
+  G.musq = at<float>(c, c->lay.musq);
+  return G;
+}
+
+int cuda_fail(sds_ctx* c, cudaError_t e) {
+  c->last_cuda = (int)e;
+  return SDS_ECUDA;
+}
+#define SDS_CU(ctx, expr)                                   \
+  do {                                                      \
+    cudaError_t e_ = (expr);                                \
+    if (e_ != cudaSuccess) return cuda_fail((ctx), e_);     \
+  } while (0)
+
+int ensure_musq(sds_ctx* c) {
+  if (c->musq_ready) return SDS_OK;
+  SDS_CU(c, launch_musq(static_cast<const float*>(c->den.means_dev), c->den.ncomp, c->d, at<float>(c, c->lay.musq),
+                        c->stream));
+  c->launches++;
+  c->musq_ready = true;
+  return SDS_OK;
+}
+
+// run the target denoiser on dense rows; the row count lives on the device (nrows_dev, may be
+// NULL) with a host upper bound for the grid
+int run_denoiser(sds_ctx* c, const float* X, const int* rowk, const int* nrows_dev, int64_t rows_ub, float* out) {
+  if (rows_ub <= 0) return SDS_OK;
+  switch (c->den.kind) {
+    case SDS_DEN_GMM: {
+      const int rc = ensure_musq(c);
+      if (rc != SDS_OK) return rc;
+      SDS_CU(c, launch_gmm_f32(gmm_args(c), X, rowk, nrows_dev, (int)rows_ub, out, c->stream));
+      c->launches++;
+      return SDS_OK;
+    }
+    case SDS_DEN_CALLBACK: {
+      int32_t rows = (int32_t)rows_ub;         // the callback needs the row count on the host
+      if (nrows_dev) {
+        SDS_CU(c, cudaMemcpyAsync(c->h_pin + 4, nrows_dev, 4, cudaMemcpyDeviceToHost, c->stream));
+        SDS_CU(c, cudaStreamSynchronize(c->stream));
+        rows = c->h_pin[4];
+      }
+      if (rows <= 0) return SDS_OK;
+      const int rc = c->den.fn(c->den.user, X, rowk, rows, c->d, out, (void*)c->stream);
+      return rc == 0 ? SDS_OK : SDS_ECALLBACK;
+    }
+    default:
+      return SDS_EUNSUPPORTED;
+  }
+}
+
+int sync_active(sds_ctx* c, int64_t* n_active) {
+  WinArgs A = win_args(c);
+  SDS_CU(c, cudaMemcpyAsync(c->h_pin, A.ctl, kCtlWords * 4, cudaMemcpyDeviceToHost, c->stream));
+  SDS_CU(c, cudaStreamSynchronize(c->stream));
+  c->ub = c->h_pin[kCtlNActive];
+  if (n_active) *n_active = c->ub;
+  return (c->h_pin[kCtlError] & kErrNonFinite) ? SDS_ENONFINITE : SDS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+#pragma GCC visibility push(default)
+
+int sds_workspace_bytes(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_t d, int32_t L,
+                        size_t* bytes) {
+  if (!bytes) return SDS_EINVAL;
+  const int rc = validate(sch, den, B, d, L);
+  if (rc != SDS_OK) return rc;
+  Layout l;
+  make_layout(sch, den, B, d, L, &l);
+  *bytes = l.total;
+  return SDS_OK;
+}
+
+int sds_create(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_t d, int32_t L, sds_ctx** out) {
+  if (!out) return SDS_EINVAL;
+  *out = nullptr;
+  const int rc = validate(sch, den, B, d, L);
+  if (rc != SDS_OK) return rc;
+  sds_ctx* c = new (std::nothrow) sds_ctx();
+  if (!c) return SDS_ENOMEM;
+  c->B = B; c->d = d; c->L = L; c->K = sch->K;
+  c->a.assign(sch->a, sch->a + sch->K);
+  c->c.assign(sch->c, sch->c + sch->K);
+  c->sigma.assign(sch->sigma, sch->sigma + sch->K);
+  c->tcond_dim = sch->tcond_dim > 0 ? sch->tcond_dim : 0;
+  if (sch->tcond && c->tcond_dim > 0) c->tcond.assign(sch->tcond, sch->tcond + (size_t)sch->K * c->tcond_dim);
+  c->den = *den;
+  make_layout(sch, den, B, d, L, &c->lay);
+  if (cudaHostAlloc((void**)&c->h_pin, 64 * sizeof(int32_t), cudaHostAllocDefault) != cudaSuccess) {
+    c->last_cuda = (int)cudaGetLastError();
+    delete c;
+    return SDS_ECUDA;
+  }
+  for (int i = 0; i < 2; ++i) {
+    if (cudaEventCreateWithFlags(&c->ev[i], cudaEventDisableTiming) != cudaSuccess) {
+      cudaGetLastError();
+      if (i == 1) cudaEventDestroy(c->ev[0]);
+      cudaFreeHost(c->h_pin);
+      delete c;
+      return SDS_ECUDA;
+    }
+  }
+  *out = c;
+  return SDS_OK;
+}
+
+int sds_bind(sds_ctx* c, void* workspace_dev, size_t bytes, void* cuda_stream, uint64_t seed, int32_t drafter_mode,
+             int64_t chain_id_offset) {
+  if (!c || !workspace_dev) return SDS_EINVAL;
+  if (drafter_mode != SDS_FROZEN_PREV) return SDS_EUNSUPPORTED;
+  if (chain_id_offset < 0) return SDS_EINVAL;
+  if (bytes < c->lay.total || (reinterpret_cast<uintptr_t>(workspace_dev) % kAlign) != 0) return SDS_ENOMEM;
+  c->ws = static_cast<char*>(workspace_dev);
+  c->ws_bytes = bytes;
+  c->stream = static_cast<cudaStream_t>(cuda_stream);
+  c->seed = seed;
+  c->mode = drafter_mode;
+  c->chain_off = chain_id_offset;
+  c->musq_ready = false;
+  const size_t kb = (size_t)c->K * 4;
+  SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.a, c->a.data(), kb, cudaMemcpyHostToDevice, c->stream));
+  SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.c, c->c.data(), kb, cudaMemcpyHostToDevice, c->stream));
+  SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.sigma, c->sigma.data(), kb, cudaMemcpyHostToDevice, c->stream));
+  if (!c->tcond.empty())
+    SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.tcond, c->tcond.data(), c->tcond.size() * 4, cudaMemcpyHostToDevice,
+                              c->stream));
+  SDS_CU(c, cudaMemsetAsync(c->ws + c->lay.ctl, 0, kCtlWords * 4, c->stream));
+  SDS_CU(c, cudaStreamSynchronize(c->stream));
+  c->state = kBound;
+  return SDS_OK;
+}
+
+int sds_reset(sds_ctx* c) {
+  if (!c) return SDS_EINVAL;
+  if (c->state < kBound) return SDS_ESTATE;
+  WinArgs A = win_args(c);
+  SDS_CU(c, launch_init(A, c->stream));
+  c->launches++;
+  const int rc = run_denoiser(c, A.X, A.rowk, A.ctl + kCtlNRows, c->B, A.Dq);
+  if (rc != SDS_OK) return rc;
+  SDS_CU(c, launch_after_init(A, c->stream));
+  SDS_CU(c, launch_compact(A, c->stream));
+  c->launches += 2;
+  c->ub = (int)c->B;
+  c->state = kReady;
+  return SDS_OK;
+}
+
+int sds_draft(sds_ctx* c) {
+  if (!c) return SDS_EINVAL;
+  if (c->state != kReady) return SDS_ESTATE;
+  SDS_CU(c, launch_draft(win_args(c), c->ub, c->stream));
+  c->launches++;
+  c->state = kDrafted;
+  return SDS_OK;
+}
+
+int sds_verify_window(sds_ctx* c) {
+  if (!c) return SDS_EINVAL;
+  if (c->state != kDrafted) return SDS_ESTATE;
+  WinArgs A = win_args(c);
+  const int rc = run_denoiser(c, A.X, A.rowk, A.ctl + kCtlNRows, (int64_t)c->ub * c->L, A.Dq);
+  if (rc != SDS_OK) return rc;
+  SDS_CU(c, launch_verify(A, c->ub, c->stream));
+  c->launches++;
+  c->state = kVerified;
+  return SDS_OK;
+}
+
+int sds_advance(sds_ctx* c, int64_t* n_active) {
+  if (!c) return SDS_EINVAL;
+  if (c->state != kVerified) return SDS_ESTATE;
+  SDS_CU(c, launch_advance(win_args(c), c->ub, c->stream));
+  c->launches++;
+  c->state = kReady;
+  if (n_active) return sync_active(c, n_active);
+  return SDS_OK;
+}
+
+int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* nfe_rows_dev) {
+  if (!c || !out_dev) return SDS_EINVAL;
+  if (c->state < kBound) return SDS_ESTATE;
+  WinArgs A = win_args(c);
+  int rc = SDS_OK;
+  if (c->den.kind == SDS_DEN_GMM && fused_small_supported(c->d, c->den.ncomp, c->L)) {
+    if ((rc = ensure_musq(c)) != SDS_OK) return rc;
+    SDS_CU(c, launch_fused_small(A, gmm_args(c), c->stream));
+    c->launches++;
+    c->ub = 0;
+    c->state = kReady;
+  } else {
+    rc = sds_reset(c);
+    if (rc != SDS_OK) return rc;
+    // Windows are enqueued one ahead of the host's knowledge of the active count: after window w
+    // is enqueued the host waits for window w-1's count. A window enqueued with no active chain
+    // does nothing on the device.
+    for (int w = 0;; ++w) {
+      if ((rc = sds_draft(c)) != SDS_OK) return rc;
+      if ((rc = sds_verify_window(c)) != SDS_OK) return rc;
+      if ((rc = sds_advance(c, nullptr)) != SDS_OK) return rc;
+      SDS_CU(c, cudaMemcpyAsync(c->h_pin + 8 + (w & 1) * kCtlWords, A.ctl, kCtlWords * 4, cudaMemcpyDeviceToHost,
+                                c->stream));
+      SDS_CU(c, cudaEventRecord(c->ev[w & 1], c->stream));
+      if (w >= 1) {
+        SDS_CU(c, cudaEventSynchronize(c->ev[(w - 1) & 1]));
+        const int na = c->h_pin[8 + ((w - 1) & 1) * kCtlWords + kCtlNActive];
+        if (na == 0) break;
+        c->ub = na;
+      }
+      if (w > c->K + 2) break;   // every window advances each active chain by at least one step
+    }
+  }
+  const size_t Bd = (size_t)c->B * c->d;
+  if (out_dev != A.Y) SDS_CU(c, cudaMemcpyAsync(out_dev, A.Y, Bd * 4, cudaMemcpyDeviceToDevice, c->stream));
+  if (nfe_calls_dev)
+    SDS_CU(c, cudaMemcpyAsync(nfe_calls_dev, A.nfe_calls, (size_t)c->B * 4, cudaMemcpyDeviceToDevice, c->stream));
+  if (nfe_rows_dev)
+    SDS_CU(c, cudaMemcpyAsync(nfe_rows_dev, A.nfe_rows, (size_t)c->B * 4, cudaMemcpyDeviceToDevice, c->stream));
+  int64_t na = 0;
+  return sync_active(c, &na);
+}
+
+int sds_sample_all_host(sds_ctx* c, const float* means_host, const float* logw_host, float* out_host,
+                        int32_t* nfe_calls_host, int32_t* nfe_rows_host) {
+  if (!c || !out_host) return SDS_EINVAL;
+  if (c->state < kBound) return SDS_ESTATE;
+  if ((means_host || logw_host) && c->den.kind != SDS_DEN_GMM) return SDS_EINVAL;
+  if (means_host) {
+    SDS_CU(c, cudaMemcpyAsync(const_cast<void*>(c->den.means_dev), means_host, (size_t)c->den.ncomp * c->d * 4,
+                              cudaMemcpyHostToDevice, c->stream));
+    c->musq_ready = false;
+  }
+  if (logw_host)
+    SDS_CU(c, cudaMemcpyAsync(const_cast<float*>(c->den.logw_dev), logw_host, (size_t)c->den.ncomp * 4,
+                              cudaMemcpyHostToDevice, c->stream));
+  WinArgs A = win_args(c);
+  const int rc = sds_sample_all(c, A.Y, nullptr, nullptr);
+  if (rc != SDS_OK && rc != SDS_ENONFINITE) return rc;
+  SDS_CU(c, cudaMemcpyAsync(out_host, A.Y, (size_t)c->B * c->d * 4, cudaMemcpyDeviceToHost, c->stream));
+  if (nfe_calls_host)
+    SDS_CU(c, cudaMemcpyAsync(nfe_calls_host, A.nfe_calls, (size_t)c->B * 4, cudaMemcpyDeviceToHost, c->stream));
+  if (nfe_rows_host)
+    SDS_CU(c, cudaMemcpyAsync(nfe_rows_host, A.nfe_rows, (size_t)c->B * 4, cudaMemcpyDeviceToHost, c->stream));
+  SDS_CU(c, cudaStreamSynchronize(c->stream));
+  return rc;
+}
+
+int sds_get(sds_ctx* c, int32_t what, void* dst, size_t bytes, int32_t dst_is_host) {
+  if (!c || !dst) return SDS_EINVAL;
+  if (c->state < kBound) return SDS_ESTATE;
+  const size_t B = (size_t)c->B, rows = B * c->L, d = (size_t)c->d;
+  size_t off = 0, len = 0;
+  switch (what) {
+    case SDS_GET_X: off = c->lay.X; len = rows * d * 4; break;
+    case SDS_GET_TAIL: off = c->lay.T; len = B * d * 4; break;
+    case SDS_GET_DQ: off = c->lay.Dq; len = rows * d * 4; break;
+    case SDS_GET_DC: off = c->lay.Dc; len = B * d * 4; break;
+    case SDS_GET_Y: off = c->lay.Y; len = B * d * 4; break;
+    case SDS_GET_N: off = c->lay.n; len = B * 4; break;
+    case SDS_GET_ACT: off = c->lay.act; len = B * 4; break;
+    case SDS_GET_ROWOFF: off = c->lay.rowoff; len = (B + 1) * 4; break;
+    case SDS_GET_S1: off = c->lay.S1; len = rows * 8; break;
+    case SDS_GET_S2: off = c->lay.S2; len = rows * 8; break;
+    case SDS_GET_ELL: off = c->lay.ell; len = rows * 4; break;
+    case SDS_GET_LOGU: off = c->lay.logU; len = rows * 4; break;
+    case SDS_GET_ACCMASK: off = c->lay.accmask; len = B * 4; break;
+    case SDS_GET_JSTAR: off = c->lay.jstar; len = B * 4; break;
+    case SDS_GET_NFE_CALLS: off = c->lay.nfe_calls; len = B * 4; break;
+    case SDS_GET_NFE_ROWS: off = c->lay.nfe_rows; len = B * 4; break;
+    case SDS_GET_CTL: off = c->lay.ctl; len = kCtlWords * 4; break;
+    case SDS_GET_ROWK: off = c->lay.rowk; len = rows * 4; break;
+    default: return SDS_EINVAL;
+  }
+  if (bytes > len) return SDS_EINVAL;
+  SDS_CU(c, cudaMemcpyAsync(dst, c->ws + off, bytes, dst_is_host ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice,
+                            c->stream));
+  if (dst_is_host) SDS_CU(c, cudaStreamSynchronize(c->stream));
+  return SDS_OK;
+}
+
+int sds_set_state(sds_ctx* c, const float* Y_dev, const int32_t* n_dev, const float* Dc_dev) {
+  if (!c) return SDS_EINVAL;
+  if (c->state != kReady) return SDS_ESTATE;
+  const size_t Bd = (size_t)c->B * c->d * 4;
+  if (Y_dev) SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.Y, Y_dev, Bd, cudaMemcpyDeviceToDevice, c->stream));
+  if (Dc_dev) SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.Dc, Dc_dev, Bd, cudaMemcpyDeviceToDevice, c->stream));
+  if (n_dev)
+    SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.n, n_dev, (size_t)c->B * 4, cudaMemcpyDeviceToDevice, c->stream));
+  SDS_CU(c, launch_compact(win_args(c), c->stream));
+  c->launches++;
+  c->ub = (int)c->B;
+  return SDS_OK;
+}
+
+int sds_denoise(sds_ctx* c, const float* x_dev, const int32_t* k_dev, int64_t rows, float* out_dev) {
+  if (!c || !x_dev || !k_dev || !out_dev) return SDS_EINVAL;
+  if (c->state < kBound) return SDS_ESTATE;
+  if (rows < 0 || rows > c->B * c->L) return SDS_EINVAL;
+  return run_denoiser(c, x_dev, k_dev, nullptr, rows, out_dev);
+}
+
+int sds_rng_normals(uint64_t seed, int32_t stream_id, int64_t b0, int64_t nb, int32_t k, int32_t d, float* out_dev,
+                    void* cuda_stream) {
+  if (!out_dev || nb < 0 || d <= 0 || k < 0 || b0 < 0) return SDS_EINVAL;
+  if (nb == 0) return SDS_OK;
+  return launch_rng_normals(seed, stream_id, (uint64_t)b0, nb, k, d, out_dev, (cudaStream_t)cuda_stream) == cudaSuccess
+             ? SDS_OK
+             : SDS_ECUDA;
+}
+
+int sds_rng_uniforms(uint64_t seed, int64_t b0, int64_t nb, int32_t k, float* u_dev, void* cuda_stream) {
+  if (!u_dev || nb < 0 || k < 0 || b0 < 0) return SDS_EINVAL;
+  if (nb == 0) return SDS_OK;
+  return launch_rng_uniforms(seed, (uint64_t)b0, nb, k, u_dev, (cudaStream_t)cuda_stream) == cudaSuccess ? SDS_OK
+                                                                                                           : SDS_ECUDA;
+}
+
+int64_t sds_launch_count(const sds_ctx* c) { return c ? c->launches : 0; }
+
+const char* sds_strerror(int code) {
+  switch (code) {
+    case SDS_OK: return "ok";
+    case SDS_EINVAL: return "invalid argument";
+    case SDS_ESTATE: return "call out of order";
+    case SDS_ENOMEM: return "workspace too small or misaligned";
+    case SDS_EUNSUPPORTED: return "unsupported configuration";
+    case SDS_ECUDA: return "CUDA error";
+    case SDS_ETIMEOUT: return "device-side wait timed out";
+    case SDS_ENONFINITE: return "non-finite log ratio: chain frozen";
+    case SDS_ECALLBACK: return "denoiser callback failed";
+    default: return "unknown error";
+  }
+}
+
+int sds_last_cuda_error(const sds_ctx* c) { return c ? c->last_cuda : 0; }
+
+void sds_destroy(sds_ctx* c) {
+  if (!c) return;
+  for (int i = 0; i < 2; ++i)
+    if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+  if (c->h_pin) cudaFreeHost(c->h_pin);
+  delete c;
+}
+
+#pragma GCC visibility pop
+}  // extern "C"

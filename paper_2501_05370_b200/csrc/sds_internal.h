@@ -1,0 +1,67 @@
+// Host-side view of the kernels: argument blocks and launcher prototypes.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace sds {
+
+// Everything a window kernel needs; passed by value. All pointers are device pointers into the
+// caller's workspace (or the caller's parameter arrays).
+struct WinArgs {
+  int B, d, L, K;
+  uint64_t seed;
+  uint64_t chain_off;
+  const float* a;        // [K]
+  const float* c;        // [K]
+  const float* sigma;    // [K]
+  float* Y;              // [B, d]   state Y_n
+  float* Dc;             // [B, d]   carried denoiser output
+  float* T;              // [B, d]   last drafted state of the window (position Lt)
+  float* X;              // [B*L, d] drafted states fed to the target, dense rows
+  float* Dq;             // [B*L, d] target outputs, same rows
+  uint16_t* Xb;          // [B*L, d] bf16 copy of X (NULL unless a tensor-core denoiser wants it)
+  int* n;                // [B]
+  int* act;              // [B]      active chain ids (ascending)
+  int* rowoff;           // [B+1]    first row of each active slot
+  int* rowk;             // [B*L]    transition index of each row
+  int* ctl;              // [kCtlWords]
+  double* S1;            // [B, L]
+  double* S2;            // [B, L]
+  float* ell;            // [B, L]
+  float* logU;           // [B, L]
+  uint32_t* accmask;     // [B]
+  int* jstar;            // [B]
+  int* nfe_calls;        // [B]
+  int* nfe_rows;         // [B]
+};
+
+struct GmmArgs {
+  int d, ncomp, K;
+  const float* tcond;    // [K, 4] (A, Bq, C, E)
+  const float* means;    // [ncomp, d]
+  const float* logw;     // [ncomp]
+  const float* musq;     // [ncomp]
+};
+
+// streaming kernels (sds_kernels.cu). ub_chains: host upper bound on the number of active chains.
+cudaError_t launch_init(const WinArgs& A, cudaStream_t st);
+cudaError_t launch_after_init(const WinArgs& A, cudaStream_t st);
+cudaError_t launch_compact(const WinArgs& A, cudaStream_t st);
+cudaError_t launch_draft(const WinArgs& A, int ub_chains, cudaStream_t st);
+cudaError_t launch_verify(const WinArgs& A, int ub_chains, cudaStream_t st);
+cudaError_t launch_advance(const WinArgs& A, int ub_chains, cudaStream_t st);
+cudaError_t launch_rng_normals(uint64_t seed, int stream_id, uint64_t b0, int64_t nb, int k, int d, float* out,
+                               cudaStream_t st);
+cudaError_t launch_rng_uniforms(uint64_t seed, uint64_t b0, int64_t nb, int k, float* out, cudaStream_t st);
+
+// mixture denoiser, float path (sds_gmm.cu)
+cudaError_t launch_musq(const float* means, int ncomp, int d, float* musq, cudaStream_t st);
+cudaError_t launch_gmm_f32(const GmmArgs& G, const float* X, const int* rowk, const int* nrows_dev, int rows_ub,
+                           float* out, cudaStream_t st);
+
+// whole-chain persistent kernel for small mixtures (sds_fused.cu)
+bool fused_small_supported(int d, int ncomp, int L);
+cudaError_t launch_fused_small(const WinArgs& A, const GmmArgs& G, cudaStream_t st);
+
+}  // namespace sds

@@ -1,0 +1,439 @@
+// Streaming kernels of the speculative window: initial state, draft, verify (log-ratio
+// reductions, accept uniforms, first rejection, reflection) and advance/compaction.
+//
+// Mapping: a "group" of TPC threads owns one chain (TPC = 32: a warp, several chains per CTA;
+// TPC = 256: the whole CTA). Rows are read and written with 128-bit accesses when d % 4 == 0.
+// All reductions combine partial sums in a fixed order, so results are reproducible and do not
+// depend on how many chains share the launch.
+#include "sds_device.cuh"
+#include "sds_internal.h"
+
+namespace sds {
+
+namespace {
+
+template <int TPC>
+struct Group {
+  static constexpr int kChainsPerBlock = kBlock / TPC;
+  __device__ static int slot() { return blockIdx.x * kChainsPerBlock + threadIdx.x / TPC; }
+  __device__ static int lane() { return threadIdx.x % TPC; }
+};
+
+__device__ __forceinline__ int window_len(const WinArgs& A, int nb) { return min(A.L, A.K - nb); }
+
+// ---------------------------------------------------------------------------------------
+// compaction: dense ascending list of chains with n < K and their first rows (one CTA)
+// ---------------------------------------------------------------------------------------
+__device__ void compact_scan(const WinArgs& A) {
+  __shared__ int s_cnt[kBlock / 32], s_row[kBlock / 32];
+  __shared__ int s_base_cnt, s_base_row;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) { s_base_cnt = 0; s_base_row = 0; }
+  __syncthreads();
+  for (int b0 = 0; b0 < A.B; b0 += kBlock) {
+    const int b = b0 + tid;
+    int flag = 0, lt = 0;
+    if (b < A.B) {
+      const int nb = __ldcg(A.n + b);
+      if (nb < A.K) { flag = 1; lt = min(A.L, A.K - nb); }
+    }
+    int c = flag, r = lt;                 // inclusive warp scans
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int c2 = __shfl_up_sync(0xffffffffu, c, o), r2 = __shfl_up_sync(0xffffffffu, r, o);
+      if (lane >= o) { c += c2; r += r2; }
+    }
+    if (lane == 31) { s_cnt[warp] = c; s_row[warp] = r; }
+    __syncthreads();
+    int wc = 0, wr = 0;
+    for (int w = 0; w < warp; ++w) { wc += s_cnt[w]; wr += s_row[w]; }
+    const int pos = s_base_cnt + wc + c - flag;
+    const int row = s_base_row + wr + r - lt;
+    if (flag) { A.act[pos] = b; A.rowoff[pos] = row; }
+    __syncthreads();
+    if (tid == kBlock - 1) { s_base_cnt = pos + flag; s_base_row = row + lt; }
+    __syncthreads();
+  }
+  if (tid == 0) {
+    A.rowoff[s_base_cnt] = s_base_row;
+    A.ctl[kCtlNActive] = s_base_cnt;
+    A.ctl[kCtlNRows] = s_base_row;
+  }
+}
+
+__global__ void __launch_bounds__(kBlock) k_compact(WinArgs A) { compact_scan(A); }
+
+// ---------------------------------------------------------------------------------------
+// I0: Y_0 ~ N(0, I) from stream 2; rows 0..B-1 of X carry Y_0 for the initial target call
+// ---------------------------------------------------------------------------------------
+template <int TPC, int VEC>
+__global__ void __launch_bounds__(kBlock) k_init(WinArgs A) {
+  using G = Group<TPC>;
+  const int b = G::slot(), t = G::lane();
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    A.ctl[kCtlNActive] = A.B;
+    A.ctl[kCtlNRows] = A.B;
+    A.ctl[kCtlWindows] = 0;
+    A.ctl[kCtlError] = 0;
+    A.ctl[kCtlFrozen] = 0;
+    A.ctl[kCtlDone] = 0;
+  }
+  if (b >= A.B) return;
+  const uint64_t bg = A.chain_off + (uint64_t)b;
+  const size_t off = (size_t)b * A.d;
+  if (VEC == 4) {
+    for (int i = t * 4; i < A.d; i += TPC * 4) {
+      const float4 z = normal4(A.seed, kStreamInit, bg, 0u, (uint32_t)(i >> 2));
+      st4(A.Y + off + i, z);
+      st4(A.X + off + i, z);
+      if (A.Xb)
+        *reinterpret_cast<uint2*>(A.Xb + off + i) = make_uint2(pack_bf16x2(z.x, z.y), pack_bf16x2(z.z, z.w));
+    }
+  } else {
+    for (int i = t; i < A.d; i += TPC) {
+      const float z = normal1(A.seed, kStreamInit, bg, 0u, (uint32_t)i);
+      A.Y[off + i] = z;
+      A.X[off + i] = z;
+      if (A.Xb) A.Xb[off + i] = (uint16_t)(pack_bf16x2(z, 0.f) & 0xffffu);
+    }
+  }
+  if (t == 0) {
+    A.n[b] = 0;
+    A.rowk[b] = 0;
+    A.nfe_calls[b] = 1;
+    A.nfe_rows[b] = 1;
+    A.accmask[b] = 0u;
+    A.jstar[b] = 0;
+  }
+}
+
+// after the initial target call: carried output <- its rows (row b belongs to chain b)
+__global__ void __launch_bounds__(kBlock) k_after_init(WinArgs A) {
+  const size_t total = (size_t)A.B * A.d;
+  for (size_t i = (size_t)blockIdx.x * kBlock + threadIdx.x; i < total; i += (size_t)gridDim.x * kBlock)
+    A.Dc[i] = A.Dq[i];
+}
+
+// ---------------------------------------------------------------------------------------
+// D1 draft: W_j = a_k W_{j-1} + c_k D_c + sigma_k xi_{b,k},  k = n + j - 1, j = 1..Lt
+// rows r0 .. r0+Lt-1 of X get W_0 .. W_{Lt-1}; T[b] gets W_Lt
+// ---------------------------------------------------------------------------------------
+template <int TPC, int VEC>
+__global__ void __launch_bounds__(kBlock) k_draft(WinArgs A) {
+  using G = Group<TPC>;
+  const int s = G::slot(), t = G::lane();
+  if (s >= A.ctl[kCtlNActive]) return;
+  const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
+  const int Lt = window_len(A, nb);
+  const uint64_t bg = A.chain_off + (uint64_t)b;
+  const size_t cb = (size_t)b * A.d;
+  if (t < Lt) A.rowk[r0 + t] = nb + t;            // TPC >= 32 >= Lt
+  if (VEC == 4) {
+    for (int i = t * 4; i < A.d; i += TPC * 4) {
+      float4 y = ld4(A.Y + cb + i);
+      const float4 dc = ld4(A.Dc + cb + i);
+      for (int j = 0; j < Lt; ++j) {
+        const size_t ro = (size_t)(r0 + j) * A.d + i;
+        st4(A.X + ro, y);
+        if (A.Xb) *reinterpret_cast<uint2*>(A.Xb + ro) = make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
+        const int k = nb + j;
+        const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
+        const float4 xi = normal4(A.seed, kStreamDraft, bg, (uint32_t)k, (uint32_t)(i >> 2));
+        y.x = draft_step(y.x, dc.x, xi.x, ak, ck, sk);
+        y.y = draft_step(y.y, dc.y, xi.y, ak, ck, sk);
+        y.z = draft_step(y.z, dc.z, xi.z, ak, ck, sk);
+        y.w = draft_step(y.w, dc.w, xi.w, ak, ck, sk);
+      }
+      st4(A.T + cb + i, y);
+    }
+  } else {
+    for (int i = t; i < A.d; i += TPC) {
+      float y = A.Y[cb + i];
+      const float dc = A.Dc[cb + i];
+      for (int j = 0; j < Lt; ++j) {
+        const size_t ro = (size_t)(r0 + j) * A.d + i;
+        A.X[ro] = y;
+        if (A.Xb) A.Xb[ro] = (uint16_t)(pack_bf16x2(y, 0.f) & 0xffffu);
+        const int k = nb + j;
+        const float xi = normal1(A.seed, kStreamDraft, bg, (uint32_t)k, (uint32_t)i);
+        y = draft_step(y, dc, xi, __ldg(A.a + k), __ldg(A.c + k), __ldg(A.sigma + k));
+      }
+      A.T[cb + i] = y;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// V1-V5 verify: per position S1 = |Delta|^2, S2 = Delta.Z (double accumulation), log ratio
+// -S1/2 - S2, accept iff log U <= log ratio, first rejection by ballot/ffs, reflection in place
+// ---------------------------------------------------------------------------------------
+template <int TPC, int VEC>
+__global__ void __launch_bounds__(kBlock) k_verify(WinArgs A) {
+  using G = Group<TPC>;
+  constexpr int kWarps = TPC / 32;
+  __shared__ double s_red[(TPC > 32) ? 2 * kMaxL * kWarps : 1];
+  __shared__ int s_jstar;
+  __shared__ float s_coef;
+  const int s = G::slot(), t = G::lane();
+  const int lane = threadIdx.x & 31, warp = t >> 5;
+  if (s >= A.ctl[kCtlNActive]) return;              // uniform per group (a warp, or the whole CTA)
+  const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
+  const int Lt = window_len(A, nb);
+  const uint64_t bg = A.chain_off + (uint64_t)b;
+  const size_t cb = (size_t)b * A.d;
+
+  double myS1 = 0.0, myS2 = 0.0;
+  for (int j = 1; j <= Lt; ++j) {
+    const int k = nb + j - 1;
+    const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
+    const float inv_s = 1.0f / sk, cs = ck * inv_s;
+    const float* wp = A.X + (size_t)(r0 + j - 1) * A.d;
+    const float* wj = (j < Lt) ? A.X + (size_t)(r0 + j) * A.d : A.T + cb;
+    const float* dq = A.Dq + (size_t)(r0 + j - 1) * A.d;
+    const float* dc = A.Dc + cb;
+    double p1 = 0.0, p2 = 0.0;
+    if (VEC == 4) {
+      for (int i = t * 4; i < A.d; i += TPC * 4) {
+        const float4 vp = ld4(wp + i), vj = ld4(wj + i), vq = ld4(dq + i), vc = ld4(dc + i);
+        float D, Z;
+        delta_z(vp.x, vj.x, vq.x, vc.x, ak, ck, cs, inv_s, D, Z);
+        p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+        delta_z(vp.y, vj.y, vq.y, vc.y, ak, ck, cs, inv_s, D, Z);
+        p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+        delta_z(vp.z, vj.z, vq.z, vc.z, ak, ck, cs, inv_s, D, Z);
+        p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+        delta_z(vp.w, vj.w, vq.w, vc.w, ak, ck, cs, inv_s, D, Z);
+        p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+      }
+    } else {
+      for (int i = t; i < A.d; i += TPC) {
+        float D, Z;
+        delta_z(wp[i], wj[i], dq[i], dc[i], ak, ck, cs, inv_s, D, Z);
+        p1 = fma((double)D, (double)D, p1);
+        p2 = fma((double)D, (double)Z, p2);
+      }
+    }
+    p1 = warp_sum(p1);
+    p2 = warp_sum(p2);
+    if (TPC == 32) {
+      if (lane == j - 1) { myS1 = p1; myS2 = p2; }
+    } else if (lane == 0) {
+      s_red[(j - 1) * kWarps + warp] = p1;
+      s_red[kMaxL * kWarps + (j - 1) * kWarps + warp] = p2;
+    }
+  }
+  if (TPC > 32) {
+    __syncthreads();
+    if (warp == 0 && lane < Lt) {
+      for (int w = 0; w < kWarps; ++w) {
+        myS1 += s_red[lane * kWarps + w];
+        myS2 += s_red[kMaxL * kWarps + lane * kWarps + w];
+      }
+    }
+  }
+
+  int jstar = 0;
+  float coef = 0.f;
+  if (warp == 0) {
+    const bool valid = lane < Lt;
+    bool acc = true, bad = false;
+    if (valid) {
+      const float U = uniform01(A.seed, bg, (uint32_t)(nb + lane));
+      const float lu = logf(U);
+      const float ellf = (float)(-0.5 * myS1 - myS2);
+      acc = (myS1 < 1e-30) || (lu <= ellf);
+      bad = !isfinite(ellf);
+      const size_t o = (size_t)b * A.L + lane;
+      A.S1[o] = myS1;
+      A.S2[o] = myS2;
+      A.ell[o] = ellf;
+      A.logU[o] = lu;
+    }
+    const uint32_t vmask = (Lt >= 32) ? 0xffffffffu : ((1u << Lt) - 1u);
+    const uint32_t amask = __ballot_sync(0xffffffffu, acc) & vmask;
+    const uint32_t bmask = __ballot_sync(0xffffffffu, bad) & vmask;
+    const uint32_t rej = ~amask & vmask;
+    jstar = rej ? __ffs(rej) : Lt + 1;
+    if (bmask) jstar = -1;                            // freeze the chain (handled by advance)
+    const int src = (jstar >= 1 && jstar <= Lt) ? jstar - 1 : 0;
+    const float mycoef = (float)(2.0 * myS2 / myS1);
+    coef = __shfl_sync(0xffffffffu, mycoef, src);
+    if (lane == 0) {
+      A.accmask[b] = amask;
+      A.jstar[b] = jstar;
+      if (bmask) atomicOr(A.ctl + kCtlError, kErrNonFinite);
+      if (TPC > 32) { s_jstar = jstar; s_coef = coef; }
+    }
+  }
+  if (TPC > 32) {
+    __syncthreads();
+    jstar = s_jstar;
+    coef = s_coef;
+  }
+  if (jstar < 1 || jstar > Lt) return;
+
+  // reflection of the rejected draft, in place
+  const int k = nb + jstar - 1;
+  const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
+  const float inv_s = 1.0f / sk, cs = ck * inv_s;
+  const float* wp = A.X + (size_t)(r0 + jstar - 1) * A.d;
+  float* wj = (jstar < Lt) ? A.X + (size_t)(r0 + jstar) * A.d : A.T + cb;
+  const float* dq = A.Dq + (size_t)(r0 + jstar - 1) * A.d;
+  const float* dc = A.Dc + cb;
+  if (VEC == 4) {
+    for (int i = t * 4; i < A.d; i += TPC * 4) {
+      const float4 vp = ld4(wp + i), vj = ld4(wj + i), vq = ld4(dq + i), vc = ld4(dc + i);
+      float4 o;
+      float D, Z;
+      delta_z(vp.x, vj.x, vq.x, vc.x, ak, ck, cs, inv_s, D, Z); o.x = reflect_elem(vp.x, vq.x, Z, D, ak, ck, sk, coef);
+      delta_z(vp.y, vj.y, vq.y, vc.y, ak, ck, cs, inv_s, D, Z); o.y = reflect_elem(vp.y, vq.y, Z, D, ak, ck, sk, coef);
+      delta_z(vp.z, vj.z, vq.z, vc.z, ak, ck, cs, inv_s, D, Z); o.z = reflect_elem(vp.z, vq.z, Z, D, ak, ck, sk, coef);
+      delta_z(vp.w, vj.w, vq.w, vc.w, ak, ck, cs, inv_s, D, Z); o.w = reflect_elem(vp.w, vq.w, Z, D, ak, ck, sk, coef);
+      st4(wj + i, o);
+    }
+  } else {
+    for (int i = t; i < A.d; i += TPC) {
+      float D, Z;
+      delta_z(wp[i], wj[i], dq[i], dc[i], ak, ck, cs, inv_s, D, Z);
+      wj[i] = reflect_elem(wp[i], dq[i], Z, D, ak, ck, sk, coef);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// C1 advance: Y <- W_adv, carried output <- target row adv, n += adv, counters; the CTA that
+// finishes last rebuilds the active list
+// ---------------------------------------------------------------------------------------
+template <int TPC, int VEC>
+__global__ void __launch_bounds__(kBlock) k_advance(WinArgs A) {
+  using G = Group<TPC>;
+  __shared__ int s_last;
+  const int s = G::slot(), t = G::lane();
+  const int n_active = A.ctl[kCtlNActive];
+  if (s < n_active) {
+    const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
+    const int Lt = window_len(A, nb);
+    const int js = A.jstar[b];
+    const size_t cb = (size_t)b * A.d;
+    if (js >= 1) {
+      const int adv = min(js, Lt);
+      const float* src = (adv < Lt) ? A.X + (size_t)(r0 + adv) * A.d : A.T + cb;
+      const float* dsrc = A.Dq + (size_t)(r0 + adv - 1) * A.d;
+      if (VEC == 4) {
+        for (int i = t * 4; i < A.d; i += TPC * 4) {
+          st4(A.Y + cb + i, ld4(src + i));
+          st4(A.Dc + cb + i, ld4(dsrc + i));
+        }
+      } else {
+        for (int i = t; i < A.d; i += TPC) {
+          A.Y[cb + i] = src[i];
+          A.Dc[cb + i] = dsrc[i];
+        }
+      }
+      if (t == 0) {
+        A.n[b] = nb + adv;
+        A.nfe_calls[b] += 1;
+        A.nfe_rows[b] += Lt;
+      }
+    } else if (t == 0) {                              // non-finite log ratio: stop this chain
+      A.n[b] = A.K;
+      atomicAdd(A.ctl + kCtlFrozen, 1);
+    }
+  }
+  // the last CTA to arrive rebuilds the list (no CTA waits on another)
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int prev = atomicAdd(A.ctl + kCtlDone, 1);
+    s_last = (prev == (int)gridDim.x - 1);
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  compact_scan(A);
+  if (threadIdx.x == 0) {
+    A.ctl[kCtlDone] = 0;
+    if (n_active > 0) A.ctl[kCtlWindows] += 1;
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// generator taps (parity of the random numbers themselves)
+// ---------------------------------------------------------------------------------------
+__global__ void k_rng_normals(uint64_t seed, int stream_id, uint64_t b0, int64_t nb, int k, int d, float* out) {
+  const int64_t total = nb * (int64_t)d;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t b = e / d;
+    const int i = (int)(e % d);
+    out[e] = normal1(seed, stream_id, b0 + (uint64_t)b, (uint32_t)k, (uint32_t)i);
+  }
+}
+__global__ void k_rng_uniforms(uint64_t seed, uint64_t b0, int64_t nb, int k, float* out) {
+  for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < nb; b += (int64_t)gridDim.x * blockDim.x)
+    out[b] = uniform01(seed, b0 + (uint64_t)b, (uint32_t)k);
+}
+
+inline int tpc_for(int d) { return d <= 256 ? 32 : 256; }
+inline bool vec4_ok(int d) { return (d % 4) == 0; }
+inline int blocks_for(int chains, int tpc) { const int cpb = kBlock / tpc; return (chains + cpb - 1) / cpb; }
+
+#define SDS_DISPATCH(KERNEL, A, chains, st)                                                       \
+  do {                                                                                            \
+    const int tpc_ = tpc_for((A).d);                                                              \
+    const int nb_ = blocks_for((chains) > 0 ? (chains) : 1, tpc_);                                \
+    if (tpc_ == 32) {                                                                             \
+      if (vec4_ok((A).d)) KERNEL<32, 4><<<nb_, kBlock, 0, st>>>(A);                               \
+      else KERNEL<32, 1><<<nb_, kBlock, 0, st>>>(A);                                              \
+    } else {                                                                                      \
+      if (vec4_ok((A).d)) KERNEL<256, 4><<<nb_, kBlock, 0, st>>>(A);                              \
+      else KERNEL<256, 1><<<nb_, kBlock, 0, st>>>(A);                                             \
+    }                                                                                             \
+  } while (0)
+
+}  // namespace
+
+cudaError_t launch_init(const WinArgs& A, cudaStream_t st) {
+  SDS_DISPATCH(k_init, A, A.B, st);
+  return cudaGetLastError();
+}
+cudaError_t launch_after_init(const WinArgs& A, cudaStream_t st) {
+  const size_t total = (size_t)A.B * A.d;
+  int nb = (int)((total + kBlock - 1) / kBlock);
+  if (nb > 148 * 8) nb = 148 * 8;
+  k_after_init<<<nb, kBlock, 0, st>>>(A);
+  return cudaGetLastError();
+}
+cudaError_t launch_compact(const WinArgs& A, cudaStream_t st) {
+  k_compact<<<1, kBlock, 0, st>>>(A);
+  return cudaGetLastError();
+}
+cudaError_t launch_draft(const WinArgs& A, int ub, cudaStream_t st) {
+  SDS_DISPATCH(k_draft, A, ub, st);
+  return cudaGetLastError();
+}
+cudaError_t launch_verify(const WinArgs& A, int ub, cudaStream_t st) {
+  SDS_DISPATCH(k_verify, A, ub, st);
+  return cudaGetLastError();
+}
+cudaError_t launch_advance(const WinArgs& A, int ub, cudaStream_t st) {
+  SDS_DISPATCH(k_advance, A, ub, st);
+  return cudaGetLastError();
+}
+cudaError_t launch_rng_normals(uint64_t seed, int stream_id, uint64_t b0, int64_t nb, int k, int d, float* out,
+                               cudaStream_t st) {
+  const int64_t total = nb * (int64_t)d;
+  int blocks = (int)((total + 255) / 256);
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  k_rng_normals<<<blocks, 256, 0, st>>>(seed, stream_id, b0, nb, k, d, out);
+  return cudaGetLastError();
+}
+cudaError_t launch_rng_uniforms(uint64_t seed, uint64_t b0, int64_t nb, int k, float* out, cudaStream_t st) {
+  int blocks = (int)((nb + 255) / 256);
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  k_rng_uniforms<<<blocks, 256, 0, st>>>(seed, b0, nb, k, out);
+  return cudaGetLastError();
+}
+
+}  // namespace sds
