@@ -1,0 +1,292 @@
+"""Thin ctypes binding of libsds (include/sds.h). Argument marshalling only: every step of the
+window runs in the library's CUDA kernels. PyTorch provides device memory and streams.
+
+There is no CPU fallback: importing works without a GPU (so that symbols can be inspected), but
+constructing a Sampler without CUDA raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import math
+import os
+from typing import Optional
+
+import numpy as np
+
+from . import build as _build
+
+# ---- constants mirrored from sds.h ----
+SDS_OK = 0
+SDS_EINVAL, SDS_ESTATE, SDS_ENOMEM, SDS_EUNSUPPORTED = -1, -2, -3, -4
+SDS_ECUDA, SDS_ETIMEOUT, SDS_ENONFINITE, SDS_ECALLBACK = -5, -6, -7, -8
+SDS_DEN_GMM, SDS_DEN_MLP, SDS_DEN_CALLBACK = 1, 2, 3
+SDS_F32, SDS_BF16 = 0, 1
+SDS_FROZEN_PREV = 0
+(GET_X, GET_TAIL, GET_DQ, GET_DC, GET_Y, GET_N, GET_ACT, GET_ROWOFF, GET_S1, GET_S2, GET_ELL, GET_LOGU,
+ GET_ACCMASK, GET_JSTAR, GET_NFE_CALLS, GET_NFE_ROWS, GET_CTL, GET_ROWK) = range(1, 19)
+
+DENOISE_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p)
+
+
+class SdsSchedule(C.Structure):
+    _fields_ = [("K", C.c_int32), ("a", C.c_void_p), ("c", C.c_void_p), ("sigma", C.c_void_p),
+                ("tcond", C.c_void_p), ("tcond_dim", C.c_int32)]
+
+
+class SdsDenoiser(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("ncomp", C.c_int32), ("means_dev", C.c_void_p), ("logw_dev", C.c_void_p),
+                ("means_dtype", C.c_int32), ("nlayer", C.c_int32), ("W_dev", C.c_void_p), ("bias_dev", C.c_void_p),
+                ("temb_dev", C.c_void_p), ("dims", C.c_void_p), ("fn", DENOISE_FN), ("user", C.c_void_p)]
+
+
+EXPORTS = {
+    "sds_workspace_bytes": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.POINTER(C.c_size_t)]),
+    "sds_create": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.POINTER(C.c_void_p)]),
+    "sds_bind": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_uint64, C.c_int32, C.c_int64]),
+    "sds_reset": (C.c_int, [C.c_void_p]),
+    "sds_draft": (C.c_int, [C.c_void_p]),
+    "sds_verify_window": (C.c_int, [C.c_void_p]),
+    "sds_advance": (C.c_int, [C.c_void_p, C.POINTER(C.c_int64)]),
+    "sds_sample_all": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "sds_sample_all_host": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "sds_get": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t, C.c_int32]),
+    "sds_set_state": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "sds_denoise": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]),
+    "sds_rng_normals": (C.c_int, [C.c_uint64, C.c_int32, C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
+    "sds_rng_uniforms": (C.c_int, [C.c_uint64, C.c_int64, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p]),
+    "sds_launch_count": (C.c_int64, [C.c_void_p]),
+    "sds_strerror": (C.c_char_p, [C.c_int]),
+    "sds_last_cuda_error": (C.c_int, [C.c_void_p]),
+    "sds_destroy": (None, [C.c_void_p]),
+}
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def load() -> C.CDLL:
+    """Load libsds.so (building it with nvcc first if the sources are newer). Raises if neither the
+    library nor a compiler is available: there is no other implementation to fall back to."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if _build.needs_build():
+        _build.build()
+    if not os.path.exists(_build.LIB):
+        raise RuntimeError("libsds.so is missing and could not be built")
+    lib = C.CDLL(_build.LIB)
+    for name, (res, args) in EXPORTS.items():
+        fn = getattr(lib, name)          # AttributeError if an export is missing
+        fn.restype = res
+        fn.argtypes = args
+    _lib = lib
+    return lib
+
+
+class SdsError(RuntimeError):
+    def __init__(self, code: int, where: str, cuda: int = 0):
+        msg = load().sds_strerror(code).decode()
+        super().__init__(f"{where}: {msg} (code {code}" + (f", cuda error {cuda})" if cuda else ")"))
+        self.code = code
+
+
+# ---------------------------------------------------------------------------------------------
+# host-side schedule helpers (float32 arrays handed to the library)
+# ---------------------------------------------------------------------------------------------
+
+def ddpm_schedule(beta: np.ndarray):
+    """Ancestral-sampler coefficients for an x0-predicting denoiser. Transition k moves noise level
+    t = K - k to t - 1: mean = a_k x_t + c_k x0_hat, std = sqrt(beta_t). Returns float32 (a, c, sigma)
+    and float64 abar[k] = abar_{K-k}."""
+    beta = np.asarray(beta, dtype=np.float64)
+    K = len(beta)
+    abar_full = np.concatenate([[1.0], np.cumprod(1.0 - beta)])
+    t = K - np.arange(K)
+    ab_t, ab_p, b_t = abar_full[t], abar_full[t - 1], beta[t - 1]
+    a = np.sqrt(1.0 - b_t) * (1.0 - ab_p) / (1.0 - ab_t)
+    c = np.sqrt(ab_p) * b_t / (1.0 - ab_t)
+    return a.astype(np.float32), c.astype(np.float32), np.sqrt(b_t).astype(np.float32), ab_t
+
+
+def gmm_tcond_posterior_mean(abar: np.ndarray, comp_std: float) -> np.ndarray:
+    """(A, Bq, C, E) per step for E[x0 | x_t] of a mixture with shared std s under x_t = al x0 + sqrt(1-al^2) eps:
+    v = al^2 s^2 + 1 - al^2;  A = al/v, Bq = -al^2/(2v), C = (1-al^2)/v, E = al s^2/v."""
+    abar = np.asarray(abar, dtype=np.float64)
+    al = np.sqrt(abar)
+    v = abar * comp_std ** 2 + 1.0 - abar
+    return np.stack([al / v, -abar / (2 * v), (1.0 - abar) / v, al * comp_std ** 2 / v], axis=1).astype(np.float32)
+
+
+def ula_schedule(K: int, gamma: float):
+    """Unadjusted Langevin: mean = x - gamma grad E(x), std = sqrt(2 gamma)."""
+    return (np.ones(K, np.float32), np.full(K, -gamma, np.float32), np.full(K, math.sqrt(2 * gamma), np.float32))
+
+
+def gmm_tcond_grad_energy(K: int, comp_std: float) -> np.ndarray:
+    """(A, Bq, C, E) for grad E of E = -log sum_c w_c N(x; mu_c, s^2 I): (1/s^2, -1/(2 s^2), -1/s^2, 1/s^2)."""
+    s2 = comp_std ** 2
+    return np.tile(np.array([1 / s2, -0.5 / s2, -1 / s2, 1 / s2], dtype=np.float32), (K, 1))
+
+
+# ---------------------------------------------------------------------------------------------
+# sampler object
+# ---------------------------------------------------------------------------------------------
+
+class Sampler:
+    """One libsds context with its device buffers.
+
+    Methods mirror the C entry points: reset, draft, verify_window, advance, sample_all,
+    sample_all_host, get, set_state, denoise.
+    """
+
+    def __init__(self, a, c, sigma, B: int, d: int, L: int, *, gmm_means=None, gmm_logw=None, tcond=None,
+                 callback=None, seed: int = 0, chain_id_offset: int = 0, device="cuda:0", stream=None):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("libsds needs a CUDA device; there is no CPU path")
+        self.torch = torch
+        self.lib = load()
+        self.device = torch.device(device)
+        torch.cuda.set_device(self.device)
+        self.B, self.d, self.L, self.K = int(B), int(d), int(L), len(a)
+        self._keep = []
+        a = np.ascontiguousarray(a, np.float32)
+        c = np.ascontiguousarray(c, np.float32)
+        sigma = np.ascontiguousarray(sigma, np.float32)
+        sch = SdsSchedule()
+        sch.K = self.K
+        sch.a, sch.c, sch.sigma = a.ctypes.data, c.ctypes.data, sigma.ctypes.data
+        if tcond is not None:
+            tcond = np.ascontiguousarray(tcond, np.float32)
+            sch.tcond, sch.tcond_dim = tcond.ctypes.data, tcond.shape[1]
+        self._keep += [a, c, sigma, tcond]
+        den = SdsDenoiser()
+        if gmm_means is not None:
+            means = np.ascontiguousarray(gmm_means, np.float32)
+            self.means = torch.from_numpy(means).to(self.device)
+            self.logw = torch.from_numpy(np.ascontiguousarray(gmm_logw, np.float32)).to(self.device)
+            den.kind, den.ncomp = SDS_DEN_GMM, means.shape[0]
+            den.means_dev, den.logw_dev, den.means_dtype = self.means.data_ptr(), self.logw.data_ptr(), SDS_F32
+        elif callback is not None:
+            self._cb = DENOISE_FN(callback)
+            den.kind, den.fn = SDS_DEN_CALLBACK, self._cb
+        else:
+            raise ValueError("a denoiser is required")
+        self._sch, self._den = sch, den
+        nbytes = C.c_size_t(0)
+        self._chk(self.lib.sds_workspace_bytes(C.byref(sch), C.byref(den), self.B, self.d, self.L, C.byref(nbytes)),
+                  "sds_workspace_bytes")
+        self.workspace_bytes = nbytes.value
+        self.ws = torch.empty(nbytes.value + 256, dtype=torch.uint8, device=self.device)
+        base = (self.ws.data_ptr() + 255) // 256 * 256
+        self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+        h = C.c_void_p()
+        self._chk(self.lib.sds_create(C.byref(sch), C.byref(den), self.B, self.d, self.L, C.byref(h)), "sds_create")
+        self.h = h
+        self._chk(self.lib.sds_bind(self.h, base, nbytes.value, self.stream.cuda_stream, seed, SDS_FROZEN_PREV,
+                                    chain_id_offset), "sds_bind")
+
+    # -- helpers --
+    def _chk(self, rc: int, where: str, allow=()):
+        if rc != SDS_OK and rc not in allow:
+            cuda = self.lib.sds_last_cuda_error(self.h) if getattr(self, "h", None) else 0
+            raise SdsError(rc, where, cuda)
+        return rc
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.lib.sds_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the path --
+    def reset(self):
+        self._chk(self.lib.sds_reset(self.h), "sds_reset")
+
+    def draft(self):
+        self._chk(self.lib.sds_draft(self.h), "sds_draft")
+
+    def verify_window(self):
+        self._chk(self.lib.sds_verify_window(self.h), "sds_verify_window")
+
+    def advance(self, sync: bool = True) -> Optional[int]:
+        if not sync:
+            self._chk(self.lib.sds_advance(self.h, None), "sds_advance")
+            return None
+        n = C.c_int64(0)
+        self._chk(self.lib.sds_advance(self.h, C.byref(n)), "sds_advance", allow=(SDS_ENONFINITE,))
+        return n.value
+
+    def sample_all(self, out=None, nfe_calls=None, nfe_rows=None):
+        t = self.torch
+        out = out if out is not None else t.empty((self.B, self.d), dtype=t.float32, device=self.device)
+        nfe_calls = nfe_calls if nfe_calls is not None else t.empty((self.B,), dtype=t.int32, device=self.device)
+        nfe_rows = nfe_rows if nfe_rows is not None else t.empty((self.B,), dtype=t.int32, device=self.device)
+        self._chk(self.lib.sds_sample_all(self.h, out.data_ptr(), nfe_calls.data_ptr(), nfe_rows.data_ptr()),
+                  "sds_sample_all", allow=(SDS_ENONFINITE,))
+        return out, nfe_calls, nfe_rows
+
+    def sample_all_host(self, means_host, logw_host, out_host, nfe_calls_host, nfe_rows_host):
+        """Host (pinned) tensors in and out; parameter upload and result download are part of the call."""
+        p = lambda x: x.data_ptr() if x is not None else None
+        self._chk(self.lib.sds_sample_all_host(self.h, p(means_host), p(logw_host), p(out_host), p(nfe_calls_host),
+                                               p(nfe_rows_host)), "sds_sample_all_host", allow=(SDS_ENONFINITE,))
+
+    _GET = {
+        GET_X: ("float32", "rows_d"), GET_TAIL: ("float32", "B_d"), GET_DQ: ("float32", "rows_d"),
+        GET_DC: ("float32", "B_d"), GET_Y: ("float32", "B_d"), GET_N: ("int32", "B"), GET_ACT: ("int32", "B"),
+        GET_ROWOFF: ("int32", "B1"), GET_S1: ("float64", "B_L"), GET_S2: ("float64", "B_L"),
+        GET_ELL: ("float32", "B_L"), GET_LOGU: ("float32", "B_L"), GET_ACCMASK: ("uint32", "B"),
+        GET_JSTAR: ("int32", "B"), GET_NFE_CALLS: ("int32", "B"), GET_NFE_ROWS: ("int32", "B"),
+        GET_CTL: ("int32", "ctl"), GET_ROWK: ("int32", "rows"),
+    }
+
+    def get(self, what: int) -> np.ndarray:
+        """Host copy of an internal array."""
+        dt, shp = self._GET[what]
+        B, L, d = self.B, self.L, self.d
+        shape = {"rows_d": (B * L, d), "B_d": (B, d), "B": (B,), "B1": (B + 1,), "B_L": (B, L), "ctl": (8,),
+                 "rows": (B * L,)}[shp]
+        arr = np.empty(shape, dtype=dt)
+        self._chk(self.lib.sds_get(self.h, what, arr.ctypes.data, arr.nbytes, 1), "sds_get")
+        return arr
+
+    def set_state(self, Y=None, n=None, Dc=None):
+        p = lambda x: x.data_ptr() if x is not None else None
+        self._keep_state = (Y, n, Dc)
+        self._chk(self.lib.sds_set_state(self.h, p(Y), p(n), p(Dc)), "sds_set_state")
+
+    def denoise(self, x, k, out=None):
+        t = self.torch
+        out = out if out is not None else t.empty_like(x)
+        self._chk(self.lib.sds_denoise(self.h, x.data_ptr(), k.data_ptr(), x.shape[0], out.data_ptr()), "sds_denoise")
+        return out
+
+    def launch_count(self) -> int:
+        return int(self.lib.sds_launch_count(self.h))
+
+
+def rng_normals(seed: int, stream_id: int, b0: int, nb: int, k: int, d: int, device="cuda:0"):
+    import torch
+    out = torch.empty((nb, d), dtype=torch.float32, device=device)
+    rc = load().sds_rng_normals(seed, stream_id, b0, nb, k, d, out.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    if rc != SDS_OK:
+        raise SdsError(rc, "sds_rng_normals")
+    return out
+
+
+def rng_uniforms(seed: int, b0: int, nb: int, k: int, device="cuda:0"):
+    import torch
+    out = torch.empty((nb,), dtype=torch.float32, device=device)
+    rc = load().sds_rng_uniforms(seed, b0, nb, k, out.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    if rc != SDS_OK:
+        raise SdsError(rc, "sds_rng_uniforms")
+    return out

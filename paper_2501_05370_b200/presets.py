@@ -1,0 +1,30 @@
+"""Builds a Sampler for a workload description (any object with the fields of workloads.Workload)."""
+from __future__ import annotations
+
+import numpy as np
+
+from . import binding as sb
+
+
+def schedule_for(w):
+    """float32 (a, c, sigma) and the mixture conditioning table for workload w (None for non-mixtures)."""
+    if w.sampler == "ddpm":
+        a, c, sigma, abar = sb.ddpm_schedule(w.beta())
+        tcond = sb.gmm_tcond_posterior_mean(abar, w.gmm["comp_std"]) if w.denoiser == "gmm" else None
+    elif w.sampler == "ula":
+        a, c, sigma = sb.ula_schedule(w.K, w.ula_gamma)
+        tcond = sb.gmm_tcond_grad_energy(w.K, w.gmm["comp_std"]) if w.denoiser == "gmm" else None
+    else:
+        raise ValueError(w.sampler)
+    return a, c, sigma, tcond
+
+
+def sampler_for(w, *, seed=None, chain_id_offset=0, B=None, device="cuda:0", gmm=None):
+    a, c, sigma, tcond = schedule_for(w)
+    seed = w.sample_seed if seed is None else seed
+    B = w.B if B is None else B
+    if w.denoiser == "gmm":
+        gp = gmm if gmm is not None else w.gmm_params()
+        return sb.Sampler(a, c, sigma, B, w.d, w.L, gmm_means=gp.means, gmm_logw=gp.logw, tcond=tcond, seed=seed,
+                          chain_id_offset=chain_id_offset, device=device)
+    raise NotImplementedError(w.denoiser)

@@ -1,0 +1,302 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs. Tiers: generator and denoiser kernels alone; one window on forced arrays (decisions
+exact outside the rounding band); free-running chains end to end."""
+import math
+
+import numpy as np
+import pytest
+
+import paper_2501_05370_b200 as sds
+from paper_2501_05370_b200 import binding as sb
+from oracle import sds_oracle as o
+import workloads as wl
+from helpers import BAND, ell_close, oracle_setup, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+
+def _torch():
+    import torch
+    return torch
+
+
+# ------------------------------------------------------------------ generator -----------
+
+@pytest.mark.parametrize("b0,k,d", [(0, 0, 1), (5, 17, 7), (123456, 499, 64), ((1 << 32) + 9, 3, 130), (7, 1999, 1024)])
+def test_rng_normals_and_uniforms(b0, k, d):
+    seed = 0x1234_5678_9ABC_DEF1
+    nb = 5
+    for stream in (o.STREAM_DRAFT, o.STREAM_INIT):
+        got = sb.rng_normals(seed, stream, b0, nb, k, d).cpu().numpy()
+        want = np.stack([o.normals(seed, stream, b0 + i, k, d) for i in range(nb)])
+        assert np.max(np.abs(got - want)) <= 3e-6
+    u = sb.rng_uniforms(seed, b0, nb, k).cpu().numpy()
+    uw = np.array([o.uniform01(seed, b0 + i, k) for i in range(nb)])
+    assert np.array_equal(u.astype(np.float64), uw)          # exact: multiples of 2^-24
+
+
+# ------------------------------------------------------------------ denoiser ------------
+
+@pytest.mark.parametrize("name,d,ncomp,rows", [("cfg1", 2, 4, 37), ("cfg2", 64, 16, 515), ("cfg2", 33, 5, 70),
+                                              ("cfg5", 96, 40, 130), ("cfg5", 1024, 24, 21)])
+def test_gmm_denoiser_rows(name, d, ncomp, rows):
+    torch = _torch()
+    w = wl.WORKLOADS[name].scaled(d=d, B=max(rows, 1), L=1)
+    gp = w.gmm_params(d=d, ncomp=ncomp)
+    s = sds.sampler_for(w, gmm=gp)
+    den, a, c, sig = oracle_setup(w, gmm=gp)
+    rng = np.random.default_rng(1)
+    scale = 4.0 if w.sampler == "ula" else 1.5
+    x = (rng.standard_normal((rows, d)) * scale).astype(np.float32)
+    # some rows sit near a component mean (sharp responsibilities)
+    x[::7] = gp.means[rng.integers(0, ncomp, size=len(x[::7]))] * (0.9 if w.sampler == "ddpm" else 1.0) + 0.1 * x[::7]
+    k = rng.integers(0, w.K, size=rows).astype(np.int32)
+    out = s.denoise(torch.from_numpy(x).cuda(), torch.from_numpy(k).cuda()).cpu().numpy()
+    for r in range(rows):
+        want = den(x[r].astype(np.float64), int(k[r]))
+        assert rel_l2(out[r], want) <= 1e-5, (r, rel_l2(out[r], want))
+    s.close()
+
+
+# ------------------------------------------------------------------ one window, forced ---
+
+def _window_check(s, w, den, a32, c32, s32, seed, chain_off, stats):
+    """Runs draft + verify on the GPU and replays the verification on the GPU's own arrays."""
+    B, L, d, K = s.B, s.L, s.d, s.K
+    ctl = s.get(sb.GET_CTL)
+    na, nrows = int(ctl[0]), int(ctl[1])
+    act, rowoff, n = s.get(sb.GET_ACT)[:na], s.get(sb.GET_ROWOFF)[:na + 1], s.get(sb.GET_N)
+    assert np.all(np.diff(act) > 0)
+    assert int(rowoff[na]) == nrows == int(sum(min(L, K - n[b]) for b in act))
+    Y, Dc = s.get(sb.GET_Y), s.get(sb.GET_DC)
+    s.draft()
+    X, T, rowk = s.get(sb.GET_X), s.get(sb.GET_TAIL), s.get(sb.GET_ROWK)
+    s.verify_window()
+    Dq = s.get(sb.GET_DQ)
+    X2, T2 = s.get(sb.GET_X), s.get(sb.GET_TAIL)
+    S1, S2, ell, logU = s.get(sb.GET_S1), s.get(sb.GET_S2), s.get(sb.GET_ELL), s.get(sb.GET_LOGU)
+    accmask, jstar = s.get(sb.GET_ACCMASK), s.get(sb.GET_JSTAR)
+    a64, c64, s64 = a32.astype(np.float64), c32.astype(np.float64), s32.astype(np.float64)
+    for si, b in enumerate(act):
+        nb = int(n[b]); Lt = min(L, K - nb); r0 = int(rowoff[si])
+        assert np.array_equal(rowk[r0:r0 + Lt], nb + np.arange(Lt))
+        W = np.concatenate([X[r0:r0 + Lt], T[b:b + 1]]).astype(np.float64)
+        assert np.array_equal(X[r0], Y[b])
+        # draft: W_j = a W_{j-1} + c D_c + sigma xi with the oracle's normals
+        for j in range(1, Lt + 1):
+            k = nb + j - 1
+            xi = o.normals(seed, o.STREAM_DRAFT, chain_off + int(b), k, d)
+            want = a64[k] * W[j - 1] + c64[k] * Dc[b].astype(np.float64) + s64[k] * xi
+            assert rel_l2(W[j], want) <= 1e-5
+        # target rows
+        for j in range(1, Lt + 1):
+            assert rel_l2(Dq[r0 + j - 1], den(W[j - 1], nb + j - 1)) <= 1e-5
+        lu = np.array([math.log(o.uniform01(seed, chain_off + int(b), nb + j)) for j in range(Lt)])
+        assert np.max(np.abs(logU[b, :Lt] - lu)) <= 2e-6
+        v = o.verify_window(W, Dq[r0:r0 + Lt], Dc[b], a64, c64, s64, nb, logU[b, :Lt].astype(np.float64))
+        amb = np.abs(v["ell"] - logU[b, :Lt]) < BAND
+        for j in range(Lt):
+            assert ell_close(float(ell[b, j]), float(v["ell"][j])), (b, j, ell[b, j], v["ell"][j])
+            assert abs(S1[b, j] - v["S1"][j]) <= 1e-5 * max(v["S1"][j], 1e-12) + 1e-12
+            gacc = bool((int(accmask[b]) >> j) & 1)
+            stats["tests"] += 1
+            if amb[j]:
+                stats["band"] += 1
+            else:
+                assert gacc == bool(v["acc"][j]), (b, j)
+        if not amb.any():
+            assert int(jstar[b]) == v["jstar"]
+        js = int(jstar[b])
+        assert 1 <= js <= Lt + 1
+        if js <= Lt and js == v["jstar"]:
+            got = X2[r0 + js] if js < Lt else T2[b]
+            assert rel_l2(got, v["Y_reflect"]) <= 1e-5
+            stats["reflected"] += 1
+            # reflection is an isometry about the target mean
+            k = nb + js - 1
+            m_q = a64[k] * W[js - 1] + c64[k] * Dq[r0 + js - 1].astype(np.float64)
+            m_p = a64[k] * W[js - 1] + c64[k] * Dc[b].astype(np.float64)
+            assert abs(np.linalg.norm(got - m_q) - np.linalg.norm(W[js] - m_p)) <= 1e-4 * np.linalg.norm(W[js] - m_p) + 1e-6
+        # rows other than the reflected one are untouched
+        for j in range(Lt + 1):
+            if j != js:
+                assert np.array_equal(X2[r0 + j] if j < Lt else T2[b], X[r0 + j] if j < Lt else T[b])
+    n_before = n.copy()
+    na2 = s.advance()
+    n2, Y2, Dc2 = s.get(sb.GET_N), s.get(sb.GET_Y), s.get(sb.GET_DC)
+    for si, b in enumerate(act):
+        nb = int(n_before[b]); Lt = min(L, K - nb); r0 = int(rowoff[si])
+        adv = min(int(jstar[b]), Lt)
+        assert n2[b] == nb + adv
+        assert np.array_equal(Y2[b], X2[r0 + adv] if adv < Lt else T2[b])
+        assert np.array_equal(Dc2[b], Dq[r0 + adv - 1])
+    assert na2 == int(np.sum(n2 < K))
+    return na2
+
+
+SHAPES = [
+    # name, B, d, L, K, ncomp, windows
+    ("cfg1", 64, 2, 4, 100, 4, 6),
+    ("cfg2", 96, 64, 8, 200, 16, 4),
+    ("cfg2", 65, 33, 5, 23, 7, 8),
+    ("cfg2", 3, 5, 2, 9, 3, 9),
+    ("cfg1", 1, 1, 1, 6, 2, 6),
+    ("cfg2", 9, 3, 32, 70, 4, 5),
+    ("cfg5", 20, 1024, 6, 40, 12, 4),
+    ("cfg5", 7, 516, 32, 64, 5, 3),
+    ("cfg2", 5, 1030, 3, 11, 6, 5),
+]
+
+
+@pytest.mark.parametrize("name,B,d,L,K,ncomp,windows", SHAPES)
+def test_window_forced_parity(name, B, d, L, K, ncomp, windows):
+    w = wl.WORKLOADS[name].scaled(B=B, d=d, L=L, K=K)
+    gp = w.gmm_params(d=d, ncomp=ncomp)
+    seed, off = 4242 + d, 1000
+    s = sds.sampler_for(w, gmm=gp, seed=seed, chain_id_offset=off)
+    den, a, c, sig = oracle_setup(w, gmm=gp)
+    a32, c32, s32, _ = sds.schedule_for(w)
+    s.reset()
+    # initial state and carried output
+    Y0, Dc0 = s.get(sb.GET_Y), s.get(sb.GET_DC)
+    for b in range(min(B, 8)):
+        want = o.normals(seed, o.STREAM_INIT, off + b, 0, d)
+        assert np.max(np.abs(Y0[b] - want)) <= 3e-6
+        assert rel_l2(Dc0[b], den(Y0[b].astype(np.float64), 0)) <= 1e-5
+    stats = dict(tests=0, band=0, reflected=0)
+    na = B
+    for _ in range(windows):
+        if na == 0:
+            break
+        na = _window_check(s, w, den, a32, c32, s32, seed, off, stats)
+    assert stats["band"] <= max(2, 2e-3 * stats["tests"])
+    s.close()
+
+
+# ------------------------------------------------------------------ free running ---------
+
+def _free_run_compare(w, gp, chains, seed, off=0, B=None):
+    torch = _torch()
+    s = sds.sampler_for(w, gmm=gp, seed=seed, chain_id_offset=off, B=B)
+    out, calls, rows = s.sample_all()
+    out, calls, rows = out.cpu().numpy(), calls.cpu().numpy(), rows.cpu().numpy()
+    assert np.all(np.isfinite(out))
+    assert np.array_equal(s.get(sb.GET_N), np.full(s.B, w.K))
+    den, a, c, sig = oracle_setup(w, gmm=gp)
+    diverged = 0
+    for b in chains:
+        r = o.speculative_chain(den, a, c, sig, w.L, seed, off + b, w.d, record=True)
+        same = (r["nfe_calls"] == calls[b] and r["nfe_rows"] == rows[b] and rel_l2(out[b], r["Y"]) <= 1e-4)
+        if not same:
+            gaps = [np.min(np.abs(win["ell"] - win["logU"])) for win in r["windows"]]
+            assert min(gaps) < BAND, (b, min(gaps), r["nfe_calls"], calls[b])
+            diverged += 1
+        # counters are consistent on their own
+        assert calls[b] >= 1 + math.ceil(w.K / w.L) and rows[b] >= w.K + 1 - 0
+    assert diverged <= max(1, len(chains) // 20)
+    s.close()
+    return out, calls, rows
+
+
+def test_free_running_cfg1_all_chains():
+    w = wl.WORKLOADS["cfg1"]
+    _free_run_compare(w, w.gmm_params(), range(w.B), w.sample_seed)
+
+
+def test_free_running_cfg2_sampled_chains():
+    w = wl.WORKLOADS["cfg2"]
+    rng = np.random.default_rng(0)
+    chains = sorted(rng.choice(w.B, size=24, replace=False).tolist())
+    out, calls, rows = _free_run_compare(w, w.gmm_params(), chains, w.sample_seed)
+    # whole-batch properties at full size
+    assert np.all(calls <= 1 + w.K) and np.all(rows <= 1 + w.K * w.L)
+    assert calls.mean() < 1 + w.K          # speculation saves sequential calls
+
+
+def test_free_running_ula_small():
+    w = wl.WORKLOADS["cfg5"].scaled(B=12, d=128, K=120, L=16)
+    gp = w.gmm_params(d=128, ncomp=12)
+    _free_run_compare(w, gp, range(12), 99)
+
+
+def test_stepwise_loop_equals_sample_all_and_is_deterministic():
+    w = wl.WORKLOADS["cfg2"].scaled(B=200, K=60)
+    gp = w.gmm_params()
+    s = sds.sampler_for(w, gmm=gp, seed=5)
+    o1, c1, r1 = [x.cpu().numpy() for x in s.sample_all()]
+    o2, c2, r2 = [x.cpu().numpy() for x in s.sample_all()]
+    assert np.array_equal(o1, o2) and np.array_equal(c1, c2) and np.array_equal(r1, r2)
+    s.reset()
+    na, windows = s.B, 0
+    while na > 0:
+        s.draft(); s.verify_window(); na = s.advance(); windows += 1
+        assert windows <= w.K
+    assert np.array_equal(s.get(sb.GET_Y), o1)
+    assert np.array_equal(s.get(sb.GET_NFE_CALLS), c1) and np.array_equal(s.get(sb.GET_NFE_ROWS), r1)
+    assert int(s.get(sb.GET_CTL)[2]) == windows
+    s.close()
+
+
+def test_chain_shards_reproduce_the_unsharded_run_bitwise():
+    w = wl.WORKLOADS["cfg2"].scaled(B=96, K=50)
+    gp = w.gmm_params()
+    full = sds.sampler_for(w, gmm=gp, seed=11)
+    of, cf, rf = [x.cpu().numpy() for x in full.sample_all()]
+    parts = []
+    for off, nb in ((0, 40), (40, 56)):
+        s = sds.sampler_for(w, gmm=gp, seed=11, chain_id_offset=off, B=nb)
+        parts.append([x.cpu().numpy() for x in s.sample_all()])
+        s.close()
+    assert np.array_equal(np.concatenate([p[0] for p in parts]), of)
+    assert np.array_equal(np.concatenate([p[1] for p in parts]), cf)
+    assert np.array_equal(np.concatenate([p[2] for p in parts]), rf)
+    full.close()
+
+
+def test_identical_drafter_and_target_accepts_everything():
+    """With c_k = 0 the draft and target means coincide (Delta = 0): every draft is accepted and
+    every window advances by its full length."""
+    w = wl.WORKLOADS["cfg2"].scaled(B=32, K=30)
+    gp = w.gmm_params()
+    a, c, sig, tcond = sds.schedule_for(w)
+    s = sb.Sampler(a, np.zeros_like(c), sig, 32, w.d, w.L, gmm_means=gp.means, gmm_logw=gp.logw, tcond=tcond, seed=3)
+    out, calls, rows = s.sample_all()
+    # Delta = 0 everywhere: every window is accepted in full
+    assert np.array_equal(calls.cpu().numpy(), np.full(32, 1 + math.ceil(30 / w.L)))
+    assert np.all(s.get(sb.GET_S1) == 0.0)
+    s.close()
+
+
+def test_call_order_is_enforced():
+    w = wl.WORKLOADS["cfg1"]
+    s = sds.sampler_for(w)
+    lib = s.lib
+    assert lib.sds_draft(s.h) == sb.SDS_ESTATE
+    s.reset()
+    assert lib.sds_verify_window(s.h) == sb.SDS_ESTATE
+    assert lib.sds_advance(s.h, None) == sb.SDS_ESTATE
+    s.draft()
+    assert lib.sds_draft(s.h) == sb.SDS_ESTATE
+    s.verify_window()
+    assert lib.sds_reset(s.h) == sb.SDS_OK
+    s.close()
+
+
+def test_set_state_resume_is_bitwise():
+    torch = _torch()
+    w = wl.WORKLOADS["cfg2"].scaled(B=50, K=40)
+    gp = w.gmm_params()
+    s = sds.sampler_for(w, gmm=gp, seed=21)
+    ref = s.sample_all()[0].cpu().numpy()
+    s.reset()
+    for _ in range(3):
+        s.draft(); s.verify_window(); s.advance()
+    Y, n, Dc = (torch.from_numpy(s.get(x)).cuda() for x in (sb.GET_Y, sb.GET_N, sb.GET_DC))
+    s2 = sds.sampler_for(w, gmm=gp, seed=21)
+    s2.reset()
+    s2.set_state(Y, n, Dc)
+    na = 1
+    while na > 0:
+        s2.draft(); s2.verify_window(); na = s2.advance()
+    assert np.array_equal(s2.get(sb.GET_Y), ref)
+    s.close(); s2.close()
