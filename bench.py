@@ -1,0 +1,335 @@
+#!/usr/bin/env python
+"""Benchmark of the speculative-sampling hot path.
+
+One "step" is one full sds_sample_all over a batch of chains of the chosen workload: initial
+state and target call, then draft / batched target / verify / advance windows until every chain
+has made its K transitions. The metric is accepted chain-steps per second (B*K per run; both
+accepted and reflected steps are valid target steps).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+
+Prints one JSON line (rank 0). N > 1 (under torch.distributed.run): chains are sharded across
+ranks by global chain id, no collective on the data path (weak scaling: B chains per rank).
+--impl reference times the CPU oracle, as it stands, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+METRIC = "accepted_chain_steps_per_sec"
+UNIT = "chain-steps/s"
+FP32_LANES_PER_SM, SMS = 128, 148
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"], bf16_sustained=d["bf16_tflops_sustained"],
+                    sm_max_mhz=d.get("sm_max_mhz", 1965.0), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_sustained=1400.0, sm_max_mhz=1965.0, source="fallback")
+
+
+# --------------------------------------------------------------------------------------------
+# CPU oracle legs
+# --------------------------------------------------------------------------------------------
+
+def oracle_closure(w):
+    from oracle import sds_oracle as o
+    gp = w.gmm_params()
+    if w.sampler == "ddpm":
+        a, c, sig, abar = o.ddpm_affine(w.beta())
+        den = lambda x, k: o.gmm_posterior_mean(x, abar[k], gp.means, gp.logw, gp.comp_std, bf16_operands=gp.means_bf16)
+    else:
+        a, c, sig = o.ula_affine(w.K, w.ula_gamma)
+        den = lambda x, k: o.gmm_grad_energy(x, gp.means, gp.logw, gp.comp_std)
+    return o, den, a, c, sig
+
+
+def oracle_time(w, budget_s: float, min_chains: int = 2, first_chain: int = 0):
+    """Runs oracle chains one after another for about budget_s seconds. Returns (chains, seconds)."""
+    o, den, a, c, sig = oracle_closure(w)
+    t0 = time.perf_counter()
+    n = 0
+    while True:
+        o.speculative_chain(den, a, c, sig, w.L, w.sample_seed, first_chain + n, w.d)
+        n += 1
+        el = time.perf_counter() - t0
+        if n >= min_chains and el >= budget_s:
+            return n, el
+        if n >= w.B:
+            return n, el
+
+
+def run_reference(args, w):
+    """--impl reference: the oracle on the host cores, same metric, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    per_step_budget = max(1.0, min(8.0, 60.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        oracle_time(w, per_step_budget, min_chains=1)
+    tot_chains, tot_s = 0, 0.0
+    for i in range(args.steps):
+        n, s = oracle_time(w, per_step_budget, min_chains=1, first_chain=i * 16)
+        tot_chains += n
+        tot_s += s
+    value = tot_chains * w.K / tot_s
+    sample = f"{tot_chains} chains of {w.name} (K={w.K}, L={w.L}, d={w.d}) over {args.steps} steps, one NumPy thread"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot_s / max(1, args.steps),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w, args),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w, args):
+    return {"workload": f"{w.name}: B={w.B} chains/GPU, d={w.d}, L={w.L}, K={w.K}, {w.sampler} "
+                        f"{w.schedule or 'gamma=%g' % w.ula_gamma}, {w.denoiser} denoiser"
+                        + (f" ncomp={w.gmm['ncomp']}" if w.denoiser == 'gmm' else ""),
+            "drafter": "frozen target output (carried)", "seed": w.sample_seed,
+            "l2": "256 MiB buffer written between timed steps (working set may fit L2)",
+            "sharding": "chains by global id, no data-path collective"}
+
+
+# --------------------------------------------------------------------------------------------
+# clocks
+# --------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.path = tempfile.mktemp(prefix="sds_clocks_", suffix=".csv")
+        self.proc = None
+        self.idx = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.idx), "-lms", "100"], stdout=open(self.path, "w"),
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for ln in open(self.path):
+                f = [x.strip() for x in ln.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# --------------------------------------------------------------------------------------------
+# GPU arm
+# --------------------------------------------------------------------------------------------
+
+def algorithmic(kind: str, w, rows_per_step: float, windows_chains: float, launches: float):
+    """Algorithmic bytes or flops one average launch of `kind` must move / compute.
+    rows_per_step: target rows verified per step (sum of window lengths); windows_chains: chain-windows."""
+    d = w.d
+    if kind == "verify":        # two fp32 streams per verified chain-step (target output + drafted state)
+        return "hbm", 8.0 * d * rows_per_step / launches
+    if kind == "draft":         # read state + carried output, write the drafted rows
+        return "hbm", (8.0 * d * windows_chains + 4.0 * d * rows_per_step) / launches
+    if kind == "advance":
+        return "hbm", 16.0 * d * windows_chains / launches
+    if kind == "denoise":       # logits + mixing contractions
+        return "alu", 4.0 * w.gmm["ncomp"] * d * (rows_per_step + w.B) / launches
+    if kind == "fused":         # whole chain in one launch: mixture contractions dominate the arithmetic
+        return "alu", 4.0 * w.gmm["ncomp"] * d * (rows_per_step + w.B) / launches
+    return "hbm", 0.0
+
+
+def run_gpu(args, w):
+    import torch
+    import torch.distributed as dist
+    import paper_2501_05370_b200 as sds
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (no CPU fallback); use --impl reference for the oracle")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    s = sds.sampler_for(w, chain_id_offset=rank * w.B, device=dev)
+    B, d, K = w.B, w.d, w.K
+    out = torch.empty((B, d), dtype=torch.float32, device=dev)
+    calls = torch.empty((B,), dtype=torch.int32, device=dev)
+    rows = torch.empty((B,), dtype=torch.int32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    gp = w.gmm_params()
+    means_h = torch.from_numpy(gp.means).pin_memory()
+    logw_h = torch.from_numpy(gp.logw).pin_memory()
+    out_h = torch.empty((B, d), dtype=torch.float32).pin_memory()
+    calls_h = torch.empty((B,), dtype=torch.int32).pin_memory()
+    rows_h = torch.empty((B,), dtype=torch.int32).pin_memory()
+    stream = torch.cuda.current_stream()
+
+    def timed(fn, steps):
+        tot = 0.0
+        for _ in range(steps):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            fn()
+            e1.record(stream)
+            e1.synchronize()
+            tot += e0.elapsed_time(e1)
+        return tot
+
+    dev_step = lambda: s.sample_all(out, calls, rows)
+    e2e_step = lambda: s.sample_all_host(means_h, logw_h, out_h, calls_h, rows_h)
+
+    for _ in range(args.warmup):
+        dev_step()
+    clocks = ClockSampler(local)
+    barrier()
+    if rank == 0:
+        clocks.start()
+    l0 = s.launch_count()
+    s.profile(True)
+    s.profile_read(reset=True)
+    ms_total = timed(dev_step, args.steps)
+    barrier()
+    prof = s.profile_read(reset=True)
+    s.profile(False)
+    launches = s.launch_count() - l0
+    clk = clocks.stop() if rank == 0 else None
+    calls_np, rows_np = calls.cpu().numpy().astype(np.int64), rows.cpu().numpy().astype(np.int64)
+
+    # the same metric through the host-buffer entry point
+    for _ in range(min(args.warmup, 3)):
+        e2e_step()
+    barrier()
+    ms_e2e = timed(e2e_step, args.steps)
+    barrier()
+
+    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, ms_e2e = float(t[0]), float(t[1])
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    pk = peaks()
+    steps = args.steps
+    ms_per_step = ms_total / steps
+    value = world * B * K / (ms_per_step * 1e-3)
+    e2e_value = world * B * K / (ms_e2e / steps * 1e-3)
+    rows_per_step = float(rows_np.sum() - B)                  # rows verified (the initial call is not a window)
+    windows_chains = float(calls_np.sum() - B)
+    kinds = {k: v for k, v in prof.items() if v[1] > 0}
+    dom = max(kinds, key=lambda k: kinds[k][0]) if kinds else "fused"
+    dom_ms, dom_n = kinds.get(dom, (ms_total, steps))
+    bound, per_launch = algorithmic(dom, w, rows_per_step, windows_chains, dom_n / steps)
+    avg_s = dom_ms / max(dom_n, 1) * 1e-3
+    if bound == "hbm":
+        achieved, peak, unit = per_launch / avg_s / 1e9, pk["hbm_gbs"], "GB/s"
+    else:
+        peak = SMS * FP32_LANES_PER_SM * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
+        achieved, unit = per_launch / avg_s / 1e12, "TFLOP/s"
+    roofline = {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
+                "frac": achieved / peak, "traffic": None,
+                "peak_source": pk["source"] if bound == "hbm" else "derived: 148 SMs x 128 fp32 lanes x 2 x max SM clock",
+                "avg_launch_us": avg_s * 1e6, "launches_per_step": dom_n / steps,
+                "share_of_kernel_time": dom_ms / max(sum(v[0] for v in kinds.values()), 1e-9),
+                "kernel_ms_per_step": {k: v[0] / steps for k, v in kinds.items()}}
+
+    nchain, sec = oracle_time(w, args.cpu_seconds)
+    cpu = {"value": nchain * K / sec, "unit": UNIT, "cores": 1, "kind": "oracle",
+           "sample": f"{nchain} chains of {w.name} run to completion in {sec:.1f} s, one NumPy thread"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic", "config": workload_config(w, args),
+        "nfe": {"K": K, "mean_target_calls": float(calls_np.mean()), "mean_target_rows": float(rows_np.mean()),
+                "mean_advance": float(K * B / max(windows_chains, 1)), "calls_saved_frac": float(1 - calls_np.mean() / K)},
+        "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e / steps,
+                "h2d_bytes_per_step": int(means_h.numel() * 4 + logw_h.numel() * 4),
+                "d2h_bytes_per_step": int(out_h.numel() * 4 + calls_h.numel() * 4 + rows_h.numel() * 4)},
+        "gpu_launches": int(launches),
+        "roofline": roofline, "cpu_baseline": cpu, "clocks": clk,
+    }
+    print(json.dumps(line), flush=True)
+    s.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="sds", choices=["sds", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--cpu-seconds", type=float, default=15.0, help="budget of the cpu_baseline leg")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "sds":
+        args.warmup = 3
+    w = wl.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_gpu(args, w)
+
+
+if __name__ == "__main__":
+    main()

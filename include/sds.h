@@ -190,6 +190,22 @@ int sds_rng_uniforms(uint64_t seed, int64_t b0, int64_t nb, int32_t k, float* u_
 /* Number of kernels this context has launched since create (for launch accounting). */
 int64_t sds_launch_count(const sds_ctx* ctx);
 
+/* Per-kernel timing (measurement aid; the paper's only cost unit is the target call, Section 7).
+ * sds_profile(ctx, 1) makes every later kernel launch of the context bracketed by a pair of CUDA
+ * events on the bound stream; sds_profile_read waits for the stream and returns, per kernel kind,
+ * the summed device time in milliseconds (ms[SDS_PROF_KINDS], host) and the number of launches
+ * (launches[SDS_PROF_KINDS], host); reset != 0 clears the sums. Off by default. */
+#define SDS_PROF_INIT     0
+#define SDS_PROF_DENOISE  1
+#define SDS_PROF_DRAFT    2
+#define SDS_PROF_VERIFY   3
+#define SDS_PROF_ADVANCE  4
+#define SDS_PROF_FUSED    5     /* whole-chain persistent kernel */
+#define SDS_PROF_AUX      6     /* |mu|^2, list rebuild, copies of the initial call */
+#define SDS_PROF_KINDS    7
+int sds_profile(sds_ctx* ctx, int32_t enable);
+int sds_profile_read(sds_ctx* ctx, double* ms, int64_t* launches, int32_t reset);
+
 const char* sds_strerror(int code);
 int sds_last_cuda_error(const sds_ctx* ctx);
 void sds_destroy(sds_ctx* ctx);

@@ -55,6 +55,8 @@ EXPORTS = {
     "sds_rng_normals": (C.c_int, [C.c_uint64, C.c_int32, C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
     "sds_rng_uniforms": (C.c_int, [C.c_uint64, C.c_int64, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p]),
     "sds_launch_count": (C.c_int64, [C.c_void_p]),
+    "sds_profile": (C.c_int, [C.c_void_p, C.c_int32]),
+    "sds_profile_read": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32]),
     "sds_strerror": (C.c_char_p, [C.c_int]),
     "sds_last_cuda_error": (C.c_int, [C.c_void_p]),
     "sds_destroy": (None, [C.c_void_p]),
@@ -269,6 +271,18 @@ class Sampler:
         out = out if out is not None else t.empty_like(x)
         self._chk(self.lib.sds_denoise(self.h, x.data_ptr(), k.data_ptr(), x.shape[0], out.data_ptr()), "sds_denoise")
         return out
+
+    PROF_KINDS = ("init", "denoise", "draft", "verify", "advance", "fused", "aux")
+
+    def profile(self, enable: bool):
+        self._chk(self.lib.sds_profile(self.h, int(enable)), "sds_profile")
+
+    def profile_read(self, reset: bool = True) -> dict:
+        """{kind: (milliseconds, launches)} accumulated since the last reset."""
+        ms = np.zeros(len(self.PROF_KINDS), np.float64)
+        n = np.zeros(len(self.PROF_KINDS), np.int64)
+        self._chk(self.lib.sds_profile_read(self.h, ms.ctypes.data, n.ctypes.data, int(reset)), "sds_profile_read")
+        return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(self.PROF_KINDS)}
 
     def launch_count(self) -> int:
         return int(self.lib.sds_launch_count(self.h))

@@ -62,6 +62,12 @@ struct sds_ctx {
   int32_t* h_pin = nullptr;         // pinned host words for the window loop
   cudaEvent_t ev[2] = {nullptr, nullptr};
   bool musq_ready = false;
+  // optional per-kernel timing: event pairs recorded around each launch, summed on read
+  bool prof_on = false;
+  std::vector<cudaEvent_t> prof_ev[SDS_PROF_KINDS];
+  size_t prof_used[SDS_PROF_KINDS] = {};
+  double prof_ms[SDS_PROF_KINDS] = {};
+  int64_t prof_n[SDS_PROF_KINDS] = {};
 };
 
 namespace {
@@ -167,11 +173,47 @@ int cuda_fail(sds_ctx* c, cudaError_t e) {
     if (e_ != cudaSuccess) return cuda_fail((ctx), e_);     \
   } while (0)
 
+// event pair around one launch of the given kind (only when profiling is on)
+cudaError_t prof_mark(sds_ctx* c, int kind) {
+  if (!c->prof_on) return cudaSuccess;
+  std::vector<cudaEvent_t>& v = c->prof_ev[kind];
+  if (c->prof_used[kind] == v.size()) {
+    cudaEvent_t e;
+    const cudaError_t rc = cudaEventCreate(&e);
+    if (rc != cudaSuccess) return rc;
+    v.push_back(e);
+  }
+  return cudaEventRecord(v[c->prof_used[kind]++], c->stream);
+}
+
+// fold finished event pairs into the sums (the stream must be idle)
+void prof_collect(sds_ctx* c) {
+  for (int k = 0; k < SDS_PROF_KINDS; ++k) {
+    for (size_t i = 0; i + 1 < c->prof_used[k]; i += 2) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, c->prof_ev[k][i], c->prof_ev[k][i + 1]) == cudaSuccess) {
+        c->prof_ms[k] += ms;
+        c->prof_n[k] += 1;
+      } else {
+        cudaGetLastError();
+      }
+    }
+    c->prof_used[k] = 0;
+  }
+}
+
+#define SDS_LAUNCH(ctx, kind, expr)            \
+  do {                                         \
+    SDS_CU(ctx, prof_mark(ctx, kind));         \
+    SDS_CU(ctx, expr);                         \
+    SDS_CU(ctx, prof_mark(ctx, kind));         \
+    (ctx)->launches++;                         \
+  } while (0)
+
 int ensure_musq(sds_ctx* c) {
   if (c->musq_ready) return SDS_OK;
-  SDS_CU(c, launch_musq(static_cast<const float*>(c->den.means_dev), c->den.ncomp, c->d, at<float>(c, c->lay.musq),
-                        c->stream));
-  c->launches++;
+  SDS_LAUNCH(c, SDS_PROF_AUX, launch_musq(static_cast<const float*>(c->den.means_dev), c->den.ncomp, c->d,
+                                          at<float>(c, c->lay.musq), c->stream));
   c->musq_ready = true;
   return SDS_OK;
 }
@@ -184,8 +226,7 @@ int run_denoiser(sds_ctx* c, const float* X, const int* rowk, const int* nrows_d
     case SDS_DEN_GMM: {
       const int rc = ensure_musq(c);
       if (rc != SDS_OK) return rc;
-      SDS_CU(c, launch_gmm_f32(gmm_args(c), X, rowk, nrows_dev, (int)rows_ub, out, c->stream));
-      c->launches++;
+      SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gmm_f32(gmm_args(c), X, rowk, nrows_dev, (int)rows_ub, out, c->stream));
       return SDS_OK;
     }
     case SDS_DEN_CALLBACK: {
@@ -292,13 +333,11 @@ int sds_reset(sds_ctx* c) {
   if (!c) return SDS_EINVAL;
   if (c->state < kBound) return SDS_ESTATE;
   WinArgs A = win_args(c);
-  SDS_CU(c, launch_init(A, c->stream));
-  c->launches++;
+  SDS_LAUNCH(c, SDS_PROF_INIT, launch_init(A, c->stream));
   const int rc = run_denoiser(c, A.X, A.rowk, A.ctl + kCtlNRows, c->B, A.Dq);
   if (rc != SDS_OK) return rc;
-  SDS_CU(c, launch_after_init(A, c->stream));
-  SDS_CU(c, launch_compact(A, c->stream));
-  c->launches += 2;
+  SDS_LAUNCH(c, SDS_PROF_AUX, launch_after_init(A, c->stream));
+  SDS_LAUNCH(c, SDS_PROF_AUX, launch_compact(A, c->stream));
   c->ub = (int)c->B;
   c->state = kReady;
   return SDS_OK;
@@ -307,8 +346,7 @@ int sds_reset(sds_ctx* c) {
 int sds_draft(sds_ctx* c) {
   if (!c) return SDS_EINVAL;
   if (c->state != kReady) return SDS_ESTATE;
-  SDS_CU(c, launch_draft(win_args(c), c->ub, c->stream));
-  c->launches++;
+  SDS_LAUNCH(c, SDS_PROF_DRAFT, launch_draft(win_args(c), c->ub, c->stream));
   c->state = kDrafted;
   return SDS_OK;
 }
@@ -319,8 +357,7 @@ int sds_verify_window(sds_ctx* c) {
   WinArgs A = win_args(c);
   const int rc = run_denoiser(c, A.X, A.rowk, A.ctl + kCtlNRows, (int64_t)c->ub * c->L, A.Dq);
   if (rc != SDS_OK) return rc;
-  SDS_CU(c, launch_verify(A, c->ub, c->stream));
-  c->launches++;
+  SDS_LAUNCH(c, SDS_PROF_VERIFY, launch_verify(A, c->ub, c->stream));
   c->state = kVerified;
   return SDS_OK;
 }
@@ -328,8 +365,7 @@ int sds_verify_window(sds_ctx* c) {
 int sds_advance(sds_ctx* c, int64_t* n_active) {
   if (!c) return SDS_EINVAL;
   if (c->state != kVerified) return SDS_ESTATE;
-  SDS_CU(c, launch_advance(win_args(c), c->ub, c->stream));
-  c->launches++;
+  SDS_LAUNCH(c, SDS_PROF_ADVANCE, launch_advance(win_args(c), c->ub, c->stream));
   c->state = kReady;
   if (n_active) return sync_active(c, n_active);
   return SDS_OK;
@@ -342,8 +378,7 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
   int rc = SDS_OK;
   if (c->den.kind == SDS_DEN_GMM && fused_small_supported(c->d, c->den.ncomp, c->L)) {
     if ((rc = ensure_musq(c)) != SDS_OK) return rc;
-    SDS_CU(c, launch_fused_small(A, gmm_args(c), c->stream));
-    c->launches++;
+    SDS_LAUNCH(c, SDS_PROF_FUSED, launch_fused_small(A, gmm_args(c), c->stream));
     c->ub = 0;
     c->state = kReady;
   } else {
@@ -444,8 +479,7 @@ int sds_set_state(sds_ctx* c, const float* Y_dev, const int32_t* n_dev, const fl
   if (Dc_dev) SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.Dc, Dc_dev, Bd, cudaMemcpyDeviceToDevice, c->stream));
   if (n_dev)
     SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.n, n_dev, (size_t)c->B * 4, cudaMemcpyDeviceToDevice, c->stream));
-  SDS_CU(c, launch_compact(win_args(c), c->stream));
-  c->launches++;
+  SDS_LAUNCH(c, SDS_PROF_AUX, launch_compact(win_args(c), c->stream));
   c->ub = (int)c->B;
   return SDS_OK;
 }
@@ -475,6 +509,26 @@ int sds_rng_uniforms(uint64_t seed, int64_t b0, int64_t nb, int32_t k, float* u_
 
 int64_t sds_launch_count(const sds_ctx* c) { return c ? c->launches : 0; }
 
+int sds_profile(sds_ctx* c, int32_t enable) {
+  if (!c) return SDS_EINVAL;
+  if (c->state >= kBound) SDS_CU(c, cudaStreamSynchronize(c->stream));
+  prof_collect(c);
+  c->prof_on = enable != 0;
+  return SDS_OK;
+}
+
+int sds_profile_read(sds_ctx* c, double* ms, int64_t* launches, int32_t reset) {
+  if (!c || !ms || !launches) return SDS_EINVAL;
+  if (c->state >= kBound) SDS_CU(c, cudaStreamSynchronize(c->stream));
+  prof_collect(c);
+  for (int k = 0; k < SDS_PROF_KINDS; ++k) {
+    ms[k] = c->prof_ms[k];
+    launches[k] = c->prof_n[k];
+    if (reset) { c->prof_ms[k] = 0.0; c->prof_n[k] = 0; }
+  }
+  return SDS_OK;
+}
+
 const char* sds_strerror(int code) {
   switch (code) {
     case SDS_OK: return "ok";
@@ -496,6 +550,8 @@ void sds_destroy(sds_ctx* c) {
   if (!c) return;
   for (int i = 0; i < 2; ++i)
     if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+  for (int k = 0; k < SDS_PROF_KINDS; ++k)
+    for (cudaEvent_t e : c->prof_ev[k]) cudaEventDestroy(e);
   if (c->h_pin) cudaFreeHost(c->h_pin);
   delete c;
 }
