@@ -206,6 +206,30 @@ int64_t sds_launch_count(const sds_ctx* ctx);
 int sds_profile(sds_ctx* ctx, int32_t enable);
 int sds_profile_read(sds_ctx* ctx, double* ms, int64_t* launches, int32_t reset);
 
+/* Mixture denoiser pass that allocates nothing and needs no context or workspace.
+ * (The paper has no counterpart: this call exists for the way the library is deployed.)
+ * For callers that cannot obtain device memory when they need a target pass: code running inside
+ * a host application that owns the GPU memory pool, code that must not hit the implicit
+ * device synchronisation of an allocation, or a process whose memory budget is fixed at start-up.
+ * Computes out_dev[r] = D(x_dev[r], k_dev[r]) exactly as sds_denoise does for a float mixture:
+ *   x_dev [rows, d] float, k_dev [rows] int32 in [0, K), means_dev [ncomp, d] float,
+ *   logw_dev [ncomp] float, tcond_dev [K, 4] float (A, Bq, C, E per step, device), out_dev [rows, d].
+ * All pointers are device pointers owned by the caller; work is enqueued on cuda_stream
+ * (cudaStream_t, NULL = default stream) of the current device and the call does not wait for it.
+ * The |mu_c|^2 table the kernel needs lives in a fixed array inside the library (16 KiB on every
+ * GPU that loads it, until the process exits), so ncomp <= SDS_STATIC_MAX_NCOMP; larger mixtures
+ * return SDS_EUNSUPPORTED and do nothing. The call never calls cudaMalloc/cudaFree or any
+ * allocating routine.
+ * The first call on each device looks up the array's device address; make that first call
+ * outside any stream capture.
+ * Every call on a device shares the one array and overwrites the entries it uses (nothing needs
+ * clearing between calls); two calls whose kernels can overlap on the GPU (different streams, no
+ * ordering between them) race on it - order them on one stream or with events. */
+#define SDS_STATIC_MAX_NCOMP 4096
+int sds_gmm_denoise_static(const float* x_dev, const int32_t* k_dev, int64_t rows, int32_t d, int32_t ncomp,
+                           const float* means_dev, const float* logw_dev, const float* tcond_dev, int32_t K,
+                           float* out_dev, void* cuda_stream);
+
 const char* sds_strerror(int code);
 int sds_last_cuda_error(const sds_ctx* ctx);
 void sds_destroy(sds_ctx* ctx);

@@ -57,6 +57,8 @@ EXPORTS = {
     "sds_launch_count": (C.c_int64, [C.c_void_p]),
     "sds_profile": (C.c_int, [C.c_void_p, C.c_int32]),
     "sds_profile_read": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32]),
+    "sds_gmm_denoise_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                         C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
     "sds_strerror": (C.c_char_p, [C.c_int]),
     "sds_last_cuda_error": (C.c_int, [C.c_void_p]),
     "sds_destroy": (None, [C.c_void_p]),
@@ -303,4 +305,19 @@ def rng_uniforms(seed: int, b0: int, nb: int, k: int, device="cuda:0"):
     rc = load().sds_rng_uniforms(seed, b0, nb, k, out.data_ptr(), torch.cuda.current_stream().cuda_stream)
     if rc != SDS_OK:
         raise SdsError(rc, "sds_rng_uniforms")
+    return out
+
+
+STATIC_MAX_NCOMP = 4096
+
+
+def gmm_denoise_static(x, k, means, logw, tcond, out):
+    """sds_gmm_denoise_static on torch CUDA tensors (all caller-allocated, including out): a mixture
+    denoiser pass for callers that cannot allocate device memory. Enqueues on the current stream."""
+    import torch
+    rc = load().sds_gmm_denoise_static(x.data_ptr(), k.data_ptr(), x.shape[0], x.shape[1], means.shape[0],
+                                       means.data_ptr(), logw.data_ptr(), tcond.data_ptr(), tcond.shape[0],
+                                       out.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    if rc != SDS_OK:
+        raise SdsError(rc, "sds_gmm_denoise_static")
     return out
