@@ -164,6 +164,12 @@ int sds_advance(sds_ctx* ctx, int64_t* n_active);
  * Small float mixtures run as one persistent kernel, one warp per chain, same results. */
 int sds_sample_all(sds_ctx* ctx, float* out_dev, int32_t* nfe_calls_dev, int32_t* nfe_rows_dev);
 
+/* Options. SDS_OPT_WHOLE_CHAIN_KERNEL (default 1): let sds_sample_all run small float mixtures
+ * (d <= 256, <= 32 components) as one persistent kernel; 0 forces the window-by-window kernels.
+ * After the whole-chain kernel only Y, N, DC and the NFE counters are meaningful for sds_get. */
+#define SDS_OPT_WHOLE_CHAIN_KERNEL 1
+int sds_set_option(sds_ctx* ctx, int32_t option, int64_t value);
+
 /* Same with host buffers: copies the mixture parameters means_host [ncomp, d] / logw_host [ncomp]
  * (float; NULL = keep what is on the device) to the device arrays named at create, runs
  * sds_sample_all, copies the results to host memory. All copies are on the bound stream. */

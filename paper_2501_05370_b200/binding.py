@@ -55,6 +55,7 @@ EXPORTS = {
     "sds_rng_normals": (C.c_int, [C.c_uint64, C.c_int32, C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
     "sds_rng_uniforms": (C.c_int, [C.c_uint64, C.c_int64, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p]),
     "sds_launch_count": (C.c_int64, [C.c_void_p]),
+    "sds_set_option": (C.c_int, [C.c_void_p, C.c_int32, C.c_int64]),
     "sds_profile": (C.c_int, [C.c_void_p, C.c_int32]),
     "sds_profile_read": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32]),
     "sds_gmm_denoise_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
@@ -273,6 +274,11 @@ class Sampler:
         out = out if out is not None else t.empty_like(x)
         self._chk(self.lib.sds_denoise(self.h, x.data_ptr(), k.data_ptr(), x.shape[0], out.data_ptr()), "sds_denoise")
         return out
+
+    OPT_WHOLE_CHAIN_KERNEL = 1
+
+    def set_option(self, option: int, value: int):
+        self._chk(self.lib.sds_set_option(self.h, option, value), "sds_set_option")
 
     PROF_KINDS = ("init", "denoise", "draft", "verify", "advance", "fused", "aux")
 

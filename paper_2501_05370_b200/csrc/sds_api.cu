@@ -62,6 +62,7 @@ struct sds_ctx {
   int32_t* h_pin = nullptr;         // pinned host words for the window loop
   cudaEvent_t ev[2] = {nullptr, nullptr};
   bool musq_ready = false;
+  bool whole_chain = true;          // sds_sample_all may use the whole-chain kernel
   // optional per-kernel timing: event pairs recorded around each launch, summed on read
   bool prof_on = false;
   std::vector<cudaEvent_t> prof_ev[SDS_PROF_KINDS];
@@ -376,8 +377,9 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
   if (c->state < kBound) return SDS_ESTATE;
   WinArgs A = win_args(c);
   int rc = SDS_OK;
-  if (c->den.kind == SDS_DEN_GMM && fused_small_supported(c->d, c->den.ncomp, c->L)) {
+  if (c->whole_chain && c->den.kind == SDS_DEN_GMM && fused_small_supported(c->d, c->den.ncomp, c->L)) {
     if ((rc = ensure_musq(c)) != SDS_OK) return rc;
+    SDS_CU(c, cudaMemsetAsync(A.ctl, 0, kCtlWords * 4, c->stream));   // no chain active afterwards, error bits clear
     SDS_LAUNCH(c, SDS_PROF_FUSED, launch_fused_small(A, gmm_args(c), c->stream));
     c->ub = 0;
     c->state = kReady;
@@ -508,6 +510,14 @@ int sds_rng_uniforms(uint64_t seed, int64_t b0, int64_t nb, int32_t k, float* u_
 }
 
 int64_t sds_launch_count(const sds_ctx* c) { return c ? c->launches : 0; }
+
+int sds_set_option(sds_ctx* c, int32_t option, int64_t value) {
+  if (!c) return SDS_EINVAL;
+  switch (option) {
+    case SDS_OPT_WHOLE_CHAIN_KERNEL: c->whole_chain = value != 0; return SDS_OK;
+    default: return SDS_EINVAL;
+  }
+}
 
 int sds_profile(sds_ctx* c, int32_t enable) {
   if (!c) return SDS_EINVAL;

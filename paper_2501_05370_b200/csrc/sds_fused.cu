@@ -1,10 +1,240 @@
-// Whole-chain persistent kernel for small float mixtures (placeholder until the kernel lands).
+// Whole-chain persistent kernel for small float mixtures: one warp carries one chain through
+// every window (draft, target rows, verify, reflection, advance) with the window buffer, the
+// mixture and the carried output in shared memory. Nothing but the final state and the counters
+// touches HBM. At these sizes (d <= 256, <= 32 components) the step-wise path is launch-bound;
+// here the bound is plain ALU work (Philox, Box-Muller, the mixture's dot products).
+//
+// Per-element arithmetic and the reduction trees are those of the step-wise kernels
+// (sds_device.cuh, sds_gmm_small.cuh), so both paths return the same bits.
 #include "sds_device.cuh"
+#include "sds_gmm_small.cuh"
 #include "sds_internal.h"
 
 namespace sds {
 
-bool fused_small_supported(int, int, int) { return false; }
-cudaError_t launch_fused_small(const WinArgs&, const GmmArgs&, cudaStream_t) { return cudaErrorNotSupported; }
+namespace {
+
+// floats of shared memory: parameters (rounded to 16 bytes) and per-warp window storage
+__host__ __device__ inline int fused_param_floats(int ncomp, int d) {
+  return (ncomp * small_ldm(d) + 2 * ncomp + 3) / 4 * 4;
+}
+__host__ __device__ inline int fused_warp_floats(int d, int L) {
+  return (2 * L + 2) * small_ldx(d) + 32 + 4 * kMaxL;   // W[L+1], Dq[L], Dc, e-scratch, S1/S2 as doubles
+}
+
+template <int G, bool VEC4>
+__global__ void k_fused_small(WinArgs A, GmmArgs P) {
+  extern __shared__ __align__(16) float smem[];
+  constexpr int RPW = 32 / G;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  const int g = lane / G, gl = lane % G;
+  const int d = A.d, L = A.L, K = A.K;
+  const int ldm = small_ldm(d), ldx = small_ldx(d);
+  float* s_means = smem;
+  float* s_musq = s_means + P.ncomp * ldm;
+  float* s_logw = s_musq + P.ncomp;
+  float* sW = smem + fused_param_floats(P.ncomp, d) + (size_t)warp * fused_warp_floats(d, L);
+  float* sDq = sW + (L + 1) * ldx;
+  float* sDc = sDq + L * ldx;
+  float* sEs = sDc + ldx;
+  double* sS = reinterpret_cast<double*>(sEs + 32);           // [2][kMaxL]
+  small_stage_params(P.means, P.musq, P.logw, P.ncomp, d, s_means, s_musq, s_logw);
+  __syncthreads();
+
+  // verify lane mapping: same partition as the step-wise warp-per-chain kernel; when only the
+  // lower half-warp would hold elements, the two halves take two positions at once
+  const bool pack2 = VEC4 ? (d <= 64) : (d <= 16);
+  const int PW = pack2 ? 16 : 32;
+  const int vh = lane / PW, vt = lane % PW;
+
+  for (int b = blockIdx.x * nwarps + warp; b < A.B; b += gridDim.x * nwarps) {
+    const uint64_t bg = A.chain_off + (uint64_t)b;
+    // I0: Y_0 and the carried output D(Y_0, 0)
+    if (VEC4) {
+      for (int q = lane; q < d / 4; q += 32) st4(sW + 4 * q, normal4(A.seed, kStreamInit, bg, 0u, (uint32_t)q));
+    } else {
+      for (int i = lane; i < d; i += 32) sW[i] = normal1(A.seed, kStreamInit, bg, 0u, (uint32_t)i);
+    }
+    __syncwarp();
+    gmm_row_small<G>(sW, g == 0, s_means, ldm, s_musq, s_logw, P.ncomp, d, __ldg(P.tcond + 0), __ldg(P.tcond + 1),
+                     __ldg(P.tcond + 2), __ldg(P.tcond + 3), sEs + g * G, sDc, gl);
+    int n = 0, calls = 1, rows = 1;
+    bool frozen = false;
+    while (n < K) {
+      const int Lt = min(L, K - n);
+      // draft noise for all positions at once, then the sequential recurrence per element
+      if (VEC4) {
+        const int nq = d / 4;
+        for (int e = lane; e < Lt * nq; e += 32) {
+          const int j = e / nq, q = e - j * nq;
+          st4(sW + (j + 1) * ldx + 4 * q, normal4(A.seed, kStreamDraft, bg, (uint32_t)(n + j), (uint32_t)q));
+        }
+      } else {
+        for (int e = lane; e < Lt * d; e += 32) {
+          const int j = e / d, i = e - j * d;
+          sW[(j + 1) * ldx + i] = normal1(A.seed, kStreamDraft, bg, (uint32_t)(n + j), (uint32_t)i);
+        }
+      }
+      __syncwarp();
+      for (int i = lane; i < d; i += 32) {
+        float y = sW[i];
+        const float dc = sDc[i];
+        for (int j = 0; j < Lt; ++j) {
+          const int k = n + j;
+          y = draft_step(y, dc, sW[(j + 1) * ldx + i], __ldg(A.a + k), __ldg(A.c + k), __ldg(A.sigma + k));
+          sW[(j + 1) * ldx + i] = y;
+        }
+      }
+      __syncwarp();
+      // target rows W_0 .. W_{Lt-1}
+      for (int j0 = 0; j0 < Lt; j0 += RPW) {
+        const int j = j0 + g;
+        const bool valid = j < Lt;
+        const int jj = valid ? j : 0;
+        const int k = n + jj;
+        gmm_row_small<G>(sW + jj * ldx, valid, s_means, ldm, s_musq, s_logw, P.ncomp, d, __ldg(P.tcond + 4 * k + 0),
+                         __ldg(P.tcond + 4 * k + 1), __ldg(P.tcond + 4 * k + 2), __ldg(P.tcond + 4 * k + 3),
+                         sEs + g * G, sDq + jj * ldx, gl);
+      }
+      // S1 = |Delta|^2, S2 = Delta.Z per position
+      for (int j0 = 1; j0 <= Lt; j0 += (pack2 ? 2 : 1)) {
+        const int j = j0 + vh;
+        double p1 = 0.0, p2 = 0.0;
+        if (j <= Lt) {
+          const int k = n + j - 1;
+          const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
+          const float inv_s = 1.0f / sk, cs = ck * inv_s;
+          const float* wp = sW + (j - 1) * ldx;
+          const float* wj = sW + j * ldx;
+          const float* dq = sDq + (j - 1) * ldx;
+          if (VEC4) {
+            for (int i = vt * 4; i < d; i += 128) {
+              const float4 vp = ld4(wp + i), vj = ld4(wj + i), vq = ld4(dq + i), vc = ld4(sDc + i);
+              float D, Z;
+              delta_z(vp.x, vj.x, vq.x, vc.x, ak, ck, cs, inv_s, D, Z);
+              p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+              delta_z(vp.y, vj.y, vq.y, vc.y, ak, ck, cs, inv_s, D, Z);
+              p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+              delta_z(vp.z, vj.z, vq.z, vc.z, ak, ck, cs, inv_s, D, Z);
+              p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+              delta_z(vp.w, vj.w, vq.w, vc.w, ak, ck, cs, inv_s, D, Z);
+              p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+            }
+          } else {
+            for (int i = vt; i < d; i += 32) {
+              float D, Z;
+              delta_z(wp[i], wj[i], dq[i], sDc[i], ak, ck, cs, inv_s, D, Z);
+              p1 = fma((double)D, (double)D, p1);
+              p2 = fma((double)D, (double)Z, p2);
+            }
+          }
+        }
+        for (int o = PW / 2; o > 0; o >>= 1) {
+          p1 += __shfl_xor_sync(0xffffffffu, p1, o);
+          p2 += __shfl_xor_sync(0xffffffffu, p2, o);
+        }
+        if (vt == 0 && j <= Lt) { sS[j - 1] = p1; sS[kMaxL + j - 1] = p2; }
+      }
+      __syncwarp();
+      // accept tests for all positions at once, first rejection by ballot
+      const bool valid = lane < Lt;
+      bool acc = true, bad = false;
+      double myS1 = 1.0, myS2 = 0.0;
+      if (valid) {
+        myS1 = sS[lane];
+        myS2 = sS[kMaxL + lane];
+        const float lu = logf(uniform01(A.seed, bg, (uint32_t)(n + lane)));
+        const float ellf = (float)(-0.5 * myS1 - myS2);
+        acc = (myS1 < 1e-30) || (lu <= ellf);
+        bad = !isfinite(ellf);
+      }
+      const uint32_t vmask = (Lt >= 32) ? 0xffffffffu : ((1u << Lt) - 1u);
+      const uint32_t amask = __ballot_sync(0xffffffffu, acc) & vmask;
+      const uint32_t bmask = __ballot_sync(0xffffffffu, bad) & vmask;
+      const uint32_t rej = ~amask & vmask;
+      int jstar = rej ? __ffs(rej) : Lt + 1;
+      if (bmask) { frozen = true; break; }
+      const float coef = __shfl_sync(0xffffffffu, (float)(2.0 * myS2 / myS1), (jstar <= Lt) ? jstar - 1 : 0);
+      if (jstar <= Lt) {                                       // reflection of the rejected draft
+        const int k = n + jstar - 1;
+        const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
+        const float inv_s = 1.0f / sk, cs = ck * inv_s;
+        const float* wp = sW + (jstar - 1) * ldx;
+        float* wj = sW + jstar * ldx;
+        const float* dq = sDq + (jstar - 1) * ldx;
+        for (int i = lane; i < d; i += 32) {
+          float D, Z;
+          delta_z(wp[i], wj[i], dq[i], sDc[i], ak, ck, cs, inv_s, D, Z);
+          wj[i] = reflect_elem(wp[i], dq[i], Z, D, ak, ck, sk, coef);
+        }
+      }
+      __syncwarp();
+      const int adv = min(jstar, Lt);                           // restart at the accepted prefix
+      for (int i = lane; i < d; i += 32) {
+        sW[i] = sW[adv * ldx + i];
+        sDc[i] = sDq[(adv - 1) * ldx + i];
+      }
+      __syncwarp();
+      n += adv;
+      calls += 1;
+      rows += Lt;
+    }
+    for (int i = lane; i < d; i += 32) {
+      A.Y[(size_t)b * d + i] = sW[i];
+      A.Dc[(size_t)b * d + i] = sDc[i];
+    }
+    if (lane == 0) {
+      A.n[b] = K;
+      A.nfe_calls[b] = calls;
+      A.nfe_rows[b] = rows;
+      if (frozen) {
+        atomicOr(A.ctl + kCtlError, kErrNonFinite);
+        atomicAdd(A.ctl + kCtlFrozen, 1);
+      }
+    }
+    __syncwarp();
+  }
+}
+
+int fused_warps(int d, int ncomp, int L) {
+  for (int w = 8; w >= 2; w >>= 1) {
+    const size_t bytes = ((size_t)fused_param_floats(ncomp, d) + (size_t)w * fused_warp_floats(d, L)) * 4;
+    if (bytes <= 100 * 1024) return w;
+  }
+  return 0;
+}
+
+}  // namespace
+
+bool fused_small_supported(int d, int ncomp, int L) {
+  return d <= 256 && ncomp <= kSmallMaxComp && L <= kMaxL && fused_warps(d, ncomp, L) > 0;
+}
+
+cudaError_t launch_fused_small(const WinArgs& A, const GmmArgs& P, cudaStream_t st) {
+  const int w = fused_warps(A.d, P.ncomp, A.L);
+  if (w == 0) return cudaErrorInvalidConfiguration;
+  const size_t smem = ((size_t)fused_param_floats(P.ncomp, A.d) + (size_t)w * fused_warp_floats(A.d, A.L)) * 4;
+  int blocks = (A.B + w - 1) / w;
+  const int cap = 148 * 16;
+  if (blocks > cap) blocks = cap;
+  const bool vec4 = (A.d % 4) == 0;
+  const int grp = small_group(P.ncomp);
+#define SDS_FUSED_LAUNCH(GG, VV)                                                                              \
+  do {                                                                                                        \
+    if (smem > 48 * 1024) {                                                                                   \
+      const cudaError_t e_ =                                                                                  \
+          cudaFuncSetAttribute(k_fused_small<GG, VV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+      if (e_ != cudaSuccess) return e_;                                                                       \
+    }                                                                                                         \
+    k_fused_small<GG, VV><<<blocks, w * 32, smem, st>>>(A, P);                                                \
+  } while (0)
+  if (grp == 16) {
+    if (vec4) SDS_FUSED_LAUNCH(16, true); else SDS_FUSED_LAUNCH(16, false);
+  } else {
+    if (vec4) SDS_FUSED_LAUNCH(32, true); else SDS_FUSED_LAUNCH(32, false);
+  }
+#undef SDS_FUSED_LAUNCH
+  return cudaGetLastError();
+}
 
 }  // namespace sds

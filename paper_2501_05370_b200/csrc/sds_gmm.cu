@@ -4,6 +4,7 @@
 // variance-preserving diffusion of the mixture and the mixture's energy gradient both take this
 // form. One warp per row; the means are staged in shared memory when they fit.
 #include "sds_device.cuh"
+#include "sds_gmm_small.cuh"
 #include "sds_internal.h"
 
 namespace sds {
@@ -75,6 +76,52 @@ __global__ void __launch_bounds__(kGmmWarps * 32) k_gmm_f32(GmmArgs G, const flo
   }
 }
 
+// Small mixtures (ncomp <= 32, means fit shared memory): G lanes per row, 32/G rows per warp at a
+// time, rows staged in shared memory. smem: [means padded][musq][logw][per warp: rows, e-scratch]
+constexpr int kSmallWarps = 8;
+
+template <int G>
+__global__ void __launch_bounds__(kSmallWarps * 32) k_gmm_small(GmmArgs P, const float* __restrict__ X,
+                                                                const int* __restrict__ rowk,
+                                                                const int* __restrict__ nrows_dev, int rows_host,
+                                                                float* __restrict__ out) {
+  extern __shared__ float smem[];
+  constexpr int RPW = 32 / G;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane / G, gl = lane % G;
+  const int nrows = nrows_dev ? min(*nrows_dev, rows_host) : rows_host;
+  const int ldm = small_ldm(P.d), ldx = small_ldx(P.d);
+  float* s_means = smem;
+  float* s_musq = s_means + P.ncomp * ldm;
+  float* s_logw = s_musq + P.ncomp;
+  float* s_x = s_logw + P.ncomp + (size_t)warp * (RPW * ldx + 32);
+  float* s_es = s_x + RPW * ldx + g * G;
+  small_stage_params(P.means, P.musq, P.logw, P.ncomp, P.d, s_means, s_musq, s_logw);
+  __syncthreads();
+  const int stride = gridDim.x * kSmallWarps * RPW;
+  for (int row0 = (blockIdx.x * kSmallWarps + warp) * RPW; row0 < nrows; row0 += stride) {
+    for (int e = lane; e < RPW * P.d; e += 32) {
+      const int r = e / P.d, i = e - r * P.d;
+      if (row0 + r < nrows) s_x[r * ldx + i] = X[(size_t)(row0 + r) * P.d + i];
+    }
+    __syncwarp();
+    const int row = row0 + g;
+    const bool valid = row < nrows;
+    float tA = 0.f, tB = 0.f, tC = 0.f, tE = 0.f;
+    if (valid) {
+      const int k = rowk[row];
+      tA = __ldg(P.tcond + 4 * k + 0); tB = __ldg(P.tcond + 4 * k + 1);
+      tC = __ldg(P.tcond + 4 * k + 2); tE = __ldg(P.tcond + 4 * k + 3);
+    }
+    gmm_row_small<G>(s_x + g * ldx, valid, s_means, ldm, s_musq, s_logw, P.ncomp, P.d, tA, tB, tC, tE, s_es,
+                     out + (size_t)(valid ? row : 0) * P.d, gl);
+  }
+}
+
+size_t small_smem_bytes(int ncomp, int d) {
+  const int G = small_group(ncomp), RPW = 32 / G;
+  return ((size_t)ncomp * small_ldm(d) + 2 * (size_t)ncomp + (size_t)kSmallWarps * (RPW * small_ldx(d) + 32)) * 4;
+}
+
 }  // namespace
 
 cudaError_t launch_musq(const float* means, int ncomp, int d, float* musq, cudaStream_t st) {
@@ -85,6 +132,27 @@ cudaError_t launch_musq(const float* means, int ncomp, int d, float* musq, cudaS
 
 cudaError_t launch_gmm_f32(const GmmArgs& G, const float* X, const int* rowk, const int* nrows_dev, int rows_ub,
                            float* out, cudaStream_t st) {
+  if (G.ncomp <= kSmallMaxComp && small_smem_bytes(G.ncomp, G.d) <= 200 * 1024) {
+    const size_t smem = small_smem_bytes(G.ncomp, G.d);
+    const int grp = small_group(G.ncomp), rows_per_cta = kSmallWarps * (32 / grp);
+    int blocks = (rows_ub + rows_per_cta - 1) / rows_per_cta;
+    if (blocks > 148 * 4) blocks = 148 * 4;
+    if (blocks < 1) blocks = 1;
+    if (grp == 16) {
+      if (smem > 48 * 1024) {
+        const cudaError_t e = cudaFuncSetAttribute(k_gmm_small<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+      }
+      k_gmm_small<16><<<blocks, kSmallWarps * 32, smem, st>>>(G, X, rowk, nrows_dev, rows_ub, out);
+    } else {
+      if (smem > 48 * 1024) {
+        const cudaError_t e = cudaFuncSetAttribute(k_gmm_small<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+      }
+      k_gmm_small<32><<<blocks, kSmallWarps * 32, smem, st>>>(G, X, rowk, nrows_dev, rows_ub, out);
+    }
+    return cudaGetLastError();
+  }
   const size_t means_bytes = (size_t)G.ncomp * G.d * sizeof(float);
   const size_t logit_bytes = (size_t)kGmmWarps * G.ncomp * sizeof(float);
   const bool in_smem = means_bytes + logit_bytes <= 96 * 1024;

@@ -237,6 +237,25 @@ def test_stepwise_loop_equals_sample_all_and_is_deterministic():
     s.close()
 
 
+FUSED_SHAPES = [(64, 2, 4, 100, 4), (300, 64, 8, 200, 16), (65, 33, 5, 23, 7), (3, 5, 2, 9, 3), (1, 1, 1, 6, 2),
+                (9, 3, 32, 70, 4), (20, 128, 6, 40, 20), (10, 256, 4, 30, 32), (40, 16, 8, 50, 16), (40, 20, 8, 50, 17),
+                (33, 68, 3, 31, 9)]
+
+
+@pytest.mark.parametrize("B,d,L,K,ncomp", FUSED_SHAPES)
+def test_whole_chain_kernel_equals_window_kernels_bitwise(B, d, L, K, ncomp):
+    for name in ("cfg2", "cfg5"):
+        w = wl.WORKLOADS[name].scaled(B=B, d=d, L=L, K=K)
+        gp = w.gmm_params(d=d, ncomp=ncomp)
+        s = sds.sampler_for(w, gmm=gp, seed=77 + d, chain_id_offset=5)
+        f = [x.cpu().numpy() for x in s.sample_all()]
+        s.set_option(s.OPT_WHOLE_CHAIN_KERNEL, 0)
+        g = [x.cpu().numpy() for x in s.sample_all()]
+        assert np.array_equal(f[0], g[0]) and np.array_equal(f[1], g[1]) and np.array_equal(f[2], g[2])
+        assert np.all(np.isfinite(f[0]))
+        s.close()
+
+
 def test_chain_shards_reproduce_the_unsharded_run_bitwise():
     w = wl.WORKLOADS["cfg2"].scaled(B=96, K=50)
     gp = w.gmm_params()
@@ -260,6 +279,9 @@ def test_identical_drafter_and_target_accepts_everything():
     gp = w.gmm_params()
     a, c, sig, tcond = sds.schedule_for(w)
     s = sb.Sampler(a, np.zeros_like(c), sig, 32, w.d, w.L, gmm_means=gp.means, gmm_logw=gp.logw, tcond=tcond, seed=3)
+    out, calls, rows = s.sample_all()
+    assert np.array_equal(calls.cpu().numpy(), np.full(32, 1 + math.ceil(30 / w.L)))
+    s.set_option(s.OPT_WHOLE_CHAIN_KERNEL, 0)          # window-by-window kernels keep S1 for inspection
     out, calls, rows = s.sample_all()
     # Delta = 0 everywhere: every window is accepted in full
     assert np.array_equal(calls.cpu().numpy(), np.full(32, 1 + math.ceil(30 / w.L)))
