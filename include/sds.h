@@ -85,13 +85,14 @@ typedef struct sds_ctx sds_ctx;   /* opaque, owned by the library */
 /* Transition schedule, caller-owned host arrays copied at create.
  * mean_k(y, D) = a[k]*y + c[k]*D, std sigma[k] > 0 shared by target and drafter (the method needs
  * equal covariances: Section 3.3 and the appendix on unequal variances).
- * tcond: [K, tcond_dim] per-step scalars handed to the denoiser (GMM: 4 per step, see below). */
+ * tcond: [K, tcond_dim] per-step scalars handed to the denoiser (GMM: 4 per step, see below), in
+ * double: the mixture logits are differences of large terms, so their coefficients keep full precision. */
 typedef struct {
   int32_t K;
   const float* a;
   const float* c;
   const float* sigma;
-  const float* tcond;
+  const double* tcond;
   int32_t tcond_dim;
 } sds_schedule;
 
@@ -219,10 +220,10 @@ int sds_profile_read(sds_ctx* ctx, double* ms, int64_t* launches, int32_t reset)
  * device synchronisation of an allocation, or a process whose memory budget is fixed at start-up.
  * Computes out_dev[r] = D(x_dev[r], k_dev[r]) exactly as sds_denoise does for a float mixture:
  *   x_dev [rows, d] float, k_dev [rows] int32 in [0, K), means_dev [ncomp, d] float,
- *   logw_dev [ncomp] float, tcond_dev [K, 4] float (A, Bq, C, E per step, device), out_dev [rows, d].
+ *   logw_dev [ncomp] float, tcond_dev [K, 4] double (A, Bq, C, E per step, device), out_dev [rows, d].
  * All pointers are device pointers owned by the caller; work is enqueued on cuda_stream
  * (cudaStream_t, NULL = default stream) of the current device and the call does not wait for it.
- * The |mu_c|^2 table the kernel needs lives in a fixed array inside the library (16 KiB on every
+ * The |mu_c|^2 table the kernel needs lives in a fixed array inside the library (32 KiB on every
  * GPU that loads it, until the process exits), so ncomp <= SDS_STATIC_MAX_NCOMP; larger mixtures
  * return SDS_EUNSUPPORTED and do nothing. The call never calls cudaMalloc/cudaFree or any
  * allocating routine.
@@ -233,7 +234,7 @@ int sds_profile_read(sds_ctx* ctx, double* ms, int64_t* launches, int32_t reset)
  * ordering between them) race on it - order them on one stream or with events. */
 #define SDS_STATIC_MAX_NCOMP 4096
 int sds_gmm_denoise_static(const float* x_dev, const int32_t* k_dev, int64_t rows, int32_t d, int32_t ncomp,
-                           const float* means_dev, const float* logw_dev, const float* tcond_dev, int32_t K,
+                           const float* means_dev, const float* logw_dev, const double* tcond_dev, int32_t K,
                            float* out_dev, void* cuda_stream);
 
 const char* sds_strerror(int code);

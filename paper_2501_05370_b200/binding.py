@@ -122,7 +122,7 @@ def gmm_tcond_posterior_mean(abar: np.ndarray, comp_std: float) -> np.ndarray:
     abar = np.asarray(abar, dtype=np.float64)
     al = np.sqrt(abar)
     v = abar * comp_std ** 2 + 1.0 - abar
-    return np.stack([al / v, -abar / (2 * v), (1.0 - abar) / v, al * comp_std ** 2 / v], axis=1).astype(np.float32)
+    return np.stack([al / v, -abar / (2 * v), (1.0 - abar) / v, al * comp_std ** 2 / v], axis=1)
 
 
 def ula_schedule(K: int, gamma: float):
@@ -133,7 +133,7 @@ def ula_schedule(K: int, gamma: float):
 def gmm_tcond_grad_energy(K: int, comp_std: float) -> np.ndarray:
     """(A, Bq, C, E) for grad E of E = -log sum_c w_c N(x; mu_c, s^2 I): (1/s^2, -1/(2 s^2), -1/s^2, 1/s^2)."""
     s2 = comp_std ** 2
-    return np.tile(np.array([1 / s2, -0.5 / s2, -1 / s2, 1 / s2], dtype=np.float32), (K, 1))
+    return np.tile(np.array([1 / s2, -0.5 / s2, -1 / s2, 1 / s2], dtype=np.float64), (K, 1))
 
 
 # ---------------------------------------------------------------------------------------------
@@ -165,7 +165,7 @@ class Sampler:
         sch.K = self.K
         sch.a, sch.c, sch.sigma = a.ctypes.data, c.ctypes.data, sigma.ctypes.data
         if tcond is not None:
-            tcond = np.ascontiguousarray(tcond, np.float32)
+            tcond = np.ascontiguousarray(tcond, np.float64)
             sch.tcond, sch.tcond_dim = tcond.ctypes.data, tcond.shape[1]
         self._keep += [a, c, sigma, tcond]
         den = SdsDenoiser()

@@ -45,7 +45,8 @@ struct Layout {
 struct sds_ctx {
   int64_t B = 0;
   int32_t d = 0, L = 0, K = 0;
-  std::vector<float> a, c, sigma, tcond;
+  std::vector<float> a, c, sigma;
+  std::vector<double> tcond;
   int32_t tcond_dim = 0;
   sds_denoiser den{};
   Layout lay{};
@@ -84,7 +85,7 @@ void make_layout(const sds_schedule* sch, const sds_denoiser* den, int64_t B, in
   l.a = cv.take(K * 4);
   l.c = cv.take(K * 4);
   l.sigma = cv.take(K * 4);
-  l.tcond = cv.take(K * (size_t)(sch->tcond_dim > 0 ? sch->tcond_dim : 1) * 4);
+  l.tcond = cv.take(K * (size_t)(sch->tcond_dim > 0 ? sch->tcond_dim : 1) * 8);
   l.Y = cv.take(Bd * 4);
   l.Dc = cv.take(Bd * 4);
   l.T = cv.take(Bd * 4);
@@ -104,7 +105,7 @@ void make_layout(const sds_schedule* sch, const sds_denoiser* den, int64_t B, in
   l.jstar = cv.take((size_t)B * 4);
   l.nfe_calls = cv.take((size_t)B * 4);
   l.nfe_rows = cv.take((size_t)B * 4);
-  l.musq = (den->kind == SDS_DEN_GMM) ? cv.take((size_t)den->ncomp * 4) : kNone;
+  l.musq = (den->kind == SDS_DEN_GMM) ? cv.take((size_t)den->ncomp * 8) : kNone;
   l.total = cv.off;
   *out = l;
 }
@@ -157,10 +158,10 @@ WinArgs win_args(sds_ctx* c) {
 GmmArgs gmm_args(sds_ctx* c) {
   GmmArgs G{};
   G.d = c->d; G.ncomp = c->den.ncomp; G.K = c->K;
-  G.tcond = at<float>(c, c->lay.tcond);
+  G.tcond = at<double>(c, c->lay.tcond);
   G.means = static_cast<const float*>(c->den.means_dev);
   G.logw = c->den.logw_dev;
-  G.musq = at<float>(c, c->lay.musq);
+  G.musq = at<double>(c, c->lay.musq);
   return G;
 }
 
@@ -214,7 +215,7 @@ void prof_collect(sds_ctx* c) {
 int ensure_musq(sds_ctx* c) {
   if (c->musq_ready) return SDS_OK;
   SDS_LAUNCH(c, SDS_PROF_AUX, launch_musq(static_cast<const float*>(c->den.means_dev), c->den.ncomp, c->d,
-                                          at<float>(c, c->lay.musq), c->stream));
+                                          at<double>(c, c->lay.musq), c->stream));
   c->musq_ready = true;
   return SDS_OK;
 }
@@ -322,7 +323,7 @@ int sds_bind(sds_ctx* c, void* workspace_dev, size_t bytes, void* cuda_stream, u
   SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.c, c->c.data(), kb, cudaMemcpyHostToDevice, c->stream));
   SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.sigma, c->sigma.data(), kb, cudaMemcpyHostToDevice, c->stream));
   if (!c->tcond.empty())
-    SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.tcond, c->tcond.data(), c->tcond.size() * 4, cudaMemcpyHostToDevice,
+    SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.tcond, c->tcond.data(), c->tcond.size() * 8, cudaMemcpyHostToDevice,
                               c->stream));
   SDS_CU(c, cudaMemsetAsync(c->ws + c->lay.ctl, 0, kCtlWords * 4, c->stream));
   SDS_CU(c, cudaStreamSynchronize(c->stream));

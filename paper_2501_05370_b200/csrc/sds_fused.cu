@@ -15,11 +15,10 @@ namespace sds {
 namespace {
 
 // floats of shared memory: parameters (rounded to 16 bytes) and per-warp window storage
-__host__ __device__ inline int fused_param_floats(int ncomp, int d) {
-  return (ncomp * small_ldm(d) + 2 * ncomp + 3) / 4 * 4;
-}
+__host__ __device__ inline int fused_param_floats(int ncomp, int d) { return small_param_floats(ncomp, d); }
 __host__ __device__ inline int fused_warp_floats(int d, int L) {
-  return (2 * L + 2) * small_ldx(d) + 32 + 4 * kMaxL;   // W[L+1], Dq[L], Dc, e-scratch, S1/S2 as doubles
+  // S1/S2 (doubles), two converted rows (doubles), W[L+1], Dq[L], Dc, e-scratch
+  return 4 * kMaxL + 4 * small_ldd(d) + (2 * L + 2) * small_ldx(d) + 32;
 }
 
 template <int G, bool VEC4>
@@ -29,16 +28,15 @@ __global__ void k_fused_small(WinArgs A, GmmArgs P) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   const int g = lane / G, gl = lane % G;
   const int d = A.d, L = A.L, K = A.K;
-  const int ldm = small_ldm(d), ldx = small_ldx(d);
-  float* s_means = smem;
-  float* s_musq = s_means + P.ncomp * ldm;
-  float* s_logw = s_musq + P.ncomp;
-  float* sW = smem + fused_param_floats(P.ncomp, d) + (size_t)warp * fused_warp_floats(d, L);
+  const int ldx = small_ldx(d), ldd = small_ldd(d);
+  const SmallParams S = small_stage_params(P.means, P.musq, P.logw, P.ncomp, d, smem);
+  float* wbase = smem + fused_param_floats(P.ncomp, d) + (size_t)warp * fused_warp_floats(d, L);
+  double* sS = reinterpret_cast<double*>(wbase);               // [2][kMaxL]
+  double* sXd = sS + 2 * kMaxL + g * ldd;                      // converted row of this lane group
+  float* sW = wbase + 4 * kMaxL + 4 * ldd;
   float* sDq = sW + (L + 1) * ldx;
   float* sDc = sDq + L * ldx;
   float* sEs = sDc + ldx;
-  double* sS = reinterpret_cast<double*>(sEs + 32);           // [2][kMaxL]
-  small_stage_params(P.means, P.musq, P.logw, P.ncomp, d, s_means, s_musq, s_logw);
   __syncthreads();
 
   // verify lane mapping: same partition as the step-wise warp-per-chain kernel; when only the
@@ -56,8 +54,8 @@ __global__ void k_fused_small(WinArgs A, GmmArgs P) {
       for (int i = lane; i < d; i += 32) sW[i] = normal1(A.seed, kStreamInit, bg, 0u, (uint32_t)i);
     }
     __syncwarp();
-    gmm_row_small<G>(sW, g == 0, s_means, ldm, s_musq, s_logw, P.ncomp, d, __ldg(P.tcond + 0), __ldg(P.tcond + 1),
-                     __ldg(P.tcond + 2), __ldg(P.tcond + 3), sEs + g * G, sDc, gl);
+    gmm_row_small<G>(sW, sXd, g == 0, S, __ldg(P.tcond + 0), __ldg(P.tcond + 1), __ldg(P.tcond + 2),
+                     __ldg(P.tcond + 3), sEs + g * G, sDc, gl);
     int n = 0, calls = 1, rows = 1;
     bool frozen = false;
     while (n < K) {
@@ -92,9 +90,8 @@ __global__ void k_fused_small(WinArgs A, GmmArgs P) {
         const bool valid = j < Lt;
         const int jj = valid ? j : 0;
         const int k = n + jj;
-        gmm_row_small<G>(sW + jj * ldx, valid, s_means, ldm, s_musq, s_logw, P.ncomp, d, __ldg(P.tcond + 4 * k + 0),
-                         __ldg(P.tcond + 4 * k + 1), __ldg(P.tcond + 4 * k + 2), __ldg(P.tcond + 4 * k + 3),
-                         sEs + g * G, sDq + jj * ldx, gl);
+        gmm_row_small<G>(sW + jj * ldx, sXd, valid, S, __ldg(P.tcond + 4 * k + 0), __ldg(P.tcond + 4 * k + 1),
+                         __ldg(P.tcond + 4 * k + 2), __ldg(P.tcond + 4 * k + 3), sEs + g * G, sDq + jj * ldx, gl);
       }
       // S1 = |Delta|^2, S2 = Delta.Z per position
       for (int j0 = 1; j0 <= Lt; j0 += (pack2 ? 2 : 1)) {

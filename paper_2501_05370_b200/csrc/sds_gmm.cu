@@ -13,7 +13,7 @@ namespace {
 
 constexpr int kGmmWarps = 4;
 
-__global__ void k_musq(const float* __restrict__ means, int ncomp, int d, float* __restrict__ musq) {
+__global__ void k_musq(const float* __restrict__ means, int ncomp, int d, double* __restrict__ musq) {
   const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (c >= ncomp) return;
@@ -23,7 +23,7 @@ __global__ void k_musq(const float* __restrict__ means, int ncomp, int d, float*
     acc = fma(m, m, acc);
   }
   acc = warp_sum(acc);
-  if (lane == 0) musq[c] = (float)acc;
+  if (lane == 0) musq[c] = acc;
 }
 
 // smem layout: [means ncomp*d (optional)] [per-warp logits kGmmWarps*ncomp]
@@ -45,15 +45,15 @@ __global__ void __launch_bounds__(kGmmWarps * 32) k_gmm_f32(GmmArgs G, const flo
   for (int row = blockIdx.x * kGmmWarps + warp; row < nrows; row += gridDim.x * kGmmWarps) {
     const float* x = X + (size_t)row * G.d;
     const int k = rowk[row];
-    const float tA = __ldg(G.tcond + 4 * k + 0), tB = __ldg(G.tcond + 4 * k + 1);
-    const float tC = __ldg(G.tcond + 4 * k + 2), tE = __ldg(G.tcond + 4 * k + 3);
+    const double tA = __ldg(G.tcond + 4 * k + 0), tB = __ldg(G.tcond + 4 * k + 1);
+    const float tC = (float)__ldg(G.tcond + 4 * k + 2), tE = (float)__ldg(G.tcond + 4 * k + 3);
     float mx = -INFINITY;
     for (int c = 0; c < G.ncomp; ++c) {
       const float* mu = M + (size_t)c * G.d;
       float acc = 0.f;
       for (int i = lane; i < G.d; i += 32) acc = fmaf(x[i], mu[i], acc);
       acc = warp_sum(acc);
-      const float lg = fmaf(tA, acc, fmaf(tB, __ldg(G.musq + c), __ldg(G.logw + c)));
+      const float lg = (float)fma(tA, (double)acc, fma(tB, __ldg(G.musq + c), (double)__ldg(G.logw + c)));
       if (lane == 0) s_logit[c] = lg;
       mx = fmaxf(mx, lg);
     }
@@ -89,13 +89,14 @@ __global__ void __launch_bounds__(kSmallWarps * 32) k_gmm_small(GmmArgs P, const
   constexpr int RPW = 32 / G;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane / G, gl = lane % G;
   const int nrows = nrows_dev ? min(*nrows_dev, rows_host) : rows_host;
-  const int ldm = small_ldm(P.d), ldx = small_ldx(P.d);
-  float* s_means = smem;
-  float* s_musq = s_means + P.ncomp * ldm;
-  float* s_logw = s_musq + P.ncomp;
-  float* s_x = s_logw + P.ncomp + (size_t)warp * (RPW * ldx + 32);
+  const int ldx = small_ldx(P.d), ldd = small_ldd(P.d);
+  const SmallParams S = small_stage_params(P.means, P.musq, P.logw, P.ncomp, P.d, smem);
+  // per warp: [RPW converted rows (double)] [RPW rows (float)] [32 floats of e-scratch]
+  const int per_warp = RPW * (2 * ldd + ldx) + 32;
+  float* wbase = smem + small_param_floats(P.ncomp, P.d) + (size_t)warp * per_warp;
+  double* s_xd = reinterpret_cast<double*>(wbase) + g * ldd;
+  float* s_x = wbase + RPW * 2 * ldd;
   float* s_es = s_x + RPW * ldx + g * G;
-  small_stage_params(P.means, P.musq, P.logw, P.ncomp, P.d, s_means, s_musq, s_logw);
   __syncthreads();
   const int stride = gridDim.x * kSmallWarps * RPW;
   for (int row0 = (blockIdx.x * kSmallWarps + warp) * RPW; row0 < nrows; row0 += stride) {
@@ -106,25 +107,24 @@ __global__ void __launch_bounds__(kSmallWarps * 32) k_gmm_small(GmmArgs P, const
     __syncwarp();
     const int row = row0 + g;
     const bool valid = row < nrows;
-    float tA = 0.f, tB = 0.f, tC = 0.f, tE = 0.f;
+    double tA = 0., tB = 0., tC = 0., tE = 0.;
     if (valid) {
       const int k = rowk[row];
       tA = __ldg(P.tcond + 4 * k + 0); tB = __ldg(P.tcond + 4 * k + 1);
       tC = __ldg(P.tcond + 4 * k + 2); tE = __ldg(P.tcond + 4 * k + 3);
     }
-    gmm_row_small<G>(s_x + g * ldx, valid, s_means, ldm, s_musq, s_logw, P.ncomp, P.d, tA, tB, tC, tE, s_es,
-                     out + (size_t)(valid ? row : 0) * P.d, gl);
+    gmm_row_small<G>(s_x + g * ldx, s_xd, valid, S, tA, tB, tC, tE, s_es, out + (size_t)(valid ? row : 0) * P.d, gl);
   }
 }
 
 size_t small_smem_bytes(int ncomp, int d) {
   const int G = small_group(ncomp), RPW = 32 / G;
-  return ((size_t)ncomp * small_ldm(d) + 2 * (size_t)ncomp + (size_t)kSmallWarps * (RPW * small_ldx(d) + 32)) * 4;
+  return ((size_t)small_param_floats(ncomp, d) + (size_t)kSmallWarps * (RPW * (2 * small_ldd(d) + small_ldx(d)) + 32)) * 4;
 }
 
 }  // namespace
 
-cudaError_t launch_musq(const float* means, int ncomp, int d, float* musq, cudaStream_t st) {
+cudaError_t launch_musq(const float* means, int ncomp, int d, double* musq, cudaStream_t st) {
   const int warps = 4;
   k_musq<<<(ncomp + warps - 1) / warps, warps * 32, 0, st>>>(means, ncomp, d, musq);
   return cudaGetLastError();

@@ -38,10 +38,10 @@ struct WinArgs {
 
 struct GmmArgs {
   int d, ncomp, K;
-  const float* tcond;    // [K, 4] (A, Bq, C, E)
+  const double* tcond;   // [K, 4] (A, Bq, C, E)
   const float* means;    // [ncomp, d]
   const float* logw;     // [ncomp]
-  const float* musq;     // [ncomp]
+  const double* musq;    // [ncomp] |mu_c|^2
 };
 
 // streaming kernels (sds_kernels.cu). ub_chains: host upper bound on the number of active chains.
@@ -56,7 +56,7 @@ cudaError_t launch_rng_normals(uint64_t seed, int stream_id, uint64_t b0, int64_
 cudaError_t launch_rng_uniforms(uint64_t seed, uint64_t b0, int64_t nb, int k, float* out, cudaStream_t st);
 
 // mixture denoiser, float path (sds_gmm.cu)
-cudaError_t launch_musq(const float* means, int ncomp, int d, float* musq, cudaStream_t st);
+cudaError_t launch_musq(const float* means, int ncomp, int d, double* musq, cudaStream_t st);
 cudaError_t launch_gmm_f32(const GmmArgs& G, const float* X, const int* rowk, const int* nrows_dev, int rows_ub,
                            float* out, cudaStream_t st);
 

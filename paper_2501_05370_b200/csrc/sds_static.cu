@@ -16,16 +16,16 @@
 
 namespace {
 
-// scratch: |mu_c|^2 for up to SDS_STATIC_MAX_NCOMP components (16 KiB per GPU, lives until exit)
-static __device__ __align__(256) float g_musq_scratch[SDS_STATIC_MAX_NCOMP];
+// scratch: |mu_c|^2 for up to SDS_STATIC_MAX_NCOMP components (32 KiB per GPU, lives until exit)
+static __device__ __align__(256) double g_musq_scratch[SDS_STATIC_MAX_NCOMP];
 
 constexpr int kMaxDevices = 64;
 std::mutex g_mu;
-float* g_scratch_addr[kMaxDevices] = {};
+double* g_scratch_addr[kMaxDevices] = {};
 
 // Device address of the scratch array on the current device. In host code the symbol's name is
 // only a handle, so the address is looked up once per device and cached.
-int scratch_for_current_device(float** out) {
+int scratch_for_current_device(double** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SDS_ECUDA;
   std::lock_guard<std::mutex> lock(g_mu);
@@ -35,7 +35,7 @@ int scratch_for_current_device(float** out) {
       cudaGetLastError();
       return SDS_ECUDA;
     }
-    g_scratch_addr[dev] = static_cast<float*>(p);
+    g_scratch_addr[dev] = static_cast<double*>(p);
   }
   *out = g_scratch_addr[dev];
   return SDS_OK;
@@ -47,13 +47,13 @@ extern "C" {
 #pragma GCC visibility push(default)
 
 int sds_gmm_denoise_static(const float* x_dev, const int32_t* k_dev, int64_t rows, int32_t d, int32_t ncomp,
-                           const float* means_dev, const float* logw_dev, const float* tcond_dev, int32_t K,
+                           const float* means_dev, const float* logw_dev, const double* tcond_dev, int32_t K,
                            float* out_dev, void* cuda_stream) {
   if (!x_dev || !k_dev || !means_dev || !logw_dev || !tcond_dev || !out_dev) return SDS_EINVAL;
   if (rows < 0 || rows > (int64_t)1 << 30 || d <= 0 || ncomp <= 0 || K <= 0) return SDS_EINVAL;
   if (ncomp > SDS_STATIC_MAX_NCOMP) return SDS_EUNSUPPORTED;   // does not fit the built-in scratch
   if (rows == 0) return SDS_OK;
-  float* musq = nullptr;
+  double* musq = nullptr;
   const int rc = scratch_for_current_device(&musq);
   if (rc != SDS_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

@@ -38,7 +38,7 @@ def _sched(K=5, sigma0=0.1):
     a = np.full(K, 0.9, np.float32)
     c = np.full(K, 0.1, np.float32)
     s = np.full(K, sigma0, np.float32)
-    t = np.zeros((K, 4), np.float32)
+    t = np.zeros((K, 4), np.float64)
     sch = sb.SdsSchedule(K, a.ctypes.data, c.ctypes.data, s.ctypes.data, t.ctypes.data, 4)
     return sch, (a, c, s, t)
 
