@@ -22,7 +22,7 @@ __host__ __device__ inline int fused_warp_floats(int d, int L) {
 }
 
 template <int G, bool VEC4>
-__global__ void k_fused_small(WinArgs A, GmmArgs P) {
+__global__ void __maxnreg__(72) k_fused_small(WinArgs A, GmmArgs P) {
   extern __shared__ __align__(16) float smem[];
   constexpr int RPW = 32 / G;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
@@ -74,13 +74,26 @@ __global__ void k_fused_small(WinArgs A, GmmArgs P) {
         }
       }
       __syncwarp();
-      for (int i = lane; i < d; i += 32) {
-        float y = sW[i];
-        const float dc = sDc[i];
+      for (int i0 = 0; i0 < d; i0 += 128) {                     // up to four elements per lane in registers
+        float y[4], dc[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int i = i0 + lane + 32 * u;
+          y[u] = (i < d) ? sW[i] : 0.f;
+          dc[u] = (i < d) ? sDc[i] : 0.f;
+        }
         for (int j = 0; j < Lt; ++j) {
           const int k = n + j;
-          y = draft_step(y, dc, sW[(j + 1) * ldx + i], __ldg(A.a + k), __ldg(A.c + k), __ldg(A.sigma + k));
-          sW[(j + 1) * ldx + i] = y;
+          const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
+          float* row = sW + (j + 1) * ldx;
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int i = i0 + lane + 32 * u;
+            if (i < d) {
+              y[u] = draft_step(y[u], dc[u], row[i], ak, ck, sk);
+              row[i] = y[u];
+            }
+          }
         }
       }
       __syncwarp();
@@ -193,45 +206,53 @@ __global__ void k_fused_small(WinArgs A, GmmArgs P) {
   }
 }
 
-int fused_warps(int d, int ncomp, int L) {
-  for (int w = 8; w >= 2; w >>= 1) {
-    const size_t bytes = ((size_t)fused_param_floats(ncomp, d) + (size_t)w * fused_warp_floats(d, L)) * 4;
-    if (bytes <= 100 * 1024) return w;
-  }
+size_t fused_smem_bytes(int d, int ncomp, int L, int warps) {
+  return ((size_t)fused_param_floats(ncomp, d) + (size_t)warps * fused_warp_floats(d, L)) * 4;
+}
+
+// largest CTA (in warps) whose shared memory still fits; 0 if even two warps do not
+int fused_max_warps(int d, int ncomp, int L) {
+  for (int w = 16; w >= 2; w -= 2)
+    if (fused_smem_bytes(d, ncomp, L, w) <= 220 * 1024) return w;
   return 0;
+}
+
+template <int G, bool VEC4>
+cudaError_t fused_launch_t(const WinArgs& A, const GmmArgs& P, cudaStream_t st) {
+  // pick the CTA size that keeps the most warps resident per SM (one wave if the batch allows)
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  int best_w = 0, best_res = 0, best_blocks = 0;
+  for (int w = fused_max_warps(A.d, P.ncomp, A.L); w >= 2; w -= 2) {
+    const size_t smem = fused_smem_bytes(A.d, P.ncomp, A.L, w);
+    cudaError_t e = cudaFuncSetAttribute(k_fused_small<G, VEC4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    int nb = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_fused_small<G, VEC4>, w * 32, smem);
+    if (e != cudaSuccess) return e;
+    if (nb * w > best_res) { best_res = nb * w; best_w = w; best_blocks = nb; }
+  }
+  if (best_w == 0) return cudaErrorInvalidConfiguration;
+  const size_t smem = fused_smem_bytes(A.d, P.ncomp, A.L, best_w);
+  cudaError_t e = cudaFuncSetAttribute(k_fused_small<G, VEC4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  int blocks = (A.B + best_w - 1) / best_w;
+  if (blocks > best_blocks * sms) blocks = best_blocks * sms;
+  k_fused_small<G, VEC4><<<blocks, best_w * 32, smem, st>>>(A, P);
+  return cudaGetLastError();
 }
 
 }  // namespace
 
 bool fused_small_supported(int d, int ncomp, int L) {
-  return d <= 256 && ncomp <= kSmallMaxComp && L <= kMaxL && fused_warps(d, ncomp, L) > 0;
+  return d <= 256 && ncomp <= kSmallMaxComp && L <= kMaxL && fused_max_warps(d, ncomp, L) > 0;
 }
 
 cudaError_t launch_fused_small(const WinArgs& A, const GmmArgs& P, cudaStream_t st) {
-  const int w = fused_warps(A.d, P.ncomp, A.L);
-  if (w == 0) return cudaErrorInvalidConfiguration;
-  const size_t smem = ((size_t)fused_param_floats(P.ncomp, A.d) + (size_t)w * fused_warp_floats(A.d, A.L)) * 4;
-  int blocks = (A.B + w - 1) / w;
-  const int cap = 148 * 16;
-  if (blocks > cap) blocks = cap;
   const bool vec4 = (A.d % 4) == 0;
-  const int grp = small_group(P.ncomp);
-#define SDS_FUSED_LAUNCH(GG, VV)                                                                              \
-  do {                                                                                                        \
-    if (smem > 48 * 1024) {                                                                                   \
-      const cudaError_t e_ =                                                                                  \
-          cudaFuncSetAttribute(k_fused_small<GG, VV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
-      if (e_ != cudaSuccess) return e_;                                                                       \
-    }                                                                                                         \
-    k_fused_small<GG, VV><<<blocks, w * 32, smem, st>>>(A, P);                                                \
-  } while (0)
-  if (grp == 16) {
-    if (vec4) SDS_FUSED_LAUNCH(16, true); else SDS_FUSED_LAUNCH(16, false);
-  } else {
-    if (vec4) SDS_FUSED_LAUNCH(32, true); else SDS_FUSED_LAUNCH(32, false);
-  }
-#undef SDS_FUSED_LAUNCH
-  return cudaGetLastError();
+  if (small_group(P.ncomp) == 16) return vec4 ? fused_launch_t<16, true>(A, P, st) : fused_launch_t<16, false>(A, P, st);
+  return vec4 ? fused_launch_t<32, true>(A, P, st) : fused_launch_t<32, false>(A, P, st);
 }
 
 }  // namespace sds
