@@ -171,10 +171,11 @@ int sds_sample_all(sds_ctx* ctx, float* out_dev, int32_t* nfe_calls_dev, int32_t
 #define SDS_OPT_WHOLE_CHAIN_KERNEL 1
 int sds_set_option(sds_ctx* ctx, int32_t option, int64_t value);
 
-/* Same with host buffers: copies the mixture parameters means_host [ncomp, d] / logw_host [ncomp]
- * (float; NULL = keep what is on the device) to the device arrays named at create, runs
- * sds_sample_all, copies the results to host memory. All copies are on the bound stream. */
-int sds_sample_all_host(sds_ctx* ctx, const float* means_host, const float* logw_host,
+/* Same with host buffers: copies the mixture parameters means_host [ncomp, d] (float or bf16, the
+ * dtype named at create) and logw_host [ncomp] (float) to the device arrays named at create
+ * (NULL = keep what is on the device), runs sds_sample_all, copies the results to host memory.
+ * All copies are on the bound stream. */
+int sds_sample_all_host(sds_ctx* ctx, const void* means_host, const float* logw_host,
                         float* out_host, int32_t* nfe_calls_host, int32_t* nfe_rows_host);
 
 /* Copy an internal array (selector above) to dst; dst_is_host != 0 waits for the stream. */

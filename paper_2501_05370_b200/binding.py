@@ -148,7 +148,8 @@ class Sampler:
     """
 
     def __init__(self, a, c, sigma, B: int, d: int, L: int, *, gmm_means=None, gmm_logw=None, tcond=None,
-                 callback=None, seed: int = 0, chain_id_offset: int = 0, device="cuda:0", stream=None):
+                 gmm_bf16: bool = False, mlp=None, callback=None, seed: int = 0, chain_id_offset: int = 0,
+                 device="cuda:0", stream=None):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("libsds needs a CUDA device; there is no CPU path")
@@ -171,10 +172,32 @@ class Sampler:
         den = SdsDenoiser()
         if gmm_means is not None:
             means = np.ascontiguousarray(gmm_means, np.float32)
-            self.means = torch.from_numpy(means).to(self.device)
+            if gmm_bf16:
+                bits = means.view(np.uint32)
+                if np.any(bits & np.uint32(0xFFFF)):
+                    raise ValueError("gmm_bf16 needs bf16-representable means")
+                self.means = torch.from_numpy((bits >> np.uint32(16)).astype(np.uint16).view(np.int16)).to(self.device)
+            else:
+                self.means = torch.from_numpy(means).to(self.device)
             self.logw = torch.from_numpy(np.ascontiguousarray(gmm_logw, np.float32)).to(self.device)
             den.kind, den.ncomp = SDS_DEN_GMM, means.shape[0]
-            den.means_dev, den.logw_dev, den.means_dtype = self.means.data_ptr(), self.logw.data_ptr(), SDS_F32
+            den.means_dev, den.logw_dev = self.means.data_ptr(), self.logw.data_ptr()
+            den.means_dtype = SDS_BF16 if gmm_bf16 else SDS_F32
+        elif mlp is not None:
+            nl = len(mlp.weights)
+            dev_bits = lambda x: torch.from_numpy(np.ascontiguousarray(x, np.uint16).view(np.int16)).to(self.device)
+            self.mlp_W = [dev_bits(w) for w in mlp.weights]
+            self.mlp_bias = [torch.from_numpy(np.ascontiguousarray(x, np.float32)).to(self.device) for x in mlp.bias]
+            self.mlp_temb = [dev_bits(x) if x is not None else None for x in mlp.temb]
+            self._mlp_dims = np.ascontiguousarray(mlp.dims, np.int32)
+            self._mlp_Wp = (C.c_void_p * nl)(*[x.data_ptr() for x in self.mlp_W])
+            self._mlp_bp = (C.c_void_p * nl)(*[x.data_ptr() for x in self.mlp_bias])
+            self._mlp_tp = (C.c_void_p * nl)(*[(x.data_ptr() if x is not None else None) for x in self.mlp_temb])
+            den.kind, den.nlayer = SDS_DEN_MLP, nl
+            den.W_dev = C.cast(self._mlp_Wp, C.c_void_p)
+            den.bias_dev = C.cast(self._mlp_bp, C.c_void_p)
+            den.temb_dev = C.cast(self._mlp_tp, C.c_void_p)
+            den.dims = self._mlp_dims.ctypes.data
         elif callback is not None:
             self._cb = DENOISE_FN(callback)
             den.kind, den.fn = SDS_DEN_CALLBACK, self._cb

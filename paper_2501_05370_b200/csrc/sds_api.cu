@@ -2,6 +2,7 @@
 // host loop of sds_sample_all. All device work is in the kernels this file launches.
 #include "../../include/sds.h"
 
+#include <algorithm>
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
@@ -10,6 +11,7 @@
 
 #include "sds_device.cuh"
 #include "sds_internal.h"
+#include "sds_tc.h"
 
 using namespace sds;
 
@@ -37,6 +39,8 @@ struct Layout {
   size_t n, act, rowoff, rowk, ctl;
   size_t S1, S2, ell, logU, accmask, jstar, nfe_calls, nfe_rows;
   size_t musq;
+  size_t H0, H1;          // MLP hidden activations (bf16)
+  size_t logits, R, Mt;   // large mixture: logits (f32), responsibilities (bf16), transposed means (bf16)
   size_t total;
 };
 
@@ -49,6 +53,9 @@ struct sds_ctx {
   std::vector<double> tcond;
   int32_t tcond_dim = 0;
   sds_denoiser den{};
+  std::vector<int32_t> mlp_dims;                 // copies of the caller's MLP description
+  std::vector<const void*> mlp_W, mlp_temb;
+  std::vector<const float*> mlp_bias;
   Layout lay{};
   char* ws = nullptr;
   size_t ws_bytes = 0;
@@ -106,6 +113,18 @@ void make_layout(const sds_schedule* sch, const sds_denoiser* den, int64_t B, in
   l.nfe_calls = cv.take((size_t)B * 4);
   l.nfe_rows = cv.take((size_t)B * 4);
   l.musq = (den->kind == SDS_DEN_GMM) ? cv.take((size_t)den->ncomp * 8) : kNone;
+  l.H0 = l.H1 = l.logits = l.R = l.Mt = kNone;
+  if (den->kind == SDS_DEN_MLP) {
+    size_t width = 0;
+    for (int i = 1; i < den->nlayer; ++i) width = std::max(width, (size_t)den->dims[i]);
+    l.H0 = cv.take(rows * width * 2);
+    l.H1 = cv.take(rows * width * 2);
+  }
+  if (den->kind == SDS_DEN_GMM && den->means_dtype == SDS_BF16) {
+    l.logits = cv.take(rows * (size_t)den->ncomp * 4);
+    l.R = cv.take(rows * (size_t)den->ncomp * 2);
+    l.Mt = cv.take((size_t)d * den->ncomp * 2);
+  }
   l.total = cv.off;
   *out = l;
 }
@@ -123,13 +142,27 @@ int validate(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_
     case SDS_DEN_GMM:
       if (den->ncomp <= 0 || !den->means_dev || !den->logw_dev) return SDS_EINVAL;
       if (!sch->tcond || sch->tcond_dim != 4) return SDS_EINVAL;
-      if (den->means_dtype != SDS_F32) return SDS_EUNSUPPORTED;
+      if (den->means_dtype == SDS_BF16) {
+        // tensor-core path: both contractions tile by 128
+        if (den->ncomp % 128 != 0 || d % 128 != 0) return SDS_EUNSUPPORTED;
+      } else if (den->means_dtype != SDS_F32) {
+        return SDS_EUNSUPPORTED;
+      }
       break;
     case SDS_DEN_CALLBACK:
       if (!den->fn) return SDS_EINVAL;
       break;
     case SDS_DEN_MLP:
-      return SDS_EUNSUPPORTED;
+      if (den->nlayer < 1 || den->nlayer > 16 || !den->dims || !den->W_dev || !den->bias_dev || !den->temb_dev)
+        return SDS_EINVAL;
+      if (den->dims[0] != d || den->dims[den->nlayer] != d) return SDS_EINVAL;
+      for (int i = 0; i <= den->nlayer; ++i)
+        if (den->dims[i] <= 0 || den->dims[i] % 128 != 0) return SDS_EUNSUPPORTED;
+      for (int i = 0; i < den->nlayer; ++i) {
+        if (!den->W_dev[i] || !den->bias_dev[i]) return SDS_EINVAL;
+        if (i < den->nlayer - 1 && !den->temb_dev[i]) return SDS_EINVAL;
+      }
+      break;
     default:
       return SDS_EUNSUPPORTED;
   }
@@ -220,15 +253,80 @@ int ensure_musq(sds_ctx* c) {
   return SDS_OK;
 }
 
-// run the target denoiser on dense rows; the row count lives on the device (nrows_dev, may be
-// NULL) with a host upper bound for the grid
-int run_denoiser(sds_ctx* c, const float* X, const int* rowk, const int* nrows_dev, int64_t rows_ub, float* out) {
+// bf16 copy of the rows for the tensor-core denoisers (the draft kernel writes it on the hot path)
+int ensure_bf16_rows(sds_ctx* c, const float* X, const uint16_t** Xb, int64_t rows_ub) {
+  if (*Xb) return SDS_OK;
+  uint16_t* dst = at<uint16_t>(c, c->lay.Xb);
+  SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_f32_to_bf16(X, (size_t)rows_ub * c->d, dst, c->stream));
+  *Xb = dst;
+  return SDS_OK;
+}
+
+TcGemmArgs tc_args(sds_ctx* c, const int* rowk, const int* nrows_dev, int64_t rows_ub) {
+  TcGemmArgs g{};
+  g.nrows_dev = nrows_dev;
+  g.rows_host = (int)rows_ub;
+  g.rows_cap = (int)(c->B * c->L);
+  g.rowk = rowk;
+  g.err = at<int>(c, c->lay.ctl) + kCtlTcError;
+  return g;
+}
+
+// run the target denoiser on dense rows X (and their bf16 copy Xb, NULL = make one); the row count
+// lives on the device (nrows_dev, may be NULL) with a host upper bound for the grids
+int run_denoiser(sds_ctx* c, const float* X, const uint16_t* Xb, const int* rowk, const int* nrows_dev,
+                 int64_t rows_ub, float* out) {
   if (rows_ub <= 0) return SDS_OK;
   switch (c->den.kind) {
     case SDS_DEN_GMM: {
-      const int rc = ensure_musq(c);
+      if (c->den.means_dtype == SDS_F32) {
+        const int rc = ensure_musq(c);
+        if (rc != SDS_OK) return rc;
+        SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gmm_f32(gmm_args(c), X, rowk, nrows_dev, (int)rows_ub, out, c->stream));
+        return SDS_OK;
+      }
+      // large mixture on tensor cores: logits = X M^T, softmax, mix = R M, affine epilogue
+      const uint16_t* means = static_cast<const uint16_t*>(c->den.means_dev);
+      uint16_t* Mt = at<uint16_t>(c, c->lay.Mt);
+      uint16_t* R = at<uint16_t>(c, c->lay.R);
+      float* logits = at<float>(c, c->lay.logits);
+      if (!c->musq_ready) {
+        SDS_LAUNCH(c, SDS_PROF_AUX, launch_musq_bf16(means, c->den.ncomp, c->d, at<double>(c, c->lay.musq), c->stream));
+        SDS_LAUNCH(c, SDS_PROF_AUX, launch_transpose_bf16(means, c->den.ncomp, c->d, Mt, c->stream));
+        c->musq_ready = true;
+      }
+      int rc = ensure_bf16_rows(c, X, &Xb, rows_ub);
       if (rc != SDS_OK) return rc;
-      SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gmm_f32(gmm_args(c), X, rowk, nrows_dev, (int)rows_ub, out, c->stream));
+      TcGemmArgs g = tc_args(c, rowk, nrows_dev, rows_ub);
+      g.N = c->den.ncomp; g.K = c->d; g.out = logits; g.ldo = c->den.ncomp;
+      g.tcond = at<double>(c, c->lay.tcond); g.musq = at<double>(c, c->lay.musq); g.logw = c->den.logw_dev;
+      SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiGmmLogits, g, Xb, means, c->stream));
+      SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_softmax_bf16(logits, nrows_dev, (int)rows_ub, c->den.ncomp, R, c->stream));
+      TcGemmArgs m = tc_args(c, rowk, nrows_dev, rows_ub);
+      m.N = c->d; m.K = c->den.ncomp; m.out = out; m.ldo = c->d;
+      m.tcond = at<double>(c, c->lay.tcond); m.xrows = X;
+      SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiGmmMix, m, R, Mt, c->stream));
+      return SDS_OK;
+    }
+    case SDS_DEN_MLP: {
+      int rc = ensure_bf16_rows(c, X, &Xb, rows_ub);
+      if (rc != SDS_OK) return rc;
+      const void* in = Xb;
+      const int nl = (int)c->mlp_W.size();
+      for (int l = 0; l < nl; ++l) {
+        TcGemmArgs g = tc_args(c, rowk, nrows_dev, rows_ub);
+        g.N = c->mlp_dims[l + 1]; g.K = c->mlp_dims[l];
+        g.bias = c->mlp_bias[l];
+        if (l < nl - 1) {
+          uint16_t* h = at<uint16_t>(c, (l & 1) ? c->lay.H1 : c->lay.H0);
+          g.out = h; g.ldo = g.N; g.temb = static_cast<const uint16_t*>(c->mlp_temb[l]);
+          SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiMlpHidden, g, in, c->mlp_W[l], c->stream));
+          in = h;
+        } else {
+          g.out = out; g.ldo = g.N;
+          SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiBiasF32, g, in, c->mlp_W[l], c->stream));
+        }
+      }
       return SDS_OK;
     }
     case SDS_DEN_CALLBACK: {
@@ -253,6 +351,7 @@ int sync_active(sds_ctx* c, int64_t* n_active) {
   SDS_CU(c, cudaStreamSynchronize(c->stream));
   c->ub = c->h_pin[kCtlNActive];
   if (n_active) *n_active = c->ub;
+  if (c->h_pin[kCtlTcError] != 0) return SDS_ETIMEOUT;
   return (c->h_pin[kCtlError] & kErrNonFinite) ? SDS_ENONFINITE : SDS_OK;
 }
 
@@ -286,6 +385,13 @@ int sds_create(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int3
   c->tcond_dim = sch->tcond_dim > 0 ? sch->tcond_dim : 0;
   if (sch->tcond && c->tcond_dim > 0) c->tcond.assign(sch->tcond, sch->tcond + (size_t)sch->K * c->tcond_dim);
   c->den = *den;
+  if (den->kind == SDS_DEN_MLP) {
+    c->mlp_dims.assign(den->dims, den->dims + den->nlayer + 1);
+    c->mlp_W.assign(den->W_dev, den->W_dev + den->nlayer);
+    c->mlp_bias.assign(den->bias_dev, den->bias_dev + den->nlayer);
+    c->mlp_temb.assign(den->temb_dev, den->temb_dev + den->nlayer);
+    c->den.dims = c->mlp_dims.data();
+  }
   make_layout(sch, den, B, d, L, &c->lay);
   if (cudaHostAlloc((void**)&c->h_pin, 64 * sizeof(int32_t), cudaHostAllocDefault) != cudaSuccess) {
     c->last_cuda = (int)cudaGetLastError();
@@ -336,7 +442,7 @@ int sds_reset(sds_ctx* c) {
   if (c->state < kBound) return SDS_ESTATE;
   WinArgs A = win_args(c);
   SDS_LAUNCH(c, SDS_PROF_INIT, launch_init(A, c->stream));
-  const int rc = run_denoiser(c, A.X, A.rowk, A.ctl + kCtlNRows, c->B, A.Dq);
+  const int rc = run_denoiser(c, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, c->B, A.Dq);
   if (rc != SDS_OK) return rc;
   SDS_LAUNCH(c, SDS_PROF_AUX, launch_after_init(A, c->stream));
   SDS_LAUNCH(c, SDS_PROF_AUX, launch_compact(A, c->stream));
@@ -357,7 +463,7 @@ int sds_verify_window(sds_ctx* c) {
   if (!c) return SDS_EINVAL;
   if (c->state != kDrafted) return SDS_ESTATE;
   WinArgs A = win_args(c);
-  const int rc = run_denoiser(c, A.X, A.rowk, A.ctl + kCtlNRows, (int64_t)c->ub * c->L, A.Dq);
+  const int rc = run_denoiser(c, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, (int64_t)c->ub * c->L, A.Dq);
   if (rc != SDS_OK) return rc;
   SDS_LAUNCH(c, SDS_PROF_VERIFY, launch_verify(A, c->ub, c->stream));
   c->state = kVerified;
@@ -416,13 +522,14 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
   return sync_active(c, &na);
 }
 
-int sds_sample_all_host(sds_ctx* c, const float* means_host, const float* logw_host, float* out_host,
+int sds_sample_all_host(sds_ctx* c, const void* means_host, const float* logw_host, float* out_host,
                         int32_t* nfe_calls_host, int32_t* nfe_rows_host) {
   if (!c || !out_host) return SDS_EINVAL;
   if (c->state < kBound) return SDS_ESTATE;
   if ((means_host || logw_host) && c->den.kind != SDS_DEN_GMM) return SDS_EINVAL;
   if (means_host) {
-    SDS_CU(c, cudaMemcpyAsync(const_cast<void*>(c->den.means_dev), means_host, (size_t)c->den.ncomp * c->d * 4,
+    const size_t esz = c->den.means_dtype == SDS_BF16 ? 2 : 4;
+    SDS_CU(c, cudaMemcpyAsync(const_cast<void*>(c->den.means_dev), means_host, (size_t)c->den.ncomp * c->d * esz,
                               cudaMemcpyHostToDevice, c->stream));
     c->musq_ready = false;
   }
@@ -491,7 +598,7 @@ int sds_denoise(sds_ctx* c, const float* x_dev, const int32_t* k_dev, int64_t ro
   if (!c || !x_dev || !k_dev || !out_dev) return SDS_EINVAL;
   if (c->state < kBound) return SDS_ESTATE;
   if (rows < 0 || rows > c->B * c->L) return SDS_EINVAL;
-  return run_denoiser(c, x_dev, k_dev, nullptr, rows, out_dev);
+  return run_denoiser(c, x_dev, nullptr, k_dev, nullptr, rows, out_dev);
 }
 
 int sds_rng_normals(uint64_t seed, int32_t stream_id, int64_t b0, int64_t nb, int32_t k, int32_t d, float* out_dev,

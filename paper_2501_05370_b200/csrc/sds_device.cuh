@@ -22,7 +22,7 @@ enum Ctl : int {
   kCtlError = 3,      // sticky error bits
   kCtlFrozen = 4,     // chains frozen because of a non-finite log ratio
   kCtlDone = 5,       // block-completion counter of the advance kernel
-  kCtlSpare0 = 6,
+  kCtlTcError = 6,    // set by a tensor-core kernel whose bounded wait gave up
   kCtlSpare1 = 7,
   kCtlWords = 8
 };

@@ -77,6 +77,7 @@ __global__ void __launch_bounds__(kBlock) k_init(WinArgs A) {
     A.ctl[kCtlError] = 0;
     A.ctl[kCtlFrozen] = 0;
     A.ctl[kCtlDone] = 0;
+    A.ctl[kCtlTcError] = 0;
   }
   if (b >= A.B) return;
   const uint64_t bg = A.chain_off + (uint64_t)b;

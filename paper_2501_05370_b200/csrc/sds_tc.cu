@@ -1,0 +1,475 @@
+// Tensor-core GEMM of the denoisers: C[M, N] = A[M, K] * B[N, K]^T, bf16 operands (both K-major),
+// fp32 accumulation in tensor memory, fused epilogues. Written for sm_100a:
+//   - operand tiles move global -> shared with TMA (cp.async.bulk.tensor, 128-byte swizzle),
+//     completion counted on mbarriers;
+//   - one elected thread issues tcgen05.mma (M = 128, N = BN, K = 16 per instruction) with the
+//     accumulator in TMEM; tcgen05.commit releases shared stages and publishes the accumulator;
+//   - four epilogue warps read the accumulator with tcgen05.ld (each warp its 32 TMEM lanes) and
+//     apply the epilogue; two accumulator buffers let the epilogue of tile i overlap the main loop
+//     of tile i+1 (persistent CTAs, static round-robin over tiles).
+// Every wait is bounded: when a wait gives up the kernel records an error word and winds down.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
+#include "sds_device.cuh"
+#include "sds_tc.h"
+
+namespace sds {
+
+namespace {
+
+constexpr int BM = 128;            // rows per tile = TMEM lanes
+constexpr int BK = 64;             // bf16 elements per K block = one 128-byte swizzle row
+constexpr int UK = 16;             // K per tcgen05.mma of kind::f16
+constexpr int kThreads = 192;      // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..5: epilogue
+constexpr uint32_t kSpinCap = 1u << 22;
+
+template <int BN> struct TileCfg {
+  static constexpr int kStages = (BN == 256) ? 4 : 6;
+  static constexpr int kABytes = BM * BK * 2;
+  static constexpr int kBBytes = BN * BK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kTmemCols = 2 * BN;                                  // two accumulator buffers
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// bounded wait: false when the cap is reached or another role has already given up
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t it = 0; it < kSpinCap; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 1023u) == 1023u && *abort_flag) return false;
+  }
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int c0, int c1, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
+          smem_u32(dst)),
+      "l"(reinterpret_cast<uint64_t>(tm)), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+      : "memory");
+}
+
+// shared-memory matrix descriptor, K-major operand, 128-byte swizzle: rows of 128 bytes, groups of
+// eight rows 1024 bytes apart (stride byte offset), descriptor version 1
+__device__ __forceinline__ uint64_t make_sdesc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(1024u >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
+// instruction descriptor, kind::f16: D = f32, A = B = bf16, both K-major, N >> 3 at bit 17, M >> 4 at bit 24
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// one 32-column chunk of one output row
+template <int EPI>
+__device__ __forceinline__ void epilogue_chunk(const TcGemmArgs& g, const uint32_t (&acc)[32], int row, int col, int krow) {
+  float v[32];
+#pragma unroll
+  for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(acc[j]);
+  if (EPI == kEpiMlpHidden) {
+    // h = SiLU(acc + bias + E[k]) stored as bf16
+    const uint4* te = reinterpret_cast<const uint4*>(g.temb + (size_t)krow * g.N + col);
+    uint4* o = reinterpret_cast<uint4*>(static_cast<uint16_t*>(g.out) + (size_t)row * g.ldo + col);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const uint4 t = __ldg(te + q);
+      const uint32_t tw[4] = {t.x, t.y, t.z, t.w};
+      uint32_t pk[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int j = q * 8 + u * 2;
+        float a = v[j] + __ldg(g.bias + col + j) + bf16_lo(tw[u]);
+        float b = v[j + 1] + __ldg(g.bias + col + j + 1) + bf16_hi(tw[u]);
+        a = __fdividef(a, 1.0f + __expf(-a));
+        b = __fdividef(b, 1.0f + __expf(-b));
+        pk[u] = pack_bf16x2(a, b);
+      }
+      o[q] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+    }
+  } else if (EPI == kEpiBiasF32) {
+    float4* o = reinterpret_cast<float4*>(static_cast<float*>(g.out) + (size_t)row * g.ldo + col);
+#pragma unroll
+    for (int q = 0; q < 8; ++q)
+      o[q] = make_float4(v[4 * q] + __ldg(g.bias + col + 4 * q), v[4 * q + 1] + __ldg(g.bias + col + 4 * q + 1),
+                         v[4 * q + 2] + __ldg(g.bias + col + 4 * q + 2), v[4 * q + 3] + __ldg(g.bias + col + 4 * q + 3));
+  } else if (EPI == kEpiGmmLogits) {
+    // logit = logw + A * <x, mu> + Bq * |mu|^2
+    const float tA = (float)__ldg(g.tcond + 4 * krow + 0);
+    const double tB = __ldg(g.tcond + 4 * krow + 1);
+    float4* o = reinterpret_cast<float4*>(static_cast<float*>(g.out) + (size_t)row * g.ldo + col);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      float w[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int n = col + 4 * q + u;
+        w[u] = fmaf(tA, v[4 * q + u], (float)fma(tB, __ldg(g.musq + n), (double)__ldg(g.logw + n)));
+      }
+      o[q] = make_float4(w[0], w[1], w[2], w[3]);
+    }
+  } else {  // kEpiGmmMix: D = C * sum_c r_c mu_c + E * x
+    const float tC = (float)__ldg(g.tcond + 4 * krow + 2), tE = (float)__ldg(g.tcond + 4 * krow + 3);
+    const float4* xr = reinterpret_cast<const float4*>(g.xrows + (size_t)row * g.N + col);
+    float4* o = reinterpret_cast<float4*>(static_cast<float*>(g.out) + (size_t)row * g.ldo + col);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const float4 x = __ldg(xr + q);
+      o[q] = make_float4(fmaf(tC, v[4 * q], tE * x.x), fmaf(tC, v[4 * q + 1], tE * x.y),
+                         fmaf(tC, v[4 * q + 2], tE * x.z), fmaf(tC, v[4 * q + 3], tE * x.w));
+    }
+  }
+}
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(kThreads, 1)
+    k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, TcGemmArgs g) {
+  using C = TileCfg<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  // 1024-byte aligned operand stages (required by the 128-byte swizzle), barriers behind them
+  uint8_t* stages = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(stages + C::kStages * C::kStageBytes);
+  uint64_t* empty_bar = full_bar + C::kStages;
+  uint64_t* tfull_bar = empty_bar + C::kStages;      // accumulator ready     [2]
+  uint64_t* tempty_bar = tfull_bar + 2;              // accumulator drained   [2]
+  uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+  volatile int* abort_s = reinterpret_cast<volatile int*>(tmem_base_s + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int M = g.nrows_dev ? min(*g.nrows_dev, g.rows_host) : g.rows_host;
+  const int m_tiles = (M + BM - 1) / BM, n_tiles = g.N / BN;
+  const int total_tiles = m_tiles * n_tiles;
+  const int kblocks = (g.K + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::kStages; ++s) { mbar_init(full_bar + s, 1); mbar_init(empty_bar + s, 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(tfull_bar + s, 1); mbar_init(tempty_bar + s, 4); }
+    *abort_s = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_s)),
+                 "r"((uint32_t)C::kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_base_s;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        const int m0 = (t / n_tiles) * BM, n0 = (t % n_tiles) * BN;
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait(empty_bar + stage, phase ^ 1u, abort_s)) { ok = false; break; }
+          uint8_t* sa = stages + stage * C::kStageBytes;
+          mbar_expect_tx(full_bar + stage, (uint32_t)C::kStageBytes);
+          tma_load_2d(sa, &tmA, kb * BK, m0, full_bar + stage);
+          tma_load_2d(sa + C::kABytes, &tmB, kb * BK, n0, full_bar + stage);
+          if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        *abort_s = 1;
+        atomicExch(g.err, 1);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(BM, BN);
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+        const int buf = it & 1;
+        const uint32_t bphase = (uint32_t)(it >> 1) & 1u;
+        if (!mbar_wait(tempty_bar + buf, bphase ^ 1u, abort_s)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait(full_bar + stage, phase, abort_s)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(stages + stage * C::kStageBytes);
+          const uint64_t adesc = make_sdesc(sa), bdesc = make_sdesc(sa + C::kABytes);
+#pragma unroll
+          for (int k = 0; k < BK / UK; ++k) {
+            // 32 bytes further along K inside the 128-byte swizzle row: +2 in the (>>4) address field
+            umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb | k) ? 1u : 0u);
+          }
+          umma_commit(empty_bar + stage);                    // frees the stage once these MMAs have read it
+          if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) umma_commit(tfull_bar + buf);                // accumulator complete
+      }
+      if (!ok) {
+        *abort_s = 1;
+        atomicExch(g.err, 2);
+      }
+    }
+  } else {
+    // ---------------- epilogue: warp q owns TMEM lanes 32q .. 32q+31 ----------------
+    const int q = warp & 3;
+    int it = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+      const int buf = it & 1;
+      const uint32_t bphase = (uint32_t)(it >> 1) & 1u;
+      const int m0 = (t / n_tiles) * BM, n0 = (t % n_tiles) * BN;
+      if (!mbar_wait(tfull_bar + buf, bphase, abort_s)) { ok = false; break; }
+      tc_fence_after();
+      const int row = m0 + q * 32 + lane;
+      const bool live = row < M;
+      const int krow = (live && g.rowk) ? __ldg(g.rowk + row) : 0;
+      const uint32_t tbase = tmem_base + (uint32_t)(buf * BN) + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+      for (int c = 0; c < BN; c += 32) {
+        uint32_t acc[32];
+        tmem_ld32(tbase + (uint32_t)c, acc);
+        if (live) epilogue_chunk<EPI>(g, acc, row, n0 + c, krow);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar + buf);
+    }
+    if (!ok && lane == 0) {
+      *abort_s = 1;
+      atomicExch(g.err, 3);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_s && threadIdx.x == 0) {
+    // give copies that may still be in flight time to land before the CTA's shared memory is released
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::kTmemCols)
+                 : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// helpers around the GEMMs of the large mixture
+// ------------------------------------------------------------------------------------------
+
+// softmax over ncomp logits per row -> normalised responsibilities in bf16
+__global__ void __launch_bounds__(256) k_softmax_bf16(const float* __restrict__ logits, const int* __restrict__ nrows_dev,
+                                                      int rows_host, int ncomp, uint16_t* __restrict__ R) {
+  const int nrows = nrows_dev ? min(*nrows_dev, rows_host) : rows_host;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int row = blockIdx.x * 8 + warp; row < nrows; row += gridDim.x * 8) {
+    const float* lg = logits + (size_t)row * ncomp;
+    float mx = -INFINITY;
+    for (int c = lane; c < ncomp; c += 32) mx = fmaxf(mx, lg[c]);
+    mx = warp_max(mx);
+    float den = 0.f;
+    for (int c = lane; c < ncomp; c += 32) den += expf(lg[c] - mx);
+    den = warp_sum(den);
+    const float inv = 1.0f / den;
+    for (int c = lane * 2; c < ncomp; c += 64) {
+      const float a = expf(lg[c] - mx) * inv, b = expf(lg[c + 1] - mx) * inv;
+      *reinterpret_cast<uint32_t*>(R + (size_t)row * ncomp + c) = pack_bf16x2(a, b);
+    }
+  }
+}
+
+// Mt[i, c] = M[c, i] (bf16), so that the mixing product is again a K-major x K-major GEMM
+__global__ void k_transpose_bf16(const uint16_t* __restrict__ Min, int ncomp, int d, uint16_t* __restrict__ Mt) {
+  __shared__ uint16_t tile[32][33];
+  const int c0 = blockIdx.y * 32, i0 = blockIdx.x * 32;
+  for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+    const int c = c0 + r, i = i0 + threadIdx.x;
+    tile[r][threadIdx.x] = (c < ncomp && i < d) ? Min[(size_t)c * d + i] : (uint16_t)0;
+  }
+  __syncthreads();
+  for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+    const int i = i0 + r, c = c0 + threadIdx.x;
+    if (i < d && c < ncomp) Mt[(size_t)i * ncomp + c] = tile[threadIdx.x][r];
+  }
+}
+
+__global__ void k_musq_bf16(const uint16_t* __restrict__ means, int ncomp, int d, double* __restrict__ musq) {
+  const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (c >= ncomp) return;
+  double acc = 0.0;
+  for (int i = lane; i < d; i += 32) {
+    const double m = (double)__uint_as_float((uint32_t)means[(size_t)c * d + i] << 16);
+    acc = fma(m, m, acc);
+  }
+  acc = warp_sum(acc);
+  if (lane == 0) musq[c] = acc;
+}
+
+__global__ void k_f32_to_bf16(const float* __restrict__ x, size_t n, uint16_t* __restrict__ out) {
+  for (size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 2; i < n; i += (size_t)gridDim.x * blockDim.x * 2) {
+    if (i + 1 < n) *reinterpret_cast<uint32_t*>(out + i) = pack_bf16x2(x[i], x[i + 1]);
+    else out[i] = (uint16_t)(pack_bf16x2(x[i], 0.f) & 0xffffu);
+  }
+}
+
+PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
+  static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(p);
+  }
+  return fn;
+}
+
+// [rows, K] bf16 row-major, box = [box_rows, 64] with the 128-byte swizzle; out-of-range reads give zeros
+bool make_tmap(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t K, uint32_t box_rows) {
+  PFN_cuTensorMapEncodeTiled_v12000 fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {K, rows};
+  const cuuint64_t strides[1] = {K * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN, int EPI>
+cudaError_t launch_t(const TcGemmArgs& g, const void* A, const void* B, int grid_tiles_ub, cudaStream_t st) {
+  using C = TileCfg<BN>;
+  CUtensorMap tmA, tmB;
+  if (!make_tmap(&tmA, A, (uint64_t)g.rows_cap, (uint64_t)g.K, BM)) return cudaErrorInvalidValue;
+  if (!make_tmap(&tmB, B, (uint64_t)g.N, (uint64_t)g.K, BN)) return cudaErrorInvalidValue;
+  cudaError_t e = cudaFuncSetAttribute(k_gemm_tc<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+  if (e != cudaSuccess) return e;
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  int grid = grid_tiles_ub < sms ? grid_tiles_ub : sms;
+  if (grid < 1) grid = 1;
+  k_gemm_tc<BN, EPI><<<grid, kThreads, C::kSmemBytes, st>>>(tmA, tmB, g);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool tc_shape_ok(int N, int K) { return N % 128 == 0 && K % 8 == 0 && K >= 8; }
+
+cudaError_t launch_gemm_tc(int epi, const TcGemmArgs& g, const void* A_bf16, const void* B_bf16, cudaStream_t st) {
+  if (!tc_shape_ok(g.N, g.K) || g.rows_cap <= 0 || g.rows_host > g.rows_cap) return cudaErrorInvalidValue;
+  if (g.rows_host <= 0) return cudaSuccess;
+  const bool wide = (g.N % 256) == 0;
+  const int m_tiles = (g.rows_host + BM - 1) / BM;
+  const int tiles = m_tiles * (g.N / (wide ? 256 : 128));
+#define SDS_TC_CASE(E)                                                                     \
+  case E:                                                                                  \
+    return wide ? launch_t<256, E>(g, A_bf16, B_bf16, tiles, st) : launch_t<128, E>(g, A_bf16, B_bf16, tiles, st);
+  switch (epi) {
+    SDS_TC_CASE(kEpiMlpHidden)
+    SDS_TC_CASE(kEpiBiasF32)
+    SDS_TC_CASE(kEpiGmmLogits)
+    SDS_TC_CASE(kEpiGmmMix)
+    default:
+      return cudaErrorInvalidValue;
+  }
+#undef SDS_TC_CASE
+}
+
+cudaError_t launch_softmax_bf16(const float* logits, const int* nrows_dev, int rows_host, int ncomp, uint16_t* R,
+                                cudaStream_t st) {
+  int blocks = (rows_host + 7) / 8;
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  if (blocks < 1) blocks = 1;
+  k_softmax_bf16<<<blocks, 256, 0, st>>>(logits, nrows_dev, rows_host, ncomp, R);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_transpose_bf16(const uint16_t* M, int ncomp, int d, uint16_t* Mt, cudaStream_t st) {
+  dim3 grid((d + 31) / 32, (ncomp + 31) / 32), block(32, 8);
+  k_transpose_bf16<<<grid, block, 0, st>>>(M, ncomp, d, Mt);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_musq_bf16(const uint16_t* means, int ncomp, int d, double* musq, cudaStream_t st) {
+  k_musq_bf16<<<(ncomp + 3) / 4, 128, 0, st>>>(means, ncomp, d, musq);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_f32_to_bf16(const float* x, size_t n, uint16_t* out, cudaStream_t st) {
+  size_t blocks = (n / 2 + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  k_f32_to_bf16<<<(int)blocks, 256, 0, st>>>(x, n, out);
+  return cudaGetLastError();
+}
+
+}  // namespace sds

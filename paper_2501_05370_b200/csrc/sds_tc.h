@@ -1,0 +1,42 @@
+// Tensor-core GEMM launcher and the helper kernels of the bf16 denoisers (sds_tc.cu).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace sds {
+
+enum TcEpilogue : int {
+  kEpiMlpHidden = 0,   // out(bf16) = SiLU(acc + bias[n] + temb[k_row][n])
+  kEpiBiasF32 = 1,     // out(f32)  = acc + bias[n]
+  kEpiGmmLogits = 2,   // out(f32)  = logw[n] + A_k * acc + Bq_k * musq[n]
+  kEpiGmmMix = 3,      // out(f32)  = C_k * acc + E_k * xrows[m][n]
+};
+
+// C[M, N] = A[M, K] * B[N, K]^T with M = min(*nrows_dev, rows_host) (or rows_host if nrows_dev is NULL).
+struct TcGemmArgs {
+  const int* nrows_dev;
+  int rows_host;         // row count (upper bound when nrows_dev is given)
+  int rows_cap;          // rows of the A buffer (tensor-map extent)
+  int N, K;
+  void* out;             // [M, ldo] bf16 or f32 depending on the epilogue
+  int ldo;
+  const int* rowk;       // [M] transition index per row
+  const float* bias;     // [N]
+  const uint16_t* temb;  // [Ksteps, N] bf16
+  const double* tcond;   // [Ksteps, 4]
+  const double* musq;    // [N]
+  const float* logw;     // [N]
+  const float* xrows;    // [M, N] f32
+  int* err;              // device word, set non-zero if a bounded wait gave up
+};
+
+bool tc_shape_ok(int N, int K);
+cudaError_t launch_gemm_tc(int epi, const TcGemmArgs& g, const void* A_bf16, const void* B_bf16, cudaStream_t st);
+cudaError_t launch_softmax_bf16(const float* logits, const int* nrows_dev, int rows_host, int ncomp, uint16_t* R,
+                                cudaStream_t st);
+cudaError_t launch_transpose_bf16(const uint16_t* M, int ncomp, int d, uint16_t* Mt, cudaStream_t st);
+cudaError_t launch_musq_bf16(const uint16_t* means, int ncomp, int d, double* musq, cudaStream_t st);
+cudaError_t launch_f32_to_bf16(const float* x, size_t n, uint16_t* out, cudaStream_t st);
+
+}  // namespace sds

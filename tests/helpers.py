@@ -6,7 +6,7 @@ import numpy as np
 from oracle import sds_oracle as o
 
 
-def oracle_setup(w, gmm=None):
+def oracle_setup(w, gmm=None, mlp=None):
     """(denoise(x, k), a, c, sigma) in double for workload w, all from the oracle's own formulas."""
     if w.sampler == "ddpm":
         a, c, sig, abar = o.ddpm_affine(w.beta())
@@ -21,7 +21,11 @@ def oracle_setup(w, gmm=None):
         else:
             den = lambda x, k: o.gmm_grad_energy(x, gp.means, gp.logw, gp.comp_std)
     else:
-        raise NotImplementedError
+        import workloads as wl
+        mp = mlp if mlp is not None else w.mlp_params()
+        W = [wl.bf16_bits_to_f32(x).astype(np.float64) for x in mp.weights]
+        T = [wl.bf16_bits_to_f32(x).astype(np.float64) if x is not None else None for x in mp.temb]
+        den = lambda x, k: o.mlp_forward(x, k, W, mp.bias, T)
     return den, a, c, sig
 
 
