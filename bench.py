@@ -50,29 +50,50 @@ def peaks():
 
 def oracle_closure(w):
     from oracle import sds_oracle as o
-    gp = w.gmm_params()
     if w.sampler == "ddpm":
         a, c, sig, abar = o.ddpm_affine(w.beta())
-        den = lambda x, k: o.gmm_posterior_mean(x, abar[k], gp.means, gp.logw, gp.comp_std, bf16_operands=gp.means_bf16)
     else:
         a, c, sig = o.ula_affine(w.K, w.ula_gamma)
-        den = lambda x, k: o.gmm_grad_energy(x, gp.means, gp.logw, gp.comp_std)
+    if w.denoiser == "mlp":
+        mp = w.mlp_params()
+        W = [wl.bf16_bits_to_f32(x).astype(np.float64) for x in mp.weights]
+        T = [wl.bf16_bits_to_f32(x).astype(np.float64) if x is not None else None for x in mp.temb]
+        den = lambda x, k: o.mlp_forward(x, k, W, mp.bias, T)
+    else:
+        gp = w.gmm_params()
+        if w.sampler == "ddpm":
+            den = lambda x, k: o.gmm_posterior_mean(x, abar[k], gp.means, gp.logw, gp.comp_std,
+                                                    bf16_operands=gp.means_bf16)
+        else:
+            den = lambda x, k: o.gmm_grad_energy(x, gp.means, gp.logw, gp.comp_std)
     return o, den, a, c, sig
 
 
-def oracle_time(w, budget_s: float, min_chains: int = 2, first_chain: int = 0):
-    """Runs oracle chains one after another for about budget_s seconds. Returns (chains, seconds)."""
+def oracle_time(w, budget_s: float, min_chains: int = 1, first_chain: int = 0):
+    """Runs oracle chains one after another for about budget_s seconds of CPU work.
+
+    Heavy workloads cannot finish even one chain in the budget, so a chain is run over the first
+    Kp transitions only (Kp starts small and grows while chains stay cheap); the sample is then a
+    prefix of the chain, which the returned description says. Returns (chain_steps, seconds, text)."""
     o, den, a, c, sig = oracle_closure(w)
     t0 = time.perf_counter()
-    n = 0
+    n, steps, Kp = 0, 0, min(w.K, 2 * w.L)
+    prefix = False
     while True:
-        o.speculative_chain(den, a, c, sig, w.L, w.sample_seed, first_chain + n, w.d)
+        t1 = time.perf_counter()
+        o.speculative_chain(den, a[:Kp], c[:Kp], sig[:Kp], w.L, w.sample_seed, first_chain + n, w.d)
+        dt = time.perf_counter() - t1
         n += 1
+        steps += Kp
+        prefix |= Kp < w.K
         el = time.perf_counter() - t0
-        if n >= min_chains and el >= budget_s:
-            return n, el
-        if n >= w.B:
-            return n, el
+        if (n >= min_chains and el >= budget_s) or n >= w.B:
+            break
+        if Kp < w.K and dt < budget_s / 8:
+            Kp = min(w.K, Kp * 4)
+    what = (f"{n} chains of {w.name}, {steps} chain-steps" + (" (chains cut to their first transitions)" if prefix else "")
+            + f" in {el:.1f} s, one NumPy thread")
+    return steps, el, what
 
 
 def run_reference(args, w):
@@ -82,14 +103,14 @@ def run_reference(args, w):
         return
     per_step_budget = max(1.0, min(8.0, 60.0 / max(1, args.steps + args.warmup)))
     for _ in range(args.warmup):
-        oracle_time(w, per_step_budget, min_chains=1)
-    tot_chains, tot_s = 0, 0.0
+        oracle_time(w, per_step_budget / 2)
+    tot_steps, tot_s, what = 0, 0.0, ""
     for i in range(args.steps):
-        n, s = oracle_time(w, per_step_budget, min_chains=1, first_chain=i * 16)
-        tot_chains += n
+        n, s, what = oracle_time(w, per_step_budget, first_chain=i * 16)
+        tot_steps += n
         tot_s += s
-    value = tot_chains * w.K / tot_s
-    sample = f"{tot_chains} chains of {w.name} (K={w.K}, L={w.L}, d={w.d}) over {args.steps} steps, one NumPy thread"
+    value = tot_steps / tot_s
+    sample = f"{args.steps} steps, each: {what}"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot_s / max(1, args.steps),
@@ -133,6 +154,13 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
+    def mark(self):
+        """Samples taken before this call are ignored by stop()."""
+        try:
+            self.skip = sum(1 for _ in open(self.path))
+        except Exception:
+            self.skip = 0
+
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
@@ -144,7 +172,9 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         try:
-            for ln in open(self.path):
+            for i, ln in enumerate(open(self.path)):
+                if i < getattr(self, "skip", 0):
+                    continue
                 f = [x.strip() for x in ln.split(",")]
                 if len(f) < 9:
                     continue
@@ -178,10 +208,13 @@ def algorithmic(kind: str, w, rows_per_step: float, windows_chains: float, launc
         return "hbm", (8.0 * d * windows_chains + 4.0 * d * rows_per_step) / launches
     if kind == "advance":
         return "hbm", 16.0 * d * windows_chains / launches
-    if kind == "denoise":       # logits + mixing contractions
-        return "alu", 4.0 * w.gmm["ncomp"] * d * (rows_per_step + w.B) / launches
-    if kind == "fused":         # whole chain in one launch: mixture contractions dominate the arithmetic
-        return "alu", 4.0 * w.gmm["ncomp"] * d * (rows_per_step + w.B) / launches
+    if kind in ("denoise", "fused"):
+        if w.denoiser == "mlp":     # 2 * sum of layer products per row, bf16 tensor cores
+            per_row = 2.0 * sum(w.mlp_dims[i] * w.mlp_dims[i + 1] for i in range(len(w.mlp_dims) - 1))
+            return "tensor", per_row * (rows_per_step + w.B) / launches
+        per_row = 4.0 * w.gmm["ncomp"] * d      # logits + mixing contractions
+        bound = "tensor" if w.gmm.get("means_bf16") else "alu"
+        return bound, per_row * (rows_per_step + w.B) / launches
     return "hbm", 0.0
 
 
@@ -211,9 +244,15 @@ def run_gpu(args, w):
     calls = torch.empty((B,), dtype=torch.int32, device=dev)
     rows = torch.empty((B,), dtype=torch.int32, device=dev)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    gp = w.gmm_params()
-    means_h = torch.from_numpy(gp.means).pin_memory()
-    logw_h = torch.from_numpy(gp.logw).pin_memory()
+    if w.denoiser == "gmm":
+        gp = w.gmm_params()
+        if gp.means_bf16:
+            means_h = torch.from_numpy((gp.means.view(np.uint32) >> np.uint32(16)).astype(np.uint16).view(np.int16)).pin_memory()
+        else:
+            means_h = torch.from_numpy(gp.means).pin_memory()
+        logw_h = torch.from_numpy(gp.logw).pin_memory()
+    else:
+        means_h = logw_h = None      # network weights stay resident on the device
     out_h = torch.empty((B, d), dtype=torch.float32).pin_memory()
     calls_h = torch.empty((B,), dtype=torch.int32).pin_memory()
     rows_h = torch.empty((B,), dtype=torch.int32).pin_memory()
@@ -234,12 +273,15 @@ def run_gpu(args, w):
     dev_step = lambda: s.sample_all(out, calls, rows)
     e2e_step = lambda: s.sample_all_host(means_h, logw_h, out_h, calls_h, rows_h)
 
-    for _ in range(args.warmup):
-        dev_step()
     clocks = ClockSampler(local)
-    barrier()
     if rank == 0:
         clocks.start()
+        time.sleep(0.5)                 # let the sampler come up before any timed work
+    for _ in range(args.warmup):
+        dev_step()
+    barrier()
+    if rank == 0:
+        clocks.mark()
     l0 = s.launch_count()
     s.profile(True)
     s.profile_read(reset=True)
@@ -277,32 +319,35 @@ def run_gpu(args, w):
     kinds = {k: v for k, v in prof.items() if v[1] > 0}
     dom = max(kinds, key=lambda k: kinds[k][0]) if kinds else "fused"
     dom_ms, dom_n = kinds.get(dom, (ms_total, steps))
+    denoise_launch_groups = {"mlp": len(w.mlp_dims) - 1}.get(w.denoiser, 3 if (w.denoiser == "gmm" and w.gmm.get("means_bf16")) else 1)
     bound, per_launch = algorithmic(dom, w, rows_per_step, windows_chains, dom_n / steps)
     avg_s = dom_ms / max(dom_n, 1) * 1e-3
     if bound == "hbm":
         achieved, peak, unit = per_launch / avg_s / 1e9, pk["hbm_gbs"], "GB/s"
+    elif bound == "tensor":
+        achieved, peak, unit = per_launch / avg_s / 1e12, pk["bf16_sustained"], "TFLOP/s"
     else:
         peak = SMS * FP32_LANES_PER_SM * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
         achieved, unit = per_launch / avg_s / 1e12, "TFLOP/s"
     roofline = {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
                 "frac": achieved / peak, "traffic": None,
-                "peak_source": pk["source"] if bound == "hbm" else "derived: 148 SMs x 128 fp32 lanes x 2 x max SM clock",
+                "peak_source": (pk["source"] + (" (sustained bf16 GEMM)" if bound == "tensor" else " (copy)")) if bound != "alu"
+                else "derived: 148 SMs x 128 fp32 lanes x 2 x max SM clock",
                 "avg_launch_us": avg_s * 1e6, "launches_per_step": dom_n / steps,
                 "share_of_kernel_time": dom_ms / max(sum(v[0] for v in kinds.values()), 1e-9),
                 "kernel_ms_per_step": {k: v[0] / steps for k, v in kinds.items()}}
 
-    nchain, sec = oracle_time(w, args.cpu_seconds)
-    cpu = {"value": nchain * K / sec, "unit": UNIT, "cores": 1, "kind": "oracle",
-           "sample": f"{nchain} chains of {w.name} run to completion in {sec:.1f} s, one NumPy thread"}
+    osteps, sec, what = oracle_time(w, args.cpu_seconds)
+    cpu = {"value": osteps / sec, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic", "config": workload_config(w, args),
+        "dtype": ("bf16" if w.dtype == "bf16" else "f32"), "data": "synthetic", "config": workload_config(w, args),
         "nfe": {"K": K, "mean_target_calls": float(calls_np.mean()), "mean_target_rows": float(rows_np.mean()),
                 "mean_advance": float(K * B / max(windows_chains, 1)), "calls_saved_frac": float(1 - calls_np.mean() / K)},
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e / steps,
-                "h2d_bytes_per_step": int(means_h.numel() * 4 + logw_h.numel() * 4),
+                "h2d_bytes_per_step": int(means_h.numel() * means_h.element_size() + logw_h.numel() * 4) if means_h is not None else 0,
                 "d2h_bytes_per_step": int(out_h.numel() * 4 + calls_h.numel() * 4 + rows_h.numel() * 4)},
         "gpu_launches": int(launches),
         "roofline": roofline, "cpu_baseline": cpu, "clocks": clk,
