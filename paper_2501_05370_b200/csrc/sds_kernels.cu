@@ -301,6 +301,143 @@ __global__ void __launch_bounds__(kBlock) k_verify(WinArgs A) {
   }
 }
 
+// Register-resident variant for d % 4 == 0 and d <= 4 * EPT * TPC: each thread keeps its slice of
+// the carried output and of the previous drafted state in registers, so every position reads only
+// its own drafted state and target output from memory (8d bytes per verified step), with 2*EPT
+// independent 128-bit loads in flight per thread. Same per-thread element order and reduction
+// tree as k_verify, hence the same bits.
+template <int TPC, int EPT>
+__global__ void __launch_bounds__(TPC > kBlock ? TPC : kBlock) k_verify_reg(WinArgs A) {
+  constexpr int kThreadsPerCta = TPC > kBlock ? TPC : kBlock;
+  constexpr int kChains = kThreadsPerCta / TPC;
+  constexpr int kWarps = TPC / 32;
+  __shared__ double s_red[(TPC > 32) ? 2 * kMaxL * kWarps : 1];
+  __shared__ int s_jstar;
+  __shared__ float s_coef;
+  const int s = blockIdx.x * kChains + threadIdx.x / TPC, t = threadIdx.x % TPC;
+  const int lane = threadIdx.x & 31, warp = t >> 5;
+  if (s >= A.ctl[kCtlNActive]) return;
+  const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
+  const int Lt = window_len(A, nb);
+  const uint64_t bg = A.chain_off + (uint64_t)b;
+  const size_t cb = (size_t)b * A.d;
+  const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+
+  float4 vc[EPT], vp[EPT];
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) {
+    const int i = (t + e * TPC) * 4;
+    vc[e] = (i < A.d) ? ld4(A.Dc + cb + i) : zero4;
+    vp[e] = (i < A.d) ? ld4(A.X + (size_t)r0 * A.d + i) : zero4;
+  }
+  double myS1 = 0.0, myS2 = 0.0;
+  for (int j = 1; j <= Lt; ++j) {
+    const int k = nb + j - 1;
+    const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
+    const float inv_s = 1.0f / sk, cs = ck * inv_s;
+    const float* wj = (j < Lt) ? A.X + (size_t)(r0 + j) * A.d : A.T + cb;
+    const float* dq = A.Dq + (size_t)(r0 + j - 1) * A.d;
+    float4 vj[EPT], vq[EPT];
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) {
+      const int i = (t + e * TPC) * 4;
+      vj[e] = (i < A.d) ? ld4(wj + i) : zero4;
+      vq[e] = (i < A.d) ? ld4(dq + i) : zero4;
+    }
+    double p1 = 0.0, p2 = 0.0;
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) {
+      if ((t + e * TPC) * 4 < A.d) {
+        float D, Z;
+        delta_z(vp[e].x, vj[e].x, vq[e].x, vc[e].x, ak, ck, cs, inv_s, D, Z);
+        p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+        delta_z(vp[e].y, vj[e].y, vq[e].y, vc[e].y, ak, ck, cs, inv_s, D, Z);
+        p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+        delta_z(vp[e].z, vj[e].z, vq[e].z, vc[e].z, ak, ck, cs, inv_s, D, Z);
+        p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+        delta_z(vp[e].w, vj[e].w, vq[e].w, vc[e].w, ak, ck, cs, inv_s, D, Z);
+        p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+      }
+      vp[e] = vj[e];
+    }
+    p1 = warp_sum(p1);
+    p2 = warp_sum(p2);
+    if (TPC == 32) {
+      if (lane == j - 1) { myS1 = p1; myS2 = p2; }
+    } else if (lane == 0) {
+      s_red[(j - 1) * kWarps + warp] = p1;
+      s_red[kMaxL * kWarps + (j - 1) * kWarps + warp] = p2;
+    }
+  }
+  if (TPC > 32) {
+    __syncthreads();
+    if (warp == 0 && lane < Lt) {
+      for (int w = 0; w < kWarps; ++w) {
+        myS1 += s_red[lane * kWarps + w];
+        myS2 += s_red[kMaxL * kWarps + lane * kWarps + w];
+      }
+    }
+  }
+  int jstar = 0;
+  float coef = 0.f;
+  if (warp == 0) {
+    const bool valid = lane < Lt;
+    bool acc = true, bad = false;
+    if (valid) {
+      const float U = uniform01(A.seed, bg, (uint32_t)(nb + lane));
+      const float lu = logf(U);
+      const float ellf = (float)(-0.5 * myS1 - myS2);
+      acc = (myS1 < 1e-30) || (lu <= ellf);
+      bad = !isfinite(ellf);
+      const size_t o = (size_t)b * A.L + lane;
+      A.S1[o] = myS1;
+      A.S2[o] = myS2;
+      A.ell[o] = ellf;
+      A.logU[o] = lu;
+    }
+    const uint32_t vmask = (Lt >= 32) ? 0xffffffffu : ((1u << Lt) - 1u);
+    const uint32_t amask = __ballot_sync(0xffffffffu, acc) & vmask;
+    const uint32_t bmask = __ballot_sync(0xffffffffu, bad) & vmask;
+    const uint32_t rej = ~amask & vmask;
+    jstar = rej ? __ffs(rej) : Lt + 1;
+    if (bmask) jstar = -1;
+    const int src = (jstar >= 1 && jstar <= Lt) ? jstar - 1 : 0;
+    coef = __shfl_sync(0xffffffffu, (float)(2.0 * myS2 / myS1), src);
+    if (lane == 0) {
+      A.accmask[b] = amask;
+      A.jstar[b] = jstar;
+      if (bmask) atomicOr(A.ctl + kCtlError, kErrNonFinite);
+      if (TPC > 32) { s_jstar = jstar; s_coef = coef; }
+    }
+  }
+  if (TPC > 32) {
+    __syncthreads();
+    jstar = s_jstar;
+    coef = s_coef;
+  }
+  if (jstar < 1 || jstar > Lt) return;
+  const int k = nb + jstar - 1;
+  const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
+  const float inv_s = 1.0f / sk, cs = ck * inv_s;
+  const float* wp = A.X + (size_t)(r0 + jstar - 1) * A.d;
+  float* wj = (jstar < Lt) ? A.X + (size_t)(r0 + jstar) * A.d : A.T + cb;
+  const float* dq = A.Dq + (size_t)(r0 + jstar - 1) * A.d;
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) {
+    const int i = (t + e * TPC) * 4;
+    if (i < A.d) {
+      const float4 p = ld4(wp + i), w = ld4(wj + i), q = ld4(dq + i), c4 = vc[e];
+      float4 o;
+      float D, Z;
+      delta_z(p.x, w.x, q.x, c4.x, ak, ck, cs, inv_s, D, Z); o.x = reflect_elem(p.x, q.x, Z, D, ak, ck, sk, coef);
+      delta_z(p.y, w.y, q.y, c4.y, ak, ck, cs, inv_s, D, Z); o.y = reflect_elem(p.y, q.y, Z, D, ak, ck, sk, coef);
+      delta_z(p.z, w.z, q.z, c4.z, ak, ck, cs, inv_s, D, Z); o.z = reflect_elem(p.z, q.z, Z, D, ak, ck, sk, coef);
+      delta_z(p.w, w.w, q.w, c4.w, ak, ck, cs, inv_s, D, Z); o.w = reflect_elem(p.w, q.w, Z, D, ak, ck, sk, coef);
+      st4(wj + i, o);
+    }
+  }
+}
+
 // ---------------------------------------------------------------------------------------
 // C1 advance: Y <- W_adv, carried output <- target row adv, n += adv, counters; the CTA that
 // finishes last rebuilds the active list
@@ -413,6 +550,18 @@ cudaError_t launch_draft(const WinArgs& A, int ub, cudaStream_t st) {
   return cudaGetLastError();
 }
 cudaError_t launch_verify(const WinArgs& A, int ub, cudaStream_t st) {
+  const int chains = ub > 0 ? ub : 1;
+  if (vec4_ok(A.d)) {
+    if (A.d <= 256) {
+      k_verify_reg<32, 2><<<blocks_for(chains, 32), kBlock, 0, st>>>(A);
+      return cudaGetLastError();
+    }
+    if (A.d <= 1024) { k_verify_reg<256, 1><<<chains, 256, 0, st>>>(A); return cudaGetLastError(); }
+    if (A.d <= 2048) { k_verify_reg<256, 2><<<chains, 256, 0, st>>>(A); return cudaGetLastError(); }
+    if (A.d <= 4096) { k_verify_reg<512, 2><<<chains, 512, 0, st>>>(A); return cudaGetLastError(); }
+    if (A.d <= 8192) { k_verify_reg<1024, 2><<<chains, 1024, 0, st>>>(A); return cudaGetLastError(); }
+    if (A.d <= 16384) { k_verify_reg<1024, 4><<<chains, 1024, 0, st>>>(A); return cudaGetLastError(); }
+  }
   SDS_DISPATCH(k_verify, A, ub, st);
   return cudaGetLastError();
 }
