@@ -117,6 +117,192 @@ __global__ void __launch_bounds__(kSmallWarps * 32) k_gmm_small(GmmArgs P, const
   }
 }
 
+// ---------------------------------------------------------------------------------------
+// Mid-size mixtures (33..256 components, d % 4 == 0): register-tiled float kernel. One CTA takes
+// 64 rows through both contractions without leaving the SM:
+//   1. logits[64, ncomp] = X[64, d] M^T, 4 rows x 16 components per thread, operands staged
+//      k-major in shared memory (one 128-bit load per 4 values);
+//   2. affine + row softmax in shared memory (weights kept transposed: [component][row]);
+//   3. out[64, d] = R[64, ncomp] M, tiles of 128 columns, 4 rows x 8 columns per thread,
+//      epilogue C * acc / den + E * x.
+// The mixture is re-read from L2 by every CTA (2 * ncomp * d * 4 bytes per 64 rows).
+// ---------------------------------------------------------------------------------------
+constexpr int kTR = 64;            // rows per CTA
+constexpr int kTK = 16;            // k-chunk
+constexpr int kTNC = 256;          // components held per CTA
+constexpr int kXS = kTR + 4;       // padded row counts (floats) of the k-major stages
+constexpr int kMS = kTNC + 4;
+constexpr int kRS = kTR + 4;       // stride of the transposed weight table
+constexpr int kM2S = 128 + 4;
+
+__global__ void __launch_bounds__(256, 2) k_gmm_tiled(GmmArgs P, const float* __restrict__ X,
+                                                      const int* __restrict__ rowk, const int* __restrict__ nrows_dev,
+                                                      int rows_host, float* __restrict__ out) {
+  extern __shared__ __align__(16) float sm[];
+  float* sRt = sm;                          // [kTNC][kRS]   logits, then exp weights
+  float* sA = sRt + kTNC * kRS;             // phase 1: Xs [kTK][kXS];  phase 3: Ms2 [kTK][kM2S]
+  float* sB = sA + kTK * kM2S;              // phase 1: Ms [kTK][kMS]
+  float* sInv = sB + kTK * kMS;             // [kTR] 1 / softmax denominator
+  const int nrows = nrows_dev ? min(*nrows_dev, rows_host) : rows_host;
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int d = P.d, nc = P.ncomp;
+  for (int row0 = blockIdx.x * kTR; row0 < nrows; row0 += gridDim.x * kTR) {
+    // ---- phase 1: logits ----
+    float acc[4][16];
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int c = 0; c < 16; ++c) acc[r][c] = 0.f;
+    const int xr = tid >> 2, xq = tid & 3;                 // X loader: row, float4 within the chunk
+    for (int k0 = 0; k0 < d; k0 += kTK) {
+      float4 xv = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (row0 + xr < nrows && k0 + 4 * xq < d) xv = ld4(X + (size_t)(row0 + xr) * d + k0 + 4 * xq);
+      float4 mv[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        mv[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (tid < nc && k0 + 4 * q < d) mv[q] = ld4(P.means + (size_t)tid * d + k0 + 4 * q);
+      }
+      __syncthreads();                                      // previous chunk fully consumed
+      sA[(4 * xq + 0) * kXS + xr] = xv.x; sA[(4 * xq + 1) * kXS + xr] = xv.y;
+      sA[(4 * xq + 2) * kXS + xr] = xv.z; sA[(4 * xq + 3) * kXS + xr] = xv.w;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        sB[(4 * q + 0) * kMS + tid] = mv[q].x; sB[(4 * q + 1) * kMS + tid] = mv[q].y;
+        sB[(4 * q + 2) * kMS + tid] = mv[q].z; sB[(4 * q + 3) * kMS + tid] = mv[q].w;
+      }
+      __syncthreads();
+#pragma unroll
+      for (int kk = 0; kk < kTK; ++kk) {
+        const float4 a = ld4(sA + kk * kXS + 4 * ty);
+        const float av[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          const float4 bq = ld4(sB + kk * kMS + 64 * v + 4 * tx);
+          const float bv[4] = {bq.x, bq.y, bq.z, bq.w};
+#pragma unroll
+          for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int u = 0; u < 4; ++u) acc[r][4 * v + u] = fmaf(av[r], bv[u], acc[r][4 * v + u]);
+        }
+      }
+    }
+    // ---- phase 2: affine, softmax ----
+    {
+      double tA[4], tB[4];
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int row = row0 + 4 * ty + r;
+        const int k = (row < nrows) ? rowk[row] : 0;
+        tA[r] = __ldg(P.tcond + 4 * k + 0);
+        tB[r] = __ldg(P.tcond + 4 * k + 1);
+      }
+#pragma unroll
+      for (int v = 0; v < 4; ++v)
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int c = 64 * v + 4 * tx + u;
+          float4 lg = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+          if (c < nc) {
+            const double mq = __ldg(P.musq + c), lw = (double)__ldg(P.logw + c);
+            lg.x = (float)fma(tA[0], (double)acc[0][4 * v + u], fma(tB[0], mq, lw));
+            lg.y = (float)fma(tA[1], (double)acc[1][4 * v + u], fma(tB[1], mq, lw));
+            lg.z = (float)fma(tA[2], (double)acc[2][4 * v + u], fma(tB[2], mq, lw));
+            lg.w = (float)fma(tA[3], (double)acc[3][4 * v + u], fma(tB[3], mq, lw));
+          }
+          st4(sRt + c * kRS + 4 * ty, lg);
+        }
+    }
+    __syncthreads();
+    {
+      const int row = tid >> 2, part = tid & 3;            // four threads per row
+      float mx = -INFINITY;
+      for (int c = part; c < nc; c += 4) mx = fmaxf(mx, sRt[c * kRS + row]);
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      float den = 0.f;
+      for (int c = part; c < nc; c += 4) {
+        const float e = expf(sRt[c * kRS + row] - mx);
+        sRt[c * kRS + row] = e;
+        den += e;
+      }
+      den += __shfl_xor_sync(0xffffffffu, den, 1);
+      den += __shfl_xor_sync(0xffffffffu, den, 2);
+      if (part == 0) sInv[row] = 1.0f / den;
+    }
+    __syncthreads();
+    // ---- phase 3: mixing ----
+    float tC[4], tE[4], inv[4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const int row = row0 + 4 * ty + r;
+      const int k = (row < nrows) ? rowk[row] : 0;
+      tC[r] = (float)__ldg(P.tcond + 4 * k + 2);
+      tE[r] = (float)__ldg(P.tcond + 4 * k + 3);
+      inv[r] = sInv[4 * ty + r];
+    }
+    for (int col0 = 0; col0 < d; col0 += 128) {
+      float o[4][8];
+#pragma unroll
+      for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int c = 0; c < 8; ++c) o[r][c] = 0.f;
+      for (int c0 = 0; c0 < nc; c0 += kTK) {
+        // stage M[c0 .. c0+15][col0 .. col0+127]: 512 float4, two per thread
+        float4 m2[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int f = tid + 256 * h, cc = f >> 5, cq = f & 31;
+          m2[h] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (c0 + cc < nc && col0 + 4 * cq < d) m2[h] = ld4(P.means + (size_t)(c0 + cc) * d + col0 + 4 * cq);
+        }
+        __syncthreads();
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int f = tid + 256 * h, cc = f >> 5, cq = f & 31;
+          st4(sA + cc * kM2S + 4 * cq, m2[h]);
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < kTK; ++kk) {
+          if (c0 + kk < nc) {
+            const float4 a = ld4(sRt + (c0 + kk) * kRS + 4 * ty);
+            const float av[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+            for (int v = 0; v < 2; ++v) {
+              const float4 bq = ld4(sA + kk * kM2S + 64 * v + 4 * tx);
+              const float bv[4] = {bq.x, bq.y, bq.z, bq.w};
+#pragma unroll
+              for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int u = 0; u < 4; ++u) o[r][4 * v + u] = fmaf(av[r], bv[u], o[r][4 * v + u]);
+            }
+          }
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int row = row0 + 4 * ty + r;
+        if (row >= nrows) continue;
+        const float sc = tC[r] * inv[r];
+#pragma unroll
+        for (int v = 0; v < 2; ++v) {
+          const int col = col0 + 64 * v + 4 * tx;
+          if (col < d) {
+            const float4 xx = ld4(X + (size_t)row * d + col);
+            st4(out + (size_t)row * d + col,
+                make_float4(fmaf(sc, o[r][4 * v + 0], tE[r] * xx.x), fmaf(sc, o[r][4 * v + 1], tE[r] * xx.y),
+                            fmaf(sc, o[r][4 * v + 2], tE[r] * xx.z), fmaf(sc, o[r][4 * v + 3], tE[r] * xx.w)));
+          }
+        }
+      }
+    }
+    __syncthreads();                                        // sRt / sInv are reused by the next row tile
+  }
+}
+
+constexpr size_t kTiledSmem = (size_t)(kTNC * kRS + kTK * kM2S + kTK * kMS + kTR) * 4;
+
 size_t small_smem_bytes(int ncomp, int d) {
   const int G = small_group(ncomp), RPW = 32 / G;
   return ((size_t)small_param_floats(ncomp, d) + (size_t)kSmallWarps * (RPW * (2 * small_ldd(d) + small_ldx(d)) + 32)) * 4;
@@ -151,6 +337,16 @@ cudaError_t launch_gmm_f32(const GmmArgs& G, const float* X, const int* rowk, co
       }
       k_gmm_small<32><<<blocks, kSmallWarps * 32, smem, st>>>(G, X, rowk, nrows_dev, rows_ub, out);
     }
+    return cudaGetLastError();
+  }
+  if (G.ncomp <= kTNC && (G.d % 4) == 0) {
+    const cudaError_t e =
+        cudaFuncSetAttribute(k_gmm_tiled, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTiledSmem);
+    if (e != cudaSuccess) return e;
+    int blocks = (rows_ub + kTR - 1) / kTR;
+    if (blocks > 148 * 2 * 8) blocks = 148 * 2 * 8;
+    if (blocks < 1) blocks = 1;
+    k_gmm_tiled<<<blocks, 256, kTiledSmem, st>>>(G, X, rowk, nrows_dev, rows_ub, out);
     return cudaGetLastError();
   }
   const size_t means_bytes = (size_t)G.ncomp * G.d * sizeof(float);

@@ -38,7 +38,8 @@ def test_rng_normals_and_uniforms(b0, k, d):
 # ------------------------------------------------------------------ denoiser ------------
 
 @pytest.mark.parametrize("name,d,ncomp,rows", [("cfg1", 2, 4, 37), ("cfg2", 64, 16, 515), ("cfg2", 33, 5, 70),
-                                              ("cfg5", 96, 40, 130), ("cfg5", 1024, 24, 21)])
+                                              ("cfg5", 96, 40, 130), ("cfg5", 1024, 24, 21), ("cfg5", 1024, 256, 150),
+                                              ("cfg2", 200, 100, 131), ("cfg5", 260, 33, 64)])
 def test_gmm_denoiser_rows(name, d, ncomp, rows):
     torch = _torch()
     w = wl.WORKLOADS[name].scaled(d=d, B=max(rows, 1), L=1)
