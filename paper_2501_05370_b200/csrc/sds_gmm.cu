@@ -215,14 +215,50 @@ __global__ void __launch_bounds__(256, 2) k_gmm_tiled(GmmArgs P, const float* __
     }
     __syncthreads();
     {
-      const int row = tid >> 2, part = tid & 3;            // four threads per row
+      // Four threads per row. The float logits above carry an absolute error that grows with
+      // |x||mu|; components within 30 of the row maximum are therefore recomputed in double (their
+      // dot product split over the four threads, fixed combination order) and stored relative to
+      // the maximum; all others have weight < e^-29 and keep their float value.
+      const int row = tid >> 2, part = tid & 3;
+      const int grow = row0 + row;
+      const bool live = grow < nrows;
+      const unsigned gmask = 0xFu << ((tid & 31) & ~3);
       float mx = -INFINITY;
       for (int c = part; c < nc; c += 4) mx = fmaxf(mx, sRt[c * kRS + row]);
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      double rA = 0.0, rB = 0.0;
+      if (live) {
+        const int k = rowk[grow];
+        rA = __ldg(P.tcond + 4 * k + 0);
+        rB = __ldg(P.tcond + 4 * k + 1);
+      }
+      const int seg = ((d + 3) / 4 + 3) / 4 * 4;            // elements per thread, multiple of 4
+      const int i0 = part * seg, i1 = min(d, i0 + seg);
+      const float* xrow = X + (size_t)(live ? grow : 0) * d;
+      for (int c = 0; c < nc; ++c) {
+        const float lg = sRt[c * kRS + row];
+        float val = lg - mx;
+        if (live && lg >= mx - 30.0f) {                      // uniform over the four threads of the row
+          const float* mu = P.means + (size_t)c * d;
+          double a0 = 0.0;
+          for (int i = i0; i < i1; ++i) a0 = fma((double)xrow[i], (double)mu[i], a0);
+          a0 += __shfl_xor_sync(gmask, a0, 1);
+          a0 += __shfl_xor_sync(gmask, a0, 2);
+          const double exact = fma(rA, a0, fma(rB, __ldg(P.musq + c), (double)__ldg(P.logw + c)));
+          val = (float)(exact - (double)mx);
+        }
+        __syncwarp();
+        if (part == 0) sRt[c * kRS + row] = val;
+      }
+      __syncwarp();
+      float m2 = -INFINITY;
+      for (int c = part; c < nc; c += 4) m2 = fmaxf(m2, sRt[c * kRS + row]);
+      m2 = fmaxf(m2, __shfl_xor_sync(0xffffffffu, m2, 1));
+      m2 = fmaxf(m2, __shfl_xor_sync(0xffffffffu, m2, 2));
       float den = 0.f;
       for (int c = part; c < nc; c += 4) {
-        const float e = expf(sRt[c * kRS + row] - mx);
+        const float e = expf(sRt[c * kRS + row] - m2);
         sRt[c * kRS + row] = e;
         den += e;
       }
