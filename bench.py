@@ -238,7 +238,8 @@ def run_gpu(args, w):
             dist.barrier()
         torch.cuda.synchronize()
 
-    s = sds.sampler_for(w, chain_id_offset=rank * w.B, device=dev)
+    from paper_2501_05370_b200 import sharding
+    s = sds.sampler_for(w, chain_id_offset=sharding.weak_offset(rank, w.B), device=dev)
     B, d, K = w.B, w.d, w.K
     out = torch.empty((B, d), dtype=torch.float32, device=dev)
     calls = torch.empty((B,), dtype=torch.int32, device=dev)
@@ -300,10 +301,7 @@ def run_gpu(args, w):
     ms_e2e = timed(e2e_step, args.steps)
     barrier()
 
-    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_total, ms_e2e = sharding.max_over_ranks([ms_total, ms_e2e], dist if world > 1 else None, dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()

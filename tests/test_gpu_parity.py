@@ -61,7 +61,7 @@ def test_gmm_denoiser_rows(name, d, ncomp, rows):
 
 # ------------------------------------------------------------------ one window, forced ---
 
-def _window_check(s, w, den, a32, c32, s32, seed, chain_off, stats):
+def _window_check(s, w, den, a32, c32, s32, seed, chain_off, stats, chains=None):
     """Runs draft + verify on the GPU and replays the verification on the GPU's own arrays."""
     B, L, d, K = s.B, s.L, s.d, s.K
     ctl = s.get(sb.GET_CTL)
@@ -79,6 +79,8 @@ def _window_check(s, w, den, a32, c32, s32, seed, chain_off, stats):
     accmask, jstar = s.get(sb.GET_ACCMASK), s.get(sb.GET_JSTAR)
     a64, c64, s64 = a32.astype(np.float64), c32.astype(np.float64), s32.astype(np.float64)
     for si, b in enumerate(act):
+        if chains is not None and int(b) not in chains:
+            continue
         nb = int(n[b]); Lt = min(L, K - nb); r0 = int(rowoff[si])
         assert np.array_equal(rowk[r0:r0 + Lt], nb + np.arange(Lt))
         W = np.concatenate([X[r0:r0 + Lt], T[b:b + 1]]).astype(np.float64)
@@ -126,6 +128,8 @@ def _window_check(s, w, den, a32, c32, s32, seed, chain_off, stats):
     na2 = s.advance()
     n2, Y2, Dc2 = s.get(sb.GET_N), s.get(sb.GET_Y), s.get(sb.GET_DC)
     for si, b in enumerate(act):
+        if chains is not None and int(b) not in chains:
+            continue
         nb = int(n_before[b]); Lt = min(L, K - nb); r0 = int(rowoff[si])
         adv = min(int(jstar[b]), Lt)
         assert n2[b] == nb + adv
@@ -172,6 +176,31 @@ def test_window_forced_parity(name, B, d, L, K, ncomp, windows):
         na = _window_check(s, w, den, a32, c32, s32, seed, off, stats)
     assert stats["band"] <= max(2, 2e-3 * stats["tests"])
     s.close()
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg5"])
+def test_full_size_windows_on_sampled_chains(name):
+    """The window kernels at the benchmark's full sizes and launch shapes; the oracle replays a
+    sample of chains (every position of their windows)."""
+    w = wl.WORKLOADS[name]
+    gp = w.gmm_params()
+    s = sds.sampler_for(w, gmm=gp)
+    den, a, c, sig = oracle_setup(w, gmm=gp)
+    a32, c32, s32, _ = sds.schedule_for(w)
+    rng = np.random.default_rng(5)
+    chains = set(int(x) for x in rng.choice(w.B, size=6, replace=False)) | {0, w.B - 1}
+    s.reset()
+    stats = dict(tests=0, band=0, reflected=0)
+    for _ in range(2):
+        _window_check(s, w, den, a32, c32, s32, w.sample_seed, 0, stats, chains=chains)
+    assert stats["tests"] >= 8 * w.L and stats["band"] <= 2
+    s.close()
+
+
+def test_full_size_cfg5_free_run_sampled():
+    w = wl.WORKLOADS["cfg5"]
+    out, calls, rows = _free_run_compare(w, w.gmm_params(), [3, 8191], w.sample_seed)
+    assert np.all(calls <= 1 + w.K) and calls.mean() < 0.2 * w.K
 
 
 # ------------------------------------------------------------------ free running ---------

@@ -54,7 +54,7 @@ def test_large_mixture_denoiser_rows(d, ncomp, rows):
     s.close()
 
 
-def _forced_window(s, w, den, seed, off, windows):
+def _forced_window(s, w, den, seed, off, windows, chains=None):
     """Decisions and log ratios of the verify step replayed by the oracle on the GPU's own arrays
     (the denoiser outputs are the GPU's; their parity is checked separately at 2e-2)."""
     import math
@@ -77,6 +77,8 @@ def _forced_window(s, w, den, seed, off, windows):
         ell, logU, accmask, jstar = s.get(sb.GET_ELL), s.get(sb.GET_LOGU), s.get(sb.GET_ACCMASK), s.get(sb.GET_JSTAR)
         X2, T2 = s.get(sb.GET_X), s.get(sb.GET_TAIL)
         for si, b in enumerate(act):
+            if chains is not None and int(b) not in chains:
+                continue
             nb = int(n[b]); Lt = min(L, K - nb); r0 = int(rowoff[si])
             W = np.concatenate([X[r0:r0 + Lt], T[b:b + 1]]).astype(np.float64)
             for j in (1, Lt):
@@ -126,4 +128,27 @@ def test_large_mixture_window_forced_and_free_run():
     # trajectories are compared in law, not bit by bit): mean number of target calls
     oc = [o.speculative_chain(den, a, c, sig, w.L, 41, b, w.d)["nfe_calls"] for b in range(12)]
     assert abs(np.mean(oc) - calls.mean()) <= 4 * (np.std(oc) / np.sqrt(12) + calls.std() / np.sqrt(40)) + 1.0
+    s.close()
+
+
+@pytest.mark.parametrize("name", ["cfg3", "cfg4"])
+def test_full_size_tensor_core_windows_on_sampled_chains(name):
+    """Full benchmark sizes and launch shapes (thousands of GEMM tiles, ragged row counts after the
+    first window); the oracle replays a sample of chains. Then the whole run: every chain ends at
+    n = K with finite state and consistent counters."""
+    w = wl.WORKLOADS[name]
+    if name == "cfg3":
+        mp_ = w.mlp_params()
+        s = sds.sampler_for(w, mlp=mp_)
+        den, a, c, sig = oracle_setup(w, mlp=mp_)
+    else:
+        gp = w.gmm_params()
+        s = sds.sampler_for(w, gmm=gp)
+        den, a, c, sig = oracle_setup(w, gmm=gp)
+    chains = {0, 1, w.B // 2 + 1, w.B - 1}
+    _forced_window(s, w, den, w.sample_seed, 0, 2, chains=chains)
+    out, calls, rows = [x.cpu().numpy() for x in s.sample_all()]
+    assert np.all(np.isfinite(out)) and np.array_equal(s.get(sb.GET_N), np.full(w.B, w.K))
+    assert np.all(calls >= 1 + -(-w.K // w.L)) and np.all(calls <= 1 + w.K)
+    assert np.all(rows >= w.K + 1) and np.all(rows <= 1 + (calls - 1) * w.L)
     s.close()
