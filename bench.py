@@ -364,10 +364,13 @@ def main():
     ap.add_argument("--impl", default="sds", choices=["sds", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="budget of the cpu_baseline leg")
+    ap.add_argument("--chains", type=int, default=0, help="chains per GPU (default: the workload's own B)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "sds":
         args.warmup = 3
     w = wl.WORKLOADS[args.workload]
+    if args.chains > 0:
+        w = w.scaled(B=args.chains)
     if args.impl == "reference":
         run_reference(args, w)
     else:
