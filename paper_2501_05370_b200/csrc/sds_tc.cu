@@ -4,9 +4,10 @@
 //     completion counted on mbarriers;
 //   - one elected thread issues tcgen05.mma (M = 128, N = BN, K = 16 per instruction) with the
 //     accumulator in TMEM; tcgen05.commit releases shared stages and publishes the accumulator;
-//   - four epilogue warps read the accumulator with tcgen05.ld (each warp its 32 TMEM lanes) and
-//     apply the epilogue; two accumulator buffers let the epilogue of tile i overlap the main loop
-//     of tile i+1 (persistent CTAs, static round-robin over tiles).
+//   - eight epilogue warps read the accumulator with tcgen05.ld (a warp reaches the 32 TMEM lanes
+//     of its quarter; two warps per quarter split the columns) and apply the epilogue; two
+//     accumulator buffers let the epilogue of tile i overlap the main loop of tile i+1
+//     (persistent CTAs, static round-robin over tiles).
 // Every wait is bounded: when a wait gives up the kernel records an error word and winds down.
 #include <cuda.h>
 #include <cudaTypedefs.h>
@@ -21,7 +22,8 @@ namespace {
 constexpr int BM = 128;            // rows per tile = TMEM lanes
 constexpr int BK = 64;             // bf16 elements per K block = one 128-byte swizzle row
 constexpr int UK = 16;             // K per tcgen05.mma of kind::f16
-constexpr int kThreads = 192;      // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..5: epilogue
+constexpr int kEpiWarps = 8;       // two warps per TMEM lane quarter, each takes half of the tile's columns
+constexpr int kThreads = 64 + 32 * kEpiWarps;   // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..9: epilogue
 constexpr uint32_t kSpinCap = 1u << 22;
 
 template <int BN> struct TileCfg {
@@ -121,7 +123,8 @@ __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w 
 
 // one 32-column chunk of one output row
 template <int EPI>
-__device__ __forceinline__ void epilogue_chunk(const TcGemmArgs& g, const uint32_t (&acc)[32], int row, int col, int krow) {
+__device__ __forceinline__ void epilogue_chunk(const TcGemmArgs& g, const uint32_t (&acc)[32], int row, int col, int krow,
+                                               const float4 (&xpre)[8]) {
   float v[32];
 #pragma unroll
   for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(acc[j]);
@@ -168,11 +171,10 @@ __device__ __forceinline__ void epilogue_chunk(const TcGemmArgs& g, const uint32
     }
   } else {  // kEpiGmmMix: D = C * sum_c r_c mu_c + E * x
     const float tC = (float)__ldg(g.tcond + 4 * krow + 2), tE = (float)__ldg(g.tcond + 4 * krow + 3);
-    const float4* xr = reinterpret_cast<const float4*>(g.xrows + (size_t)row * g.N + col);
     float4* o = reinterpret_cast<float4*>(static_cast<float*>(g.out) + (size_t)row * g.ldo + col);
 #pragma unroll
     for (int q = 0; q < 8; ++q) {
-      const float4 x = __ldg(xr + q);
+      const float4 x = xpre[q];
       o[q] = make_float4(fmaf(tC, v[4 * q], tE * x.x), fmaf(tC, v[4 * q + 1], tE * x.y),
                          fmaf(tC, v[4 * q + 2], tE * x.z), fmaf(tC, v[4 * q + 3], tE * x.w));
     }
@@ -201,7 +203,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::kStages; ++s) { mbar_init(full_bar + s, 1); mbar_init(empty_bar + s, 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(tfull_bar + s, 1); mbar_init(tempty_bar + s, 4); }
+    for (int s = 0; s < 2; ++s) { mbar_init(tfull_bar + s, 1); mbar_init(tempty_bar + s, kEpiWarps); }
     *abort_s = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -273,25 +275,43 @@ __global__ void __launch_bounds__(kThreads, 1)
       }
     }
   } else {
-    // ---------------- epilogue: warp q owns TMEM lanes 32q .. 32q+31 ----------------
-    const int q = warp & 3;
+    // ---------------- epilogue: warps with (warp & 3) == q reach TMEM lanes 32q .. 32q+31 ----------------
+    const int q = warp & 3, half = (warp - 2) >> 2;
+    constexpr int kCols = BN / 2;                      // columns per epilogue warp
     int it = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
       const int buf = it & 1;
       const uint32_t bphase = (uint32_t)(it >> 1) & 1u;
-      const int m0 = (t / n_tiles) * BM, n0 = (t % n_tiles) * BN;
-      if (!mbar_wait(tfull_bar + buf, bphase, abort_s)) { ok = false; break; }
-      tc_fence_after();
+      const int m0 = (t / n_tiles) * BM, n0 = (t % n_tiles) * BN + half * kCols;
       const int row = m0 + q * 32 + lane;
       const bool live = row < M;
       const int krow = (live && g.rowk) ? __ldg(g.rowk + row) : 0;
-      const uint32_t tbase = tmem_base + (uint32_t)(buf * BN) + ((uint32_t)(q * 32) << 16);
+      // the mixing epilogue adds E * x: its rows are fetched one 32-column chunk ahead
+      float4 xnext[8];
+      if (EPI == kEpiGmmMix && live) {
+        const float4* xr = reinterpret_cast<const float4*>(g.xrows + (size_t)row * g.N + n0);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) xnext[u] = __ldg(xr + u);
+      }
+      if (!mbar_wait(tfull_bar + buf, bphase, abort_s)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t tbase = tmem_base + (uint32_t)(buf * BN + half * kCols) + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
-      for (int c = 0; c < BN; c += 32) {
+      for (int c = 0; c < kCols; c += 32) {
+        float4 xcur[8];
+        if (EPI == kEpiGmmMix) {
+#pragma unroll
+          for (int u = 0; u < 8; ++u) xcur[u] = xnext[u];
+          if (live && c + 32 < kCols) {
+            const float4* xr = reinterpret_cast<const float4*>(g.xrows + (size_t)row * g.N + n0 + c + 32);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) xnext[u] = __ldg(xr + u);
+          }
+        }
         uint32_t acc[32];
         tmem_ld32(tbase + (uint32_t)c, acc);
-        if (live) epilogue_chunk<EPI>(g, acc, row, n0 + c, krow);
+        if (live) epilogue_chunk<EPI>(g, acc, row, n0 + c, krow, xcur);
       }
       tc_fence_before();
       __syncwarp();
