@@ -458,9 +458,19 @@ __global__ void __launch_bounds__(kBlock) k_advance(WinArgs A) {
       const float* src = (adv < Lt) ? A.X + (size_t)(r0 + adv) * A.d : A.T + cb;
       const float* dsrc = A.Dq + (size_t)(r0 + adv - 1) * A.d;
       if (VEC == 4) {
-        for (int i = t * 4; i < A.d; i += TPC * 4) {
-          st4(A.Y + cb + i, ld4(src + i));
-          st4(A.Dc + cb + i, ld4(dsrc + i));
+        // four iterations' loads are issued before their stores (eight 128-bit loads in flight)
+        for (int i0 = t * 4; i0 < A.d; i0 += TPC * 16) {
+          float4 vy[4], vd[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int i = i0 + u * TPC * 4;
+            if (i < A.d) { vy[u] = ld4(src + i); vd[u] = ld4(dsrc + i); }
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int i = i0 + u * TPC * 4;
+            if (i < A.d) { st4(A.Y + cb + i, vy[u]); st4(A.Dc + cb + i, vd[u]); }
+          }
         }
       } else {
         for (int i = t; i < A.d; i += TPC) {
