@@ -32,7 +32,8 @@ template <int BN> struct TileCfg {
   static constexpr int kBBytes = BN * BK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kTmemCols = 2 * BN;                                  // two accumulator buffers
-  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+  static constexpr int kEpiStageBytes = kEpiWarps * 32 * 33 * 4;            // one padded 32x32 float tile per epilogue warp
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/ + kEpiStageBytes;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -123,8 +124,7 @@ __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w 
 
 // one 32-column chunk of one output row
 template <int EPI>
-__device__ __forceinline__ void epilogue_chunk(const TcGemmArgs& g, const uint32_t (&acc)[32], int row, int col, int krow,
-                                               const float4 (&xpre)[8]) {
+__device__ __forceinline__ void epilogue_chunk(const TcGemmArgs& g, const uint32_t (&acc)[32], int row, int col, int krow) {
   float v[32];
 #pragma unroll
   for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(acc[j]);
@@ -148,12 +148,6 @@ __device__ __forceinline__ void epilogue_chunk(const TcGemmArgs& g, const uint32
       }
       o[q] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
     }
-  } else if (EPI == kEpiBiasF32) {
-    float4* o = reinterpret_cast<float4*>(static_cast<float*>(g.out) + (size_t)row * g.ldo + col);
-#pragma unroll
-    for (int q = 0; q < 8; ++q)
-      o[q] = make_float4(v[4 * q] + __ldg(g.bias + col + 4 * q), v[4 * q + 1] + __ldg(g.bias + col + 4 * q + 1),
-                         v[4 * q + 2] + __ldg(g.bias + col + 4 * q + 2), v[4 * q + 3] + __ldg(g.bias + col + 4 * q + 3));
   } else if (EPI == kEpiGmmLogits) {
     // logit = logw + A * <x, mu> + Bq * |mu|^2
     const float tA = (float)__ldg(g.tcond + 4 * krow + 0);
@@ -169,16 +163,8 @@ __device__ __forceinline__ void epilogue_chunk(const TcGemmArgs& g, const uint32
       }
       o[q] = make_float4(w[0], w[1], w[2], w[3]);
     }
-  } else {  // kEpiGmmMix: D = C * sum_c r_c mu_c + E * x
-    const float tC = (float)__ldg(g.tcond + 4 * krow + 2), tE = (float)__ldg(g.tcond + 4 * krow + 3);
-    float4* o = reinterpret_cast<float4*>(static_cast<float*>(g.out) + (size_t)row * g.ldo + col);
-#pragma unroll
-    for (int q = 0; q < 8; ++q) {
-      const float4 x = xpre[q];
-      o[q] = make_float4(fmaf(tC, v[4 * q], tE * x.x), fmaf(tC, v[4 * q + 1], tE * x.y),
-                         fmaf(tC, v[4 * q + 2], tE * x.z), fmaf(tC, v[4 * q + 3], tE * x.w));
-    }
   }
+  // the float-output epilogues (acc + bias; C * acc + E * x) are written in the kernel body
 }
 
 template <int BN, int EPI>
@@ -194,6 +180,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   uint64_t* tempty_bar = tfull_bar + 2;              // accumulator drained   [2]
   uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(tempty_bar + 2);
   volatile int* abort_s = reinterpret_cast<volatile int*>(tmem_base_s + 1);
+  float* epi_stage = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(full_bar) + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int M = g.nrows_dev ? min(*g.nrows_dev, g.rows_host) : g.rows_host;
@@ -287,35 +274,83 @@ __global__ void __launch_bounds__(kThreads, 1)
       const int row = m0 + q * 32 + lane;
       const bool live = row < M;
       const int krow = (live && g.rowk) ? __ldg(g.rowk + row) : 0;
-      // the mixing epilogue adds E * x: its rows are fetched one 32-column chunk ahead
-      float4 xnext[8];
-      if (EPI == kEpiGmmMix && live) {
-        const float4* xr = reinterpret_cast<const float4*>(g.xrows + (size_t)row * g.N + n0);
-#pragma unroll
-        for (int u = 0; u < 8; ++u) xnext[u] = __ldg(xr + u);
-      }
-      if (!mbar_wait(tfull_bar + buf, bphase, abort_s)) { ok = false; break; }
-      tc_fence_after();
       const uint32_t tbase = tmem_base + (uint32_t)(buf * BN + half * kCols) + ((uint32_t)(q * 32) << 16);
-#pragma unroll 1
-      for (int c = 0; c < kCols; c += 32) {
-        float4 xcur[8];
+      if (EPI == kEpiGmmMix || EPI == kEpiBiasF32) {
+        // Float outputs. In TMEM a thread owns a row, so direct 128-bit accesses of a warp would
+        // touch 32 different lines each and saturate the L1 tag stage. The 32x32 chunk is turned
+        // through shared memory instead: eight lanes cover the 32 columns of a row, a warp access
+        // covers four rows of 128 contiguous bytes. All eight x loads of a chunk are in flight
+        // before the accumulator chunk is read.
+        float* stg = epi_stage + (warp - 2) * (32 * 33);
+        float rowC = 0.f, rowE = 0.f;
         if (EPI == kEpiGmmMix) {
-#pragma unroll
-          for (int u = 0; u < 8; ++u) xcur[u] = xnext[u];
-          if (live && c + 32 < kCols) {
-            const float4* xr = reinterpret_cast<const float4*>(g.xrows + (size_t)row * g.N + n0 + c + 32);
-#pragma unroll
-            for (int u = 0; u < 8; ++u) xnext[u] = __ldg(xr + u);
-          }
+          rowC = (float)__ldg(g.tcond + 4 * krow + 2);
+          rowE = (float)__ldg(g.tcond + 4 * krow + 3);
         }
-        uint32_t acc[32];
-        tmem_ld32(tbase + (uint32_t)c, acc);
-        if (live) epilogue_chunk<EPI>(g, acc, row, n0 + c, krow, xcur);
+        const int rbase = m0 + q * 32;
+        const int nlive = min(32, M - rbase);                 // rows of this warp inside the matrix
+        const int rr4 = lane >> 3, c4 = (lane & 7) * 4;
+        bool waited = false;
+#pragma unroll 1
+        for (int c = 0; c < kCols; c += 32) {
+          const int col = n0 + c + c4;
+          float4 xv[8];
+          if (EPI == kEpiGmmMix) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int rl = 4 * i + rr4;
+              xv[i] = (rl < nlive) ? __ldg(reinterpret_cast<const float4*>(g.xrows + (size_t)(rbase + rl) * g.N + col))
+                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+          }
+          if (!waited) {
+            if (!mbar_wait(tfull_bar + buf, bphase, abort_s)) { ok = false; break; }
+            tc_fence_after();
+            waited = true;
+          }
+          uint32_t acc[32];
+          tmem_ld32(tbase + (uint32_t)c, acc);
+          if (c + 32 >= kCols) {                              // accumulator fully read: hand the buffer back
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar + buf);
+          }
+#pragma unroll
+          for (int j = 0; j < 32; ++j) stg[lane * 33 + j] = __uint_as_float(acc[j]);
+          __syncwarp();
+          float4 bc = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (EPI == kEpiBiasF32) bc = __ldg(reinterpret_cast<const float4*>(g.bias + col));
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int rl = 4 * i + rr4;
+            const float cC = __shfl_sync(0xffffffffu, rowC, rl), cE = __shfl_sync(0xffffffffu, rowE, rl);
+            if (rl < nlive) {
+              const float* sp = stg + rl * 33 + c4;
+              float4 o;
+              if (EPI == kEpiGmmMix) {
+                o = make_float4(fmaf(cC, sp[0], cE * xv[i].x), fmaf(cC, sp[1], cE * xv[i].y),
+                                fmaf(cC, sp[2], cE * xv[i].z), fmaf(cC, sp[3], cE * xv[i].w));
+              } else {
+                o = make_float4(sp[0] + bc.x, sp[1] + bc.y, sp[2] + bc.z, sp[3] + bc.w);
+              }
+              *reinterpret_cast<float4*>(static_cast<float*>(g.out) + (size_t)(rbase + rl) * g.ldo + col) = o;
+            }
+          }
+          __syncwarp();
+        }
+      } else {
+        if (!mbar_wait(tfull_bar + buf, bphase, abort_s)) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll 1
+        for (int c = 0; c < kCols; c += 32) {
+          uint32_t acc[32];
+          tmem_ld32(tbase + (uint32_t)c, acc);
+          if (live) epilogue_chunk<EPI>(g, acc, row, n0 + c, krow);
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar + buf);
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar + buf);
     }
     if (!ok && lane == 0) {
       *abort_s = 1;
