@@ -122,33 +122,13 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
-// one 32-column chunk of one output row
+// one 32-column chunk of one output row (thread = row form; used by the small logits output only)
 template <int EPI>
 __device__ __forceinline__ void epilogue_chunk(const TcGemmArgs& g, const uint32_t (&acc)[32], int row, int col, int krow) {
   float v[32];
 #pragma unroll
   for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(acc[j]);
-  if (EPI == kEpiMlpHidden) {
-    // h = SiLU(acc + bias + E[k]) stored as bf16
-    const uint4* te = reinterpret_cast<const uint4*>(g.temb + (size_t)krow * g.N + col);
-    uint4* o = reinterpret_cast<uint4*>(static_cast<uint16_t*>(g.out) + (size_t)row * g.ldo + col);
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const uint4 t = __ldg(te + q);
-      const uint32_t tw[4] = {t.x, t.y, t.z, t.w};
-      uint32_t pk[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int j = q * 8 + u * 2;
-        float a = v[j] + __ldg(g.bias + col + j) + bf16_lo(tw[u]);
-        float b = v[j + 1] + __ldg(g.bias + col + j + 1) + bf16_hi(tw[u]);
-        a = __fdividef(a, 1.0f + __expf(-a));
-        b = __fdividef(b, 1.0f + __expf(-b));
-        pk[u] = pack_bf16x2(a, b);
-      }
-      o[q] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-    }
-  } else if (EPI == kEpiGmmLogits) {
+  if (EPI == kEpiGmmLogits) {
     // logit = logw + A * <x, mu> + Bq * |mu|^2
     const float tA = (float)__ldg(g.tcond + 4 * krow + 0);
     const double tB = __ldg(g.tcond + 4 * krow + 1);
@@ -164,7 +144,7 @@ __device__ __forceinline__ void epilogue_chunk(const TcGemmArgs& g, const uint32
       o[q] = make_float4(w[0], w[1], w[2], w[3]);
     }
   }
-  // the float-output epilogues (acc + bias; C * acc + E * x) are written in the kernel body
+  // the other epilogues (SiLU hidden layer, acc + bias, C * acc + E * x) are written in the kernel body
 }
 
 template <int BN, int EPI>
@@ -275,8 +255,8 @@ __global__ void __launch_bounds__(kThreads, 1)
       const bool live = row < M;
       const int krow = (live && g.rowk) ? __ldg(g.rowk + row) : 0;
       const uint32_t tbase = tmem_base + (uint32_t)(buf * BN + half * kCols) + ((uint32_t)(q * 32) << 16);
-      if (EPI == kEpiGmmMix || EPI == kEpiBiasF32) {
-        // Float outputs. In TMEM a thread owns a row, so direct 128-bit accesses of a warp would
+      if (EPI == kEpiGmmMix || EPI == kEpiBiasF32 || EPI == kEpiMlpHidden) {
+        // In TMEM a thread owns a row, so direct 128-bit accesses of a warp would
         // touch 32 different lines each and saturate the L1 tag stage. The 32x32 chunk is turned
         // through shared memory instead: eight lanes cover the 32 columns of a row, a warp access
         // covers four rows of 128 contiguous bytes. All eight x loads of a chunk are in flight
@@ -294,6 +274,16 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll 1
         for (int c = 0; c < kCols; c += 32) {
           const int col = n0 + c + c4;
+          uint2 tv[8];                                        // time-embedding row pieces (4 bf16 each)
+          if (EPI == kEpiMlpHidden) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int rl = 4 * i + rr4;
+              const int kr = __shfl_sync(0xffffffffu, krow, rl);
+              tv[i] = (rl < nlive) ? __ldg(reinterpret_cast<const uint2*>(g.temb + (size_t)kr * g.N + col))
+                                   : make_uint2(0u, 0u);
+            }
+          }
           float4 xv[8];
           if (EPI == kEpiGmmMix) {
 #pragma unroll
@@ -319,13 +309,22 @@ __global__ void __launch_bounds__(kThreads, 1)
           for (int j = 0; j < 32; ++j) stg[lane * 33 + j] = __uint_as_float(acc[j]);
           __syncwarp();
           float4 bc = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (EPI == kEpiBiasF32) bc = __ldg(reinterpret_cast<const float4*>(g.bias + col));
+          if (EPI == kEpiBiasF32 || EPI == kEpiMlpHidden) bc = __ldg(reinterpret_cast<const float4*>(g.bias + col));
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             const int rl = 4 * i + rr4;
             const float cC = __shfl_sync(0xffffffffu, rowC, rl), cE = __shfl_sync(0xffffffffu, rowE, rl);
             if (rl < nlive) {
               const float* sp = stg + rl * 33 + c4;
+              if (EPI == kEpiMlpHidden) {                     // h = SiLU(acc + bias + E[k]) as bf16
+                float h0 = sp[0] + bc.x + bf16_lo(tv[i].x), h1 = sp[1] + bc.y + bf16_hi(tv[i].x);
+                float h2 = sp[2] + bc.z + bf16_lo(tv[i].y), h3 = sp[3] + bc.w + bf16_hi(tv[i].y);
+                h0 = __fdividef(h0, 1.0f + __expf(-h0)); h1 = __fdividef(h1, 1.0f + __expf(-h1));
+                h2 = __fdividef(h2, 1.0f + __expf(-h2)); h3 = __fdividef(h3, 1.0f + __expf(-h3));
+                *reinterpret_cast<uint2*>(static_cast<uint16_t*>(g.out) + (size_t)(rbase + rl) * g.ldo + col) =
+                    make_uint2(pack_bf16x2(h0, h1), pack_bf16x2(h2, h3));
+                continue;
+              }
               float4 o;
               if (EPI == kEpiGmmMix) {
                 o = make_float4(fmaf(cC, sp[0], cE * xv[i].x), fmaf(cC, sp[1], cE * xv[i].y),
