@@ -25,39 +25,43 @@ __device__ __forceinline__ int window_len(const WinArgs& A, int nb) { return min
 // compaction: dense ascending list of chains with n < K and their first rows (one CTA)
 // ---------------------------------------------------------------------------------------
 __device__ void compact_scan(const WinArgs& A) {
+  // every thread owns a contiguous range of chains: count, one block-wide exclusive scan, write
   __shared__ int s_cnt[kBlock / 32], s_row[kBlock / 32];
-  __shared__ int s_base_cnt, s_base_row;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) { s_base_cnt = 0; s_base_row = 0; }
-  __syncthreads();
-  for (int b0 = 0; b0 < A.B; b0 += kBlock) {
-    const int b = b0 + tid;
-    int flag = 0, lt = 0;
-    if (b < A.B) {
-      const int nb = __ldcg(A.n + b);
-      if (nb < A.K) { flag = 1; lt = min(A.L, A.K - nb); }
-    }
-    int c = flag, r = lt;                 // inclusive warp scans
+  const int per = (A.B + kBlock - 1) / kBlock;
+  const int b0 = min(A.B, tid * per), b1 = min(A.B, b0 + per);
+  int cnt = 0, rows = 0;
+  for (int b = b0; b < b1; ++b) {
+    const int nb = __ldcg(A.n + b);
+    if (nb < A.K) { cnt += 1; rows += min(A.L, A.K - nb); }
+  }
+  int c = cnt, r = rows;                  // inclusive warp scans
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int c2 = __shfl_up_sync(0xffffffffu, c, o), r2 = __shfl_up_sync(0xffffffffu, r, o);
-      if (lane >= o) { c += c2; r += r2; }
+  for (int o = 1; o < 32; o <<= 1) {
+    const int c2 = __shfl_up_sync(0xffffffffu, c, o), r2 = __shfl_up_sync(0xffffffffu, r, o);
+    if (lane >= o) { c += c2; r += r2; }
+  }
+  if (lane == 31) { s_cnt[warp] = c; s_row[warp] = r; }
+  __syncthreads();
+  int pos = c - cnt, row = r - rows, tot_c = 0, tot_r = 0;
+  for (int w = 0; w < kBlock / 32; ++w) {
+    if (w < warp) { pos += s_cnt[w]; row += s_row[w]; }
+    tot_c += s_cnt[w];
+    tot_r += s_row[w];
+  }
+  for (int b = b0; b < b1; ++b) {
+    const int nb = __ldcg(A.n + b);
+    if (nb < A.K) {
+      A.act[pos] = b;
+      A.rowoff[pos] = row;
+      pos += 1;
+      row += min(A.L, A.K - nb);
     }
-    if (lane == 31) { s_cnt[warp] = c; s_row[warp] = r; }
-    __syncthreads();
-    int wc = 0, wr = 0;
-    for (int w = 0; w < warp; ++w) { wc += s_cnt[w]; wr += s_row[w]; }
-    const int pos = s_base_cnt + wc + c - flag;
-    const int row = s_base_row + wr + r - lt;
-    if (flag) { A.act[pos] = b; A.rowoff[pos] = row; }
-    __syncthreads();
-    if (tid == kBlock - 1) { s_base_cnt = pos + flag; s_base_row = row + lt; }
-    __syncthreads();
   }
   if (tid == 0) {
-    A.rowoff[s_base_cnt] = s_base_row;
-    A.ctl[kCtlNActive] = s_base_cnt;
-    A.ctl[kCtlNRows] = s_base_row;
+    A.rowoff[tot_c] = tot_r;
+    A.ctl[kCtlNActive] = tot_c;
+    A.ctl[kCtlNRows] = tot_r;
   }
 }
 
@@ -576,6 +580,12 @@ cudaError_t launch_verify(const WinArgs& A, int ub, cudaStream_t st) {
   return cudaGetLastError();
 }
 cudaError_t launch_advance(const WinArgs& A, int ub, cudaStream_t st) {
+  // two row copies per chain: a warp per chain up to d = 2048 keeps enough work per CTA to hide the
+  // chain of dependent index loads in front of the copies
+  if (vec4_ok(A.d) && A.d <= 2048) {
+    k_advance<32, 4><<<blocks_for(ub > 0 ? ub : 1, 32), kBlock, 0, st>>>(A);
+    return cudaGetLastError();
+  }
   SDS_DISPATCH(k_advance, A, ub, st);
   return cudaGetLastError();
 }
