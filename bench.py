@@ -213,7 +213,12 @@ def algorithmic(kind: str, w, rows_per_step: float, windows_chains: float, launc
             per_row = 2.0 * sum(w.mlp_dims[i] * w.mlp_dims[i + 1] for i in range(len(w.mlp_dims) - 1))
             return "tensor", per_row * (rows_per_step + w.B) / launches
         per_row = 4.0 * w.gmm["ncomp"] * d      # logits + mixing contractions
-        bound = "tensor" if w.gmm.get("means_bf16") else "alu"
+        if w.gmm.get("means_bf16"):
+            bound = "tensor"
+        elif kind == "denoise" and w.gmm["ncomp"] > 32 and w.gmm["ncomp"] % 128 == 0 and d % 128 == 0:
+            bound = "tensor_split"              # float operands as three bf16 planes, six products
+        else:
+            bound = "alu"
         return bound, per_row * (rows_per_step + w.B) / launches
     return "hbm", 0.0
 
@@ -324,12 +329,14 @@ def run_gpu(args, w):
         achieved, peak, unit = per_launch / avg_s / 1e9, pk["hbm_gbs"], "GB/s"
     elif bound == "tensor":
         achieved, peak, unit = per_launch / avg_s / 1e12, pk["bf16_sustained"], "TFLOP/s"
+    elif bound == "tensor_split":
+        achieved, peak, unit = per_launch / avg_s / 1e12, pk["bf16_sustained"] / 6.0, "TFLOP/s"
     else:
         peak = SMS * FP32_LANES_PER_SM * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
         achieved, unit = per_launch / avg_s / 1e12, "TFLOP/s"
-    roofline = {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
+    roofline = {"kernel": dom, "bound": "tensor" if bound == "tensor_split" else bound, "achieved": achieved, "peak": peak, "unit": unit,
                 "frac": achieved / peak, "traffic": None,
-                "peak_source": (pk["source"] + (" (sustained bf16 GEMM)" if bound == "tensor" else " (copy)")) if bound != "alu"
+                "peak_source": (pk["source"] + {"tensor": " (sustained bf16 GEMM)", "tensor_split": " (sustained bf16 GEMM / 6 products of the 3-way split)"}.get(bound, " (copy)")) if bound != "alu"
                 else "derived: 148 SMs x 128 fp32 lanes x 2 x max SM clock",
                 "avg_launch_us": avg_s * 1e6, "launches_per_step": dom_n / steps,
                 "share_of_kernel_time": dom_ms / max(sum(v[0] for v in kinds.values()), 1e-9),

@@ -169,6 +169,11 @@ int sds_sample_all(sds_ctx* ctx, float* out_dev, int32_t* nfe_calls_dev, int32_t
  * (d <= 256, <= 32 components) as one persistent kernel; 0 forces the window-by-window kernels.
  * After the whole-chain kernel only Y, N, DC and the NFE counters are meaningful for sds_get. */
 #define SDS_OPT_WHOLE_CHAIN_KERNEL 1
+/* SDS_OPT_TENSOR_SPLIT (default 1): float mixtures with more than 32 components whose shapes tile
+ * for the tensor cores (ncomp % 128 == 0, d % 128 == 0) run both contractions as bf16 tensor-core
+ * GEMMs on a three-way split of every float operand (six partial products, float accumulation);
+ * 0 forces the float ALU kernel. */
+#define SDS_OPT_TENSOR_SPLIT 2
 int sds_set_option(sds_ctx* ctx, int32_t option, int64_t value);
 
 /* Same with host buffers: copies the mixture parameters means_host [ncomp, d] (float or bf16, the

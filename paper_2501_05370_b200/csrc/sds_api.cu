@@ -41,6 +41,7 @@ struct Layout {
   size_t musq;
   size_t H0, H1;          // MLP hidden activations (bf16)
   size_t logits, R, Mt;   // large mixture: logits (f32), responsibilities (bf16), transposed means (bf16)
+  size_t Xs, Ms, Lscr;    // float mixture on tensor cores: 3 bf16 planes of the rows / of the means, shifted logits
   size_t total;
 };
 
@@ -71,6 +72,7 @@ struct sds_ctx {
   cudaEvent_t ev[2] = {nullptr, nullptr};
   bool musq_ready = false;
   bool whole_chain = true;          // sds_sample_all may use the whole-chain kernel
+  bool tensor_split = true;         // float mixtures of tensor-core shape use the 3-way bf16 split
   // optional per-kernel timing: event pairs recorded around each launch, summed on read
   bool prof_on = false;
   std::vector<cudaEvent_t> prof_ev[SDS_PROF_KINDS];
@@ -80,6 +82,13 @@ struct sds_ctx {
 };
 
 namespace {
+
+// float mixture whose two contractions tile for the tensor cores (and is too large for the
+// one-warp-per-row kernel): eligible for the split-precision path
+bool gmm_split_shape(const sds_denoiser& den, int32_t d) {
+  return den.kind == SDS_DEN_GMM && den.means_dtype == SDS_F32 && den.ncomp > 32 && den.ncomp % 128 == 0 &&
+         d % 128 == 0;
+}
 
 bool wants_bf16_rows(const sds_denoiser& den) {
   return den.kind == SDS_DEN_MLP || (den.kind == SDS_DEN_GMM && den.means_dtype == SDS_BF16);
@@ -113,7 +122,15 @@ void make_layout(const sds_schedule* sch, const sds_denoiser* den, int64_t B, in
   l.nfe_calls = cv.take((size_t)B * 4);
   l.nfe_rows = cv.take((size_t)B * 4);
   l.musq = (den->kind == SDS_DEN_GMM) ? cv.take((size_t)den->ncomp * 8) : kNone;
-  l.H0 = l.H1 = l.logits = l.R = l.Mt = kNone;
+  l.H0 = l.H1 = l.logits = l.R = l.Mt = l.Xs = l.Ms = l.Lscr = kNone;
+  if (gmm_split_shape(*den, d)) {
+    l.Xs = cv.take(3 * rows * (size_t)d * 2);
+    l.Ms = cv.take(3 * (size_t)den->ncomp * d * 2);
+    l.Mt = cv.take(3 * (size_t)d * den->ncomp * 2);
+    l.R = cv.take(3 * rows * (size_t)den->ncomp * 2);
+    l.logits = cv.take(rows * (size_t)den->ncomp * 4);
+    l.Lscr = cv.take(rows * (size_t)den->ncomp * 4);
+  }
   if (den->kind == SDS_DEN_MLP) {
     size_t width = 0;
     for (int i = 1; i < den->nlayer; ++i) width = std::max(width, (size_t)den->dims[i]);
@@ -279,6 +296,45 @@ int run_denoiser(sds_ctx* c, const float* X, const uint16_t* Xb, const int* rowk
   if (rows_ub <= 0) return SDS_OK;
   switch (c->den.kind) {
     case SDS_DEN_GMM: {
+      if (c->den.means_dtype == SDS_F32 && c->tensor_split && gmm_split_shape(c->den, c->d)) {
+        // Float mixture on the tensor cores: rows, means and responsibilities are split into three
+        // bf16 planes each (x = h + m + l carries the 24-bit significand); the six products of
+        // total order <= 2 are accumulated, smallest first, in one TMEM accumulator.
+        const float* means = static_cast<const float*>(c->den.means_dev);
+        const size_t nc = (size_t)c->den.ncomp, dd = (size_t)c->d, cap = (size_t)(c->B * c->L);
+        uint16_t* Ms = at<uint16_t>(c, c->lay.Ms);
+        uint16_t* Mt = at<uint16_t>(c, c->lay.Mt);
+        uint16_t* Xs = at<uint16_t>(c, c->lay.Xs);
+        uint16_t* Rs = at<uint16_t>(c, c->lay.R);
+        float* logits = at<float>(c, c->lay.logits);
+        const bool fresh = !c->musq_ready;
+        int rc = ensure_musq(c);
+        if (rc != SDS_OK) return rc;
+        if (fresh) {
+          SDS_LAUNCH(c, SDS_PROF_AUX, launch_split3(means, nc * dd, nc * dd, Ms, c->stream));
+          for (int i = 0; i < 3; ++i)
+            SDS_LAUNCH(c, SDS_PROF_AUX, launch_transpose_bf16(Ms + i * nc * dd, (int)nc, (int)dd, Mt + i * nc * dd, c->stream));
+        }
+        SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_split3(X, (size_t)rows_ub * dd, cap * dd, Xs, c->stream));
+        static const uint8_t kA[6] = {2, 1, 0, 1, 0, 0}, kB[6] = {0, 1, 2, 0, 1, 0};
+        TcGemmArgs g = tc_args(c, rowk, nrows_dev, rows_ub);
+        g.N = (int)nc; g.K = (int)dd; g.out = logits; g.ldo = (int)nc;
+        g.tcond = at<double>(c, c->lay.tcond); g.musq = at<double>(c, c->lay.musq); g.logw = c->den.logw_dev;
+        g.nseg = 6; g.nplanes = 3; g.a_plane = cap * dd; g.b_plane = nc * dd;
+        for (int i = 0; i < 6; ++i) { g.a_idx[i] = kA[i]; g.b_idx[i] = kB[i]; }
+        SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiGmmLogits, g, Xs, Ms, c->stream));
+        SDS_LAUNCH(c, SDS_PROF_DENOISE,
+                   launch_softmax_split3(logits, nrows_dev, (int)rows_ub, (int)nc, (int)dd, X, means,
+                                         at<double>(c, c->lay.musq), c->den.logw_dev, at<double>(c, c->lay.tcond), rowk,
+                                         cap * nc, Rs, at<float>(c, c->lay.Lscr), c->stream));
+        TcGemmArgs m = tc_args(c, rowk, nrows_dev, rows_ub);
+        m.N = (int)dd; m.K = (int)nc; m.out = out; m.ldo = (int)dd;
+        m.tcond = at<double>(c, c->lay.tcond); m.xrows = X;
+        m.nseg = 6; m.nplanes = 3; m.a_plane = cap * nc; m.b_plane = nc * dd;
+        for (int i = 0; i < 6; ++i) { m.a_idx[i] = kA[i]; m.b_idx[i] = kB[i]; }
+        SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiGmmMix, m, Rs, Mt, c->stream));
+        return SDS_OK;
+      }
       if (c->den.means_dtype == SDS_F32) {
         const int rc = ensure_musq(c);
         if (rc != SDS_OK) return rc;
@@ -623,6 +679,7 @@ int sds_set_option(sds_ctx* c, int32_t option, int64_t value) {
   if (!c) return SDS_EINVAL;
   switch (option) {
     case SDS_OPT_WHOLE_CHAIN_KERNEL: c->whole_chain = value != 0; return SDS_OK;
+    case SDS_OPT_TENSOR_SPLIT: c->tensor_split = value != 0; return SDS_OK;
     default: return SDS_EINVAL;
   }
 }

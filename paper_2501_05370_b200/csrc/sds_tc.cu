@@ -149,7 +149,9 @@ __device__ __forceinline__ void epilogue_chunk(const TcGemmArgs& g, const uint32
 
 template <int BN, int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
-    k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, TcGemmArgs g) {
+    k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
+              const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB0,
+              const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, TcGemmArgs g) {
   using C = TileCfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte aligned operand stages (required by the 128-byte swizzle), barriers behind them
@@ -166,7 +168,10 @@ __global__ void __launch_bounds__(kThreads, 1)
   const int M = g.nrows_dev ? min(*g.nrows_dev, g.rows_host) : g.rows_host;
   const int m_tiles = (M + BM - 1) / BM, n_tiles = g.N / BN;
   const int total_tiles = m_tiles * n_tiles;
-  const int kblocks = (g.K + BK - 1) / BK;
+  // K loop = nseg segments of K/BK blocks; segment s multiplies plane a_idx[s] of A with plane
+  // b_idx[s] of B into the same accumulator (split-precision products; one segment otherwise)
+  const int kb_seg = (g.K + BK - 1) / BK;
+  const int kblocks = kb_seg * g.nseg;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::kStages; ++s) { mbar_init(full_bar + s, 1); mbar_init(empty_bar + s, 1); }
@@ -197,8 +202,10 @@ __global__ void __launch_bounds__(kThreads, 1)
           if (!mbar_wait(empty_bar + stage, phase ^ 1u, abort_s)) { ok = false; break; }
           uint8_t* sa = stages + stage * C::kStageBytes;
           mbar_expect_tx(full_bar + stage, (uint32_t)C::kStageBytes);
-          tma_load_2d(sa, &tmA, kb * BK, m0, full_bar + stage);
-          tma_load_2d(sa + C::kABytes, &tmB, kb * BK, n0, full_bar + stage);
+          const int seg = kb / kb_seg, kk = (kb - seg * kb_seg) * BK;
+          const int ai = g.a_idx[seg], bi = g.b_idx[seg];
+          tma_load_2d(sa, ai == 0 ? &tmA0 : (ai == 1 ? &tmA1 : &tmA2), kk, m0, full_bar + stage);
+          tma_load_2d(sa + C::kABytes, bi == 0 ? &tmB0 : (bi == 1 ? &tmB1 : &tmB2), kk, n0, full_bar + stage);
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -431,6 +438,92 @@ __global__ void k_f32_to_bf16(const float* __restrict__ x, size_t n, uint16_t* _
   }
 }
 
+// x = h + m + l with h, m, l bfloat16 (each the rounded remainder of the previous ones): three
+// planes that together carry the 24-bit significand of a float
+__device__ __forceinline__ void split3(float x, uint16_t& h, uint16_t& m, uint16_t& l) {
+  const uint32_t ph = pack_bf16x2(x, 0.f) & 0xffffu;
+  const float r1 = x - __uint_as_float(ph << 16);
+  const uint32_t pm = pack_bf16x2(r1, 0.f) & 0xffffu;
+  const float r2 = r1 - __uint_as_float(pm << 16);
+  h = (uint16_t)ph; m = (uint16_t)pm; l = (uint16_t)(pack_bf16x2(r2, 0.f) & 0xffffu);
+}
+
+__global__ void k_split3(const float* __restrict__ x, size_t n, size_t plane, uint16_t* __restrict__ out) {
+  for (size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4; i < n; i += (size_t)gridDim.x * blockDim.x * 4) {
+    float v[4] = {0.f, 0.f, 0.f, 0.f};
+    if (i + 3 < n) { const float4 t = ld4(x + i); v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; }
+    else for (int u = 0; u < 4 && i + u < n; ++u) v[u] = x[i + u];
+    uint16_t p[3][4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) split3(v[u], p[0][u], p[1][u], p[2][u]);
+#pragma unroll
+    for (int q = 0; q < 3; ++q) {
+      if (i + 3 < n) {
+        *reinterpret_cast<uint2*>(out + q * plane + i) =
+            make_uint2((uint32_t)p[q][0] | ((uint32_t)p[q][1] << 16), (uint32_t)p[q][2] | ((uint32_t)p[q][3] << 16));
+      } else {
+        for (int u = 0; u < 4 && i + u < n; ++u) out[q * plane + i + u] = p[q][u];
+      }
+    }
+  }
+}
+
+// Row softmax for the split-precision mixture. The tensor-core logits are float sums of large
+// terms; components within 30 of the row maximum get their logit again in double (warp-wide dot
+// product, fixed combination order), all others weigh less than e^-29. Writes the normalised
+// responsibilities as three bf16 planes. One warp per row.
+__global__ void __launch_bounds__(256)
+    k_softmax_split3(const float* __restrict__ logits, const int* __restrict__ nrows_dev, int rows_host, int ncomp,
+                     int d, const float* __restrict__ X, const float* __restrict__ means,
+                     const double* __restrict__ musq, const float* __restrict__ logw,
+                     const double* __restrict__ tcond, const int* __restrict__ rowk, size_t rplane,
+                     uint16_t* __restrict__ R, float* __restrict__ scratch) {
+  const int nrows = nrows_dev ? min(*nrows_dev, rows_host) : rows_host;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int row = blockIdx.x * 8 + warp; row < nrows; row += gridDim.x * 8) {
+    const float* lg = logits + (size_t)row * ncomp;
+    float* sh = scratch + (size_t)row * ncomp;           // shifted logits (in place is not possible: logits is const)
+    float mx = -INFINITY;
+    for (int c = lane; c < ncomp; c += 32) mx = fmaxf(mx, lg[c]);
+    mx = warp_max(mx);
+    const int k = rowk[row];
+    const double tA = __ldg(tcond + 4 * k + 0), tB = __ldg(tcond + 4 * k + 1);
+    const float* x = X + (size_t)row * d;
+    for (int c0 = 0; c0 < ncomp; c0 += 32) {
+      const int c = c0 + lane;
+      const float v = (c < ncomp) ? lg[c] : -INFINITY;
+      float val = v - mx;
+      unsigned sel = __ballot_sync(0xffffffffu, v >= mx - 30.0f);
+      while (sel) {                                        // warp-uniform loop over the selected components
+        const int l = __ffs(sel) - 1;
+        sel &= sel - 1;
+        const float* mu = means + (size_t)(c0 + l) * d;
+        double a = 0.0;
+        for (int i = lane; i < d; i += 32) a = fma((double)x[i], (double)mu[i], a);
+        a = warp_sum(a);
+        const double exact = fma(tA, a, fma(tB, __ldg(musq + c0 + l), (double)__ldg(logw + c0 + l)));
+        if (lane == l) val = (float)(exact - (double)mx);
+      }
+      if (c < ncomp) sh[c] = val;
+    }
+    __syncwarp();
+    float m2 = -INFINITY;
+    for (int c = lane; c < ncomp; c += 32) m2 = fmaxf(m2, sh[c]);
+    m2 = warp_max(m2);
+    float den = 0.f;
+    for (int c = lane; c < ncomp; c += 32) den += expf(sh[c] - m2);
+    den = warp_sum(den);
+    const float inv = 1.0f / den;
+    for (int c = lane; c < ncomp; c += 32) {
+      uint16_t h, m, l;
+      split3(expf(sh[c] - m2) * inv, h, m, l);
+      R[(size_t)row * ncomp + c] = h;
+      R[rplane + (size_t)row * ncomp + c] = m;
+      R[2 * rplane + (size_t)row * ncomp + c] = l;
+    }
+  }
+}
+
 PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
   static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
   if (!fn) {
@@ -460,9 +553,13 @@ bool make_tmap(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t K, uin
 template <int BN, int EPI>
 cudaError_t launch_t(const TcGemmArgs& g, const void* A, const void* B, int grid_tiles_ub, cudaStream_t st) {
   using C = TileCfg<BN>;
-  CUtensorMap tmA, tmB;
-  if (!make_tmap(&tmA, A, (uint64_t)g.rows_cap, (uint64_t)g.K, BM)) return cudaErrorInvalidValue;
-  if (!make_tmap(&tmB, B, (uint64_t)g.N, (uint64_t)g.K, BN)) return cudaErrorInvalidValue;
+  CUtensorMap tmA[3], tmB[3];
+  for (int i = 0; i < 3; ++i) {
+    const uint16_t* a = static_cast<const uint16_t*>(A) + (size_t)i * g.a_plane;
+    const uint16_t* b = static_cast<const uint16_t*>(B) + (size_t)i * g.b_plane;
+    if (!make_tmap(&tmA[i], g.nplanes > i ? a : A, (uint64_t)g.rows_cap, (uint64_t)g.K, BM)) return cudaErrorInvalidValue;
+    if (!make_tmap(&tmB[i], g.nplanes > i ? b : B, (uint64_t)g.N, (uint64_t)g.K, BN)) return cudaErrorInvalidValue;
+  }
   cudaError_t e = cudaFuncSetAttribute(k_gemm_tc<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
   if (e != cudaSuccess) return e;
   int dev = 0, sms = 148;
@@ -470,7 +567,7 @@ cudaError_t launch_t(const TcGemmArgs& g, const void* A, const void* B, int grid
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   int grid = grid_tiles_ub < sms ? grid_tiles_ub : sms;
   if (grid < 1) grid = 1;
-  k_gemm_tc<BN, EPI><<<grid, kThreads, C::kSmemBytes, st>>>(tmA, tmB, g);
+  k_gemm_tc<BN, EPI><<<grid, kThreads, C::kSmemBytes, st>>>(tmA[0], tmA[1], tmA[2], tmB[0], tmB[1], tmB[2], g);
   return cudaGetLastError();
 }
 
@@ -478,7 +575,10 @@ cudaError_t launch_t(const TcGemmArgs& g, const void* A, const void* B, int grid
 
 bool tc_shape_ok(int N, int K) { return N % 128 == 0 && K % 8 == 0 && K >= 8; }
 
-cudaError_t launch_gemm_tc(int epi, const TcGemmArgs& g, const void* A_bf16, const void* B_bf16, cudaStream_t st) {
+cudaError_t launch_gemm_tc(int epi, const TcGemmArgs& g_in, const void* A_bf16, const void* B_bf16, cudaStream_t st) {
+  TcGemmArgs g = g_in;
+  if (g.nseg <= 0) { g.nseg = 1; g.nplanes = 1; g.a_idx[0] = g.b_idx[0] = 0; }
+  if (g.nseg > 8 || g.nplanes < 1 || g.nplanes > 3) return cudaErrorInvalidValue;
   if (!tc_shape_ok(g.N, g.K) || g.rows_cap <= 0 || g.rows_host > g.rows_cap) return cudaErrorInvalidValue;
   if (g.rows_host <= 0) return cudaSuccess;
   const bool wide = (g.N % 256) == 0;
@@ -515,6 +615,26 @@ cudaError_t launch_transpose_bf16(const uint16_t* M, int ncomp, int d, uint16_t*
 
 cudaError_t launch_musq_bf16(const uint16_t* means, int ncomp, int d, double* musq, cudaStream_t st) {
   k_musq_bf16<<<(ncomp + 3) / 4, 128, 0, st>>>(means, ncomp, d, musq);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_split3(const float* x, size_t n, size_t plane, uint16_t* out, cudaStream_t st) {
+  size_t blocks = (n / 4 + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  k_split3<<<(int)blocks, 256, 0, st>>>(x, n, plane, out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_softmax_split3(const float* logits, const int* nrows_dev, int rows_host, int ncomp, int d,
+                                  const float* X, const float* means, const double* musq, const float* logw,
+                                  const double* tcond, const int* rowk, size_t rplane, uint16_t* R, float* scratch,
+                                  cudaStream_t st) {
+  int blocks = (rows_host + 7) / 8;
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  if (blocks < 1) blocks = 1;
+  k_softmax_split3<<<blocks, 256, 0, st>>>(logits, nrows_dev, rows_host, ncomp, d, X, means, musq, logw, tcond, rowk,
+                                           rplane, R, scratch);
   return cudaGetLastError();
 }
 

@@ -29,6 +29,12 @@ struct TcGemmArgs {
   const float* logw;     // [N]
   const float* xrows;    // [M, N] f32
   int* err;              // device word, set non-zero if a bounded wait gave up
+  // split-precision products: A and B each come as nplanes bf16 planes (a_plane / b_plane elements
+  // apart); segment s of the K loop multiplies plane a_idx[s] of A with plane b_idx[s] of B.
+  // nseg = 0 means one plane, one segment.
+  int nseg, nplanes;
+  size_t a_plane, b_plane;
+  uint8_t a_idx[8], b_idx[8];
 };
 
 bool tc_shape_ok(int N, int K);
@@ -37,6 +43,11 @@ cudaError_t launch_softmax_bf16(const float* logits, const int* nrows_dev, int r
                                 cudaStream_t st);
 cudaError_t launch_transpose_bf16(const uint16_t* M, int ncomp, int d, uint16_t* Mt, cudaStream_t st);
 cudaError_t launch_musq_bf16(const uint16_t* means, int ncomp, int d, double* musq, cudaStream_t st);
+cudaError_t launch_split3(const float* x, size_t n, size_t plane, uint16_t* out, cudaStream_t st);
+cudaError_t launch_softmax_split3(const float* logits, const int* nrows_dev, int rows_host, int ncomp, int d,
+                                  const float* X, const float* means, const double* musq, const float* logw,
+                                  const double* tcond, const int* rowk, size_t rplane, uint16_t* R, float* scratch,
+                                  cudaStream_t st);
 cudaError_t launch_f32_to_bf16(const float* x, size_t n, uint16_t* out, cudaStream_t st);
 
 }  // namespace sds

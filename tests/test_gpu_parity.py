@@ -39,7 +39,8 @@ def test_rng_normals_and_uniforms(b0, k, d):
 
 @pytest.mark.parametrize("name,d,ncomp,rows", [("cfg1", 2, 4, 37), ("cfg2", 64, 16, 515), ("cfg2", 33, 5, 70),
                                               ("cfg5", 96, 40, 130), ("cfg5", 1024, 24, 21), ("cfg5", 1024, 256, 150),
-                                              ("cfg2", 200, 100, 131), ("cfg5", 260, 33, 64)])
+                                              ("cfg2", 200, 100, 131), ("cfg5", 260, 33, 64), ("cfg2", 256, 128, 300),
+                                              ("cfg5", 384, 256, 77)])
 def test_gmm_denoiser_rows(name, d, ncomp, rows):
     torch = _torch()
     w = wl.WORKLOADS[name].scaled(d=d, B=max(rows, 1), L=1)
@@ -57,6 +58,26 @@ def test_gmm_denoiser_rows(name, d, ncomp, rows):
         want = den(x[r].astype(np.float64), int(k[r]))
         assert rel_l2(out[r], want) <= 1e-5, (r, rel_l2(out[r], want))
     s.close()
+
+
+def test_split_precision_tensor_path_agrees_with_float_alu_path():
+    """Float mixtures of tensor-core shape run as bf16 GEMMs on a three-way split of every operand;
+    the float ALU kernel (option off) must give the same rows to float accuracy."""
+    torch = _torch()
+    for name, d, ncomp in (("cfg2", 256, 128), ("cfg5", 1024, 256)):
+        rows = 333
+        w = wl.WORKLOADS[name].scaled(d=d, B=rows, L=1)
+        gp = w.gmm_params(d=d, ncomp=ncomp)
+        s = sds.sampler_for(w, gmm=gp)
+        rng = np.random.default_rng(9)
+        x = torch.from_numpy((rng.standard_normal((rows, d)) * (4.0 if w.sampler == "ula" else 1.5)).astype(np.float32)).cuda()
+        k = torch.from_numpy(rng.integers(0, w.K, size=rows).astype(np.int32)).cuda()
+        a = s.denoise(x, k).cpu().numpy()
+        s.set_option(s.OPT_TENSOR_SPLIT, 0)
+        b = s.denoise(x, k).cpu().numpy()
+        err = np.linalg.norm(a - b, axis=1) / np.maximum(np.linalg.norm(b, axis=1), 1e-6)
+        assert err.max() <= 1e-5, err.max()
+        s.close()
 
 
 # ------------------------------------------------------------------ one window, forced ---
