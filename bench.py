@@ -215,7 +215,7 @@ def algorithmic(kind: str, w, rows_per_step: float, windows_chains: float, launc
         per_row = 4.0 * w.gmm["ncomp"] * d      # logits + mixing contractions
         if w.gmm.get("means_bf16"):
             bound = "tensor"
-        elif kind == "denoise" and w.gmm["ncomp"] > 32 and w.gmm["ncomp"] % 128 == 0 and d % 128 == 0:
+        elif kind == "denoise" and 32 < w.gmm["ncomp"] <= 1024 and w.gmm["ncomp"] % 128 == 0 and d % 128 == 0:
             bound = "tensor_split"              # float operands as three bf16 planes, six products
         else:
             bound = "alu"

@@ -41,7 +41,7 @@ struct Layout {
   size_t musq;
   size_t H0, H1;          // MLP hidden activations (bf16)
   size_t logits, R, Mt;   // large mixture: logits (f32), responsibilities (bf16), transposed means (bf16)
-  size_t Xs, Ms, Lscr;    // float mixture on tensor cores: 3 bf16 planes of the rows / of the means, shifted logits
+  size_t Xs, Ms;          // float mixture on tensor cores: 3 bf16 planes of the rows / of the means
   size_t total;
 };
 
@@ -87,7 +87,7 @@ namespace {
 // one-warp-per-row kernel): eligible for the split-precision path
 bool gmm_split_shape(const sds_denoiser& den, int32_t d) {
   return den.kind == SDS_DEN_GMM && den.means_dtype == SDS_F32 && den.ncomp > 32 && den.ncomp % 128 == 0 &&
-         d % 128 == 0;
+         den.ncomp <= 1024 && d % 128 == 0;
 }
 
 bool wants_bf16_rows(const sds_denoiser& den) {
@@ -122,14 +122,13 @@ void make_layout(const sds_schedule* sch, const sds_denoiser* den, int64_t B, in
   l.nfe_calls = cv.take((size_t)B * 4);
   l.nfe_rows = cv.take((size_t)B * 4);
   l.musq = (den->kind == SDS_DEN_GMM) ? cv.take((size_t)den->ncomp * 8) : kNone;
-  l.H0 = l.H1 = l.logits = l.R = l.Mt = l.Xs = l.Ms = l.Lscr = kNone;
+  l.H0 = l.H1 = l.logits = l.R = l.Mt = l.Xs = l.Ms = kNone;
   if (gmm_split_shape(*den, d)) {
     l.Xs = cv.take(3 * rows * (size_t)d * 2);
     l.Ms = cv.take(3 * (size_t)den->ncomp * d * 2);
     l.Mt = cv.take(3 * (size_t)d * den->ncomp * 2);
     l.R = cv.take(3 * rows * (size_t)den->ncomp * 2);
     l.logits = cv.take(rows * (size_t)den->ncomp * 4);
-    l.Lscr = cv.take(rows * (size_t)den->ncomp * 4);
   }
   if (den->kind == SDS_DEN_MLP) {
     size_t width = 0;
@@ -326,7 +325,7 @@ int run_denoiser(sds_ctx* c, const float* X, const uint16_t* Xb, const int* rowk
         SDS_LAUNCH(c, SDS_PROF_DENOISE,
                    launch_softmax_split3(logits, nrows_dev, (int)rows_ub, (int)nc, (int)dd, X, means,
                                          at<double>(c, c->lay.musq), c->den.logw_dev, at<double>(c, c->lay.tcond), rowk,
-                                         cap * nc, Rs, at<float>(c, c->lay.Lscr), c->stream));
+                                         cap * nc, Rs, c->stream));
         TcGemmArgs m = tc_args(c, rowk, nrows_dev, rows_ub);
         m.N = (int)dd; m.K = (int)nc; m.out = out; m.ldo = (int)dd;
         m.tcond = at<double>(c, c->lay.tcond); m.xrows = X;

@@ -472,54 +472,76 @@ __global__ void k_split3(const float* __restrict__ x, size_t n, size_t plane, ui
 // terms; components within 30 of the row maximum get their logit again in double (warp-wide dot
 // product, fixed combination order), all others weigh less than e^-29. Writes the normalised
 // responsibilities as three bf16 planes. One warp per row.
+template <int NQ>   // ncomp = 128 * NQ: a lane holds NQ groups of four consecutive components in registers
 __global__ void __launch_bounds__(256)
-    k_softmax_split3(const float* __restrict__ logits, const int* __restrict__ nrows_dev, int rows_host, int ncomp,
-                     int d, const float* __restrict__ X, const float* __restrict__ means,
+    k_softmax_split3(const float* __restrict__ logits, const int* __restrict__ nrows_dev, int rows_host, int d,
+                     const float* __restrict__ X, const float* __restrict__ means,
                      const double* __restrict__ musq, const float* __restrict__ logw,
                      const double* __restrict__ tcond, const int* __restrict__ rowk, size_t rplane,
-                     uint16_t* __restrict__ R, float* __restrict__ scratch) {
+                     uint16_t* __restrict__ R) {
+  constexpr int ncomp = 128 * NQ;
   const int nrows = nrows_dev ? min(*nrows_dev, rows_host) : rows_host;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int row = blockIdx.x * 8 + warp; row < nrows; row += gridDim.x * 8) {
     const float* lg = logits + (size_t)row * ncomp;
-    float* sh = scratch + (size_t)row * ncomp;           // shifted logits (in place is not possible: logits is const)
+    float v[NQ][4];
     float mx = -INFINITY;
-    for (int c = lane; c < ncomp; c += 32) mx = fmaxf(mx, lg[c]);
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) {
+      const float4 t = ld4(lg + 4 * (lane + 32 * q));
+      v[q][0] = t.x; v[q][1] = t.y; v[q][2] = t.z; v[q][3] = t.w;
+      mx = fmaxf(mx, fmaxf(fmaxf(t.x, t.y), fmaxf(t.z, t.w)));
+    }
     mx = warp_max(mx);
     const int k = rowk[row];
     const double tA = __ldg(tcond + 4 * k + 0), tB = __ldg(tcond + 4 * k + 1);
     const float* x = X + (size_t)row * d;
-    for (int c0 = 0; c0 < ncomp; c0 += 32) {
-      const int c = c0 + lane;
-      const float v = (c < ncomp) ? lg[c] : -INFINITY;
-      float val = v - mx;
-      unsigned sel = __ballot_sync(0xffffffffu, v >= mx - 30.0f);
-      while (sel) {                                        // warp-uniform loop over the selected components
-        const int l = __ffs(sel) - 1;
-        sel &= sel - 1;
-        const float* mu = means + (size_t)(c0 + l) * d;
-        double a = 0.0;
-        for (int i = lane; i < d; i += 32) a = fma((double)x[i], (double)mu[i], a);
-        a = warp_sum(a);
-        const double exact = fma(tA, a, fma(tB, __ldg(musq + c0 + l), (double)__ldg(logw + c0 + l)));
-        if (lane == l) val = (float)(exact - (double)mx);
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        float val = v[q][u] - mx;
+        unsigned sel = __ballot_sync(0xffffffffu, v[q][u] >= mx - 30.0f);
+        while (sel) {                                      // warp-uniform loop over the selected components
+          const int l = __ffs(sel) - 1;
+          sel &= sel - 1;
+          const int c = 4 * (l + 32 * q) + u;
+          const float* mu = means + (size_t)c * d;
+          double a = 0.0;
+          for (int i = lane; i < d; i += 32) a = fma((double)x[i], (double)mu[i], a);
+          a = warp_sum(a);
+          const double exact = fma(tA, a, fma(tB, __ldg(musq + c), (double)__ldg(logw + c)));
+          if (lane == l) val = (float)(exact - (double)mx);
+        }
+        v[q][u] = val;
       }
-      if (c < ncomp) sh[c] = val;
     }
-    __syncwarp();
     float m2 = -INFINITY;
-    for (int c = lane; c < ncomp; c += 32) m2 = fmaxf(m2, sh[c]);
+#pragma unroll
+    for (int q = 0; q < NQ; ++q)
+#pragma unroll
+      for (int u = 0; u < 4; ++u) m2 = fmaxf(m2, v[q][u]);
     m2 = warp_max(m2);
     float den = 0.f;
-    for (int c = lane; c < ncomp; c += 32) den += expf(sh[c] - m2);
+#pragma unroll
+    for (int q = 0; q < NQ; ++q)
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        v[q][u] = expf(v[q][u] - m2);
+        den += v[q][u];
+      }
     den = warp_sum(den);
     const float inv = 1.0f / den;
-    for (int c = lane; c < ncomp; c += 32) {
-      uint16_t h, m, l;
-      split3(expf(sh[c] - m2) * inv, h, m, l);
-      R[(size_t)row * ncomp + c] = h;
-      R[rplane + (size_t)row * ncomp + c] = m;
-      R[2 * rplane + (size_t)row * ncomp + c] = l;
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) {
+      uint16_t p[3][4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) split3(v[q][u] * inv, p[0][u], p[1][u], p[2][u]);
+      const size_t o = (size_t)row * ncomp + 4 * (lane + 32 * q);
+#pragma unroll
+      for (int pl = 0; pl < 3; ++pl)
+        *reinterpret_cast<uint2*>(R + pl * rplane + o) = make_uint2((uint32_t)p[pl][0] | ((uint32_t)p[pl][1] << 16),
+                                                                    (uint32_t)p[pl][2] | ((uint32_t)p[pl][3] << 16));
     }
   }
 }
@@ -628,13 +650,20 @@ cudaError_t launch_split3(const float* x, size_t n, size_t plane, uint16_t* out,
 
 cudaError_t launch_softmax_split3(const float* logits, const int* nrows_dev, int rows_host, int ncomp, int d,
                                   const float* X, const float* means, const double* musq, const float* logw,
-                                  const double* tcond, const int* rowk, size_t rplane, uint16_t* R, float* scratch,
-                                  cudaStream_t st) {
+                                  const double* tcond, const int* rowk, size_t rplane, uint16_t* R, cudaStream_t st) {
   int blocks = (rows_host + 7) / 8;
   if (blocks > 148 * 8) blocks = 148 * 8;
   if (blocks < 1) blocks = 1;
-  k_softmax_split3<<<blocks, 256, 0, st>>>(logits, nrows_dev, rows_host, ncomp, d, X, means, musq, logw, tcond, rowk,
-                                           rplane, R, scratch);
+#define SDS_SM3(NQ)                                                                                              \
+  case NQ:                                                                                                       \
+    k_softmax_split3<NQ><<<blocks, 256, 0, st>>>(logits, nrows_dev, rows_host, d, X, means, musq, logw, tcond,   \
+                                                 rowk, rplane, R);                                               \
+    break;
+  switch (ncomp / 128) {
+    SDS_SM3(1) SDS_SM3(2) SDS_SM3(3) SDS_SM3(4) SDS_SM3(5) SDS_SM3(6) SDS_SM3(7) SDS_SM3(8)
+    default: return cudaErrorInvalidValue;
+  }
+#undef SDS_SM3
   return cudaGetLastError();
 }
 

@@ -46,8 +46,7 @@ cudaError_t launch_musq_bf16(const uint16_t* means, int ncomp, int d, double* mu
 cudaError_t launch_split3(const float* x, size_t n, size_t plane, uint16_t* out, cudaStream_t st);
 cudaError_t launch_softmax_split3(const float* logits, const int* nrows_dev, int rows_host, int ncomp, int d,
                                   const float* X, const float* means, const double* musq, const float* logw,
-                                  const double* tcond, const int* rowk, size_t rplane, uint16_t* R, float* scratch,
-                                  cudaStream_t st);
+                                  const double* tcond, const int* rowk, size_t rplane, uint16_t* R, cudaStream_t st);
 cudaError_t launch_f32_to_bf16(const float* x, size_t n, uint16_t* out, cudaStream_t st);
 
 }  // namespace sds
