@@ -373,3 +373,90 @@ def test_set_state_resume_is_bitwise():
         s2.draft(); s2.verify_window(); na = s2.advance()
     assert np.array_equal(s2.get(sb.GET_Y), ref)
     s.close(); s2.close()
+
+
+# ------------------------------------------------------------------ callback denoiser, failures ---
+
+class _DevArray:
+    """Zero-copy view of device memory handed to a callback (CUDA array interface)."""
+
+    def __init__(self, ptr, shape, typestr):
+        self.__cuda_array_interface__ = {"data": (int(ptr), False), "shape": tuple(shape), "typestr": typestr,
+                                         "version": 2, "strides": None}
+
+
+def _make_callback(torch, means_t, logw_t, tcond_t, poison_row=None, fail=False):
+    """User denoiser written with torch ops on the library's stream: the same mixture formula."""
+    state = {"poisoned": False}
+
+    def cb(user, x_ptr, k_ptr, rows, d, out_ptr, stream):
+        if fail:
+            return 7
+        with torch.cuda.stream(torch.cuda.ExternalStream(int(stream or 0))):
+            x = torch.as_tensor(_DevArray(x_ptr, (rows, d), "<f4"), device="cuda")
+            k = torch.as_tensor(_DevArray(k_ptr, (rows,), "<i4"), device="cuda").long()
+            out = torch.as_tensor(_DevArray(out_ptr, (rows, d), "<f4"), device="cuda")
+            tc = tcond_t[k]                                              # [rows, 4] double
+            xd = x.double()
+            lg = logw_t.double()[None, :] + tc[:, 0:1] * (xd @ means_t.double().T) \
+                + tc[:, 1:2] * (means_t.double() ** 2).sum(1)[None, :]
+            r = torch.softmax(lg, dim=1)
+            res = tc[:, 2:3] * (r @ means_t.double()) + tc[:, 3:4] * xd
+            if poison_row is not None and not state["poisoned"] and rows > poison_row:
+                res[poison_row] = float("nan")            # only the first (initial) target call is hit
+                state["poisoned"] = True
+            out.copy_(res.float())
+        return 0
+    return cb
+
+
+def test_callback_denoiser_matches_builtin_mixture_and_oracle():
+    torch = _torch()
+    w = wl.WORKLOADS["cfg2"].scaled(B=40, K=30)
+    gp = w.gmm_params()
+    a, c, sig, tcond = sds.schedule_for(w)
+    means_t, logw_t = torch.from_numpy(gp.means).cuda(), torch.from_numpy(gp.logw).cuda()
+    tcond_t = torch.from_numpy(tcond).cuda()
+    s_cb = sb.Sampler(a, c, sig, 40, w.d, w.L, callback=_make_callback(torch, means_t, logw_t, tcond_t), seed=9)
+    out, calls, rows = [x.cpu().numpy() for x in s_cb.sample_all()]
+    den, ao, co, so = oracle_setup(w, gmm=gp)
+    bad = 0
+    for b in range(12):
+        r = o.speculative_chain(den, ao, co, so, w.L, 9, b, w.d)
+        ok = r["nfe_calls"] == calls[b] and r["nfe_rows"] == rows[b] and rel_l2(out[b], r["Y"]) <= 1e-4
+        bad += (not ok)
+    assert bad <= 1
+    s_cb.close()
+
+
+def test_non_finite_target_output_freezes_only_that_chain():
+    torch = _torch()
+    w = wl.WORKLOADS["cfg2"].scaled(B=16, K=24)
+    gp = w.gmm_params()
+    a, c, sig, tcond = sds.schedule_for(w)
+    means_t, logw_t = torch.from_numpy(gp.means).cuda(), torch.from_numpy(gp.logw).cuda()
+    tcond_t = torch.from_numpy(tcond).cuda()
+    clean = sb.Sampler(a, c, sig, 16, w.d, w.L, callback=_make_callback(torch, means_t, logw_t, tcond_t), seed=4)
+    ref = clean.sample_all()[0].cpu().numpy()
+    # row 3 of the initial target call is poisoned: chain 3 starts with a NaN carried output
+    s = sb.Sampler(a, c, sig, 16, w.d, w.L, callback=_make_callback(torch, means_t, logw_t, tcond_t, poison_row=3), seed=4)
+    out_t = torch.empty((16, w.d), dtype=torch.float32, device="cuda")
+    rc = s.lib.sds_sample_all(s.h, out_t.data_ptr(), None, None)
+    assert rc == sb.SDS_ENONFINITE
+    ctl = s.get(sb.GET_CTL)
+    assert ctl[0] == 0 and ctl[4] == 1                      # nobody active, exactly one chain frozen
+    assert np.array_equal(s.get(sb.GET_N), np.full(16, w.K))
+    out = out_t.cpu().numpy()
+    # every other chain is bit-identical to the clean run
+    same = [b for b in range(16) if np.array_equal(out[b], ref[b])]
+    assert same == [b for b in range(16) if b != 3]
+    clean.close(); s.close()
+
+
+def test_failing_callback_is_reported():
+    torch = _torch()
+    w = wl.WORKLOADS["cfg1"].scaled(K=10)
+    a, c, sig, _ = sds.schedule_for(w)
+    s = sb.Sampler(a, c, sig, 8, w.d, w.L, callback=_make_callback(torch, None, None, None, fail=True), seed=1)
+    assert s.lib.sds_reset(s.h) == sb.SDS_ECALLBACK
+    s.close()
