@@ -200,6 +200,12 @@ int sds_rng_normals(uint64_t seed, int32_t stream_id, int64_t b0, int64_t nb, in
                     float* out_dev, void* cuda_stream);
 int sds_rng_uniforms(uint64_t seed, int64_t b0, int64_t nb, int32_t k, float* u_dev, void* cuda_stream);
 
+/* Self-test of the device-side bounded wait used by the tensor-core kernels (their mbarrier waits
+ * give up after a fixed number of polls and report SDS_ETIMEOUT instead of spinning): launches one
+ * thread that waits `polls` times on a barrier nobody arrives on and stores 1 in *status_dev when
+ * the wait ran out (0 would mean the barrier completed). The kernel always terminates. */
+int sds_selftest_bounded_wait(int32_t polls, int32_t* status_dev, void* cuda_stream);
+
 /* Number of kernels this context has launched since create (for launch accounting). */
 int64_t sds_launch_count(const sds_ctx* ctx);
 

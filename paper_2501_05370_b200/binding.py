@@ -54,6 +54,7 @@ EXPORTS = {
     "sds_denoise": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]),
     "sds_rng_normals": (C.c_int, [C.c_uint64, C.c_int32, C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
     "sds_rng_uniforms": (C.c_int, [C.c_uint64, C.c_int64, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p]),
+    "sds_selftest_bounded_wait": (C.c_int, [C.c_int32, C.c_void_p, C.c_void_p]),
     "sds_launch_count": (C.c_int64, [C.c_void_p]),
     "sds_set_option": (C.c_int, [C.c_void_p, C.c_int32, C.c_int64]),
     "sds_profile": (C.c_int, [C.c_void_p, C.c_int32]),

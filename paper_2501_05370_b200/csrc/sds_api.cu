@@ -672,6 +672,12 @@ int sds_rng_uniforms(uint64_t seed, int64_t b0, int64_t nb, int32_t k, float* u_
                                                                                                            : SDS_ECUDA;
 }
 
+int sds_selftest_bounded_wait(int32_t polls, int32_t* status_dev, void* cuda_stream) {
+  if (!status_dev || polls <= 0 || polls > (1 << 24)) return SDS_EINVAL;
+  return launch_wait_selftest((uint32_t)polls, status_dev, (cudaStream_t)cuda_stream) == cudaSuccess ? SDS_OK
+                                                                                                       : SDS_ECUDA;
+}
+
 int64_t sds_launch_count(const sds_ctx* c) { return c ? c->launches : 0; }
 
 int sds_set_option(sds_ctx* c, int32_t option, int64_t value) {

@@ -546,6 +546,19 @@ __global__ void __launch_bounds__(256)
   }
 }
 
+// Self-test of the bounded wait: one thread waits on an mbarrier that nobody ever arrives on. The
+// wait must give up after `polls` attempts and report it; the kernel then ends normally.
+__global__ void k_wait_selftest(uint32_t polls, int* status) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    bool done = false;
+    for (uint32_t it = 0; it < polls && !done; ++it) done = mbar_try_wait(&bar, 0u);
+    *status = done ? 0 : 1;               // 1 = the wait ran out, as it must
+  }
+}
+
 PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
   static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
   if (!fn) {
@@ -637,6 +650,11 @@ cudaError_t launch_transpose_bf16(const uint16_t* M, int ncomp, int d, uint16_t*
 
 cudaError_t launch_musq_bf16(const uint16_t* means, int ncomp, int d, double* musq, cudaStream_t st) {
   k_musq_bf16<<<(ncomp + 3) / 4, 128, 0, st>>>(means, ncomp, d, musq);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_wait_selftest(uint32_t polls, int* status_dev, cudaStream_t st) {
+  k_wait_selftest<<<1, 32, 0, st>>>(polls, status_dev);
   return cudaGetLastError();
 }
 

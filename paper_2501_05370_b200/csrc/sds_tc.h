@@ -43,6 +43,7 @@ cudaError_t launch_softmax_bf16(const float* logits, const int* nrows_dev, int r
                                 cudaStream_t st);
 cudaError_t launch_transpose_bf16(const uint16_t* M, int ncomp, int d, uint16_t* Mt, cudaStream_t st);
 cudaError_t launch_musq_bf16(const uint16_t* means, int ncomp, int d, double* musq, cudaStream_t st);
+cudaError_t launch_wait_selftest(uint32_t polls, int* status_dev, cudaStream_t st);
 cudaError_t launch_split3(const float* x, size_t n, size_t plane, uint16_t* out, cudaStream_t st);
 cudaError_t launch_softmax_split3(const float* logits, const int* nrows_dev, int rows_host, int ncomp, int d,
                                   const float* X, const float* means, const double* musq, const float* logw,

@@ -152,3 +152,15 @@ def test_full_size_tensor_core_windows_on_sampled_chains(name):
     assert np.all(calls >= 1 + -(-w.K // w.L)) and np.all(calls <= 1 + w.K)
     assert np.all(rows >= w.K + 1) and np.all(rows <= 1 + (calls - 1) * w.L)
     s.close()
+
+
+def test_bounded_wait_runs_out_and_reports():
+    """A wait on a barrier that nothing completes gives up after its poll limit and says so; the
+    context stays usable (the next kernel runs)."""
+    import torch
+    st = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    rc = sb.load().sds_selftest_bounded_wait(2000, st.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    assert rc == sb.SDS_OK
+    torch.cuda.synchronize()
+    assert int(st.item()) == 1
+    assert float((torch.ones(4, device="cuda") * 2).sum().item()) == 8.0
