@@ -59,7 +59,11 @@ extern "C" {
 #define SDS_F32           0
 #define SDS_BF16          1
 
-#define SDS_FROZEN_PREV   0     /* drafter reuses the newest target output on the accepted path (no extra call) */
+#define SDS_FROZEN_PREV   0     /* drafter reuses the newest target output on the accepted path (no extra call;
+                                   the fallback the "efficient frozen draft strategy" paragraph offers, used always) */
+#define SDS_FROZEN_EXACT  1     /* main-text frozen drafter (Eq. 6): sds_draft first evaluates the target at
+                                   (Y_n, t_n) for every active chain; that output is also row 1 of the batch,
+                                   so position 1 always accepts. Two sequential target calls per window. */
 
 #define SDS_GET_X         1     /* float  [nrows, d]  drafted states fed to the target (row r = rowoff[s]+j-1) */
 #define SDS_GET_TAIL      2     /* float  [B, d]      last drafted state of each chain's window */

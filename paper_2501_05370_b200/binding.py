@@ -21,7 +21,7 @@ SDS_EINVAL, SDS_ESTATE, SDS_ENOMEM, SDS_EUNSUPPORTED = -1, -2, -3, -4
 SDS_ECUDA, SDS_ETIMEOUT, SDS_ENONFINITE, SDS_ECALLBACK = -5, -6, -7, -8
 SDS_DEN_GMM, SDS_DEN_MLP, SDS_DEN_CALLBACK = 1, 2, 3
 SDS_F32, SDS_BF16 = 0, 1
-SDS_FROZEN_PREV = 0
+SDS_FROZEN_PREV, SDS_FROZEN_EXACT = 0, 1
 (GET_X, GET_TAIL, GET_DQ, GET_DC, GET_Y, GET_N, GET_ACT, GET_ROWOFF, GET_S1, GET_S2, GET_ELL, GET_LOGU,
  GET_ACCMASK, GET_JSTAR, GET_NFE_CALLS, GET_NFE_ROWS, GET_CTL, GET_ROWK) = range(1, 19)
 
@@ -150,7 +150,7 @@ class Sampler:
 
     def __init__(self, a, c, sigma, B: int, d: int, L: int, *, gmm_means=None, gmm_logw=None, tcond=None,
                  gmm_bf16: bool = False, mlp=None, callback=None, seed: int = 0, chain_id_offset: int = 0,
-                 device="cuda:0", stream=None):
+                 drafter_mode: int = 0, device="cuda:0", stream=None):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("libsds needs a CUDA device; there is no CPU path")
@@ -215,7 +215,7 @@ class Sampler:
         h = C.c_void_p()
         self._chk(self.lib.sds_create(C.byref(sch), C.byref(den), self.B, self.d, self.L, C.byref(h)), "sds_create")
         self.h = h
-        self._chk(self.lib.sds_bind(self.h, base, nbytes.value, self.stream.cuda_stream, seed, SDS_FROZEN_PREV,
+        self._chk(self.lib.sds_bind(self.h, base, nbytes.value, self.stream.cuda_stream, seed, drafter_mode,
                                     chain_id_offset), "sds_bind")
 
     # -- helpers --

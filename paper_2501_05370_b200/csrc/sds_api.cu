@@ -191,6 +191,7 @@ T* at(sds_ctx* c, size_t off) { return off == kNone ? nullptr : reinterpret_cast
 WinArgs win_args(sds_ctx* c) {
   WinArgs A{};
   A.B = (int)c->B; A.d = c->d; A.L = c->L; A.K = c->K;
+  A.exact = c->mode == SDS_FROZEN_EXACT ? 1 : 0;
   A.seed = c->seed; A.chain_off = (uint64_t)c->chain_off;
   A.a = at<float>(c, c->lay.a); A.c = at<float>(c, c->lay.c); A.sigma = at<float>(c, c->lay.sigma);
   A.Y = at<float>(c, c->lay.Y); A.Dc = at<float>(c, c->lay.Dc); A.T = at<float>(c, c->lay.T);
@@ -469,7 +470,7 @@ int sds_create(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int3
 int sds_bind(sds_ctx* c, void* workspace_dev, size_t bytes, void* cuda_stream, uint64_t seed, int32_t drafter_mode,
              int64_t chain_id_offset) {
   if (!c || !workspace_dev) return SDS_EINVAL;
-  if (drafter_mode != SDS_FROZEN_PREV) return SDS_EUNSUPPORTED;
+  if (drafter_mode != SDS_FROZEN_PREV && drafter_mode != SDS_FROZEN_EXACT) return SDS_EUNSUPPORTED;
   if (chain_id_offset < 0) return SDS_EINVAL;
   if (bytes < c->lay.total || (reinterpret_cast<uintptr_t>(workspace_dev) % kAlign) != 0) return SDS_ENOMEM;
   c->ws = static_cast<char*>(workspace_dev);
@@ -497,9 +498,11 @@ int sds_reset(sds_ctx* c) {
   if (c->state < kBound) return SDS_ESTATE;
   WinArgs A = win_args(c);
   SDS_LAUNCH(c, SDS_PROF_INIT, launch_init(A, c->stream));
-  const int rc = run_denoiser(c, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, c->B, A.Dq);
-  if (rc != SDS_OK) return rc;
-  SDS_LAUNCH(c, SDS_PROF_AUX, launch_after_init(A, c->stream));
+  if (c->mode == SDS_FROZEN_PREV) {
+    const int rc = run_denoiser(c, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, c->B, A.Dq);
+    if (rc != SDS_OK) return rc;
+    SDS_LAUNCH(c, SDS_PROF_AUX, launch_after_init(A, c->stream));
+  }
   SDS_LAUNCH(c, SDS_PROF_AUX, launch_compact(A, c->stream));
   c->ub = (int)c->B;
   c->state = kReady;
@@ -509,7 +512,15 @@ int sds_reset(sds_ctx* c) {
 int sds_draft(sds_ctx* c) {
   if (!c) return SDS_EINVAL;
   if (c->state != kReady) return SDS_ESTATE;
-  SDS_LAUNCH(c, SDS_PROF_DRAFT, launch_draft(win_args(c), c->ub, c->stream));
+  WinArgs A = win_args(c);
+  if (c->mode == SDS_FROZEN_EXACT) {
+    // frozen output = target output at (Y_n, t_n): one row per active chain
+    SDS_LAUNCH(c, SDS_PROF_DRAFT, launch_gather_state(A, c->ub, c->stream));
+    const int rc = run_denoiser(c, A.X, A.Xb, A.rowk, A.ctl + kCtlNActive, c->ub, A.Dq);
+    if (rc != SDS_OK) return rc;
+    SDS_LAUNCH(c, SDS_PROF_DRAFT, launch_scatter_carried(A, c->ub, c->stream));
+  }
+  SDS_LAUNCH(c, SDS_PROF_DRAFT, launch_draft(A, c->ub, c->stream));
   c->state = kDrafted;
   return SDS_OK;
 }
@@ -539,7 +550,7 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
   if (c->state < kBound) return SDS_ESTATE;
   WinArgs A = win_args(c);
   int rc = SDS_OK;
-  if (c->whole_chain && c->den.kind == SDS_DEN_GMM && fused_small_supported(c->d, c->den.ncomp, c->L)) {
+  if (c->whole_chain && c->mode == SDS_FROZEN_PREV && c->den.kind == SDS_DEN_GMM && fused_small_supported(c->d, c->den.ncomp, c->L)) {
     if ((rc = ensure_musq(c)) != SDS_OK) return rc;
     SDS_CU(c, cudaMemsetAsync(A.ctl, 0, kCtlWords * 4, c->stream));   // no chain active afterwards, error bits clear
     SDS_LAUNCH(c, SDS_PROF_FUSED, launch_fused_small(A, gmm_args(c), c->stream));

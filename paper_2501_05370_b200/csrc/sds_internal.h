@@ -10,6 +10,7 @@ namespace sds {
 // caller's workspace (or the caller's parameter arrays).
 struct WinArgs {
   int B, d, L, K;
+  int exact;             // 1: the drafter's frozen output is recomputed at Y_n before every window
   uint64_t seed;
   uint64_t chain_off;
   const float* a;        // [K]
@@ -48,6 +49,8 @@ struct GmmArgs {
 cudaError_t launch_init(const WinArgs& A, cudaStream_t st);
 cudaError_t launch_after_init(const WinArgs& A, cudaStream_t st);
 cudaError_t launch_compact(const WinArgs& A, cudaStream_t st);
+cudaError_t launch_gather_state(const WinArgs& A, int ub_chains, cudaStream_t st);
+cudaError_t launch_scatter_carried(const WinArgs& A, int ub_chains, cudaStream_t st);
 cudaError_t launch_draft(const WinArgs& A, int ub_chains, cudaStream_t st);
 cudaError_t launch_verify(const WinArgs& A, int ub_chains, cudaStream_t st);
 cudaError_t launch_advance(const WinArgs& A, int ub_chains, cudaStream_t st);

@@ -105,8 +105,8 @@ __global__ void __launch_bounds__(kBlock) k_init(WinArgs A) {
   if (t == 0) {
     A.n[b] = 0;
     A.rowk[b] = 0;
-    A.nfe_calls[b] = 1;
-    A.nfe_rows[b] = 1;
+    A.nfe_calls[b] = A.exact ? 0 : 1;      // the carried-output drafter starts with one target call
+    A.nfe_rows[b] = A.exact ? 0 : 1;
     A.accmask[b] = 0u;
     A.jstar[b] = 0;
   }
@@ -117,6 +117,48 @@ __global__ void __launch_bounds__(kBlock) k_after_init(WinArgs A) {
   const size_t total = (size_t)A.B * A.d;
   for (size_t i = (size_t)blockIdx.x * kBlock + threadIdx.x; i < total; i += (size_t)gridDim.x * kBlock)
     A.Dc[i] = A.Dq[i];
+}
+
+// ---------------------------------------------------------------------------------------
+// Main-text frozen drafter (Eq. 6): the frozen output is the target's output at (Y_n, t_n). Before
+// drafting, the states of the active chains are gathered into dense rows, the target runs on
+// them, and the result is scattered into the carried-output array.
+// ---------------------------------------------------------------------------------------
+template <int TPC, int VEC>
+__global__ void __launch_bounds__(kBlock) k_gather_state(WinArgs A) {
+  using G = Group<TPC>;
+  const int s = G::slot(), t = G::lane();
+  if (s >= A.ctl[kCtlNActive]) return;
+  const int b = A.act[s];
+  const size_t cb = (size_t)b * A.d, ro = (size_t)s * A.d;
+  if (t == 0) A.rowk[s] = A.n[b];
+  if (VEC == 4) {
+    for (int i = t * 4; i < A.d; i += TPC * 4) {
+      const float4 y = ld4(A.Y + cb + i);
+      st4(A.X + ro + i, y);
+      if (A.Xb) *reinterpret_cast<uint2*>(A.Xb + ro + i) = make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
+    }
+  } else {
+    for (int i = t; i < A.d; i += TPC) {
+      const float y = A.Y[cb + i];
+      A.X[ro + i] = y;
+      if (A.Xb) A.Xb[ro + i] = (uint16_t)(pack_bf16x2(y, 0.f) & 0xffffu);
+    }
+  }
+}
+
+template <int TPC, int VEC>
+__global__ void __launch_bounds__(kBlock) k_scatter_carried(WinArgs A) {
+  using G = Group<TPC>;
+  const int s = G::slot(), t = G::lane();
+  if (s >= A.ctl[kCtlNActive]) return;
+  const int b = A.act[s];
+  const size_t cb = (size_t)b * A.d, ro = (size_t)s * A.d;
+  if (VEC == 4) {
+    for (int i = t * 4; i < A.d; i += TPC * 4) st4(A.Dc + cb + i, ld4(A.Dq + ro + i));
+  } else {
+    for (int i = t; i < A.d; i += TPC) A.Dc[cb + i] = A.Dq[ro + i];
+  }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -484,7 +526,9 @@ __global__ void __launch_bounds__(kBlock) k_advance(WinArgs A) {
       }
       if (t == 0) {
         A.n[b] = nb + adv;
-        A.nfe_calls[b] += 1;
+        // sequential target calls of this window: the batched pass, plus (main-text drafter) the
+        // call at Y_n, which is row 1 of the batch (a window of one row is a single call)
+        A.nfe_calls[b] += (A.exact && Lt > 1) ? 2 : 1;
         A.nfe_rows[b] += Lt;
       }
     } else if (t == 0) {                              // non-finite log ratio: stop this chain
@@ -557,6 +601,14 @@ cudaError_t launch_after_init(const WinArgs& A, cudaStream_t st) {
 }
 cudaError_t launch_compact(const WinArgs& A, cudaStream_t st) {
   k_compact<<<1, kBlock, 0, st>>>(A);
+  return cudaGetLastError();
+}
+cudaError_t launch_gather_state(const WinArgs& A, int ub, cudaStream_t st) {
+  SDS_DISPATCH(k_gather_state, A, ub, st);
+  return cudaGetLastError();
+}
+cudaError_t launch_scatter_carried(const WinArgs& A, int ub, cudaStream_t st) {
+  SDS_DISPATCH(k_scatter_carried, A, ub, st);
   return cudaGetLastError();
 }
 cudaError_t launch_draft(const WinArgs& A, int ub, cudaStream_t st) {

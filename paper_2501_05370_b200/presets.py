@@ -19,7 +19,7 @@ def schedule_for(w):
     return a, c, sigma, tcond
 
 
-def sampler_for(w, *, seed=None, chain_id_offset=0, B=None, device="cuda:0", gmm=None, mlp=None):
+def sampler_for(w, *, seed=None, chain_id_offset=0, B=None, device="cuda:0", gmm=None, mlp=None, drafter_mode=0):
     a, c, sigma, tcond = schedule_for(w)
     seed = w.sample_seed if seed is None else seed
     B = w.B if B is None else B
@@ -27,8 +27,8 @@ def sampler_for(w, *, seed=None, chain_id_offset=0, B=None, device="cuda:0", gmm
         gp = gmm if gmm is not None else w.gmm_params()
         return sb.Sampler(a, c, sigma, B, w.d, w.L, gmm_means=gp.means, gmm_logw=gp.logw, tcond=tcond,
                           gmm_bf16=bool(getattr(gp, "means_bf16", False)), seed=seed,
-                          chain_id_offset=chain_id_offset, device=device)
+                          chain_id_offset=chain_id_offset, drafter_mode=drafter_mode, device=device)
     if w.denoiser == "mlp":
         mp = mlp if mlp is not None else w.mlp_params()
-        return sb.Sampler(a, c, sigma, B, w.d, w.L, mlp=mp, seed=seed, chain_id_offset=chain_id_offset, device=device)
+        return sb.Sampler(a, c, sigma, B, w.d, w.L, mlp=mp, seed=seed, chain_id_offset=chain_id_offset, drafter_mode=drafter_mode, device=device)
     raise NotImplementedError(w.denoiser)

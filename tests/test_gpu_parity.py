@@ -460,3 +460,39 @@ def test_failing_callback_is_reported():
     s = sb.Sampler(a, c, sig, 8, w.d, w.L, callback=_make_callback(torch, None, None, None, fail=True), seed=1)
     assert s.lib.sds_reset(s.h) == sb.SDS_ECALLBACK
     s.close()
+
+
+# ------------------------------------------------------------------ main-text frozen drafter ---
+
+def test_exact_frozen_drafter_matches_oracle():
+    w = wl.WORKLOADS["cfg2"].scaled(B=48, K=40)
+    gp = w.gmm_params()
+    s = sds.sampler_for(w, gmm=gp, seed=13, drafter_mode=sb.SDS_FROZEN_EXACT)
+    # one window by hand: position 1 compares the frozen output with itself and always accepts
+    s.reset()
+    s.draft(); s.verify_window()
+    assert np.all(s.get(sb.GET_ACCMASK) & 1 == 1)
+    assert np.all(s.get(sb.GET_S1)[:, 0] == 0.0)
+    s.advance()
+    out, calls, rows = [x.cpu().numpy() for x in s.sample_all()]
+    den, a, c, sig = oracle_setup(w, gmm=gp)
+    bad = 0
+    for b in range(16):
+        r = o.speculative_chain(den, a, c, sig, w.L, 13, b, w.d, mode=o.FROZEN_EXACT)
+        ok = r["nfe_calls"] == calls[b] and r["nfe_rows"] == rows[b] and rel_l2(out[b], r["Y"]) <= 1e-4
+        bad += (not ok)
+    assert bad <= 1
+    s.close()
+
+
+def test_exact_frozen_drafter_with_window_one_is_the_plain_chain():
+    w = wl.WORKLOADS["cfg2"].scaled(B=8, K=25, L=1)
+    gp = w.gmm_params()
+    s = sds.sampler_for(w, gmm=gp, seed=17, drafter_mode=sb.SDS_FROZEN_EXACT)
+    out, calls, rows = [x.cpu().numpy() for x in s.sample_all()]
+    den, a, c, sig = oracle_setup(w, gmm=gp)
+    assert np.all(calls == 25) and np.all(rows == 25)
+    for b in range(8):
+        y = o.plain_chain(den, a, c, sig, seed=17, b=b, d=w.d)
+        assert rel_l2(out[b], y) <= 1e-4
+    s.close()
