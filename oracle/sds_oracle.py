@@ -11,6 +11,7 @@ What each function follows:
                                        (Eq. 3 target transition; Langevin Eq. 13)
   gmm_posterior_mean, gmm_grad_energy  exact denoiser / score of a Gaussian mixture (Tweedie)
   mlp_forward                          bf16-operand MLP denoiser
+  phi4_energy, phi4_grad_energy        the lattice energy of the Langevin experiment (Appendix K)
   rejection_discrete                   Algorithm 2 (generic maximal coupling), finite space
   rejection_reflection                 Algorithm 3 (reflection maximal coupling)
   rejection_incorrect                  the biased rule of Appendix "need for adjusted rejection"
@@ -201,6 +202,40 @@ def gmm_grad_energy(x, means, logw, s):
     logit = np.asarray(logw, dtype=np.float64) - 0.5 * np.sum(diff * diff, axis=1) / (s * s)
     r = _log_softmax_weights(logit)
     return (r @ diff) / (s * s)
+
+
+def phi4_energy(x, side, beta, periodic=False):
+    """E(x) = beta/2 sum_{|i-j|=1} (x_i - x_j)^2 + sum_i (x_i^2 - 1)^2 on a side x side grid
+    (Appendix K; each neighbouring pair counted once; free boundaries unless periodic)."""
+    g = np.asarray(x, dtype=np.float64).reshape(side, side)
+    e = np.sum((g * g - 1.0) ** 2)
+    for axis in (0, 1):
+        if periodic:
+            dif = g - np.roll(g, -1, axis=axis)
+        else:
+            dif = np.diff(g, axis=axis)
+        e += 0.5 * beta * np.sum(dif * dif)
+    return float(e)
+
+
+def phi4_grad_energy(x, side, beta, periodic=False):
+    """Gradient of phi4_energy: beta * sum over neighbours (x_i - x_j) + 4 x_i (x_i^2 - 1)."""
+    g = np.asarray(x, dtype=np.float64).reshape(side, side)
+    grad = 4.0 * g * (g * g - 1.0)
+    for axis in (0, 1):
+        if periodic:
+            grad += beta * (2.0 * g - np.roll(g, 1, axis=axis) - np.roll(g, -1, axis=axis))
+        else:
+            fwd = np.zeros_like(g)
+            bwd = np.zeros_like(g)
+            sl_a = [slice(None)] * 2
+            sl_b = [slice(None)] * 2
+            sl_a[axis] = slice(0, -1)
+            sl_b[axis] = slice(1, None)
+            fwd[tuple(sl_a)] = g[tuple(sl_a)] - g[tuple(sl_b)]      # pair (i, i+1) seen from i
+            bwd[tuple(sl_b)] = g[tuple(sl_b)] - g[tuple(sl_a)]      # same pair seen from i+1
+            grad += beta * (fwd + bwd)
+    return grad.reshape(-1)
 
 
 def silu(x):

@@ -465,3 +465,39 @@ def test_ula_affine():
     x = np.array([1.0, 2.0])
     m_p, m_q = a[0] * x + c[0] * gh, a[0] * x + c[0] * g
     assert np.allclose((m_p - m_q) / s[0], math.sqrt(1e-3 / 2) * (g - gh))
+
+
+# ------------------------------------------------------------------ phi^4 Langevin experiment ----
+
+def test_phi4_gradient_is_the_gradient_of_the_energy():
+    rng = np.random.default_rng(21)
+    for periodic in (False, True):
+        x = rng.standard_normal(36)
+        h = 1e-6
+        fd = np.array([(o.phi4_energy(x + h * np.eye(36)[i], 6, 7.5, periodic)
+                        - o.phi4_energy(x - h * np.eye(36)[i], 6, 7.5, periodic)) / (2 * h) for i in range(36)])
+        assert np.allclose(o.phi4_grad_energy(x, 6, 7.5, periodic), fd, rtol=1e-6, atol=1e-6)
+    # a constant field at a minimum of the site potential has zero energy and zero gradient
+    assert o.phi4_energy(np.ones(64), 8, 100.0) == 0.0
+    assert np.all(o.phi4_grad_energy(-np.ones(64), 8, 100.0) == 0.0)
+    # 2x1 lattice by hand: E = beta/2 (a-b)^2 + (a^2-1)^2 + (b^2-1)^2 on the pair, second row independent
+    x = np.array([0.5, -0.25, 0.0, 0.0])
+    e_pairs = 0.5 * 3.0 * ((0.5 + 0.25) ** 2 + 0.5 ** 2 + 0.25 ** 2 + 0.0)
+    e_site = (0.25 - 1) ** 2 + (0.0625 - 1) ** 2 + 2.0
+    assert abs(o.phi4_energy(x, 2, 3.0) - (e_pairs + e_site)) < 1e-12
+
+
+def test_phi4_speculative_langevin_reproduces_the_papers_nfe():
+    """The one experiment with printed numbers that needs no data: 100000 Langevin steps cost 48564
+    target calls with window 20 and the frozen drafter (Appendix K). With the target evaluated at
+    Y_n before drafting and one call counted per window, windows per step must come out at 0.4856."""
+    g = GOLD["phi4_table"]
+    K = 7000
+    a, c, sig = o.ula_affine(K, g["gamma"])
+    den = lambda x, k: o.phi4_grad_energy(x, g["side"], g["beta"])
+    ratios = []
+    for b in range(2):
+        r = o.speculative_chain(den, a, c, sig, g["window"], 5, b, g["side"] ** 2, mode=o.FROZEN_EXACT)
+        ratios.append(len(r["adv"]) / K)
+        assert 2 * len(r["adv"]) - 1 <= r["nfe_calls"] <= 2 * len(r["adv"])   # the oracle counts both sequential calls
+    assert abs(np.mean(ratios) - g["nfe_per_step"]) < 0.012, ratios
