@@ -54,7 +54,10 @@ def oracle_closure(w):
         a, c, sig, abar = o.ddpm_affine(w.beta())
     else:
         a, c, sig = o.ula_affine(w.K, w.ula_gamma)
-    if w.denoiser == "mlp":
+    if w.denoiser == "phi4":
+        p4 = w.phi4
+        den = lambda x, k: o.phi4_grad_energy(x, p4["side"], p4["beta"], p4.get("periodic", False))
+    elif w.denoiser == "mlp":
         mp = w.mlp_params()
         W = [wl.bf16_bits_to_f32(x).astype(np.float64) for x in mp.weights]
         T = [wl.bf16_bits_to_f32(x).astype(np.float64) if x is not None else None for x in mp.temb]
@@ -81,7 +84,8 @@ def oracle_time(w, budget_s: float, min_chains: int = 1, first_chain: int = 0):
     prefix = False
     while True:
         t1 = time.perf_counter()
-        o.speculative_chain(den, a[:Kp], c[:Kp], sig[:Kp], w.L, w.sample_seed, first_chain + n, w.d)
+        o.speculative_chain(den, a[:Kp], c[:Kp], sig[:Kp], w.L, w.sample_seed, first_chain + n, w.d,
+                            mode=getattr(w, "drafter_mode", 0))
         dt = time.perf_counter() - t1
         n += 1
         steps += Kp
@@ -127,7 +131,8 @@ def workload_config(w, args):
     return {"workload": f"{w.name}: B={w.B} chains/GPU, d={w.d}, L={w.L}, K={w.K}, {w.sampler} "
                         f"{w.schedule or 'gamma=%g' % w.ula_gamma}, {w.denoiser} denoiser"
                         + (f" ncomp={w.gmm['ncomp']}" if w.denoiser == 'gmm' else ""),
-            "drafter": "frozen target output (carried)", "seed": w.sample_seed,
+            "drafter": "frozen target output " + ("evaluated at Y_n" if getattr(w, "drafter_mode", 0) else "(carried)"),
+            "seed": w.sample_seed,
             "l2": "256 MiB buffer written between timed steps (working set may fit L2)",
             "sharding": "chains by global id, no data-path collective"}
 
@@ -209,6 +214,8 @@ def algorithmic(kind: str, w, rows_per_step: float, windows_chains: float, launc
     if kind == "advance":
         return "hbm", 16.0 * d * windows_chains / launches
     if kind in ("denoise", "fused"):
+        if w.denoiser == "phi4":    # four neighbour differences, the site term, one fma per site
+            return "alu", 12.0 * d * (rows_per_step + w.B) / launches
         if w.denoiser == "mlp":     # 2 * sum of layer products per row, bf16 tensor cores
             per_row = 2.0 * sum(w.mlp_dims[i] * w.mlp_dims[i + 1] for i in range(len(w.mlp_dims) - 1))
             return "tensor", per_row * (rows_per_step + w.B) / launches

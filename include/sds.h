@@ -55,6 +55,7 @@ extern "C" {
 #define SDS_DEN_GMM       1     /* closed-form Gaussian-mixture posterior mean / energy gradient */
 #define SDS_DEN_MLP       2     /* bf16 MLP with per-step embedding rows */
 #define SDS_DEN_CALLBACK  3     /* user function on device buffers */
+#define SDS_DEN_PHI4      4     /* energy gradient of the phi^4 lattice model (Langevin chains, Appendix K) */
 
 #define SDS_F32           0
 #define SDS_BF16          1
@@ -115,7 +116,10 @@ typedef int (*sds_denoise_fn)(void* user, const float* x_dev, const int32_t* k_d
  * MLP: nlayer linear layers dims[0]=d -> ... -> dims[nlayer]=d.
  *   h_l = SiLU(W_l h_{l-1} + bias_l + temb_l[k]) for l < nlayer, output = W_nlayer h + bias (float).
  *   W_dev[l]: [dims[l+1], dims[l]] bf16 row-major; bias_dev[l]: [dims[l+1]] float;
- *   temb_dev[l]: [K, dims[l+1]] bf16 (NULL for the last layer). Every dims[] a multiple of 128. */
+ *   temb_dev[l]: [K, dims[l+1]] bf16 (NULL for the last layer). Every dims[] a multiple of 128.
+ * PHI4: D(x) = grad E(x), E(x) = coupling/2 sum_{|i-j|=1} (x_i - x_j)^2 + sum_i (x_i^2 - 1)^2 on a
+ *   grid_side x grid_side lattice (d = grid_side^2), every neighbouring pair once, free boundaries
+ *   unless periodic != 0. Used with the Langevin schedule a = 1, c = -gamma, sigma = sqrt(2 gamma). */
 typedef struct {
   int32_t kind;
   int32_t ncomp;
@@ -129,6 +133,9 @@ typedef struct {
   const int32_t* dims;
   sds_denoise_fn fn;
   void* user;
+  int32_t grid_side;
+  float coupling;
+  int32_t periodic;
 } sds_denoiser;
 
 /* Bytes of device workspace sds_bind needs for this problem (256-byte aligned base required). */

@@ -19,7 +19,7 @@ from . import build as _build
 SDS_OK = 0
 SDS_EINVAL, SDS_ESTATE, SDS_ENOMEM, SDS_EUNSUPPORTED = -1, -2, -3, -4
 SDS_ECUDA, SDS_ETIMEOUT, SDS_ENONFINITE, SDS_ECALLBACK = -5, -6, -7, -8
-SDS_DEN_GMM, SDS_DEN_MLP, SDS_DEN_CALLBACK = 1, 2, 3
+SDS_DEN_GMM, SDS_DEN_MLP, SDS_DEN_CALLBACK, SDS_DEN_PHI4 = 1, 2, 3, 4
 SDS_F32, SDS_BF16 = 0, 1
 SDS_FROZEN_PREV, SDS_FROZEN_EXACT = 0, 1
 (GET_X, GET_TAIL, GET_DQ, GET_DC, GET_Y, GET_N, GET_ACT, GET_ROWOFF, GET_S1, GET_S2, GET_ELL, GET_LOGU,
@@ -36,7 +36,8 @@ class SdsSchedule(C.Structure):
 class SdsDenoiser(C.Structure):
     _fields_ = [("kind", C.c_int32), ("ncomp", C.c_int32), ("means_dev", C.c_void_p), ("logw_dev", C.c_void_p),
                 ("means_dtype", C.c_int32), ("nlayer", C.c_int32), ("W_dev", C.c_void_p), ("bias_dev", C.c_void_p),
-                ("temb_dev", C.c_void_p), ("dims", C.c_void_p), ("fn", DENOISE_FN), ("user", C.c_void_p)]
+                ("temb_dev", C.c_void_p), ("dims", C.c_void_p), ("fn", DENOISE_FN), ("user", C.c_void_p),
+                ("grid_side", C.c_int32), ("coupling", C.c_float), ("periodic", C.c_int32)]
 
 
 EXPORTS = {
@@ -149,7 +150,7 @@ class Sampler:
     """
 
     def __init__(self, a, c, sigma, B: int, d: int, L: int, *, gmm_means=None, gmm_logw=None, tcond=None,
-                 gmm_bf16: bool = False, mlp=None, callback=None, seed: int = 0, chain_id_offset: int = 0,
+                 gmm_bf16: bool = False, mlp=None, callback=None, phi4=None, seed: int = 0, chain_id_offset: int = 0,
                  drafter_mode: int = 0, device="cuda:0", stream=None):
         import torch
         if not torch.cuda.is_available():
@@ -199,6 +200,8 @@ class Sampler:
             den.bias_dev = C.cast(self._mlp_bp, C.c_void_p)
             den.temb_dev = C.cast(self._mlp_tp, C.c_void_p)
             den.dims = self._mlp_dims.ctypes.data
+        elif phi4 is not None:                   # (grid side, coupling beta, periodic)
+            den.kind, den.grid_side, den.coupling, den.periodic = SDS_DEN_PHI4, int(phi4[0]), float(phi4[1]), int(bool(phi4[2]))
         elif callback is not None:
             self._cb = DENOISE_FN(callback)
             den.kind, den.fn = SDS_DEN_CALLBACK, self._cb

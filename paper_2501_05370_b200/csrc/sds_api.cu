@@ -168,6 +168,10 @@ int validate(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_
     case SDS_DEN_CALLBACK:
       if (!den->fn) return SDS_EINVAL;
       break;
+    case SDS_DEN_PHI4:
+      if (den->grid_side < 2 || (int64_t)den->grid_side * den->grid_side != d) return SDS_EINVAL;
+      if (!std::isfinite(den->coupling)) return SDS_EINVAL;
+      break;
     case SDS_DEN_MLP:
       if (den->nlayer < 1 || den->nlayer > 16 || !den->dims || !den->W_dev || !den->bias_dev || !den->temb_dev)
         return SDS_EINVAL;
@@ -385,6 +389,10 @@ int run_denoiser(sds_ctx* c, const float* X, const uint16_t* Xb, const int* rowk
       }
       return SDS_OK;
     }
+    case SDS_DEN_PHI4:
+      SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_phi4_grad(X, nrows_dev, (int)rows_ub, c->den.grid_side, c->den.coupling,
+                                                        c->den.periodic, out, c->stream));
+      return SDS_OK;
     case SDS_DEN_CALLBACK: {
       int32_t rows = (int32_t)rows_ub;         // the callback needs the row count on the host
       if (nrows_dev) {

@@ -63,6 +63,10 @@ cudaError_t launch_musq(const float* means, int ncomp, int d, double* musq, cuda
 cudaError_t launch_gmm_f32(const GmmArgs& G, const float* X, const int* rowk, const int* nrows_dev, int rows_ub,
                            float* out, cudaStream_t st);
 
+// lattice energy gradient (sds_phi4.cu)
+cudaError_t launch_phi4_grad(const float* X, const int* nrows_dev, int rows_ub, int side, float beta, int periodic,
+                             float* out, cudaStream_t st);
+
 // whole-chain persistent kernel for small mixtures (sds_fused.cu)
 bool fused_small_supported(int d, int ncomp, int L);
 cudaError_t launch_fused_small(const WinArgs& A, const GmmArgs& G, cudaStream_t st);

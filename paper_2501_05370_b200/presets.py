@@ -19,8 +19,10 @@ def schedule_for(w):
     return a, c, sigma, tcond
 
 
-def sampler_for(w, *, seed=None, chain_id_offset=0, B=None, device="cuda:0", gmm=None, mlp=None, drafter_mode=0):
+def sampler_for(w, *, seed=None, chain_id_offset=0, B=None, device="cuda:0", gmm=None, mlp=None, drafter_mode=None):
     a, c, sigma, tcond = schedule_for(w)
+    if drafter_mode is None:
+        drafter_mode = getattr(w, "drafter_mode", 0)
     seed = w.sample_seed if seed is None else seed
     B = w.B if B is None else B
     if w.denoiser == "gmm":
@@ -31,4 +33,8 @@ def sampler_for(w, *, seed=None, chain_id_offset=0, B=None, device="cuda:0", gmm
     if w.denoiser == "mlp":
         mp = mlp if mlp is not None else w.mlp_params()
         return sb.Sampler(a, c, sigma, B, w.d, w.L, mlp=mp, seed=seed, chain_id_offset=chain_id_offset, drafter_mode=drafter_mode, device=device)
+    if w.denoiser == "phi4":
+        p4 = w.phi4
+        return sb.Sampler(a, c, sigma, B, w.d, w.L, phi4=(p4["side"], p4["beta"], p4.get("periodic", False)), seed=seed,
+                          chain_id_offset=chain_id_offset, drafter_mode=drafter_mode, device=device)
     raise NotImplementedError(w.denoiser)

@@ -20,6 +20,9 @@ def oracle_setup(w, gmm=None, mlp=None):
                                                     bf16_operands=gp.means_bf16)
         else:
             den = lambda x, k: o.gmm_grad_energy(x, gp.means, gp.logw, gp.comp_std)
+    elif w.denoiser == "phi4":
+        p4 = w.phi4
+        den = lambda x, k: o.phi4_grad_energy(x, p4["side"], p4["beta"], p4.get("periodic", False))
     else:
         import workloads as wl
         mp = mlp if mlp is not None else w.mlp_params()

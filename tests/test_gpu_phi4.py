@@ -1,0 +1,68 @@
+"""GPU parity and the paper's printed figure for the phi^4 Langevin workload (Appendix K)."""
+import json
+import os
+
+import numpy as np
+import pytest
+
+import paper_2501_05370_b200 as sds
+from paper_2501_05370_b200 import binding as sb
+from oracle import sds_oracle as o
+import workloads as wl
+from helpers import oracle_setup, rel_l2
+from test_gpu_parity import _window_check
+
+pytestmark = pytest.mark.gpu
+GOLD = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "worked_examples.json")))
+
+
+@pytest.mark.parametrize("side,beta,periodic,rows", [(8, 100.0, False, 300), (5, 7.5, True, 77), (2, 3.0, False, 9),
+                                                     (16, 40.0, False, 50)])
+def test_phi4_gradient_rows(side, beta, periodic, rows):
+    import torch
+    w = wl.WORKLOADS["phi4"].scaled(d=side * side, B=rows, L=1, K=4, phi4=dict(side=side, beta=beta, periodic=periodic))
+    s = sds.sampler_for(w)
+    rng = np.random.default_rng(side)
+    x = (1.0 + 0.3 * rng.standard_normal((rows, side * side))).astype(np.float32)
+    k = np.zeros(rows, np.int32)
+    out = s.denoise(torch.from_numpy(x).cuda(), torch.from_numpy(k).cuda()).cpu().numpy()
+    for r in range(rows):
+        assert rel_l2(out[r], o.phi4_grad_energy(x[r].astype(np.float64), side, beta, periodic)) <= 1e-5
+    s.close()
+
+
+def test_phi4_windows_and_free_run_against_oracle():
+    w = wl.WORKLOADS["phi4"].scaled(B=24, K=600)
+    s = sds.sampler_for(w, seed=3)
+    den, a, c, sig = oracle_setup(w)
+    a32, c32, s32, _ = sds.schedule_for(w)
+    s.reset()
+    stats = dict(tests=0, band=0, reflected=0)
+    for _ in range(3):
+        _window_check(s, w, den, a32, c32, s32, 3, 0, stats)
+    assert stats["band"] <= 2 and stats["reflected"] > 0
+    out, calls, rows = [x.cpu().numpy() for x in s.sample_all()]
+    diverged = 0
+    for b in range(8):
+        r = o.speculative_chain(den, a, c, sig, w.L, 3, b, w.d, mode=o.FROZEN_EXACT)
+        same = r["nfe_calls"] == calls[b] and r["nfe_rows"] == rows[b] and rel_l2(out[b], r["Y"]) <= 1e-4
+        diverged += (not same)
+    assert diverged <= 1
+    s.close()
+
+
+def test_phi4_full_run_reproduces_the_papers_nfe():
+    """500 chains x 100000 Langevin steps, window 20: the paper reports 48564 target calls per
+    100000 steps. One call per window is what it counts, i.e. windows per step = 0.4856."""
+    g = GOLD["phi4_table"]
+    w = wl.WORKLOADS["phi4"]
+    assert (w.K, w.L, w.phi4["side"], w.phi4["beta"], w.ula_gamma) == (g["steps"], g["window"], g["side"], g["beta"], g["gamma"])
+    s = sds.sampler_for(w)
+    out, calls, rows = [x.cpu().numpy().astype(np.float64) for x in s.sample_all()]
+    assert np.all(np.isfinite(out)) and np.array_equal(s.get(sb.GET_N), np.full(w.B, w.K))
+    windows_per_step = (calls / 2.0).mean() / w.K           # two sequential calls per window in this mode
+    assert abs(windows_per_step - g["nfe_per_step"]) < 0.004, windows_per_step
+    energies = np.array([o.phi4_energy(x, g["side"], g["beta"]) for x in out])
+    print(f"windows per step {windows_per_step:.5f} (paper {g['nfe_per_step']}), "
+          f"final energy {energies.mean():.2f} +- {energies.std():.2f}")
+    s.close()

@@ -146,6 +146,8 @@ class Workload:
     denoiser: str = "gmm"       # "gmm" | "mlp"
     gmm: dict = field(default_factory=dict)
     mlp_dims: list = field(default_factory=list)
+    phi4: dict = field(default_factory=dict)     # side, beta, periodic (lattice energy workload)
+    drafter_mode: int = 0                        # 0: carried target output, 1: target evaluated at Y_n
     param_seed: int = 0
     sample_seed: int = 2025
     dtype: str = "f32"
@@ -190,4 +192,8 @@ WORKLOADS = {
     # unadjusted Langevin on a mixture energy: d = 1024, 256 comps, means ~ N(0, 16 I), s = 1
     "cfg5": Workload("cfg5", B=8192, d=1024, L=32, K=2000, sampler="ula", ula_gamma=1e-3,
                      gmm=dict(ncomp=256, mean_scale=4.0, comp_std=1.0), param_seed=1005, sample_seed=2029),
+    # Langevin chains on the phi^4 lattice energy (Appendix K): 8x8 grid, beta = 100, step 1e-3,
+    # 100000 iterations, window 20, 500 runs, frozen drafter evaluated at Y_n
+    "phi4": Workload("phi4", B=500, d=64, L=20, K=100000, sampler="ula", ula_gamma=1e-3, denoiser="phi4",
+                     phi4=dict(side=8, beta=100.0, periodic=False), drafter_mode=1, sample_seed=2030),
 }
