@@ -90,8 +90,9 @@ def _window_check(s, w, den, a32, c32, s32, seed, chain_off, stats, chains=None)
     act, rowoff, n = s.get(sb.GET_ACT)[:na], s.get(sb.GET_ROWOFF)[:na + 1], s.get(sb.GET_N)
     assert np.all(np.diff(act) > 0)
     assert int(rowoff[na]) == nrows == int(sum(min(L, K - n[b]) for b in act))
-    Y, Dc = s.get(sb.GET_Y), s.get(sb.GET_DC)
+    Y = s.get(sb.GET_Y)
     s.draft()
+    Dc = s.get(sb.GET_DC)            # the frozen output the draft used (recomputed by the draft call in exact mode)
     X, T, rowk = s.get(sb.GET_X), s.get(sb.GET_TAIL), s.get(sb.GET_ROWK)
     s.verify_window()
     Dq = s.get(sb.GET_DQ)
