@@ -328,7 +328,8 @@ def verify_window(W, Dq, D_c, a, c, sigma, n, logU, decide_f32=True):
 
     W   [Lt+1, d]  W[0] = Y_n, W[j] = drafted state for transition k = n+j-1
     Dq  [Lt, d]    target denoiser outputs, Dq[j-1] = D(W[j-1], k)
-    D_c [d]        the frozen (carried) denoiser output the drafter used
+    D_c [d]        the frozen (carried) denoiser output the drafter used, or [Lt, d]: the draft
+                   model's own output per position (independent drafter)
     logU[Lt]       log of the accept uniforms
     Draft mean m^p = a_k W[j-1] + c_k D_c, target mean m^q = a_k W[j-1] + c_k Dq[j-1].
     decide_f32: compare log U and the log-ratio after rounding both to single precision
@@ -339,6 +340,8 @@ def verify_window(W, Dq, D_c, a, c, sigma, n, logU, decide_f32=True):
     Dq = np.asarray(Dq, dtype=np.float64)
     D_c = np.asarray(D_c, dtype=np.float64)
     Lt = Dq.shape[0]
+    if D_c.ndim == 1:                      # frozen drafter: one output for the whole window
+        D_c = np.broadcast_to(D_c, Dq.shape)
     S1 = np.zeros(Lt)
     S2 = np.zeros(Lt)
     ell = np.zeros(Lt)
@@ -347,7 +350,7 @@ def verify_window(W, Dq, D_c, a, c, sigma, n, logU, decide_f32=True):
     Y_reflect = None
     for j in range(1, Lt + 1):
         k = n + j - 1
-        m_p = a[k] * W[j - 1] + c[k] * D_c
+        m_p = a[k] * W[j - 1] + c[k] * D_c[j - 1]
         m_q = a[k] * W[j - 1] + c[k] * Dq[j - 1]
         Delta = (m_p - m_q) / sigma[k]
         Z = (W[j] - m_p) / sigma[k]
@@ -368,11 +371,13 @@ def verify_window(W, Dq, D_c, a, c, sigma, n, logU, decide_f32=True):
 
 FROZEN_PREV = 0     # carry the latest target output on the accepted trajectory (no extra call)
 FROZEN_EXACT = 1    # evaluate the target at Y_n before drafting (main-text frozen drafter)
+INDEPENDENT = 2     # a second, cheaper model proposes every draft step (Eq. 5)
 
 
 def speculative_chain(denoise, a, c, sigma, L, seed, b, d, mode=FROZEN_PREV, Y0=None,
-                      record=False, decide_f32=True):
-    """Algorithm 4 for chain b with the frozen-target drafter.
+                      record=False, decide_f32=True, draft_denoise=None):
+    """Algorithm 4 for chain b with the frozen-target drafter, or (mode INDEPENDENT) with the draft
+    model draft_denoise(x, k): m^p_k(y) = a_k y + c_k D^p(y, k) evaluated at every drafted state.
 
     denoise(x, k) -> D; transition means are a_k y + c_k D, std sigma_k.
     Returns dict(Y, nfe_calls, nfe_rows, adv (list), windows (list of per-window records if record)).
@@ -402,22 +407,28 @@ def speculative_chain(denoise, a, c, sigma, L, seed, b, d, mode=FROZEN_PREV, Y0=
             nfe_rows += 1
             first = 2
         xi = np.empty((Lt, d))
+        Dp = np.empty((Lt, d)) if mode == INDEPENDENT else None
         for j in range(1, Lt + 1):         # sequential draft
             k = n + j - 1
             xi[j - 1] = normals(seed, STREAM_DRAFT, b, k, d)
-            W[j] = a[k] * W[j - 1] + c[k] * D_c + sigma[k] * xi[j - 1]
+            if mode == INDEPENDENT:
+                Dp[j - 1] = draft_denoise(W[j - 1], k)
+                W[j] = a[k] * W[j - 1] + c[k] * Dp[j - 1] + sigma[k] * xi[j - 1]
+            else:
+                W[j] = a[k] * W[j - 1] + c[k] * D_c + sigma[k] * xi[j - 1]
         for j in range(first, Lt + 1):     # one batched target call on the drafted states
             Dq[j - 1] = denoise(W[j - 1], n + j - 1)
         if Lt >= first:
             nfe_calls += 1
             nfe_rows += Lt - first + 1
         logU = np.array([math.log(uniform01(seed, b, n + j - 1)) for j in range(1, Lt + 1)])
-        v = verify_window(W, Dq, D_c, a, c, sigma, n, logU, decide_f32=decide_f32)
+        v = verify_window(W, Dq, Dp if mode == INDEPENDENT else D_c, a, c, sigma, n, logU, decide_f32=decide_f32)
         adv = min(v["jstar"], Lt)
         if v["jstar"] <= Lt:
             W[adv] = v["Y_reflect"]
         if record:
-            windows.append(dict(n=n, W=W.copy(), Dq=Dq.copy(), D_c=D_c.copy(), logU=logU, xi=xi, **v))
+            windows.append(dict(n=n, W=W.copy(), Dq=Dq.copy(), D_c=(Dp if mode == INDEPENDENT else D_c).copy(),
+                                logU=logU, xi=xi, **v))
         Y = W[adv].copy()
         D_c = Dq[adv - 1].copy()
         n += adv

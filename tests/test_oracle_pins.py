@@ -501,3 +501,34 @@ def test_phi4_speculative_langevin_reproduces_the_papers_nfe():
         ratios.append(len(r["adv"]) / K)
         assert 2 * len(r["adv"]) - 1 <= r["nfe_calls"] <= 2 * len(r["adv"])   # the oracle counts both sequential calls
     assert abs(np.mean(ratios) - g["nfe_per_step"]) < 0.012, ratios
+
+
+# ------------------------------------------------------------------ independent drafter ----------
+
+def test_independent_drafter_equal_to_target_is_the_plain_chain():
+    den, a, c, sig = _cfg1_denoiser(K=30)
+    for b in range(3):
+        r = o.speculative_chain(den, a, c, sig, L=4, seed=31, b=b, d=2, mode=o.INDEPENDENT, draft_denoise=den)
+        assert r["adv"] == [4] * 7 + [2]                      # every draft accepted
+        assert r["nfe_calls"] == 8 and r["nfe_rows"] == 30    # one batched target call per window, no initial call
+        assert np.array_equal(r["Y"], o.plain_chain(den, a, c, sig, seed=31, b=b, d=2))
+
+
+def test_independent_drafter_keeps_the_target_law():
+    den, a, c, sig = _cfg1_denoiser(K=40)
+    w = wl.WORKLOADS["cfg1"]
+    gp = w.gmm_params()
+    abar = o.ddpm_affine(wl.beta_linear(40))[3]
+    # the cheaper model knows only two of the four components, and those slightly displaced
+    cheap = lambda x, k: o.gmm_posterior_mean(x, abar[k], gp.means[:2] * 1.1, gp.logw[:2], gp.comp_std * 1.5)
+    N = 400
+    S = np.array([o.speculative_chain(den, a, c, sig, L=4, seed=3, b=b, d=2, mode=o.INDEPENDENT, draft_denoise=cheap)["Y"]
+                  for b in range(N)])
+    P = np.array([o.plain_chain(den, a, c, sig, seed=4, b=b, d=2) for b in range(N)])
+    for i in range(2):
+        se = math.sqrt(S[:, i].var() / N + P[:, i].var() / N)
+        assert abs(S[:, i].mean() - P[:, i].mean()) < 4 * se
+    assert _mmd_perm_pvalue(S, P, np.random.default_rng(1)) > 0.01
+    # and the draft model alone does NOT have that law (the test above is not vacuous)
+    Q = np.array([o.plain_chain(cheap, a, c, sig, seed=5, b=b, d=2) for b in range(N)])
+    assert _mmd_perm_pvalue(Q, P, np.random.default_rng(2)) < 0.01
