@@ -66,6 +66,9 @@ extern "C" {
                                    (Y_n, t_n) for every active chain; that output is also row 1 of the batch,
                                    so position 1 always accepts. Two sequential target calls per window. */
 
+#define SDS_INDEPENDENT   2     /* a second, cheaper model proposes every draft step (Eq. 5); needs
+                                   sds_create_with_drafter */
+
 #define SDS_GET_X         1     /* float  [nrows, d]  drafted states fed to the target (row r = rowoff[s]+j-1) */
 #define SDS_GET_TAIL      2     /* float  [B, d]      last drafted state of each chain's window */
 #define SDS_GET_DQ        3     /* float  [nrows, d]  target denoiser outputs, same rows as X */
@@ -84,6 +87,7 @@ extern "C" {
 #define SDS_GET_NFE_ROWS  16    /* int32  [B]         target rows evaluated for the chain */
 #define SDS_GET_CTL       17    /* int32  [8]         n_active, nrows, windows done, error word, frozen chains, ... */
 #define SDS_GET_ROWK      18    /* int32  [nrows]     transition index of each row */
+#define SDS_GET_DP        19    /* float  [nrows, d]  independent drafter: the draft model's output per drafted row */
 
 typedef struct sds_ctx sds_ctx;   /* opaque, owned by the library */
 
@@ -146,6 +150,16 @@ int sds_workspace_bytes(const sds_schedule* sch, const sds_denoiser* den, int64_
  * Validates and copies the schedule. No device work. */
 int sds_create(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_t d, int32_t L,
                sds_ctx** out);
+
+/* Same with a second, cheaper denoiser as independent draft model (Eq. 5): the draft mean at
+ * every position is a_k y + c_k D^p(y, k) with D^p = `drafter` (any kind but the callback), evaluated
+ * sequentially, one position of all chains per call. drafter_tcond: [K, 4] host doubles (the
+ * mixture coefficients of the draft model; NULL unless the drafter is a mixture). Bind with
+ * SDS_INDEPENDENT. One batched target call per window; sds_sample_all uses the window kernels. */
+int sds_workspace_bytes_with_drafter(const sds_schedule* sch, const sds_denoiser* den, const sds_denoiser* drafter,
+                                     const double* drafter_tcond, int64_t B, int32_t d, int32_t L, size_t* bytes);
+int sds_create_with_drafter(const sds_schedule* sch, const sds_denoiser* den, const sds_denoiser* drafter,
+                            const double* drafter_tcond, int64_t B, int32_t d, int32_t L, sds_ctx** out);
 
 /* Attach workspace, stream (cudaStream_t, may be NULL for the default stream), seed, drafter mode
  * and the global id of local chain 0. Uploads the schedule into the workspace and waits for it. */

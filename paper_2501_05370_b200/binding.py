@@ -21,9 +21,9 @@ SDS_EINVAL, SDS_ESTATE, SDS_ENOMEM, SDS_EUNSUPPORTED = -1, -2, -3, -4
 SDS_ECUDA, SDS_ETIMEOUT, SDS_ENONFINITE, SDS_ECALLBACK = -5, -6, -7, -8
 SDS_DEN_GMM, SDS_DEN_MLP, SDS_DEN_CALLBACK, SDS_DEN_PHI4 = 1, 2, 3, 4
 SDS_F32, SDS_BF16 = 0, 1
-SDS_FROZEN_PREV, SDS_FROZEN_EXACT = 0, 1
+SDS_FROZEN_PREV, SDS_FROZEN_EXACT, SDS_INDEPENDENT = 0, 1, 2
 (GET_X, GET_TAIL, GET_DQ, GET_DC, GET_Y, GET_N, GET_ACT, GET_ROWOFF, GET_S1, GET_S2, GET_ELL, GET_LOGU,
- GET_ACCMASK, GET_JSTAR, GET_NFE_CALLS, GET_NFE_ROWS, GET_CTL, GET_ROWK) = range(1, 19)
+ GET_ACCMASK, GET_JSTAR, GET_NFE_CALLS, GET_NFE_ROWS, GET_CTL, GET_ROWK, GET_DP) = range(1, 20)
 
 DENOISE_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p)
 
@@ -43,6 +43,10 @@ class SdsDenoiser(C.Structure):
 EXPORTS = {
     "sds_workspace_bytes": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.POINTER(C.c_size_t)]),
     "sds_create": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.POINTER(C.c_void_p)]),
+    "sds_workspace_bytes_with_drafter": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int32,
+                                                   C.c_int32, C.POINTER(C.c_size_t)]),
+    "sds_create_with_drafter": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32,
+                                          C.POINTER(C.c_void_p)]),
     "sds_bind": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_uint64, C.c_int32, C.c_int64]),
     "sds_reset": (C.c_int, [C.c_void_p]),
     "sds_draft": (C.c_int, [C.c_void_p]),
@@ -151,7 +155,7 @@ class Sampler:
 
     def __init__(self, a, c, sigma, B: int, d: int, L: int, *, gmm_means=None, gmm_logw=None, tcond=None,
                  gmm_bf16: bool = False, mlp=None, callback=None, phi4=None, seed: int = 0, chain_id_offset: int = 0,
-                 drafter_mode: int = 0, device="cuda:0", stream=None):
+                 drafter_mode: int = 0, drafter=None, device="cuda:0", stream=None):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("libsds needs a CUDA device; there is no CPU path")
@@ -171,6 +175,43 @@ class Sampler:
             tcond = np.ascontiguousarray(tcond, np.float64)
             sch.tcond, sch.tcond_dim = tcond.ctypes.data, tcond.shape[1]
         self._keep += [a, c, sigma, tcond]
+        den = self._make_denoiser("tgt", gmm_means, gmm_logw, gmm_bf16, mlp, phi4, callback)
+        if den is None:
+            raise ValueError("a denoiser is required")
+        dden, dtc = None, None
+        if drafter is not None:                  # independent draft model: dict(gmm_means=, gmm_logw=, tcond=, gmm_bf16=, mlp=, phi4=)
+            dden = self._make_denoiser("drf", drafter.get("gmm_means"), drafter.get("gmm_logw"),
+                                       drafter.get("gmm_bf16", False), drafter.get("mlp"), drafter.get("phi4"), None)
+            if dden is None:
+                raise ValueError("the drafter needs a denoiser")
+            if drafter.get("tcond") is not None:
+                dtc = np.ascontiguousarray(drafter["tcond"], np.float64)
+            drafter_mode = SDS_INDEPENDENT
+        self._sch, self._den, self._dden, self._dtc = sch, den, dden, dtc
+        nbytes = C.c_size_t(0)
+        h = C.c_void_p()
+        if dden is None:
+            self._chk(self.lib.sds_workspace_bytes(C.byref(sch), C.byref(den), self.B, self.d, self.L, C.byref(nbytes)),
+                      "sds_workspace_bytes")
+            self._chk(self.lib.sds_create(C.byref(sch), C.byref(den), self.B, self.d, self.L, C.byref(h)), "sds_create")
+        else:
+            tcp = dtc.ctypes.data if dtc is not None else None
+            self._chk(self.lib.sds_workspace_bytes_with_drafter(C.byref(sch), C.byref(den), C.byref(dden), tcp, self.B,
+                                                                self.d, self.L, C.byref(nbytes)),
+                      "sds_workspace_bytes_with_drafter")
+            self._chk(self.lib.sds_create_with_drafter(C.byref(sch), C.byref(den), C.byref(dden), tcp, self.B, self.d,
+                                                       self.L, C.byref(h)), "sds_create_with_drafter")
+        self.h = h
+        self.workspace_bytes = nbytes.value
+        self.ws = torch.empty(nbytes.value + 256, dtype=torch.uint8, device=self.device)
+        base = (self.ws.data_ptr() + 255) // 256 * 256
+        self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+        self._chk(self.lib.sds_bind(self.h, base, nbytes.value, self.stream.cuda_stream, seed, drafter_mode,
+                                    chain_id_offset), "sds_bind")
+
+    def _make_denoiser(self, tag, gmm_means, gmm_logw, gmm_bf16, mlp, phi4, callback):
+        """Fills an SdsDenoiser and keeps the device arrays it names alive under self.<tag>_*."""
+        torch = self.torch
         den = SdsDenoiser()
         if gmm_means is not None:
             means = np.ascontiguousarray(gmm_means, np.float32)
@@ -178,48 +219,41 @@ class Sampler:
                 bits = means.view(np.uint32)
                 if np.any(bits & np.uint32(0xFFFF)):
                     raise ValueError("gmm_bf16 needs bf16-representable means")
-                self.means = torch.from_numpy((bits >> np.uint32(16)).astype(np.uint16).view(np.int16)).to(self.device)
+                means_t = torch.from_numpy((bits >> np.uint32(16)).astype(np.uint16).view(np.int16)).to(self.device)
             else:
-                self.means = torch.from_numpy(means).to(self.device)
-            self.logw = torch.from_numpy(np.ascontiguousarray(gmm_logw, np.float32)).to(self.device)
+                means_t = torch.from_numpy(means).to(self.device)
+            logw_t = torch.from_numpy(np.ascontiguousarray(gmm_logw, np.float32)).to(self.device)
+            setattr(self, tag + "_means", means_t)
+            setattr(self, tag + "_logw", logw_t)
+            if tag == "tgt":
+                self.means, self.logw = means_t, logw_t
             den.kind, den.ncomp = SDS_DEN_GMM, means.shape[0]
-            den.means_dev, den.logw_dev = self.means.data_ptr(), self.logw.data_ptr()
+            den.means_dev, den.logw_dev = means_t.data_ptr(), logw_t.data_ptr()
             den.means_dtype = SDS_BF16 if gmm_bf16 else SDS_F32
         elif mlp is not None:
             nl = len(mlp.weights)
             dev_bits = lambda x: torch.from_numpy(np.ascontiguousarray(x, np.uint16).view(np.int16)).to(self.device)
-            self.mlp_W = [dev_bits(w) for w in mlp.weights]
-            self.mlp_bias = [torch.from_numpy(np.ascontiguousarray(x, np.float32)).to(self.device) for x in mlp.bias]
-            self.mlp_temb = [dev_bits(x) if x is not None else None for x in mlp.temb]
-            self._mlp_dims = np.ascontiguousarray(mlp.dims, np.int32)
-            self._mlp_Wp = (C.c_void_p * nl)(*[x.data_ptr() for x in self.mlp_W])
-            self._mlp_bp = (C.c_void_p * nl)(*[x.data_ptr() for x in self.mlp_bias])
-            self._mlp_tp = (C.c_void_p * nl)(*[(x.data_ptr() if x is not None else None) for x in self.mlp_temb])
+            W = [dev_bits(w) for w in mlp.weights]
+            bias = [torch.from_numpy(np.ascontiguousarray(x, np.float32)).to(self.device) for x in mlp.bias]
+            temb = [dev_bits(x) if x is not None else None for x in mlp.temb]
+            dims = np.ascontiguousarray(mlp.dims, np.int32)
+            Wp = (C.c_void_p * nl)(*[x.data_ptr() for x in W])
+            bp = (C.c_void_p * nl)(*[x.data_ptr() for x in bias])
+            tp = (C.c_void_p * nl)(*[(x.data_ptr() if x is not None else None) for x in temb])
+            setattr(self, tag + "_mlp", (W, bias, temb, dims, Wp, bp, tp))
             den.kind, den.nlayer = SDS_DEN_MLP, nl
-            den.W_dev = C.cast(self._mlp_Wp, C.c_void_p)
-            den.bias_dev = C.cast(self._mlp_bp, C.c_void_p)
-            den.temb_dev = C.cast(self._mlp_tp, C.c_void_p)
-            den.dims = self._mlp_dims.ctypes.data
+            den.W_dev = C.cast(Wp, C.c_void_p)
+            den.bias_dev = C.cast(bp, C.c_void_p)
+            den.temb_dev = C.cast(tp, C.c_void_p)
+            den.dims = dims.ctypes.data
         elif phi4 is not None:                   # (grid side, coupling beta, periodic)
             den.kind, den.grid_side, den.coupling, den.periodic = SDS_DEN_PHI4, int(phi4[0]), float(phi4[1]), int(bool(phi4[2]))
         elif callback is not None:
             self._cb = DENOISE_FN(callback)
             den.kind, den.fn = SDS_DEN_CALLBACK, self._cb
         else:
-            raise ValueError("a denoiser is required")
-        self._sch, self._den = sch, den
-        nbytes = C.c_size_t(0)
-        self._chk(self.lib.sds_workspace_bytes(C.byref(sch), C.byref(den), self.B, self.d, self.L, C.byref(nbytes)),
-                  "sds_workspace_bytes")
-        self.workspace_bytes = nbytes.value
-        self.ws = torch.empty(nbytes.value + 256, dtype=torch.uint8, device=self.device)
-        base = (self.ws.data_ptr() + 255) // 256 * 256
-        self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
-        h = C.c_void_p()
-        self._chk(self.lib.sds_create(C.byref(sch), C.byref(den), self.B, self.d, self.L, C.byref(h)), "sds_create")
-        self.h = h
-        self._chk(self.lib.sds_bind(self.h, base, nbytes.value, self.stream.cuda_stream, seed, drafter_mode,
-                                    chain_id_offset), "sds_bind")
+            return None
+        return den
 
     # -- helpers --
     def _chk(self, rc: int, where: str, allow=()):
@@ -278,7 +312,7 @@ class Sampler:
         GET_ROWOFF: ("int32", "B1"), GET_S1: ("float64", "B_L"), GET_S2: ("float64", "B_L"),
         GET_ELL: ("float32", "B_L"), GET_LOGU: ("float32", "B_L"), GET_ACCMASK: ("uint32", "B"),
         GET_JSTAR: ("int32", "B"), GET_NFE_CALLS: ("int32", "B"), GET_NFE_ROWS: ("int32", "B"),
-        GET_CTL: ("int32", "ctl"), GET_ROWK: ("int32", "rows"),
+        GET_CTL: ("int32", "ctl"), GET_ROWK: ("int32", "rows"), GET_DP: ("float32", "rows_d"),
     }
 
     def get(self, what: int) -> np.ndarray:

@@ -38,11 +38,29 @@ struct Layout {
   size_t Y, Dc, T, X, Dq, Xb;
   size_t n, act, rowoff, rowk, ctl;
   size_t S1, S2, ell, logU, accmask, jstar, nfe_calls, nfe_rows;
-  size_t musq;
+  size_t Gk;
+  size_t Gx, Gb, Pb, Dp;  // independent drafter: gathered rows (f32, bf16), its outputs per call and per row
+  size_t total;
+};
+
+// workspace regions private to one denoiser (the target, or the independent draft model)
+struct DenLayout {
+  size_t tcond, musq;
   size_t H0, H1;          // MLP hidden activations (bf16)
   size_t logits, R, Mt;   // large mixture: logits (f32), responsibilities (bf16), transposed means (bf16)
   size_t Xs, Ms;          // float mixture on tensor cores: 3 bf16 planes of the rows / of the means
-  size_t total;
+  size_t xb;              // where a bf16 copy of this denoiser's input rows goes when the caller has none
+};
+
+struct Engine {
+  sds_denoiser den{};
+  std::vector<int32_t> mlp_dims;                 // copies of the caller's MLP description
+  std::vector<const void*> mlp_W, mlp_temb;
+  std::vector<const float*> mlp_bias;
+  std::vector<double> tcond;
+  DenLayout lay{};
+  int64_t cap_rows = 0;                          // rows of the buffers this denoiser's GEMMs read
+  bool musq_ready = false;
 };
 
 }  // namespace
@@ -51,12 +69,9 @@ struct sds_ctx {
   int64_t B = 0;
   int32_t d = 0, L = 0, K = 0;
   std::vector<float> a, c, sigma;
-  std::vector<double> tcond;
   int32_t tcond_dim = 0;
-  sds_denoiser den{};
-  std::vector<int32_t> mlp_dims;                 // copies of the caller's MLP description
-  std::vector<const void*> mlp_W, mlp_temb;
-  std::vector<const float*> mlp_bias;
+  Engine tgt, drf;                  // target denoiser; independent draft model (optional)
+  bool has_drafter = false;
   Layout lay{};
   char* ws = nullptr;
   size_t ws_bytes = 0;
@@ -70,7 +85,6 @@ struct sds_ctx {
   int64_t launches = 0;
   int32_t* h_pin = nullptr;         // pinned host words for the window loop
   cudaEvent_t ev[2] = {nullptr, nullptr};
-  bool musq_ready = false;
   bool whole_chain = true;          // sds_sample_all may use the whole-chain kernel
   bool tensor_split = true;         // float mixtures of tensor-core shape use the 3-way bf16 split
   // optional per-kernel timing: event pairs recorded around each launch, summed on read
@@ -94,14 +108,38 @@ bool wants_bf16_rows(const sds_denoiser& den) {
   return den.kind == SDS_DEN_MLP || (den.kind == SDS_DEN_GMM && den.means_dtype == SDS_BF16);
 }
 
-void make_layout(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_t d, int32_t L, Layout* out) {
+void den_layout(Carve& cv, const sds_denoiser* den, size_t K, int tcond_dim, size_t rows, int32_t d, DenLayout* l) {
+  l->tcond = cv.take(K * (size_t)(tcond_dim > 0 ? tcond_dim : 1) * 8);
+  l->musq = (den->kind == SDS_DEN_GMM) ? cv.take((size_t)den->ncomp * 8) : kNone;
+  l->H0 = l->H1 = l->logits = l->R = l->Mt = l->Xs = l->Ms = kNone;
+  if (gmm_split_shape(*den, d)) {
+    l->Xs = cv.take(3 * rows * (size_t)d * 2);
+    l->Ms = cv.take(3 * (size_t)den->ncomp * d * 2);
+    l->Mt = cv.take(3 * (size_t)d * den->ncomp * 2);
+    l->R = cv.take(3 * rows * (size_t)den->ncomp * 2);
+    l->logits = cv.take(rows * (size_t)den->ncomp * 4);
+  }
+  if (den->kind == SDS_DEN_MLP) {
+    size_t width = 0;
+    for (int i = 1; i < den->nlayer; ++i) width = std::max(width, (size_t)den->dims[i]);
+    l->H0 = cv.take(rows * width * 2);
+    l->H1 = cv.take(rows * width * 2);
+  }
+  if (den->kind == SDS_DEN_GMM && den->means_dtype == SDS_BF16) {
+    l->logits = cv.take(rows * (size_t)den->ncomp * 4);
+    l->R = cv.take(rows * (size_t)den->ncomp * 2);
+    l->Mt = cv.take((size_t)d * den->ncomp * 2);
+  }
+}
+
+void make_layout(const sds_schedule* sch, const sds_denoiser* den, const sds_denoiser* drafter, int64_t B, int32_t d,
+                 int32_t L, Layout* out, DenLayout* tl, DenLayout* dl) {
   Carve cv;
   Layout l{};
   const size_t K = (size_t)sch->K, rows = (size_t)B * L, Bd = (size_t)B * d;
   l.a = cv.take(K * 4);
   l.c = cv.take(K * 4);
   l.sigma = cv.take(K * 4);
-  l.tcond = cv.take(K * (size_t)(sch->tcond_dim > 0 ? sch->tcond_dim : 1) * 8);
   l.Y = cv.take(Bd * 4);
   l.Dc = cv.take(Bd * 4);
   l.T = cv.take(Bd * 4);
@@ -121,29 +159,23 @@ void make_layout(const sds_schedule* sch, const sds_denoiser* den, int64_t B, in
   l.jstar = cv.take((size_t)B * 4);
   l.nfe_calls = cv.take((size_t)B * 4);
   l.nfe_rows = cv.take((size_t)B * 4);
-  l.musq = (den->kind == SDS_DEN_GMM) ? cv.take((size_t)den->ncomp * 8) : kNone;
-  l.H0 = l.H1 = l.logits = l.R = l.Mt = l.Xs = l.Ms = kNone;
-  if (gmm_split_shape(*den, d)) {
-    l.Xs = cv.take(3 * rows * (size_t)d * 2);
-    l.Ms = cv.take(3 * (size_t)den->ncomp * d * 2);
-    l.Mt = cv.take(3 * (size_t)d * den->ncomp * 2);
-    l.R = cv.take(3 * rows * (size_t)den->ncomp * 2);
-    l.logits = cv.take(rows * (size_t)den->ncomp * 4);
-  }
-  if (den->kind == SDS_DEN_MLP) {
-    size_t width = 0;
-    for (int i = 1; i < den->nlayer; ++i) width = std::max(width, (size_t)den->dims[i]);
-    l.H0 = cv.take(rows * width * 2);
-    l.H1 = cv.take(rows * width * 2);
-  }
-  if (den->kind == SDS_DEN_GMM && den->means_dtype == SDS_BF16) {
-    l.logits = cv.take(rows * (size_t)den->ncomp * 4);
-    l.R = cv.take(rows * (size_t)den->ncomp * 2);
-    l.Mt = cv.take((size_t)d * den->ncomp * 2);
+  den_layout(cv, den, K, sch->tcond_dim, rows, d, tl);
+  tl->xb = l.Xb;
+  l.Gx = l.Gb = l.Pb = l.Dp = l.Gk = kNone;
+  if (drafter) {
+    l.Gk = cv.take((size_t)B * 4);
+    l.Gx = cv.take(Bd * 4);
+    l.Gb = cv.take(Bd * 2);
+    l.Pb = cv.take(Bd * 4);
+    l.Dp = cv.take(rows * d * 4);
+    den_layout(cv, drafter, K, 4, (size_t)B, d, dl);
+    dl->xb = l.Gb;
   }
   l.total = cv.off;
   *out = l;
 }
+
+int validate_den(const sds_denoiser* den, const double* tcond, int tcond_dim, int32_t d);
 
 int validate(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_t d, int32_t L) {
   if (!sch || !den) return SDS_EINVAL;
@@ -154,10 +186,14 @@ int validate(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_
     if (!std::isfinite(sch->a[k]) || !std::isfinite(sch->c[k]) || !std::isfinite(sch->sigma[k])) return SDS_EINVAL;
     if (!(sch->sigma[k] > 0.f)) return SDS_EINVAL;
   }
+  return validate_den(den, sch->tcond, sch->tcond_dim, d);
+}
+
+int validate_den(const sds_denoiser* den, const double* tcond, int tcond_dim, int32_t d) {
   switch (den->kind) {
     case SDS_DEN_GMM:
       if (den->ncomp <= 0 || !den->means_dev || !den->logw_dev) return SDS_EINVAL;
-      if (!sch->tcond || sch->tcond_dim != 4) return SDS_EINVAL;
+      if (!tcond || tcond_dim != 4) return SDS_EINVAL;
       if (den->means_dtype == SDS_BF16) {
         // tensor-core path: both contractions tile by 128
         if (den->ncomp % 128 != 0 || d % 128 != 0) return SDS_EUNSUPPORTED;
@@ -195,7 +231,7 @@ T* at(sds_ctx* c, size_t off) { return off == kNone ? nullptr : reinterpret_cast
 WinArgs win_args(sds_ctx* c) {
   WinArgs A{};
   A.B = (int)c->B; A.d = c->d; A.L = c->L; A.K = c->K;
-  A.exact = c->mode == SDS_FROZEN_EXACT ? 1 : 0;
+  A.mode = c->mode;
   A.seed = c->seed; A.chain_off = (uint64_t)c->chain_off;
   A.a = at<float>(c, c->lay.a); A.c = at<float>(c, c->lay.c); A.sigma = at<float>(c, c->lay.sigma);
   A.Y = at<float>(c, c->lay.Y); A.Dc = at<float>(c, c->lay.Dc); A.T = at<float>(c, c->lay.T);
@@ -206,16 +242,18 @@ WinArgs win_args(sds_ctx* c) {
   A.ell = at<float>(c, c->lay.ell); A.logU = at<float>(c, c->lay.logU);
   A.accmask = at<uint32_t>(c, c->lay.accmask); A.jstar = at<int>(c, c->lay.jstar);
   A.nfe_calls = at<int>(c, c->lay.nfe_calls); A.nfe_rows = at<int>(c, c->lay.nfe_rows);
+  A.Gx = at<float>(c, c->lay.Gx); A.Gb = at<uint16_t>(c, c->lay.Gb); A.Gk = at<int>(c, c->lay.Gk);
+  A.Pb = at<float>(c, c->lay.Pb); A.Dp = at<float>(c, c->lay.Dp);
   return A;
 }
 
-GmmArgs gmm_args(sds_ctx* c) {
+GmmArgs gmm_args(sds_ctx* c, Engine& e) {
   GmmArgs G{};
-  G.d = c->d; G.ncomp = c->den.ncomp; G.K = c->K;
-  G.tcond = at<double>(c, c->lay.tcond);
-  G.means = static_cast<const float*>(c->den.means_dev);
-  G.logw = c->den.logw_dev;
-  G.musq = at<double>(c, c->lay.musq);
+  G.d = c->d; G.ncomp = e.den.ncomp; G.K = c->K;
+  G.tcond = at<double>(c, e.lay.tcond);
+  G.means = static_cast<const float*>(e.den.means_dev);
+  G.logw = e.den.logw_dev;
+  G.musq = at<double>(c, e.lay.musq);
   return G;
 }
 
@@ -266,28 +304,28 @@ void prof_collect(sds_ctx* c) {
     (ctx)->launches++;                         \
   } while (0)
 
-int ensure_musq(sds_ctx* c) {
-  if (c->musq_ready) return SDS_OK;
-  SDS_LAUNCH(c, SDS_PROF_AUX, launch_musq(static_cast<const float*>(c->den.means_dev), c->den.ncomp, c->d,
-                                          at<double>(c, c->lay.musq), c->stream));
-  c->musq_ready = true;
+int ensure_musq(sds_ctx* c, Engine& e) {
+  if (e.musq_ready) return SDS_OK;
+  SDS_LAUNCH(c, SDS_PROF_AUX, launch_musq(static_cast<const float*>(e.den.means_dev), e.den.ncomp, c->d,
+                                          at<double>(c, e.lay.musq), c->stream));
+  e.musq_ready = true;
   return SDS_OK;
 }
 
 // bf16 copy of the rows for the tensor-core denoisers (the draft kernel writes it on the hot path)
-int ensure_bf16_rows(sds_ctx* c, const float* X, const uint16_t** Xb, int64_t rows_ub) {
+int ensure_bf16_rows(sds_ctx* c, Engine& e, const float* X, const uint16_t** Xb, int64_t rows_ub) {
   if (*Xb) return SDS_OK;
-  uint16_t* dst = at<uint16_t>(c, c->lay.Xb);
+  uint16_t* dst = at<uint16_t>(c, e.lay.xb);
   SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_f32_to_bf16(X, (size_t)rows_ub * c->d, dst, c->stream));
   *Xb = dst;
   return SDS_OK;
 }
 
-TcGemmArgs tc_args(sds_ctx* c, const int* rowk, const int* nrows_dev, int64_t rows_ub) {
+TcGemmArgs tc_args(sds_ctx* c, Engine& e, const int* rowk, const int* nrows_dev, int64_t rows_ub) {
   TcGemmArgs g{};
   g.nrows_dev = nrows_dev;
   g.rows_host = (int)rows_ub;
-  g.rows_cap = (int)(c->B * c->L);
+  g.rows_cap = (int)e.cap_rows;
   g.rowk = rowk;
   g.err = at<int>(c, c->lay.ctl) + kCtlTcError;
   return g;
@@ -295,24 +333,24 @@ TcGemmArgs tc_args(sds_ctx* c, const int* rowk, const int* nrows_dev, int64_t ro
 
 // run the target denoiser on dense rows X (and their bf16 copy Xb, NULL = make one); the row count
 // lives on the device (nrows_dev, may be NULL) with a host upper bound for the grids
-int run_denoiser(sds_ctx* c, const float* X, const uint16_t* Xb, const int* rowk, const int* nrows_dev,
+int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, const int* rowk, const int* nrows_dev,
                  int64_t rows_ub, float* out) {
   if (rows_ub <= 0) return SDS_OK;
-  switch (c->den.kind) {
+  switch (e.den.kind) {
     case SDS_DEN_GMM: {
-      if (c->den.means_dtype == SDS_F32 && c->tensor_split && gmm_split_shape(c->den, c->d)) {
+      if (e.den.means_dtype == SDS_F32 && c->tensor_split && gmm_split_shape(e.den, c->d)) {
         // Float mixture on the tensor cores: rows, means and responsibilities are split into three
         // bf16 planes each (x = h + m + l carries the 24-bit significand); the six products of
         // total order <= 2 are accumulated, smallest first, in one TMEM accumulator.
-        const float* means = static_cast<const float*>(c->den.means_dev);
-        const size_t nc = (size_t)c->den.ncomp, dd = (size_t)c->d, cap = (size_t)(c->B * c->L);
-        uint16_t* Ms = at<uint16_t>(c, c->lay.Ms);
-        uint16_t* Mt = at<uint16_t>(c, c->lay.Mt);
-        uint16_t* Xs = at<uint16_t>(c, c->lay.Xs);
-        uint16_t* Rs = at<uint16_t>(c, c->lay.R);
-        float* logits = at<float>(c, c->lay.logits);
-        const bool fresh = !c->musq_ready;
-        int rc = ensure_musq(c);
+        const float* means = static_cast<const float*>(e.den.means_dev);
+        const size_t nc = (size_t)e.den.ncomp, dd = (size_t)c->d, cap = (size_t)e.cap_rows;
+        uint16_t* Ms = at<uint16_t>(c, e.lay.Ms);
+        uint16_t* Mt = at<uint16_t>(c, e.lay.Mt);
+        uint16_t* Xs = at<uint16_t>(c, e.lay.Xs);
+        uint16_t* Rs = at<uint16_t>(c, e.lay.R);
+        float* logits = at<float>(c, e.lay.logits);
+        const bool fresh = !e.musq_ready;
+        int rc = ensure_musq(c, e);
         if (rc != SDS_OK) return rc;
         if (fresh) {
           SDS_LAUNCH(c, SDS_PROF_AUX, launch_split3(means, nc * dd, nc * dd, Ms, c->stream));
@@ -321,77 +359,77 @@ int run_denoiser(sds_ctx* c, const float* X, const uint16_t* Xb, const int* rowk
         }
         SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_split3(X, (size_t)rows_ub * dd, cap * dd, Xs, c->stream));
         static const uint8_t kA[6] = {2, 1, 0, 1, 0, 0}, kB[6] = {0, 1, 2, 0, 1, 0};
-        TcGemmArgs g = tc_args(c, rowk, nrows_dev, rows_ub);
+        TcGemmArgs g = tc_args(c, e, rowk, nrows_dev, rows_ub);
         g.N = (int)nc; g.K = (int)dd; g.out = logits; g.ldo = (int)nc;
-        g.tcond = at<double>(c, c->lay.tcond); g.musq = at<double>(c, c->lay.musq); g.logw = c->den.logw_dev;
+        g.tcond = at<double>(c, e.lay.tcond); g.musq = at<double>(c, e.lay.musq); g.logw = e.den.logw_dev;
         g.nseg = 6; g.nplanes = 3; g.a_plane = cap * dd; g.b_plane = nc * dd;
         for (int i = 0; i < 6; ++i) { g.a_idx[i] = kA[i]; g.b_idx[i] = kB[i]; }
         SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiGmmLogits, g, Xs, Ms, c->stream));
         SDS_LAUNCH(c, SDS_PROF_DENOISE,
                    launch_softmax_split3(logits, nrows_dev, (int)rows_ub, (int)nc, (int)dd, X, means,
-                                         at<double>(c, c->lay.musq), c->den.logw_dev, at<double>(c, c->lay.tcond), rowk,
+                                         at<double>(c, e.lay.musq), e.den.logw_dev, at<double>(c, e.lay.tcond), rowk,
                                          cap * nc, Rs, c->stream));
-        TcGemmArgs m = tc_args(c, rowk, nrows_dev, rows_ub);
+        TcGemmArgs m = tc_args(c, e, rowk, nrows_dev, rows_ub);
         m.N = (int)dd; m.K = (int)nc; m.out = out; m.ldo = (int)dd;
-        m.tcond = at<double>(c, c->lay.tcond); m.xrows = X;
+        m.tcond = at<double>(c, e.lay.tcond); m.xrows = X;
         m.nseg = 6; m.nplanes = 3; m.a_plane = cap * nc; m.b_plane = nc * dd;
         for (int i = 0; i < 6; ++i) { m.a_idx[i] = kA[i]; m.b_idx[i] = kB[i]; }
         SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiGmmMix, m, Rs, Mt, c->stream));
         return SDS_OK;
       }
-      if (c->den.means_dtype == SDS_F32) {
-        const int rc = ensure_musq(c);
+      if (e.den.means_dtype == SDS_F32) {
+        const int rc = ensure_musq(c, e);
         if (rc != SDS_OK) return rc;
-        SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gmm_f32(gmm_args(c), X, rowk, nrows_dev, (int)rows_ub, out, c->stream));
+        SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gmm_f32(gmm_args(c, e), X, rowk, nrows_dev, (int)rows_ub, out, c->stream));
         return SDS_OK;
       }
       // large mixture on tensor cores: logits = X M^T, softmax, mix = R M, affine epilogue
-      const uint16_t* means = static_cast<const uint16_t*>(c->den.means_dev);
-      uint16_t* Mt = at<uint16_t>(c, c->lay.Mt);
-      uint16_t* R = at<uint16_t>(c, c->lay.R);
-      float* logits = at<float>(c, c->lay.logits);
-      if (!c->musq_ready) {
-        SDS_LAUNCH(c, SDS_PROF_AUX, launch_musq_bf16(means, c->den.ncomp, c->d, at<double>(c, c->lay.musq), c->stream));
-        SDS_LAUNCH(c, SDS_PROF_AUX, launch_transpose_bf16(means, c->den.ncomp, c->d, Mt, c->stream));
-        c->musq_ready = true;
+      const uint16_t* means = static_cast<const uint16_t*>(e.den.means_dev);
+      uint16_t* Mt = at<uint16_t>(c, e.lay.Mt);
+      uint16_t* R = at<uint16_t>(c, e.lay.R);
+      float* logits = at<float>(c, e.lay.logits);
+      if (!e.musq_ready) {
+        SDS_LAUNCH(c, SDS_PROF_AUX, launch_musq_bf16(means, e.den.ncomp, c->d, at<double>(c, e.lay.musq), c->stream));
+        SDS_LAUNCH(c, SDS_PROF_AUX, launch_transpose_bf16(means, e.den.ncomp, c->d, Mt, c->stream));
+        e.musq_ready = true;
       }
-      int rc = ensure_bf16_rows(c, X, &Xb, rows_ub);
+      int rc = ensure_bf16_rows(c, e, X, &Xb, rows_ub);
       if (rc != SDS_OK) return rc;
-      TcGemmArgs g = tc_args(c, rowk, nrows_dev, rows_ub);
-      g.N = c->den.ncomp; g.K = c->d; g.out = logits; g.ldo = c->den.ncomp;
-      g.tcond = at<double>(c, c->lay.tcond); g.musq = at<double>(c, c->lay.musq); g.logw = c->den.logw_dev;
+      TcGemmArgs g = tc_args(c, e, rowk, nrows_dev, rows_ub);
+      g.N = e.den.ncomp; g.K = c->d; g.out = logits; g.ldo = e.den.ncomp;
+      g.tcond = at<double>(c, e.lay.tcond); g.musq = at<double>(c, e.lay.musq); g.logw = e.den.logw_dev;
       SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiGmmLogits, g, Xb, means, c->stream));
-      SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_softmax_bf16(logits, nrows_dev, (int)rows_ub, c->den.ncomp, R, c->stream));
-      TcGemmArgs m = tc_args(c, rowk, nrows_dev, rows_ub);
-      m.N = c->d; m.K = c->den.ncomp; m.out = out; m.ldo = c->d;
-      m.tcond = at<double>(c, c->lay.tcond); m.xrows = X;
+      SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_softmax_bf16(logits, nrows_dev, (int)rows_ub, e.den.ncomp, R, c->stream));
+      TcGemmArgs m = tc_args(c, e, rowk, nrows_dev, rows_ub);
+      m.N = c->d; m.K = e.den.ncomp; m.out = out; m.ldo = c->d;
+      m.tcond = at<double>(c, e.lay.tcond); m.xrows = X;
       SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiGmmMix, m, R, Mt, c->stream));
       return SDS_OK;
     }
     case SDS_DEN_MLP: {
-      int rc = ensure_bf16_rows(c, X, &Xb, rows_ub);
+      int rc = ensure_bf16_rows(c, e, X, &Xb, rows_ub);
       if (rc != SDS_OK) return rc;
       const void* in = Xb;
-      const int nl = (int)c->mlp_W.size();
+      const int nl = (int)e.mlp_W.size();
       for (int l = 0; l < nl; ++l) {
-        TcGemmArgs g = tc_args(c, rowk, nrows_dev, rows_ub);
-        g.N = c->mlp_dims[l + 1]; g.K = c->mlp_dims[l];
-        g.bias = c->mlp_bias[l];
+        TcGemmArgs g = tc_args(c, e, rowk, nrows_dev, rows_ub);
+        g.N = e.mlp_dims[l + 1]; g.K = e.mlp_dims[l];
+        g.bias = e.mlp_bias[l];
         if (l < nl - 1) {
-          uint16_t* h = at<uint16_t>(c, (l & 1) ? c->lay.H1 : c->lay.H0);
-          g.out = h; g.ldo = g.N; g.temb = static_cast<const uint16_t*>(c->mlp_temb[l]);
-          SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiMlpHidden, g, in, c->mlp_W[l], c->stream));
+          uint16_t* h = at<uint16_t>(c, (l & 1) ? e.lay.H1 : e.lay.H0);
+          g.out = h; g.ldo = g.N; g.temb = static_cast<const uint16_t*>(e.mlp_temb[l]);
+          SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiMlpHidden, g, in, e.mlp_W[l], c->stream));
           in = h;
         } else {
           g.out = out; g.ldo = g.N;
-          SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiBiasF32, g, in, c->mlp_W[l], c->stream));
+          SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiBiasF32, g, in, e.mlp_W[l], c->stream));
         }
       }
       return SDS_OK;
     }
     case SDS_DEN_PHI4:
-      SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_phi4_grad(X, nrows_dev, (int)rows_ub, c->den.grid_side, c->den.coupling,
-                                                        c->den.periodic, out, c->stream));
+      SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_phi4_grad(X, nrows_dev, (int)rows_ub, e.den.grid_side, e.den.coupling,
+                                                        e.den.periodic, out, c->stream));
       return SDS_OK;
     case SDS_DEN_CALLBACK: {
       int32_t rows = (int32_t)rows_ub;         // the callback needs the row count on the host
@@ -401,7 +439,7 @@ int run_denoiser(sds_ctx* c, const float* X, const uint16_t* Xb, const int* rowk
         rows = c->h_pin[4];
       }
       if (rows <= 0) return SDS_OK;
-      const int rc = c->den.fn(c->den.user, X, rowk, rows, c->d, out, (void*)c->stream);
+      const int rc = e.den.fn(e.den.user, X, rowk, rows, c->d, out, (void*)c->stream);
       return rc == 0 ? SDS_OK : SDS_ECALLBACK;
     }
     default:
@@ -424,22 +462,37 @@ int sync_active(sds_ctx* c, int64_t* n_active) {
 extern "C" {
 #pragma GCC visibility push(default)
 
-int sds_workspace_bytes(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_t d, int32_t L,
-                        size_t* bytes) {
-  if (!bytes) return SDS_EINVAL;
-  const int rc = validate(sch, den, B, d, L);
-  if (rc != SDS_OK) return rc;
-  Layout l;
-  make_layout(sch, den, B, d, L, &l);
-  *bytes = l.total;
-  return SDS_OK;
+namespace {
+
+void engine_init(Engine& e, const sds_denoiser* den, const double* tcond, int tcond_dim, int K, int64_t cap_rows) {
+  e.den = *den;
+  e.cap_rows = cap_rows;
+  if (tcond && tcond_dim > 0) e.tcond.assign(tcond, tcond + (size_t)K * tcond_dim);
+  if (den->kind == SDS_DEN_MLP) {
+    e.mlp_dims.assign(den->dims, den->dims + den->nlayer + 1);
+    e.mlp_W.assign(den->W_dev, den->W_dev + den->nlayer);
+    e.mlp_bias.assign(den->bias_dev, den->bias_dev + den->nlayer);
+    e.mlp_temb.assign(den->temb_dev, den->temb_dev + den->nlayer);
+    e.den.dims = e.mlp_dims.data();
+  }
 }
 
-int sds_create(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_t d, int32_t L, sds_ctx** out) {
-  if (!out) return SDS_EINVAL;
-  *out = nullptr;
-  const int rc = validate(sch, den, B, d, L);
+int create_impl(const sds_schedule* sch, const sds_denoiser* den, const sds_denoiser* drafter,
+                const double* drafter_tcond, int64_t B, int32_t d, int32_t L, sds_ctx** out, size_t* bytes_only) {
+  int rc = validate(sch, den, B, d, L);
   if (rc != SDS_OK) return rc;
+  if (drafter) {
+    if (drafter->kind == SDS_DEN_CALLBACK) return SDS_EUNSUPPORTED;
+    rc = validate_den(drafter, drafter_tcond, 4, d);
+    if (rc != SDS_OK) return rc;
+  }
+  if (bytes_only) {
+    Layout l;
+    DenLayout tl, dl;
+    make_layout(sch, den, drafter, B, d, L, &l, &tl, &dl);
+    *bytes_only = l.total;
+    return SDS_OK;
+  }
   sds_ctx* c = new (std::nothrow) sds_ctx();
   if (!c) return SDS_ENOMEM;
   c->B = B; c->d = d; c->L = L; c->K = sch->K;
@@ -447,16 +500,10 @@ int sds_create(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int3
   c->c.assign(sch->c, sch->c + sch->K);
   c->sigma.assign(sch->sigma, sch->sigma + sch->K);
   c->tcond_dim = sch->tcond_dim > 0 ? sch->tcond_dim : 0;
-  if (sch->tcond && c->tcond_dim > 0) c->tcond.assign(sch->tcond, sch->tcond + (size_t)sch->K * c->tcond_dim);
-  c->den = *den;
-  if (den->kind == SDS_DEN_MLP) {
-    c->mlp_dims.assign(den->dims, den->dims + den->nlayer + 1);
-    c->mlp_W.assign(den->W_dev, den->W_dev + den->nlayer);
-    c->mlp_bias.assign(den->bias_dev, den->bias_dev + den->nlayer);
-    c->mlp_temb.assign(den->temb_dev, den->temb_dev + den->nlayer);
-    c->den.dims = c->mlp_dims.data();
-  }
-  make_layout(sch, den, B, d, L, &c->lay);
+  engine_init(c->tgt, den, sch->tcond, c->tcond_dim, sch->K, B * L);
+  c->has_drafter = drafter != nullptr;
+  if (drafter) engine_init(c->drf, drafter, drafter_tcond, 4, sch->K, B);
+  make_layout(sch, den, drafter, B, d, L, &c->lay, &c->tgt.lay, &c->drf.lay);
   if (cudaHostAlloc((void**)&c->h_pin, 64 * sizeof(int32_t), cudaHostAllocDefault) != cudaSuccess) {
     c->last_cuda = (int)cudaGetLastError();
     delete c;
@@ -475,10 +522,39 @@ int sds_create(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int3
   return SDS_OK;
 }
 
+}  // namespace
+
+int sds_workspace_bytes(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_t d, int32_t L,
+                        size_t* bytes) {
+  if (!bytes) return SDS_EINVAL;
+  return create_impl(sch, den, nullptr, nullptr, B, d, L, nullptr, bytes);
+}
+
+int sds_create(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_t d, int32_t L, sds_ctx** out) {
+  if (!out) return SDS_EINVAL;
+  *out = nullptr;
+  return create_impl(sch, den, nullptr, nullptr, B, d, L, out, nullptr);
+}
+
+int sds_workspace_bytes_with_drafter(const sds_schedule* sch, const sds_denoiser* den, const sds_denoiser* drafter,
+                                     const double* drafter_tcond, int64_t B, int32_t d, int32_t L, size_t* bytes) {
+  if (!bytes || !drafter) return SDS_EINVAL;
+  return create_impl(sch, den, drafter, drafter_tcond, B, d, L, nullptr, bytes);
+}
+
+int sds_create_with_drafter(const sds_schedule* sch, const sds_denoiser* den, const sds_denoiser* drafter,
+                            const double* drafter_tcond, int64_t B, int32_t d, int32_t L, sds_ctx** out) {
+  if (!out || !drafter) return SDS_EINVAL;
+  *out = nullptr;
+  return create_impl(sch, den, drafter, drafter_tcond, B, d, L, out, nullptr);
+}
+
 int sds_bind(sds_ctx* c, void* workspace_dev, size_t bytes, void* cuda_stream, uint64_t seed, int32_t drafter_mode,
              int64_t chain_id_offset) {
   if (!c || !workspace_dev) return SDS_EINVAL;
-  if (drafter_mode != SDS_FROZEN_PREV && drafter_mode != SDS_FROZEN_EXACT) return SDS_EUNSUPPORTED;
+  if (drafter_mode != SDS_FROZEN_PREV && drafter_mode != SDS_FROZEN_EXACT && drafter_mode != SDS_INDEPENDENT)
+    return SDS_EUNSUPPORTED;
+  if ((drafter_mode == SDS_INDEPENDENT) != c->has_drafter) return SDS_EINVAL;   // the draft model and the mode go together
   if (chain_id_offset < 0) return SDS_EINVAL;
   if (bytes < c->lay.total || (reinterpret_cast<uintptr_t>(workspace_dev) % kAlign) != 0) return SDS_ENOMEM;
   c->ws = static_cast<char*>(workspace_dev);
@@ -487,14 +563,15 @@ int sds_bind(sds_ctx* c, void* workspace_dev, size_t bytes, void* cuda_stream, u
   c->seed = seed;
   c->mode = drafter_mode;
   c->chain_off = chain_id_offset;
-  c->musq_ready = false;
+  c->tgt.musq_ready = c->drf.musq_ready = false;
   const size_t kb = (size_t)c->K * 4;
   SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.a, c->a.data(), kb, cudaMemcpyHostToDevice, c->stream));
   SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.c, c->c.data(), kb, cudaMemcpyHostToDevice, c->stream));
   SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.sigma, c->sigma.data(), kb, cudaMemcpyHostToDevice, c->stream));
-  if (!c->tcond.empty())
-    SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.tcond, c->tcond.data(), c->tcond.size() * 8, cudaMemcpyHostToDevice,
-                              c->stream));
+  for (Engine* e : {&c->tgt, &c->drf})
+    if (!e->tcond.empty())
+      SDS_CU(c, cudaMemcpyAsync(c->ws + e->lay.tcond, e->tcond.data(), e->tcond.size() * 8, cudaMemcpyHostToDevice,
+                                c->stream));
   SDS_CU(c, cudaMemsetAsync(c->ws + c->lay.ctl, 0, kCtlWords * 4, c->stream));
   SDS_CU(c, cudaStreamSynchronize(c->stream));
   c->state = kBound;
@@ -507,7 +584,7 @@ int sds_reset(sds_ctx* c) {
   WinArgs A = win_args(c);
   SDS_LAUNCH(c, SDS_PROF_INIT, launch_init(A, c->stream));
   if (c->mode == SDS_FROZEN_PREV) {
-    const int rc = run_denoiser(c, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, c->B, A.Dq);
+    const int rc = run_denoiser(c, c->tgt, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, c->B, A.Dq);
     if (rc != SDS_OK) return rc;
     SDS_LAUNCH(c, SDS_PROF_AUX, launch_after_init(A, c->stream));
   }
@@ -524,11 +601,21 @@ int sds_draft(sds_ctx* c) {
   if (c->mode == SDS_FROZEN_EXACT) {
     // frozen output = target output at (Y_n, t_n): one row per active chain
     SDS_LAUNCH(c, SDS_PROF_DRAFT, launch_gather_state(A, c->ub, c->stream));
-    const int rc = run_denoiser(c, A.X, A.Xb, A.rowk, A.ctl + kCtlNActive, c->ub, A.Dq);
+    const int rc = run_denoiser(c, c->tgt, A.X, A.Xb, A.rowk, A.ctl + kCtlNActive, c->ub, A.Dq);
     if (rc != SDS_OK) return rc;
     SDS_LAUNCH(c, SDS_PROF_DRAFT, launch_scatter_carried(A, c->ub, c->stream));
   }
-  SDS_LAUNCH(c, SDS_PROF_DRAFT, launch_draft(A, c->ub, c->stream));
+  if (c->mode == SDS_INDEPENDENT) {
+    // sequential draft: position j needs the draft model at W_{j-1}
+    for (int j = 1; j <= c->L; ++j) {
+      SDS_LAUNCH(c, SDS_PROF_DRAFT, launch_gather_pos(A, j, c->ub, c->stream));
+      const int rc = run_denoiser(c, c->drf, A.Gx, A.Gb, A.Gk, A.ctl + kCtlNActive, c->ub, A.Pb);
+      if (rc != SDS_OK) return rc;
+      SDS_LAUNCH(c, SDS_PROF_DRAFT, launch_draft_pos(A, j, c->ub, c->stream));
+    }
+  } else {
+    SDS_LAUNCH(c, SDS_PROF_DRAFT, launch_draft(A, c->ub, c->stream));
+  }
   c->state = kDrafted;
   return SDS_OK;
 }
@@ -537,7 +624,7 @@ int sds_verify_window(sds_ctx* c) {
   if (!c) return SDS_EINVAL;
   if (c->state != kDrafted) return SDS_ESTATE;
   WinArgs A = win_args(c);
-  const int rc = run_denoiser(c, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, (int64_t)c->ub * c->L, A.Dq);
+  const int rc = run_denoiser(c, c->tgt, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, (int64_t)c->ub * c->L, A.Dq);
   if (rc != SDS_OK) return rc;
   SDS_LAUNCH(c, SDS_PROF_VERIFY, launch_verify(A, c->ub, c->stream));
   c->state = kVerified;
@@ -558,10 +645,10 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
   if (c->state < kBound) return SDS_ESTATE;
   WinArgs A = win_args(c);
   int rc = SDS_OK;
-  if (c->whole_chain && c->mode == SDS_FROZEN_PREV && c->den.kind == SDS_DEN_GMM && fused_small_supported(c->d, c->den.ncomp, c->L)) {
-    if ((rc = ensure_musq(c)) != SDS_OK) return rc;
+  if (c->whole_chain && c->mode == SDS_FROZEN_PREV && c->tgt.den.kind == SDS_DEN_GMM && fused_small_supported(c->d, c->tgt.den.ncomp, c->L)) {
+    if ((rc = ensure_musq(c, c->tgt)) != SDS_OK) return rc;
     SDS_CU(c, cudaMemsetAsync(A.ctl, 0, kCtlWords * 4, c->stream));   // no chain active afterwards, error bits clear
-    SDS_LAUNCH(c, SDS_PROF_FUSED, launch_fused_small(A, gmm_args(c), c->stream));
+    SDS_LAUNCH(c, SDS_PROF_FUSED, launch_fused_small(A, gmm_args(c, c->tgt), c->stream));
     c->ub = 0;
     c->state = kReady;
   } else {
@@ -600,15 +687,15 @@ int sds_sample_all_host(sds_ctx* c, const void* means_host, const float* logw_ho
                         int32_t* nfe_calls_host, int32_t* nfe_rows_host) {
   if (!c || !out_host) return SDS_EINVAL;
   if (c->state < kBound) return SDS_ESTATE;
-  if ((means_host || logw_host) && c->den.kind != SDS_DEN_GMM) return SDS_EINVAL;
+  if ((means_host || logw_host) && c->tgt.den.kind != SDS_DEN_GMM) return SDS_EINVAL;
   if (means_host) {
-    const size_t esz = c->den.means_dtype == SDS_BF16 ? 2 : 4;
-    SDS_CU(c, cudaMemcpyAsync(const_cast<void*>(c->den.means_dev), means_host, (size_t)c->den.ncomp * c->d * esz,
+    const size_t esz = c->tgt.den.means_dtype == SDS_BF16 ? 2 : 4;
+    SDS_CU(c, cudaMemcpyAsync(const_cast<void*>(c->tgt.den.means_dev), means_host, (size_t)c->tgt.den.ncomp * c->d * esz,
                               cudaMemcpyHostToDevice, c->stream));
-    c->musq_ready = false;
+    c->tgt.musq_ready = false;
   }
   if (logw_host)
-    SDS_CU(c, cudaMemcpyAsync(const_cast<float*>(c->den.logw_dev), logw_host, (size_t)c->den.ncomp * 4,
+    SDS_CU(c, cudaMemcpyAsync(const_cast<float*>(c->tgt.den.logw_dev), logw_host, (size_t)c->tgt.den.ncomp * 4,
                               cudaMemcpyHostToDevice, c->stream));
   WinArgs A = win_args(c);
   const int rc = sds_sample_all(c, A.Y, nullptr, nullptr);
@@ -646,6 +733,9 @@ int sds_get(sds_ctx* c, int32_t what, void* dst, size_t bytes, int32_t dst_is_ho
     case SDS_GET_NFE_ROWS: off = c->lay.nfe_rows; len = B * 4; break;
     case SDS_GET_CTL: off = c->lay.ctl; len = kCtlWords * 4; break;
     case SDS_GET_ROWK: off = c->lay.rowk; len = rows * 4; break;
+    case SDS_GET_DP:
+      if (c->lay.Dp == kNone) return SDS_EINVAL;
+      off = c->lay.Dp; len = rows * d * 4; break;
     default: return SDS_EINVAL;
   }
   if (bytes > len) return SDS_EINVAL;
@@ -672,7 +762,7 @@ int sds_denoise(sds_ctx* c, const float* x_dev, const int32_t* k_dev, int64_t ro
   if (!c || !x_dev || !k_dev || !out_dev) return SDS_EINVAL;
   if (c->state < kBound) return SDS_ESTATE;
   if (rows < 0 || rows > c->B * c->L) return SDS_EINVAL;
-  return run_denoiser(c, x_dev, nullptr, k_dev, nullptr, rows, out_dev);
+  return run_denoiser(c, c->tgt, x_dev, nullptr, k_dev, nullptr, rows, out_dev);
 }
 
 int sds_rng_normals(uint64_t seed, int32_t stream_id, int64_t b0, int64_t nb, int32_t k, int32_t d, float* out_dev,

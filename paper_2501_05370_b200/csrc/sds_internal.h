@@ -10,7 +10,8 @@ namespace sds {
 // caller's workspace (or the caller's parameter arrays).
 struct WinArgs {
   int B, d, L, K;
-  int exact;             // 1: the drafter's frozen output is recomputed at Y_n before every window
+  int mode;              // 0: carried target output; 1: target output at Y_n, recomputed before every
+                         // window; 2: independent draft model evaluated at every drafted state
   uint64_t seed;
   uint64_t chain_off;
   const float* a;        // [K]
@@ -35,6 +36,12 @@ struct WinArgs {
   int* jstar;            // [B]
   int* nfe_calls;        // [B]
   int* nfe_rows;         // [B]
+  // independent drafter only
+  float* Gx;             // [B, d]   one position's input rows of the draft model, dense over active chains
+  uint16_t* Gb;          // [B, d]   their bf16 copy
+  int* Gk;               // [B]      their transition indices
+  float* Pb;             // [B, d]   the draft model's outputs for that position
+  float* Dp;             // [B*L, d] draft-model output per drafted row (NULL in the frozen modes)
 };
 
 struct GmmArgs {
@@ -52,6 +59,8 @@ cudaError_t launch_compact(const WinArgs& A, cudaStream_t st);
 cudaError_t launch_gather_state(const WinArgs& A, int ub_chains, cudaStream_t st);
 cudaError_t launch_scatter_carried(const WinArgs& A, int ub_chains, cudaStream_t st);
 cudaError_t launch_draft(const WinArgs& A, int ub_chains, cudaStream_t st);
+cudaError_t launch_gather_pos(const WinArgs& A, int j, int ub_chains, cudaStream_t st);
+cudaError_t launch_draft_pos(const WinArgs& A, int j, int ub_chains, cudaStream_t st);
 cudaError_t launch_verify(const WinArgs& A, int ub_chains, cudaStream_t st);
 cudaError_t launch_advance(const WinArgs& A, int ub_chains, cudaStream_t st);
 cudaError_t launch_rng_normals(uint64_t seed, int stream_id, uint64_t b0, int64_t nb, int k, int d, float* out,

@@ -105,8 +105,8 @@ __global__ void __launch_bounds__(kBlock) k_init(WinArgs A) {
   if (t == 0) {
     A.n[b] = 0;
     A.rowk[b] = 0;
-    A.nfe_calls[b] = A.exact ? 0 : 1;      // the carried-output drafter starts with one target call
-    A.nfe_rows[b] = A.exact ? 0 : 1;
+    A.nfe_calls[b] = A.mode == 0 ? 1 : 0;      // the carried-output drafter starts with one target call
+    A.nfe_rows[b] = A.mode == 0 ? 1 : 0;
     A.accmask[b] = 0u;
     A.jstar[b] = 0;
   }
@@ -211,6 +211,87 @@ __global__ void __launch_bounds__(kBlock) k_draft(WinArgs A) {
 }
 
 // ---------------------------------------------------------------------------------------
+// Independent draft model (Eq. 5): the draft mean at position j needs the draft model's output at
+// W_{j-1}, so the window is drafted one position at a time. k_gather_pos collects W_{j-1} of every
+// active chain into dense rows (for j = 1 it also opens the window: W_0 = Y_n and the row indices);
+// the draft model runs on them; k_draft_pos makes W_j and keeps the model's output for verify.
+// Chains whose window is shorter than j contribute a valid dummy row that is never used.
+// ---------------------------------------------------------------------------------------
+template <int TPC, int VEC>
+__global__ void __launch_bounds__(kBlock) k_gather_pos(WinArgs A, int j) {
+  using G = Group<TPC>;
+  const int s = G::slot(), t = G::lane();
+  if (s >= A.ctl[kCtlNActive]) return;
+  const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
+  const int Lt = window_len(A, nb);
+  const int jj = min(j, Lt);
+  const float* src = (j == 1) ? A.Y + (size_t)b * A.d : A.X + (size_t)(r0 + jj - 1) * A.d;
+  const size_t go = (size_t)s * A.d, x0 = (size_t)r0 * A.d;
+  if (t == 0) A.Gk[s] = nb + jj - 1;
+  if (j == 1 && t < Lt) A.rowk[r0 + t] = nb + t;
+  if (VEC == 4) {
+    for (int i = t * 4; i < A.d; i += TPC * 4) {
+      const float4 v = ld4(src + i);
+      const uint2 pk = make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
+      st4(A.Gx + go + i, v);
+      *reinterpret_cast<uint2*>(A.Gb + go + i) = pk;
+      if (j == 1) {
+        st4(A.X + x0 + i, v);
+        if (A.Xb) *reinterpret_cast<uint2*>(A.Xb + x0 + i) = pk;
+      }
+    }
+  } else {
+    for (int i = t; i < A.d; i += TPC) {
+      const float v = src[i];
+      const uint16_t pk = (uint16_t)(pack_bf16x2(v, 0.f) & 0xffffu);
+      A.Gx[go + i] = v;
+      A.Gb[go + i] = pk;
+      if (j == 1) {
+        A.X[x0 + i] = v;
+        if (A.Xb) A.Xb[x0 + i] = pk;
+      }
+    }
+  }
+}
+
+template <int TPC, int VEC>
+__global__ void __launch_bounds__(kBlock) k_draft_pos(WinArgs A, int j) {
+  using G = Group<TPC>;
+  const int s = G::slot(), t = G::lane();
+  if (s >= A.ctl[kCtlNActive]) return;
+  const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
+  const int Lt = window_len(A, nb);
+  if (j > Lt) return;
+  const int k = nb + j - 1;
+  const uint64_t bg = A.chain_off + (uint64_t)b;
+  const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
+  const float* wp = A.X + (size_t)(r0 + j - 1) * A.d;
+  const float* pp = A.Pb + (size_t)s * A.d;
+  float* dp = A.Dp + (size_t)(r0 + j - 1) * A.d;
+  float* dst = (j < Lt) ? A.X + (size_t)(r0 + j) * A.d : A.T + (size_t)b * A.d;
+  uint16_t* dstb = (j < Lt && A.Xb) ? A.Xb + (size_t)(r0 + j) * A.d : nullptr;
+  if (VEC == 4) {
+    for (int i = t * 4; i < A.d; i += TPC * 4) {
+      const float4 y = ld4(wp + i), p = ld4(pp + i);
+      const float4 xi = normal4(A.seed, kStreamDraft, bg, (uint32_t)k, (uint32_t)(i >> 2));
+      const float4 o = make_float4(draft_step(y.x, p.x, xi.x, ak, ck, sk), draft_step(y.y, p.y, xi.y, ak, ck, sk),
+                                   draft_step(y.z, p.z, xi.z, ak, ck, sk), draft_step(y.w, p.w, xi.w, ak, ck, sk));
+      st4(dst + i, o);
+      st4(dp + i, p);
+      if (dstb) *reinterpret_cast<uint2*>(dstb + i) = make_uint2(pack_bf16x2(o.x, o.y), pack_bf16x2(o.z, o.w));
+    }
+  } else {
+    for (int i = t; i < A.d; i += TPC) {
+      const float p = pp[i];
+      const float o = draft_step(wp[i], p, normal1(A.seed, kStreamDraft, bg, (uint32_t)k, (uint32_t)i), ak, ck, sk);
+      dst[i] = o;
+      dp[i] = p;
+      if (dstb) dstb[i] = (uint16_t)(pack_bf16x2(o, 0.f) & 0xffffu);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
 // V1-V5 verify: per position S1 = |Delta|^2, S2 = Delta.Z (double accumulation), log ratio
 // -S1/2 - S2, accept iff log U <= log ratio, first rejection by ballot/ffs, reflection in place
 // ---------------------------------------------------------------------------------------
@@ -237,7 +318,7 @@ __global__ void __launch_bounds__(kBlock) k_verify(WinArgs A) {
     const float* wp = A.X + (size_t)(r0 + j - 1) * A.d;
     const float* wj = (j < Lt) ? A.X + (size_t)(r0 + j) * A.d : A.T + cb;
     const float* dq = A.Dq + (size_t)(r0 + j - 1) * A.d;
-    const float* dc = A.Dc + cb;
+    const float* dc = A.Dp ? A.Dp + (size_t)(r0 + j - 1) * A.d : A.Dc + cb;   // draft model's or frozen output
     double p1 = 0.0, p2 = 0.0;
     if (VEC == 4) {
       for (int i = t * 4; i < A.d; i += TPC * 4) {
@@ -326,7 +407,7 @@ __global__ void __launch_bounds__(kBlock) k_verify(WinArgs A) {
   const float* wp = A.X + (size_t)(r0 + jstar - 1) * A.d;
   float* wj = (jstar < Lt) ? A.X + (size_t)(r0 + jstar) * A.d : A.T + cb;
   const float* dq = A.Dq + (size_t)(r0 + jstar - 1) * A.d;
-  const float* dc = A.Dc + cb;
+  const float* dc = A.Dp ? A.Dp + (size_t)(r0 + jstar - 1) * A.d : A.Dc + cb;
   if (VEC == 4) {
     for (int i = t * 4; i < A.d; i += TPC * 4) {
       const float4 vp = ld4(wp + i), vj = ld4(wj + i), vq = ld4(dq + i), vc = ld4(dc + i);
@@ -389,6 +470,7 @@ __global__ void __launch_bounds__(TPC > kBlock ? TPC : kBlock) k_verify_reg(WinA
       const int i = (t + e * TPC) * 4;
       vj[e] = (i < A.d) ? ld4(wj + i) : zero4;
       vq[e] = (i < A.d) ? ld4(dq + i) : zero4;
+      if (A.Dp && i < A.d) vc[e] = ld4(A.Dp + (size_t)(r0 + j - 1) * A.d + i);   // independent draft model
     }
     double p1 = 0.0, p2 = 0.0;
 #pragma unroll
@@ -472,7 +554,8 @@ __global__ void __launch_bounds__(TPC > kBlock ? TPC : kBlock) k_verify_reg(WinA
   for (int e = 0; e < EPT; ++e) {
     const int i = (t + e * TPC) * 4;
     if (i < A.d) {
-      const float4 p = ld4(wp + i), w = ld4(wj + i), q = ld4(dq + i), c4 = vc[e];
+      const float4 p = ld4(wp + i), w = ld4(wj + i), q = ld4(dq + i);
+      const float4 c4 = A.Dp ? ld4(A.Dp + (size_t)(r0 + jstar - 1) * A.d + i) : vc[e];
       float4 o;
       float D, Z;
       delta_z(p.x, w.x, q.x, c4.x, ak, ck, cs, inv_s, D, Z); o.x = reflect_elem(p.x, q.x, Z, D, ak, ck, sk, coef);
@@ -528,7 +611,7 @@ __global__ void __launch_bounds__(kBlock) k_advance(WinArgs A) {
         A.n[b] = nb + adv;
         // sequential target calls of this window: the batched pass, plus (main-text drafter) the
         // call at Y_n, which is row 1 of the batch (a window of one row is a single call)
-        A.nfe_calls[b] += (A.exact && Lt > 1) ? 2 : 1;
+        A.nfe_calls[b] += (A.mode == 1 && Lt > 1) ? 2 : 1;
         A.nfe_rows[b] += Lt;
       }
     } else if (t == 0) {                              // non-finite log ratio: stop this chain
@@ -613,6 +696,24 @@ cudaError_t launch_scatter_carried(const WinArgs& A, int ub, cudaStream_t st) {
 }
 cudaError_t launch_draft(const WinArgs& A, int ub, cudaStream_t st) {
   SDS_DISPATCH(k_draft, A, ub, st);
+  return cudaGetLastError();
+}
+cudaError_t launch_gather_pos(const WinArgs& A, int j, int ub, cudaStream_t st) {
+  const int tpc = tpc_for(A.d), nb = blocks_for(ub > 0 ? ub : 1, tpc);
+  if (tpc == 32) {
+    if (vec4_ok(A.d)) k_gather_pos<32, 4><<<nb, kBlock, 0, st>>>(A, j); else k_gather_pos<32, 1><<<nb, kBlock, 0, st>>>(A, j);
+  } else {
+    if (vec4_ok(A.d)) k_gather_pos<256, 4><<<nb, kBlock, 0, st>>>(A, j); else k_gather_pos<256, 1><<<nb, kBlock, 0, st>>>(A, j);
+  }
+  return cudaGetLastError();
+}
+cudaError_t launch_draft_pos(const WinArgs& A, int j, int ub, cudaStream_t st) {
+  const int tpc = tpc_for(A.d), nb = blocks_for(ub > 0 ? ub : 1, tpc);
+  if (tpc == 32) {
+    if (vec4_ok(A.d)) k_draft_pos<32, 4><<<nb, kBlock, 0, st>>>(A, j); else k_draft_pos<32, 1><<<nb, kBlock, 0, st>>>(A, j);
+  } else {
+    if (vec4_ok(A.d)) k_draft_pos<256, 4><<<nb, kBlock, 0, st>>>(A, j); else k_draft_pos<256, 1><<<nb, kBlock, 0, st>>>(A, j);
+  }
   return cudaGetLastError();
 }
 cudaError_t launch_verify(const WinArgs& A, int ub, cudaStream_t st) {

@@ -19,7 +19,21 @@ def schedule_for(w):
     return a, c, sigma, tcond
 
 
-def sampler_for(w, *, seed=None, chain_id_offset=0, B=None, device="cuda:0", gmm=None, mlp=None, drafter_mode=None):
+def drafter_for(w, *, gmm=None, mlp=None):
+    """Description of an independent draft model for workload w: a (smaller) mixture or MLP."""
+    if gmm is not None:
+        if w.sampler == "ddpm":
+            tc = sb.gmm_tcond_posterior_mean(sb.ddpm_schedule(w.beta())[3], gmm.comp_std)
+        else:
+            tc = sb.gmm_tcond_grad_energy(w.K, gmm.comp_std)
+        return dict(gmm_means=gmm.means, gmm_logw=gmm.logw, tcond=tc, gmm_bf16=bool(getattr(gmm, "means_bf16", False)))
+    if mlp is not None:
+        return dict(mlp=mlp)
+    raise ValueError("a draft model is required")
+
+
+def sampler_for(w, *, seed=None, chain_id_offset=0, B=None, device="cuda:0", gmm=None, mlp=None, drafter_mode=None,
+                drafter=None):
     a, c, sigma, tcond = schedule_for(w)
     if drafter_mode is None:
         drafter_mode = getattr(w, "drafter_mode", 0)
@@ -29,12 +43,12 @@ def sampler_for(w, *, seed=None, chain_id_offset=0, B=None, device="cuda:0", gmm
         gp = gmm if gmm is not None else w.gmm_params()
         return sb.Sampler(a, c, sigma, B, w.d, w.L, gmm_means=gp.means, gmm_logw=gp.logw, tcond=tcond,
                           gmm_bf16=bool(getattr(gp, "means_bf16", False)), seed=seed,
-                          chain_id_offset=chain_id_offset, drafter_mode=drafter_mode, device=device)
+                          chain_id_offset=chain_id_offset, drafter_mode=drafter_mode, drafter=drafter, device=device)
     if w.denoiser == "mlp":
         mp = mlp if mlp is not None else w.mlp_params()
-        return sb.Sampler(a, c, sigma, B, w.d, w.L, mlp=mp, seed=seed, chain_id_offset=chain_id_offset, drafter_mode=drafter_mode, device=device)
+        return sb.Sampler(a, c, sigma, B, w.d, w.L, mlp=mp, seed=seed, chain_id_offset=chain_id_offset, drafter_mode=drafter_mode, drafter=drafter, device=device)
     if w.denoiser == "phi4":
         p4 = w.phi4
         return sb.Sampler(a, c, sigma, B, w.d, w.L, phi4=(p4["side"], p4["beta"], p4.get("periodic", False)), seed=seed,
-                          chain_id_offset=chain_id_offset, drafter_mode=drafter_mode, device=device)
+                          chain_id_offset=chain_id_offset, drafter_mode=drafter_mode, drafter=drafter, device=device)
     raise NotImplementedError(w.denoiser)

@@ -82,7 +82,7 @@ def test_split_precision_tensor_path_agrees_with_float_alu_path():
 
 # ------------------------------------------------------------------ one window, forced ---
 
-def _window_check(s, w, den, a32, c32, s32, seed, chain_off, stats, chains=None):
+def _window_check(s, w, den, a32, c32, s32, seed, chain_off, stats, chains=None, draft_den=None):
     """Runs draft + verify on the GPU and replays the verification on the GPU's own arrays."""
     B, L, d, K = s.B, s.L, s.d, s.K
     ctl = s.get(sb.GET_CTL)
@@ -94,6 +94,7 @@ def _window_check(s, w, den, a32, c32, s32, seed, chain_off, stats, chains=None)
     s.draft()
     Dc = s.get(sb.GET_DC)            # the frozen output the draft used (recomputed by the draft call in exact mode)
     X, T, rowk = s.get(sb.GET_X), s.get(sb.GET_TAIL), s.get(sb.GET_ROWK)
+    Dp = s.get(sb.GET_DP) if draft_den is not None else None     # independent draft model: output per drafted row
     s.verify_window()
     Dq = s.get(sb.GET_DQ)
     X2, T2 = s.get(sb.GET_X), s.get(sb.GET_TAIL)
@@ -111,14 +112,20 @@ def _window_check(s, w, den, a32, c32, s32, seed, chain_off, stats, chains=None)
         for j in range(1, Lt + 1):
             k = nb + j - 1
             xi = o.normals(seed, o.STREAM_DRAFT, chain_off + int(b), k, d)
-            want = a64[k] * W[j - 1] + c64[k] * Dc[b].astype(np.float64) + s64[k] * xi
+            if draft_den is not None:
+                assert rel_l2(Dp[r0 + j - 1], draft_den(W[j - 1], k)) <= 1e-5
+                dcj = Dp[r0 + j - 1].astype(np.float64)
+            else:
+                dcj = Dc[b].astype(np.float64)
+            want = a64[k] * W[j - 1] + c64[k] * dcj + s64[k] * xi
             assert rel_l2(W[j], want) <= 1e-5
         # target rows
         for j in range(1, Lt + 1):
             assert rel_l2(Dq[r0 + j - 1], den(W[j - 1], nb + j - 1)) <= 1e-5
         lu = np.array([math.log(o.uniform01(seed, chain_off + int(b), nb + j)) for j in range(Lt)])
         assert np.max(np.abs(logU[b, :Lt] - lu)) <= 2e-6
-        v = o.verify_window(W, Dq[r0:r0 + Lt], Dc[b], a64, c64, s64, nb, logU[b, :Lt].astype(np.float64))
+        dc_arg = Dp[r0:r0 + Lt] if draft_den is not None else Dc[b]
+        v = o.verify_window(W, Dq[r0:r0 + Lt], dc_arg, a64, c64, s64, nb, logU[b, :Lt].astype(np.float64))
         amb = np.abs(v["ell"] - logU[b, :Lt]) < BAND
         for j in range(Lt):
             assert ell_close(float(ell[b, j]), float(v["ell"][j])), (b, j, ell[b, j], v["ell"][j])
@@ -140,7 +147,7 @@ def _window_check(s, w, den, a32, c32, s32, seed, chain_off, stats, chains=None)
             # reflection is an isometry about the target mean
             k = nb + js - 1
             m_q = a64[k] * W[js - 1] + c64[k] * Dq[r0 + js - 1].astype(np.float64)
-            m_p = a64[k] * W[js - 1] + c64[k] * Dc[b].astype(np.float64)
+            m_p = a64[k] * W[js - 1] + c64[k] * (Dp[r0 + js - 1] if draft_den is not None else Dc[b]).astype(np.float64)
             assert abs(np.linalg.norm(got - m_q) - np.linalg.norm(W[js] - m_p)) <= 1e-4 * np.linalg.norm(W[js] - m_p) + 1e-6
         # rows other than the reflected one are untouched
         for j in range(Lt + 1):
@@ -156,7 +163,7 @@ def _window_check(s, w, den, a32, c32, s32, seed, chain_off, stats, chains=None)
         adv = min(int(jstar[b]), Lt)
         assert n2[b] == nb + adv
         assert np.array_equal(Y2[b], X2[r0 + adv] if adv < Lt else T2[b])
-        assert np.array_equal(Dc2[b], Dq[r0 + adv - 1])
+        assert np.array_equal(Dc2[b], Dq[r0 + adv - 1])          # carry rule (unused by the other drafters)
     assert na2 == int(np.sum(n2 < K))
     return na2
 
@@ -496,4 +503,68 @@ def test_exact_frozen_drafter_with_window_one_is_the_plain_chain():
     for b in range(8):
         y = o.plain_chain(den, a, c, sig, seed=17, b=b, d=w.d)
         assert rel_l2(out[b], y) <= 1e-4
+    s.close()
+
+
+# ------------------------------------------------------------------ independent drafter ----------
+
+def _cheap_mixture(w, gp, keep):
+    """A cheaper draft model: the first `keep` components, slightly displaced and wider."""
+    return wl.GmmParams(means=(gp.means[:keep] * 1.05).astype(np.float32), logw=np.full(keep, -math.log(keep), np.float32),
+                        comp_std=gp.comp_std * 1.3)
+
+
+def _oracle_cheap(w, cheap):
+    if w.sampler == "ddpm":
+        abar = o.ddpm_affine(w.beta())[3]
+        return lambda x, k: o.gmm_posterior_mean(x, abar[k], cheap.means, cheap.logw, cheap.comp_std)
+    return lambda x, k: o.gmm_grad_energy(x, cheap.means, cheap.logw, cheap.comp_std)
+
+
+@pytest.mark.parametrize("name,B,d,L,K,ncomp,keep", [("cfg2", 40, 64, 8, 60, 16, 6), ("cfg2", 9, 33, 5, 23, 7, 3),
+                                                     ("cfg5", 12, 512, 6, 40, 40, 12)])
+def test_independent_drafter_windows_and_free_run(name, B, d, L, K, ncomp, keep):
+    w = wl.WORKLOADS[name].scaled(B=B, d=d, L=L, K=K)
+    gp = w.gmm_params(d=d, ncomp=ncomp)
+    cheap = _cheap_mixture(w, gp, keep)
+    s = sds.sampler_for(w, gmm=gp, seed=23, drafter=sds.drafter_for(w, gmm=cheap))
+    den, a, c, sig = oracle_setup(w, gmm=gp)
+    dden = _oracle_cheap(w, cheap)
+    a32, c32, s32, _ = sds.schedule_for(w)
+    s.reset()
+    stats = dict(tests=0, band=0, reflected=0)
+    for _ in range(3):
+        _window_check(s, w, den, a32, c32, s32, 23, 0, stats, draft_den=dden)
+    assert stats["band"] <= 2
+    out, calls, rows = [x.cpu().numpy() for x in s.sample_all()]
+    bad = 0
+    for b in range(min(B, 10)):
+        r = o.speculative_chain(den, a, c, sig, L, 23, b, d, mode=o.INDEPENDENT, draft_denoise=dden)
+        ok = r["nfe_calls"] == calls[b] and r["nfe_rows"] == rows[b] and rel_l2(out[b], r["Y"]) <= 1e-4
+        bad += (not ok)
+    assert bad <= 1
+    s.close()
+
+
+def test_independent_drafter_equal_to_target_accepts_everything():
+    w = wl.WORKLOADS["cfg2"].scaled(B=20, K=50)
+    gp = w.gmm_params()
+    s = sds.sampler_for(w, gmm=gp, seed=29, drafter=sds.drafter_for(w, gmm=gp))
+    out, calls, rows = [x.cpu().numpy() for x in s.sample_all()]
+    assert np.all(calls == math.ceil(50 / w.L)) and np.all(rows == 50)
+    den, a, c, sig = oracle_setup(w, gmm=gp)
+    for b in range(6):
+        assert rel_l2(out[b], o.plain_chain(den, a, c, sig, seed=29, b=b, d=w.d)) <= 1e-4
+    s.close()
+
+
+def test_independent_mlp_drafter_for_mlp_target_runs():
+    dims, ddims = [256, 384, 384, 256], [256, 128, 256]
+    w = wl.WORKLOADS["cfg3"].scaled(d=256, B=64, L=4, K=24, mlp_dims=dims)
+    mp = w.mlp_params()
+    dmp = wl.mlp_params(77, ddims, 24)
+    s = sds.sampler_for(w, mlp=mp, seed=5, drafter=sds.drafter_for(w, mlp=dmp))
+    out, calls, rows = [x.cpu().numpy() for x in s.sample_all()]
+    assert np.all(np.isfinite(out)) and np.array_equal(s.get(sb.GET_N), np.full(64, 24))
+    assert np.all(calls >= 6) and np.all(calls <= 24) and np.all(rows >= 24)
     s.close()
