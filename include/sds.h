@@ -201,6 +201,12 @@ int sds_sample_all(sds_ctx* ctx, float* out_dev, int32_t* nfe_calls_dev, int32_t
 #define SDS_OPT_TENSOR_SPLIT 2
 int sds_set_option(sds_ctx* ctx, int32_t option, int64_t value);
 
+/* Temperature of the accept test (Appendix D, temperature rejection): a draft is accepted iff
+ * log U <= (log ratio) / tau; the reflection is unchanged. tau = 1 (default) is the exact method;
+ * tau > 1 accepts more and moves the output toward the draft model, tau < 1 the other way: the
+ * samples then no longer follow the target law exactly. SDS_GET_ELL returns the tempered value. */
+int sds_set_temperature(sds_ctx* ctx, double tau);
+
 /* Same with host buffers: copies the mixture parameters means_host [ncomp, d] (float or bf16, the
  * dtype named at create) and logw_host [ncomp] (float) to the device arrays named at create
  * (NULL = keep what is on the device), runs sds_sample_all, copies the results to host memory.

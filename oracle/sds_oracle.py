@@ -292,15 +292,18 @@ def log_ratio_expanded(Z: np.ndarray, Delta: np.ndarray) -> float:
     return float(-0.5 * np.dot(Delta + 2.0 * Z, Delta))
 
 
-def rejection_reflection(m_p, m_q, sigma, y_tilde, U):
+def rejection_reflection(m_p, m_q, sigma, y_tilde, U, tau=1.0):
     """Algorithm 3: reflection maximal coupling of N(m^p, sigma^2 I) and N(m^q, sigma^2 I).
-    Returns (Y, accept, log_ratio). Delta = 0 accepts (ratio 1; e is never needed)."""
+    Returns (Y, accept, log_ratio). Delta = 0 accepts (ratio 1; e is never needed).
+    tau != 1 is the temperature variant (Algorithm 6): the accept test compares U with
+    N(Z + Delta; 0, tau I) / N(Z; 0, tau I) = ratio^(1/tau); the reflection is unchanged and the
+    output law is no longer exactly the target's. The returned log ratio is the tempered one."""
     m_p = np.asarray(m_p, dtype=np.float64)
     m_q = np.asarray(m_q, dtype=np.float64)
     y_tilde = np.asarray(y_tilde, dtype=np.float64)
     Delta = (m_p - m_q) / sigma
     Z = (y_tilde - m_p) / sigma
-    ell = log_ratio_expanded(Z, Delta)
+    ell = log_ratio_expanded(Z, Delta) / tau
     nrm2 = float(np.dot(Delta, Delta))
     accept = (nrm2 < 1e-30) or (math.log(U) <= min(0.0, ell))
     if accept:
@@ -323,7 +326,7 @@ def rejection_incorrect_gaussian(m_p, m_q, sigma, y_tilde, U, fresh_normal):
 # ----------------------------------------------------------------------------------------
 
 
-def verify_window(W, Dq, D_c, a, c, sigma, n, logU, decide_f32=True):
+def verify_window(W, Dq, D_c, a, c, sigma, n, logU, decide_f32=True, tau=1.0):
     """The verification loop of Algorithm 4 for one chain on given arrays.
 
     W   [Lt+1, d]  W[0] = Y_n, W[j] = drafted state for transition k = n+j-1
@@ -356,7 +359,7 @@ def verify_window(W, Dq, D_c, a, c, sigma, n, logU, decide_f32=True):
         Z = (W[j] - m_p) / sigma[k]
         S1[j - 1] = np.dot(Delta, Delta)
         S2[j - 1] = np.dot(Delta, Z)
-        ell[j - 1] = log_ratio_expanded(Z, Delta)
+        ell[j - 1] = log_ratio_expanded(Z, Delta) / tau          # tau = 1: the exact method
         if decide_f32:
             ok = np.float32(logU[j - 1]) <= np.float32(ell[j - 1])
         else:
@@ -375,7 +378,7 @@ INDEPENDENT = 2     # a second, cheaper model proposes every draft step (Eq. 5)
 
 
 def speculative_chain(denoise, a, c, sigma, L, seed, b, d, mode=FROZEN_PREV, Y0=None,
-                      record=False, decide_f32=True, draft_denoise=None):
+                      record=False, decide_f32=True, draft_denoise=None, tau=1.0):
     """Algorithm 4 for chain b with the frozen-target drafter, or (mode INDEPENDENT) with the draft
     model draft_denoise(x, k): m^p_k(y) = a_k y + c_k D^p(y, k) evaluated at every drafted state.
 
@@ -422,7 +425,8 @@ def speculative_chain(denoise, a, c, sigma, L, seed, b, d, mode=FROZEN_PREV, Y0=
             nfe_calls += 1
             nfe_rows += Lt - first + 1
         logU = np.array([math.log(uniform01(seed, b, n + j - 1)) for j in range(1, Lt + 1)])
-        v = verify_window(W, Dq, Dp if mode == INDEPENDENT else D_c, a, c, sigma, n, logU, decide_f32=decide_f32)
+        v = verify_window(W, Dq, Dp if mode == INDEPENDENT else D_c, a, c, sigma, n, logU, decide_f32=decide_f32,
+                          tau=tau)
         adv = min(v["jstar"], Lt)
         if v["jstar"] <= Lt:
             W[adv] = v["Y_reflect"]

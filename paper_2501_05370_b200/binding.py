@@ -62,6 +62,7 @@ EXPORTS = {
     "sds_selftest_bounded_wait": (C.c_int, [C.c_int32, C.c_void_p, C.c_void_p]),
     "sds_launch_count": (C.c_int64, [C.c_void_p]),
     "sds_set_option": (C.c_int, [C.c_void_p, C.c_int32, C.c_int64]),
+    "sds_set_temperature": (C.c_int, [C.c_void_p, C.c_double]),
     "sds_profile": (C.c_int, [C.c_void_p, C.c_int32]),
     "sds_profile_read": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32]),
     "sds_gmm_denoise_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
@@ -341,6 +342,9 @@ class Sampler:
 
     def set_option(self, option: int, value: int):
         self._chk(self.lib.sds_set_option(self.h, option, value), "sds_set_option")
+
+    def set_temperature(self, tau: float):
+        self._chk(self.lib.sds_set_temperature(self.h, float(tau)), "sds_set_temperature")
 
     PROF_KINDS = ("init", "denoise", "draft", "verify", "advance", "fused", "aux")
 

@@ -85,6 +85,7 @@ struct sds_ctx {
   int64_t launches = 0;
   int32_t* h_pin = nullptr;         // pinned host words for the window loop
   cudaEvent_t ev[2] = {nullptr, nullptr};
+  double tau = 1.0;                 // temperature of the accept test
   bool whole_chain = true;          // sds_sample_all may use the whole-chain kernel
   bool tensor_split = true;         // float mixtures of tensor-core shape use the 3-way bf16 split
   // optional per-kernel timing: event pairs recorded around each launch, summed on read
@@ -232,6 +233,7 @@ WinArgs win_args(sds_ctx* c) {
   WinArgs A{};
   A.B = (int)c->B; A.d = c->d; A.L = c->L; A.K = c->K;
   A.mode = c->mode;
+  A.inv_tau = 1.0 / c->tau;
   A.seed = c->seed; A.chain_off = (uint64_t)c->chain_off;
   A.a = at<float>(c, c->lay.a); A.c = at<float>(c, c->lay.c); A.sigma = at<float>(c, c->lay.sigma);
   A.Y = at<float>(c, c->lay.Y); A.Dc = at<float>(c, c->lay.Dc); A.T = at<float>(c, c->lay.T);
@@ -796,6 +798,12 @@ int sds_set_option(sds_ctx* c, int32_t option, int64_t value) {
     case SDS_OPT_TENSOR_SPLIT: c->tensor_split = value != 0; return SDS_OK;
     default: return SDS_EINVAL;
   }
+}
+
+int sds_set_temperature(sds_ctx* c, double tau) {
+  if (!c || !(tau > 0.0) || !std::isfinite(tau)) return SDS_EINVAL;
+  c->tau = tau;
+  return SDS_OK;
 }
 
 int sds_profile(sds_ctx* c, int32_t enable) {

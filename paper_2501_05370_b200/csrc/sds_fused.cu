@@ -154,7 +154,7 @@ __global__ void __maxnreg__(72) k_fused_small(WinArgs A, GmmArgs P) {
         myS1 = sS[lane];
         myS2 = sS[kMaxL + lane];
         const float lu = logf(uniform01(A.seed, bg, (uint32_t)(n + lane)));
-        const float ellf = (float)(-0.5 * myS1 - myS2);
+        const float ellf = (float)((-0.5 * myS1 - myS2) * A.inv_tau);   // tempered log ratio (inv_tau = 1: exact method)
         acc = (myS1 < 1e-30) || (lu <= ellf);
         bad = !isfinite(ellf);
       }

@@ -12,6 +12,7 @@ struct WinArgs {
   int B, d, L, K;
   int mode;              // 0: carried target output; 1: target output at Y_n, recomputed before every
                          // window; 2: independent draft model evaluated at every drafted state
+  double inv_tau;        // 1 / temperature of the accept test (1 = the exact method)
   uint64_t seed;
   uint64_t chain_off;
   const float* a;        // [K]

@@ -368,7 +368,7 @@ __global__ void __launch_bounds__(kBlock) k_verify(WinArgs A) {
     if (valid) {
       const float U = uniform01(A.seed, bg, (uint32_t)(nb + lane));
       const float lu = logf(U);
-      const float ellf = (float)(-0.5 * myS1 - myS2);
+      const float ellf = (float)((-0.5 * myS1 - myS2) * A.inv_tau);   // tempered log ratio (inv_tau = 1: exact method)
       acc = (myS1 < 1e-30) || (lu <= ellf);
       bad = !isfinite(ellf);
       const size_t o = (size_t)b * A.L + lane;
@@ -514,7 +514,7 @@ __global__ void __launch_bounds__(TPC > kBlock ? TPC : kBlock) k_verify_reg(WinA
     if (valid) {
       const float U = uniform01(A.seed, bg, (uint32_t)(nb + lane));
       const float lu = logf(U);
-      const float ellf = (float)(-0.5 * myS1 - myS2);
+      const float ellf = (float)((-0.5 * myS1 - myS2) * A.inv_tau);   // tempered log ratio (inv_tau = 1: exact method)
       acc = (myS1 < 1e-30) || (lu <= ellf);
       bad = !isfinite(ellf);
       const size_t o = (size_t)b * A.L + lane;

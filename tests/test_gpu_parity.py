@@ -568,3 +568,36 @@ def test_independent_mlp_drafter_for_mlp_target_runs():
     assert np.all(np.isfinite(out)) and np.array_equal(s.get(sb.GET_N), np.full(64, 24))
     assert np.all(calls >= 6) and np.all(calls <= 24) and np.all(rows >= 24)
     s.close()
+
+
+# ------------------------------------------------------------------ temperature variant ----------
+
+@pytest.mark.parametrize("tau", [0.5, 2.0])
+def test_temperature_variant_matches_oracle(tau):
+    w = wl.WORKLOADS["cfg2"].scaled(B=64, K=40)
+    gp = w.gmm_params()
+    den, a, c, sig = oracle_setup(w, gmm=gp)
+    res = {}
+    for fused in (1, 0):
+        s = sds.sampler_for(w, gmm=gp, seed=37)
+        s.set_temperature(tau)
+        s.set_option(s.OPT_WHOLE_CHAIN_KERNEL, fused)
+        res[fused] = [x.cpu().numpy() for x in s.sample_all()]
+        if not fused:                                   # tempered log ratio is what the library reports
+            s.reset(); s.draft(); s.verify_window()
+            ell, S1, S2 = s.get(sb.GET_ELL), s.get(sb.GET_S1), s.get(sb.GET_S2)
+            assert np.allclose(ell, (-0.5 * S1 - S2) / tau, rtol=1e-6, atol=1e-6)
+        s.close()
+    assert all(np.array_equal(x, y) for x, y in zip(res[0], res[1]))
+    out, calls, rows = res[1]
+    bad = 0
+    for b in range(12):
+        r = o.speculative_chain(den, a, c, sig, w.L, 37, b, w.d, tau=tau)
+        bad += not (r["nfe_calls"] == calls[b] and r["nfe_rows"] == rows[b] and rel_l2(out[b], r["Y"]) <= 1e-4)
+    assert bad <= 1
+    # a higher temperature accepts more
+    if tau > 1:
+        s = sds.sampler_for(w, gmm=gp, seed=37)
+        base = s.sample_all()[1].cpu().numpy()
+        assert calls.mean() < base.mean()
+        s.close()

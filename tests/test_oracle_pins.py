@@ -532,3 +532,45 @@ def test_independent_drafter_keeps_the_target_law():
     # and the draft model alone does NOT have that law (the test above is not vacuous)
     Q = np.array([o.plain_chain(cheap, a, c, sig, seed=5, b=b, d=2) for b in range(N)])
     assert _mmd_perm_pvalue(Q, P, np.random.default_rng(2)) < 0.01
+
+
+# ------------------------------------------------------------------ temperature variant ----------
+
+def _tempered_accept_prob(delta, tau):
+    """E[min(1, exp(l / tau))] for l ~ N(-delta^2/2, delta^2): X = l/tau ~ N(mu, s^2),
+    P = Phi(mu/s) + exp(mu + s^2/2) Phi(-(mu + s^2)/s)."""
+    mu, s = -delta ** 2 / (2 * tau), delta / tau
+    return stats.norm.cdf(mu / s) + math.exp(mu + s * s / 2) * stats.norm.cdf(-(mu + s * s) / s)
+
+
+@pytest.mark.parametrize("tau", [0.5, 2.0, 8.0])
+def test_temperature_accept_probability_and_mean_shift(tau):
+    g = GOLD["fig_temperature"]                       # draft mean 1, target mean 3, std 0.5
+    m_p, m_q, s = np.array([g["m_p"]]), np.array([g["m_q"]]), g["sigma"]
+    delta = abs(g["m_p"] - g["m_q"]) / s
+    assert abs(_tempered_accept_prob(delta, 1.0) - (2 - 2 * stats.norm.cdf(delta / 2))) < 1e-12
+    rng = np.random.default_rng(int(tau * 10))
+    N = 80_000
+    acc = 0
+    ys = np.empty(N)
+    for i in range(N):
+        y = m_p + s * rng.standard_normal(1)
+        Y, a_, _ = o.rejection_reflection(m_p, m_q, s, y, 1.0 - rng.random(), tau=tau)
+        acc += a_
+        ys[i] = Y[0]
+    p = _tempered_accept_prob(delta, tau)
+    assert abs(acc / N - p) < 4 * math.sqrt(p * (1 - p) / N) + 1e-4
+    # Proposition "link with guidance": the output mean moves toward the draft mean for tau > 1
+    # and away from it for tau < 1 (target mean 3 > draft mean 1)
+    shift = ys.mean() - m_q[0]
+    se = ys.std() / math.sqrt(N)
+    assert (shift < -3 * se) if tau > 1 else (shift > 3 * se)
+
+
+def test_temperature_one_is_the_exact_method_and_large_tau_accepts_the_draft():
+    den, a, c, sig = _cfg1_denoiser(K=20)
+    r1 = o.speculative_chain(den, a, c, sig, L=4, seed=8, b=0, d=2)
+    r2 = o.speculative_chain(den, a, c, sig, L=4, seed=8, b=0, d=2, tau=1.0)
+    assert np.array_equal(r1["Y"], r2["Y"]) and r1["adv"] == r2["adv"]
+    r3 = o.speculative_chain(den, a, c, sig, L=4, seed=8, b=0, d=2, tau=1e9)
+    assert r3["adv"] == [4] * 5                        # every draft accepted
