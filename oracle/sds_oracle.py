@@ -313,6 +313,30 @@ def rejection_reflection(m_p, m_q, sigma, y_tilde, U, tau=1.0):
     return Y, False, ell
 
 
+def rejection_reflection_projected(m_p, m_q, sigma, y_tilde, U, A):
+    """Reflection coupling decided in the image of a matrix A, written in the original space
+    (Appendix F, the algorithm for a full matrix A): with P = A^+ A (the orthogonal projector onto
+    the row space of A), accept iff U <= min(1, exp(-(Delta + 2 Z)^T P Delta / 2)); a rejected draft
+    becomes m^q + sigma (Z - 2 (Z^T P Delta)/(Delta^T P Delta) Delta). For invertible A, P = I and
+    this is Algorithm 3; otherwise the output law is not the target's, but (A Y~, A Y) are maximally
+    coupled. Returns (Y, accept, log_ratio). P Delta = 0 accepts."""
+    m_p = np.asarray(m_p, dtype=np.float64)
+    m_q = np.asarray(m_q, dtype=np.float64)
+    y_tilde = np.asarray(y_tilde, dtype=np.float64)
+    A = np.atleast_2d(np.asarray(A, dtype=np.float64))
+    P = np.linalg.pinv(A) @ A
+    Delta = (m_p - m_q) / sigma
+    Z = (y_tilde - m_p) / sigma
+    PD = P @ Delta
+    ell = -0.5 * float(np.dot(Delta + 2.0 * Z, PD))
+    dPd = float(np.dot(Delta, PD))
+    accept = (dPd < 1e-30) or (math.log(U) <= min(0.0, ell))
+    if accept:
+        return y_tilde.copy(), True, ell
+    Y = m_q + sigma * (Z - 2.0 * (float(np.dot(Z, PD)) / dPd) * Delta)
+    return Y, False, ell
+
+
 def rejection_incorrect_gaussian(m_p, m_q, sigma, y_tilde, U, fresh_normal):
     """Same accept test, but on rejection a fresh draw from N(m^q, sigma^2 I) (biased)."""
     Y, acc, ell = rejection_reflection(m_p, m_q, sigma, y_tilde, U)
@@ -326,7 +350,7 @@ def rejection_incorrect_gaussian(m_p, m_q, sigma, y_tilde, U, fresh_normal):
 # ----------------------------------------------------------------------------------------
 
 
-def verify_window(W, Dq, D_c, a, c, sigma, n, logU, decide_f32=True, tau=1.0):
+def verify_window(W, Dq, D_c, a, c, sigma, n, logU, decide_f32=True, tau=1.0, proj=None):
     """The verification loop of Algorithm 4 for one chain on given arrays.
 
     W   [Lt+1, d]  W[0] = Y_n, W[j] = drafted state for transition k = n+j-1
@@ -337,6 +361,8 @@ def verify_window(W, Dq, D_c, a, c, sigma, n, logU, decide_f32=True, tau=1.0):
     Draft mean m^p = a_k W[j-1] + c_k D_c, target mean m^q = a_k W[j-1] + c_k Dq[j-1].
     decide_f32: compare log U and the log-ratio after rounding both to single precision
     (the precision in which the GPU path stores and compares them).
+    proj: a matrix A [r, d]; the test and the reflection coefficient then use P = A^+ A as in
+    rejection_reflection_projected, and S1 = Delta^T P Delta, S2 = Z^T P Delta.
     Returns dict(S1, S2, ell, acc, jstar, Y_reflect) with jstar in 1..Lt+1 (Lt+1 = all accepted).
     """
     W = np.asarray(W, dtype=np.float64)
@@ -351,12 +377,30 @@ def verify_window(W, Dq, D_c, a, c, sigma, n, logU, decide_f32=True, tau=1.0):
     acc = np.zeros(Lt, dtype=bool)
     jstar = Lt + 1
     Y_reflect = None
+    P = None
+    if proj is not None:
+        Amat = np.atleast_2d(np.asarray(proj, dtype=np.float64))
+        P = np.linalg.pinv(Amat) @ Amat
     for j in range(1, Lt + 1):
         k = n + j - 1
         m_p = a[k] * W[j - 1] + c[k] * D_c[j - 1]
         m_q = a[k] * W[j - 1] + c[k] * Dq[j - 1]
         Delta = (m_p - m_q) / sigma[k]
         Z = (W[j] - m_p) / sigma[k]
+        if P is not None:                                        # ratio decided in the image of A
+            PD = P @ Delta
+            S1[j - 1] = np.dot(Delta, PD)
+            S2[j - 1] = np.dot(Z, PD)
+            ell[j - 1] = -0.5 * np.dot(Delta + 2.0 * Z, PD) / tau
+            if decide_f32:
+                ok = np.float32(logU[j - 1]) <= np.float32(ell[j - 1])
+            else:
+                ok = logU[j - 1] <= ell[j - 1]
+            acc[j - 1] = bool(ok) or S1[j - 1] < 1e-30
+            if not acc[j - 1] and jstar == Lt + 1:
+                jstar = j
+                Y_reflect = m_q + sigma[k] * (Z - 2.0 * (S2[j - 1] / S1[j - 1]) * Delta)
+            continue
         S1[j - 1] = np.dot(Delta, Delta)
         S2[j - 1] = np.dot(Delta, Z)
         ell[j - 1] = log_ratio_expanded(Z, Delta) / tau          # tau = 1: the exact method
@@ -378,7 +422,7 @@ INDEPENDENT = 2     # a second, cheaper model proposes every draft step (Eq. 5)
 
 
 def speculative_chain(denoise, a, c, sigma, L, seed, b, d, mode=FROZEN_PREV, Y0=None,
-                      record=False, decide_f32=True, draft_denoise=None, tau=1.0):
+                      record=False, decide_f32=True, draft_denoise=None, tau=1.0, proj=None):
     """Algorithm 4 for chain b with the frozen-target drafter, or (mode INDEPENDENT) with the draft
     model draft_denoise(x, k): m^p_k(y) = a_k y + c_k D^p(y, k) evaluated at every drafted state.
 
@@ -426,7 +470,7 @@ def speculative_chain(denoise, a, c, sigma, L, seed, b, d, mode=FROZEN_PREV, Y0=
             nfe_rows += Lt - first + 1
         logU = np.array([math.log(uniform01(seed, b, n + j - 1)) for j in range(1, Lt + 1)])
         v = verify_window(W, Dq, Dp if mode == INDEPENDENT else D_c, a, c, sigma, n, logU, decide_f32=decide_f32,
-                          tau=tau)
+                          tau=tau, proj=proj)
         adv = min(v["jstar"], Lt)
         if v["jstar"] <= Lt:
             W[adv] = v["Y_reflect"]

@@ -574,3 +574,85 @@ def test_temperature_one_is_the_exact_method_and_large_tau_accepts_the_draft():
     assert np.array_equal(r1["Y"], r2["Y"]) and r1["adv"] == r2["adv"]
     r3 = o.speculative_chain(den, a, c, sig, L=4, seed=8, b=0, d=2, tau=1e9)
     assert r3["adv"] == [4] * 5                        # every draft accepted
+
+
+# ----------------------------------------------------------------------------------------
+# projected acceptance ratio (Appendix F: the rule for a full matrix A, in the original space)
+# ----------------------------------------------------------------------------------------
+
+
+def test_projected_rule_with_invertible_matrix_is_algorithm_3():
+    rng = np.random.default_rng(77)
+    for _ in range(50):
+        d = 3
+        A = rng.standard_normal((d, d)) + 2 * np.eye(d)
+        m_p, m_q = rng.standard_normal(d), rng.standard_normal(d)
+        s = 0.7
+        y = m_p + s * rng.standard_normal(d)
+        U = 1.0 - rng.random()
+        Y1, a1, l1 = o.rejection_reflection(m_p, m_q, s, y, U)
+        Y2, a2, l2 = o.rejection_reflection_projected(m_p, m_q, s, y, U, A)
+        assert a1 == a2 and abs(l1 - l2) < 1e-10 and np.allclose(Y1, Y2, atol=1e-10)
+
+
+def test_projected_log_ratio_equals_the_whitened_image_form():
+    # (Delta + 2Z)^T A^+ A Delta = |Z_A + Delta_A|^2 - |Z_A|^2 with v_A = (A A^T)^(-1/2) A v
+    rng = np.random.default_rng(78)
+    A = rng.standard_normal((2, 5))
+    w, V = np.linalg.eigh(A @ A.T)
+    Wh = V @ np.diag(w ** -0.5) @ V.T @ A
+    m_p, m_q = rng.standard_normal(5), rng.standard_normal(5)
+    s = 1.3
+    y = m_p + s * rng.standard_normal(5)
+    _, _, ell = o.rejection_reflection_projected(m_p, m_q, s, y, 0.5, A)
+    Z, D = (y - m_p) / s, (m_p - m_q) / s
+    ZA, DA = Wh @ Z, Wh @ D
+    assert abs(ell - (-0.5) * (np.dot(ZA + DA, ZA + DA) - np.dot(ZA, ZA))) < 1e-10
+
+
+def test_projected_rule_couples_the_images_maximally():
+    # accept frequency = 2 - 2 Phi(|Delta_A| / 2) with |Delta_A|^2 = Delta^T A^+ A Delta, and the image
+    # A Y has the image of the target law although Y itself does not follow the target law
+    rng = np.random.default_rng(79)
+    A = np.array([[0.6, 0.8]])                        # one orthonormal row: A Y is a scalar
+    m_p, m_q, s = np.array([0.0, 0.0]), np.array([2.0, -0.5]), 1.0
+    dA = abs((A @ (m_p - m_q))[0]) / s
+    N = 60_000
+    acc = 0
+    img = np.empty(N)
+    for i in range(N):
+        y = m_p + s * rng.standard_normal(2)
+        Y, a_, _ = o.rejection_reflection_projected(m_p, m_q, s, y, 1.0 - rng.random(), A)
+        acc += a_
+        img[i] = (A @ Y)[0]
+    p = 2 - 2 * stats.norm.cdf(dA / 2)
+    assert abs(acc / N - p) < 4 * math.sqrt(p * (1 - p) / N)
+    assert abs(p - (2 - 2 * stats.norm.cdf(np.linalg.norm(m_p - m_q) / 2))) > 0.02   # not the full-space rate
+    assert stats.kstest(img, stats.norm(loc=(A @ m_q)[0], scale=s).cdf).pvalue > 1e-3
+
+
+def test_window_with_projection_follows_the_single_step_rule():
+    rng = np.random.default_rng(80)
+    d, Lt, n = 6, 4, 3
+    K = 12
+    a, c, sig = 0.9 + 0.01 * np.arange(K), 0.05 + 0.01 * np.arange(K), 0.3 + 0.02 * np.arange(K)
+    A = rng.standard_normal((2, d))
+    W = rng.standard_normal((Lt + 1, d))
+    Dq = rng.standard_normal((Lt, d))
+    Dc = rng.standard_normal(d)
+    logU = np.log(1.0 - rng.random(Lt))
+    v = o.verify_window(W, Dq, Dc, a, c, sig, n, logU, decide_f32=False, proj=A)
+    first = None
+    for j in range(1, Lt + 1):
+        k = n + j - 1
+        m_p, m_q = a[k] * W[j - 1] + c[k] * Dc, a[k] * W[j - 1] + c[k] * Dq[j - 1]
+        Y, ok, ell = o.rejection_reflection_projected(m_p, m_q, sig[k], W[j], math.exp(logU[j - 1]), A)
+        assert abs(ell - v["ell"][j - 1]) < 1e-10 and ok == bool(v["acc"][j - 1])
+        if not ok and first is None:
+            first = j
+            assert np.allclose(Y, v["Y_reflect"], atol=1e-10)
+    assert v["jstar"] == (first if first is not None else Lt + 1)
+    # a square invertible matrix changes nothing
+    v0 = o.verify_window(W, Dq, Dc, a, c, sig, n, logU, decide_f32=False)
+    v1 = o.verify_window(W, Dq, Dc, a, c, sig, n, logU, decide_f32=False, proj=rng.standard_normal((d, d)) + 3 * np.eye(d))
+    assert np.allclose(v0["ell"], v1["ell"], atol=1e-9) and v0["jstar"] == v1["jstar"]
