@@ -207,6 +207,17 @@ int sds_set_option(sds_ctx* ctx, int32_t option, int64_t value);
  * samples then no longer follow the target law exactly. SDS_GET_ELL returns the tempered value. */
 int sds_set_temperature(sds_ctx* ctx, double tau);
 
+/* Accept test decided in the image of a matrix A (Appendix F, reflection coupling with a full
+ * matrix, written in the original space): with P = A^+ A the log ratio is -(Delta + 2Z)^T P Delta / 2
+ * and a rejected draft becomes m^q + sigma (Z - 2 (Z^T P Delta)/(Delta^T P Delta) Delta).
+ * Q_dev: device array [r, d] of floats, ORTHONORMAL rows spanning the row space of A (so that
+ * P = Q^T Q; the caller orthonormalises, the library does not check), caller-owned and alive for
+ * as long as it is set; r in [1, d], d <= 16384 (else SDS_EUNSUPPORTED). NULL with r = 0 restores
+ * the full-space test (the exact method). With r < d the samples no longer follow the target law;
+ * the images A Y~ and A Y are maximally coupled. SDS_GET_S1 / SDS_GET_S2 then return
+ * Delta^T P Delta and Z^T P Delta. The whole-chain kernel is not used while a projection is set. */
+int sds_set_projection(sds_ctx* ctx, const float* Q_dev, int32_t r);
+
 /* Same with host buffers: copies the mixture parameters means_host [ncomp, d] (float or bf16, the
  * dtype named at create) and logw_host [ncomp] (float) to the device arrays named at create
  * (NULL = keep what is on the device), runs sds_sample_all, copies the results to host memory.

@@ -63,6 +63,7 @@ EXPORTS = {
     "sds_launch_count": (C.c_int64, [C.c_void_p]),
     "sds_set_option": (C.c_int, [C.c_void_p, C.c_int32, C.c_int64]),
     "sds_set_temperature": (C.c_int, [C.c_void_p, C.c_double]),
+    "sds_set_projection": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32]),
     "sds_profile": (C.c_int, [C.c_void_p, C.c_int32]),
     "sds_profile_read": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32]),
     "sds_gmm_denoise_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
@@ -146,6 +147,15 @@ def gmm_tcond_grad_energy(K: int, comp_std: float) -> np.ndarray:
 # ---------------------------------------------------------------------------------------------
 # sampler object
 # ---------------------------------------------------------------------------------------------
+
+def projection_basis(A: np.ndarray, rtol: float = 1e-10) -> np.ndarray:
+    """Orthonormal rows [r, d] spanning the row space of A (from its singular value decomposition),
+    the form sds_set_projection takes: Q^T Q = A^+ A."""
+    A = np.atleast_2d(np.asarray(A, dtype=np.float64))
+    _, sv, Vt = np.linalg.svd(A, full_matrices=False)
+    r = int(np.sum(sv > rtol * sv.max())) if sv.size else 0
+    return np.ascontiguousarray(Vt[:r], dtype=np.float32)
+
 
 class Sampler:
     """One libsds context with its device buffers.
@@ -345,6 +355,19 @@ class Sampler:
 
     def set_temperature(self, tau: float):
         self._chk(self.lib.sds_set_temperature(self.h, float(tau)), "sds_set_temperature")
+
+    def set_projection(self, Q):
+        """Q: float32 CUDA tensor [r, d] with orthonormal rows (see projection_basis), or None to
+        return to the full-space accept test. The tensor is kept alive by this object."""
+        if Q is None:
+            self._chk(self.lib.sds_set_projection(self.h, None, 0), "sds_set_projection")
+            self._proj = None
+            return
+        t = self.torch
+        if Q.dtype != t.float32 or not Q.is_cuda or Q.dim() != 2 or Q.shape[1] != self.d or not Q.is_contiguous():
+            raise ValueError("Q must be a contiguous float32 CUDA tensor [r, d]")
+        self._chk(self.lib.sds_set_projection(self.h, Q.data_ptr(), int(Q.shape[0])), "sds_set_projection")
+        self._proj = Q
 
     PROF_KINDS = ("init", "denoise", "draft", "verify", "advance", "fused", "aux")
 

@@ -86,6 +86,8 @@ struct sds_ctx {
   int32_t* h_pin = nullptr;         // pinned host words for the window loop
   cudaEvent_t ev[2] = {nullptr, nullptr};
   double tau = 1.0;                 // temperature of the accept test
+  const float* Q = nullptr;         // orthonormal rows of the subspace the ratio is decided in (caller's)
+  int32_t qr = 0;
   bool whole_chain = true;          // sds_sample_all may use the whole-chain kernel
   bool tensor_split = true;         // float mixtures of tensor-core shape use the 3-way bf16 split
   // optional per-kernel timing: event pairs recorded around each launch, summed on read
@@ -246,6 +248,7 @@ WinArgs win_args(sds_ctx* c) {
   A.nfe_calls = at<int>(c, c->lay.nfe_calls); A.nfe_rows = at<int>(c, c->lay.nfe_rows);
   A.Gx = at<float>(c, c->lay.Gx); A.Gb = at<uint16_t>(c, c->lay.Gb); A.Gk = at<int>(c, c->lay.Gk);
   A.Pb = at<float>(c, c->lay.Pb); A.Dp = at<float>(c, c->lay.Dp);
+  A.Q = c->Q; A.qr = c->qr;
   return A;
 }
 
@@ -647,7 +650,7 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
   if (c->state < kBound) return SDS_ESTATE;
   WinArgs A = win_args(c);
   int rc = SDS_OK;
-  if (c->whole_chain && c->mode == SDS_FROZEN_PREV && c->tgt.den.kind == SDS_DEN_GMM && fused_small_supported(c->d, c->tgt.den.ncomp, c->L)) {
+  if (c->whole_chain && !c->Q && c->mode == SDS_FROZEN_PREV && c->tgt.den.kind == SDS_DEN_GMM && fused_small_supported(c->d, c->tgt.den.ncomp, c->L)) {
     if ((rc = ensure_musq(c, c->tgt)) != SDS_OK) return rc;
     SDS_CU(c, cudaMemsetAsync(A.ctl, 0, kCtlWords * 4, c->stream));   // no chain active afterwards, error bits clear
     SDS_LAUNCH(c, SDS_PROF_FUSED, launch_fused_small(A, gmm_args(c, c->tgt), c->stream));
@@ -803,6 +806,14 @@ int sds_set_option(sds_ctx* c, int32_t option, int64_t value) {
 int sds_set_temperature(sds_ctx* c, double tau) {
   if (!c || !(tau > 0.0) || !std::isfinite(tau)) return SDS_EINVAL;
   c->tau = tau;
+  return SDS_OK;
+}
+
+int sds_set_projection(sds_ctx* c, const float* Q_dev, int32_t r) {
+  if (!c || r < 0 || (Q_dev && r == 0) || (!Q_dev && r != 0)) return SDS_EINVAL;
+  if (Q_dev && (r > c->d || c->d > 16384)) return SDS_EUNSUPPORTED;
+  c->Q = Q_dev;
+  c->qr = r;
   return SDS_OK;
 }
 

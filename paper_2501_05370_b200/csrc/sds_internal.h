@@ -43,6 +43,9 @@ struct WinArgs {
   int* Gk;               // [B]      their transition indices
   float* Pb;             // [B, d]   the draft model's outputs for that position
   float* Dp;             // [B*L, d] draft-model output per drafted row (NULL in the frozen modes)
+  // acceptance ratio decided in a subspace (NULL: the full space)
+  const float* Q;        // [qr, d]  orthonormal rows spanning the row space of the projection matrix
+  int qr;
 };
 
 struct GmmArgs {

@@ -292,6 +292,62 @@ __global__ void __launch_bounds__(kBlock) k_draft_pos(WinArgs A, int j) {
 }
 
 // ---------------------------------------------------------------------------------------
+// Ratio decided in a subspace (Appendix F): with P = Q^T Q the orthogonal projector onto the rows
+// of Q, S1 = Delta^T P Delta = sum_i (q_i.Delta)^2 and S2 = Z^T P Delta = sum_i (q_i.Delta)(q_i.Z).
+// One CTA per (active chain, position): Delta and Z of that position are staged in shared memory,
+// then the warps share the rows of Q. Sums in double, combined in a fixed order.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kBlock) k_project(WinArgs A) {
+  extern __shared__ __align__(16) float s_dz[];          // [2][d]
+  __shared__ double s_acc[2 * (kBlock / 32)];
+  const int s = blockIdx.x, j = blockIdx.y + 1;
+  if (s >= A.ctl[kCtlNActive]) return;
+  const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
+  const int Lt = window_len(A, nb);
+  if (j > Lt) return;
+  const int d = A.d, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const size_t cb = (size_t)b * d;
+  const int k = nb + j - 1;
+  const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
+  const float inv_s = 1.0f / sk, cs = ck * inv_s;
+  const float* wp = A.X + (size_t)(r0 + j - 1) * d;
+  const float* wj = (j < Lt) ? A.X + (size_t)(r0 + j) * d : A.T + cb;
+  const float* dq = A.Dq + (size_t)(r0 + j - 1) * d;
+  const float* dc = A.Dp ? A.Dp + (size_t)(r0 + j - 1) * d : A.Dc + cb;
+  float* sD = s_dz;
+  float* sZ = s_dz + d;
+  for (int i = tid; i < d; i += kBlock) {
+    float D, Z;
+    delta_z(wp[i], wj[i], dq[i], dc[i], ak, ck, cs, inv_s, D, Z);
+    sD[i] = D;
+    sZ[i] = Z;
+  }
+  __syncthreads();
+  double t1 = 0.0, t2 = 0.0;
+  for (int r = warp; r < A.qr; r += kBlock / 32) {
+    const float* q = A.Q + (size_t)r * d;
+    double pd = 0.0, pz = 0.0;
+    for (int i = lane; i < d; i += 32) {
+      const double qi = (double)__ldg(q + i);
+      pd = fma(qi, (double)sD[i], pd);
+      pz = fma(qi, (double)sZ[i], pz);
+    }
+    pd = warp_sum(pd);
+    pz = warp_sum(pz);
+    t1 = fma(pd, pd, t1);
+    t2 = fma(pd, pz, t2);
+  }
+  if (lane == 0) { s_acc[warp] = t1; s_acc[kBlock / 32 + warp] = t2; }
+  __syncthreads();
+  if (tid == 0) {
+    double S1 = 0.0, S2 = 0.0;
+    for (int w = 0; w < kBlock / 32; ++w) { S1 += s_acc[w]; S2 += s_acc[kBlock / 32 + w]; }
+    A.S1[(size_t)b * A.L + j - 1] = S1;
+    A.S2[(size_t)b * A.L + j - 1] = S2;
+  }
+}
+
+// ---------------------------------------------------------------------------------------
 // V1-V5 verify: per position S1 = |Delta|^2, S2 = Delta.Z (double accumulation), log ratio
 // -S1/2 - S2, accept iff log U <= log ratio, first rejection by ballot/ffs, reflection in place
 // ---------------------------------------------------------------------------------------
@@ -311,7 +367,12 @@ __global__ void __launch_bounds__(kBlock) k_verify(WinArgs A) {
   const size_t cb = (size_t)b * A.d;
 
   double myS1 = 0.0, myS2 = 0.0;
-  for (int j = 1; j <= Lt; ++j) {
+  const bool projected = A.Q != nullptr;              // S1, S2 already written by k_project
+  if (projected && warp == 0 && lane < Lt) {
+    myS1 = A.S1[(size_t)b * A.L + lane];
+    myS2 = A.S2[(size_t)b * A.L + lane];
+  }
+  for (int j = 1; j <= (projected ? 0 : Lt); ++j) {
     const int k = nb + j - 1;
     const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
     const float inv_s = 1.0f / sk, cs = ck * inv_s;
@@ -350,7 +411,7 @@ __global__ void __launch_bounds__(kBlock) k_verify(WinArgs A) {
       s_red[kMaxL * kWarps + (j - 1) * kWarps + warp] = p2;
     }
   }
-  if (TPC > 32) {
+  if (TPC > 32 && !projected) {
     __syncthreads();
     if (warp == 0 && lane < Lt) {
       for (int w = 0; w < kWarps; ++w) {
@@ -718,6 +779,16 @@ cudaError_t launch_draft_pos(const WinArgs& A, int j, int ub, cudaStream_t st) {
 }
 cudaError_t launch_verify(const WinArgs& A, int ub, cudaStream_t st) {
   const int chains = ub > 0 ? ub : 1;
+  if (A.Q) {                                            // projected sums first, then the shared accept/reflect tail
+    const size_t smem = 2 * (size_t)A.d * sizeof(float);
+    cudaError_t e = cudaFuncSetAttribute(k_project, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    k_project<<<dim3(chains, A.L), kBlock, smem, st>>>(A);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    SDS_DISPATCH(k_verify, A, ub, st);
+    return cudaGetLastError();
+  }
   if (vec4_ok(A.d)) {
     if (A.d <= 256) {
       k_verify_reg<32, 2><<<blocks_for(chains, 32), kBlock, 0, st>>>(A);
@@ -725,6 +796,7 @@ cudaError_t launch_verify(const WinArgs& A, int ub, cudaStream_t st) {
     }
     if (A.d <= 1024) { k_verify_reg<256, 1><<<chains, 256, 0, st>>>(A); return cudaGetLastError(); }
     if (A.d <= 2048) { k_verify_reg<256, 2><<<chains, 256, 0, st>>>(A); return cudaGetLastError(); }
+    if (A.d <= 3072) { k_verify_reg<256, 3><<<chains, 256, 0, st>>>(A); return cudaGetLastError(); }
     if (A.d <= 4096) { k_verify_reg<512, 2><<<chains, 512, 0, st>>>(A); return cudaGetLastError(); }
     if (A.d <= 8192) { k_verify_reg<1024, 2><<<chains, 1024, 0, st>>>(A); return cudaGetLastError(); }
     if (A.d <= 16384) { k_verify_reg<1024, 4><<<chains, 1024, 0, st>>>(A); return cudaGetLastError(); }

@@ -82,7 +82,7 @@ def test_split_precision_tensor_path_agrees_with_float_alu_path():
 
 # ------------------------------------------------------------------ one window, forced ---
 
-def _window_check(s, w, den, a32, c32, s32, seed, chain_off, stats, chains=None, draft_den=None):
+def _window_check(s, w, den, a32, c32, s32, seed, chain_off, stats, chains=None, draft_den=None, proj=None):
     """Runs draft + verify on the GPU and replays the verification on the GPU's own arrays."""
     B, L, d, K = s.B, s.L, s.d, s.K
     ctl = s.get(sb.GET_CTL)
@@ -125,11 +125,13 @@ def _window_check(s, w, den, a32, c32, s32, seed, chain_off, stats, chains=None,
         lu = np.array([math.log(o.uniform01(seed, chain_off + int(b), nb + j)) for j in range(Lt)])
         assert np.max(np.abs(logU[b, :Lt] - lu)) <= 2e-6
         dc_arg = Dp[r0:r0 + Lt] if draft_den is not None else Dc[b]
-        v = o.verify_window(W, Dq[r0:r0 + Lt], dc_arg, a64, c64, s64, nb, logU[b, :Lt].astype(np.float64))
+        v = o.verify_window(W, Dq[r0:r0 + Lt], dc_arg, a64, c64, s64, nb, logU[b, :Lt].astype(np.float64), proj=proj)
         amb = np.abs(v["ell"] - logU[b, :Lt]) < BAND
         for j in range(Lt):
             assert ell_close(float(ell[b, j]), float(v["ell"][j])), (b, j, ell[b, j], v["ell"][j])
             assert abs(S1[b, j] - v["S1"][j]) <= 1e-5 * max(v["S1"][j], 1e-12) + 1e-12
+            if proj is not None:
+                assert abs(S2[b, j] - v["S2"][j]) <= 1e-5 * math.sqrt(max(v["S1"][j], 1e-12)) * 8 + 1e-9
             gacc = bool((int(accmask[b]) >> j) & 1)
             stats["tests"] += 1
             if amb[j]:
@@ -144,6 +146,8 @@ def _window_check(s, w, den, a32, c32, s32, seed, chain_off, stats, chains=None,
             got = X2[r0 + js] if js < Lt else T2[b]
             assert rel_l2(got, v["Y_reflect"]) <= 1e-5
             stats["reflected"] += 1
+            if proj is not None:
+                continue
             # reflection is an isometry about the target mean
             k = nb + js - 1
             m_q = a64[k] * W[js - 1] + c64[k] * Dq[r0 + js - 1].astype(np.float64)
@@ -601,3 +605,63 @@ def test_temperature_variant_matches_oracle(tau):
         base = s.sample_all()[1].cpu().numpy()
         assert calls.mean() < base.mean()
         s.close()
+
+
+# ----------------------------------------------------------------------------------------
+# acceptance ratio decided in a subspace (Appendix F)
+# ----------------------------------------------------------------------------------------
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("d,r", [(64, 5), (1030, 7), (3072, 16)])
+def test_projected_ratio_matches_oracle(d, r):
+    import torch
+    w = wl.WORKLOADS["cfg2"].scaled(B=24, d=d, K=24, L=6)
+    gp = w.gmm_params(d=d)
+    den, a, c, sig = oracle_setup(w, gmm=gp)
+    a32, c32, s32 = [np.asarray(v, dtype=np.float32) for v in (a, c, sig)]
+    A = np.random.default_rng(5).standard_normal((r, d))
+    Q = sb.projection_basis(A)
+    assert Q.shape == (r, d) and np.allclose(Q @ Q.T, np.eye(r), atol=1e-5)
+    s = sds.sampler_for(w, gmm=gp, seed=41)
+    s.set_projection(torch.from_numpy(Q).cuda())
+    stats = dict(tests=0, band=0, reflected=0)
+    s.reset()
+    for _ in range(4):
+        _window_check(s, w, den, a32, c32, s32, 41, 0, stats, chains=set(range(8)), proj=A)
+    assert stats["reflected"] >= 1 and stats["band"] <= 2
+    # whole run against the oracle's chain with the same matrix
+    out, calls, rows = [x.cpu().numpy() for x in s.sample_all()]
+    bad = 0
+    for b in range(6):
+        ref = o.speculative_chain(den, a, c, sig, w.L, 41, b, d, proj=A)
+        bad += not (ref["nfe_calls"] == calls[b] and ref["nfe_rows"] == rows[b] and rel_l2(out[b], ref["Y"]) <= 1e-4)
+    assert bad <= 1
+    # deciding in a low-dimensional image accepts more than the full-space test
+    s.set_projection(None)
+    full = s.sample_all()[1].cpu().numpy()
+    assert calls.mean() < full.mean()
+    s.close()
+
+
+@pytest.mark.gpu
+def test_projection_onto_the_whole_space_is_the_exact_method():
+    import torch
+    w = wl.WORKLOADS["cfg2"].scaled(B=32, K=30)
+    gp = w.gmm_params()
+    s = sds.sampler_for(w, gmm=gp, seed=43)
+    s.set_option(s.OPT_WHOLE_CHAIN_KERNEL, 0)
+    base = [x.cpu().numpy() for x in s.sample_all()]
+    Q = sb.projection_basis(np.random.default_rng(6).standard_normal((w.d, w.d)))
+    s.set_projection(torch.from_numpy(Q).cuda())
+    s.reset(); s.draft(); s.verify_window()
+    S1p, S2p = s.get(sb.GET_S1), s.get(sb.GET_S2)
+    s.set_projection(None)
+    s.reset(); s.draft(); s.verify_window()
+    S1, S2 = s.get(sb.GET_S1), s.get(sb.GET_S2)
+    assert np.allclose(S1p, S1, rtol=1e-4, atol=1e-9) and np.allclose(S2p, S2, rtol=1e-3, atol=1e-5)
+    s.set_projection(torch.from_numpy(Q).cuda())
+    got = [x.cpu().numpy() for x in s.sample_all()]
+    same = np.sum(got[1] == base[1])
+    assert same >= w.B - 2                              # decisions can differ only inside the rounding band
+    s.close()
