@@ -17,6 +17,8 @@ What each function follows:
   rejection_incorrect                  the biased rule of Appendix "need for adjusted rejection"
   log_ratio                            log of the acceptance ratio, both printed forms
   verify_window                        the accept/reflect loop of Algorithm 4 on given arrays
+  rejection_reflection_projected       the rule of Appendix F for a matrix A, in the original space
+  ddim_affine, picard_trajectory       deterministic sampler and its Picard iterates (Appendix C)
   speculative_chain                    Algorithm 4 (detailed speculative sampling for DDM) and
                                        Algorithm 5 (Langevin) through the affine form
   plain_chain                          the target chain itself (Eq. 3), no speculation
@@ -137,6 +139,26 @@ def ddpm_affine(beta: np.ndarray):
         sig[k] = math.sqrt(beta[t - 1])
         abar_step[k] = abar[t]
     return a, c, sig, abar_step
+
+
+def ddim_affine(beta: np.ndarray):
+    """Deterministic counterpart of ddpm_affine (the sampler without noise the Picard drafter
+    iterates, Appendix C "parallel sampling"): with the denoiser output D read as x0 and the noise
+    direction (x_t - sqrt(abar_t) D)/sqrt(1 - abar_t) kept,
+        x_{t-1} = sqrt(abar_{t-1}) D + sqrt(1 - abar_{t-1}) (x_t - sqrt(abar_t) D)/sqrt(1 - abar_t)
+                = abar_det_k x_t + cbar_det_k D,
+        abar_det_k = sqrt((1 - abar_{t-1})/(1 - abar_t)),  cbar_det_k = sqrt(abar_{t-1}) - abar_det_k sqrt(abar_t),
+    t = K - k. Returns (a_det, c_det)."""
+    beta = np.asarray(beta, dtype=np.float64)
+    K = beta.shape[0]
+    abar = np.concatenate([[1.0], np.cumprod(1.0 - beta)])
+    a_det = np.empty(K)
+    c_det = np.empty(K)
+    for k in range(K):
+        t = K - k
+        a_det[k] = math.sqrt((1.0 - abar[t - 1]) / (1.0 - abar[t]))
+        c_det[k] = math.sqrt(abar[t - 1]) - a_det[k] * math.sqrt(abar[t])
+    return a_det, c_det
 
 
 def ula_affine(K: int, gamma: float):
@@ -350,7 +372,7 @@ def rejection_incorrect_gaussian(m_p, m_q, sigma, y_tilde, U, fresh_normal):
 # ----------------------------------------------------------------------------------------
 
 
-def verify_window(W, Dq, D_c, a, c, sigma, n, logU, decide_f32=True, tau=1.0, proj=None):
+def verify_window(W, Dq, D_c, a, c, sigma, n, logU, decide_f32=True, tau=1.0, proj=None, M_p=None):
     """The verification loop of Algorithm 4 for one chain on given arrays.
 
     W   [Lt+1, d]  W[0] = Y_n, W[j] = drafted state for transition k = n+j-1
@@ -361,14 +383,16 @@ def verify_window(W, Dq, D_c, a, c, sigma, n, logU, decide_f32=True, tau=1.0, pr
     Draft mean m^p = a_k W[j-1] + c_k D_c, target mean m^q = a_k W[j-1] + c_k Dq[j-1].
     decide_f32: compare log U and the log-ratio after rounding both to single precision
     (the precision in which the GPU path stores and compares them).
+    M_p [Lt, d]    explicit draft means (drafters whose mean is not a_k W[j-1] + c_k D, such as the
+                   Picard drafter); D_c is then ignored
     proj: a matrix A [r, d]; the test and the reflection coefficient then use P = A^+ A as in
     rejection_reflection_projected, and S1 = Delta^T P Delta, S2 = Z^T P Delta.
     Returns dict(S1, S2, ell, acc, jstar, Y_reflect) with jstar in 1..Lt+1 (Lt+1 = all accepted).
     """
     W = np.asarray(W, dtype=np.float64)
     Dq = np.asarray(Dq, dtype=np.float64)
-    D_c = np.asarray(D_c, dtype=np.float64)
     Lt = Dq.shape[0]
+    D_c = np.zeros(Dq.shape[1]) if D_c is None else np.asarray(D_c, dtype=np.float64)
     if D_c.ndim == 1:                      # frozen drafter: one output for the whole window
         D_c = np.broadcast_to(D_c, Dq.shape)
     S1 = np.zeros(Lt)
@@ -383,7 +407,7 @@ def verify_window(W, Dq, D_c, a, c, sigma, n, logU, decide_f32=True, tau=1.0, pr
         P = np.linalg.pinv(Amat) @ Amat
     for j in range(1, Lt + 1):
         k = n + j - 1
-        m_p = a[k] * W[j - 1] + c[k] * D_c[j - 1]
+        m_p = a[k] * W[j - 1] + c[k] * D_c[j - 1] if M_p is None else np.asarray(M_p[j - 1], dtype=np.float64)
         m_q = a[k] * W[j - 1] + c[k] * Dq[j - 1]
         Delta = (m_p - m_q) / sigma[k]
         Z = (W[j] - m_p) / sigma[k]
@@ -419,12 +443,43 @@ def verify_window(W, Dq, D_c, a, c, sigma, n, logU, decide_f32=True, tau=1.0, pr
 FROZEN_PREV = 0     # carry the latest target output on the accepted trajectory (no extra call)
 FROZEN_EXACT = 1    # evaluate the target at Y_n before drafting (main-text frozen drafter)
 INDEPENDENT = 2     # a second, cheaper model proposes every draft step (Eq. 5)
+PICARD = 3          # draft means from Picard iterations of the deterministic sampler (Appendix C)
+
+
+def picard_trajectory(denoise, a_det, c_det, Y, D_c, n, Lt, iters):
+    """Picard iterates of the deterministic sampler over one window (Appendix C, parallel sampling
+    as drafting). Points F_0 .. F_{Lt-1}, F_0 = Y_n throughout. Start: the deterministic rollout
+    with the carried output frozen, F^0_{j+1} = a_det F^0_j + c_det D_c (the paper leaves the
+    deterministic start free). Each iteration evaluates the target at all points of the previous
+    iterate in one batch and shifts: F^m_{j+1} = a_det_k F^{m-1}_j + c_det_k D(F^{m-1}_j, k),
+    k = n + j. After m iterations the first m+1 points equal the sequential deterministic chain.
+    Returns F [Lt, d]."""
+    Y = np.asarray(Y, dtype=np.float64)
+    F = np.empty((Lt, Y.shape[0]))
+    F[0] = Y
+    for j in range(Lt - 1):
+        F[j + 1] = a_det[n + j] * F[j] + c_det[n + j] * D_c
+    for _ in range(iters):
+        D = [denoise(F[j], n + j) for j in range(Lt - 1)]          # one batched target call
+        Fn = F.copy()
+        for j in range(Lt - 1):
+            Fn[j + 1] = a_det[n + j] * F[j] + c_det[n + j] * D[j]
+        F = Fn
+    return F
 
 
 def speculative_chain(denoise, a, c, sigma, L, seed, b, d, mode=FROZEN_PREV, Y0=None,
-                      record=False, decide_f32=True, draft_denoise=None, tau=1.0, proj=None):
+                      record=False, decide_f32=True, draft_denoise=None, tau=1.0, proj=None, picard=None):
     """Algorithm 4 for chain b with the frozen-target drafter, or (mode INDEPENDENT) with the draft
     model draft_denoise(x, k): m^p_k(y) = a_k y + c_k D^p(y, k) evaluated at every drafted state.
+
+    mode PICARD with picard = (p, a_det, c_det): p >= 1 parallel target calls per window build the
+    draft. p - 1 Picard iterations (picard_trajectory) give points F_0..F_{Lt-1}; the last call
+    evaluates the target there and the draft mean of position j is the stochastic sampler's step
+    from F_{j-1}: m^p_j = a_k F_{j-1} + c_k D(F_{j-1}, k), k = n+j-1, independent of the earlier
+    drafted states. Since F_0 = Y_n, position 1 is drafted from the target itself and its target
+    output is already known; the verify call evaluates positions 2..Lt. The carried output (start
+    of the next window's Picard sequence) follows the FROZEN_PREV rule.
 
     denoise(x, k) -> D; transition means are a_k y + c_k D, std sigma_k.
     Returns dict(Y, nfe_calls, nfe_rows, adv (list), windows (list of per-window records if record)).
@@ -435,7 +490,7 @@ def speculative_chain(denoise, a, c, sigma, L, seed, b, d, mode=FROZEN_PREV, Y0=
     nfe_calls = 0
     nfe_rows = 0
     D_c = None
-    if mode == FROZEN_PREV:
+    if mode in (FROZEN_PREV, PICARD):
         D_c = denoise(Y, 0)               # the one initial call
         nfe_calls += 1
         nfe_rows += 1
@@ -455,10 +510,29 @@ def speculative_chain(denoise, a, c, sigma, L, seed, b, d, mode=FROZEN_PREV, Y0=
             first = 2
         xi = np.empty((Lt, d))
         Dp = np.empty((Lt, d)) if mode == INDEPENDENT else None
+        Mp = None
+        if mode == PICARD:
+            p_calls, a_det, c_det = picard
+            F = picard_trajectory(denoise, a_det, c_det, Y, D_c, n, Lt, p_calls - 1)
+            if Lt >= 2:
+                nfe_calls += p_calls - 1
+                nfe_rows += (p_calls - 1) * (Lt - 1)
+            Mp = np.empty((Lt, d))
+            for j in range(1, Lt + 1):     # last parallel call: the target at every Picard point
+                k = n + j - 1
+                DF = denoise(F[j - 1], k)
+                if j == 1:
+                    Dq[0] = DF             # F_0 = Y_n = W_0: this is the target output of position 1
+                Mp[j - 1] = a[k] * F[j - 1] + c[k] * DF
+            nfe_calls += 1
+            nfe_rows += Lt
+            first = 2
         for j in range(1, Lt + 1):         # sequential draft
             k = n + j - 1
             xi[j - 1] = normals(seed, STREAM_DRAFT, b, k, d)
-            if mode == INDEPENDENT:
+            if mode == PICARD:
+                W[j] = Mp[j - 1] + sigma[k] * xi[j - 1]
+            elif mode == INDEPENDENT:
                 Dp[j - 1] = draft_denoise(W[j - 1], k)
                 W[j] = a[k] * W[j - 1] + c[k] * Dp[j - 1] + sigma[k] * xi[j - 1]
             else:
@@ -470,13 +544,13 @@ def speculative_chain(denoise, a, c, sigma, L, seed, b, d, mode=FROZEN_PREV, Y0=
             nfe_rows += Lt - first + 1
         logU = np.array([math.log(uniform01(seed, b, n + j - 1)) for j in range(1, Lt + 1)])
         v = verify_window(W, Dq, Dp if mode == INDEPENDENT else D_c, a, c, sigma, n, logU, decide_f32=decide_f32,
-                          tau=tau, proj=proj)
+                          tau=tau, proj=proj, M_p=Mp)
         adv = min(v["jstar"], Lt)
         if v["jstar"] <= Lt:
             W[adv] = v["Y_reflect"]
         if record:
             windows.append(dict(n=n, W=W.copy(), Dq=Dq.copy(), D_c=(Dp if mode == INDEPENDENT else D_c).copy(),
-                                logU=logU, xi=xi, **v))
+                                logU=logU, xi=xi, M_p=None if Mp is None else Mp.copy(), **v))
         Y = W[adv].copy()
         D_c = Dq[adv - 1].copy()
         n += adv

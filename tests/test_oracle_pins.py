@@ -656,3 +656,82 @@ def test_window_with_projection_follows_the_single_step_rule():
     v0 = o.verify_window(W, Dq, Dc, a, c, sig, n, logU, decide_f32=False)
     v1 = o.verify_window(W, Dq, Dc, a, c, sig, n, logU, decide_f32=False, proj=rng.standard_normal((d, d)) + 3 * np.eye(d))
     assert np.allclose(v0["ell"], v1["ell"], atol=1e-9) and v0["jstar"] == v1["jstar"]
+
+
+# ----------------------------------------------------------------------------------------
+# Picard drafter (Appendix C: parallel sampling as drafting)
+# ----------------------------------------------------------------------------------------
+
+
+def test_deterministic_sampler_keeps_the_noise_direction():
+    # if x_t = sqrt(abar_t) x0 + sqrt(1 - abar_t) eps and the denoiser returns x0, one deterministic
+    # step lands on sqrt(abar_{t-1}) x0 + sqrt(1 - abar_{t-1}) eps with the same eps
+    K = 25
+    beta = wl.beta_cosine(K)
+    a_det, c_det = o.ddim_affine(beta)
+    abar = np.concatenate([[1.0], np.cumprod(1 - beta)])
+    rng = np.random.default_rng(3)
+    x0, eps = rng.standard_normal(4), rng.standard_normal(4)
+    for k in range(K):
+        t = K - k
+        xt = math.sqrt(abar[t]) * x0 + math.sqrt(1 - abar[t]) * eps
+        want = math.sqrt(abar[t - 1]) * x0 + math.sqrt(1 - abar[t - 1]) * eps
+        assert np.allclose(a_det[k] * xt + c_det[k] * x0, want, atol=1e-12)
+
+
+def test_picard_iterates_reach_the_sequential_deterministic_chain():
+    den, a, c, sig = _cfg1_denoiser(K=30)
+    a_det, c_det = o.ddim_affine(wl.beta_linear(30))
+    rng = np.random.default_rng(4)
+    Y, Dc, n, Lt = rng.standard_normal(2), rng.standard_normal(2), 5, 6
+    seq = np.empty((Lt, 2))
+    seq[0] = Y
+    for j in range(Lt - 1):
+        seq[j + 1] = a_det[n + j] * seq[j] + c_det[n + j] * den(seq[j], n + j)
+    for m in range(Lt):
+        F = o.picard_trajectory(den, a_det, c_det, Y, Dc, n, Lt, m)
+        assert np.allclose(F[:m + 1], seq[:m + 1], atol=1e-12)       # m iterations fix the first m+1 points
+        if m < Lt - 1:
+            assert not np.allclose(F[m + 1], seq[m + 1], atol=1e-6)  # and not yet the next one
+    # no iteration: the rollout with the carried output frozen
+    F0 = o.picard_trajectory(den, a_det, c_det, Y, Dc, n, Lt, 0)
+    assert np.allclose(F0[2], a_det[n + 1] * (a_det[n] * Y + c_det[n] * Dc) + c_det[n + 1] * Dc)
+
+
+def test_picard_drafter_with_window_one_is_the_plain_chain():
+    den, a, c, sig = _cfg1_denoiser(K=20)
+    a_det, c_det = o.ddim_affine(wl.beta_linear(20))
+    for p in (1, 3):
+        r = o.speculative_chain(den, a, c, sig, L=1, seed=17, b=2, d=2, mode=o.PICARD, picard=(p, a_det, c_det))
+        assert r["adv"] == [1] * 20
+        assert r["nfe_calls"] == 1 + 20 and r["nfe_rows"] == 1 + 20   # initial call + one target row per step
+        assert np.array_equal(r["Y"], o.plain_chain(den, a, c, sig, seed=17, b=2, d=2))
+
+
+def test_picard_drafter_counters_and_first_position():
+    den, a, c, sig = _cfg1_denoiser(K=23)
+    a_det, c_det = o.ddim_affine(wl.beta_linear(23))
+    for p in (1, 2, 4):
+        r = o.speculative_chain(den, a, c, sig, L=4, seed=19, b=1, d=2, mode=o.PICARD, picard=(p, a_det, c_det),
+                                record=True)
+        assert sum(r["adv"]) == 23
+        calls, rows = 1, 1
+        for wd in r["windows"]:
+            Lt = wd["Dq"].shape[0]
+            calls += (p - 1 if Lt >= 2 else 0) + 1 + (1 if Lt >= 2 else 0)
+            rows += (p - 1) * (Lt - 1) + Lt + (Lt - 1)
+            assert wd["S1"][0] < 1e-24 and wd["acc"][0]              # position 1 is drafted from the target itself
+        assert (r["nfe_calls"], r["nfe_rows"]) == (calls, rows)
+
+
+def test_picard_drafter_keeps_the_target_law():
+    den, a, c, sig = _cfg1_denoiser(K=40)
+    a_det, c_det = o.ddim_affine(wl.beta_linear(40))
+    N = 400
+    S = np.array([o.speculative_chain(den, a, c, sig, L=4, seed=6, b=b, d=2, mode=o.PICARD, picard=(2, a_det, c_det))["Y"]
+                  for b in range(N)])
+    P = np.array([o.plain_chain(den, a, c, sig, seed=7, b=b, d=2) for b in range(N)])
+    for i in range(2):
+        se = math.sqrt(S[:, i].var() / N + P[:, i].var() / N)
+        assert abs(S[:, i].mean() - P[:, i].mean()) < 4 * se
+    assert _mmd_perm_pvalue(S, P, np.random.default_rng(3)) > 0.01
