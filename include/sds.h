@@ -69,6 +69,9 @@ extern "C" {
 #define SDS_INDEPENDENT   2     /* a second, cheaper model proposes every draft step (Eq. 5); needs
                                    sds_create_with_drafter */
 
+#define SDS_PICARD        3     /* draft means from Picard iterations of the deterministic sampler (Appendix C,
+                                   parallel sampling as drafting); needs sds_create_picard */
+
 #define SDS_GET_X         1     /* float  [nrows, d]  drafted states fed to the target (row r = rowoff[s]+j-1) */
 #define SDS_GET_TAIL      2     /* float  [B, d]      last drafted state of each chain's window */
 #define SDS_GET_DQ        3     /* float  [nrows, d]  target denoiser outputs, same rows as X */
@@ -160,6 +163,22 @@ int sds_workspace_bytes_with_drafter(const sds_schedule* sch, const sds_denoiser
                                      const double* drafter_tcond, int64_t B, int32_t d, int32_t L, size_t* bytes);
 int sds_create_with_drafter(const sds_schedule* sch, const sds_denoiser* den, const sds_denoiser* drafter,
                             const double* drafter_tcond, int64_t B, int32_t d, int32_t L, sds_ctx** out);
+
+/* Picard drafter (Appendix C, "parallel sampling and speculative correction"): per window,
+ * calls >= 1 batched target calls build the draft. Points F_0..F_{Lt-1} of the deterministic
+ * sampler F_{j+1} = a_det[k] F_j + c_det[k] D(F_j, k), k = n+j, F_0 = Y_n, start as the rollout
+ * with the carried target output frozen and are refined by calls-1 Picard iterations (each one
+ * target call on all points of the previous iterate); the last call evaluates the target at the
+ * points and the draft mean of position j is the stochastic step from F_{j-1}:
+ * m^p_j = a_k F_{j-1} + c_k D(F_{j-1}, k), independent of the earlier drafted states. Position 1
+ * is thereby drafted from the target itself and always accepts. a_det, c_det: host arrays [K]
+ * (copied), finite. Bind with SDS_PICARD. Target calls per window: calls + 1 (calls for a window
+ * of one position). SDS_GET_DP returns the draft means per drafted row. The carried output follows
+ * the SDS_FROZEN_PREV rule. sds_sample_all uses the window kernels. */
+int sds_workspace_bytes_picard(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_t d, int32_t L,
+                               size_t* bytes);
+int sds_create_picard(const sds_schedule* sch, const sds_denoiser* den, int32_t calls, const float* a_det,
+                      const float* c_det, int64_t B, int32_t d, int32_t L, sds_ctx** out);
 
 /* Attach workspace, stream (cudaStream_t, may be NULL for the default stream), seed, drafter mode
  * and the global id of local chain 0. Uploads the schedule into the workspace and waits for it. */

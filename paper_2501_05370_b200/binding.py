@@ -21,7 +21,7 @@ SDS_EINVAL, SDS_ESTATE, SDS_ENOMEM, SDS_EUNSUPPORTED = -1, -2, -3, -4
 SDS_ECUDA, SDS_ETIMEOUT, SDS_ENONFINITE, SDS_ECALLBACK = -5, -6, -7, -8
 SDS_DEN_GMM, SDS_DEN_MLP, SDS_DEN_CALLBACK, SDS_DEN_PHI4 = 1, 2, 3, 4
 SDS_F32, SDS_BF16 = 0, 1
-SDS_FROZEN_PREV, SDS_FROZEN_EXACT, SDS_INDEPENDENT = 0, 1, 2
+SDS_FROZEN_PREV, SDS_FROZEN_EXACT, SDS_INDEPENDENT, SDS_PICARD = 0, 1, 2, 3
 (GET_X, GET_TAIL, GET_DQ, GET_DC, GET_Y, GET_N, GET_ACT, GET_ROWOFF, GET_S1, GET_S2, GET_ELL, GET_LOGU,
  GET_ACCMASK, GET_JSTAR, GET_NFE_CALLS, GET_NFE_ROWS, GET_CTL, GET_ROWK, GET_DP) = range(1, 20)
 
@@ -47,6 +47,10 @@ EXPORTS = {
                                                    C.c_int32, C.POINTER(C.c_size_t)]),
     "sds_create_with_drafter": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32,
                                           C.POINTER(C.c_void_p)]),
+    "sds_workspace_bytes_picard": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32,
+                                             C.POINTER(C.c_size_t)]),
+    "sds_create_picard": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int64, C.c_int32,
+                                    C.c_int32, C.POINTER(C.c_void_p)]),
     "sds_bind": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_uint64, C.c_int32, C.c_int64]),
     "sds_reset": (C.c_int, [C.c_void_p]),
     "sds_draft": (C.c_int, [C.c_void_p]),
@@ -124,6 +128,19 @@ def ddpm_schedule(beta: np.ndarray):
     return a.astype(np.float32), c.astype(np.float32), np.sqrt(b_t).astype(np.float32), ab_t
 
 
+def ddim_schedule(beta: np.ndarray):
+    """Coefficients (a_det, c_det) of the deterministic counterpart of ddpm_schedule, the sampler the
+    Picard drafter iterates: x_{t-1} = sqrt(abar_{t-1}) D + sqrt(1 - abar_{t-1}) (x_t - sqrt(abar_t) D)/sqrt(1 - abar_t)."""
+    beta = np.asarray(beta, dtype=np.float64)
+    K = len(beta)
+    abar_full = np.concatenate([[1.0], np.cumprod(1.0 - beta)])
+    t = K - np.arange(K)
+    ab_t, ab_p = abar_full[t], abar_full[t - 1]
+    a_det = np.sqrt((1.0 - ab_p) / (1.0 - ab_t))
+    c_det = np.sqrt(ab_p) - a_det * np.sqrt(ab_t)
+    return a_det.astype(np.float32), c_det.astype(np.float32)
+
+
 def gmm_tcond_posterior_mean(abar: np.ndarray, comp_std: float) -> np.ndarray:
     """(A, Bq, C, E) per step for E[x0 | x_t] of a mixture with shared std s under x_t = al x0 + sqrt(1-al^2) eps:
     v = al^2 s^2 + 1 - al^2;  A = al/v, Bq = -al^2/(2v), C = (1-al^2)/v, E = al s^2/v."""
@@ -166,7 +183,7 @@ class Sampler:
 
     def __init__(self, a, c, sigma, B: int, d: int, L: int, *, gmm_means=None, gmm_logw=None, tcond=None,
                  gmm_bf16: bool = False, mlp=None, callback=None, phi4=None, seed: int = 0, chain_id_offset: int = 0,
-                 drafter_mode: int = 0, drafter=None, device="cuda:0", stream=None):
+                 drafter_mode: int = 0, drafter=None, picard=None, device="cuda:0", stream=None):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("libsds needs a CUDA device; there is no CPU path")
@@ -201,7 +218,21 @@ class Sampler:
         self._sch, self._den, self._dden, self._dtc = sch, den, dden, dtc
         nbytes = C.c_size_t(0)
         h = C.c_void_p()
-        if dden is None:
+        if picard is not None:                   # (calls, a_det, c_det): Picard drafter
+            if dden is not None:
+                raise ValueError("picard and drafter exclude each other")
+            calls, a_det, c_det = picard
+            a_det = np.ascontiguousarray(a_det, np.float32)
+            c_det = np.ascontiguousarray(c_det, np.float32)
+            if a_det.shape != (self.K,) or c_det.shape != (self.K,):
+                raise ValueError("a_det and c_det must have one entry per transition")
+            drafter_mode = SDS_PICARD
+            self._chk(self.lib.sds_workspace_bytes_picard(C.byref(sch), C.byref(den), self.B, self.d, self.L,
+                                                          C.byref(nbytes)), "sds_workspace_bytes_picard")
+            self._chk(self.lib.sds_create_picard(C.byref(sch), C.byref(den), int(calls), a_det.ctypes.data,
+                                                 c_det.ctypes.data, self.B, self.d, self.L, C.byref(h)),
+                      "sds_create_picard")
+        elif dden is None:
             self._chk(self.lib.sds_workspace_bytes(C.byref(sch), C.byref(den), self.B, self.d, self.L, C.byref(nbytes)),
                       "sds_workspace_bytes")
             self._chk(self.lib.sds_create(C.byref(sch), C.byref(den), self.B, self.d, self.L, C.byref(h)), "sds_create")

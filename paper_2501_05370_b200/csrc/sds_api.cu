@@ -40,6 +40,7 @@ struct Layout {
   size_t S1, S2, ell, logU, accmask, jstar, nfe_calls, nfe_rows;
   size_t Gk;
   size_t Gx, Gb, Pb, Dp;  // independent drafter: gathered rows (f32, bf16), its outputs per call and per row
+  size_t adet, cdet;      // Picard drafter: deterministic sampler coefficients (Dp then holds draft means)
   size_t total;
 };
 
@@ -72,6 +73,8 @@ struct sds_ctx {
   int32_t tcond_dim = 0;
   Engine tgt, drf;                  // target denoiser; independent draft model (optional)
   bool has_drafter = false;
+  int32_t picard_calls = 0;         // > 0: created for the Picard drafter
+  std::vector<float> a_det, c_det;
   Layout lay{};
   char* ws = nullptr;
   size_t ws_bytes = 0;
@@ -135,8 +138,8 @@ void den_layout(Carve& cv, const sds_denoiser* den, size_t K, int tcond_dim, siz
   }
 }
 
-void make_layout(const sds_schedule* sch, const sds_denoiser* den, const sds_denoiser* drafter, int64_t B, int32_t d,
-                 int32_t L, Layout* out, DenLayout* tl, DenLayout* dl) {
+void make_layout(const sds_schedule* sch, const sds_denoiser* den, const sds_denoiser* drafter, bool picard, int64_t B,
+                 int32_t d, int32_t L, Layout* out, DenLayout* tl, DenLayout* dl) {
   Carve cv;
   Layout l{};
   const size_t K = (size_t)sch->K, rows = (size_t)B * L, Bd = (size_t)B * d;
@@ -173,6 +176,12 @@ void make_layout(const sds_schedule* sch, const sds_denoiser* den, const sds_den
     l.Dp = cv.take(rows * d * 4);
     den_layout(cv, drafter, K, 4, (size_t)B, d, dl);
     dl->xb = l.Gb;
+  }
+  l.adet = l.cdet = kNone;
+  if (picard) {
+    l.adet = cv.take(K * 4);
+    l.cdet = cv.take(K * 4);
+    l.Dp = cv.take(rows * d * 4);
   }
   l.total = cv.off;
   *out = l;
@@ -249,6 +258,9 @@ WinArgs win_args(sds_ctx* c) {
   A.Gx = at<float>(c, c->lay.Gx); A.Gb = at<uint16_t>(c, c->lay.Gb); A.Gk = at<int>(c, c->lay.Gk);
   A.Pb = at<float>(c, c->lay.Pb); A.Dp = at<float>(c, c->lay.Dp);
   A.Q = c->Q; A.qr = c->qr;
+  A.mean_rows = c->mode == SDS_PICARD ? 1 : 0;
+  A.picard_calls = c->picard_calls;
+  A.a_det = at<float>(c, c->lay.adet); A.c_det = at<float>(c, c->lay.cdet);
   return A;
 }
 
@@ -482,10 +494,22 @@ void engine_init(Engine& e, const sds_denoiser* den, const double* tcond, int tc
   }
 }
 
+struct PicardSpec {
+  int32_t calls;
+  const float* a_det;
+  const float* c_det;
+};
+
 int create_impl(const sds_schedule* sch, const sds_denoiser* den, const sds_denoiser* drafter,
-                const double* drafter_tcond, int64_t B, int32_t d, int32_t L, sds_ctx** out, size_t* bytes_only) {
+                const double* drafter_tcond, const PicardSpec* pic, int64_t B, int32_t d, int32_t L, sds_ctx** out,
+                size_t* bytes_only) {
   int rc = validate(sch, den, B, d, L);
   if (rc != SDS_OK) return rc;
+  if (pic && !bytes_only) {
+    if (pic->calls < 1 || pic->calls > 64 || !pic->a_det || !pic->c_det) return SDS_EINVAL;
+    for (int k = 0; k < sch->K; ++k)
+      if (!std::isfinite(pic->a_det[k]) || !std::isfinite(pic->c_det[k])) return SDS_EINVAL;
+  }
   if (drafter) {
     if (drafter->kind == SDS_DEN_CALLBACK) return SDS_EUNSUPPORTED;
     rc = validate_den(drafter, drafter_tcond, 4, d);
@@ -494,7 +518,7 @@ int create_impl(const sds_schedule* sch, const sds_denoiser* den, const sds_deno
   if (bytes_only) {
     Layout l;
     DenLayout tl, dl;
-    make_layout(sch, den, drafter, B, d, L, &l, &tl, &dl);
+    make_layout(sch, den, drafter, pic != nullptr, B, d, L, &l, &tl, &dl);
     *bytes_only = l.total;
     return SDS_OK;
   }
@@ -508,7 +532,12 @@ int create_impl(const sds_schedule* sch, const sds_denoiser* den, const sds_deno
   engine_init(c->tgt, den, sch->tcond, c->tcond_dim, sch->K, B * L);
   c->has_drafter = drafter != nullptr;
   if (drafter) engine_init(c->drf, drafter, drafter_tcond, 4, sch->K, B);
-  make_layout(sch, den, drafter, B, d, L, &c->lay, &c->tgt.lay, &c->drf.lay);
+  if (pic) {
+    c->picard_calls = pic->calls;
+    c->a_det.assign(pic->a_det, pic->a_det + sch->K);
+    c->c_det.assign(pic->c_det, pic->c_det + sch->K);
+  }
+  make_layout(sch, den, drafter, pic != nullptr, B, d, L, &c->lay, &c->tgt.lay, &c->drf.lay);
   if (cudaHostAlloc((void**)&c->h_pin, 64 * sizeof(int32_t), cudaHostAllocDefault) != cudaSuccess) {
     c->last_cuda = (int)cudaGetLastError();
     delete c;
@@ -532,34 +561,51 @@ int create_impl(const sds_schedule* sch, const sds_denoiser* den, const sds_deno
 int sds_workspace_bytes(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_t d, int32_t L,
                         size_t* bytes) {
   if (!bytes) return SDS_EINVAL;
-  return create_impl(sch, den, nullptr, nullptr, B, d, L, nullptr, bytes);
+  return create_impl(sch, den, nullptr, nullptr, nullptr, B, d, L, nullptr, bytes);
 }
 
 int sds_create(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_t d, int32_t L, sds_ctx** out) {
   if (!out) return SDS_EINVAL;
   *out = nullptr;
-  return create_impl(sch, den, nullptr, nullptr, B, d, L, out, nullptr);
+  return create_impl(sch, den, nullptr, nullptr, nullptr, B, d, L, out, nullptr);
+}
+
+int sds_workspace_bytes_picard(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int32_t d, int32_t L,
+                               size_t* bytes) {
+  if (!bytes) return SDS_EINVAL;
+  const PicardSpec pic{1, nullptr, nullptr};
+  return create_impl(sch, den, nullptr, nullptr, &pic, B, d, L, nullptr, bytes);
+}
+
+int sds_create_picard(const sds_schedule* sch, const sds_denoiser* den, int32_t calls, const float* a_det,
+                      const float* c_det, int64_t B, int32_t d, int32_t L, sds_ctx** out) {
+  if (!out) return SDS_EINVAL;
+  *out = nullptr;
+  const PicardSpec pic{calls, a_det, c_det};
+  return create_impl(sch, den, nullptr, nullptr, &pic, B, d, L, out, nullptr);
 }
 
 int sds_workspace_bytes_with_drafter(const sds_schedule* sch, const sds_denoiser* den, const sds_denoiser* drafter,
                                      const double* drafter_tcond, int64_t B, int32_t d, int32_t L, size_t* bytes) {
   if (!bytes || !drafter) return SDS_EINVAL;
-  return create_impl(sch, den, drafter, drafter_tcond, B, d, L, nullptr, bytes);
+  return create_impl(sch, den, drafter, drafter_tcond, nullptr, B, d, L, nullptr, bytes);
 }
 
 int sds_create_with_drafter(const sds_schedule* sch, const sds_denoiser* den, const sds_denoiser* drafter,
                             const double* drafter_tcond, int64_t B, int32_t d, int32_t L, sds_ctx** out) {
   if (!out || !drafter) return SDS_EINVAL;
   *out = nullptr;
-  return create_impl(sch, den, drafter, drafter_tcond, B, d, L, out, nullptr);
+  return create_impl(sch, den, drafter, drafter_tcond, nullptr, B, d, L, out, nullptr);
 }
 
 int sds_bind(sds_ctx* c, void* workspace_dev, size_t bytes, void* cuda_stream, uint64_t seed, int32_t drafter_mode,
              int64_t chain_id_offset) {
   if (!c || !workspace_dev) return SDS_EINVAL;
-  if (drafter_mode != SDS_FROZEN_PREV && drafter_mode != SDS_FROZEN_EXACT && drafter_mode != SDS_INDEPENDENT)
+  if (drafter_mode != SDS_FROZEN_PREV && drafter_mode != SDS_FROZEN_EXACT && drafter_mode != SDS_INDEPENDENT &&
+      drafter_mode != SDS_PICARD)
     return SDS_EUNSUPPORTED;
   if ((drafter_mode == SDS_INDEPENDENT) != c->has_drafter) return SDS_EINVAL;   // the draft model and the mode go together
+  if ((drafter_mode == SDS_PICARD) != (c->picard_calls > 0)) return SDS_EINVAL; // so do the Picard context and its mode
   if (chain_id_offset < 0) return SDS_EINVAL;
   if (bytes < c->lay.total || (reinterpret_cast<uintptr_t>(workspace_dev) % kAlign) != 0) return SDS_ENOMEM;
   c->ws = static_cast<char*>(workspace_dev);
@@ -573,6 +619,10 @@ int sds_bind(sds_ctx* c, void* workspace_dev, size_t bytes, void* cuda_stream, u
   SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.a, c->a.data(), kb, cudaMemcpyHostToDevice, c->stream));
   SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.c, c->c.data(), kb, cudaMemcpyHostToDevice, c->stream));
   SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.sigma, c->sigma.data(), kb, cudaMemcpyHostToDevice, c->stream));
+  if (c->picard_calls > 0) {
+    SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.adet, c->a_det.data(), kb, cudaMemcpyHostToDevice, c->stream));
+    SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.cdet, c->c_det.data(), kb, cudaMemcpyHostToDevice, c->stream));
+  }
   for (Engine* e : {&c->tgt, &c->drf})
     if (!e->tcond.empty())
       SDS_CU(c, cudaMemcpyAsync(c->ws + e->lay.tcond, e->tcond.data(), e->tcond.size() * 8, cudaMemcpyHostToDevice,
@@ -588,7 +638,7 @@ int sds_reset(sds_ctx* c) {
   if (c->state < kBound) return SDS_ESTATE;
   WinArgs A = win_args(c);
   SDS_LAUNCH(c, SDS_PROF_INIT, launch_init(A, c->stream));
-  if (c->mode == SDS_FROZEN_PREV) {
+  if (c->mode == SDS_FROZEN_PREV || c->mode == SDS_PICARD) {
     const int rc = run_denoiser(c, c->tgt, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, c->B, A.Dq);
     if (rc != SDS_OK) return rc;
     SDS_LAUNCH(c, SDS_PROF_AUX, launch_after_init(A, c->stream));
@@ -610,7 +660,19 @@ int sds_draft(sds_ctx* c) {
     if (rc != SDS_OK) return rc;
     SDS_LAUNCH(c, SDS_PROF_DRAFT, launch_scatter_carried(A, c->ub, c->stream));
   }
-  if (c->mode == SDS_INDEPENDENT) {
+  if (c->mode == SDS_PICARD) {
+    // the rows hold the deterministic sampler's points while the target refines them in parallel
+    const int64_t rows_ub = (int64_t)c->ub * c->L;
+    SDS_LAUNCH(c, SDS_PROF_DRAFT, launch_picard_start(A, c->ub, c->stream));
+    for (int m = 1; m < c->picard_calls; ++m) {
+      const int rc = run_denoiser(c, c->tgt, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, rows_ub, A.Dq);
+      if (rc != SDS_OK) return rc;
+      SDS_LAUNCH(c, SDS_PROF_DRAFT, launch_picard_step(A, c->ub, c->stream));
+    }
+    const int rc = run_denoiser(c, c->tgt, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, rows_ub, A.Dq);
+    if (rc != SDS_OK) return rc;
+    SDS_LAUNCH(c, SDS_PROF_DRAFT, launch_picard_draft(A, c->ub, c->stream));
+  } else if (c->mode == SDS_INDEPENDENT) {
     // sequential draft: position j needs the draft model at W_{j-1}
     for (int j = 1; j <= c->L; ++j) {
       SDS_LAUNCH(c, SDS_PROF_DRAFT, launch_gather_pos(A, j, c->ub, c->stream));

@@ -129,6 +129,18 @@ __device__ __forceinline__ void delta_z(float wp, float wj, float dq, float dc, 
   Z = r * inv_s;
 }
 
+// the same for a drafter given by its mean m^p itself (not of the form a W_{j-1} + c D):
+// Delta_i = (m^p_i - a W_{j-1} - c D_q)/sigma, Z_i = (W_j - m^p_i)/sigma; `mean` selects the form
+__device__ __forceinline__ void delta_z_any(bool mean, float wp, float wj, float dq, float dc_or_mp, float a, float c,
+                                            float cs, float inv_s, float& D, float& Z) {
+  if (mean) {
+    D = (dc_or_mp - fmaf(a, wp, c * dq)) * inv_s;
+    Z = (wj - dc_or_mp) * inv_s;
+  } else {
+    delta_z(wp, wj, dq, dc_or_mp, a, c, cs, inv_s, D, Z);
+  }
+}
+
 // reflected state: m^q + sigma (Z - coef * Delta), coef = 2 (Delta.Z)/|Delta|^2
 __device__ __forceinline__ float reflect_elem(float wp, float dq, float Z, float D, float a, float c, float s,
                                               float coef) {

@@ -46,6 +46,11 @@ struct WinArgs {
   // acceptance ratio decided in a subspace (NULL: the full space)
   const float* Q;        // [qr, d]  orthonormal rows spanning the row space of the projection matrix
   int qr;
+  // Picard drafter only: Dp then holds the draft MEANS per drafted row
+  int mean_rows;         // 1: Dp rows are draft means m^p, not draft-model outputs
+  int picard_calls;      // batched target calls per window that build the draft
+  const float* a_det;    // [K] deterministic sampler F_{j+1} = a_det F_j + c_det D
+  const float* c_det;    // [K]
 };
 
 struct GmmArgs {
@@ -65,6 +70,9 @@ cudaError_t launch_scatter_carried(const WinArgs& A, int ub_chains, cudaStream_t
 cudaError_t launch_draft(const WinArgs& A, int ub_chains, cudaStream_t st);
 cudaError_t launch_gather_pos(const WinArgs& A, int j, int ub_chains, cudaStream_t st);
 cudaError_t launch_draft_pos(const WinArgs& A, int j, int ub_chains, cudaStream_t st);
+cudaError_t launch_picard_start(const WinArgs& A, int ub_chains, cudaStream_t st);
+cudaError_t launch_picard_step(const WinArgs& A, int ub_chains, cudaStream_t st);
+cudaError_t launch_picard_draft(const WinArgs& A, int ub_chains, cudaStream_t st);
 cudaError_t launch_verify(const WinArgs& A, int ub_chains, cudaStream_t st);
 cudaError_t launch_advance(const WinArgs& A, int ub_chains, cudaStream_t st);
 cudaError_t launch_rng_normals(uint64_t seed, int stream_id, uint64_t b0, int64_t nb, int k, int d, float* out,

@@ -105,8 +105,9 @@ __global__ void __launch_bounds__(kBlock) k_init(WinArgs A) {
   if (t == 0) {
     A.n[b] = 0;
     A.rowk[b] = 0;
-    A.nfe_calls[b] = A.mode == 0 ? 1 : 0;      // the carried-output drafter starts with one target call
-    A.nfe_rows[b] = A.mode == 0 ? 1 : 0;
+    const int first = (A.mode == 0 || A.mode == 3) ? 1 : 0;   // drafters that carry an output start with one target call
+    A.nfe_calls[b] = first;
+    A.nfe_rows[b] = first;
     A.accmask[b] = 0u;
     A.jstar[b] = 0;
   }
@@ -292,6 +293,134 @@ __global__ void __launch_bounds__(kBlock) k_draft_pos(WinArgs A, int j) {
 }
 
 // ---------------------------------------------------------------------------------------
+// Picard drafter (Appendix C): rows r0..r0+Lt-1 of X hold the points F_0..F_{Lt-1} of the
+// deterministic sampler while the draft is built; each thread owns its elements across positions.
+//   k_picard_start  F_0 = Y_n, F_{j+1} = a_det F_j + c_det D_c (carried output frozen)
+//   k_picard_step   after a target call on the points: F_{j+1} <- a_det F_j(old) + c_det D(F_j(old))
+//   k_picard_draft  after the last call: m^p_{j+1} = a F_j + c D(F_j) (kept per row for verify),
+//                   W_{j+1} = m^p_{j+1} + sigma xi; the rows then hold W_0..W_{Lt-1}, T holds W_Lt
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void put_row(const WinArgs& A, size_t ro, float v) {
+  A.X[ro] = v;
+  if (A.Xb) A.Xb[ro] = (uint16_t)(pack_bf16x2(v, 0.f) & 0xffffu);
+}
+__device__ __forceinline__ void put_row4(const WinArgs& A, size_t ro, float4 v) {
+  st4(A.X + ro, v);
+  if (A.Xb) *reinterpret_cast<uint2*>(A.Xb + ro) = make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
+}
+
+template <int TPC, int VEC>
+__global__ void __launch_bounds__(kBlock) k_picard_start(WinArgs A) {
+  using G = Group<TPC>;
+  const int s = G::slot(), t = G::lane();
+  if (s >= A.ctl[kCtlNActive]) return;
+  const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
+  const int Lt = window_len(A, nb);
+  const size_t cb = (size_t)b * A.d;
+  if (t < Lt) A.rowk[r0 + t] = nb + t;
+  if (VEC == 4) {
+    for (int i = t * 4; i < A.d; i += TPC * 4) {
+      float4 f = ld4(A.Y + cb + i);
+      const float4 dc = ld4(A.Dc + cb + i);
+      for (int j = 0; j < Lt; ++j) {
+        put_row4(A, (size_t)(r0 + j) * A.d + i, f);
+        const float ad = __ldg(A.a_det + nb + j), cd = __ldg(A.c_det + nb + j);
+        f = make_float4(fmaf(ad, f.x, cd * dc.x), fmaf(ad, f.y, cd * dc.y), fmaf(ad, f.z, cd * dc.z),
+                        fmaf(ad, f.w, cd * dc.w));
+      }
+    }
+  } else {
+    for (int i = t; i < A.d; i += TPC) {
+      float f = A.Y[cb + i];
+      const float dc = A.Dc[cb + i];
+      for (int j = 0; j < Lt; ++j) {
+        put_row(A, (size_t)(r0 + j) * A.d + i, f);
+        f = fmaf(__ldg(A.a_det + nb + j), f, __ldg(A.c_det + nb + j) * dc);
+      }
+    }
+  }
+}
+
+template <int TPC, int VEC>
+__global__ void __launch_bounds__(kBlock) k_picard_step(WinArgs A) {
+  using G = Group<TPC>;
+  const int s = G::slot(), t = G::lane();
+  if (s >= A.ctl[kCtlNActive]) return;
+  const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
+  const int Lt = window_len(A, nb);
+  if (VEC == 4) {
+    for (int i = t * 4; i < A.d; i += TPC * 4) {
+      float4 f = ld4(A.X + (size_t)r0 * A.d + i);                 // previous iterate's F_j
+      for (int j = 0; j + 1 < Lt; ++j) {
+        const size_t rn = (size_t)(r0 + j + 1) * A.d + i;
+        const float4 fn = ld4(A.X + rn);                          // previous iterate's F_{j+1}, needed next
+        const float4 dq = ld4(A.Dq + (size_t)(r0 + j) * A.d + i);
+        const float ad = __ldg(A.a_det + nb + j), cd = __ldg(A.c_det + nb + j);
+        put_row4(A, rn, make_float4(fmaf(ad, f.x, cd * dq.x), fmaf(ad, f.y, cd * dq.y), fmaf(ad, f.z, cd * dq.z),
+                                    fmaf(ad, f.w, cd * dq.w)));
+        f = fn;
+      }
+    }
+  } else {
+    for (int i = t; i < A.d; i += TPC) {
+      float f = A.X[(size_t)r0 * A.d + i];
+      for (int j = 0; j + 1 < Lt; ++j) {
+        const size_t rn = (size_t)(r0 + j + 1) * A.d + i;
+        const float fn = A.X[rn];
+        put_row(A, rn, fmaf(__ldg(A.a_det + nb + j), f, __ldg(A.c_det + nb + j) * A.Dq[(size_t)(r0 + j) * A.d + i]));
+        f = fn;
+      }
+    }
+  }
+}
+
+template <int TPC, int VEC>
+__global__ void __launch_bounds__(kBlock) k_picard_draft(WinArgs A) {
+  using G = Group<TPC>;
+  const int s = G::slot(), t = G::lane();
+  if (s >= A.ctl[kCtlNActive]) return;
+  const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
+  const int Lt = window_len(A, nb);
+  const uint64_t bg = A.chain_off + (uint64_t)b;
+  const size_t cb = (size_t)b * A.d;
+  if (VEC == 4) {
+    for (int i = t * 4; i < A.d; i += TPC * 4) {
+      float4 f = ld4(A.X + (size_t)r0 * A.d + i);
+      for (int j = 0; j < Lt; ++j) {
+        const int k = nb + j;
+        const size_t ro = (size_t)(r0 + j) * A.d + i;
+        const float4 fn = (j + 1 < Lt) ? ld4(A.X + ro + A.d) : f;   // F_{j+1} before W_{j+1} replaces it
+        const float4 dq = ld4(A.Dq + ro);
+        const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
+        const float4 mp = make_float4(fmaf(ak, f.x, ck * dq.x), fmaf(ak, f.y, ck * dq.y), fmaf(ak, f.z, ck * dq.z),
+                                      fmaf(ak, f.w, ck * dq.w));
+        st4(A.Dp + ro, mp);
+        const float4 xi = normal4(A.seed, kStreamDraft, bg, (uint32_t)k, (uint32_t)(i >> 2));
+        const float4 w = make_float4(fmaf(sk, xi.x, mp.x), fmaf(sk, xi.y, mp.y), fmaf(sk, xi.z, mp.z), fmaf(sk, xi.w, mp.w));
+        if (j + 1 < Lt) put_row4(A, ro + A.d, w);
+        else st4(A.T + cb + i, w);
+        f = fn;
+      }
+    }
+  } else {
+    for (int i = t; i < A.d; i += TPC) {
+      float f = A.X[(size_t)r0 * A.d + i];
+      for (int j = 0; j < Lt; ++j) {
+        const int k = nb + j;
+        const size_t ro = (size_t)(r0 + j) * A.d + i;
+        const float fn = (j + 1 < Lt) ? A.X[ro + A.d] : f;
+        const float mp = fmaf(__ldg(A.a + k), f, __ldg(A.c + k) * A.Dq[ro]);
+        A.Dp[ro] = mp;
+        const float w = fmaf(__ldg(A.sigma + k), normal1(A.seed, kStreamDraft, bg, (uint32_t)k, (uint32_t)i), mp);
+        if (j + 1 < Lt) put_row(A, ro + A.d, w);
+        else A.T[cb + i] = w;
+        f = fn;
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
 // Ratio decided in a subspace (Appendix F): with P = Q^T Q the orthogonal projector onto the rows
 // of Q, S1 = Delta^T P Delta = sum_i (q_i.Delta)^2 and S2 = Z^T P Delta = sum_i (q_i.Delta)(q_i.Z).
 // One CTA per (active chain, position): Delta and Z of that position are staged in shared memory,
@@ -318,7 +447,7 @@ __global__ void __launch_bounds__(kBlock) k_project(WinArgs A) {
   float* sZ = s_dz + d;
   for (int i = tid; i < d; i += kBlock) {
     float D, Z;
-    delta_z(wp[i], wj[i], dq[i], dc[i], ak, ck, cs, inv_s, D, Z);
+    delta_z_any(A.mean_rows != 0, wp[i], wj[i], dq[i], dc[i], ak, ck, cs, inv_s, D, Z);
     sD[i] = D;
     sZ[i] = Z;
   }
@@ -366,6 +495,7 @@ __global__ void __launch_bounds__(kBlock) k_verify(WinArgs A) {
   const uint64_t bg = A.chain_off + (uint64_t)b;
   const size_t cb = (size_t)b * A.d;
 
+  const bool mean = A.mean_rows != 0;                 // Dp rows are draft means (Picard drafter)
   double myS1 = 0.0, myS2 = 0.0;
   const bool projected = A.Q != nullptr;              // S1, S2 already written by k_project
   if (projected && warp == 0 && lane < Lt) {
@@ -385,19 +515,19 @@ __global__ void __launch_bounds__(kBlock) k_verify(WinArgs A) {
       for (int i = t * 4; i < A.d; i += TPC * 4) {
         const float4 vp = ld4(wp + i), vj = ld4(wj + i), vq = ld4(dq + i), vc = ld4(dc + i);
         float D, Z;
-        delta_z(vp.x, vj.x, vq.x, vc.x, ak, ck, cs, inv_s, D, Z);
+        delta_z_any(mean, vp.x, vj.x, vq.x, vc.x, ak, ck, cs, inv_s, D, Z);
         p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
-        delta_z(vp.y, vj.y, vq.y, vc.y, ak, ck, cs, inv_s, D, Z);
+        delta_z_any(mean, vp.y, vj.y, vq.y, vc.y, ak, ck, cs, inv_s, D, Z);
         p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
-        delta_z(vp.z, vj.z, vq.z, vc.z, ak, ck, cs, inv_s, D, Z);
+        delta_z_any(mean, vp.z, vj.z, vq.z, vc.z, ak, ck, cs, inv_s, D, Z);
         p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
-        delta_z(vp.w, vj.w, vq.w, vc.w, ak, ck, cs, inv_s, D, Z);
+        delta_z_any(mean, vp.w, vj.w, vq.w, vc.w, ak, ck, cs, inv_s, D, Z);
         p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
       }
     } else {
       for (int i = t; i < A.d; i += TPC) {
         float D, Z;
-        delta_z(wp[i], wj[i], dq[i], dc[i], ak, ck, cs, inv_s, D, Z);
+        delta_z_any(mean, wp[i], wj[i], dq[i], dc[i], ak, ck, cs, inv_s, D, Z);
         p1 = fma((double)D, (double)D, p1);
         p2 = fma((double)D, (double)Z, p2);
       }
@@ -474,16 +604,16 @@ __global__ void __launch_bounds__(kBlock) k_verify(WinArgs A) {
       const float4 vp = ld4(wp + i), vj = ld4(wj + i), vq = ld4(dq + i), vc = ld4(dc + i);
       float4 o;
       float D, Z;
-      delta_z(vp.x, vj.x, vq.x, vc.x, ak, ck, cs, inv_s, D, Z); o.x = reflect_elem(vp.x, vq.x, Z, D, ak, ck, sk, coef);
-      delta_z(vp.y, vj.y, vq.y, vc.y, ak, ck, cs, inv_s, D, Z); o.y = reflect_elem(vp.y, vq.y, Z, D, ak, ck, sk, coef);
-      delta_z(vp.z, vj.z, vq.z, vc.z, ak, ck, cs, inv_s, D, Z); o.z = reflect_elem(vp.z, vq.z, Z, D, ak, ck, sk, coef);
-      delta_z(vp.w, vj.w, vq.w, vc.w, ak, ck, cs, inv_s, D, Z); o.w = reflect_elem(vp.w, vq.w, Z, D, ak, ck, sk, coef);
+      delta_z_any(mean, vp.x, vj.x, vq.x, vc.x, ak, ck, cs, inv_s, D, Z); o.x = reflect_elem(vp.x, vq.x, Z, D, ak, ck, sk, coef);
+      delta_z_any(mean, vp.y, vj.y, vq.y, vc.y, ak, ck, cs, inv_s, D, Z); o.y = reflect_elem(vp.y, vq.y, Z, D, ak, ck, sk, coef);
+      delta_z_any(mean, vp.z, vj.z, vq.z, vc.z, ak, ck, cs, inv_s, D, Z); o.z = reflect_elem(vp.z, vq.z, Z, D, ak, ck, sk, coef);
+      delta_z_any(mean, vp.w, vj.w, vq.w, vc.w, ak, ck, cs, inv_s, D, Z); o.w = reflect_elem(vp.w, vq.w, Z, D, ak, ck, sk, coef);
       st4(wj + i, o);
     }
   } else {
     for (int i = t; i < A.d; i += TPC) {
       float D, Z;
-      delta_z(wp[i], wj[i], dq[i], dc[i], ak, ck, cs, inv_s, D, Z);
+      delta_z_any(mean, wp[i], wj[i], dq[i], dc[i], ak, ck, cs, inv_s, D, Z);
       wj[i] = reflect_elem(wp[i], dq[i], Z, D, ak, ck, sk, coef);
     }
   }
@@ -672,8 +802,13 @@ __global__ void __launch_bounds__(kBlock) k_advance(WinArgs A) {
         A.n[b] = nb + adv;
         // sequential target calls of this window: the batched pass, plus (main-text drafter) the
         // call at Y_n, which is row 1 of the batch (a window of one row is a single call)
-        A.nfe_calls[b] += (A.mode == 1 && Lt > 1) ? 2 : 1;
-        A.nfe_rows[b] += Lt;
+        if (A.mode == 3) {   // Picard: calls-1 refinements on Lt-1 points, the last draft call on Lt, verify on Lt-1
+          A.nfe_calls[b] += (Lt > 1) ? A.picard_calls + 1 : 1;
+          A.nfe_rows[b] += (A.picard_calls - 1) * (Lt - 1) + Lt + (Lt - 1);
+        } else {
+          A.nfe_calls[b] += (A.mode == 1 && Lt > 1) ? 2 : 1;
+          A.nfe_rows[b] += Lt;
+        }
       }
     } else if (t == 0) {                              // non-finite log ratio: stop this chain
       A.n[b] = A.K;
@@ -777,8 +912,24 @@ cudaError_t launch_draft_pos(const WinArgs& A, int j, int ub, cudaStream_t st) {
   }
   return cudaGetLastError();
 }
+cudaError_t launch_picard_start(const WinArgs& A, int ub, cudaStream_t st) {
+  SDS_DISPATCH(k_picard_start, A, ub, st);
+  return cudaGetLastError();
+}
+cudaError_t launch_picard_step(const WinArgs& A, int ub, cudaStream_t st) {
+  SDS_DISPATCH(k_picard_step, A, ub, st);
+  return cudaGetLastError();
+}
+cudaError_t launch_picard_draft(const WinArgs& A, int ub, cudaStream_t st) {
+  SDS_DISPATCH(k_picard_draft, A, ub, st);
+  return cudaGetLastError();
+}
 cudaError_t launch_verify(const WinArgs& A, int ub, cudaStream_t st) {
   const int chains = ub > 0 ? ub : 1;
+  if (A.mean_rows && !A.Q) {                            // draft means per row: the generic kernel handles them
+    SDS_DISPATCH(k_verify, A, ub, st);
+    return cudaGetLastError();
+  }
   if (A.Q) {                                            // projected sums first, then the shared accept/reflect tail
     const size_t smem = 2 * (size_t)A.d * sizeof(float);
     cudaError_t e = cudaFuncSetAttribute(k_project, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -32,8 +32,18 @@ def drafter_for(w, *, gmm=None, mlp=None):
     raise ValueError("a draft model is required")
 
 
+def picard_for(w, calls: int):
+    """(calls, a_det, c_det) for Sampler(picard=...): the deterministic sampler that goes with the
+    workload's schedule (noise-free ancestral step for ddpm, gradient step for Langevin)."""
+    if w.sampler == "ddpm":
+        a_det, c_det = sb.ddim_schedule(w.beta())
+    else:
+        a_det, c_det, _ = sb.ula_schedule(w.K, w.ula_gamma)
+    return (int(calls), a_det, c_det)
+
+
 def sampler_for(w, *, seed=None, chain_id_offset=0, B=None, device="cuda:0", gmm=None, mlp=None, drafter_mode=None,
-                drafter=None):
+                drafter=None, picard=None):
     a, c, sigma, tcond = schedule_for(w)
     if drafter_mode is None:
         drafter_mode = getattr(w, "drafter_mode", 0)
@@ -43,12 +53,12 @@ def sampler_for(w, *, seed=None, chain_id_offset=0, B=None, device="cuda:0", gmm
         gp = gmm if gmm is not None else w.gmm_params()
         return sb.Sampler(a, c, sigma, B, w.d, w.L, gmm_means=gp.means, gmm_logw=gp.logw, tcond=tcond,
                           gmm_bf16=bool(getattr(gp, "means_bf16", False)), seed=seed,
-                          chain_id_offset=chain_id_offset, drafter_mode=drafter_mode, drafter=drafter, device=device)
+                          chain_id_offset=chain_id_offset, drafter_mode=drafter_mode, drafter=drafter, picard=picard, device=device)
     if w.denoiser == "mlp":
         mp = mlp if mlp is not None else w.mlp_params()
-        return sb.Sampler(a, c, sigma, B, w.d, w.L, mlp=mp, seed=seed, chain_id_offset=chain_id_offset, drafter_mode=drafter_mode, drafter=drafter, device=device)
+        return sb.Sampler(a, c, sigma, B, w.d, w.L, mlp=mp, seed=seed, chain_id_offset=chain_id_offset, drafter_mode=drafter_mode, drafter=drafter, picard=picard, device=device)
     if w.denoiser == "phi4":
         p4 = w.phi4
         return sb.Sampler(a, c, sigma, B, w.d, w.L, phi4=(p4["side"], p4["beta"], p4.get("periodic", False)), seed=seed,
-                          chain_id_offset=chain_id_offset, drafter_mode=drafter_mode, drafter=drafter, device=device)
+                          chain_id_offset=chain_id_offset, drafter_mode=drafter_mode, drafter=drafter, picard=picard, device=device)
     raise NotImplementedError(w.denoiser)
