@@ -28,7 +28,9 @@ closed form 2 - 2*Phi(|m^p - m^q| / (2 sigma)) (Proposition 2) on the two worked
 the paper draws; output law of the reflection step by KS at d = 1, 2 (and the incorrect rule
 failing it); the discrete worked example; E[log a] = -|Delta|^2/2; mean window advance against
 the geometric sum; speculative vs plain chain in law; mixture denoiser against brute force and
-finite differences; DDPM coefficient identities.
+finite differences; DDPM coefficient identities; the projected rule against Algorithm 3 (invertible
+matrix), the whitened-image identity and the image's law; the Picard iterates against the sequential
+deterministic chain, window 1 against the plain chain, and the chain's law.
 Parity unpinned: agreement of the NFE counters with the paper's tables (the paper does not say
 which frozen-drafter variant or call count produced them).
 """
