@@ -119,7 +119,7 @@ void den_layout(Carve& cv, const sds_denoiser* den, size_t K, int tcond_dim, siz
   l->musq = (den->kind == SDS_DEN_GMM) ? cv.take((size_t)den->ncomp * 8) : kNone;
   l->H0 = l->H1 = l->logits = l->R = l->Mt = l->Xs = l->Ms = kNone;
   if (gmm_split_shape(*den, d)) {
-    l->Xs = cv.take(3 * rows * (size_t)d * 2);
+    l->Xs = cv.take(2 * rows * (size_t)d * 2);
     l->Ms = cv.take(3 * (size_t)den->ncomp * d * 2);
     l->Mt = cv.take(3 * (size_t)d * den->ncomp * 2);
     l->R = cv.take(3 * rows * (size_t)den->ncomp * 2);
@@ -257,6 +257,10 @@ WinArgs win_args(sds_ctx* c) {
   A.nfe_calls = at<int>(c, c->lay.nfe_calls); A.nfe_rows = at<int>(c, c->lay.nfe_rows);
   A.Gx = at<float>(c, c->lay.Gx); A.Gb = at<uint16_t>(c, c->lay.Gb); A.Gk = at<int>(c, c->lay.Gk);
   A.Pb = at<float>(c, c->lay.Pb); A.Dp = at<float>(c, c->lay.Dp);
+  if (c->tensor_split && gmm_split_shape(c->tgt.den, c->d)) {   // draft and init write the row planes themselves
+    A.Xs = at<uint16_t>(c, c->tgt.lay.Xs);
+    A.xs_plane = (size_t)c->tgt.cap_rows * c->d;
+  }
   A.Q = c->Q; A.qr = c->qr;
   A.mean_rows = c->mode == SDS_PICARD ? 1 : 0;
   A.picard_calls = c->picard_calls;
@@ -351,14 +355,17 @@ TcGemmArgs tc_args(sds_ctx* c, Engine& e, const int* rowk, const int* nrows_dev,
 // run the target denoiser on dense rows X (and their bf16 copy Xb, NULL = make one); the row count
 // lives on the device (nrows_dev, may be NULL) with a host upper bound for the grids
 int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, const int* rowk, const int* nrows_dev,
-                 int64_t rows_ub, float* out) {
+                 int64_t rows_ub, float* out, bool planes_ready = false) {
   if (rows_ub <= 0) return SDS_OK;
   switch (e.den.kind) {
     case SDS_DEN_GMM: {
       if (e.den.means_dtype == SDS_F32 && c->tensor_split && gmm_split_shape(e.den, c->d)) {
-        // Float mixture on the tensor cores: rows, means and responsibilities are split into three
-        // bf16 planes each (x = h + m + l carries the 24-bit significand); the six products of
-        // total order <= 2 are accumulated, smallest first, in one TMEM accumulator.
+        // Float mixture on the tensor cores: means and responsibilities are split into three bf16
+        // planes each (x = h + m + l carries the 24-bit significand) and the mixing contraction
+        // accumulates the six products of total order <= 2, smallest first, in one TMEM accumulator.
+        // The logits only have to find the components within 30 of the row maximum (the softmax
+        // kernel recomputes those in double; the rest weigh less than e^-29), so the rows are split in
+        // two planes and three products (orders <= 1, a 16-bit significand) are enough.
         const float* means = static_cast<const float*>(e.den.means_dev);
         const size_t nc = (size_t)e.den.ncomp, dd = (size_t)c->d, cap = (size_t)e.cap_rows;
         uint16_t* Ms = at<uint16_t>(c, e.lay.Ms);
@@ -370,17 +377,19 @@ int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, cons
         int rc = ensure_musq(c, e);
         if (rc != SDS_OK) return rc;
         if (fresh) {
-          SDS_LAUNCH(c, SDS_PROF_AUX, launch_split3(means, nc * dd, nc * dd, Ms, c->stream));
+          SDS_LAUNCH(c, SDS_PROF_AUX, launch_split3(means, nc * dd, nc * dd, 3, Ms, c->stream));
           for (int i = 0; i < 3; ++i)
             SDS_LAUNCH(c, SDS_PROF_AUX, launch_transpose_bf16(Ms + i * nc * dd, (int)nc, (int)dd, Mt + i * nc * dd, c->stream));
         }
-        SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_split3(X, (size_t)rows_ub * dd, cap * dd, Xs, c->stream));
+        if (!planes_ready)   // the draft and init kernels write the two row planes as they write the rows
+          SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_split3(X, (size_t)rows_ub * dd, cap * dd, 2, Xs, c->stream));
         static const uint8_t kA[6] = {2, 1, 0, 1, 0, 0}, kB[6] = {0, 1, 2, 0, 1, 0};
+        static const uint8_t kLa[3] = {1, 0, 0}, kLb[3] = {0, 1, 0};
         TcGemmArgs g = tc_args(c, e, rowk, nrows_dev, rows_ub);
         g.N = (int)nc; g.K = (int)dd; g.out = logits; g.ldo = (int)nc;
         g.tcond = at<double>(c, e.lay.tcond); g.musq = at<double>(c, e.lay.musq); g.logw = e.den.logw_dev;
-        g.nseg = 6; g.nplanes = 3; g.a_plane = cap * dd; g.b_plane = nc * dd;
-        for (int i = 0; i < 6; ++i) { g.a_idx[i] = kA[i]; g.b_idx[i] = kB[i]; }
+        g.nseg = 3; g.nplanes = 2; g.a_plane = cap * dd; g.b_plane = nc * dd;
+        for (int i = 0; i < 3; ++i) { g.a_idx[i] = kLa[i]; g.b_idx[i] = kLb[i]; }
         SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiGmmLogits, g, Xs, Ms, c->stream));
         SDS_LAUNCH(c, SDS_PROF_DENOISE,
                    launch_softmax_split3(logits, nrows_dev, (int)rows_ub, (int)nc, (int)dd, X, means,
@@ -639,7 +648,7 @@ int sds_reset(sds_ctx* c) {
   WinArgs A = win_args(c);
   SDS_LAUNCH(c, SDS_PROF_INIT, launch_init(A, c->stream));
   if (c->mode == SDS_FROZEN_PREV || c->mode == SDS_PICARD) {
-    const int rc = run_denoiser(c, c->tgt, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, c->B, A.Dq);
+    const int rc = run_denoiser(c, c->tgt, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, c->B, A.Dq, A.Xs != nullptr);
     if (rc != SDS_OK) return rc;
     SDS_LAUNCH(c, SDS_PROF_AUX, launch_after_init(A, c->stream));
   }
@@ -691,7 +700,9 @@ int sds_verify_window(sds_ctx* c) {
   if (!c) return SDS_EINVAL;
   if (c->state != kDrafted) return SDS_ESTATE;
   WinArgs A = win_args(c);
-  const int rc = run_denoiser(c, c->tgt, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, (int64_t)c->ub * c->L, A.Dq);
+  // rows drafted by k_draft (the two frozen-output modes) come with their bf16 planes
+  const bool planes_ready = A.Xs != nullptr && (c->mode == SDS_FROZEN_PREV || c->mode == SDS_FROZEN_EXACT);
+  const int rc = run_denoiser(c, c->tgt, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, (int64_t)c->ub * c->L, A.Dq, planes_ready);
   if (rc != SDS_OK) return rc;
   SDS_LAUNCH(c, SDS_PROF_VERIFY, launch_verify(A, c->ub, c->stream));
   c->state = kVerified;

@@ -34,9 +34,9 @@ constexpr int kErrNonFinite = 1;
 __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
 #pragma unroll
   for (int r = 0; r < 10; ++r) {
-    const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
-    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
-    c = make_uint4(hi1 ^ c.y ^ k.x, lo1, hi0 ^ c.w ^ k.y, lo0);
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c.x;        // one wide multiply gives hi and lo
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * c.z;
+    c = make_uint4((uint32_t)(p1 >> 32) ^ c.y ^ k.x, (uint32_t)p1, (uint32_t)(p0 >> 32) ^ c.w ^ k.y, (uint32_t)p0);
     k.x += 0x9E3779B9u;
     k.y += 0xBB67AE85u;
   }
@@ -51,13 +51,28 @@ __device__ __forceinline__ uint4 philox_block(uint64_t seed, int stream, uint64_
 
 // Box-Muller on one word pair; both uniforms carry 24 bits so they are exact in float:
 // u1 = ((x_even >> 8) + 1) 2^-24 in (0, 1], u2 = (x_odd >> 8) 2^-24 in [0, 1).
+// The transcendental steps use the special-function unit (lg2, sqrt, sin, cos approximations): with
+// the accurate library routines this transform, not memory, bounds the draft kernel. Documented
+// error of the approximations: lg2 2^-22 (absolute on (0.5, 2), relative elsewhere), sqrt 2^-23
+// relative, sin/cos 2^-20.5 absolute on [-2 pi, 2 pi]; the angle is shifted to [-pi, pi) exactly
+// (u2 - 1/2 is exact) and cos(t + pi) = -cos t. A normal z = r cos(.) thus differs from the exactly
+// rounded one by at most about 1e-6 r + 1.7e-7/r for r >= 1/8 (r <= 5.77), less below.
+__device__ __forceinline__ float sqrt_approx(float x) {
+  float y;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ float2 box_muller(uint32_t xe, uint32_t xo) {
   const float u1 = (float)((xe >> 8) + 1u) * 0x1p-24f;
   const float u2 = (float)(xo >> 8) * 0x1p-24f;
-  const float r = sqrtf(-2.0f * logf(u1));
-  float s, c;
-  sincospif(2.0f * u2, &s, &c);
-  return make_float2(r * c, r * s);
+  // -2 ln u1; next to 1 the approximation's absolute error would dominate, so the series of
+  // -2 ln(1 - t), t = 1 - u1 (exact), takes over below t = 2^-7 (truncation t^4/5 relative)
+  const float t = 1.0f - u1;
+  float r2 = -1.38629436111989f * __log2f(u1);
+  if (t < 0x1p-7f) r2 = 2.0f * t * fmaf(t, fmaf(t, fmaf(t, 0.25f, 0.333333343f), 0.5f), 1.0f);
+  const float r = sqrt_approx(r2);
+  const float th = (u2 - 0.5f) * 6.28318530717959f;                            // 2 pi u2 - pi
+  return make_float2(-r * __cosf(th), -r * __sinf(th));
 }
 
 // four normals of block q (elements 4q .. 4q+3)
@@ -108,6 +123,25 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
+}
+
+// x = h + m + l with h, m, l bfloat16 (each the rounded remainder of the previous ones): three
+// planes that together carry the 24-bit significand of a float
+__device__ __forceinline__ void split3(float x, uint16_t& h, uint16_t& m, uint16_t& l) {
+  const uint32_t ph = pack_bf16x2(x, 0.f) & 0xffffu;
+  const float r1 = x - __uint_as_float(ph << 16);
+  const uint32_t pm = pack_bf16x2(r1, 0.f) & 0xffffu;
+  const float r2 = r1 - __uint_as_float(pm << 16);
+  h = (uint16_t)ph; m = (uint16_t)pm; l = (uint16_t)(pack_bf16x2(r2, 0.f) & 0xffffu);
+}
+
+// the first two planes (h, m) of four consecutive floats, stored `plane` elements apart
+__device__ __forceinline__ void store_split2x4(uint16_t* out, size_t plane, float4 v) {
+  const uint32_t h01 = pack_bf16x2(v.x, v.y), h23 = pack_bf16x2(v.z, v.w);
+  const float rx = v.x - __uint_as_float(h01 << 16), ry = v.y - __uint_as_float(h01 & 0xffff0000u);
+  const float rz = v.z - __uint_as_float(h23 << 16), rw = v.w - __uint_as_float(h23 & 0xffff0000u);
+  *reinterpret_cast<uint2*>(out) = make_uint2(h01, h23);
+  *reinterpret_cast<uint2*>(out + plane) = make_uint2(pack_bf16x2(rx, ry), pack_bf16x2(rz, rw));
 }
 
 // ---------------------------------------------------------------------------------------

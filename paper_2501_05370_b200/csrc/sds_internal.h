@@ -24,6 +24,8 @@ struct WinArgs {
   float* X;              // [B*L, d] drafted states fed to the target, dense rows
   float* Dq;             // [B*L, d] target outputs, same rows
   uint16_t* Xb;          // [B*L, d] bf16 copy of X (NULL unless a tensor-core denoiser wants it)
+  uint16_t* Xs;          // two bf16 planes (high part, first remainder) of X, xs_plane elements apart (NULL unless
+  size_t xs_plane;       // the float mixture runs its logits on the tensor cores)
   int* n;                // [B]
   int* act;              // [B]      active chain ids (ascending)
   int* rowoff;           // [B+1]    first row of each active slot

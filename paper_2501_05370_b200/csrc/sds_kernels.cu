@@ -93,6 +93,7 @@ __global__ void __launch_bounds__(kBlock) k_init(WinArgs A) {
       st4(A.X + off + i, z);
       if (A.Xb)
         *reinterpret_cast<uint2*>(A.Xb + off + i) = make_uint2(pack_bf16x2(z.x, z.y), pack_bf16x2(z.z, z.w));
+      if (A.Xs) store_split2x4(A.Xs + off + i, A.xs_plane, z);
     }
   } else {
     for (int i = t; i < A.d; i += TPC) {
@@ -184,6 +185,7 @@ __global__ void __launch_bounds__(kBlock) k_draft(WinArgs A) {
         const size_t ro = (size_t)(r0 + j) * A.d + i;
         st4(A.X + ro, y);
         if (A.Xb) *reinterpret_cast<uint2*>(A.Xb + ro) = make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
+        if (A.Xs) store_split2x4(A.Xs + ro, A.xs_plane, y);
         const int k = nb + j;
         const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
         const float4 xi = normal4(A.seed, kStreamDraft, bg, (uint32_t)k, (uint32_t)(i >> 2));

@@ -438,17 +438,7 @@ __global__ void k_f32_to_bf16(const float* __restrict__ x, size_t n, uint16_t* _
   }
 }
 
-// x = h + m + l with h, m, l bfloat16 (each the rounded remainder of the previous ones): three
-// planes that together carry the 24-bit significand of a float
-__device__ __forceinline__ void split3(float x, uint16_t& h, uint16_t& m, uint16_t& l) {
-  const uint32_t ph = pack_bf16x2(x, 0.f) & 0xffffu;
-  const float r1 = x - __uint_as_float(ph << 16);
-  const uint32_t pm = pack_bf16x2(r1, 0.f) & 0xffffu;
-  const float r2 = r1 - __uint_as_float(pm << 16);
-  h = (uint16_t)ph; m = (uint16_t)pm; l = (uint16_t)(pack_bf16x2(r2, 0.f) & 0xffffu);
-}
-
-__global__ void k_split3(const float* __restrict__ x, size_t n, size_t plane, uint16_t* __restrict__ out) {
+__global__ void k_split3(const float* __restrict__ x, size_t n, size_t plane, int nplanes, uint16_t* __restrict__ out) {
   for (size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4; i < n; i += (size_t)gridDim.x * blockDim.x * 4) {
     float v[4] = {0.f, 0.f, 0.f, 0.f};
     if (i + 3 < n) { const float4 t = ld4(x + i); v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; }
@@ -458,6 +448,7 @@ __global__ void k_split3(const float* __restrict__ x, size_t n, size_t plane, ui
     for (int u = 0; u < 4; ++u) split3(v[u], p[0][u], p[1][u], p[2][u]);
 #pragma unroll
     for (int q = 0; q < 3; ++q) {
+      if (q >= nplanes) break;
       if (i + 3 < n) {
         *reinterpret_cast<uint2*>(out + q * plane + i) =
             make_uint2((uint32_t)p[q][0] | ((uint32_t)p[q][1] << 16), (uint32_t)p[q][2] | ((uint32_t)p[q][3] << 16));
@@ -658,11 +649,11 @@ cudaError_t launch_wait_selftest(uint32_t polls, int* status_dev, cudaStream_t s
   return cudaGetLastError();
 }
 
-cudaError_t launch_split3(const float* x, size_t n, size_t plane, uint16_t* out, cudaStream_t st) {
+cudaError_t launch_split3(const float* x, size_t n, size_t plane, int nplanes, uint16_t* out, cudaStream_t st) {
   size_t blocks = (n / 4 + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
   if (blocks < 1) blocks = 1;
-  k_split3<<<(int)blocks, 256, 0, st>>>(x, n, plane, out);
+  k_split3<<<(int)blocks, 256, 0, st>>>(x, n, plane, nplanes, out);
   return cudaGetLastError();
 }
 

@@ -44,7 +44,8 @@ cudaError_t launch_softmax_bf16(const float* logits, const int* nrows_dev, int r
 cudaError_t launch_transpose_bf16(const uint16_t* M, int ncomp, int d, uint16_t* Mt, cudaStream_t st);
 cudaError_t launch_musq_bf16(const uint16_t* means, int ncomp, int d, double* musq, cudaStream_t st);
 cudaError_t launch_wait_selftest(uint32_t polls, int* status_dev, cudaStream_t st);
-cudaError_t launch_split3(const float* x, size_t n, size_t plane, uint16_t* out, cudaStream_t st);
+// the first nplanes (1..3) of the three-way bf16 split of x, planes `plane` elements apart
+cudaError_t launch_split3(const float* x, size_t n, size_t plane, int nplanes, uint16_t* out, cudaStream_t st);
 cudaError_t launch_softmax_split3(const float* logits, const int* nrows_dev, int rows_host, int ncomp, int d,
                                   const float* X, const float* means, const double* musq, const float* logw,
                                   const double* tcond, const int* rowk, size_t rplane, uint16_t* R, cudaStream_t st);

@@ -29,7 +29,10 @@ def test_rng_normals_and_uniforms(b0, k, d):
     for stream in (o.STREAM_DRAFT, o.STREAM_INIT):
         got = sb.rng_normals(seed, stream, b0, nb, k, d).cpu().numpy()
         want = np.stack([o.normals(seed, stream, b0 + i, k, d) for i in range(nb)])
-        assert np.max(np.abs(got - want)) <= 3e-6
+        # the library's Box-Muller uses the special-function unit: lg2 (2^-22), sqrt (2^-23 relative),
+        # sin/cos (2^-20.5 absolute) give at most ~1e-6 r + 1.7e-7/r per normal, r <= 5.77
+        assert np.max(np.abs(got - want)) <= 7e-6
+        assert np.mean(np.abs(got - want)) <= 1e-6
     u = sb.rng_uniforms(seed, b0, nb, k).cpu().numpy()
     uw = np.array([o.uniform01(seed, b0 + i, k) for i in range(nb)])
     assert np.array_equal(u.astype(np.float64), uw)          # exact: multiples of 2^-24
