@@ -218,6 +218,11 @@ int sds_sample_all(sds_ctx* ctx, float* out_dev, int32_t* nfe_calls_dev, int32_t
  * GEMMs on a three-way split of every float operand (six partial products, float accumulation);
  * 0 forces the float ALU kernel. */
 #define SDS_OPT_TENSOR_SPLIT 2
+/* SDS_OPT_GEMM_PAIR (default 1): tensor-core GEMMs whose N is a multiple of 256 run on clusters of
+ * two CTAs that share one 256 x 256 tile (each CTA stages half of the B tile); 0 keeps one CTA
+ * per 128 x 256 tile. Same products, same accumulation order per output element: both give the
+ * same bits. Falls back to one CTA per tile where no cluster can be resident. */
+#define SDS_OPT_GEMM_PAIR 3
 int sds_set_option(sds_ctx* ctx, int32_t option, int64_t value);
 
 /* Temperature of the accept test (Appendix D, temperature rejection): a draft is accepted iff

@@ -93,6 +93,7 @@ struct sds_ctx {
   int32_t qr = 0;
   bool whole_chain = true;          // sds_sample_all may use the whole-chain kernel
   bool tensor_split = true;         // float mixtures of tensor-core shape use the 3-way bf16 split
+  bool gemm_pair = true;            // tensor-core GEMMs with N % 256 == 0 run on CTA pairs
   // optional per-kernel timing: event pairs recorded around each launch, summed on read
   bool prof_on = false;
   std::vector<cudaEvent_t> prof_ev[SDS_PROF_KINDS];
@@ -349,6 +350,7 @@ TcGemmArgs tc_args(sds_ctx* c, Engine& e, const int* rowk, const int* nrows_dev,
   g.rows_cap = (int)e.cap_rows;
   g.rowk = rowk;
   g.err = at<int>(c, c->lay.ctl) + kCtlTcError;
+  g.pair = c->gemm_pair ? 1 : 0;
   return g;
 }
 
@@ -872,6 +874,7 @@ int sds_set_option(sds_ctx* c, int32_t option, int64_t value) {
   switch (option) {
     case SDS_OPT_WHOLE_CHAIN_KERNEL: c->whole_chain = value != 0; return SDS_OK;
     case SDS_OPT_TENSOR_SPLIT: c->tensor_split = value != 0; return SDS_OK;
+    case SDS_OPT_GEMM_PAIR: c->gemm_pair = value != 0; return SDS_OK;
     default: return SDS_EINVAL;
   }
 }

@@ -8,6 +8,11 @@
 //     of its quarter; two warps per quarter split the columns) and apply the epilogue; two
 //     accumulator buffers let the epilogue of tile i overlap the main loop of tile i+1
 //     (persistent CTAs, static round-robin over tiles).
+//   - PAIR variant (N % 256 == 0): two CTAs of a cluster share one 256 x 256 tile
+//     (tcgen05.mma.cta_group::2). Each CTA loads its own 128 rows of A and HALF of the B tile, so
+//     the operand bytes a CTA pulls from L2 per k-block drop from 48 KB to 32 KB and six stages
+//     fit; the leader CTA issues the MMAs for both, each CTA keeps and drains the accumulator of
+//     its own 128 rows. No load is multicast: every CTA fetches what it stages itself.
 // Every wait is bounded: when a wait gives up the kernel records an error word and winds down.
 #include <cuda.h>
 #include <cudaTypedefs.h>
@@ -26,10 +31,11 @@ constexpr int kEpiWarps = 8;       // two warps per TMEM lane quarter, each take
 constexpr int kThreads = 64 + 32 * kEpiWarps;   // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..9: epilogue
 constexpr uint32_t kSpinCap = 1u << 22;
 
-template <int BN> struct TileCfg {
-  static constexpr int kStages = (BN == 256) ? 4 : 6;
+template <int BN, bool PAIR> struct TileCfg {
+  static constexpr int kStages = PAIR ? 6 : ((BN == 256) ? 4 : 6);
+  static constexpr int kBRows = PAIR ? BN / 2 : BN;                         // rows of B one CTA stages
   static constexpr int kABytes = BM * BK * 2;
-  static constexpr int kBBytes = BN * BK * 2;
+  static constexpr int kBBytes = kBRows * BK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kTmemCols = 2 * BN;                                  // two accumulator buffers
   static constexpr int kEpiStageBytes = kEpiWarps * 32 * 33 * 4;            // one padded 32x32 float tile per epilogue warp
@@ -73,6 +79,49 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, in
           smem_u32(dst)),
       "l"(reinterpret_cast<uint64_t>(tm)), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
       : "memory");
+}
+
+// ---- CTA-pair forms ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// address of the same shared-memory object in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load of one CTA of a pair; the bytes are counted on the barrier at cluster address bar_addr
+// (the leader's). Not a multicast: the data lands in the issuing CTA's shared memory only.
+__device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* tm, int c0, int c1, uint32_t bar_addr) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
+          smem_u32(dst)),
+      "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar_addr), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+// arrive on the barrier at the same offset in both CTAs of the pair once the MMAs issued so far are done
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
+                   smem_u32(bar)),
+               "h"((uint16_t)3)
+               : "memory");
 }
 
 // shared-memory matrix descriptor, K-major operand, 128-byte swizzle: rows of 128 bytes, groups of
@@ -147,12 +196,13 @@ __device__ __forceinline__ void epilogue_chunk(const TcGemmArgs& g, const uint32
   // the other epilogues (SiLU hidden layer, acc + bias, C * acc + E * x) are written in the kernel body
 }
 
-template <int BN, int EPI>
+template <int BN, int EPI, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
     k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
               const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB0,
               const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, TcGemmArgs g) {
-  using C = TileCfg<BN>;
+  using C = TileCfg<BN, PAIR>;
+  constexpr int TM = PAIR ? 2 * BM : BM;               // rows of one tile (of the pair's tile)
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte aligned operand stages (required by the 128-byte swizzle), barriers behind them
   uint8_t* stages = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -165,8 +215,11 @@ __global__ void __launch_bounds__(kThreads, 1)
   float* epi_stage = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(full_bar) + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;              // 0: leader (issues the MMAs of the pair)
+  const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int nworkers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   const int M = g.nrows_dev ? min(*g.nrows_dev, g.rows_host) : g.rows_host;
-  const int m_tiles = (M + BM - 1) / BM, n_tiles = g.N / BN;
+  const int m_tiles = (M + TM - 1) / TM, n_tiles = g.N / BN;
   const int total_tiles = m_tiles * n_tiles;
   // K loop = nseg segments of K/BK blocks; segment s multiplies plane a_idx[s] of A with plane
   // b_idx[s] of B into the same accumulator (split-precision products; one segment otherwise)
@@ -175,18 +228,27 @@ __global__ void __launch_bounds__(kThreads, 1)
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::kStages; ++s) { mbar_init(full_bar + s, 1); mbar_init(empty_bar + s, 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(tfull_bar + s, 1); mbar_init(tempty_bar + s, kEpiWarps); }
+    // the leader's "drained" barriers collect the epilogue warps of both CTAs
+    for (int s = 0; s < 2; ++s) { mbar_init(tfull_bar + s, 1); mbar_init(tempty_bar + s, PAIR ? 2 * kEpiWarps : kEpiWarps); }
     *abort_s = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_s)),
-                 "r"((uint32_t)C::kTmemCols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (PAIR) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_s)),
+                   "r"((uint32_t)C::kTmemCols)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_s)),
+                   "r"((uint32_t)C::kTmemCols)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();          // the peer's barriers exist before anything is sent to them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_base_s;
 
@@ -196,16 +258,27 @@ __global__ void __launch_bounds__(kThreads, 1)
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-        const int m0 = (t / n_tiles) * BM, n0 = (t % n_tiles) * BN;
+      const uint32_t leader_full0 = PAIR ? map_to_cta(smem_u32(full_bar), 0u) : 0u;
+      for (int t = worker; t < total_tiles && ok; t += nworkers) {
+        const int m0 = (t / n_tiles) * TM + (int)rank * BM, n0 = (t % n_tiles) * BN + (int)rank * C::kBRows;
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(empty_bar + stage, phase ^ 1u, abort_s)) { ok = false; break; }
           uint8_t* sa = stages + stage * C::kStageBytes;
-          mbar_expect_tx(full_bar + stage, (uint32_t)C::kStageBytes);
           const int seg = kb / kb_seg, kk = (kb - seg * kb_seg) * BK;
           const int ai = g.a_idx[seg], bi = g.b_idx[seg];
-          tma_load_2d(sa, ai == 0 ? &tmA0 : (ai == 1 ? &tmA1 : &tmA2), kk, m0, full_bar + stage);
-          tma_load_2d(sa + C::kABytes, bi == 0 ? &tmB0 : (bi == 1 ? &tmB1 : &tmB2), kk, n0, full_bar + stage);
+          const CUtensorMap* ta = ai == 0 ? &tmA0 : (ai == 1 ? &tmA1 : &tmA2);
+          const CUtensorMap* tb = bi == 0 ? &tmB0 : (bi == 1 ? &tmB1 : &tmB2);
+          if (PAIR) {
+            // the leader's barrier counts the bytes of both CTAs' loads
+            if (rank == 0) mbar_expect_tx(full_bar + stage, 2u * (uint32_t)C::kStageBytes);
+            const uint32_t fb = leader_full0 + (uint32_t)stage * 8u;
+            tma_load_2d_pair(sa, ta, kk, m0, fb);
+            tma_load_2d_pair(sa + C::kABytes, tb, kk, n0, fb);
+          } else {
+            mbar_expect_tx(full_bar + stage, (uint32_t)C::kStageBytes);
+            tma_load_2d(sa, ta, kk, m0, full_bar + stage);
+            tma_load_2d(sa + C::kABytes, tb, kk, n0, full_bar + stage);
+          }
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -216,13 +289,13 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc(BM, BN);
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = make_idesc(TM, BN);
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+      for (int t = worker; t < total_tiles && ok; t += nworkers, ++it) {
         const int buf = it & 1;
         const uint32_t bphase = (uint32_t)(it >> 1) & 1u;
         if (!mbar_wait(tempty_bar + buf, bphase ^ 1u, abort_s)) { ok = false; break; }
@@ -236,12 +309,14 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll
           for (int k = 0; k < BK / UK; ++k) {
             // 32 bytes further along K inside the 128-byte swizzle row: +2 in the (>>4) address field
-            umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb | k) ? 1u : 0u);
+            if (PAIR) umma_bf16_pair(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb | k) ? 1u : 0u);
+            else umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb | k) ? 1u : 0u);
           }
-          umma_commit(empty_bar + stage);                    // frees the stage once these MMAs have read it
+          // frees the stage (in both CTAs of a pair) once these MMAs have read it
+          if (PAIR) umma_commit_pair(empty_bar + stage); else umma_commit(empty_bar + stage);
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
         }
-        if (ok) umma_commit(tfull_bar + buf);                // accumulator complete
+        if (ok) { if (PAIR) umma_commit_pair(tfull_bar + buf); else umma_commit(tfull_bar + buf); }   // accumulator complete
       }
       if (!ok) {
         *abort_s = 1;
@@ -254,10 +329,12 @@ __global__ void __launch_bounds__(kThreads, 1)
     constexpr int kCols = BN / 2;                      // columns per epilogue warp
     int it = 0;
     bool ok = true;
-    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+    // "drained" goes to the leader's barrier (the MMA issuer of the pair waits there)
+    const uint32_t drained0 = (PAIR && rank != 0) ? map_to_cta(smem_u32(tempty_bar), 0u) : 0u;
+    for (int t = worker; t < total_tiles && ok; t += nworkers, ++it) {
       const int buf = it & 1;
       const uint32_t bphase = (uint32_t)(it >> 1) & 1u;
-      const int m0 = (t / n_tiles) * BM, n0 = (t % n_tiles) * BN + half * kCols;
+      const int m0 = (t / n_tiles) * TM + (int)rank * BM, n0 = (t % n_tiles) * BN + half * kCols;
       const int row = m0 + q * 32 + lane;
       const bool live = row < M;
       const int krow = (live && g.rowk) ? __ldg(g.rowk + row) : 0;
@@ -310,7 +387,10 @@ __global__ void __launch_bounds__(kThreads, 1)
           if (c + 32 >= kCols) {                              // accumulator fully read: hand the buffer back
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar + buf);
+            if (lane == 0) {
+              if (PAIR && rank != 0) mbar_arrive_cluster(drained0 + (uint32_t)buf * 8u);
+              else mbar_arrive(tempty_bar + buf);
+            }
           }
 #pragma unroll
           for (int j = 0; j < 32; ++j) stg[lane * 33 + j] = __uint_as_float(acc[j]);
@@ -355,7 +435,10 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(tempty_bar + buf);
+        if (lane == 0) {
+              if (PAIR && rank != 0) mbar_arrive_cluster(drained0 + (uint32_t)buf * 8u);
+              else mbar_arrive(tempty_bar + buf);
+            }
       }
     }
     if (!ok && lane == 0) {
@@ -371,10 +454,15 @@ __global__ void __launch_bounds__(kThreads, 1)
     for (int i = 0; i < 2000; ++i) __nanosleep(1000);
   }
   __syncthreads();
+  if (PAIR) cluster_sync_all();          // neither CTA leaves while the other may still reach its memory
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::kTmemCols)
-                 : "memory");
+    if (PAIR)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::kTmemCols)
+                   : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::kTmemCols)
+                   : "memory");
   }
 }
 
@@ -576,24 +664,50 @@ bool make_tmap(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t K, uin
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, int EPI>
+template <int BN, int EPI, bool PAIR>
 cudaError_t launch_t(const TcGemmArgs& g, const void* A, const void* B, int grid_tiles_ub, cudaStream_t st) {
-  using C = TileCfg<BN>;
+  using C = TileCfg<BN, PAIR>;
   CUtensorMap tmA[3], tmB[3];
   for (int i = 0; i < 3; ++i) {
     const uint16_t* a = static_cast<const uint16_t*>(A) + (size_t)i * g.a_plane;
     const uint16_t* b = static_cast<const uint16_t*>(B) + (size_t)i * g.b_plane;
     if (!make_tmap(&tmA[i], g.nplanes > i ? a : A, (uint64_t)g.rows_cap, (uint64_t)g.K, BM)) return cudaErrorInvalidValue;
-    if (!make_tmap(&tmB[i], g.nplanes > i ? b : B, (uint64_t)g.N, (uint64_t)g.K, BN)) return cudaErrorInvalidValue;
+    if (!make_tmap(&tmB[i], g.nplanes > i ? b : B, (uint64_t)g.N, (uint64_t)g.K, C::kBRows)) return cudaErrorInvalidValue;
   }
-  cudaError_t e = cudaFuncSetAttribute(k_gemm_tc<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(k_gemm_tc<BN, EPI, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
   if (e != cudaSuccess) return e;
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (PAIR) {
+    // one cluster of two CTAs per tile of 256 rows; grid_tiles_ub counts those tiles
+    int pairs = grid_tiles_ub < sms / 2 ? grid_tiles_ub : sms / 2;
+    if (pairs < 1) pairs = 1;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(2 * pairs);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = C::kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int resident = 0;                      // clusters that fit at once (a GPC with an odd SM count leaves one SM out)
+    e = cudaOccupancyMaxActiveClusters(&resident, k_gemm_tc<BN, EPI, PAIR>, &cfg);
+    if (e != cudaSuccess || resident < 1) {            // no room for a cluster here: the caller takes the one-CTA kernel
+      cudaGetLastError();
+      return cudaErrorLaunchOutOfResources;
+    }
+    if (pairs > resident) {
+      pairs = resident;
+      cfg.gridDim = dim3(2 * pairs);
+    }
+    return cudaLaunchKernelEx(&cfg, k_gemm_tc<BN, EPI, PAIR>, tmA[0], tmA[1], tmA[2], tmB[0], tmB[1], tmB[2], g);
+  }
   int grid = grid_tiles_ub < sms ? grid_tiles_ub : sms;
   if (grid < 1) grid = 1;
-  k_gemm_tc<BN, EPI><<<grid, kThreads, C::kSmemBytes, st>>>(tmA[0], tmA[1], tmA[2], tmB[0], tmB[1], tmB[2], g);
+  k_gemm_tc<BN, EPI, PAIR><<<grid, kThreads, C::kSmemBytes, st>>>(tmA[0], tmA[1], tmA[2], tmB[0], tmB[1], tmB[2], g);
   return cudaGetLastError();
 }
 
@@ -608,11 +722,18 @@ cudaError_t launch_gemm_tc(int epi, const TcGemmArgs& g_in, const void* A_bf16, 
   if (!tc_shape_ok(g.N, g.K) || g.rows_cap <= 0 || g.rows_host > g.rows_cap) return cudaErrorInvalidValue;
   if (g.rows_host <= 0) return cudaSuccess;
   const bool wide = (g.N % 256) == 0;
-  const int m_tiles = (g.rows_host + BM - 1) / BM;
-  const int tiles = m_tiles * (g.N / (wide ? 256 : 128));
+  const bool pair = wide && g.pair != 0;
+  const int tm = pair ? 2 * BM : BM;
+  const int m_tiles = (g.rows_host + tm - 1) / tm;
+  int tiles = m_tiles * (g.N / (wide ? 256 : 128));
 #define SDS_TC_CASE(E)                                                                     \
   case E:                                                                                  \
-    return wide ? launch_t<256, E>(g, A_bf16, B_bf16, tiles, st) : launch_t<128, E>(g, A_bf16, B_bf16, tiles, st);
+    if (pair) {                                                                            \
+      const cudaError_t e_ = launch_t<256, E, true>(g, A_bf16, B_bf16, tiles, st);         \
+      if (e_ != cudaErrorLaunchOutOfResources) return e_;                                  \
+      tiles = ((g.rows_host + BM - 1) / BM) * (g.N / 256);                                 \
+    }                                                                                      \
+    return wide ? launch_t<256, E, false>(g, A_bf16, B_bf16, tiles, st) : launch_t<128, E, false>(g, A_bf16, B_bf16, tiles, st);
   switch (epi) {
     SDS_TC_CASE(kEpiMlpHidden)
     SDS_TC_CASE(kEpiBiasF32)

@@ -32,6 +32,7 @@ struct TcGemmArgs {
   // split-precision products: A and B each come as nplanes bf16 planes (a_plane / b_plane elements
   // apart); segment s of the K loop multiplies plane a_idx[s] of A with plane b_idx[s] of B.
   // nseg = 0 means one plane, one segment.
+  int pair;              // 1: two CTAs share a 256 x 256 tile (needs N % 256 == 0; ignored otherwise)
   int nseg, nplanes;
   size_t a_plane, b_plane;
   uint8_t a_idx[8], b_idx[8];
