@@ -17,8 +17,8 @@ namespace {
 // floats of shared memory: parameters (rounded to 16 bytes) and per-warp window storage
 __host__ __device__ inline int fused_param_floats(int ncomp, int d) { return small_param_floats(ncomp, d); }
 __host__ __device__ inline int fused_warp_floats(int d, int L) {
-  // S1/S2 (doubles), two converted rows (doubles), W[L+1], Dq[L], Dc, e-scratch
-  return 4 * kMaxL + 4 * small_ldd(d) + (2 * L + 2) * small_ldx(d) + 32;
+  // S1/S2 (doubles), logit hand-off (doubles), W[L+1], Dq[L], Dc, e-scratch
+  return 4 * kMaxL + kSmallScratchFloats + (2 * L + 2) * small_ldx(d) + 32;
 }
 
 template <int G, bool VEC4>
@@ -28,12 +28,12 @@ __global__ void __maxnreg__(72) k_fused_small(WinArgs A, GmmArgs P) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   const int g = lane / G, gl = lane % G;
   const int d = A.d, L = A.L, K = A.K;
-  const int ldx = small_ldx(d), ldd = small_ldd(d);
+  const int ldx = small_ldx(d);
   const SmallParams S = small_stage_params(P.means, P.musq, P.logw, P.ncomp, d, smem);
   float* wbase = smem + fused_param_floats(P.ncomp, d) + (size_t)warp * fused_warp_floats(d, L);
   double* sS = reinterpret_cast<double*>(wbase);               // [2][kMaxL]
-  double* sXd = sS + 2 * kMaxL + g * ldd;                      // converted row of this lane group
-  float* sW = wbase + 4 * kMaxL + 4 * ldd;
+  double* sLg = sS + 2 * kMaxL;                                // logit hand-off of the row routine
+  float* sW = wbase + 4 * kMaxL + kSmallScratchFloats;
   float* sDq = sW + (L + 1) * ldx;
   float* sDc = sDq + L * ldx;
   float* sEs = sDc + ldx;
@@ -54,7 +54,7 @@ __global__ void __maxnreg__(72) k_fused_small(WinArgs A, GmmArgs P) {
       for (int i = lane; i < d; i += 32) sW[i] = normal1(A.seed, kStreamInit, bg, 0u, (uint32_t)i);
     }
     __syncwarp();
-    gmm_row_small<G>(sW, sXd, g == 0, S, __ldg(P.tcond + 0), __ldg(P.tcond + 1), __ldg(P.tcond + 2),
+    gmm_row_small<G>(sW, ldx, sLg, g == 0, S, __ldg(P.tcond + 0), __ldg(P.tcond + 1), __ldg(P.tcond + 2),
                      __ldg(P.tcond + 3), sEs + g * G, sDc, gl);
     int n = 0, calls = 1, rows = 1;
     bool frozen = false;
@@ -103,7 +103,7 @@ __global__ void __maxnreg__(72) k_fused_small(WinArgs A, GmmArgs P) {
         const bool valid = j < Lt;
         const int jj = valid ? j : 0;
         const int k = n + jj;
-        gmm_row_small<G>(sW + jj * ldx, sXd, valid, S, __ldg(P.tcond + 4 * k + 0), __ldg(P.tcond + 4 * k + 1),
+        gmm_row_small<G>(sW + j0 * ldx, ldx, sLg, valid, S, __ldg(P.tcond + 4 * k + 0), __ldg(P.tcond + 4 * k + 1),
                          __ldg(P.tcond + 4 * k + 2), __ldg(P.tcond + 4 * k + 3), sEs + g * G, sDq + jj * ldx, gl);
       }
       // S1 = |Delta|^2, S2 = Delta.Z per position

@@ -89,13 +89,13 @@ __global__ void __launch_bounds__(kSmallWarps * 32) k_gmm_small(GmmArgs P, const
   constexpr int RPW = 32 / G;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane / G, gl = lane % G;
   const int nrows = nrows_dev ? min(*nrows_dev, rows_host) : rows_host;
-  const int ldx = small_ldx(P.d), ldd = small_ldd(P.d);
+  const int ldx = small_ldx(P.d);
   const SmallParams S = small_stage_params(P.means, P.musq, P.logw, P.ncomp, P.d, smem);
-  // per warp: [RPW converted rows (double)] [RPW rows (float)] [32 floats of e-scratch]
-  const int per_warp = RPW * (2 * ldd + ldx) + 32;
+  // per warp: [logit hand-off (32 doubles)] [RPW rows (float)] [32 floats of e-scratch]
+  const int per_warp = kSmallScratchFloats + RPW * ldx + 32;
   float* wbase = smem + small_param_floats(P.ncomp, P.d) + (size_t)warp * per_warp;
-  double* s_xd = reinterpret_cast<double*>(wbase) + g * ldd;
-  float* s_x = wbase + RPW * 2 * ldd;
+  double* s_lg = reinterpret_cast<double*>(wbase);
+  float* s_x = wbase + kSmallScratchFloats;
   float* s_es = s_x + RPW * ldx + g * G;
   __syncthreads();
   const int stride = gridDim.x * kSmallWarps * RPW;
@@ -113,7 +113,7 @@ __global__ void __launch_bounds__(kSmallWarps * 32) k_gmm_small(GmmArgs P, const
       tA = __ldg(P.tcond + 4 * k + 0); tB = __ldg(P.tcond + 4 * k + 1);
       tC = __ldg(P.tcond + 4 * k + 2); tE = __ldg(P.tcond + 4 * k + 3);
     }
-    gmm_row_small<G>(s_x + g * ldx, s_xd, valid, S, tA, tB, tC, tE, s_es, out + (size_t)(valid ? row : 0) * P.d, gl);
+    gmm_row_small<G>(s_x, ldx, s_lg, valid, S, tA, tB, tC, tE, s_es, out + (size_t)(valid ? row : 0) * P.d, gl);
   }
 }
 
@@ -341,7 +341,7 @@ constexpr size_t kTiledSmem = (size_t)(kTNC * kRS + kTK * kM2S + kTK * kMS + kTR
 
 size_t small_smem_bytes(int ncomp, int d) {
   const int G = small_group(ncomp), RPW = 32 / G;
-  return ((size_t)small_param_floats(ncomp, d) + (size_t)kSmallWarps * (RPW * (2 * small_ldd(d) + small_ldx(d)) + 32)) * 4;
+  return ((size_t)small_param_floats(ncomp, d) + (size_t)kSmallWarps * (kSmallScratchFloats + RPW * small_ldx(d) + 32)) * 4;
 }
 
 }  // namespace
