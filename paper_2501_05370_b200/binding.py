@@ -381,6 +381,7 @@ class Sampler:
     OPT_WHOLE_CHAIN_KERNEL = 1
     OPT_TENSOR_SPLIT = 2
     OPT_GEMM_PAIR = 3
+    OPT_VERIFY_EARLY_EXIT = 4
 
     def set_option(self, option: int, value: int):
         self._chk(self.lib.sds_set_option(self.h, option, value), "sds_set_option")

@@ -94,6 +94,7 @@ struct sds_ctx {
   bool whole_chain = true;          // sds_sample_all may use the whole-chain kernel
   bool tensor_split = true;         // float mixtures of tensor-core shape use the 3-way bf16 split
   bool gemm_pair = true;            // tensor-core GEMMs with N % 256 == 0 run on CTA pairs
+  bool early_exit = true;           // verify stops reading a window after the block with the first rejection
   // optional per-kernel timing: event pairs recorded around each launch, summed on read
   bool prof_on = false;
   std::vector<cudaEvent_t> prof_ev[SDS_PROF_KINDS];
@@ -246,6 +247,7 @@ WinArgs win_args(sds_ctx* c) {
   A.B = (int)c->B; A.d = c->d; A.L = c->L; A.K = c->K;
   A.mode = c->mode;
   A.inv_tau = 1.0 / c->tau;
+  A.early_exit = c->early_exit ? 1 : 0;
   A.seed = c->seed; A.chain_off = (uint64_t)c->chain_off;
   A.a = at<float>(c, c->lay.a); A.c = at<float>(c, c->lay.c); A.sigma = at<float>(c, c->lay.sigma);
   A.Y = at<float>(c, c->lay.Y); A.Dc = at<float>(c, c->lay.Dc); A.T = at<float>(c, c->lay.T);
@@ -875,6 +877,7 @@ int sds_set_option(sds_ctx* c, int32_t option, int64_t value) {
     case SDS_OPT_WHOLE_CHAIN_KERNEL: c->whole_chain = value != 0; return SDS_OK;
     case SDS_OPT_TENSOR_SPLIT: c->tensor_split = value != 0; return SDS_OK;
     case SDS_OPT_GEMM_PAIR: c->gemm_pair = value != 0; return SDS_OK;
+    case SDS_OPT_VERIFY_EARLY_EXIT: c->early_exit = value != 0; return SDS_OK;
     default: return SDS_EINVAL;
   }
 }

@@ -13,6 +13,8 @@ struct WinArgs {
   int mode;              // 0: carried target output; 1: target output at Y_n, recomputed before every
                          // window; 2: independent draft model evaluated at every drafted state
   double inv_tau;        // 1 / temperature of the accept test (1 = the exact method)
+  int early_exit;        // verify stops reading a chain's window after the block of four positions
+                         // that holds its first rejection (large-d kernels only)
   uint64_t seed;
   uint64_t chain_off;
   const float* a;        // [K]

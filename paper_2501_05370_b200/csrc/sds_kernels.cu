@@ -650,84 +650,115 @@ __global__ void __launch_bounds__(TPC > kBlock ? TPC : kBlock) k_verify_reg(WinA
     vc[e] = (i < A.d) ? ld4(A.Dc + cb + i) : zero4;
     vp[e] = (i < A.d) ? ld4(A.X + (size_t)r0 * A.d + i) : zero4;
   }
-  double myS1 = 0.0, myS2 = 0.0;
-  for (int j = 1; j <= Lt; ++j) {
-    const int k = nb + j - 1;
-    const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
-    const float inv_s = 1.0f / sk, cs = ck * inv_s;
-    const float* wj = (j < Lt) ? A.X + (size_t)(r0 + j) * A.d : A.T + cb;
-    const float* dq = A.Dq + (size_t)(r0 + j - 1) * A.d;
-    float4 vj[EPT], vq[EPT];
-#pragma unroll
-    for (int e = 0; e < EPT; ++e) {
-      const int i = (t + e * TPC) * 4;
-      vj[e] = (i < A.d) ? ld4(wj + i) : zero4;
-      vq[e] = (i < A.d) ? ld4(dq + i) : zero4;
-      if (A.Dp && i < A.d) vc[e] = ld4(A.Dp + (size_t)(r0 + j - 1) * A.d + i);   // independent draft model
-    }
-    double p1 = 0.0, p2 = 0.0;
-#pragma unroll
-    for (int e = 0; e < EPT; ++e) {
-      if ((t + e * TPC) * 4 < A.d) {
-        float D, Z;
-        delta_z(vp[e].x, vj[e].x, vq[e].x, vc[e].x, ak, ck, cs, inv_s, D, Z);
-        p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
-        delta_z(vp[e].y, vj[e].y, vq[e].y, vc[e].y, ak, ck, cs, inv_s, D, Z);
-        p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
-        delta_z(vp[e].z, vj[e].z, vq[e].z, vc[e].z, ak, ck, cs, inv_s, D, Z);
-        p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
-        delta_z(vp[e].w, vj[e].w, vq[e].w, vc[e].w, ak, ck, cs, inv_s, D, Z);
-        p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
-      }
-      vp[e] = vj[e];
-    }
-    p1 = warp_sum(p1);
-    p2 = warp_sum(p2);
-    if (TPC == 32) {
-      if (lane == j - 1) { myS1 = p1; myS2 = p2; }
-    } else if (lane == 0) {
-      s_red[(j - 1) * kWarps + warp] = p1;
-      s_red[kMaxL * kWarps + (j - 1) * kWarps + warp] = p2;
-    }
-  }
-  if (TPC > 32) {
-    __syncthreads();
-    if (warp == 0 && lane < Lt) {
-      for (int w = 0; w < kWarps; ++w) {
-        myS1 += s_red[lane * kWarps + w];
-        myS2 += s_red[kMaxL * kWarps + lane * kWarps + w];
-      }
-    }
-  }
-  int jstar = 0;
+  // Positions are taken in blocks; with early exit (one chain per CTA, option on) the accept tests
+  // of a block are decided before the next block is read, and nothing after the block that holds
+  // the first rejection is read at all: those positions report zeros.
+  const bool early = (TPC > 32) && A.early_exit != 0;
+  const int blk = early ? 4 : Lt;
+  int jstar = Lt + 1;
   float coef = 0.f;
-  if (warp == 0) {
-    const bool valid = lane < Lt;
-    bool acc = true, bad = false;
-    if (valid) {
-      const float U = uniform01(A.seed, bg, (uint32_t)(nb + lane));
-      const float lu = logf(U);
-      const float ellf = (float)((-0.5 * myS1 - myS2) * A.inv_tau);   // tempered log ratio (inv_tau = 1: exact method)
-      acc = (myS1 < 1e-30) || (lu <= ellf);
-      bad = !isfinite(ellf);
-      const size_t o = (size_t)b * A.L + lane;
-      A.S1[o] = myS1;
-      A.S2[o] = myS2;
-      A.ell[o] = ellf;
-      A.logU[o] = lu;
+  uint32_t amask = 0u;
+  bool frozen = false;
+  int done = 0;                                          // positions evaluated so far
+  for (int jb = 1; jb <= Lt; jb += blk) {
+    const int je = min(Lt, jb + blk - 1);
+    double myS1 = 0.0, myS2 = 0.0;
+    for (int j = jb; j <= je; ++j) {
+      const int k = nb + j - 1;
+      const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
+      const float inv_s = 1.0f / sk, cs = ck * inv_s;
+      const float* wj = (j < Lt) ? A.X + (size_t)(r0 + j) * A.d : A.T + cb;
+      const float* dq = A.Dq + (size_t)(r0 + j - 1) * A.d;
+      float4 vj[EPT], vq[EPT];
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) {
+        const int i = (t + e * TPC) * 4;
+        vj[e] = (i < A.d) ? ld4(wj + i) : zero4;
+        vq[e] = (i < A.d) ? ld4(dq + i) : zero4;
+        if (A.Dp && i < A.d) vc[e] = ld4(A.Dp + (size_t)(r0 + j - 1) * A.d + i);   // independent draft model
+      }
+      double p1 = 0.0, p2 = 0.0;
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) {
+        if ((t + e * TPC) * 4 < A.d) {
+          float D, Z;
+          delta_z(vp[e].x, vj[e].x, vq[e].x, vc[e].x, ak, ck, cs, inv_s, D, Z);
+          p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+          delta_z(vp[e].y, vj[e].y, vq[e].y, vc[e].y, ak, ck, cs, inv_s, D, Z);
+          p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+          delta_z(vp[e].z, vj[e].z, vq[e].z, vc[e].z, ak, ck, cs, inv_s, D, Z);
+          p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+          delta_z(vp[e].w, vj[e].w, vq[e].w, vc[e].w, ak, ck, cs, inv_s, D, Z);
+          p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+        }
+        vp[e] = vj[e];
+      }
+      p1 = warp_sum(p1);
+      p2 = warp_sum(p2);
+      if (TPC == 32) {
+        if (lane == j - 1) { myS1 = p1; myS2 = p2; }
+      } else if (lane == 0) {
+        s_red[(j - 1) * kWarps + warp] = p1;
+        s_red[kMaxL * kWarps + (j - 1) * kWarps + warp] = p2;
+      }
     }
-    const uint32_t vmask = (Lt >= 32) ? 0xffffffffu : ((1u << Lt) - 1u);
-    const uint32_t amask = __ballot_sync(0xffffffffu, acc) & vmask;
-    const uint32_t bmask = __ballot_sync(0xffffffffu, bad) & vmask;
-    const uint32_t rej = ~amask & vmask;
-    jstar = rej ? __ffs(rej) : Lt + 1;
-    if (bmask) jstar = -1;
-    const int src = (jstar >= 1 && jstar <= Lt) ? jstar - 1 : 0;
-    coef = __shfl_sync(0xffffffffu, (float)(2.0 * myS2 / myS1), src);
+    const bool mine = lane >= jb - 1 && lane <= je - 1;   // positions of this block, one per lane of warp 0
+    if (TPC > 32) {
+      __syncthreads();
+      if (warp == 0 && mine) {
+        for (int w = 0; w < kWarps; ++w) {
+          myS1 += s_red[lane * kWarps + w];
+          myS2 += s_red[kMaxL * kWarps + lane * kWarps + w];
+        }
+      }
+    }
+    if (warp == 0) {
+      bool acc = true, bad = false;
+      if (mine) {
+        const float U = uniform01(A.seed, bg, (uint32_t)(nb + lane));
+        const float lu = logf(U);
+        const float ellf = (float)((-0.5 * myS1 - myS2) * A.inv_tau);   // tempered log ratio (inv_tau = 1: exact method)
+        acc = (myS1 < 1e-30) || (lu <= ellf);
+        bad = !isfinite(ellf);
+        const size_t o = (size_t)b * A.L + lane;
+        A.S1[o] = myS1;
+        A.S2[o] = myS2;
+        A.ell[o] = ellf;
+        A.logU[o] = lu;
+      }
+      const uint32_t bmask_all = (je >= 32) ? 0xffffffffu : ((1u << je) - 1u);
+      const uint32_t vmask = bmask_all & ~((1u << (jb - 1)) - 1u);
+      const uint32_t am = __ballot_sync(0xffffffffu, acc) & vmask;
+      const uint32_t bm = __ballot_sync(0xffffffffu, bad) & vmask;
+      const uint32_t rej = ~am & vmask;
+      amask |= am;
+      if (bm) frozen = true;
+      if (rej && jstar > Lt) {
+        jstar = __ffs(rej);
+        coef = __shfl_sync(0xffffffffu, (float)(2.0 * myS2 / myS1), jstar - 1);
+      }
+      if (TPC > 32 && lane == 0) { s_jstar = frozen ? -1 : jstar; s_coef = coef; }
+    }
+    done = je;
+    if (TPC > 32) {
+      __syncthreads();
+      const int js = s_jstar;
+      if (js < 0 || js <= Lt) break;                      // frozen, or first rejection found
+    }
+  }
+  if (warp == 0) {
+    if (lane >= done && lane < Lt) {                      // positions that were not evaluated
+      const size_t o = (size_t)b * A.L + lane;
+      A.S1[o] = 0.0;
+      A.S2[o] = 0.0;
+      A.ell[o] = 0.f;
+      A.logU[o] = 0.f;
+    }
+    if (frozen) jstar = -1;
     if (lane == 0) {
       A.accmask[b] = amask;
       A.jstar[b] = jstar;
-      if (bmask) atomicOr(A.ctl + kCtlError, kErrNonFinite);
+      if (frozen) atomicOr(A.ctl + kCtlError, kErrNonFinite);
       if (TPC > 32) { s_jstar = jstar; s_coef = coef; }
     }
   }

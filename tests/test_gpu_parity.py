@@ -87,6 +87,7 @@ def test_split_precision_tensor_path_agrees_with_float_alu_path():
 
 def _window_check(s, w, den, a32, c32, s32, seed, chain_off, stats, chains=None, draft_den=None, proj=None):
     """Runs draft + verify on the GPU and replays the verification on the GPU's own arrays."""
+    s.set_option(s.OPT_VERIFY_EARLY_EXIT, 0)      # these checks look at every position of the window
     B, L, d, K = s.B, s.L, s.d, s.K
     ctl = s.get(sb.GET_CTL)
     na, nrows = int(ctl[0]), int(ctl[1])
@@ -667,4 +668,62 @@ def test_projection_onto_the_whole_space_is_the_exact_method():
     got = [x.cpu().numpy() for x in s.sample_all()]
     same = np.sum(got[1] == base[1])
     assert same >= w.B - 2                              # decisions can differ only inside the rounding band
+    s.close()
+
+
+# ----------------------------------------------------------------------------------------
+# verify with early exit (blocks of four positions; nothing after the first rejection is read)
+# ----------------------------------------------------------------------------------------
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("d,L,B", [(1024, 12, 40), (3072, 8, 24), (4096, 16, 12), (16384, 16, 6)])
+def test_verify_early_exit_only_skips_diagnostics(d, L, B):
+    w = wl.WORKLOADS["cfg2"].scaled(B=B, d=d, K=3 * L + 5, L=L)
+    gp = w.gmm_params(d=d, ncomp=8)
+    res = {}
+    for early in (1, 0):
+        s = sds.sampler_for(w, gmm=gp, seed=61)
+        s.set_option(s.OPT_VERIFY_EARLY_EXIT, early)
+        s.reset()
+        wins = []
+        for _ in range(3):
+            s.draft(); s.verify_window()
+            wins.append(dict(n=s.get(sb.GET_N).copy(), X=s.get(sb.GET_X).copy(), T=s.get(sb.GET_TAIL).copy(),
+                             js=s.get(sb.GET_JSTAR).copy(), am=s.get(sb.GET_ACCMASK).copy(), S1=s.get(sb.GET_S1).copy(),
+                             S2=s.get(sb.GET_S2).copy(), ell=s.get(sb.GET_ELL).copy(), lu=s.get(sb.GET_LOGU).copy()))
+            s.advance()
+        full = [x.cpu().numpy() for x in s.sample_all()]
+        res[early] = (wins, full)
+        s.close()
+    skipped = 0
+    for a, b in zip(res[1][0], res[0][0]):
+        assert np.array_equal(a["n"], b["n"]) and np.array_equal(a["js"], b["js"])
+        assert np.array_equal(a["X"], b["X"]) and np.array_equal(a["T"], b["T"])      # same reflected states
+        for c in range(B):
+            Lt = min(L, w.K - int(a["n"][c]))
+            js = int(a["js"][c])
+            n_eval = Lt if js > Lt else min(Lt, 4 * ((js + 3) // 4))
+            keep = (1 << n_eval) - 1
+            assert int(a["am"][c]) == int(b["am"][c]) & keep
+            for key in ("S1", "S2", "ell", "lu"):
+                assert np.array_equal(a[key][c, :n_eval], b[key][c, :n_eval])
+                assert not np.any(a[key][c, n_eval:Lt])
+            skipped += Lt - n_eval
+    assert skipped > 0                                                                # the case does skip positions
+    assert all(np.array_equal(x, y) for x, y in zip(res[1][1], res[0][1]))            # whole runs agree bit for bit
+
+
+@pytest.mark.gpu
+def test_early_exit_run_matches_oracle():
+    w = wl.WORKLOADS["cfg2"].scaled(B=16, d=1024, K=40, L=12)
+    gp = w.gmm_params(d=1024, ncomp=6)
+    den, a, c, sig = oracle_setup(w, gmm=gp)
+    s = sds.sampler_for(w, gmm=gp, seed=62)
+    out, calls, rows = [x.cpu().numpy() for x in s.sample_all()]
+    bad = 0
+    for b in range(6):
+        r = o.speculative_chain(den, a, c, sig, w.L, 62, b, w.d)
+        bad += not (r["nfe_calls"] == calls[b] and r["nfe_rows"] == rows[b] and rel_l2(out[b], r["Y"]) <= 1e-4)
+    assert bad <= 1
     s.close()

@@ -23,6 +23,7 @@ def _det_coeffs(w):
 def _picard_window(s, w, den, a, c, sig, a_det, c_det, calls, seed, chains, stats, tol=1e-5):
     """One window on the GPU (draft, verify, advance), replayed by the oracle: the Picard points and
     draft means from the oracle's own trajectory, the verification on the GPU's arrays."""
+    s.set_option(s.OPT_VERIFY_EARLY_EXIT, 0)      # these checks look at every position of the window
     B, L, d, K = s.B, s.L, s.d, s.K
     na = int(s.get(sb.GET_CTL)[0])
     act, rowoff, n = s.get(sb.GET_ACT)[:na], s.get(sb.GET_ROWOFF)[:na + 1], s.get(sb.GET_N)

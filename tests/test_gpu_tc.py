@@ -57,6 +57,7 @@ def test_large_mixture_denoiser_rows(d, ncomp, rows):
 def _forced_window(s, w, den, seed, off, windows, chains=None):
     """Decisions and log ratios of the verify step replayed by the oracle on the GPU's own arrays
     (the denoiser outputs are the GPU's; their parity is checked separately at 2e-2)."""
+    s.set_option(s.OPT_VERIFY_EARLY_EXIT, 0)      # these checks look at every position of the window
     import math
     a32, c32, s32, _ = sds.schedule_for(w)
     a64, c64, s64 = a32.astype(np.float64), c32.astype(np.float64), s32.astype(np.float64)
