@@ -324,8 +324,13 @@ def run_gpu(args, w):
     ms_per_step = ms_total / steps
     value = world * B * K / (ms_per_step * 1e-3)
     e2e_value = world * B * K / (ms_e2e / steps * 1e-3)
-    rows_per_step = float(rows_np.sum() - B)                  # rows verified (the initial call is not a window)
-    windows_chains = float(calls_np.sum() - B)
+    if getattr(w, "drafter_mode", 0) == 1:
+        # drafter evaluated at Y_n: no initial call, two sequential calls per window (one for a last window of one row)
+        rows_per_step = float(rows_np.sum())
+        windows_chains = float(np.ceil(calls_np / 2.0).sum())
+    else:
+        rows_per_step = float(rows_np.sum() - B)              # rows verified (the initial call is not a window)
+        windows_chains = float(calls_np.sum() - B)
     kinds = {k: v for k, v in prof.items() if v[1] > 0}
     dom = max(kinds, key=lambda k: kinds[k][0]) if kinds else "fused"
     dom_ms, dom_n = kinds.get(dom, (ms_total, steps))
