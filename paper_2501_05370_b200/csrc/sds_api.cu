@@ -733,6 +733,12 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
     SDS_LAUNCH(c, SDS_PROF_FUSED, launch_fused_small(A, gmm_args(c, c->tgt), c->stream));
     c->ub = 0;
     c->state = kReady;
+  } else if (c->whole_chain && !c->Q && c->mode == SDS_FROZEN_EXACT && c->tgt.den.kind == SDS_DEN_PHI4 &&
+             fused_phi4_ok(c->d, c->L)) {
+    SDS_CU(c, cudaMemsetAsync(A.ctl, 0, kCtlWords * 4, c->stream));
+    SDS_LAUNCH(c, SDS_PROF_FUSED, launch_fused_phi4(A, c->tgt.den.grid_side, c->tgt.den.coupling, c->tgt.den.periodic, c->stream));
+    c->ub = 0;
+    c->state = kReady;
   } else {
     rc = sds_reset(c);
     if (rc != SDS_OK) return rc;

@@ -181,4 +181,27 @@ __device__ __forceinline__ float reflect_elem(float wp, float dq, float Z, float
   return fmaf(s, fmaf(-coef, D, Z), fmaf(a, wp, c * dq));
 }
 
+// ---------------------------------------------------------------------------------------
+// phi^4 lattice energy gradient at site i of a side x side grid (Appendix K): beta times the sum
+// of the differences to the neighbours (order up, down, left, right; free or periodic boundaries)
+// plus the derivative 4 x (x^2 - 1) of the site potential
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ float phi4_site(const float* x, int i, int side, float beta, int periodic) {
+  const int r = i / side, c = i - r * side;
+  const float xi = x[i];
+  float acc = 0.f;
+  if (periodic) {
+    acc += xi - x[((r + side - 1) % side) * side + c];
+    acc += xi - x[((r + 1) % side) * side + c];
+    acc += xi - x[r * side + (c + side - 1) % side];
+    acc += xi - x[r * side + (c + 1) % side];
+  } else {
+    if (r > 0) acc += xi - x[i - side];
+    if (r < side - 1) acc += xi - x[i + side];
+    if (c > 0) acc += xi - x[i - 1];
+    if (c < side - 1) acc += xi - x[i + 1];
+  }
+  return fmaf(beta, acc, 4.0f * xi * fmaf(xi, xi, -1.0f));
+}
+
 }  // namespace sds

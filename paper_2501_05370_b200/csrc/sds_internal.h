@@ -96,4 +96,8 @@ cudaError_t launch_phi4_grad(const float* X, const int* nrows_dev, int rows_ub, 
 bool fused_small_supported(int d, int ncomp, int L);
 cudaError_t launch_fused_small(const WinArgs& A, const GmmArgs& G, cudaStream_t st);
 
+// whole-chain kernel for the lattice model with the drafter evaluated at Y_n (sds_fused_phi4.cu)
+bool fused_phi4_ok(int d, int L);
+cudaError_t launch_fused_phi4(const WinArgs& A, int side, float beta, int periodic, cudaStream_t st);
+
 }  // namespace sds

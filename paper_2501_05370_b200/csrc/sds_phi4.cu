@@ -17,22 +17,8 @@ __global__ void __launch_bounds__(256) k_phi4_grad(const float* __restrict__ X, 
   const size_t total = (size_t)nrows * d;
   for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
     const size_t row = e / d;
-    const int i = (int)(e - row * d), r = i / side, c = i - r * side;
-    const float* x = X + row * d;
-    const float xi = x[i];
-    float acc = 0.f;
-    if (periodic) {
-      acc += xi - x[((r + side - 1) % side) * side + c];
-      acc += xi - x[((r + 1) % side) * side + c];
-      acc += xi - x[r * side + (c + side - 1) % side];
-      acc += xi - x[r * side + (c + 1) % side];
-    } else {
-      if (r > 0) acc += xi - x[i - side];
-      if (r < side - 1) acc += xi - x[i + side];
-      if (c > 0) acc += xi - x[i - 1];
-      if (c < side - 1) acc += xi - x[i + 1];
-    }
-    out[e] = fmaf(beta, acc, 4.0f * xi * fmaf(xi, xi, -1.0f));
+    const int i = (int)(e - row * d);
+    out[e] = phi4_site(X + row * d, i, side, beta, periodic);
   }
 }
 

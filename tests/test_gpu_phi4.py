@@ -66,3 +66,19 @@ def test_phi4_full_run_reproduces_the_papers_nfe():
     print(f"windows per step {windows_per_step:.5f} (paper {g['nfe_per_step']}), "
           f"final energy {energies.mean():.2f} +- {energies.std():.2f}")
     s.close()
+
+
+@pytest.mark.parametrize("side,L,periodic", [(8, 20, False), (6, 7, True), (5, 4, False)])
+def test_phi4_whole_chain_kernel_equals_window_kernels(side, L, periodic):
+    """The one-launch path and the window-by-window path give the same bits (states and counters)."""
+    w = wl.WORKLOADS["phi4"].scaled(B=40, K=257, L=L, d=side * side,
+                                    phi4=dict(side=side, beta=100.0, periodic=periodic))
+    res = {}
+    for fused in (1, 0):
+        s = sds.sampler_for(w, seed=9)
+        s.set_option(s.OPT_WHOLE_CHAIN_KERNEL, fused)
+        res[fused] = [x.cpu().numpy() for x in s.sample_all()] + [s.launch_count()]
+        s.close()
+    for x, y in zip(res[1][:3], res[0][:3]):
+        assert np.array_equal(x, y)
+    assert res[1][3] < 10 < res[0][3]                       # one launch against hundreds
