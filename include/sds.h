@@ -231,6 +231,11 @@ int sds_sample_all(sds_ctx* ctx, float* out_dev, int32_t* nfe_calls_dev, int32_t
  * diagnostic arrays (SDS_GET_S1, _S2, _ELL, _LOGU, bits of _ACCMASK) hold zeros for the skipped
  * positions. 0 evaluates every position of every window. */
 #define SDS_OPT_VERIFY_EARLY_EXIT 4
+/* SDS_OPT_FUSE_ADVANCE (default 1): inside sds_sample_all, for d % 4 == 0 with d <= 256 or
+ * 2048 < d <= 16384, the verify kernel also performs the advance step of its chain, and the CTA that finishes
+ * last rebuilds the active list, so a window is draft, denoiser, verify: one launch less. Same
+ * results. The step-wise calls sds_verify_window / sds_advance are not affected. */
+#define SDS_OPT_FUSE_ADVANCE 5
 int sds_set_option(sds_ctx* ctx, int32_t option, int64_t value);
 
 /* Temperature of the accept test (Appendix D, temperature rejection): a draft is accepted iff

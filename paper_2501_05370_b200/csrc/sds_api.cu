@@ -95,6 +95,8 @@ struct sds_ctx {
   bool tensor_split = true;         // float mixtures of tensor-core shape use the 3-way bf16 split
   bool gemm_pair = true;            // tensor-core GEMMs with N % 256 == 0 run on CTA pairs
   bool early_exit = true;           // verify stops reading a window after the block with the first rejection
+  bool fuse_advance = true;         // sds_sample_all lets the verify kernel do the advance step where it can
+  bool fusing = false;              // set around the verify call of the sds_sample_all loop
   // optional per-kernel timing: event pairs recorded around each launch, summed on read
   bool prof_on = false;
   std::vector<cudaEvent_t> prof_ev[SDS_PROF_KINDS];
@@ -248,6 +250,7 @@ WinArgs win_args(sds_ctx* c) {
   A.mode = c->mode;
   A.inv_tau = 1.0 / c->tau;
   A.early_exit = c->early_exit ? 1 : 0;
+  A.fuse_advance = c->fusing ? 1 : 0;
   A.seed = c->seed; A.chain_off = (uint64_t)c->chain_off;
   A.a = at<float>(c, c->lay.a); A.c = at<float>(c, c->lay.c); A.sigma = at<float>(c, c->lay.sigma);
   A.Y = at<float>(c, c->lay.Y); A.Dc = at<float>(c, c->lay.Dc); A.T = at<float>(c, c->lay.T);
@@ -747,8 +750,14 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
     // does nothing on the device.
     for (int w = 0;; ++w) {
       if ((rc = sds_draft(c)) != SDS_OK) return rc;
-      if ((rc = sds_verify_window(c)) != SDS_OK) return rc;
-      if ((rc = sds_advance(c, nullptr)) != SDS_OK) return rc;
+      // where the register-resident verify kernel runs, it also advances its chains and compacts
+      c->fusing = c->fuse_advance && verify_can_advance(A);
+      rc = sds_verify_window(c);
+      const bool fused_adv = c->fusing;
+      c->fusing = false;
+      if (rc != SDS_OK) return rc;
+      if (fused_adv) c->state = kReady;
+      else if ((rc = sds_advance(c, nullptr)) != SDS_OK) return rc;
       SDS_CU(c, cudaMemcpyAsync(c->h_pin + 8 + (w & 1) * kCtlWords, A.ctl, kCtlWords * 4, cudaMemcpyDeviceToHost,
                                 c->stream));
       SDS_CU(c, cudaEventRecord(c->ev[w & 1], c->stream));
@@ -884,6 +893,7 @@ int sds_set_option(sds_ctx* c, int32_t option, int64_t value) {
     case SDS_OPT_TENSOR_SPLIT: c->tensor_split = value != 0; return SDS_OK;
     case SDS_OPT_GEMM_PAIR: c->gemm_pair = value != 0; return SDS_OK;
     case SDS_OPT_VERIFY_EARLY_EXIT: c->early_exit = value != 0; return SDS_OK;
+    case SDS_OPT_FUSE_ADVANCE: c->fuse_advance = value != 0; return SDS_OK;
     default: return SDS_EINVAL;
   }
 }

@@ -26,9 +26,11 @@ __device__ __forceinline__ int window_len(const WinArgs& A, int nb) { return min
 // ---------------------------------------------------------------------------------------
 __device__ void compact_scan(const WinArgs& A) {
   // every thread owns a contiguous range of chains: count, one block-wide exclusive scan, write
-  __shared__ int s_cnt[kBlock / 32], s_row[kBlock / 32];
+  // (any CTA size up to 1024 threads; the result does not depend on it)
+  __shared__ int s_cnt[32], s_row[32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int per = (A.B + kBlock - 1) / kBlock;
+  const int nthr = blockDim.x, nwarp = nthr >> 5;
+  const int per = (A.B + nthr - 1) / nthr;
   const int b0 = min(A.B, tid * per), b1 = min(A.B, b0 + per);
   int cnt = 0, rows = 0;
   for (int b = b0; b < b1; ++b) {
@@ -44,7 +46,7 @@ __device__ void compact_scan(const WinArgs& A) {
   if (lane == 31) { s_cnt[warp] = c; s_row[warp] = r; }
   __syncthreads();
   int pos = c - cnt, row = r - rows, tot_c = 0, tot_r = 0;
-  for (int w = 0; w < kBlock / 32; ++w) {
+  for (int w = 0; w < nwarp; ++w) {
     if (w < warp) { pos += s_cnt[w]; row += s_row[w]; }
     tot_c += s_cnt[w];
     tot_r += s_row[w];
@@ -62,6 +64,38 @@ __device__ void compact_scan(const WinArgs& A) {
     A.rowoff[tot_c] = tot_r;
     A.ctl[kCtlNActive] = tot_c;
     A.ctl[kCtlNRows] = tot_r;
+  }
+}
+
+// counters of one finished window of chain b (Lt positions)
+__device__ __forceinline__ void count_window(const WinArgs& A, int b, int Lt) {
+  if (A.mode == 3) {   // Picard: calls-1 refinements on Lt-1 points, the last draft call on Lt, verify on Lt-1
+    A.nfe_calls[b] += (Lt > 1) ? A.picard_calls + 1 : 1;
+    A.nfe_rows[b] += (A.picard_calls - 1) * (Lt - 1) + Lt + (Lt - 1);
+  } else {
+    // sequential target calls of this window: the batched pass, plus (main-text drafter) the
+    // call at Y_n, which is row 1 of the batch (a window of one row is a single call)
+    A.nfe_calls[b] += (A.mode == 1 && Lt > 1) ? 2 : 1;
+    A.nfe_rows[b] += Lt;
+  }
+}
+
+// end of a window, CTA-wide: the CTA that arrives last rebuilds the active list (no CTA waits on another)
+__device__ __forceinline__ void window_tail(const WinArgs& A, int n_active_before) {
+  __shared__ int s_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int prev = atomicAdd(A.ctl + kCtlDone, 1);
+    s_last = (prev == (int)gridDim.x - 1);
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  compact_scan(A);
+  if (threadIdx.x == 0) {
+    A.ctl[kCtlDone] = 0;
+    if (n_active_before > 0) A.ctl[kCtlWindows] += 1;
   }
 }
 
@@ -627,16 +661,13 @@ __global__ void __launch_bounds__(kBlock) k_verify(WinArgs A) {
 // independent 128-bit loads in flight per thread. Same per-thread element order and reduction
 // tree as k_verify, hence the same bits.
 template <int TPC, int EPT>
-__global__ void __launch_bounds__(TPC > kBlock ? TPC : kBlock) k_verify_reg(WinArgs A) {
-  constexpr int kThreadsPerCta = TPC > kBlock ? TPC : kBlock;
-  constexpr int kChains = kThreadsPerCta / TPC;
+__device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t) {
   constexpr int kWarps = TPC / 32;
   __shared__ double s_red[(TPC > 32) ? 2 * kMaxL * kWarps : 1];
   __shared__ int s_jstar;
   __shared__ float s_coef;
-  const int s = blockIdx.x * kChains + threadIdx.x / TPC, t = threadIdx.x % TPC;
   const int lane = threadIdx.x & 31, warp = t >> 5;
-  if (s >= A.ctl[kCtlNActive]) return;
+  const bool fa = A.fuse_advance != 0;                 // also do this chain's part of the advance step
   const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
   const int Lt = window_len(A, nb);
   const uint64_t bg = A.chain_off + (uint64_t)b;
@@ -767,7 +798,28 @@ __global__ void __launch_bounds__(TPC > kBlock ? TPC : kBlock) k_verify_reg(WinA
     jstar = s_jstar;
     coef = s_coef;
   }
-  if (jstar < 1 || jstar > Lt) return;
+  if (jstar < 1 || jstar > Lt) {
+    if (fa) {
+      if (jstar >= 1) {                                  // every draft accepted: the window's last state and output carry on
+#pragma unroll
+        for (int e = 0; e < EPT; ++e) {
+          const int i = (t + e * TPC) * 4;
+          if (i < A.d) {
+            st4(A.Y + cb + i, ld4(A.T + cb + i));
+            st4(A.Dc + cb + i, ld4(A.Dq + (size_t)(r0 + Lt - 1) * A.d + i));
+          }
+        }
+        if (t == 0) {
+          A.n[b] = nb + Lt;
+          count_window(A, b, Lt);
+        }
+      } else if (t == 0) {                               // non-finite log ratio: stop this chain
+        A.n[b] = A.K;
+        atomicAdd(A.ctl + kCtlFrozen, 1);
+      }
+    }
+    return;
+  }
   const int k = nb + jstar - 1;
   const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
   const float inv_s = 1.0f / sk, cs = ck * inv_s;
@@ -787,8 +839,26 @@ __global__ void __launch_bounds__(TPC > kBlock ? TPC : kBlock) k_verify_reg(WinA
       delta_z(p.z, w.z, q.z, c4.z, ak, ck, cs, inv_s, D, Z); o.z = reflect_elem(p.z, q.z, Z, D, ak, ck, sk, coef);
       delta_z(p.w, w.w, q.w, c4.w, ak, ck, cs, inv_s, D, Z); o.w = reflect_elem(p.w, q.w, Z, D, ak, ck, sk, coef);
       st4(wj + i, o);
+      if (fa) {                                          // the reflected state is the next state; its target row carries on
+        st4(A.Y + cb + i, o);
+        st4(A.Dc + cb + i, q);
+      }
     }
   }
+  if (fa && t == 0) {
+    A.n[b] = nb + jstar;
+    count_window(A, b, Lt);
+  }
+}
+
+template <int TPC, int EPT>
+__global__ void __launch_bounds__(TPC > kBlock ? TPC : kBlock) k_verify_reg(WinArgs A) {
+  constexpr int kThreadsPerCta = TPC > kBlock ? TPC : kBlock;
+  constexpr int kChains = kThreadsPerCta / TPC;
+  const int s = blockIdx.x * kChains + threadIdx.x / TPC, t = threadIdx.x % TPC;
+  const int n_active = A.ctl[kCtlNActive];
+  if (s < n_active) verify_reg_chain<TPC, EPT>(A, s, t);
+  if (A.fuse_advance) window_tail(A, n_active);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -798,7 +868,6 @@ __global__ void __launch_bounds__(TPC > kBlock ? TPC : kBlock) k_verify_reg(WinA
 template <int TPC, int VEC>
 __global__ void __launch_bounds__(kBlock) k_advance(WinArgs A) {
   using G = Group<TPC>;
-  __shared__ int s_last;
   const int s = G::slot(), t = G::lane();
   const int n_active = A.ctl[kCtlNActive];
   if (s < n_active) {
@@ -833,36 +902,14 @@ __global__ void __launch_bounds__(kBlock) k_advance(WinArgs A) {
       }
       if (t == 0) {
         A.n[b] = nb + adv;
-        // sequential target calls of this window: the batched pass, plus (main-text drafter) the
-        // call at Y_n, which is row 1 of the batch (a window of one row is a single call)
-        if (A.mode == 3) {   // Picard: calls-1 refinements on Lt-1 points, the last draft call on Lt, verify on Lt-1
-          A.nfe_calls[b] += (Lt > 1) ? A.picard_calls + 1 : 1;
-          A.nfe_rows[b] += (A.picard_calls - 1) * (Lt - 1) + Lt + (Lt - 1);
-        } else {
-          A.nfe_calls[b] += (A.mode == 1 && Lt > 1) ? 2 : 1;
-          A.nfe_rows[b] += Lt;
-        }
+        count_window(A, b, Lt);
       }
     } else if (t == 0) {                              // non-finite log ratio: stop this chain
       A.n[b] = A.K;
       atomicAdd(A.ctl + kCtlFrozen, 1);
     }
   }
-  // the last CTA to arrive rebuilds the list (no CTA waits on another)
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const int prev = atomicAdd(A.ctl + kCtlDone, 1);
-    s_last = (prev == (int)gridDim.x - 1);
-  }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  compact_scan(A);
-  if (threadIdx.x == 0) {
-    A.ctl[kCtlDone] = 0;
-    if (n_active > 0) A.ctl[kCtlWindows] += 1;
-  }
+  window_tail(A, n_active);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -957,6 +1004,13 @@ cudaError_t launch_picard_draft(const WinArgs& A, int ub, cudaStream_t st) {
   SDS_DISPATCH(k_picard_draft, A, ub, st);
   return cudaGetLastError();
 }
+// whether launch_verify takes the register-resident kernel, the one that can also do the advance step
+// (and where that pays: for 256 < d <= 2048 the separate warp-per-chain advance kernel is faster than
+// one more fence and counter update in each of the many small verify CTAs)
+bool verify_can_advance(const WinArgs& A) {
+  return !A.Q && !A.mean_rows && vec4_ok(A.d) && A.d <= 16384 && (A.d <= 256 || A.d > 2048);
+}
+
 cudaError_t launch_verify(const WinArgs& A, int ub, cudaStream_t st) {
   const int chains = ub > 0 ? ub : 1;
   if (A.mean_rows && !A.Q) {                            // draft means per row: the generic kernel handles them

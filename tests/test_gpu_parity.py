@@ -727,3 +727,27 @@ def test_early_exit_run_matches_oracle():
         bad += not (r["nfe_calls"] == calls[b] and r["nfe_rows"] == rows[b] and rel_l2(out[b], r["Y"]) <= 1e-4)
     assert bad <= 1
     s.close()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("d,L,B,mode", [(64, 8, 70, 0), (1024, 12, 40, 0), (3072, 8, 24, 1), (4096, 16, 12, 0), (16384, 5, 6, 0)])
+def test_sample_all_with_fused_advance_equals_the_stepwise_calls(d, L, B, mode):
+    """sds_sample_all (verify kernel advancing its chains, early exit on) against an explicit
+    draft / verify / advance loop, and against the same run with the advance kernel: same bits."""
+    w = wl.WORKLOADS["cfg2"].scaled(B=B, d=d, K=3 * L + 7, L=L)
+    gp = w.gmm_params(d=d, ncomp=8)
+    s = sds.sampler_for(w, gmm=gp, seed=71, drafter_mode=mode)
+    s.set_option(s.OPT_WHOLE_CHAIN_KERNEL, 0)
+    got = [x.cpu().numpy() for x in s.sample_all()]
+    windows_fused = int(s.get(sb.GET_CTL)[2])
+    s.set_option(s.OPT_FUSE_ADVANCE, 0)
+    ref = [x.cpu().numpy() for x in s.sample_all()]
+    assert all(np.array_equal(x, y) for x, y in zip(got, ref))
+    assert windows_fused == int(s.get(sb.GET_CTL)[2])
+    s.reset()
+    na = B
+    while na > 0:
+        s.draft(); s.verify_window(); na = s.advance()
+    assert np.array_equal(s.get(sb.GET_Y), got[0])
+    assert np.array_equal(s.get(sb.GET_NFE_CALLS), got[1]) and np.array_equal(s.get(sb.GET_NFE_ROWS), got[2])
+    s.close()
