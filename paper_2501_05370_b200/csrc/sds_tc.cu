@@ -548,8 +548,9 @@ __global__ void k_split3(const float* __restrict__ x, size_t n, size_t plane, in
 }
 
 // Row softmax for the split-precision mixture. The tensor-core logits are float sums of large
-// terms; components within 30 of the row maximum get their logit again in double (warp-wide dot
-// product, fixed combination order), all others weigh less than e^-29. Writes the normalised
+// terms; when more than one component lies within 30 of the row maximum, those components get
+// their logit again in double (warp-wide dot product, fixed combination order); all others weigh
+// less than e^-29. Writes the normalised
 // responsibilities as three bf16 planes. One warp per row.
 template <int NQ>   // ncomp = 128 * NQ: a lane holds NQ groups of four consecutive components in registers
 __global__ void __launch_bounds__(256)
@@ -575,12 +576,20 @@ __global__ void __launch_bounds__(256)
     const int k = rowk[row];
     const double tA = __ldg(tcond + 4 * k + 0), tB = __ldg(tcond + 4 * k + 1);
     const float* x = X + (size_t)row * d;
+    // A row whose maximum stands alone (nothing else within 30) is one-hot to within e^-30 whatever
+    // the exact value of that logit: no refinement, and the row of X is not read at all.
+    int near = 0;
+#pragma unroll
+    for (int q = 0; q < NQ; ++q)
+#pragma unroll
+      for (int u = 0; u < 4; ++u) near += __popc(__ballot_sync(0xffffffffu, v[q][u] >= mx - 30.0f));
+    const bool refine = near > 1;
 #pragma unroll
     for (int q = 0; q < NQ; ++q) {
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         float val = v[q][u] - mx;
-        unsigned sel = __ballot_sync(0xffffffffu, v[q][u] >= mx - 30.0f);
+        unsigned sel = refine ? __ballot_sync(0xffffffffu, v[q][u] >= mx - 30.0f) : 0u;
         while (sel) {                                      // warp-uniform loop over the selected components
           const int l = __ffs(sel) - 1;
           sel &= sel - 1;
