@@ -14,7 +14,7 @@ struct WinArgs {
                          // window; 2: independent draft model evaluated at every drafted state
   double inv_tau;        // 1 / temperature of the accept test (1 = the exact method)
   int fuse_advance;      // the verify kernel also advances its chain and the last CTA compacts (no advance launch)
-  int early_exit;        // verify stops reading a chain's window after the block of four positions
+  int early_exit;        // verify stops reading a chain's window after the block of two (d >= 2048) or four positions
                          // that holds its first rejection (large-d kernels only)
   uint64_t seed;
   uint64_t chain_off;

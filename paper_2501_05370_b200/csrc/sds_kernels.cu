@@ -685,7 +685,7 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t)
   // of a block are decided before the next block is read, and nothing after the block that holds
   // the first rejection is read at all: those positions report zeros.
   const bool early = (TPC > 32) && A.early_exit != 0;
-  const int blk = early ? 4 : Lt;
+  const int blk = early ? (A.d >= 2048 ? 2 : 4) : Lt;   // small rows: fewer, larger blocks (two barriers per block)
   int jstar = Lt + 1;
   float coef = 0.f;
   uint32_t amask = 0u;

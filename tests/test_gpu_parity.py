@@ -672,7 +672,7 @@ def test_projection_onto_the_whole_space_is_the_exact_method():
 
 
 # ----------------------------------------------------------------------------------------
-# verify with early exit (blocks of four positions; nothing after the first rejection is read)
+# verify with early exit (blocks of two or four positions; nothing after the first rejection is read)
 # ----------------------------------------------------------------------------------------
 
 
@@ -697,13 +697,14 @@ def test_verify_early_exit_only_skips_diagnostics(d, L, B):
         res[early] = (wins, full)
         s.close()
     skipped = 0
+    blk = 2 if d >= 2048 else 4
     for a, b in zip(res[1][0], res[0][0]):
         assert np.array_equal(a["n"], b["n"]) and np.array_equal(a["js"], b["js"])
         assert np.array_equal(a["X"], b["X"]) and np.array_equal(a["T"], b["T"])      # same reflected states
         for c in range(B):
             Lt = min(L, w.K - int(a["n"][c]))
             js = int(a["js"][c])
-            n_eval = Lt if js > Lt else min(Lt, 4 * ((js + 3) // 4))
+            n_eval = Lt if js > Lt else min(Lt, blk * ((js + blk - 1) // blk))
             keep = (1 << n_eval) - 1
             assert int(a["am"][c]) == int(b["am"][c]) & keep
             for key in ("S1", "S2", "ell", "lu"):
