@@ -44,6 +44,9 @@ __global__ void __maxnreg__(72) k_fused_small(WinArgs A, GmmArgs P) {
   const bool pack2 = VEC4 ? (d <= 64) : (d <= 16);
   const int PW = pack2 ? 16 : 32;
   const int vh = lane / PW, vt = lane % PW;
+  // noise generation walks (position, block) pairs without a division per element
+  const int nz_n = VEC4 ? d / 4 : d;
+  const int nz_j0 = lane / nz_n, nz_q0 = lane % nz_n, nz_dj = 32 / nz_n, nz_dq = 32 % nz_n;
 
   for (int b = blockIdx.x * nwarps + warp; b < A.B; b += gridDim.x * nwarps) {
     const uint64_t bg = A.chain_off + (uint64_t)b;
@@ -62,15 +65,19 @@ __global__ void __maxnreg__(72) k_fused_small(WinArgs A, GmmArgs P) {
       const int Lt = min(L, K - n);
       // draft noise for all positions at once, then the sequential recurrence per element
       if (VEC4) {
-        const int nq = d / 4;
-        for (int e = lane; e < Lt * nq; e += 32) {
-          const int j = e / nq, q = e - j * nq;
+        // element e = lane + 32 it is block q of position j; (j, q) advance by (32 / nq, 32 % nq) with carry
+        int j = nz_j0, q = nz_q0;
+        for (int e = lane; e < Lt * nz_n; e += 32) {
           st4(sW + (j + 1) * ldx + 4 * q, normal4(A.seed, kStreamDraft, bg, (uint32_t)(n + j), (uint32_t)q));
+          j += nz_dj; q += nz_dq;
+          if (q >= nz_n) { q -= nz_n; j += 1; }
         }
       } else {
-        for (int e = lane; e < Lt * d; e += 32) {
-          const int j = e / d, i = e - j * d;
+        int j = nz_j0, i = nz_q0;
+        for (int e = lane; e < Lt * nz_n; e += 32) {
           sW[(j + 1) * ldx + i] = normal1(A.seed, kStreamDraft, bg, (uint32_t)(n + j), (uint32_t)i);
+          j += nz_dj; i += nz_dq;
+          if (i >= nz_n) { i -= nz_n; j += 1; }
         }
       }
       __syncwarp();
