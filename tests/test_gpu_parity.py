@@ -187,6 +187,8 @@ SHAPES = [
     ("cfg5", 20, 1024, 6, 40, 12, 4),
     ("cfg5", 7, 516, 32, 64, 5, 3),
     ("cfg2", 5, 1030, 3, 11, 6, 5),
+    ("cfg2", 4, 8, 8, 3, 4, 1),          # the whole chain is shorter than one window
+    ("cfg5", 3, 2052, 32, 5, 3, 1),      # same, one CTA per chain
 ]
 
 
@@ -306,7 +308,7 @@ def test_stepwise_loop_equals_sample_all_and_is_deterministic():
 
 FUSED_SHAPES = [(64, 2, 4, 100, 4), (300, 64, 8, 200, 16), (65, 33, 5, 23, 7), (3, 5, 2, 9, 3), (1, 1, 1, 6, 2),
                 (9, 3, 32, 70, 4), (20, 128, 6, 40, 20), (10, 256, 4, 30, 32), (40, 16, 8, 50, 16), (40, 20, 8, 50, 17),
-                (33, 68, 3, 31, 9)]
+                (33, 68, 3, 31, 9), (4, 8, 8, 3, 4)]
 
 
 @pytest.mark.parametrize("B,d,L,K,ncomp", FUSED_SHAPES)
