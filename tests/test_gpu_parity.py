@@ -754,3 +754,50 @@ def test_sample_all_with_fused_advance_equals_the_stepwise_calls(d, L, B, mode):
     assert np.array_equal(s.get(sb.GET_Y), got[0])
     assert np.array_equal(s.get(sb.GET_NFE_CALLS), got[1]) and np.array_equal(s.get(sb.GET_NFE_ROWS), got[2])
     s.close()
+
+
+# ----------------------------------------------------------------------------------------
+# laws on the GPU at scale
+# ----------------------------------------------------------------------------------------
+
+
+@pytest.mark.gpu
+def test_gpu_normals_follow_the_standard_normal_law():
+    """The library's normals use hardware approximations of log, sqrt, sin and cos: their law is
+    checked directly (Kolmogorov-Smirnov, moments, independence of neighbours)."""
+    from scipy import stats
+    z = sb.rng_normals(20250101, o.STREAM_DRAFT, 0, 2048, 3, 1024).cpu().numpy().astype(np.float64).ravel()
+    n = z.size
+    assert stats.kstest(z[:400_000], stats.norm.cdf).pvalue > 1e-3
+    assert abs(z.mean()) < 5 / math.sqrt(n) and abs(z.var() - 1) < 5 * math.sqrt(2 / n)
+    assert abs(np.mean(z ** 4) - 3) < 5 * math.sqrt(96 / n)
+    pairs = z.reshape(-1, 2)                               # the two outputs of one Box-Muller pair
+    assert abs(np.mean(pairs[:, 0] * pairs[:, 1])) < 5 / math.sqrt(n / 2)
+    assert abs(np.mean(z[:-1] * z[1:])) < 5 / math.sqrt(n)
+
+
+@pytest.mark.gpu
+def test_speculative_and_plain_chains_agree_in_law_on_the_gpu():
+    """cfg2 at full batch: window 8 with the carried-output drafter against the plain sequential
+    chain (window 1 with the drafter evaluated at Y_n, which accepts every step) under another seed."""
+    w = wl.WORKLOADS["cfg2"]
+    gp = w.gmm_params()
+    s = sds.sampler_for(w, gmm=gp, seed=101)
+    S = s.sample_all()[0].cpu().numpy().astype(np.float64)
+    s.close()
+    wp = w.scaled(L=1)
+    p = sds.sampler_for(wp, gmm=gp, seed=202, drafter_mode=sb.SDS_FROZEN_EXACT)
+    outp, calls, _ = p.sample_all()
+    P = outp.cpu().numpy().astype(np.float64)
+    assert np.all(calls.cpu().numpy() == w.K)              # one target call per step: the plain chain
+    p.close()
+    B = w.B
+    se = np.sqrt(S.var(axis=0) / B + P.var(axis=0) / B)
+    zmean = (S.mean(axis=0) - P.mean(axis=0)) / se
+    assert np.max(np.abs(zmean)) < 4.5 and abs(zmean.mean()) < 4 / math.sqrt(w.d)
+    rv = S.var(axis=0) / P.var(axis=0)
+    assert np.max(np.abs(rv - 1)) < 6 * math.sqrt(2 / B) * 2
+    # a random projection, compared as distributions
+    u = np.random.default_rng(0).standard_normal(w.d); u /= np.linalg.norm(u)
+    from scipy import stats
+    assert stats.ks_2samp(S @ u, P @ u).pvalue > 1e-3
