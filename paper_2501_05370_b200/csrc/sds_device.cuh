@@ -181,6 +181,36 @@ __device__ __forceinline__ float reflect_elem(float wp, float dq, float Z, float
   return fmaf(s, fmaf(-coef, D, Z), fmaf(a, wp, c * dq));
 }
 
+// Sequential draft recurrence of one chain held in shared memory (whole-chain kernels): rows
+// 1..Lt of sW hold the noise and are replaced by the drafted states; a lane keeps U of its elements
+// (32 apart) in registers across the positions.
+template <int U, class Args>
+__device__ __forceinline__ void draft_recurrence(const Args& A, float* sW, const float* sDc, int ldx, int d, int n, int Lt,
+                                                 int lane) {
+  for (int i0 = 0; i0 < d; i0 += 32 * U) {
+    float y[U], dc[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int i = i0 + lane + 32 * u;
+      y[u] = (i < d) ? sW[i] : 0.f;
+      dc[u] = (i < d) ? sDc[i] : 0.f;
+    }
+    for (int j = 0; j < Lt; ++j) {
+      const int k = n + j;
+      const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
+      float* row = sW + (j + 1) * ldx;
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int i = i0 + lane + 32 * u;
+        if (i < d) {
+          y[u] = draft_step(y[u], dc[u], row[i], ak, ck, sk);
+          row[i] = y[u];
+        }
+      }
+    }
+  }
+}
+
 // ---------------------------------------------------------------------------------------
 // phi^4 lattice energy gradient at site i of a side x side grid (Appendix K): beta times the sum
 // of the differences to the neighbours (order up, down, left, right; free or periodic boundaries)

@@ -70,28 +70,8 @@ __global__ void __maxnreg__(72) k_fused_phi4(WinArgs A, int side, float beta, in
         }
       }
       __syncwarp();
-      for (int i0 = 0; i0 < d; i0 += 128) {                     // up to four elements per lane in registers
-        float y[4], dc[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int i = i0 + lane + 32 * u;
-          y[u] = (i < d) ? sW[i] : 0.f;
-          dc[u] = (i < d) ? sDc[i] : 0.f;
-        }
-        for (int j = 0; j < Lt; ++j) {
-          const int k = n + j;
-          const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
-          float* row = sW + (j + 1) * ldx;
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const int i = i0 + lane + 32 * u;
-            if (i < d) {
-              y[u] = draft_step(y[u], dc[u], row[i], ak, ck, sk);
-              row[i] = y[u];
-            }
-          }
-        }
-      }
+      if (d <= 64) draft_recurrence<2>(A, sW, sDc, ldx, d, n, Lt, lane);   // elements per lane held in registers
+      else draft_recurrence<4>(A, sW, sDc, ldx, d, n, Lt, lane);
       __syncwarp();
       // target rows W_1 .. W_{Lt-1} (row 0 is the frozen output)
       for (int e = lane; e < (Lt - 1) * d; e += 32) {
