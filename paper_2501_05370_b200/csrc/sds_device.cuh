@@ -64,17 +64,33 @@ __device__ __forceinline__ float sqrt_approx(float x) {
   asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ float lg2_approx(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float sin_approx(float x) {
+  float y;
+  asm("sin.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float cos_approx(float x) {
+  float y;
+  asm("cos.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ float2 box_muller(uint32_t xe, uint32_t xo) {
   const float u1 = (float)((xe >> 8) + 1u) * 0x1p-24f;
-  const float u2 = (float)(xo >> 8) * 0x1p-24f;
+  // angle 2 pi u2 - pi with u2 = (x_odd >> 8) 2^-24: (m - 2^23) is exact in float and 2 pi 2^-24 is the
+  // float 2 pi scaled by a power of two, so this single rounding equals that of (u2 - 1/2) * 2 pi
+  const float th = (float)((int)(xo >> 8) - (1 << 23)) * (6.28318530717959f * 0x1p-24f);
   // -2 ln u1; next to 1 the approximation's absolute error would dominate, so the series of
   // -2 ln(1 - t), t = 1 - u1 (exact), takes over below t = 2^-7 (truncation t^4/5 relative)
   const float t = 1.0f - u1;
-  float r2 = -1.38629436111989f * __log2f(u1);
+  float r2 = -1.38629436111989f * lg2_approx(u1);
   if (t < 0x1p-7f) r2 = 2.0f * t * fmaf(t, fmaf(t, fmaf(t, 0.25f, 0.333333343f), 0.5f), 1.0f);
   const float r = sqrt_approx(r2);
-  const float th = (u2 - 0.5f) * 6.28318530717959f;                            // 2 pi u2 - pi
-  return make_float2(-r * __cosf(th), -r * __sinf(th));
+  return make_float2(-r * cos_approx(th), -r * sin_approx(th));
 }
 
 // four normals of block q (elements 4q .. 4q+3)
