@@ -100,6 +100,26 @@ def oracle_time(w, budget_s: float, min_chains: int = 1, first_chain: int = 0):
     return steps, el, what
 
 
+def oracle_plain_time(w, budget_s: float):
+    """The oracle's plain (non-speculative) chain, same sampling rule as oracle_time: the context
+    for the saving in sequential target calls. Returns (chain_steps, seconds)."""
+    o, den, a, c, sig = oracle_closure(w)
+    t0 = time.perf_counter()
+    n, steps, Kp = 0, 0, min(w.K, 2 * w.L)
+    while True:
+        t1 = time.perf_counter()
+        o.plain_chain(den, a[:Kp], c[:Kp], sig[:Kp], w.sample_seed, n, w.d)
+        dt = time.perf_counter() - t1
+        n += 1
+        steps += Kp
+        el = time.perf_counter() - t0
+        if el >= budget_s or n >= w.B:
+            break
+        if Kp < w.K and dt < budget_s / 8:
+            Kp = min(w.K, Kp * 4)
+    return steps, el
+
+
 def run_reference(args, w):
     """--impl reference: the oracle on the host cores, same metric, bounded sample per step."""
     rank = int(os.environ.get("RANK", "0"))
@@ -376,6 +396,8 @@ def run_gpu(args, w):
 
     osteps, sec, what = oracle_time(w, args.cpu_seconds)
     cpu = {"value": osteps / sec, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what}
+    psteps, psec = oracle_plain_time(w, max(1.0, args.cpu_seconds / 5))
+    cpu["plain_chain_value"] = psteps / psec          # the oracle's plain sequential chain, same unit, for context
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": args.warmup,
