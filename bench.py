@@ -257,6 +257,39 @@ def algorithmic(kind: str, w, rows_per_step: float, windows_chains: float, launc
     return "hbm", 0.0
 
 
+def acceptance_by_step(sds, w, dev, chains: int = 64, bins: int = 10):
+    """Acceptance rate of the drafted steps by position in the chain (ten equal ranges of the step
+    index), from a window-by-window run of a few chains outside the timed region: a draft tested
+    at step k counts once, as accepted or rejected; drafts after a window's first rejection are
+    never tested."""
+    from paper_2501_05370_b200 import binding as sb
+    B = min(chains, w.B)
+    s = sds.sampler_for(w, B=B, device=dev)
+    s.set_option(s.OPT_VERIFY_EARLY_EXIT, 0)
+    s.reset()
+    tested, accepted = np.zeros(bins), np.zeros(bins)
+    na, windows, cap = B, 0, 800                        # very long chains: the first 800 windows only
+    while na > 0 and windows < cap:
+        n = s.get(sb.GET_N).astype(np.int64)
+        s.draft(); s.verify_window()
+        js, am = s.get(sb.GET_JSTAR).astype(np.int64), s.get(sb.GET_ACCMASK).astype(np.int64)
+        live = (n < w.K) & (js >= 1)
+        Lt = np.minimum(w.L, w.K - n)
+        last = np.minimum(js, Lt)                           # positions 1..last were tested
+        for j in range(1, w.L + 1):
+            m = live & (j <= last)
+            if not m.any():
+                break
+            bi = np.minimum(bins - 1, (n[m] + j - 1) * bins // w.K)
+            np.add.at(tested, bi, 1)
+            np.add.at(accepted, bi, (am[m] >> (j - 1)) & 1)
+        na = s.advance()
+        windows += 1
+    s.close()
+    return {"chains": B, "bins": bins, "windows": windows,
+            "rate": [round(float(a / t), 4) if t > 0 else None for a, t in zip(accepted, tested)]}
+
+
 def run_gpu(args, w):
     import torch
     import torch.distributed as dist
@@ -394,6 +427,8 @@ def run_gpu(args, w):
                 "share_of_kernel_time": dom_ms / max(sum(v[0] for v in kinds.values()), 1e-9),
                 "kernel_ms_per_step": {k: v[0] / steps for k, v in kinds.items()}}
 
+    acc_profile = acceptance_by_step(sds, w, dev)
+
     osteps, sec, what = oracle_time(w, args.cpu_seconds)
     cpu = {"value": osteps / sec, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what}
     psteps, psec = oracle_plain_time(w, max(1.0, args.cpu_seconds / 5))
@@ -404,7 +439,8 @@ def run_gpu(args, w):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": ("bf16" if w.dtype == "bf16" else "f32"), "data": "synthetic", "config": workload_config(w, args),
         "nfe": {"K": K, "mean_target_calls": float(calls_np.mean()), "mean_target_rows": float(rows_np.mean()),
-                "mean_advance": float(K * B / max(windows_chains, 1)), "calls_saved_frac": float(1 - calls_np.mean() / K)},
+                "mean_advance": float(K * B / max(windows_chains, 1)), "calls_saved_frac": float(1 - calls_np.mean() / K),
+                "acceptance_by_step": acc_profile},
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e / steps,
                 "h2d_bytes_per_step": int(means_h.numel() * means_h.element_size() + logw_h.numel() * 4) if means_h is not None else 0,
                 "d2h_bytes_per_step": int(out_h.numel() * 4 + calls_h.numel() * 4 + rows_h.numel() * 4)},
