@@ -165,3 +165,24 @@ def test_bounded_wait_runs_out_and_reports():
     torch.cuda.synchronize()
     assert int(st.item()) == 1
     assert float((torch.ones(4, device="cuda") * 2).sum().item()) == 8.0
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4", "cfg5"])
+def test_full_size_runs_agree_bitwise_across_kernel_options(name):
+    """At the benchmark sizes: the verify kernel that exits early and advances its chains, the
+    CTA-pair GEMM and the whole-chain kernel change how the work is done, not one bit of the result,
+    and a repeated run reproduces itself."""
+    import torch
+    w = wl.WORKLOADS[name]
+    s = sds.sampler_for(w)
+    ref = None
+    for fuse, early, pair, whole in [(1, 1, 1, 1), (1, 1, 1, 1), (0, 1, 1, 1), (1, 0, 1, 1), (0, 0, 0, 0)]:
+        s.set_option(s.OPT_FUSE_ADVANCE, fuse); s.set_option(s.OPT_VERIFY_EARLY_EXIT, early)
+        s.set_option(s.OPT_GEMM_PAIR, pair); s.set_option(s.OPT_WHOLE_CHAIN_KERNEL, whole)
+        got = [x.clone() for x in s.sample_all()]
+        if ref is None:
+            ref = got
+            assert torch.isfinite(ref[0]).all()
+        else:
+            assert all(torch.equal(a, b) for a, b in zip(ref, got)), (fuse, early, pair, whole)
+    s.close()
