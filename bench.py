@@ -406,6 +406,8 @@ def run_gpu(args, w):
     dom = max(kinds, key=lambda k: kinds[k][0]) if kinds else "fused"
     dom_ms, dom_n = kinds.get(dom, (ms_total, steps))
     denoise_launch_groups = {"mlp": len(w.mlp_dims) - 1}.get(w.denoiser, 3 if (w.denoiser == "gmm" and w.gmm.get("means_bf16")) else 1)
+    from paper_2501_05370_b200 import binding as sb
+    split_products, t_full, t_brief = 4.5, 0, 0
     bound, per_launch = algorithmic(dom, w, rows_per_step, windows_chains, dom_n / steps)
     avg_s = dom_ms / max(dom_n, 1) * 1e-3
     if bound == "hbm":
@@ -414,14 +416,20 @@ def run_gpu(args, w):
         achieved, peak, unit = per_launch / avg_s / 1e12, pk["bf16_sustained"], "TFLOP/s"
     elif bound == "tensor_split":
         # float-equivalent flops: the logits contraction costs 3 bf16 products per float product, the
-        # mixing contraction 6, and the two contractions are the same size: 4.5 on average
-        achieved, peak, unit = per_launch / avg_s / 1e12, pk["bf16_sustained"] / 4.5, "TFLOP/s"
+        # mixing contraction 6 (or 3, see below), and the two contractions are the same size
+        # where a tile of responsibilities needs only its first plane (one-hot rows) the mixing contraction
+        # runs 3 products instead of 6; the library counts both kinds of tile
+        ctl = s.get(sb.GET_CTL)
+        t_full, t_brief = int(ctl[8]), int(ctl[9])
+        mix_products = (6.0 * t_full + 3.0 * t_brief) / max(1, t_full + t_brief)
+        split_products = (3.0 + mix_products) / 2.0
+        achieved, peak, unit = per_launch / avg_s / 1e12, pk["bf16_sustained"] / split_products, "TFLOP/s"
     else:
         peak = SMS * FP32_LANES_PER_SM * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
         achieved, unit = per_launch / avg_s / 1e12, "TFLOP/s"
     roofline = {"kernel": dom, "bound": "tensor" if bound == "tensor_split" else bound, "achieved": achieved, "peak": peak, "unit": unit,
                 "frac": achieved / peak, "traffic": None,
-                "peak_source": (pk["source"] + {"tensor": " (sustained bf16 GEMM)", "tensor_split": " (sustained bf16 GEMM / 4.5: 3 bf16 products per float product in the logits, 6 in the mixing)"}.get(bound, " (copy)")) if bound != "alu"
+                "peak_source": (pk["source"] + {"tensor": " (sustained bf16 GEMM)", "tensor_split": f" (sustained bf16 GEMM / {split_products:.2f}: 3 bf16 products per float product in the logits, 6 in the mixing, 3 for tiles of one-hot rows: {t_brief} of {t_full + t_brief} tiles)"}.get(bound, " (copy)")) if bound != "alu"
                 else "derived: 148 SMs x 128 fp32 lanes x 2 x max SM clock",
                 "avg_launch_us": avg_s * 1e6, "launches_per_step": dom_n / steps,
                 "share_of_kernel_time": dom_ms / max(sum(v[0] for v in kinds.values()), 1e-9),

@@ -88,7 +88,9 @@ extern "C" {
 #define SDS_GET_JSTAR     14    /* int32  [B]         first rejected position, Lt+1 if none */
 #define SDS_GET_NFE_CALLS 15    /* int32  [B]         sequential batched target calls the chain took part in */
 #define SDS_GET_NFE_ROWS  16    /* int32  [B]         target rows evaluated for the chain */
-#define SDS_GET_CTL       17    /* int32  [8]         n_active, nrows, windows done, error word, frozen chains, ... */
+#define SDS_GET_CTL       17    /* int32  [16]        n_active, nrows, windows done, error word, frozen chains, ...;
+                                   [8], [9]: mixing-GEMM tiles of the split-precision mixture run with all six
+                                   products / with the three of the first plane since sds_reset */
 #define SDS_GET_ROWK      18    /* int32  [nrows]     transition index of each row */
 #define SDS_GET_DP        19    /* float  [nrows, d]  independent drafter: the draft model's output per drafted row */
 

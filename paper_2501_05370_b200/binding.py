@@ -361,7 +361,7 @@ class Sampler:
         """Host copy of an internal array."""
         dt, shp = self._GET[what]
         B, L, d = self.B, self.L, self.d
-        shape = {"rows_d": (B * L, d), "B_d": (B, d), "B": (B,), "B1": (B + 1,), "B_L": (B, L), "ctl": (8,),
+        shape = {"rows_d": (B * L, d), "B_d": (B, d), "B": (B,), "B1": (B + 1,), "B_L": (B, L), "ctl": (16,),
                  "rows": (B * L,)}[shp]
         arr = np.empty(shape, dtype=dt)
         self._chk(self.lib.sds_get(self.h, what, arr.ctypes.data, arr.nbytes, 1), "sds_get")

@@ -50,6 +50,7 @@ struct DenLayout {
   size_t H0, H1;          // MLP hidden activations (bf16)
   size_t logits, R, Mt;   // large mixture: logits (f32), responsibilities (bf16), transposed means (bf16)
   size_t Xs, Ms;          // float mixture on tensor cores: 3 bf16 planes of the rows / of the means
+  size_t flags;           // one int per 128 rows: responsibilities with a non-zero second or third plane
   size_t xb;              // where a bf16 copy of this denoiser's input rows goes when the caller has none
 };
 
@@ -121,13 +122,14 @@ bool wants_bf16_rows(const sds_denoiser& den) {
 void den_layout(Carve& cv, const sds_denoiser* den, size_t K, int tcond_dim, size_t rows, int32_t d, DenLayout* l) {
   l->tcond = cv.take(K * (size_t)(tcond_dim > 0 ? tcond_dim : 1) * 8);
   l->musq = (den->kind == SDS_DEN_GMM) ? cv.take((size_t)den->ncomp * 8) : kNone;
-  l->H0 = l->H1 = l->logits = l->R = l->Mt = l->Xs = l->Ms = kNone;
+  l->H0 = l->H1 = l->logits = l->R = l->Mt = l->Xs = l->Ms = l->flags = kNone;
   if (gmm_split_shape(*den, d)) {
     l->Xs = cv.take(2 * rows * (size_t)d * 2);
     l->Ms = cv.take(3 * (size_t)den->ncomp * d * 2);
     l->Mt = cv.take(3 * (size_t)d * den->ncomp * 2);
     l->R = cv.take(3 * rows * (size_t)den->ncomp * 2);
     l->logits = cv.take(rows * (size_t)den->ncomp * 4);
+    l->flags = cv.take(((rows + 255) / 256 * 2) * 4);
   }
   if (den->kind == SDS_DEN_MLP) {
     size_t width = 0;
@@ -398,15 +400,23 @@ int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, cons
         g.nseg = 3; g.nplanes = 2; g.a_plane = cap * dd; g.b_plane = nc * dd;
         for (int i = 0; i < 3; ++i) { g.a_idx[i] = kLa[i]; g.b_idx[i] = kLb[i]; }
         SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiGmmLogits, g, Xs, Ms, c->stream));
+        // rows whose responsibilities need only their first bf16 plane (one-hot rows above all) let
+        // the mixing contraction drop the three products with the other planes, tile by tile
+        int* flags = at<int>(c, e.lay.flags);
+        SDS_CU(c, cudaMemsetAsync(flags, 0, (((size_t)rows_ub + 255) / 256 * 2) * 4, c->stream));
         SDS_LAUNCH(c, SDS_PROF_DENOISE,
                    launch_softmax_split3(logits, nrows_dev, (int)rows_ub, (int)nc, (int)dd, X, means,
                                          at<double>(c, e.lay.musq), e.den.logw_dev, at<double>(c, e.lay.tcond), rowk,
-                                         cap * nc, Rs, c->stream));
+                                         cap * nc, Rs, flags, c->stream));
         TcGemmArgs m = tc_args(c, e, rowk, nrows_dev, rows_ub);
         m.N = (int)dd; m.K = (int)nc; m.out = out; m.ldo = (int)dd;
         m.tcond = at<double>(c, e.lay.tcond); m.xrows = X;
         m.nseg = 6; m.nplanes = 3; m.a_plane = cap * nc; m.b_plane = nc * dd;
         for (int i = 0; i < 6; ++i) { m.a_idx[i] = kA[i]; m.b_idx[i] = kB[i]; }
+        static const uint8_t kSa[3] = {0, 0, 0}, kSb[3] = {2, 1, 0};   // the products with the first plane, same order
+        m.tile_flags = flags; m.nseg_short = 3;
+        m.tile_counts = at<int>(c, c->lay.ctl) + kCtlTilesFull;
+        for (int i = 0; i < 3; ++i) { m.a_short[i] = kSa[i]; m.b_short[i] = kSb[i]; }
         SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiGmmMix, m, Rs, Mt, c->stream));
         return SDS_OK;
       }
@@ -758,12 +768,12 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
       if (rc != SDS_OK) return rc;
       if (fused_adv) c->state = kReady;
       else if ((rc = sds_advance(c, nullptr)) != SDS_OK) return rc;
-      SDS_CU(c, cudaMemcpyAsync(c->h_pin + 8 + (w & 1) * kCtlWords, A.ctl, kCtlWords * 4, cudaMemcpyDeviceToHost,
+      SDS_CU(c, cudaMemcpyAsync(c->h_pin + 16 + (w & 1) * kCtlWords, A.ctl, kCtlWords * 4, cudaMemcpyDeviceToHost,
                                 c->stream));
       SDS_CU(c, cudaEventRecord(c->ev[w & 1], c->stream));
       if (w >= 1) {
         SDS_CU(c, cudaEventSynchronize(c->ev[(w - 1) & 1]));
-        const int na = c->h_pin[8 + ((w - 1) & 1) * kCtlWords + kCtlNActive];
+        const int na = c->h_pin[16 + ((w - 1) & 1) * kCtlWords + kCtlNActive];
         if (na == 0) break;
         c->ub = na;
       }

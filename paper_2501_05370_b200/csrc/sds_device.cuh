@@ -24,7 +24,9 @@ enum Ctl : int {
   kCtlDone = 5,       // block-completion counter of the advance kernel
   kCtlTcError = 6,    // set by a tensor-core kernel whose bounded wait gave up
   kCtlSpare1 = 7,
-  kCtlWords = 8
+  kCtlTilesFull = 8,  // mixing-GEMM tiles of the split-precision mixture run with all six products since reset
+  kCtlTilesBrief = 9, // ... and with the three products of the first plane only
+  kCtlWords = 16
 };
 constexpr int kErrNonFinite = 1;
 

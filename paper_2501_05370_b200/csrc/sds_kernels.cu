@@ -116,6 +116,8 @@ __global__ void __launch_bounds__(kBlock) k_init(WinArgs A) {
     A.ctl[kCtlFrozen] = 0;
     A.ctl[kCtlDone] = 0;
     A.ctl[kCtlTcError] = 0;
+    A.ctl[kCtlTilesFull] = 0;
+    A.ctl[kCtlTilesBrief] = 0;
   }
   if (b >= A.B) return;
   const uint64_t bg = A.chain_off + (uint64_t)b;

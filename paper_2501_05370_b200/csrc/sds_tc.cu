@@ -196,6 +196,15 @@ __device__ __forceinline__ void epilogue_chunk(const TcGemmArgs& g, const uint32
   // the other epilogues (SiLU hidden layer, acc + bias, C * acc + E * x) are written in the kernel body
 }
 
+// whether tile row `tm` (TM rows) may take the short segment list: no flag set in its row blocks of 128
+template <int TM>
+__device__ __forceinline__ bool tile_is_brief(const TcGemmArgs& g, int tm) {
+  if (!g.tile_flags || g.nseg_short <= 0) return false;
+  int f = __ldg(g.tile_flags + tm * (TM / 128));
+  if (TM == 256) f |= __ldg(g.tile_flags + tm * 2 + 1);
+  return f == 0;
+}
+
 template <int BN, int EPI, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
     k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
@@ -261,11 +270,13 @@ __global__ void __launch_bounds__(kThreads, 1)
       const uint32_t leader_full0 = PAIR ? map_to_cta(smem_u32(full_bar), 0u) : 0u;
       for (int t = worker; t < total_tiles && ok; t += nworkers) {
         const int m0 = (t / n_tiles) * TM + (int)rank * BM, n0 = (t % n_tiles) * BN + (int)rank * C::kBRows;
-        for (int kb = 0; kb < kblocks; ++kb) {
+        const bool brief = tile_is_brief<TM>(g, t / n_tiles);
+        const int nkb = brief ? kb_seg * g.nseg_short : kblocks;
+        for (int kb = 0; kb < nkb; ++kb) {
           if (!mbar_wait(empty_bar + stage, phase ^ 1u, abort_s)) { ok = false; break; }
           uint8_t* sa = stages + stage * C::kStageBytes;
           const int seg = kb / kb_seg, kk = (kb - seg * kb_seg) * BK;
-          const int ai = g.a_idx[seg], bi = g.b_idx[seg];
+          const int ai = brief ? g.a_short[seg] : g.a_idx[seg], bi = brief ? g.b_short[seg] : g.b_idx[seg];
           const CUtensorMap* ta = ai == 0 ? &tmA0 : (ai == 1 ? &tmA1 : &tmA2);
           const CUtensorMap* tb = bi == 0 ? &tmB0 : (bi == 1 ? &tmB1 : &tmB2);
           if (PAIR) {
@@ -301,7 +312,10 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (!mbar_wait(tempty_bar + buf, bphase ^ 1u, abort_s)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
-        for (int kb = 0; kb < kblocks; ++kb) {
+        const bool brief = tile_is_brief<TM>(g, t / n_tiles);
+        const int nkb = brief ? kb_seg * g.nseg_short : kblocks;
+        if (g.tile_counts) atomicAdd(g.tile_counts + (brief ? 1 : 0), 1);
+        for (int kb = 0; kb < nkb; ++kb) {
           if (!mbar_wait(full_bar + stage, phase, abort_s)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_u32(stages + stage * C::kStageBytes);
@@ -558,7 +572,7 @@ __global__ void __launch_bounds__(256)
                      const float* __restrict__ X, const float* __restrict__ means,
                      const double* __restrict__ musq, const float* __restrict__ logw,
                      const double* __restrict__ tcond, const int* __restrict__ rowk, size_t rplane,
-                     uint16_t* __restrict__ R) {
+                     uint16_t* __restrict__ R, int* __restrict__ tile_flags) {
   constexpr int ncomp = 128 * NQ;
   const int nrows = nrows_dev ? min(*nrows_dev, rows_host) : rows_host;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -620,17 +634,24 @@ __global__ void __launch_bounds__(256)
       }
     den = warp_sum(den);
     const float inv = 1.0f / den;
+    uint32_t lower = 0u;                          // any non-zero entry in the second or third plane of this row
 #pragma unroll
     for (int q = 0; q < NQ; ++q) {
       uint16_t p[3][4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) split3(v[q][u] * inv, p[0][u], p[1][u], p[2][u]);
+      for (int u = 0; u < 4; ++u) {
+        float r = v[q][u] * inv;
+        if (r < 0x1p-40f) r = 0.f;               // below 1e-12 of the row: dropped (keeps one-hot rows exactly one-hot)
+        split3(r, p[0][u], p[1][u], p[2][u]);
+        lower |= (uint32_t)p[1][u] | (uint32_t)p[2][u];
+      }
       const size_t o = (size_t)row * ncomp + 4 * (lane + 32 * q);
 #pragma unroll
       for (int pl = 0; pl < 3; ++pl)
         *reinterpret_cast<uint2*>(R + pl * rplane + o) = make_uint2((uint32_t)p[pl][0] | ((uint32_t)p[pl][1] << 16),
                                                                     (uint32_t)p[pl][2] | ((uint32_t)p[pl][3] << 16));
     }
+    if (tile_flags && __any_sync(0xffffffffu, lower != 0u) && lane == 0) tile_flags[row >> 7] = 1;
   }
 }
 
@@ -789,14 +810,15 @@ cudaError_t launch_split3(const float* x, size_t n, size_t plane, int nplanes, u
 
 cudaError_t launch_softmax_split3(const float* logits, const int* nrows_dev, int rows_host, int ncomp, int d,
                                   const float* X, const float* means, const double* musq, const float* logw,
-                                  const double* tcond, const int* rowk, size_t rplane, uint16_t* R, cudaStream_t st) {
+                                  const double* tcond, const int* rowk, size_t rplane, uint16_t* R, int* tile_flags,
+                                  cudaStream_t st) {
   int blocks = (rows_host + 7) / 8;
   if (blocks > 148 * 8) blocks = 148 * 8;
   if (blocks < 1) blocks = 1;
 #define SDS_SM3(NQ)                                                                                              \
   case NQ:                                                                                                       \
     k_softmax_split3<NQ><<<blocks, 256, 0, st>>>(logits, nrows_dev, rows_host, d, X, means, musq, logw, tcond,   \
-                                                 rowk, rplane, R);                                               \
+                                                 rowk, rplane, R, tile_flags);                                   \
     break;
   switch (ncomp / 128) {
     SDS_SM3(1) SDS_SM3(2) SDS_SM3(3) SDS_SM3(4) SDS_SM3(5) SDS_SM3(6) SDS_SM3(7) SDS_SM3(8)

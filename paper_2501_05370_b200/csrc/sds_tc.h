@@ -36,6 +36,13 @@ struct TcGemmArgs {
   int nseg, nplanes;
   size_t a_plane, b_plane;
   uint8_t a_idx[8], b_idx[8];
+  // optional short segment list per row block: tile_flags[r] (one int per 128 rows of A) == 0 for
+  // every row block of a tile means planes 1.. of A are all zero there, and the tile runs the
+  // nseg_short segments a_short/b_short instead (the products left out are exact zeros)
+  const int* tile_flags;
+  int* tile_counts;      // optional: [0] += tiles run with the full list, [1] += tiles run with the short one
+  int nseg_short;
+  uint8_t a_short[8], b_short[8];
 };
 
 bool tc_shape_ok(int N, int K);
@@ -47,9 +54,12 @@ cudaError_t launch_musq_bf16(const uint16_t* means, int ncomp, int d, double* mu
 cudaError_t launch_wait_selftest(uint32_t polls, int* status_dev, cudaStream_t st);
 // the first nplanes (1..3) of the three-way bf16 split of x, planes `plane` elements apart
 cudaError_t launch_split3(const float* x, size_t n, size_t plane, int nplanes, uint16_t* out, cudaStream_t st);
+// tile_flags: one int per 128 rows, zeroed by the caller; set where a row has a non-zero entry in the
+// second or third plane of its responsibilities
 cudaError_t launch_softmax_split3(const float* logits, const int* nrows_dev, int rows_host, int ncomp, int d,
                                   const float* X, const float* means, const double* musq, const float* logw,
-                                  const double* tcond, const int* rowk, size_t rplane, uint16_t* R, cudaStream_t st);
+                                  const double* tcond, const int* rowk, size_t rplane, uint16_t* R, int* tile_flags,
+                                  cudaStream_t st);
 cudaError_t launch_f32_to_bf16(const float* x, size_t n, uint16_t* out, cudaStream_t st);
 
 }  // namespace sds
