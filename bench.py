@@ -72,7 +72,65 @@ def oracle_closure(w):
     return o, den, a, c, sig
 
 
-def oracle_time(w, budget_s: float, min_chains: int = 1, first_chain: int = 0):
+VARIANTS = ("default", "exact", "independent", "picard2", "tau2", "proj16")
+
+
+def draft_mixture(w):
+    """The cheaper draft model of the `independent` variant: the first half of the mixture's components."""
+    gp = w.gmm_params()
+    half = max(1, w.gmm["ncomp"] // 2)
+    return wl.GmmParams(means=gp.means[:half].copy(), logw=np.full((half,), -np.log(half), dtype=np.float32),
+                        comp_std=gp.comp_std, means_bf16=gp.means_bf16)
+
+
+def proj_matrix(w, r: int = 16):
+    return np.random.default_rng(1234).standard_normal((r, w.d))
+
+
+def gpu_sampler(sds, w, variant: str, **kw):
+    """The sampler of a bench variant: the default drafter, or one of the other drafters / accept tests."""
+    import torch
+    from paper_2501_05370_b200 import binding as sb
+    if variant == "exact":
+        s = sds.sampler_for(w, drafter_mode=sb.SDS_FROZEN_EXACT, **kw)
+    elif variant == "independent":
+        if w.denoiser != "gmm":
+            raise SystemExit("--variant independent is defined for the mixture workloads")
+        s = sds.sampler_for(w, drafter=sds.drafter_for(w, gmm=draft_mixture(w)), **kw)
+    elif variant == "picard2":
+        s = sds.sampler_for(w, picard=sds.picard_for(w, 2), **kw)
+    else:
+        s = sds.sampler_for(w, **kw)
+    if variant == "tau2":
+        s.set_temperature(2.0)
+    if variant == "proj16":
+        s.set_projection(torch.from_numpy(sb.projection_basis(proj_matrix(w))).to(kw.get("device", "cuda:0")))
+    return s
+
+
+def oracle_chain_kwargs(w, variant: str, o, a, c, sig):
+    """Keyword arguments that make the oracle's chain follow the same variant."""
+    if variant == "exact":
+        return dict(mode=o.FROZEN_EXACT)
+    if variant == "independent":
+        gp = draft_mixture(w)
+        if w.sampler == "ddpm":
+            abar = o.ddpm_affine(w.beta())[3]
+            dd = lambda x, k: o.gmm_posterior_mean(x, abar[k], gp.means, gp.logw, gp.comp_std, bf16_operands=gp.means_bf16)
+        else:
+            dd = lambda x, k: o.gmm_grad_energy(x, gp.means, gp.logw, gp.comp_std)
+        return dict(mode=o.INDEPENDENT, draft_denoise=dd)
+    if variant == "picard2":
+        ad, cd = o.ddim_affine(w.beta()) if w.sampler == "ddpm" else o.ula_affine(w.K, w.ula_gamma)[:2]
+        return dict(mode=o.PICARD, picard=(2, ad, cd))
+    if variant == "tau2":
+        return dict(mode=getattr(w, "drafter_mode", 0), tau=2.0)
+    if variant == "proj16":
+        return dict(mode=getattr(w, "drafter_mode", 0), proj=proj_matrix(w))
+    return dict(mode=getattr(w, "drafter_mode", 0))
+
+
+def oracle_time(w, budget_s: float, min_chains: int = 1, first_chain: int = 0, variant: str = "default"):
     """Runs oracle chains one after another for about budget_s seconds of CPU work.
 
     Heavy workloads cannot finish even one chain in the budget, so a chain is run over the first
@@ -84,8 +142,10 @@ def oracle_time(w, budget_s: float, min_chains: int = 1, first_chain: int = 0):
     prefix = False
     while True:
         t1 = time.perf_counter()
-        o.speculative_chain(den, a[:Kp], c[:Kp], sig[:Kp], w.L, w.sample_seed, first_chain + n, w.d,
-                            mode=getattr(w, "drafter_mode", 0))
+        okw = oracle_chain_kwargs(w, variant, o, a, c, sig)
+        if "picard" in okw:
+            okw["picard"] = (okw["picard"][0], okw["picard"][1][:Kp], okw["picard"][2][:Kp])
+        o.speculative_chain(den, a[:Kp], c[:Kp], sig[:Kp], w.L, w.sample_seed, first_chain + n, w.d, **okw)
         dt = time.perf_counter() - t1
         n += 1
         steps += Kp
@@ -127,10 +187,10 @@ def run_reference(args, w):
         return
     per_step_budget = max(1.0, min(8.0, 60.0 / max(1, args.steps + args.warmup)))
     for _ in range(args.warmup):
-        oracle_time(w, per_step_budget / 2)
+        oracle_time(w, per_step_budget / 2, variant=args.variant)
     tot_steps, tot_s, what = 0, 0.0, ""
     for i in range(args.steps):
-        n, s, what = oracle_time(w, per_step_budget, first_chain=i * 16)
+        n, s, what = oracle_time(w, per_step_budget, first_chain=i * 16, variant=args.variant)
         tot_steps += n
         tot_s += s
     value = tot_steps / tot_s
@@ -151,7 +211,13 @@ def workload_config(w, args):
     return {"workload": f"{w.name}: B={w.B} chains/GPU, d={w.d}, L={w.L}, K={w.K}, {w.sampler} "
                         f"{w.schedule or 'gamma=%g' % w.ula_gamma}, {w.denoiser} denoiser"
                         + (f" ncomp={w.gmm['ncomp']}" if w.denoiser == 'gmm' else ""),
-            "drafter": "frozen target output " + ("evaluated at Y_n" if getattr(w, "drafter_mode", 0) else "(carried)"),
+            "drafter": {"exact": "frozen target output evaluated at Y_n",
+                        "independent": "independent draft model: the first half of the mixture's components",
+                        "picard2": "Picard drafter, 2 parallel target calls per window"}.get(
+                            getattr(args, "variant", "default"),
+                            "frozen target output " + ("evaluated at Y_n" if getattr(w, "drafter_mode", 0) else "(carried)")),
+            "accept_test": {"tau2": "temperature 2 (inexact)", "proj16": "decided in the image of a 16 x d matrix (inexact)"}.get(
+                getattr(args, "variant", "default"), "exact"),
             "seed": w.sample_seed,
             "l2": "256 MiB buffer written between timed steps (working set may fit L2)",
             "sharding": "chains by global id, no data-path collective"}
@@ -257,14 +323,14 @@ def algorithmic(kind: str, w, rows_per_step: float, windows_chains: float, launc
     return "hbm", 0.0
 
 
-def acceptance_by_step(sds, w, dev, chains: int = 64, bins: int = 10):
+def acceptance_by_step(sds, w, dev, variant: str = "default", chains: int = 64, bins: int = 10):
     """Acceptance rate of the drafted steps by position in the chain (ten equal ranges of the step
     index), from a window-by-window run of a few chains outside the timed region: a draft tested
     at step k counts once, as accepted or rejected; drafts after a window's first rejection are
     never tested."""
     from paper_2501_05370_b200 import binding as sb
     B = min(chains, w.B)
-    s = sds.sampler_for(w, B=B, device=dev)
+    s = gpu_sampler(sds, w, variant, B=B, device=dev)
     s.set_option(s.OPT_VERIFY_EARLY_EXIT, 0)
     s.reset()
     tested, accepted = np.zeros(bins), np.zeros(bins)
@@ -311,7 +377,7 @@ def run_gpu(args, w):
         torch.cuda.synchronize()
 
     from paper_2501_05370_b200 import sharding
-    s = sds.sampler_for(w, chain_id_offset=sharding.weak_offset(rank, w.B), device=dev)
+    s = gpu_sampler(sds, w, args.variant, chain_id_offset=sharding.weak_offset(rank, w.B), device=dev)
     B, d, K = w.B, w.d, w.K
     out = torch.empty((B, d), dtype=torch.float32, device=dev)
     calls = torch.empty((B,), dtype=torch.int32, device=dev)
@@ -395,10 +461,16 @@ def run_gpu(args, w):
     ms_per_step = ms_total / steps
     value = world * B * K / (ms_per_step * 1e-3)
     e2e_value = world * B * K / (ms_e2e / steps * 1e-3)
-    if getattr(w, "drafter_mode", 0) == 1:
+    if getattr(w, "drafter_mode", 0) == 1 or args.variant == "exact":
         # drafter evaluated at Y_n: no initial call, two sequential calls per window (one for a last window of one row)
         rows_per_step = float(rows_np.sum())
         windows_chains = float(np.ceil(calls_np / 2.0).sum())
+    elif args.variant == "independent":                       # no initial call, one target call per window
+        rows_per_step = float(rows_np.sum())
+        windows_chains = float(calls_np.sum())
+    elif args.variant == "picard2":                           # initial call, then 2 draft calls + 1 verify call per window
+        windows_chains = float(np.ceil((calls_np - 1) / 3.0).sum())
+        rows_per_step = float(w.L * windows_chains)           # rows of the verify calls (full windows assumed)
     else:
         rows_per_step = float(rows_np.sum() - B)              # rows verified (the initial call is not a window)
         windows_chains = float(calls_np.sum() - B)
@@ -435,9 +507,9 @@ def run_gpu(args, w):
                 "share_of_kernel_time": dom_ms / max(sum(v[0] for v in kinds.values()), 1e-9),
                 "kernel_ms_per_step": {k: v[0] / steps for k, v in kinds.items()}}
 
-    acc_profile = acceptance_by_step(sds, w, dev)
+    acc_profile = acceptance_by_step(sds, w, dev, args.variant)
 
-    osteps, sec, what = oracle_time(w, args.cpu_seconds)
+    osteps, sec, what = oracle_time(w, args.cpu_seconds, variant=args.variant)
     cpu = {"value": osteps / sec, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what}
     psteps, psec = oracle_plain_time(w, max(1.0, args.cpu_seconds / 5))
     cpu["plain_chain_value"] = psteps / psec          # the oracle's plain sequential chain, same unit, for context
@@ -470,6 +542,8 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="budget of the cpu_baseline leg")
     ap.add_argument("--chains", type=int, default=0, help="chains per GPU (default: the workload's own B)")
+    ap.add_argument("--variant", default="default", choices=VARIANTS,
+                    help="another drafter or accept test on the same workload (default: the workload's own)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "sds":
         args.warmup = 3
