@@ -740,7 +740,8 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
   if (c->state < kBound) return SDS_ESTATE;
   WinArgs A = win_args(c);
   int rc = SDS_OK;
-  if (c->whole_chain && !c->Q && c->mode == SDS_FROZEN_PREV && c->tgt.den.kind == SDS_DEN_GMM && fused_small_supported(c->d, c->tgt.den.ncomp, c->L)) {
+  if (c->whole_chain && !c->Q && (c->mode == SDS_FROZEN_PREV || c->mode == SDS_FROZEN_EXACT) &&
+      c->tgt.den.kind == SDS_DEN_GMM && fused_small_supported(c->d, c->tgt.den.ncomp, c->L)) {
     if ((rc = ensure_musq(c, c->tgt)) != SDS_OK) return rc;
     SDS_CU(c, cudaMemsetAsync(A.ctl, 0, kCtlWords * 4, c->stream));   // no chain active afterwards, error bits clear
     SDS_LAUNCH(c, SDS_PROF_FUSED, launch_fused_small(A, gmm_args(c, c->tgt), c->stream));

@@ -21,7 +21,9 @@ __host__ __device__ inline int fused_warp_floats(int d, int L) {
   return 4 * kMaxL + kSmallScratchFloats + (2 * L + 2) * small_ldx(d) + 32;
 }
 
-template <int G, bool VEC4>
+// EXACT: the frozen drafter of the main text (Eq. 6), whose frozen output is the target at (Y_n, t_n),
+// evaluated at the start of every window; otherwise the carried output of the previous window.
+template <int G, bool VEC4, bool EXACT>
 __global__ void __maxnreg__(72) k_fused_small(WinArgs A, GmmArgs P) {
   extern __shared__ __align__(16) float smem[];
   constexpr int RPW = 32 / G;
@@ -57,12 +59,19 @@ __global__ void __maxnreg__(72) k_fused_small(WinArgs A, GmmArgs P) {
       for (int i = lane; i < d; i += 32) sW[i] = normal1(A.seed, kStreamInit, bg, 0u, (uint32_t)i);
     }
     __syncwarp();
-    gmm_row_small<G>(sW, ldx, sLg, g == 0, S, __ldg(P.tcond + 0), __ldg(P.tcond + 1), __ldg(P.tcond + 2),
-                     __ldg(P.tcond + 3), sEs + g * G, sDc, gl);
-    int n = 0, calls = 1, rows = 1;
+    if (!EXACT)
+      gmm_row_small<G>(sW, ldx, sLg, g == 0, S, __ldg(P.tcond + 0), __ldg(P.tcond + 1), __ldg(P.tcond + 2),
+                       __ldg(P.tcond + 3), sEs + g * G, sDc, gl);
+    int n = 0, calls = EXACT ? 0 : 1, rows = EXACT ? 0 : 1;
     bool frozen = false;
     while (n < K) {
       const int Lt = min(L, K - n);
+      if (EXACT) {      // frozen output = the target at (Y_n, t_n); it is also the target output of position 1
+        gmm_row_small<G>(sW, ldx, sLg, g == 0, S, __ldg(P.tcond + 4 * n + 0), __ldg(P.tcond + 4 * n + 1),
+                         __ldg(P.tcond + 4 * n + 2), __ldg(P.tcond + 4 * n + 3), sEs + g * G, sDc, gl);
+        for (int i = lane; i < d; i += 32) sDq[i] = sDc[i];
+        __syncwarp();
+      }
       // draft noise for all positions at once, then the sequential recurrence per element
       if (VEC4) {
         // element e = lane + 32 it is block q of position j; (j, q) advance by (32 / nq, 32 % nq) with carry
@@ -85,7 +94,7 @@ __global__ void __maxnreg__(72) k_fused_small(WinArgs A, GmmArgs P) {
       else draft_recurrence<4>(A, sW, sDc, ldx, d, n, Lt, lane);
       __syncwarp();
       // target rows W_0 .. W_{Lt-1}
-      for (int j0 = 0; j0 < Lt; j0 += RPW) {
+      for (int j0 = EXACT ? 1 : 0; j0 < Lt; j0 += RPW) {
         const int j = j0 + g;
         const bool valid = j < Lt;
         const int jj = valid ? j : 0;
@@ -173,7 +182,7 @@ __global__ void __maxnreg__(72) k_fused_small(WinArgs A, GmmArgs P) {
       }
       __syncwarp();
       n += adv;
-      calls += 1;
+      calls += (EXACT && Lt > 1) ? 2 : 1;   // with the drafter at Y_n: that call and the batched one
       rows += Lt;
     }
     for (int i = lane; i < d; i += 32) {
@@ -204,7 +213,7 @@ int fused_max_warps(int d, int ncomp, int L) {
   return 0;
 }
 
-template <int G, bool VEC4>
+template <int G, bool VEC4, bool EXACT>
 cudaError_t fused_launch_t(const WinArgs& A, const GmmArgs& P, cudaStream_t st) {
   // pick the CTA size that keeps the most warps resident per SM (one wave if the batch allows)
   int dev = 0, sms = 148;
@@ -213,20 +222,20 @@ cudaError_t fused_launch_t(const WinArgs& A, const GmmArgs& P, cudaStream_t st) 
   int best_w = 0, best_res = 0, best_blocks = 0;
   for (int w = fused_max_warps(A.d, P.ncomp, A.L); w >= 2; w -= 2) {
     const size_t smem = fused_smem_bytes(A.d, P.ncomp, A.L, w);
-    cudaError_t e = cudaFuncSetAttribute(k_fused_small<G, VEC4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(k_fused_small<G, VEC4, EXACT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int nb = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_fused_small<G, VEC4>, w * 32, smem);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_fused_small<G, VEC4, EXACT>, w * 32, smem);
     if (e != cudaSuccess) return e;
     if (nb * w > best_res) { best_res = nb * w; best_w = w; best_blocks = nb; }
   }
   if (best_w == 0) return cudaErrorInvalidConfiguration;
   const size_t smem = fused_smem_bytes(A.d, P.ncomp, A.L, best_w);
-  cudaError_t e = cudaFuncSetAttribute(k_fused_small<G, VEC4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(k_fused_small<G, VEC4, EXACT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   int blocks = (A.B + best_w - 1) / best_w;
   if (blocks > best_blocks * sms) blocks = best_blocks * sms;
-  k_fused_small<G, VEC4><<<blocks, best_w * 32, smem, st>>>(A, P);
+  k_fused_small<G, VEC4, EXACT><<<blocks, best_w * 32, smem, st>>>(A, P);
   return cudaGetLastError();
 }
 
@@ -237,9 +246,13 @@ bool fused_small_supported(int d, int ncomp, int L) {
 }
 
 cudaError_t launch_fused_small(const WinArgs& A, const GmmArgs& P, cudaStream_t st) {
-  const bool vec4 = (A.d % 4) == 0;
-  if (small_group(P.ncomp) == 16) return vec4 ? fused_launch_t<16, true>(A, P, st) : fused_launch_t<16, false>(A, P, st);
-  return vec4 ? fused_launch_t<32, true>(A, P, st) : fused_launch_t<32, false>(A, P, st);
+  const bool vec4 = (A.d % 4) == 0, exact = A.mode == 1;
+  if (small_group(P.ncomp) == 16) {
+    if (exact) return vec4 ? fused_launch_t<16, true, true>(A, P, st) : fused_launch_t<16, false, true>(A, P, st);
+    return vec4 ? fused_launch_t<16, true, false>(A, P, st) : fused_launch_t<16, false, false>(A, P, st);
+  }
+  if (exact) return vec4 ? fused_launch_t<32, true, true>(A, P, st) : fused_launch_t<32, false, true>(A, P, st);
+  return vec4 ? fused_launch_t<32, true, false>(A, P, st) : fused_launch_t<32, false, false>(A, P, st);
 }
 
 }  // namespace sds

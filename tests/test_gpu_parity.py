@@ -314,15 +314,18 @@ FUSED_SHAPES = [(64, 2, 4, 100, 4), (300, 64, 8, 200, 16), (65, 33, 5, 23, 7), (
 @pytest.mark.parametrize("B,d,L,K,ncomp", FUSED_SHAPES)
 def test_whole_chain_kernel_equals_window_kernels_bitwise(B, d, L, K, ncomp):
     for name in ("cfg2", "cfg5"):
-        w = wl.WORKLOADS[name].scaled(B=B, d=d, L=L, K=K)
-        gp = w.gmm_params(d=d, ncomp=ncomp)
-        s = sds.sampler_for(w, gmm=gp, seed=77 + d, chain_id_offset=5)
-        f = [x.cpu().numpy() for x in s.sample_all()]
-        s.set_option(s.OPT_WHOLE_CHAIN_KERNEL, 0)
-        g = [x.cpu().numpy() for x in s.sample_all()]
-        assert np.array_equal(f[0], g[0]) and np.array_equal(f[1], g[1]) and np.array_equal(f[2], g[2])
-        assert np.all(np.isfinite(f[0]))
-        s.close()
+        for mode in (sb.SDS_FROZEN_PREV, sb.SDS_FROZEN_EXACT):       # carried output; target evaluated at Y_n
+            w = wl.WORKLOADS[name].scaled(B=B, d=d, L=L, K=K)
+            gp = w.gmm_params(d=d, ncomp=ncomp)
+            s = sds.sampler_for(w, gmm=gp, seed=77 + d, chain_id_offset=5, drafter_mode=mode)
+            l0 = s.launch_count()
+            f = [x.cpu().numpy() for x in s.sample_all()]
+            assert s.launch_count() - l0 <= 2                           # one kernel (plus the |mu|^2 table once)
+            s.set_option(s.OPT_WHOLE_CHAIN_KERNEL, 0)
+            g = [x.cpu().numpy() for x in s.sample_all()]
+            assert np.array_equal(f[0], g[0]) and np.array_equal(f[1], g[1]) and np.array_equal(f[2], g[2])
+            assert np.all(np.isfinite(f[0]))
+            s.close()
 
 
 def test_chain_shards_reproduce_the_unsharded_run_bitwise():
