@@ -208,11 +208,12 @@ int sds_advance(sds_ctx* ctx, int64_t* n_active);
 
 /* reset, then windows until no chain is active; copies Y_K to out_dev [B, d] and the counters to
  * nfe_calls_dev / nfe_rows_dev [B] (either may be NULL). Waits for the stream.
- * Small float mixtures run as one persistent kernel, one warp per chain, same results. */
+ * Small float mixtures and the lattice model run as one persistent kernel, one warp per chain, same results. */
 int sds_sample_all(sds_ctx* ctx, float* out_dev, int32_t* nfe_calls_dev, int32_t* nfe_rows_dev);
 
 /* Options. SDS_OPT_WHOLE_CHAIN_KERNEL (default 1): let sds_sample_all run small float mixtures
- * (d <= 256, <= 32 components) as one persistent kernel; 0 forces the window-by-window kernels.
+ * (d <= 256, <= 32 components; SDS_FROZEN_PREV or SDS_FROZEN_EXACT) and the lattice model
+ * (d <= 256, SDS_FROZEN_EXACT) as one persistent kernel; 0 forces the window-by-window kernels.
  * After the whole-chain kernel only Y, N, DC and the NFE counters are meaningful for sds_get. */
 #define SDS_OPT_WHOLE_CHAIN_KERNEL 1
 /* SDS_OPT_TENSOR_SPLIT (default 1): float mixtures with more than 32 components whose shapes tile
