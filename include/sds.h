@@ -160,7 +160,8 @@ int sds_create(const sds_schedule* sch, const sds_denoiser* den, int64_t B, int3
  * every position is a_k y + c_k D^p(y, k) with D^p = `drafter` (any kind but the callback), evaluated
  * sequentially, one position of all chains per call. drafter_tcond: [K, 4] host doubles (the
  * mixture coefficients of the draft model; NULL unless the drafter is a mixture). Bind with
- * SDS_INDEPENDENT. One batched target call per window; sds_sample_all uses the window kernels. */
+ * SDS_INDEPENDENT. One batched target call per window. sds_sample_all uses the window kernels, or the
+ * whole-chain kernel when target and draft model are both small float mixtures (<= 32 components, d <= 256). */
 int sds_workspace_bytes_with_drafter(const sds_schedule* sch, const sds_denoiser* den, const sds_denoiser* drafter,
                                      const double* drafter_tcond, int64_t B, int32_t d, int32_t L, size_t* bytes);
 int sds_create_with_drafter(const sds_schedule* sch, const sds_denoiser* den, const sds_denoiser* drafter,
@@ -212,7 +213,8 @@ int sds_advance(sds_ctx* ctx, int64_t* n_active);
 int sds_sample_all(sds_ctx* ctx, float* out_dev, int32_t* nfe_calls_dev, int32_t* nfe_rows_dev);
 
 /* Options. SDS_OPT_WHOLE_CHAIN_KERNEL (default 1): let sds_sample_all run small float mixtures
- * (d <= 256, <= 32 components; SDS_FROZEN_PREV or SDS_FROZEN_EXACT) and the lattice model
+ * (d <= 256, <= 32 components; SDS_FROZEN_PREV, SDS_FROZEN_EXACT, or SDS_INDEPENDENT with a draft model of
+ * the same kind) and the lattice model
  * (d <= 256, SDS_FROZEN_EXACT) as one persistent kernel; 0 forces the window-by-window kernels.
  * After the whole-chain kernel only Y, N, DC and the NFE counters are meaningful for sds_get. */
 #define SDS_OPT_WHOLE_CHAIN_KERNEL 1

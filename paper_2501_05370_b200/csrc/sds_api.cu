@@ -744,7 +744,18 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
       c->tgt.den.kind == SDS_DEN_GMM && fused_small_supported(c->d, c->tgt.den.ncomp, c->L)) {
     if ((rc = ensure_musq(c, c->tgt)) != SDS_OK) return rc;
     SDS_CU(c, cudaMemsetAsync(A.ctl, 0, kCtlWords * 4, c->stream));   // no chain active afterwards, error bits clear
-    SDS_LAUNCH(c, SDS_PROF_FUSED, launch_fused_small(A, gmm_args(c, c->tgt), c->stream));
+    SDS_LAUNCH(c, SDS_PROF_FUSED, launch_fused_small(A, gmm_args(c, c->tgt), nullptr, c->stream));
+    c->ub = 0;
+    c->state = kReady;
+  } else if (c->whole_chain && !c->Q && c->mode == SDS_INDEPENDENT && c->tgt.den.kind == SDS_DEN_GMM &&
+             c->tgt.den.means_dtype == SDS_F32 && c->drf.den.kind == SDS_DEN_GMM && c->drf.den.means_dtype == SDS_F32 &&
+             fused_small_supported_with_drafter(c->d, c->tgt.den.ncomp, c->drf.den.ncomp, c->L)) {
+    // small target and small independent draft model: both mixtures live in shared memory
+    if ((rc = ensure_musq(c, c->tgt)) != SDS_OK) return rc;
+    if ((rc = ensure_musq(c, c->drf)) != SDS_OK) return rc;
+    SDS_CU(c, cudaMemsetAsync(A.ctl, 0, kCtlWords * 4, c->stream));
+    const GmmArgs gd = gmm_args(c, c->drf);
+    SDS_LAUNCH(c, SDS_PROF_FUSED, launch_fused_small(A, gmm_args(c, c->tgt), &gd, c->stream));
     c->ub = 0;
     c->state = kReady;
   } else if (c->whole_chain && !c->Q && c->mode == SDS_FROZEN_EXACT && c->tgt.den.kind == SDS_DEN_PHI4 &&

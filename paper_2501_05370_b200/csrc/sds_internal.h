@@ -96,7 +96,8 @@ cudaError_t launch_phi4_grad(const float* X, const int* nrows_dev, int rows_ub, 
 
 // whole-chain persistent kernel for small mixtures (sds_fused.cu)
 bool fused_small_supported(int d, int ncomp, int L);
-cudaError_t launch_fused_small(const WinArgs& A, const GmmArgs& G, cudaStream_t st);
+bool fused_small_supported_with_drafter(int d, int ncomp, int ncomp_d, int L);
+cudaError_t launch_fused_small(const WinArgs& A, const GmmArgs& G, const GmmArgs* drafter, cudaStream_t st);
 
 // whole-chain kernel for the lattice model with the drafter evaluated at Y_n (sds_fused_phi4.cu)
 bool fused_phi4_ok(int d, int L);

@@ -311,6 +311,24 @@ FUSED_SHAPES = [(64, 2, 4, 100, 4), (300, 64, 8, 200, 16), (65, 33, 5, 23, 7), (
                 (33, 68, 3, 31, 9), (4, 8, 8, 3, 4)]
 
 
+@pytest.mark.parametrize("B,d,L,K,ncomp,ncomp_d", [(40, 64, 8, 60, 16, 8), (9, 33, 5, 23, 7, 20), (3, 5, 2, 9, 3, 1),
+                                                   (12, 128, 6, 40, 20, 32), (17, 16, 32, 70, 16, 16)])
+def test_whole_chain_kernel_with_independent_drafter_equals_window_kernels_bitwise(B, d, L, K, ncomp, ncomp_d):
+    for name in ("cfg2", "cfg5"):
+        w = wl.WORKLOADS[name].scaled(B=B, d=d, L=L, K=K)
+        gp = w.gmm_params(d=d, ncomp=ncomp)
+        gd = wl.gmm_params(4321, ncomp_d, d, w.gmm["mean_scale"] * 1.1, w.gmm["comp_std"] * 1.3)
+        res = {}
+        for fused in (1, 0):
+            s = sds.sampler_for(w, gmm=gp, seed=91 + d, chain_id_offset=3, drafter=sds.drafter_for(w, gmm=gd))
+            s.set_option(s.OPT_WHOLE_CHAIN_KERNEL, fused)
+            l0 = s.launch_count()
+            res[fused] = [x.cpu().numpy() for x in s.sample_all()] + [s.launch_count() - l0]
+            s.close()
+        assert all(np.array_equal(x, y) for x, y in zip(res[1][:3], res[0][:3]))
+        assert res[1][3] <= 3 < res[0][3]
+
+
 @pytest.mark.parametrize("B,d,L,K,ncomp", FUSED_SHAPES)
 def test_whole_chain_kernel_equals_window_kernels_bitwise(B, d, L, K, ncomp):
     for name in ("cfg2", "cfg5"):
