@@ -822,3 +822,19 @@ def test_speculative_and_plain_chains_agree_in_law_on_the_gpu():
     u = np.random.default_rng(0).standard_normal(w.d); u /= np.linalg.norm(u)
     from scipy import stats
     assert stats.ks_2samp(S @ u, P @ u).pvalue > 1e-3
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("d", [2, 8, 32])
+def test_sequential_target_calls_fall_with_the_window_size(d):
+    """Section 7, low-dimensional mixtures (16 components, 200 steps): the number of sequential
+    target calls falls as the window grows, and window 1 is the plain chain's count."""
+    calls = []
+    for L in (1, 2, 4, 8, 16):
+        w = wl.WORKLOADS["cfg2"].scaled(B=512, d=d, L=L)
+        s = sds.sampler_for(w, gmm=w.gmm_params(d=d), seed=5)
+        calls.append(float(s.sample_all()[1].float().mean().item()))
+        s.close()
+    assert calls[0] == 1 + 200
+    assert all(a > b for a, b in zip(calls, calls[1:])), calls
+    assert calls[-1] < 0.6 * 200
