@@ -236,15 +236,14 @@ __device__ __forceinline__ void draft_recurrence(const Args& A, float* sW, const
 // of the differences to the neighbours (order up, down, left, right; free or periodic boundaries)
 // plus the derivative 4 x (x^2 - 1) of the site potential
 // ---------------------------------------------------------------------------------------
-__device__ __forceinline__ float phi4_site(const float* x, int i, int side, float beta, int periodic) {
-  const int r = i / side, c = i - r * side;
+__device__ __forceinline__ float phi4_site_rc(const float* x, int i, int r, int c, int side, float beta, int periodic) {
   const float xi = x[i];
   float acc = 0.f;
   if (periodic) {
-    acc += xi - x[((r + side - 1) % side) * side + c];
-    acc += xi - x[((r + 1) % side) * side + c];
-    acc += xi - x[r * side + (c + side - 1) % side];
-    acc += xi - x[r * side + (c + 1) % side];
+    acc += xi - x[(r > 0 ? r - 1 : side - 1) * side + c];
+    acc += xi - x[(r < side - 1 ? r + 1 : 0) * side + c];
+    acc += xi - x[r * side + (c > 0 ? c - 1 : side - 1)];
+    acc += xi - x[r * side + (c < side - 1 ? c + 1 : 0)];
   } else {
     if (r > 0) acc += xi - x[i - side];
     if (r < side - 1) acc += xi - x[i + side];
@@ -252,6 +251,10 @@ __device__ __forceinline__ float phi4_site(const float* x, int i, int side, floa
     if (c < side - 1) acc += xi - x[i + 1];
   }
   return fmaf(beta, acc, 4.0f * xi * fmaf(xi, xi, -1.0f));
+}
+__device__ __forceinline__ float phi4_site(const float* x, int i, int side, float beta, int periodic) {
+  const int r = i / side;
+  return phi4_site_rc(x, i, r, i - r * side, side, beta, periodic);
 }
 
 }  // namespace sds

@@ -28,6 +28,13 @@ __global__ void __maxnreg__(72) k_fused_phi4(WinArgs A, int side, float beta, in
   const bool pack2 = VEC4 ? (d <= 64) : (d <= 16);
   const int PW = pack2 ? 16 : 32;
   const int vh = lane / PW, vt = lane % PW;
+  // grid coordinates of this lane's sites (lane + 32 u), found once: row << 8 | column
+  int site_rc[2];                                             // lattices of up to 64 sites: two sites per lane
+#pragma unroll
+  for (int u = 0; u < 2; ++u) {
+    const int i = lane + 32 * u, r = i / side;
+    site_rc[u] = (r << 8) | (i - r * side);
+  }
   // noise generation walks (position, block) pairs without a division per element
   const int nz_n = VEC4 ? d / 4 : d;
   const int nz_j0 = lane / nz_n, nz_q0 = lane % nz_n, nz_dj = 32 / nz_n, nz_dq = 32 % nz_n;
@@ -46,10 +53,22 @@ __global__ void __maxnreg__(72) k_fused_phi4(WinArgs A, int side, float beta, in
     while (n < K) {
       const int Lt = min(L, K - n);
       // frozen output = the target at (Y_n, t_n); it is also the target output of position 1
-      for (int i = lane; i < d; i += 32) {
-        const float g0 = phi4_site(sW, i, side, beta, periodic);
-        sDc[i] = g0;
-        sDq[i] = g0;
+      if (d <= 64) {
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int i = lane + 32 * u;
+          if (i < d) {
+            const float g0 = phi4_site_rc(sW, i, site_rc[u] >> 8, site_rc[u] & 255, side, beta, periodic);
+            sDc[i] = g0;
+            sDq[i] = g0;
+          }
+        }
+      } else {
+        for (int i = lane; i < d; i += 32) {
+          const float g0 = phi4_site(sW, i, side, beta, periodic);
+          sDc[i] = g0;
+          sDq[i] = g0;
+        }
       }
       __syncwarp();
       // draft noise for all positions at once, then the sequential recurrence per element
@@ -74,9 +93,19 @@ __global__ void __maxnreg__(72) k_fused_phi4(WinArgs A, int side, float beta, in
       else draft_recurrence<4>(A, sW, sDc, ldx, d, n, Lt, lane);
       __syncwarp();
       // target rows W_1 .. W_{Lt-1} (row 0 is the frozen output)
-      for (int e = lane; e < (Lt - 1) * d; e += 32) {
-        const int j = 1 + e / d, i = e - (j - 1) * d;
-        sDq[j * ldx + i] = phi4_site(sW + j * ldx, i, side, beta, periodic);
+      if (d <= 64) {
+        for (int j = 1; j < Lt; ++j) {
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            const int i = lane + 32 * u;
+            if (i < d) sDq[j * ldx + i] = phi4_site_rc(sW + j * ldx, i, site_rc[u] >> 8, site_rc[u] & 255, side, beta, periodic);
+          }
+        }
+      } else {
+        for (int e = lane; e < (Lt - 1) * d; e += 32) {
+          const int j = 1 + e / d, i = e - (j - 1) * d;
+          sDq[j * ldx + i] = phi4_site(sW + j * ldx, i, side, beta, periodic);
+        }
       }
       __syncwarp();
       // S1 = |Delta|^2, S2 = Delta.Z per position
