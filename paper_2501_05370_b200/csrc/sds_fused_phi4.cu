@@ -12,8 +12,11 @@ namespace {
 __host__ __device__ inline int lat_ldx(int d) { return (d + 3) / 4 * 4 + 4; }
 __host__ __device__ inline int lat_warp_floats(int d, int L) { return 4 * kMaxL + (2 * L + 2) * lat_ldx(d); }
 
-template <bool VEC4>
-__global__ void __maxnreg__(72) k_fused_phi4(WinArgs A, int side, float beta, int periodic) {
+// ROOMY: few chains (not more warps than fit at 128 registers each): the kernel is latency-bound,
+// so it takes the registers that keep everything out of local memory; otherwise the cap that keeps
+// 28 warps per SM resident.
+template <bool VEC4, bool ROOMY>
+__global__ void __maxnreg__(ROOMY ? 128 : 72) k_fused_phi4(WinArgs A, int side, float beta, int periodic) {
   extern __shared__ __align__(16) float smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   const int d = A.d, L = A.L, K = A.K;
@@ -212,7 +215,7 @@ bool fused_phi4_supported(int d, int L) {
   return d <= 256 && L <= kMaxL && (size_t)2 * lat_warp_floats(d, L) * 4 <= 220 * 1024;
 }
 
-template <bool VEC4>
+template <bool VEC4, bool ROOMY>
 cudaError_t fused_phi4_launch_t(const WinArgs& A, int side, float beta, int periodic, cudaStream_t st) {
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
@@ -221,15 +224,15 @@ cudaError_t fused_phi4_launch_t(const WinArgs& A, int side, float beta, int peri
   int w = 4;
   while (w > 1 && (size_t)w * lat_warp_floats(A.d, A.L) * 4 > 220 * 1024) w >>= 1;
   const size_t smem = (size_t)w * lat_warp_floats(A.d, A.L) * 4;
-  cudaError_t e = cudaFuncSetAttribute(k_fused_phi4<VEC4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(k_fused_phi4<VEC4, ROOMY>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   int nb = 0;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_fused_phi4<VEC4>, w * 32, smem);
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_fused_phi4<VEC4, ROOMY>, w * 32, smem);
   if (e != cudaSuccess) return e;
   if (nb < 1) return cudaErrorInvalidConfiguration;
   int blocks = (A.B + w - 1) / w;
   if (blocks > nb * sms) blocks = nb * sms;
-  k_fused_phi4<VEC4><<<blocks, w * 32, smem, st>>>(A, side, beta, periodic);
+  k_fused_phi4<VEC4, ROOMY><<<blocks, w * 32, smem, st>>>(A, side, beta, periodic);
   return cudaGetLastError();
 }
 
@@ -238,8 +241,15 @@ cudaError_t fused_phi4_launch_t(const WinArgs& A, int side, float beta, int peri
 bool fused_phi4_ok(int d, int L) { return fused_phi4_supported(d, L); }
 
 cudaError_t launch_fused_phi4(const WinArgs& A, int side, float beta, int periodic, cudaStream_t st) {
-  return (A.d % 4) == 0 ? fused_phi4_launch_t<true>(A, side, beta, periodic, st)
-                        : fused_phi4_launch_t<false>(A, side, beta, periodic, st);
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const bool roomy = (long long)A.B <= (long long)sms * 16;       // 16 warps of 128 registers per SM
+  if ((A.d % 4) == 0)
+    return roomy ? fused_phi4_launch_t<true, true>(A, side, beta, periodic, st)
+                 : fused_phi4_launch_t<true, false>(A, side, beta, periodic, st);
+  return roomy ? fused_phi4_launch_t<false, true>(A, side, beta, periodic, st)
+               : fused_phi4_launch_t<false, false>(A, side, beta, periodic, st);
 }
 
 }  // namespace sds
