@@ -241,6 +241,11 @@ int sds_sample_all(sds_ctx* ctx, float* out_dev, int32_t* nfe_calls_dev, int32_t
  * last rebuilds the active list, so a window is draft, denoiser, verify: one launch less. Same
  * results. The step-wise calls sds_verify_window / sds_advance are not affected. */
 #define SDS_OPT_FUSE_ADVANCE 5
+/* SDS_OPT_RAW_ROWS (default 1): inside sds_sample_all, for mixture denoisers on the tensor cores with a
+ * frozen drafter, the mixing GEMM stores its accumulators and the verify and advance kernels, which
+ * hold the rows' inputs anyway, apply the affine map C acc + E x with the same operations: the GEMM's
+ * epilogue no longer reads the rows. Same results, bit for bit. */
+#define SDS_OPT_RAW_ROWS 6
 int sds_set_option(sds_ctx* ctx, int32_t option, int64_t value);
 
 /* Temperature of the accept test (Appendix D, temperature rejection): a draft is accepted iff

@@ -98,6 +98,8 @@ struct sds_ctx {
   bool early_exit = true;           // verify stops reading a window after the block with the first rejection
   bool fuse_advance = true;         // sds_sample_all lets the verify kernel do the advance step where it can
   bool fusing = false;              // set around the verify call of the sds_sample_all loop
+  bool raw_rows = true;             // sds_sample_all lets the mixing GEMM store accumulators, verify applies C acc + E x
+  bool raw_now = false;             // set around the verify and advance calls of the sds_sample_all loop
   // optional per-kernel timing: event pairs recorded around each launch, summed on read
   bool prof_on = false;
   std::vector<cudaEvent_t> prof_ev[SDS_PROF_KINDS];
@@ -253,6 +255,7 @@ WinArgs win_args(sds_ctx* c) {
   A.inv_tau = 1.0 / c->tau;
   A.early_exit = c->early_exit ? 1 : 0;
   A.fuse_advance = c->fusing ? 1 : 0;
+  A.raw_tcond = c->raw_now ? at<double>(c, c->tgt.lay.tcond) : nullptr;
   A.seed = c->seed; A.chain_off = (uint64_t)c->chain_off;
   A.a = at<float>(c, c->lay.a); A.c = at<float>(c, c->lay.c); A.sigma = at<float>(c, c->lay.sigma);
   A.Y = at<float>(c, c->lay.Y); A.Dc = at<float>(c, c->lay.Dc); A.T = at<float>(c, c->lay.T);
@@ -364,7 +367,7 @@ TcGemmArgs tc_args(sds_ctx* c, Engine& e, const int* rowk, const int* nrows_dev,
 // run the target denoiser on dense rows X (and their bf16 copy Xb, NULL = make one); the row count
 // lives on the device (nrows_dev, may be NULL) with a host upper bound for the grids
 int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, const int* rowk, const int* nrows_dev,
-                 int64_t rows_ub, float* out, bool planes_ready = false) {
+                 int64_t rows_ub, float* out, bool planes_ready = false, bool raw = false) {
   if (rows_ub <= 0) return SDS_OK;
   switch (e.den.kind) {
     case SDS_DEN_GMM: {
@@ -410,7 +413,7 @@ int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, cons
                                          cap * nc, Rs, flags, c->stream));
         TcGemmArgs m = tc_args(c, e, rowk, nrows_dev, rows_ub);
         m.N = (int)dd; m.K = (int)nc; m.out = out; m.ldo = (int)dd;
-        m.tcond = at<double>(c, e.lay.tcond); m.xrows = X;
+        m.tcond = at<double>(c, e.lay.tcond); m.xrows = raw ? nullptr : X;
         m.nseg = 6; m.nplanes = 3; m.a_plane = cap * nc; m.b_plane = nc * dd;
         for (int i = 0; i < 6; ++i) { m.a_idx[i] = kA[i]; m.b_idx[i] = kB[i]; }
         static const uint8_t kSa[3] = {0, 0, 0}, kSb[3] = {2, 1, 0};   // the products with the first plane, same order
@@ -445,7 +448,7 @@ int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, cons
       SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_softmax_bf16(logits, nrows_dev, (int)rows_ub, e.den.ncomp, R, c->stream));
       TcGemmArgs m = tc_args(c, e, rowk, nrows_dev, rows_ub);
       m.N = c->d; m.K = e.den.ncomp; m.out = out; m.ldo = c->d;
-      m.tcond = at<double>(c, e.lay.tcond); m.xrows = X;
+      m.tcond = at<double>(c, e.lay.tcond); m.xrows = raw ? nullptr : X;
       SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiGmmMix, m, R, Mt, c->stream));
       return SDS_OK;
     }
@@ -719,7 +722,8 @@ int sds_verify_window(sds_ctx* c) {
   WinArgs A = win_args(c);
   // rows drafted by k_draft (the two frozen-output modes) come with their bf16 planes
   const bool planes_ready = A.Xs != nullptr && (c->mode == SDS_FROZEN_PREV || c->mode == SDS_FROZEN_EXACT);
-  const int rc = run_denoiser(c, c->tgt, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, (int64_t)c->ub * c->L, A.Dq, planes_ready);
+  const int rc = run_denoiser(c, c->tgt, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, (int64_t)c->ub * c->L, A.Dq, planes_ready,
+                              c->raw_now);
   if (rc != SDS_OK) return rc;
   SDS_LAUNCH(c, SDS_PROF_VERIFY, launch_verify(A, c->ub, c->stream));
   c->state = kVerified;
@@ -774,12 +778,21 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
       if ((rc = sds_draft(c)) != SDS_OK) return rc;
       // where the register-resident verify kernel runs, it also advances its chains and compacts
       c->fusing = c->fuse_advance && verify_can_advance(A);
+      // mixtures on the tensor cores: the mixing GEMM stores its accumulators and the verify (and advance)
+      // kernels, which hold the rows' inputs anyway, apply C acc + E x: the GEMM's epilogue reads nothing
+      const bool tensor_mix = c->tgt.den.kind == SDS_DEN_GMM &&
+                              (c->tgt.den.means_dtype == SDS_BF16 || (c->tensor_split && gmm_split_shape(c->tgt.den, c->d)));
+      c->raw_now = c->raw_rows && tensor_mix && (c->mode == SDS_FROZEN_PREV || c->mode == SDS_FROZEN_EXACT) &&
+                   verify_reads_raw_rows(A);
       rc = sds_verify_window(c);
       const bool fused_adv = c->fusing;
       c->fusing = false;
+      if (rc == SDS_OK) {
+        if (fused_adv) c->state = kReady;
+        else rc = sds_advance(c, nullptr);
+      }
+      c->raw_now = false;
       if (rc != SDS_OK) return rc;
-      if (fused_adv) c->state = kReady;
-      else if ((rc = sds_advance(c, nullptr)) != SDS_OK) return rc;
       SDS_CU(c, cudaMemcpyAsync(c->h_pin + 16 + (w & 1) * kCtlWords, A.ctl, kCtlWords * 4, cudaMemcpyDeviceToHost,
                                 c->stream));
       SDS_CU(c, cudaEventRecord(c->ev[w & 1], c->stream));
@@ -916,6 +929,7 @@ int sds_set_option(sds_ctx* c, int32_t option, int64_t value) {
     case SDS_OPT_GEMM_PAIR: c->gemm_pair = value != 0; return SDS_OK;
     case SDS_OPT_VERIFY_EARLY_EXIT: c->early_exit = value != 0; return SDS_OK;
     case SDS_OPT_FUSE_ADVANCE: c->fuse_advance = value != 0; return SDS_OK;
+    case SDS_OPT_RAW_ROWS: c->raw_rows = value != 0; return SDS_OK;
     default: return SDS_EINVAL;
   }
 }

@@ -195,6 +195,11 @@ __device__ __forceinline__ void delta_z_any(bool mean, float wp, float wj, float
   }
 }
 
+// target output from a stored accumulator (rows kept raw by the mixing contraction): C acc + E x
+__device__ __forceinline__ float4 affine_row4(float cC, float cE, float4 acc, float4 x) {
+  return make_float4(fmaf(cC, acc.x, cE * x.x), fmaf(cC, acc.y, cE * x.y), fmaf(cC, acc.z, cE * x.z), fmaf(cC, acc.w, cE * x.w));
+}
+
 // reflected state: m^q + sigma (Z - coef * Delta), coef = 2 (Delta.Z)/|Delta|^2
 __device__ __forceinline__ float reflect_elem(float wp, float dq, float Z, float D, float a, float c, float s,
                                               float coef) {

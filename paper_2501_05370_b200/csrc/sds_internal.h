@@ -13,6 +13,8 @@ struct WinArgs {
   int mode;              // 0: carried target output; 1: target output at Y_n, recomputed before every
                          // window; 2: independent draft model evaluated at every drafted state
   double inv_tau;        // 1 / temperature of the accept test (1 = the exact method)
+  const double* raw_tcond;  // non-NULL: Dq holds the mixing contraction's accumulators; the target output of row r
+                            // (input X[r], step k = rowk[r]) is fma(C_k, Dq[r], E_k X[r]) with (.., .., C, E) = raw_tcond[4k..]
   int fuse_advance;      // the verify kernel also advances its chain and the last CTA compacts (no advance launch)
   int early_exit;        // verify stops reading a chain's window after the block of two (d >= 2048) or four positions
                          // that holds its first rejection (large-d kernels only)
@@ -79,6 +81,7 @@ cudaError_t launch_picard_start(const WinArgs& A, int ub_chains, cudaStream_t st
 cudaError_t launch_picard_step(const WinArgs& A, int ub_chains, cudaStream_t st);
 cudaError_t launch_picard_draft(const WinArgs& A, int ub_chains, cudaStream_t st);
 bool verify_can_advance(const WinArgs& A);
+bool verify_reads_raw_rows(const WinArgs& A);
 cudaError_t launch_verify(const WinArgs& A, int ub_chains, cudaStream_t st);
 cudaError_t launch_advance(const WinArgs& A, int ub_chains, cudaStream_t st);
 cudaError_t launch_rng_normals(uint64_t seed, int stream_id, uint64_t b0, int64_t nb, int k, int d, float* out,

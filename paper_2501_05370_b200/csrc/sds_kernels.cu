@@ -710,6 +710,11 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t)
         vq[e] = (i < A.d) ? ld4(dq + i) : zero4;
         if (A.Dp && i < A.d) vc[e] = ld4(A.Dp + (size_t)(r0 + j - 1) * A.d + i);   // independent draft model
       }
+      if (A.raw_tcond) {                 // rows kept raw: the row's input W_{j-1} is in registers already
+        const float cC = (float)__ldg(A.raw_tcond + 4 * k + 2), cE = (float)__ldg(A.raw_tcond + 4 * k + 3);
+#pragma unroll
+        for (int e = 0; e < EPT; ++e) vq[e] = affine_row4(cC, cE, vq[e], vp[e]);
+      }
       double p1 = 0.0, p2 = 0.0;
 #pragma unroll
       for (int e = 0; e < EPT; ++e) {
@@ -808,7 +813,13 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t)
           const int i = (t + e * TPC) * 4;
           if (i < A.d) {
             st4(A.Y + cb + i, ld4(A.T + cb + i));
-            st4(A.Dc + cb + i, ld4(A.Dq + (size_t)(r0 + Lt - 1) * A.d + i));
+            float4 q = ld4(A.Dq + (size_t)(r0 + Lt - 1) * A.d + i);
+            if (A.raw_tcond) {
+              const int kl = nb + Lt - 1;
+              q = affine_row4((float)__ldg(A.raw_tcond + 4 * kl + 2), (float)__ldg(A.raw_tcond + 4 * kl + 3), q,
+                              ld4(A.X + (size_t)(r0 + Lt - 1) * A.d + i));
+            }
+            st4(A.Dc + cb + i, q);
           }
         }
         if (t == 0) {
@@ -832,7 +843,9 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t)
   for (int e = 0; e < EPT; ++e) {
     const int i = (t + e * TPC) * 4;
     if (i < A.d) {
-      const float4 p = ld4(wp + i), w = ld4(wj + i), q = ld4(dq + i);
+      const float4 p = ld4(wp + i), w = ld4(wj + i);
+      float4 q = ld4(dq + i);
+      if (A.raw_tcond) q = affine_row4((float)__ldg(A.raw_tcond + 4 * k + 2), (float)__ldg(A.raw_tcond + 4 * k + 3), q, p);
       const float4 c4 = A.Dp ? ld4(A.Dp + (size_t)(r0 + jstar - 1) * A.d + i) : vc[e];
       float4 o;
       float D, Z;
@@ -888,7 +901,15 @@ __global__ void __launch_bounds__(kBlock) k_advance(WinArgs A) {
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
             const int i = i0 + u * TPC * 4;
-            if (i < A.d) { vy[u] = ld4(src + i); vd[u] = ld4(dsrc + i); }
+            if (i < A.d) {
+              vy[u] = ld4(src + i);
+              vd[u] = ld4(dsrc + i);
+              if (A.raw_tcond) {
+                const int kl = nb + adv - 1;
+                vd[u] = affine_row4((float)__ldg(A.raw_tcond + 4 * kl + 2), (float)__ldg(A.raw_tcond + 4 * kl + 3), vd[u],
+                                    ld4(A.X + (size_t)(r0 + adv - 1) * A.d + i));
+              }
+            }
           }
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
@@ -1006,6 +1027,9 @@ cudaError_t launch_picard_draft(const WinArgs& A, int ub, cudaStream_t st) {
   SDS_DISPATCH(k_picard_draft, A, ub, st);
   return cudaGetLastError();
 }
+// whether launch_verify takes the register-resident kernel (the one that also reads rows kept raw)
+bool verify_reads_raw_rows(const WinArgs& A) { return !A.Q && !A.mean_rows && !A.Dp && vec4_ok(A.d) && A.d <= 16384; }
+
 // whether launch_verify takes the register-resident kernel, the one that can also do the advance step
 // (and where that pays: for 256 < d <= 2048 the separate warp-per-chain advance kernel is faster than
 // one more fence and counter update in each of the many small verify CTAs)

@@ -361,7 +361,10 @@ __global__ void __launch_bounds__(kThreads, 1)
         // before the accumulator chunk is read.
         float* stg = epi_stage + (warp - 2) * (32 * 33);
         float rowC = 0.f, rowE = 0.f;
-        if (EPI == kEpiGmmMix) {
+        // xrows == NULL: the caller applies C acc + E x itself where it reads the rows (it holds x there
+        // anyway); the accumulator is stored as it is and this epilogue reads nothing
+        const bool affine = EPI == kEpiGmmMix && g.xrows != nullptr;
+        if (affine) {
           rowC = (float)__ldg(g.tcond + 4 * krow + 2);
           rowE = (float)__ldg(g.tcond + 4 * krow + 3);
         }
@@ -383,7 +386,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             }
           }
           float4 xv[8];
-          if (EPI == kEpiGmmMix) {
+          if (affine) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
               const int rl = 4 * i + rr4;
@@ -427,9 +430,11 @@ __global__ void __launch_bounds__(kThreads, 1)
                 continue;
               }
               float4 o;
-              if (EPI == kEpiGmmMix) {
+              if (affine) {
                 o = make_float4(fmaf(cC, sp[0], cE * xv[i].x), fmaf(cC, sp[1], cE * xv[i].y),
                                 fmaf(cC, sp[2], cE * xv[i].z), fmaf(cC, sp[3], cE * xv[i].w));
+              } else if (EPI == kEpiGmmMix) {
+                o = make_float4(sp[0], sp[1], sp[2], sp[3]);
               } else {
                 o = make_float4(sp[0] + bc.x, sp[1] + bc.y, sp[2] + bc.z, sp[3] + bc.w);
               }

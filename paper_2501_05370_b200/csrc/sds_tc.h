@@ -27,7 +27,7 @@ struct TcGemmArgs {
   const double* tcond;   // [Ksteps, 4]
   const double* musq;    // [N]
   const float* logw;     // [N]
-  const float* xrows;    // [M, N] f32
+  const float* xrows;    // [M, N] f32; NULL with the mixing epilogue: store the accumulator, no affine map
   int* err;              // device word, set non-zero if a bounded wait gave up
   // split-precision products: A and B each come as nplanes bf16 planes (a_plane / b_plane elements
   // apart); segment s of the K loop multiplies plane a_idx[s] of A with plane b_idx[s] of B.

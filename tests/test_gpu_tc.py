@@ -176,13 +176,15 @@ def test_full_size_runs_agree_bitwise_across_kernel_options(name):
     w = wl.WORKLOADS[name]
     s = sds.sampler_for(w)
     ref = None
-    for fuse, early, pair, whole in [(1, 1, 1, 1), (1, 1, 1, 1), (0, 1, 1, 1), (1, 0, 1, 1), (0, 0, 0, 0)]:
+    for fuse, early, pair, whole, raw in [(1, 1, 1, 1, 1), (1, 1, 1, 1, 1), (0, 1, 1, 1, 1), (1, 0, 1, 1, 1), (1, 1, 1, 1, 0),
+                                         (0, 0, 0, 0, 0)]:
         s.set_option(s.OPT_FUSE_ADVANCE, fuse); s.set_option(s.OPT_VERIFY_EARLY_EXIT, early)
         s.set_option(s.OPT_GEMM_PAIR, pair); s.set_option(s.OPT_WHOLE_CHAIN_KERNEL, whole)
+        s.set_option(s.OPT_RAW_ROWS, raw)
         got = [x.clone() for x in s.sample_all()]
         if ref is None:
             ref = got
             assert torch.isfinite(ref[0]).all()
         else:
-            assert all(torch.equal(a, b) for a, b in zip(ref, got)), (fuse, early, pair, whole)
+            assert all(torch.equal(a, b) for a, b in zip(ref, got)), (fuse, early, pair, whole, raw)
     s.close()
