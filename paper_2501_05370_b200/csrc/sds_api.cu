@@ -40,6 +40,7 @@ struct Layout {
   size_t S1, S2, ell, logU, accmask, jstar, nfe_calls, nfe_rows;
   size_t Gk;
   size_t Gx, Gb, Pb, Dp;  // independent drafter: gathered rows (f32, bf16), its outputs per call and per row
+  size_t ce;              // (C_k, E_k) of the target mixture as floats, for rows kept raw
   size_t adet, cdet;      // Picard drafter: deterministic sampler coefficients (Dp then holds draft means)
   size_t total;
 };
@@ -185,6 +186,7 @@ void make_layout(const sds_schedule* sch, const sds_denoiser* den, const sds_den
     den_layout(cv, drafter, K, 4, (size_t)B, d, dl);
     dl->xb = l.Gb;
   }
+  l.ce = (den->kind == SDS_DEN_GMM) ? cv.take(K * 8) : kNone;
   l.adet = l.cdet = kNone;
   if (picard) {
     l.adet = cv.take(K * 4);
@@ -255,7 +257,7 @@ WinArgs win_args(sds_ctx* c) {
   A.inv_tau = 1.0 / c->tau;
   A.early_exit = c->early_exit ? 1 : 0;
   A.fuse_advance = c->fusing ? 1 : 0;
-  A.raw_tcond = c->raw_now ? at<double>(c, c->tgt.lay.tcond) : nullptr;
+  A.raw_ce = c->raw_now ? at<float2>(c, c->lay.ce) : nullptr;
   A.seed = c->seed; A.chain_off = (uint64_t)c->chain_off;
   A.a = at<float>(c, c->lay.a); A.c = at<float>(c, c->lay.c); A.sigma = at<float>(c, c->lay.sigma);
   A.Y = at<float>(c, c->lay.Y); A.Dc = at<float>(c, c->lay.Dc); A.T = at<float>(c, c->lay.T);
@@ -648,6 +650,15 @@ int sds_bind(sds_ctx* c, void* workspace_dev, size_t bytes, void* cuda_stream, u
   SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.a, c->a.data(), kb, cudaMemcpyHostToDevice, c->stream));
   SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.c, c->c.data(), kb, cudaMemcpyHostToDevice, c->stream));
   SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.sigma, c->sigma.data(), kb, cudaMemcpyHostToDevice, c->stream));
+  if (c->lay.ce != kNone && c->tgt.tcond.size() == (size_t)c->K * 4) {
+    std::vector<float> ce((size_t)c->K * 2);
+    for (int k = 0; k < c->K; ++k) {
+      ce[2 * k] = (float)c->tgt.tcond[4 * (size_t)k + 2];
+      ce[2 * k + 1] = (float)c->tgt.tcond[4 * (size_t)k + 3];
+    }
+    SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.ce, ce.data(), ce.size() * 4, cudaMemcpyHostToDevice, c->stream));
+    SDS_CU(c, cudaStreamSynchronize(c->stream));      // the staging vector goes away
+  }
   if (c->picard_calls > 0) {
     SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.adet, c->a_det.data(), kb, cudaMemcpyHostToDevice, c->stream));
     SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.cdet, c->c_det.data(), kb, cudaMemcpyHostToDevice, c->stream));

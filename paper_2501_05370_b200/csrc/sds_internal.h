@@ -13,8 +13,8 @@ struct WinArgs {
   int mode;              // 0: carried target output; 1: target output at Y_n, recomputed before every
                          // window; 2: independent draft model evaluated at every drafted state
   double inv_tau;        // 1 / temperature of the accept test (1 = the exact method)
-  const double* raw_tcond;  // non-NULL: Dq holds the mixing contraction's accumulators; the target output of row r
-                            // (input X[r], step k = rowk[r]) is fma(C_k, Dq[r], E_k X[r]) with (.., .., C, E) = raw_tcond[4k..]
+  const float2* raw_ce;  // non-NULL: Dq holds the mixing contraction's accumulators; the target output of row r
+                         // (input X[r], step k = rowk[r]) is fma(C_k, Dq[r], E_k X[r]) with (C_k, E_k) = raw_ce[k]
   int fuse_advance;      // the verify kernel also advances its chain and the last CTA compacts (no advance launch)
   int early_exit;        // verify stops reading a chain's window after the block of two (d >= 2048) or four positions
                          // that holds its first rejection (large-d kernels only)

@@ -710,10 +710,10 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t)
         vq[e] = (i < A.d) ? ld4(dq + i) : zero4;
         if (A.Dp && i < A.d) vc[e] = ld4(A.Dp + (size_t)(r0 + j - 1) * A.d + i);   // independent draft model
       }
-      if (A.raw_tcond) {                 // rows kept raw: the row's input W_{j-1} is in registers already
-        const float cC = (float)__ldg(A.raw_tcond + 4 * k + 2), cE = (float)__ldg(A.raw_tcond + 4 * k + 3);
+      if (A.raw_ce) {                    // rows kept raw: the row's input W_{j-1} is in registers already
+        const float2 ce = __ldg(A.raw_ce + k);
 #pragma unroll
-        for (int e = 0; e < EPT; ++e) vq[e] = affine_row4(cC, cE, vq[e], vp[e]);
+        for (int e = 0; e < EPT; ++e) vq[e] = affine_row4(ce.x, ce.y, vq[e], vp[e]);
       }
       double p1 = 0.0, p2 = 0.0;
 #pragma unroll
@@ -814,10 +814,9 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t)
           if (i < A.d) {
             st4(A.Y + cb + i, ld4(A.T + cb + i));
             float4 q = ld4(A.Dq + (size_t)(r0 + Lt - 1) * A.d + i);
-            if (A.raw_tcond) {
-              const int kl = nb + Lt - 1;
-              q = affine_row4((float)__ldg(A.raw_tcond + 4 * kl + 2), (float)__ldg(A.raw_tcond + 4 * kl + 3), q,
-                              ld4(A.X + (size_t)(r0 + Lt - 1) * A.d + i));
+            if (A.raw_ce) {
+              const float2 ce = __ldg(A.raw_ce + nb + Lt - 1);
+              q = affine_row4(ce.x, ce.y, q, ld4(A.X + (size_t)(r0 + Lt - 1) * A.d + i));
             }
             st4(A.Dc + cb + i, q);
           }
@@ -845,7 +844,10 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t)
     if (i < A.d) {
       const float4 p = ld4(wp + i), w = ld4(wj + i);
       float4 q = ld4(dq + i);
-      if (A.raw_tcond) q = affine_row4((float)__ldg(A.raw_tcond + 4 * k + 2), (float)__ldg(A.raw_tcond + 4 * k + 3), q, p);
+      if (A.raw_ce) {
+        const float2 ce = __ldg(A.raw_ce + k);
+        q = affine_row4(ce.x, ce.y, q, p);
+      }
       const float4 c4 = A.Dp ? ld4(A.Dp + (size_t)(r0 + jstar - 1) * A.d + i) : vc[e];
       float4 o;
       float D, Z;
@@ -904,10 +906,9 @@ __global__ void __launch_bounds__(kBlock) k_advance(WinArgs A) {
             if (i < A.d) {
               vy[u] = ld4(src + i);
               vd[u] = ld4(dsrc + i);
-              if (A.raw_tcond) {
-                const int kl = nb + adv - 1;
-                vd[u] = affine_row4((float)__ldg(A.raw_tcond + 4 * kl + 2), (float)__ldg(A.raw_tcond + 4 * kl + 3), vd[u],
-                                    ld4(A.X + (size_t)(r0 + adv - 1) * A.d + i));
+              if (A.raw_ce) {
+                const float2 ce = __ldg(A.raw_ce + nb + adv - 1);
+                vd[u] = affine_row4(ce.x, ce.y, vd[u], ld4(A.X + (size_t)(r0 + adv - 1) * A.d + i));
               }
             }
           }
