@@ -246,6 +246,15 @@ int sds_sample_all(sds_ctx* ctx, float* out_dev, int32_t* nfe_calls_dev, int32_t
  * hold the rows' inputs anyway, apply the affine map C acc + E x with the same operations: the GEMM's
  * epilogue no longer reads the rows. Same results, bit for bit. */
 #define SDS_OPT_RAW_ROWS 6
+/* SDS_OPT_REGEN_DRAFTS (default 1; needs SDS_OPT_FUSE_ADVANCE): inside sds_sample_all, for SDS_FROZEN_PREV with
+ * d % 4 == 0, 256 < d <= 16384, the full-space test and a target that reads only the bf16 copy of its
+ * input rows (the MLP; the bf16 mixture with SDS_OPT_RAW_ROWS), the draft kernel stores only that copy and
+ * the verify kernel does not read drafted states at all. A drafted state (Algorithm 4, draft step) is a
+ * function of Y_n, the frozen target output and the chain's noise, which is a function of (seed, chain,
+ * step): verify runs the draft recurrence again in registers with the draft kernel's own operations,
+ * reads only the target outputs, and advances its chains. Same results, bit for bit. SDS_GET_X and
+ * SDS_GET_TAIL are then stale after sds_sample_all. */
+#define SDS_OPT_REGEN_DRAFTS 7
 int sds_set_option(sds_ctx* ctx, int32_t option, int64_t value);
 
 /* Temperature of the accept test (Appendix D, temperature rejection): a draft is accepted iff

@@ -384,6 +384,7 @@ class Sampler:
     OPT_VERIFY_EARLY_EXIT = 4
     OPT_FUSE_ADVANCE = 5
     OPT_RAW_ROWS = 6
+    OPT_REGEN_DRAFTS = 7
 
     def set_option(self, option: int, value: int):
         self._chk(self.lib.sds_set_option(self.h, option, value), "sds_set_option")

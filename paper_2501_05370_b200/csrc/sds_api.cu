@@ -98,9 +98,12 @@ struct sds_ctx {
   bool gemm_pair = true;            // tensor-core GEMMs with N % 256 == 0 run on CTA pairs
   bool early_exit = true;           // verify stops reading a window after the block with the first rejection
   bool fuse_advance = true;         // sds_sample_all lets the verify kernel do the advance step where it can
+  bool regen = true;                // sds_sample_all lets the verify kernel draw the drafted states again instead of reading them
   bool fusing = false;              // set around the verify call of the sds_sample_all loop
   bool raw_rows = true;             // sds_sample_all lets the mixing GEMM store accumulators, verify applies C acc + E x
   bool raw_now = false;             // set around the verify and advance calls of the sds_sample_all loop
+  bool regen_now = false;           // likewise: verify regenerates the drafted states
+  bool skipx_now = false;           // likewise: the draft kernel stores only the bf16 copy of its rows
   // optional per-kernel timing: event pairs recorded around each launch, summed on read
   bool prof_on = false;
   std::vector<cudaEvent_t> prof_ev[SDS_PROF_KINDS];
@@ -258,6 +261,8 @@ WinArgs win_args(sds_ctx* c) {
   A.early_exit = c->early_exit ? 1 : 0;
   A.fuse_advance = c->fusing ? 1 : 0;
   A.raw_ce = c->raw_now ? at<float2>(c, c->lay.ce) : nullptr;
+  A.regen = c->regen_now ? 1 : 0;
+  A.skip_x = c->skipx_now ? 1 : 0;
   A.seed = c->seed; A.chain_off = (uint64_t)c->chain_off;
   A.a = at<float>(c, c->lay.a); A.c = at<float>(c, c->lay.c); A.sigma = at<float>(c, c->lay.sigma);
   A.Y = at<float>(c, c->lay.Y); A.Dc = at<float>(c, c->lay.Dc); A.T = at<float>(c, c->lay.T);
@@ -786,15 +791,26 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
     // is enqueued the host waits for window w-1's count. A window enqueued with no active chain
     // does nothing on the device.
     for (int w = 0;; ++w) {
-      if ((rc = sds_draft(c)) != SDS_OK) return rc;
-      // where the register-resident verify kernel runs, it also advances its chains and compacts
-      c->fusing = c->fuse_advance && verify_can_advance(A);
       // mixtures on the tensor cores: the mixing GEMM stores its accumulators and the verify (and advance)
       // kernels, which hold the rows' inputs anyway, apply C acc + E x: the GEMM's epilogue reads nothing
       const bool tensor_mix = c->tgt.den.kind == SDS_DEN_GMM &&
                               (c->tgt.den.means_dtype == SDS_BF16 || (c->tensor_split && gmm_split_shape(c->tgt.den, c->d)));
       c->raw_now = c->raw_rows && tensor_mix && (c->mode == SDS_FROZEN_PREV || c->mode == SDS_FROZEN_EXACT) &&
                    verify_reads_raw_rows(A);
+      // Frozen drafter whose target reads nothing but the bf16 copy of its input rows (the MLP; the bf16 mixture
+      // with raw rows): the draft kernel stores only that copy, and verify, which then has no float rows to
+      // read, makes the drafted states again from what it holds and advances its chains (it alone knows the
+      // accepted state). Drawing the noise again costs about as much as reading the rows would, so this pays
+      // only through the draft kernel's smaller writes; where the float rows are needed anyway it stays off.
+      const bool bf16_only = A.Xb != nullptr &&
+                             (c->tgt.den.kind == SDS_DEN_MLP ||
+                              (c->tgt.den.kind == SDS_DEN_GMM && c->tgt.den.means_dtype == SDS_BF16 && c->raw_now));
+      c->regen_now = c->regen && c->fuse_advance && bf16_only && verify_can_regen(A);
+      c->skipx_now = c->regen_now;
+      // where the register-resident verify kernel runs, it also advances its chains and compacts
+      c->fusing = c->fuse_advance && (verify_can_advance(A) || c->regen_now);
+      rc = sds_draft(c);
+      if (rc != SDS_OK) { c->fusing = c->raw_now = c->regen_now = c->skipx_now = false; return rc; }
       rc = sds_verify_window(c);
       const bool fused_adv = c->fusing;
       c->fusing = false;
@@ -802,7 +818,7 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
         if (fused_adv) c->state = kReady;
         else rc = sds_advance(c, nullptr);
       }
-      c->raw_now = false;
+      c->raw_now = c->regen_now = c->skipx_now = false;
       if (rc != SDS_OK) return rc;
       SDS_CU(c, cudaMemcpyAsync(c->h_pin + 16 + (w & 1) * kCtlWords, A.ctl, kCtlWords * 4, cudaMemcpyDeviceToHost,
                                 c->stream));
@@ -941,6 +957,7 @@ int sds_set_option(sds_ctx* c, int32_t option, int64_t value) {
     case SDS_OPT_VERIFY_EARLY_EXIT: c->early_exit = value != 0; return SDS_OK;
     case SDS_OPT_FUSE_ADVANCE: c->fuse_advance = value != 0; return SDS_OK;
     case SDS_OPT_RAW_ROWS: c->raw_rows = value != 0; return SDS_OK;
+    case SDS_OPT_REGEN_DRAFTS: c->regen = value != 0; return SDS_OK;
     default: return SDS_EINVAL;
   }
 }

@@ -174,6 +174,11 @@ __device__ __forceinline__ float draft_step(float y, float dc, float xi, float a
   return fmaf(s, xi, fmaf(a, y, c * dc));
 }
 
+__device__ __forceinline__ float4 draft_step4(float4 y, float4 dc, float4 xi, float a, float c, float s) {
+  return make_float4(draft_step(y.x, dc.x, xi.x, a, c, s), draft_step(y.y, dc.y, xi.y, a, c, s),
+                     draft_step(y.z, dc.z, xi.z, a, c, s), draft_step(y.w, dc.w, xi.w, a, c, s));
+}
+
 // Delta_i = (m^p_i - m^q_i)/sigma = (c/sigma)(D_c - D_q);  Z_i = (W_j - a W_{j-1} - c D_c)/sigma
 __device__ __forceinline__ void delta_z(float wp, float wj, float dq, float dc, float a, float c, float cs,
                                         float inv_s, float& D, float& Z) {

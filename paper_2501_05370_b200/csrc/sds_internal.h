@@ -18,6 +18,9 @@ struct WinArgs {
   int fuse_advance;      // the verify kernel also advances its chain and the last CTA compacts (no advance launch)
   int early_exit;        // verify stops reading a chain's window after the block of two (d >= 2048) or four positions
                          // that holds its first rejection (large-d kernels only)
+  int regen;             // verify draws the drafted states again from Y_n, the carried output and the noise instead of
+                         // reading them (needs fuse_advance; see verify_can_regen)
+  int skip_x;            // the draft kernel stores only the bf16 copies of its rows (nothing reads the float rows)
   uint64_t seed;
   uint64_t chain_off;
   const float* a;        // [K]
@@ -82,6 +85,7 @@ cudaError_t launch_picard_step(const WinArgs& A, int ub_chains, cudaStream_t st)
 cudaError_t launch_picard_draft(const WinArgs& A, int ub_chains, cudaStream_t st);
 bool verify_can_advance(const WinArgs& A);
 bool verify_reads_raw_rows(const WinArgs& A);
+bool verify_can_regen(const WinArgs& A);
 cudaError_t launch_verify(const WinArgs& A, int ub_chains, cudaStream_t st);
 cudaError_t launch_advance(const WinArgs& A, int ub_chains, cudaStream_t st);
 cudaError_t launch_rng_normals(uint64_t seed, int stream_id, uint64_t b0, int64_t nb, int k, int d, float* out,

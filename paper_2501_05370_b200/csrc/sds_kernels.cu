@@ -219,7 +219,7 @@ __global__ void __launch_bounds__(kBlock) k_draft(WinArgs A) {
       const float4 dc = ld4(A.Dc + cb + i);
       for (int j = 0; j < Lt; ++j) {
         const size_t ro = (size_t)(r0 + j) * A.d + i;
-        st4(A.X + ro, y);
+        if (!A.skip_x) st4(A.X + ro, y);
         if (A.Xb) *reinterpret_cast<uint2*>(A.Xb + ro) = make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
         if (A.Xs) store_split2x4(A.Xs + ro, A.xs_plane, y);
         const int k = nb + j;
@@ -230,7 +230,7 @@ __global__ void __launch_bounds__(kBlock) k_draft(WinArgs A) {
         y.z = draft_step(y.z, dc.z, xi.z, ak, ck, sk);
         y.w = draft_step(y.w, dc.w, xi.w, ak, ck, sk);
       }
-      st4(A.T + cb + i, y);
+      if (!A.skip_x) st4(A.T + cb + i, y);
     }
   } else {
     for (int i = t; i < A.d; i += TPC) {
@@ -657,13 +657,30 @@ __global__ void __launch_bounds__(kBlock) k_verify(WinArgs A) {
   }
 }
 
+// Elements 4q .. 4q+3 of the drafted state W_to of a chain at step nb, continued from W_from (y) with the
+// carried output dc: the draft recurrence run again on the chain's own noise (to >= from).
+__device__ __forceinline__ float4 redraft4(const WinArgs& A, float4 y, float4 dc, uint64_t bg, int nb, int from, int to,
+                                           uint32_t q) {
+  for (int jj = from + 1; jj <= to; ++jj) {
+    const int k = nb + jj - 1;
+    y = draft_step4(y, dc, normal4(A.seed, kStreamDraft, bg, (uint32_t)k, q), __ldg(A.a + k), __ldg(A.c + k), __ldg(A.sigma + k));
+  }
+  return y;
+}
+
 // Register-resident variant for d % 4 == 0 and d <= 4 * EPT * TPC: each thread keeps its slice of
 // the carried output and of the previous drafted state in registers, so every position reads only
 // its own drafted state and target output from memory (8d bytes per verified step), with 2*EPT
 // independent 128-bit loads in flight per thread. Same per-thread element order and reduction
 // tree as k_verify, hence the same bits.
-template <int TPC, int EPT>
-__device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t) {
+// REGEN: the drafted states are not read at all. A drafted state is a function of Y_n, the carried
+// output and the chain's noise, all of which the thread holds or can draw again, so each position
+// reads only its target output (4d bytes per verified step) and the draft kernel need not store
+// the float rows. The state in front of the current block of positions stays in shared memory; the
+// tail (reflection, or the last row's input when all drafts pass) continues from it.
+template <int TPC, int EPT, bool REGEN>
+__device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t, float* snap) {
+  static_assert(!REGEN || TPC > 32, "regenerated drafts: one chain per CTA");
   constexpr int kWarps = TPC / 32;
   __shared__ double s_red[(TPC > 32) ? 2 * kMaxL * kWarps : 1];
   __shared__ int s_jstar;
@@ -681,8 +698,9 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t)
   for (int e = 0; e < EPT; ++e) {
     const int i = (t + e * TPC) * 4;
     vc[e] = (i < A.d) ? ld4(A.Dc + cb + i) : zero4;
-    vp[e] = (i < A.d) ? ld4(A.X + (size_t)r0 * A.d + i) : zero4;
+    vp[e] = (i < A.d) ? ld4((REGEN ? A.Y + cb : A.X + (size_t)r0 * A.d) + i) : zero4;   // W_0 = Y_n
   }
+  int snap_pos = 0;                                      // REGEN: snap holds this thread's slice of W_{snap_pos}
   // Positions are taken in blocks; with early exit (one chain per CTA, option on) the accept tests
   // of a block are decided before the next block is read, and nothing after the block that holds
   // the first rejection is read at all: those positions report zeros.
@@ -696,17 +714,25 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t)
   for (int jb = 1; jb <= Lt; jb += blk) {
     const int je = min(Lt, jb + blk - 1);
     double myS1 = 0.0, myS2 = 0.0;
+    if (REGEN) {                                         // the state in front of this block, kept for the tail
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) {
+        const int i = (t + e * TPC) * 4;
+        if (i < A.d) st4(snap + i, vp[e]);
+      }
+      snap_pos = jb - 1;
+    }
     for (int j = jb; j <= je; ++j) {
       const int k = nb + j - 1;
       const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
       const float inv_s = 1.0f / sk, cs = ck * inv_s;
       const float* wj = (j < Lt) ? A.X + (size_t)(r0 + j) * A.d : A.T + cb;
       const float* dq = A.Dq + (size_t)(r0 + j - 1) * A.d;
-      float4 vj[EPT], vq[EPT];
+      float4 vj[REGEN ? 1 : EPT], vq[EPT];
 #pragma unroll
       for (int e = 0; e < EPT; ++e) {
         const int i = (t + e * TPC) * 4;
-        vj[e] = (i < A.d) ? ld4(wj + i) : zero4;
+        if (!REGEN) vj[REGEN ? 0 : e] = (i < A.d) ? ld4(wj + i) : zero4;
         vq[e] = (i < A.d) ? ld4(dq + i) : zero4;
         if (A.Dp && i < A.d) vc[e] = ld4(A.Dp + (size_t)(r0 + j - 1) * A.d + i);   // independent draft model
       }
@@ -718,18 +744,23 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t)
       double p1 = 0.0, p2 = 0.0;
 #pragma unroll
       for (int e = 0; e < EPT; ++e) {
+        // the drafted state W_j: read back, or made again from W_{j-1}, the carried output and the
+        // chain's noise (the draft kernel's own operations, hence its bits)
+        const float4 w = REGEN ? draft_step4(vp[e], vc[e], normal4(A.seed, kStreamDraft, bg, (uint32_t)k, (uint32_t)(t + e * TPC)),
+                                             ak, ck, sk)
+                               : vj[REGEN ? 0 : e];
         if ((t + e * TPC) * 4 < A.d) {
           float D, Z;
-          delta_z(vp[e].x, vj[e].x, vq[e].x, vc[e].x, ak, ck, cs, inv_s, D, Z);
+          delta_z(vp[e].x, w.x, vq[e].x, vc[e].x, ak, ck, cs, inv_s, D, Z);
           p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
-          delta_z(vp[e].y, vj[e].y, vq[e].y, vc[e].y, ak, ck, cs, inv_s, D, Z);
+          delta_z(vp[e].y, w.y, vq[e].y, vc[e].y, ak, ck, cs, inv_s, D, Z);
           p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
-          delta_z(vp[e].z, vj[e].z, vq[e].z, vc[e].z, ak, ck, cs, inv_s, D, Z);
+          delta_z(vp[e].z, w.z, vq[e].z, vc[e].z, ak, ck, cs, inv_s, D, Z);
           p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
-          delta_z(vp[e].w, vj[e].w, vq[e].w, vc[e].w, ak, ck, cs, inv_s, D, Z);
+          delta_z(vp[e].w, w.w, vq[e].w, vc[e].w, ak, ck, cs, inv_s, D, Z);
           p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
         }
-        vp[e] = vj[e];
+        vp[e] = w;
       }
       p1 = warp_sum(p1);
       p2 = warp_sum(p2);
@@ -812,11 +843,13 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t)
         for (int e = 0; e < EPT; ++e) {
           const int i = (t + e * TPC) * 4;
           if (i < A.d) {
-            st4(A.Y + cb + i, ld4(A.T + cb + i));
+            st4(A.Y + cb + i, REGEN ? vp[e] : ld4(A.T + cb + i));   // REGEN: every block ran, vp holds W_Lt
             float4 q = ld4(A.Dq + (size_t)(r0 + Lt - 1) * A.d + i);
             if (A.raw_ce) {
               const float2 ce = __ldg(A.raw_ce + nb + Lt - 1);
-              q = affine_row4(ce.x, ce.y, q, ld4(A.X + (size_t)(r0 + Lt - 1) * A.d + i));
+              const float4 x = REGEN ? redraft4(A, ld4(snap + i), vc[e], bg, nb, snap_pos, Lt - 1, (uint32_t)(t + e * TPC))
+                                     : ld4(A.X + (size_t)(r0 + Lt - 1) * A.d + i);
+              q = affine_row4(ce.x, ce.y, q, x);
             }
             st4(A.Dc + cb + i, q);
           }
@@ -842,20 +875,23 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t)
   for (int e = 0; e < EPT; ++e) {
     const int i = (t + e * TPC) * 4;
     if (i < A.d) {
-      const float4 p = ld4(wp + i), w = ld4(wj + i);
+      // REGEN: the first rejection lies in the last block read, whose entry state is in snap
+      const float4 p = REGEN ? redraft4(A, ld4(snap + i), vc[e], bg, nb, snap_pos, jstar - 1, (uint32_t)(t + e * TPC)) : ld4(wp + i);
+      const float4 w = REGEN ? draft_step4(p, vc[e], normal4(A.seed, kStreamDraft, bg, (uint32_t)k, (uint32_t)(t + e * TPC)), ak, ck, sk)
+                             : ld4(wj + i);
       float4 q = ld4(dq + i);
       if (A.raw_ce) {
         const float2 ce = __ldg(A.raw_ce + k);
         q = affine_row4(ce.x, ce.y, q, p);
       }
-      const float4 c4 = A.Dp ? ld4(A.Dp + (size_t)(r0 + jstar - 1) * A.d + i) : vc[e];
+      const float4 c4 = (!REGEN && A.Dp) ? ld4(A.Dp + (size_t)(r0 + jstar - 1) * A.d + i) : vc[e];
       float4 o;
       float D, Z;
       delta_z(p.x, w.x, q.x, c4.x, ak, ck, cs, inv_s, D, Z); o.x = reflect_elem(p.x, q.x, Z, D, ak, ck, sk, coef);
       delta_z(p.y, w.y, q.y, c4.y, ak, ck, cs, inv_s, D, Z); o.y = reflect_elem(p.y, q.y, Z, D, ak, ck, sk, coef);
       delta_z(p.z, w.z, q.z, c4.z, ak, ck, cs, inv_s, D, Z); o.z = reflect_elem(p.z, q.z, Z, D, ak, ck, sk, coef);
       delta_z(p.w, w.w, q.w, c4.w, ak, ck, cs, inv_s, D, Z); o.w = reflect_elem(p.w, q.w, Z, D, ak, ck, sk, coef);
-      st4(wj + i, o);
+      if (!REGEN) st4(wj + i, o);
       if (fa) {                                          // the reflected state is the next state; its target row carries on
         st4(A.Y + cb + i, o);
         st4(A.Dc + cb + i, q);
@@ -868,13 +904,14 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t)
   }
 }
 
-template <int TPC, int EPT>
+template <int TPC, int EPT, bool REGEN>
 __global__ void __launch_bounds__(TPC > kBlock ? TPC : kBlock) k_verify_reg(WinArgs A) {
+  extern __shared__ __align__(16) float s_snap[];        // REGEN: d floats, the chain's state in front of the current block
   constexpr int kThreadsPerCta = TPC > kBlock ? TPC : kBlock;
   constexpr int kChains = kThreadsPerCta / TPC;
   const int s = blockIdx.x * kChains + threadIdx.x / TPC, t = threadIdx.x % TPC;
   const int n_active = A.ctl[kCtlNActive];
-  if (s < n_active) verify_reg_chain<TPC, EPT>(A, s, t);
+  if (s < n_active) verify_reg_chain<TPC, EPT, REGEN>(A, s, t, s_snap);
   if (A.fuse_advance) window_tail(A, n_active);
 }
 
@@ -1028,6 +1065,28 @@ cudaError_t launch_picard_draft(const WinArgs& A, int ub, cudaStream_t st) {
   SDS_DISPATCH(k_picard_draft, A, ub, st);
   return cudaGetLastError();
 }
+// one chain per CTA; with regenerated drafts the CTA keeps d floats of shared memory
+template <int TPC, int EPT>
+cudaError_t launch_verify_reg(const WinArgs& A, int chains, cudaStream_t st) {
+  if (!A.regen) {
+    k_verify_reg<TPC, EPT, false><<<chains, TPC, 0, st>>>(A);
+    return cudaGetLastError();
+  }
+  const size_t smem = (size_t)A.d * sizeof(float);
+  if (smem + 2 * kMaxL * (TPC / 32) * sizeof(double) + 64 > 48 * 1024) {   // the kernel's own shared arrays count too
+    const cudaError_t e = cudaFuncSetAttribute(k_verify_reg<TPC, EPT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  k_verify_reg<TPC, EPT, true><<<chains, TPC, smem, st>>>(A);
+  return cudaGetLastError();
+}
+
+// whether launch_verify may regenerate the drafted states instead of reading them (a chain per CTA,
+// frozen drafter, plain accept test; the caller also needs the advance step inside the kernel)
+bool verify_can_regen(const WinArgs& A) {
+  return !A.Q && !A.mean_rows && !A.Dp && vec4_ok(A.d) && A.d > 256 && A.d <= 16384 && A.mode == 0;
+}
+
 // whether launch_verify takes the register-resident kernel (the one that also reads rows kept raw)
 bool verify_reads_raw_rows(const WinArgs& A) { return !A.Q && !A.mean_rows && !A.Dp && vec4_ok(A.d) && A.d <= 16384; }
 
@@ -1056,15 +1115,15 @@ cudaError_t launch_verify(const WinArgs& A, int ub, cudaStream_t st) {
   }
   if (vec4_ok(A.d)) {
     if (A.d <= 256) {
-      k_verify_reg<32, 2><<<blocks_for(chains, 32), kBlock, 0, st>>>(A);
+      k_verify_reg<32, 2, false><<<blocks_for(chains, 32), kBlock, 0, st>>>(A);
       return cudaGetLastError();
     }
-    if (A.d <= 1024) { k_verify_reg<256, 1><<<chains, 256, 0, st>>>(A); return cudaGetLastError(); }
-    if (A.d <= 2048) { k_verify_reg<256, 2><<<chains, 256, 0, st>>>(A); return cudaGetLastError(); }
-    if (A.d <= 3072) { k_verify_reg<256, 3><<<chains, 256, 0, st>>>(A); return cudaGetLastError(); }
-    if (A.d <= 4096) { k_verify_reg<512, 2><<<chains, 512, 0, st>>>(A); return cudaGetLastError(); }
-    if (A.d <= 8192) { k_verify_reg<1024, 2><<<chains, 1024, 0, st>>>(A); return cudaGetLastError(); }
-    if (A.d <= 16384) { k_verify_reg<1024, 4><<<chains, 1024, 0, st>>>(A); return cudaGetLastError(); }
+    if (A.d <= 1024) return launch_verify_reg<256, 1>(A, chains, st);
+    if (A.d <= 2048) return launch_verify_reg<256, 2>(A, chains, st);
+    if (A.d <= 3072) return launch_verify_reg<256, 3>(A, chains, st);
+    if (A.d <= 4096) return launch_verify_reg<512, 2>(A, chains, st);
+    if (A.d <= 8192) return launch_verify_reg<1024, 2>(A, chains, st);
+    if (A.d <= 16384) return launch_verify_reg<1024, 4>(A, chains, st);
   }
   SDS_DISPATCH(k_verify, A, ub, st);
   return cudaGetLastError();

@@ -754,9 +754,11 @@ def test_early_exit_run_matches_oracle():
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("d,L,B,mode", [(64, 8, 70, 0), (1024, 12, 40, 0), (3072, 8, 24, 1), (4096, 16, 12, 0), (16384, 5, 6, 0)])
+@pytest.mark.parametrize("d,L,B,mode", [(64, 8, 70, 0), (1024, 12, 40, 0), (2048, 7, 9, 0), (3072, 8, 24, 1), (3072, 8, 24, 0), (4096, 16, 12, 0), (8192, 6, 5, 0),
+                          (16384, 5, 6, 0)])
 def test_sample_all_with_fused_advance_equals_the_stepwise_calls(d, L, B, mode):
-    """sds_sample_all (verify kernel advancing its chains, early exit on) against an explicit
+    """sds_sample_all (verify kernel advancing its chains, early exit on, drafted states drawn again
+    rather than read where d > 256 and the carried output is the drafter) against an explicit
     draft / verify / advance loop, and against the same run with the advance kernel: same bits."""
     w = wl.WORKLOADS["cfg2"].scaled(B=B, d=d, K=3 * L + 7, L=L)
     gp = w.gmm_params(d=d, ncomp=8)
@@ -764,6 +766,9 @@ def test_sample_all_with_fused_advance_equals_the_stepwise_calls(d, L, B, mode):
     s.set_option(s.OPT_WHOLE_CHAIN_KERNEL, 0)
     got = [x.cpu().numpy() for x in s.sample_all()]
     windows_fused = int(s.get(sb.GET_CTL)[2])
+    s.set_option(s.OPT_REGEN_DRAFTS, 0)                    # fused advance with the drafted states read back
+    mid = [x.cpu().numpy() for x in s.sample_all()]
+    assert all(np.array_equal(x, y) for x, y in zip(got, mid))
     s.set_option(s.OPT_FUSE_ADVANCE, 0)
     ref = [x.cpu().numpy() for x in s.sample_all()]
     assert all(np.array_equal(x, y) for x, y in zip(got, ref))

@@ -169,22 +169,22 @@ def test_bounded_wait_runs_out_and_reports():
 
 @pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4", "cfg5"])
 def test_full_size_runs_agree_bitwise_across_kernel_options(name):
-    """At the benchmark sizes: the verify kernel that exits early and advances its chains, the
-    CTA-pair GEMM and the whole-chain kernel change how the work is done, not one bit of the result,
-    and a repeated run reproduces itself."""
+    """At the benchmark sizes: the verify kernel that exits early, advances its chains and draws the
+    drafted states again instead of reading them, the CTA-pair GEMM and the whole-chain kernel change
+    how the work is done, not one bit of the result, and a repeated run reproduces itself."""
     import torch
     w = wl.WORKLOADS[name]
     s = sds.sampler_for(w)
     ref = None
-    for fuse, early, pair, whole, raw in [(1, 1, 1, 1, 1), (1, 1, 1, 1, 1), (0, 1, 1, 1, 1), (1, 0, 1, 1, 1), (1, 1, 1, 1, 0),
-                                         (0, 0, 0, 0, 0)]:
+    for fuse, early, pair, whole, raw, regen in [(1, 1, 1, 1, 1, 1), (1, 1, 1, 1, 1, 1), (1, 1, 1, 1, 1, 0), (0, 1, 1, 1, 1, 1),
+                                                (1, 0, 1, 1, 1, 1), (1, 1, 1, 1, 0, 1), (0, 0, 0, 0, 0, 0)]:
         s.set_option(s.OPT_FUSE_ADVANCE, fuse); s.set_option(s.OPT_VERIFY_EARLY_EXIT, early)
         s.set_option(s.OPT_GEMM_PAIR, pair); s.set_option(s.OPT_WHOLE_CHAIN_KERNEL, whole)
-        s.set_option(s.OPT_RAW_ROWS, raw)
+        s.set_option(s.OPT_RAW_ROWS, raw); s.set_option(s.OPT_REGEN_DRAFTS, regen)
         got = [x.clone() for x in s.sample_all()]
         if ref is None:
             ref = got
             assert torch.isfinite(ref[0]).all()
         else:
-            assert all(torch.equal(a, b) for a, b in zip(ref, got)), (fuse, early, pair, whole, raw)
+            assert all(torch.equal(a, b) for a, b in zip(ref, got)), (fuse, early, pair, whole, raw, regen)
     s.close()
