@@ -33,6 +33,10 @@ import workloads as wl  # noqa: E402
 METRIC = "accepted_chain_steps_per_sec"
 UNIT = "chain-steps/s"
 FP32_LANES_PER_SM, SMS = 128, 148
+# DRAM bytes (read + written) of one launch of the dominant kernel, from the profiler's counters of that
+# kernel as it stands, at the workload's own size (profiles/k_fused_small_cfg2.md). An entry goes back to
+# None when its kernel's source changes. Keyed by (workload, variant, kernel kind).
+CAPTURED_TRAFFIC = {("cfg2", "default", "fused"): 82176.0}
 
 
 def peaks():
@@ -500,7 +504,8 @@ def run_gpu(args, w):
         peak = SMS * FP32_LANES_PER_SM * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
         achieved, unit = per_launch / avg_s / 1e12, "TFLOP/s"
     roofline = {"kernel": dom, "bound": "tensor" if bound == "tensor_split" else bound, "achieved": achieved, "peak": peak, "unit": unit,
-                "frac": achieved / peak, "traffic": None,
+                "frac": achieved / peak,
+                "traffic": CAPTURED_TRAFFIC.get((w.name, args.variant, dom)) if not args.chains else None,
                 "peak_source": (pk["source"] + {"tensor": " (sustained bf16 GEMM)", "tensor_split": f" (sustained bf16 GEMM / {split_products:.2f}: 3 bf16 products per float product in the logits, 6 in the mixing, 3 for tiles of one-hot rows: {t_brief} of {t_full + t_brief} tiles)"}.get(bound, " (copy)")) if bound != "alu"
                 else "derived: 148 SMs x 128 fp32 lanes x 2 x max SM clock",
                 "avg_launch_us": avg_s * 1e6, "launches_per_step": dom_n / steps,
