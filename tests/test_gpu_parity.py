@@ -757,9 +757,10 @@ def test_early_exit_run_matches_oracle():
 @pytest.mark.parametrize("d,L,B,mode", [(64, 8, 70, 0), (1024, 12, 40, 0), (2048, 7, 9, 0), (3072, 8, 24, 1), (3072, 8, 24, 0), (4096, 16, 12, 0), (8192, 6, 5, 0),
                           (16384, 5, 6, 0)])
 def test_sample_all_with_fused_advance_equals_the_stepwise_calls(d, L, B, mode):
-    """sds_sample_all (verify kernel advancing its chains, early exit on, drafted states drawn again
-    rather than read where d > 256 and the carried output is the drafter) against an explicit
-    draft / verify / advance loop, and against the same run with the advance kernel: same bits."""
+    """sds_sample_all (verify kernel advancing its chains, early exit on) against an explicit
+    draft / verify / advance loop, and against the same run with the advance kernel: same bits.
+    (A float mixture reads the float rows, so the drafted states are read back here whatever the
+    option says; the bf16 targets' test covers the other path.)"""
     w = wl.WORKLOADS["cfg2"].scaled(B=B, d=d, K=3 * L + 7, L=L)
     gp = w.gmm_params(d=d, ncomp=8)
     s = sds.sampler_for(w, gmm=gp, seed=71, drafter_mode=mode)

@@ -188,3 +188,42 @@ def test_full_size_runs_agree_bitwise_across_kernel_options(name):
         else:
             assert all(torch.equal(a, b) for a, b in zip(ref, got)), (fuse, early, pair, whole, raw, regen)
     s.close()
+
+
+@pytest.mark.parametrize("kind,d,L,B", [("gmm", 512, 9, 21), ("gmm", 1536, 7, 13), ("mlp", 3072, 8, 10), ("gmm", 4096, 6, 9),
+                                         ("mlp", 8192, 5, 5), ("gmm", 16384, 6, 4)])
+def test_drafted_states_drawn_again_give_the_same_bits(kind, d, L, B):
+    """Targets that read only the bf16 rows (the MLP, the bf16 mixture): inside sds_sample_all the draft
+    kernel stores only those rows and verify runs the draft recurrence again from Y_n, the carried
+    output and the chain's noise. One case per verify kernel shape; windows whose first rejection
+    falls at every offset of a block of positions, windows that accept everything, a ragged last
+    window. Same bits as with the rows read back, as with the advance kernel, and as the step-wise calls."""
+    K = 3 * L + 4
+    if kind == "mlp":
+        w = wl.WORKLOADS["cfg3"].scaled(d=d, B=B, L=L, K=K, mlp_dims=[d, 256, d])
+        s = sds.sampler_for(w, mlp=w.mlp_params(), seed=81)
+    else:
+        w = wl.WORKLOADS["cfg4"].scaled(d=d, B=B, L=L, K=K)
+        s = sds.sampler_for(w, gmm=w.gmm_params(d=d, ncomp=128), seed=81)
+    got = [x.cpu().numpy() for x in s.sample_all()]
+    assert np.all(np.isfinite(got[0]))
+    windows = int(s.get(sb.GET_CTL)[2])
+    s.set_option(s.OPT_REGEN_DRAFTS, 0)
+    back = [x.cpu().numpy() for x in s.sample_all()]
+    assert all(np.array_equal(x, y) for x, y in zip(got, back))
+    assert windows == int(s.get(sb.GET_CTL)[2])
+    s.set_option(s.OPT_FUSE_ADVANCE, 0)
+    sep = [x.cpu().numpy() for x in s.sample_all()]
+    assert all(np.array_equal(x, y) for x, y in zip(got, sep))
+    s.reset()
+    na, advs = B, []
+    while na > 0:
+        n0 = s.get(sb.GET_N).copy()
+        s.draft(); s.verify_window(); na = s.advance()
+        advs.append(s.get(sb.GET_N) - n0)
+    assert np.array_equal(s.get(sb.GET_Y), got[0])
+    assert np.array_equal(s.get(sb.GET_NFE_CALLS), got[1]) and np.array_equal(s.get(sb.GET_NFE_ROWS), got[2])
+    adv = np.concatenate(advs)
+    if kind == "gmm":                                     # (the random network's drafts are rejected at once)
+        assert len(set(adv[adv > 0].tolist())) >= 3       # the windows did end at several different positions
+    s.close()
