@@ -230,7 +230,8 @@ int sds_sample_all(sds_ctx* ctx, float* out_dev, int32_t* nfe_calls_dev, int32_t
 #define SDS_OPT_GEMM_PAIR 3
 /* SDS_OPT_VERIFY_EARLY_EXIT (default 1): Algorithm 4 stops at the first rejection, so nothing after
  * it is needed. For d % 4 == 0, 256 < d <= 16384 (one CTA per chain) with the full-space test and a
- * frozen or independent drafter, verify takes the positions in blocks of two (four when d < 2048), decides a block's
+ * frozen or independent drafter, verify takes the positions in blocks of two (d >= 2048: the first position alone,
+ * then pairs) or four (d < 2048), decides a block's
  * accept tests before reading the next and skips every block after the one that holds the first
  * rejection. Decisions, first-reject indices, reflected states and counters are unchanged; the
  * diagnostic arrays (SDS_GET_S1, _S2, _ELL, _LOGU, bits of _ACCMASK) hold zeros for the skipped

@@ -16,8 +16,8 @@ struct WinArgs {
   const float2* raw_ce;  // non-NULL: Dq holds the mixing contraction's accumulators; the target output of row r
                          // (input X[r], step k = rowk[r]) is fma(C_k, Dq[r], E_k X[r]) with (C_k, E_k) = raw_ce[k]
   int fuse_advance;      // the verify kernel also advances its chain and the last CTA compacts (no advance launch)
-  int early_exit;        // verify stops reading a chain's window after the block of two (d >= 2048) or four positions
-                         // that holds its first rejection (large-d kernels only)
+  int early_exit;        // verify stops reading a chain's window after the block of positions that holds its first
+                         // rejection (d >= 2048: the first position, then pairs; below: fours; large-d kernels only)
   int regen;             // verify draws the drafted states again from Y_n, the carried output and the noise instead of
                          // reading them (needs fuse_advance; see verify_can_regen)
   int skip_x;            // the draft kernel stores only the bf16 copies of its rows (nothing reads the float rows)

@@ -711,8 +711,11 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t,
   uint32_t amask = 0u;
   bool frozen = false;
   int done = 0;                                          // positions evaluated so far
-  for (int jb = 1; jb <= Lt; jb += blk) {
-    const int je = min(Lt, jb + blk - 1);
+  // long rows: the first position is a block of its own (a chain whose first draft is rejected reads one
+  // position, not two)
+  const bool first_alone = early && A.d >= 2048;
+  for (int jb = 1, je; jb <= Lt; jb = je + 1) {
+    je = (first_alone && jb == 1) ? 1 : min(Lt, jb + blk - 1);
     double myS1 = 0.0, myS2 = 0.0;
     if (REGEN) {                                         // the state in front of this block, kept for the tail
 #pragma unroll
