@@ -1075,6 +1075,7 @@ cudaError_t launch_verify_reg(const WinArgs& A, int chains, cudaStream_t st) {
     k_verify_reg<TPC, EPT, false><<<chains, TPC, 0, st>>>(A);
     return cudaGetLastError();
   }
+  if (!A.fuse_advance) return cudaErrorInvalidValue;     // the regenerated states exist only in this kernel: it must advance
   const size_t smem = (size_t)A.d * sizeof(float);
   if (smem + 2 * kMaxL * (TPC / 32) * sizeof(double) + 64 > 48 * 1024) {   // the kernel's own shared arrays count too
     const cudaError_t e = cudaFuncSetAttribute(k_verify_reg<TPC, EPT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
