@@ -222,6 +222,7 @@ __global__ void __launch_bounds__(kBlock) k_draft(WinArgs A) {
         if (!A.skip_x) st4(A.X + ro, y);
         if (A.Xb) *reinterpret_cast<uint2*>(A.Xb + ro) = make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
         if (A.Xs) store_split2x4(A.Xs + ro, A.xs_plane, y);
+        if (A.skip_x && j == Lt - 1) break;            // W_Lt is no target input: verify makes it itself
         const int k = nb + j;
         const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
         const float4 xi = normal4(A.seed, kStreamDraft, bg, (uint32_t)k, (uint32_t)(i >> 2));
