@@ -881,8 +881,10 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t,
     if (i < A.d) {
       // REGEN: the first rejection lies in the last block read, whose entry state is in snap
       const float4 p = REGEN ? redraft4(A, ld4(snap + i), vc[e], bg, nb, snap_pos, jstar - 1, (uint32_t)(t + e * TPC)) : ld4(wp + i);
-      const float4 w = REGEN ? draft_step4(p, vc[e], normal4(A.seed, kStreamDraft, bg, (uint32_t)k, (uint32_t)(t + e * TPC)), ak, ck, sk)
-                             : ld4(wj + i);
+      // (when the rejected position is the last one read, its drafted state is still in registers)
+      const float4 w = !REGEN ? ld4(wj + i)
+                       : (jstar == done) ? vp[e]
+                       : draft_step4(p, vc[e], normal4(A.seed, kStreamDraft, bg, (uint32_t)k, (uint32_t)(t + e * TPC)), ak, ck, sk);
       float4 q = ld4(dq + i);
       if (A.raw_ce) {
         const float2 ce = __ldg(A.raw_ce + k);
