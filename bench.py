@@ -6,15 +6,19 @@ state and target call, then draft / batched target / verify / advance windows un
 has made its K transitions. The metric is accepted chain-steps per second (B*K per run; both
 accepted and reflected steps are valid target steps).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4] [--impl reference]
 
-Prints one JSON line (rank 0). N > 1 (under torch.distributed.run): chains are sharded across
-ranks by global chain id, no collective on the data path (weak scaling: B chains per rank).
+Prints one JSON line (rank 0). The default workload is the largest single-GPU configuration (cfg4:
+1024 chains of dimension 16384, 1024-component mixture on the tensor cores). N > 1: chains are sharded
+across ranks by global chain id, no collective on the data path (weak scaling: B chains per rank);
+started without a launcher, the script starts its own N ranks under torch.distributed.run. After the
+timed region the ranks gather the final samples and sum the counters (NCCL, off the timed path).
 --impl reference times the CPU oracle, as it stands, on a bounded sample of the same workload.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import subprocess
@@ -33,10 +37,32 @@ import workloads as wl  # noqa: E402
 METRIC = "accepted_chain_steps_per_sec"
 UNIT = "chain-steps/s"
 FP32_LANES_PER_SM, SMS = 128, 148
-# DRAM bytes (read + written) of one launch of the dominant kernel, from the profiler's counters of that
-# kernel as it stands, at the workload's own size (profiles/k_fused_small_cfg2.md). An entry goes back to
-# None when its kernel's source changes. Keyed by (workload, variant, kernel kind).
-CAPTURED_TRAFFIC = {("cfg2", "default", "fused"): 82176.0}
+DEFAULT_WORKLOAD = "cfg4"
+CSRC = os.path.join(ROOT, "paper_2501_05370_b200", "csrc")
+TRAFFIC_TABLE = os.path.join(ROOT, "profiles", "dram_traffic.md")
+
+
+def measured_traffic():
+    """DRAM bytes (read + written) and warp instructions per launch from the profiler captures listed
+    in the traffic table: rows `| workload | kernel kind | chains | DRAM bytes per launch | warp
+    instructions per launch | source file:hash | note |`. A capture is taken at a reduced number of
+    chains; every chain moves the same bytes, so a launch at B chains moves B / chains times as much.
+    A row whose source file no longer has the recorded hash describes a kernel that has changed since:
+    it is ignored (the figure is then null). Returns {(workload, kind): (chains, bytes, inst)}."""
+    out = {}
+    if not os.path.exists(TRAFFIC_TABLE):
+        return out
+    for ln in open(TRAFFIC_TABLE):
+        f = [x.strip() for x in ln.strip().strip("|").split("|")]
+        if len(f) < 6 or not f[2].isdigit():
+            continue
+        src, _, want = f[5].partition(":")
+        path = os.path.join(CSRC, src)
+        if not os.path.exists(path) or hashlib.sha256(open(path, "rb").read()).hexdigest()[:12] != want:
+            continue
+        num = lambda x: float(x) if x not in ("", "-") else None
+        out[(f[0], f[1])] = (int(f[2]), num(f[3]), num(f[4]))
+    return out
 
 
 def peaks():
@@ -108,7 +134,7 @@ def gpu_sampler(sds, w, variant: str, **kw):
     if variant == "tau2":
         s.set_temperature(2.0)
     if variant == "proj16":
-        s.set_projection(torch.from_numpy(sb.projection_basis(proj_matrix(w))).to(kw.get("device", "cuda:0")))
+        s.set_projection(torch.from_numpy(sds.projection_basis(proj_matrix(w))).to(kw.get("device", "cuda:0")))
     return s
 
 
@@ -142,7 +168,7 @@ def oracle_time(w, budget_s: float, min_chains: int = 1, first_chain: int = 0, v
     prefix of the chain, which the returned description says. Returns (chain_steps, seconds, text)."""
     o, den, a, c, sig = oracle_closure(w)
     t0 = time.perf_counter()
-    n, steps, Kp = 0, 0, min(w.K, 2 * w.L)
+    n, steps, Kp = 0, 0, min(w.K, w.L)           # at least one full window per chain
     prefix = False
     while True:
         t1 = time.perf_counter()
@@ -169,7 +195,7 @@ def oracle_plain_time(w, budget_s: float):
     for the saving in sequential target calls. Returns (chain_steps, seconds)."""
     o, den, a, c, sig = oracle_closure(w)
     t0 = time.perf_counter()
-    n, steps, Kp = 0, 0, min(w.K, 2 * w.L)
+    n, steps, Kp = 0, 0, min(w.K, w.L)
     while True:
         t1 = time.perf_counter()
         o.plain_chain(den, a[:Kp], c[:Kp], sig[:Kp], w.sample_seed, n, w.d)
@@ -300,31 +326,113 @@ class ClockSampler:
 # GPU arm
 # --------------------------------------------------------------------------------------------
 
-def algorithmic(kind: str, w, rows_per_step: float, windows_chains: float, launches: float):
-    """Algorithmic bytes or flops one average launch of `kind` must move / compute.
-    rows_per_step: target rows verified per step (sum of window lengths); windows_chains: chain-windows."""
-    d = w.d
-    if kind == "verify":        # two fp32 streams per verified chain-step (target output + drafted state)
-        return "hbm", 8.0 * d * rows_per_step / launches
-    if kind == "draft":         # read state + carried output, write the drafted rows
-        return "hbm", (8.0 * d * windows_chains + 4.0 * d * rows_per_step) / launches
-    if kind == "advance":
-        return "hbm", 16.0 * d * windows_chains / launches
-    if kind in ("denoise", "fused"):
-        if w.denoiser == "phi4":    # four neighbour differences, the site term, one fma per site
-            return "alu", 12.0 * d * (rows_per_step + w.B) / launches
-        if w.denoiser == "mlp":     # 2 * sum of layer products per row, bf16 tensor cores
-            per_row = 2.0 * sum(w.mlp_dims[i] * w.mlp_dims[i + 1] for i in range(len(w.mlp_dims) - 1))
-            return "tensor", per_row * (rows_per_step + w.B) / launches
-        per_row = 4.0 * w.gmm["ncomp"] * d      # logits + mixing contractions
-        if w.gmm.get("means_bf16"):
-            bound = "tensor"
-        elif kind == "denoise" and 32 < w.gmm["ncomp"] <= 1024 and w.gmm["ncomp"] % 128 == 0 and d % 128 == 0:
-            bound = "tensor_split"              # float operands as bf16 planes: 3 products (logits) + 6 (mixing)
+def run_counts(w, variant, calls_np, rows_np):
+    """(target rows of the windows, chain-windows) of one run, from the per-chain counters."""
+    B = len(calls_np)
+    if getattr(w, "drafter_mode", 0) == 1 or variant == "exact":
+        # drafter evaluated at Y_n: no initial call, two sequential calls per window (one for a last window of one row)
+        return float(rows_np.sum()), float(np.ceil(calls_np / 2.0).sum())
+    if variant == "independent":                       # no initial call, one target call per window
+        return float(rows_np.sum()), float(calls_np.sum())
+    if variant == "picard2":                           # initial call, then 2 draft calls + 1 verify call per window
+        cw = float(np.ceil((calls_np - 1) / 3.0).sum())
+        return float(w.L * cw), cw                     # rows of the verify calls (full windows assumed)
+    return float(rows_np.sum() - B), float(calls_np.sum() - B)   # the initial call is not a window
+
+
+def tensor_mixture(w):
+    return w.denoiser == "gmm" and (w.gmm.get("means_bf16") or
+                                    (32 < w.gmm["ncomp"] <= 1024 and w.gmm["ncomp"] % 128 == 0 and w.d % 128 == 0))
+
+
+def kernel_rooflines(w, variant, prof, steps, rows, cw, positions, pk, ctl, traffic, launch_shape):
+    """One roofline entry per kernel kind that ran in the timed region.
+
+    rows: target rows of the windows per run (sum of window lengths over chains and windows);
+    cw: chain-windows per run; positions: window positions whose accept test verify evaluated per run
+    (fewer than rows when it stops reading after the first rejection). Algorithmic bytes / flops are the
+    per-unit figures of the method (what any implementation must move or compute); `requested` is what
+    this implementation's kernels ask memory for."""
+    d, B = w.d, w.B
+    hbm, tens = pk["hbm_gbs"], pk["bf16_sustained"]
+    alu_peak = SMS * FP32_LANES_PER_SM * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
+    kinds = {k: v for k, v in prof.items() if v[1] > 0 and v[0] > 0}
+    total_ms = sum(v[0] for v in kinds.values())
+    bf16_rows = w.denoiser == "mlp" or (w.denoiser == "gmm" and w.gmm.get("means_bf16"))
+    split = tensor_mixture(w) and not w.gmm.get("means_bf16")
+    regen, cached = launch_shape.get("regen", False), launch_shape.get("noise_cache", False)
+    out = []
+    for kind, (ms, n) in sorted(kinds.items(), key=lambda kv: -kv[1][0]):
+        if kind in ("init", "aux"):
+            continue
+        per_run_launches = n / steps
+        avg_s = ms / n * 1e-3
+        e = {"kernel": kind, "launches_per_step": per_run_launches, "avg_launch_us": avg_s * 1e6,
+             "ms_per_step": ms / steps, "share_of_kernel_time": ms / max(total_ms, 1e-9)}
+        if kind in ("denoise", "fused", "draft_model"):
+            if w.denoiser == "phi4":
+                bound, per_run = "alu", 12.0 * d * (rows + B)
+            elif w.denoiser == "mlp":
+                bound, per_run = "tensor", 2.0 * sum(w.mlp_dims[i] * w.mlp_dims[i + 1] for i in range(len(w.mlp_dims) - 1)) * (rows + B)
+            else:
+                per_run = 4.0 * w.gmm["ncomp"] * d * (rows + B)
+                bound = "tensor" if (kind == "denoise" and tensor_mixture(w)) else "alu"
+            if kind == "draft_model":
+                bound, per_run = "alu", 4.0 * max(1, w.gmm["ncomp"] // 2) * d * rows
+            peak, unit, src = (tens, "TFLOP/s", pk["source"] + " (sustained bf16 GEMM)") if bound == "tensor" else \
+                              (alu_peak, "TFLOP/s", "derived: 148 SMs x 128 fp32 lanes x 2 x max SM clock")
+            if bound == "tensor" and split:
+                # float operands as bf16 planes: 3 bf16 products per float product in the logits, 6 in the
+                # mixing (3 for tiles whose responsibilities need only their first plane; the library counts both)
+                t_full, t_brief = int(ctl[8]), int(ctl[9])
+                mix = (6.0 * t_full + 3.0 * t_brief) / max(1, t_full + t_brief)
+                peak = tens / ((3.0 + mix) / 2.0)
+                src = pk["source"] + f" (sustained bf16 GEMM / {(3.0 + mix) / 2.0:.2f} bf16 products per float product; {t_brief} of {t_full + t_brief} mixing tiles one-hot)"
+            ach = per_run / (ms / steps * 1e-3) / 1e12
+            e.update(bound=bound, achieved=ach, peak=peak, unit=unit, frac=ach / peak, peak_source=src,
+                     algorithmic_per_launch=per_run / per_run_launches)
         else:
-            bound = "alu"
-        return bound, per_row * (rows_per_step + w.B) / launches
-    return "hbm", 0.0
+            if kind == "verify":
+                per_run = 8.0 * d * rows                         # two float streams per window position
+                # requested: per evaluated position the target row (and the drafted state unless it is made
+                # again in registers or read from the noise cache), per chain-window the state, the carried
+                # output, the reflected row's inputs again and the two rows the advance step writes
+                per_pos = 4.0 * d if regen else 8.0 * d
+                req = per_pos * positions + (8.0 * d + 4.0 * d + 8.0 * d) * cw
+                e.update(positions_evaluated_per_step=positions, requested_bytes_per_launch=req / per_run_launches,
+                         requested_achieved=req / (ms / steps * 1e-3) / 1e9,
+                         requested_frac=req / (ms / steps * 1e-3) / 1e9 / hbm)
+            elif kind == "draft":
+                rows_w = 4.0 * d * rows + (2.0 * d * rows if bf16_rows else 0.0) + (4.0 * d * rows if split else 0.0)
+                per_run = 8.0 * d * cw + rows_w
+                # stored by this implementation: the float rows are skipped where nothing reads them
+                moved = 8.0 * d * cw + (2.0 * d * (rows - cw) if (regen and bf16_rows) else rows_w)
+                e.update(requested_bytes_per_launch=moved / per_run_launches,
+                         requested_achieved=moved / (ms / steps * 1e-3) / 1e9,
+                         requested_frac=moved / (ms / steps * 1e-3) / 1e9 / hbm)
+            elif kind == "advance":
+                per_run = 16.0 * d * cw
+            elif kind == "softmax":
+                nc = w.gmm["ncomp"] if w.denoiser == "gmm" else 0
+                per_run = (4.0 + (6.0 if split else 2.0)) * nc * (rows + B)   # logits in, responsibilities out
+            else:
+                per_run = 0.0
+            ach = per_run / (ms / steps * 1e-3) / 1e9
+            e.update(bound="hbm", achieved=ach, peak=hbm, unit="GB/s", frac=ach / hbm, peak_source=pk["source"] + " (copy)",
+                     algorithmic_per_launch=per_run / per_run_launches)
+        t = traffic.get((w.name, kind))
+        e["traffic"] = None
+        if t is not None and t[1] is not None:
+            e["traffic"] = t[1] * B / t[0]                       # captured at t[0] chains; traffic grows with the chains
+            e["traffic_over_algorithmic"] = e["traffic"] / max(e["algorithmic_per_launch"], 1.0) if e["bound"] == "hbm" else None
+        if t is not None and t[2] is not None:
+            # issue bound: warp instructions per launch against one instruction per cycle and scheduler
+            inst = t[2] * B / t[0]
+            slots = SMS * 4 * pk["sm_max_mhz"] * 1e6
+            e["issue"] = {"warp_instructions_per_launch": inst, "issue_slots_per_s": slots,
+                          "frac_of_issue_peak": inst / avg_s / slots}
+        out.append(e)
+    return out
 
 
 def acceptance_by_step(sds, w, dev, variant: str = "default", chains: int = 64, bins: int = 10):
@@ -360,28 +468,136 @@ def acceptance_by_step(sds, w, dev, variant: str = "default", chains: int = 64, 
             "rate": [round(float(a / t), 4) if t > 0 else None for a, t in zip(accepted, tested)]}
 
 
+def quick_config(sds, name, dev, steps: int = 5, warmup: int = 2):
+    """ms per run, chain-steps/s and the counters of another workload, in the same process."""
+    import torch
+    w = wl.WORKLOADS[name]
+    s = gpu_sampler(sds, w, "default", device=dev)
+    out = torch.empty((w.B, w.d), dtype=torch.float32, device=dev)
+    calls = torch.empty((w.B,), dtype=torch.int32, device=dev)
+    rows = torch.empty((w.B,), dtype=torch.int32, device=dev)
+    st = torch.cuda.current_stream()
+    for _ in range(warmup):
+        s.sample_all(out, calls, rows)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(st)
+    for _ in range(steps):
+        s.sample_all(out, calls, rows)
+    e1.record(st)
+    e1.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    c, r = calls.cpu().numpy().astype(np.int64), rows.cpu().numpy().astype(np.int64)
+    rws, cw = run_counts(w, "default", c, r)
+    s.close()
+    del out
+    torch.cuda.empty_cache()
+    return {"B": w.B, "d": w.d, "L": w.L, "K": w.K, "ms_per_run": ms, "chain_steps_per_s": w.B * w.K / (ms * 1e-3),
+            "mean_target_calls": float(c.mean()), "mean_target_rows": float(r.mean()),
+            "mean_advance": float(w.K * w.B / max(cw, 1.0)), "steps_timed": steps}
+
+
+def phi4_energies(x, side, beta):
+    """Lattice energy of each row of x [n, side*side] with every neighbouring pair counted once
+    (free boundaries), and the same with each pair counted from both of its sites (twice)."""
+    g = np.asarray(x, np.float64).reshape(-1, side, side)
+    site = ((g * g - 1.0) ** 2).sum(axis=(1, 2))
+    pairs = (np.diff(g, axis=1) ** 2).sum(axis=(1, 2)) + (np.diff(g, axis=2) ** 2).sum(axis=(1, 2))
+    return 0.5 * beta * pairs + site, beta * pairs + site
+
+
+def phi4_energy_statistic(sds, w, dev, last: int = 500):
+    """Appendix K reports the mean and standard deviation of the energy over the last 500 simulated
+    samples of 500 runs, for the plain Langevin chain and for speculative sampling. Here: every chain is
+    run to step K - last, then stepped window by window to the end while every accepted state (the
+    samples X_{K-last+1} .. X_K) is read back; the plain chain is the same with window 1. Both energy
+    conventions are reported (the sampler itself uses each pair once)."""
+    import torch
+    from paper_2501_05370_b200 import binding as sb
+    res = {}
+    for label, L in (("speculative", w.L), ("plain", 1)):
+        head = w.scaled(K=w.K - last, L=L)
+        s = gpu_sampler(sds, head, "default", device=dev)
+        Y = s.sample_all()[0].clone()
+        s.close()
+        full = w.scaled(L=L)
+        s = gpu_sampler(sds, full, "default", device=dev)
+        s.reset()
+        s.set_state(Y=Y, n=torch.full((w.B,), w.K - last, dtype=torch.int32, device=dev))
+        e1, e2, na = [], [], w.B
+        while na > 0:
+            n0 = s.get(sb.GET_N).astype(np.int64)
+            act, rowoff = s.get(sb.GET_ACT), s.get(sb.GET_ROWOFF)
+            nact = int(s.get(sb.GET_CTL)[0])
+            s.draft(); s.verify_window()
+            X, T, js = s.get(sb.GET_X), s.get(sb.GET_TAIL), s.get(sb.GET_JSTAR).astype(np.int64)
+            for si in range(nact):
+                b = int(act[si]); r0 = int(rowoff[si]); Lt = min(L, w.K - int(n0[b]))
+                adv = min(int(js[b]), Lt)
+                states = [X[r0 + j] if j < Lt else T[b] for j in range(1, adv + 1)]   # W_1 .. W_adv (the last one reflected or accepted)
+                a, b2 = phi4_energies(np.stack(states), w.phi4["side"], w.phi4["beta"])
+                e1 += a.tolist(); e2 += b2.tolist()
+            na = s.advance()
+        s.close()
+        e1, e2 = np.array(e1), np.array(e2)
+        res[label] = {"samples": int(e1.size), "mean_pairs_once": float(e1.mean()), "std_pairs_once": float(e1.std()),
+                      "mean_pairs_twice": float(e2.mean()), "std_pairs_twice": float(e2.std())}
+    res["paper"] = {"plain": [62.27, 13.32], "speculative": [65.90, 12.48],
+                    "note": "Appendix K table; the paper does not say how the pairs of its reported energy are counted"}
+    return res
+
+
+def independent_cost_ratio(sds, w, dev, prof, steps, rows, cw, ms_per_step):
+    """Section 4.1, proposition on the average cost ratio: with C_p the cost of one draft-model call
+    (one position of all chains) and C_q the cost of one batched target call, the original sampler
+    costs K C_q and the speculative one (K / E[adv]) (L C_p + C_q): ratio E[adv] / (1 + L C_p / C_q).
+    C_p and C_q are the measured kernel times per call; the measured ratio is the plain chain's time
+    (window 1, target at every step: one call on B rows per step) over the speculative run's."""
+    import torch
+    dm, dn = prof.get("draft_model", (0.0, 0)), prof.get("denoise", (0.0, 0))
+    sm = prof.get("softmax", (0.0, 0))
+    if dm[1] == 0 or dn[1] == 0:
+        return None
+    windows = cw / w.B                                   # windows per run (every chain takes part in each)
+    calls_q = max(1.0, float(np.ceil(dn[1] / steps / max(1.0, (dn[1] / steps) / max(windows, 1.0)))))
+    c_p = dm[0] / steps / (windows * w.L)                # ms per draft-model call
+    c_q = (dn[0] + sm[0]) / steps / windows              # ms per batched target call
+    adv = w.K * w.B / max(cw, 1.0)
+    from paper_2501_05370_b200 import binding as sb
+    plain = sds.sampler_for(w.scaled(L=1), drafter_mode=sb.SDS_FROZEN_EXACT, device=dev)
+    plain.set_option(plain.OPT_WHOLE_CHAIN_KERNEL, 0)
+    plain.sample_all()
+    st = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(st); plain.sample_all(); e1.record(st); e1.synchronize()
+    ms_plain = e0.elapsed_time(e1)
+    plain.close()
+    return {"C_p_ms_per_draft_call": c_p, "C_q_ms_per_target_call": c_q, "C_p_over_C_q": c_p / c_q, "L": w.L,
+            "mean_advance": adv, "predicted_cost_ratio": adv / (1.0 + w.L * c_p / c_q),
+            "plain_chain_ms": ms_plain, "speculative_ms": ms_per_step, "measured_cost_ratio": ms_plain / ms_per_step,
+            "note": "window kernels on both sides; the proposition counts a batched call as one unit whatever its "
+                    "row count, while on the GPU a call on B*L rows costs more than a call on B rows"}
+
+
 def run_gpu(args, w):
     import torch
-    import torch.distributed as dist
     import paper_2501_05370_b200 as sds
+    from paper_2501_05370_b200 import binding as sb
+    from paper_2501_05370_b200 import sharding
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, local, world = sharding.dist_env()
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device (no CPU fallback); use --impl reference for the oracle")
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(dev))
+    dist = sharding.init_process_group("nccl", dev)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        sharding.barrier(dist)
         torch.cuda.synchronize()
 
-    from paper_2501_05370_b200 import sharding
     s = gpu_sampler(sds, w, args.variant, chain_id_offset=sharding.weak_offset(rank, w.B), device=dev)
+    if args.variant == "independent":
+        s.set_option(s.OPT_WHOLE_CHAIN_KERNEL, 0)      # the cost ratio is about the draft-model and target kernels
     B, d, K = w.B, w.d, w.K
     out = torch.empty((B, d), dtype=torch.float32, device=dev)
     calls = torch.empty((B,), dtype=torch.int32, device=dev)
@@ -446,6 +662,7 @@ def run_gpu(args, w):
     if clk is not None:
         clk["source"] = clk_source
     calls_np, rows_np = calls.cpu().numpy().astype(np.int64), rows.cpu().numpy().astype(np.int64)
+    ctl = s.get(sb.GET_CTL)
 
     # the same metric through the host-buffer entry point
     for _ in range(min(args.warmup, 3)):
@@ -454,9 +671,17 @@ def run_gpu(args, w):
     ms_e2e = timed(e2e_step, args.steps)
     barrier()
 
-    ms_total, ms_e2e = sharding.max_over_ranks([ms_total, ms_e2e], dist if world > 1 else None, dev)
+    # end of the run: every rank's samples in global chain order and the counters summed (off the timed path)
+    all_samples, tot_calls, tot_rows = sharding.gather_results(out, calls, rows, dist)
+    gathered = {"samples_shape": list(all_samples.shape), "all_finite": bool(torch.isfinite(all_samples).all().item()),
+                "target_calls_all_chains": tot_calls, "target_rows_all_chains": tot_rows,
+                "collectives": "none" if world == 1 else "one all-gather of the [B, d] samples, one all-reduce of the counters (NCCL)"}
+    del all_samples
+
+    ms_total, ms_e2e = sharding.max_over_ranks([ms_total, ms_e2e], dist, dev)
     if rank != 0:
-        if world > 1:
+        s.close()
+        if dist is not None:
             dist.destroy_process_group()
         return
 
@@ -465,54 +690,36 @@ def run_gpu(args, w):
     ms_per_step = ms_total / steps
     value = world * B * K / (ms_per_step * 1e-3)
     e2e_value = world * B * K / (ms_e2e / steps * 1e-3)
-    if getattr(w, "drafter_mode", 0) == 1 or args.variant == "exact":
-        # drafter evaluated at Y_n: no initial call, two sequential calls per window (one for a last window of one row)
-        rows_per_step = float(rows_np.sum())
-        windows_chains = float(np.ceil(calls_np / 2.0).sum())
-    elif args.variant == "independent":                       # no initial call, one target call per window
-        rows_per_step = float(rows_np.sum())
-        windows_chains = float(calls_np.sum())
-    elif args.variant == "picard2":                           # initial call, then 2 draft calls + 1 verify call per window
-        windows_chains = float(np.ceil((calls_np - 1) / 3.0).sum())
-        rows_per_step = float(w.L * windows_chains)           # rows of the verify calls (full windows assumed)
-    else:
-        rows_per_step = float(rows_np.sum() - B)              # rows verified (the initial call is not a window)
-        windows_chains = float(calls_np.sum() - B)
-    kinds = {k: v for k, v in prof.items() if v[1] > 0}
-    dom = max(kinds, key=lambda k: kinds[k][0]) if kinds else "fused"
-    dom_ms, dom_n = kinds.get(dom, (ms_total, steps))
-    denoise_launch_groups = {"mlp": len(w.mlp_dims) - 1}.get(w.denoiser, 3 if (w.denoiser == "gmm" and w.gmm.get("means_bf16")) else 1)
-    from paper_2501_05370_b200 import binding as sb
-    split_products, t_full, t_brief = 4.5, 0, 0
-    bound, per_launch = algorithmic(dom, w, rows_per_step, windows_chains, dom_n / steps)
-    avg_s = dom_ms / max(dom_n, 1) * 1e-3
-    if bound == "hbm":
-        achieved, peak, unit = per_launch / avg_s / 1e9, pk["hbm_gbs"], "GB/s"
-    elif bound == "tensor":
-        achieved, peak, unit = per_launch / avg_s / 1e12, pk["bf16_sustained"], "TFLOP/s"
-    elif bound == "tensor_split":
-        # float-equivalent flops: the logits contraction costs 3 bf16 products per float product, the
-        # mixing contraction 6 (or 3, see below), and the two contractions are the same size
-        # where a tile of responsibilities needs only its first plane (one-hot rows) the mixing contraction
-        # runs 3 products instead of 6; the library counts both kinds of tile
-        ctl = s.get(sb.GET_CTL)
-        t_full, t_brief = int(ctl[8]), int(ctl[9])
-        mix_products = (6.0 * t_full + 3.0 * t_brief) / max(1, t_full + t_brief)
-        split_products = (3.0 + mix_products) / 2.0
-        achieved, peak, unit = per_launch / avg_s / 1e12, pk["bf16_sustained"] / split_products, "TFLOP/s"
-    else:
-        peak = SMS * FP32_LANES_PER_SM * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
-        achieved, unit = per_launch / avg_s / 1e12, "TFLOP/s"
-    roofline = {"kernel": dom, "bound": "tensor" if bound == "tensor_split" else bound, "achieved": achieved, "peak": peak, "unit": unit,
-                "frac": achieved / peak,
-                "traffic": CAPTURED_TRAFFIC.get((w.name, args.variant, dom)) if not args.chains else None,
-                "peak_source": (pk["source"] + {"tensor": " (sustained bf16 GEMM)", "tensor_split": f" (sustained bf16 GEMM / {split_products:.2f}: 3 bf16 products per float product in the logits, 6 in the mixing, 3 for tiles of one-hot rows: {t_brief} of {t_full + t_brief} tiles)"}.get(bound, " (copy)")) if bound != "alu"
-                else "derived: 148 SMs x 128 fp32 lanes x 2 x max SM clock",
-                "avg_launch_us": avg_s * 1e6, "launches_per_step": dom_n / steps,
-                "share_of_kernel_time": dom_ms / max(sum(v[0] for v in kinds.values()), 1e-9),
-                "kernel_ms_per_step": {k: v[0] / steps for k, v in kinds.items()}}
+    rows_per_step, windows_chains = run_counts(w, args.variant, calls_np, rows_np)
+    positions = float(int(ctl[10]) & 0x7fffffff) if prof.get("verify", (0, 0))[1] > 0 else 0.0   # of the last run
+    launch_shape = {"regen": bool(int(ctl[11]) & 1), "noise_cache": bool(int(ctl[11]) & 2)}
+    traffic = measured_traffic() if not args.chains else {}
+    if args.chains:                                     # a reduced batch: scale the captures to it all the same
+        traffic = measured_traffic()
+    rl = kernel_rooflines(w, args.variant, prof, steps, rows_per_step, windows_chains, positions, pk, ctl, traffic, launch_shape)
+    if not rl:
+        raise RuntimeError("no kernel of the library ran inside the timed region")
+    dom = rl[0]
+    roofline = {k: dom.get(k) for k in ("kernel", "bound", "achieved", "peak", "unit", "frac", "traffic", "peak_source",
+                                        "avg_launch_us", "launches_per_step", "share_of_kernel_time")}
+    roofline["kernel_ms_per_step"] = {k: v[0] / steps for k, v in prof.items() if v[1] > 0}
 
     acc_profile = acceptance_by_step(sds, w, dev, args.variant)
+    extra = {}
+    if w.denoiser == "phi4" and not args.no_extras:
+        extra["phi4_energy"] = phi4_energy_statistic(sds, w, dev)
+    if args.variant == "independent":
+        extra["cost_ratio"] = independent_cost_ratio(sds, w, dev, prof, steps, rows_per_step, windows_chains, ms_per_step)
+    s.close()
+    del out, flush
+    torch.cuda.empty_cache()
+    if world == 1 and not args.no_extras and args.variant == "default" and not args.chains:
+        extra["per_config"] = {w.name: {"B": B, "d": d, "L": w.L, "K": K, "ms_per_run": ms_per_step, "chain_steps_per_s": value,
+                                        "mean_target_calls": float(calls_np.mean()), "mean_target_rows": float(rows_np.mean()),
+                                        "mean_advance": float(K * B / max(windows_chains, 1)), "steps_timed": steps}}
+        for name in ("cfg1", "cfg2", "cfg3", "cfg4", "cfg5"):
+            if name != w.name:
+                extra["per_config"][name] = quick_config(sds, name, dev)
 
     osteps, sec, what = oracle_time(w, args.cpu_seconds, variant=args.variant)
     cpu = {"value": osteps / sec, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what}
@@ -530,11 +737,11 @@ def run_gpu(args, w):
                 "h2d_bytes_per_step": int(means_h.numel() * means_h.element_size() + logw_h.numel() * 4) if means_h is not None else 0,
                 "d2h_bytes_per_step": int(out_h.numel() * 4 + calls_h.numel() * 4 + rows_h.numel() * 4)},
         "gpu_launches": int(launches),
-        "roofline": roofline, "cpu_baseline": cpu, "clocks": clk,
+        "roofline": roofline, "rooflines": rl, "gathered": gathered, "cpu_baseline": cpu, "clocks": clk,
     }
+    line.update(extra)
     print(json.dumps(line), flush=True)
-    s.close()
-    if world > 1:
+    if dist is not None:
         dist.destroy_process_group()
 
 
@@ -544,11 +751,13 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="sds", choices=["sds", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(wl.WORKLOADS))
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="budget of the cpu_baseline leg")
     ap.add_argument("--chains", type=int, default=0, help="chains per GPU (default: the workload's own B)")
     ap.add_argument("--variant", default="default", choices=VARIANTS,
                     help="another drafter or accept test on the same workload (default: the workload's own)")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the per-workload table and the lattice energy statistic (profiler captures)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "sds":
         args.warmup = 3
@@ -557,8 +766,12 @@ def main():
         w = w.scaled(B=args.chains)
     if args.impl == "reference":
         run_reference(args, w)
-    else:
-        run_gpu(args, w)
+        return
+    from paper_2501_05370_b200 import sharding
+    if args.gpus > 1 and not sharding.under_launcher():
+        # started as `python bench.py --gpus N`: become N ranks, one per GPU
+        sys.exit(sharding.launch_ranks(args.gpus, os.path.abspath(__file__), sys.argv[1:]))
+    run_gpu(args, w)
 
 
 if __name__ == "__main__":

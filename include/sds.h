@@ -90,7 +90,10 @@ extern "C" {
 #define SDS_GET_NFE_ROWS  16    /* int32  [B]         target rows evaluated for the chain */
 #define SDS_GET_CTL       17    /* int32  [16]        n_active, nrows, windows done, error word, frozen chains, ...;
                                    [8], [9]: mixing-GEMM tiles of the split-precision mixture run with all six
-                                   products / with the three of the first plane since sds_reset */
+                                   products / with the three of the first plane since sds_reset;
+                                   [10]: window positions whose accept test was evaluated since sds_reset
+                                   (the window kernels; with SDS_OPT_VERIFY_EARLY_EXIT fewer than the rows drafted);
+                                   [11]: how the last sds_sample_all ran its windows (bit 0: SDS_OPT_REGEN_DRAFTS in effect) */
 #define SDS_GET_ROWK      18    /* int32  [nrows]     transition index of each row */
 #define SDS_GET_DP        19    /* float  [nrows, d]  independent drafter: the draft model's output per drafted row */
 
@@ -121,7 +124,8 @@ typedef int (*sds_denoise_fn)(void* user, const float* x_dev, const int32_t* k_d
  *   Posterior mean E[x0 | x_t] of a variance-preserving forward process and the energy gradient of
  *   the mixture both have this form (binding helpers compute the four scalars).
  *   means_dev: [ncomp, d] float (SDS_F32) or bf16 (SDS_BF16; then <x,mu> and the mixing sum run on
- *   tensor cores with x and r rounded to bf16). logw_dev: [ncomp] float.
+ *   tensor cores with x and r rounded to bf16). logw_dev: [ncomp] float. Float mixtures take at most 7264
+ *   components (one logit per component and warp in shared memory); more is SDS_EUNSUPPORTED.
  * MLP: nlayer linear layers dims[0]=d -> ... -> dims[nlayer]=d.
  *   h_l = SiLU(W_l h_{l-1} + bias_l + temb_l[k]) for l < nlayer, output = W_nlayer h + bias (float).
  *   W_dev[l]: [dims[l+1], dims[l]] bf16 row-major; bias_dev[l]: [dims[l+1]] float;
@@ -314,13 +318,15 @@ int64_t sds_launch_count(const sds_ctx* ctx);
  * the summed device time in milliseconds (ms[SDS_PROF_KINDS], host) and the number of launches
  * (launches[SDS_PROF_KINDS], host); reset != 0 clears the sums. Off by default. */
 #define SDS_PROF_INIT     0
-#define SDS_PROF_DENOISE  1
+#define SDS_PROF_DENOISE  1     /* target denoiser: GEMMs of the tensor-core denoisers, or the float kernel */
 #define SDS_PROF_DRAFT    2
 #define SDS_PROF_VERIFY   3
 #define SDS_PROF_ADVANCE  4
 #define SDS_PROF_FUSED    5     /* whole-chain persistent kernel */
 #define SDS_PROF_AUX      6     /* |mu|^2, list rebuild, copies of the initial call */
-#define SDS_PROF_KINDS    7
+#define SDS_PROF_SOFTMAX  7     /* passes between the two GEMMs of a tensor-core mixture (softmax, row conversions) */
+#define SDS_PROF_DRAFT_MODEL 8  /* every kernel of the independent draft model (SDS_INDEPENDENT) */
+#define SDS_PROF_KINDS    9
 int sds_profile(sds_ctx* ctx, int32_t enable);
 int sds_profile_read(sds_ctx* ctx, double* ms, int64_t* launches, int32_t reset);
 

@@ -224,6 +224,8 @@ int validate_den(const sds_denoiser* den, const double* tcond, int tcond_dim, in
         if (den->ncomp % 128 != 0 || d % 128 != 0) return SDS_EUNSUPPORTED;
       } else if (den->means_dtype != SDS_F32) {
         return SDS_EUNSUPPORTED;
+      } else if (!gmm_f32_shape_ok(den->ncomp, d)) {
+        return SDS_EUNSUPPORTED;          // more components than the float kernels hold logits for
       }
       break;
     case SDS_DEN_CALLBACK:
@@ -355,7 +357,7 @@ int ensure_musq(sds_ctx* c, Engine& e) {
 int ensure_bf16_rows(sds_ctx* c, Engine& e, const float* X, const uint16_t** Xb, int64_t rows_ub) {
   if (*Xb) return SDS_OK;
   uint16_t* dst = at<uint16_t>(c, e.lay.xb);
-  SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_f32_to_bf16(X, (size_t)rows_ub * c->d, dst, c->stream));
+  SDS_LAUNCH(c, &e == &c->drf ? SDS_PROF_DRAFT_MODEL : SDS_PROF_SOFTMAX, launch_f32_to_bf16(X, (size_t)rows_ub * c->d, dst, c->stream));
   *Xb = dst;
   return SDS_OK;
 }
@@ -376,6 +378,10 @@ TcGemmArgs tc_args(sds_ctx* c, Engine& e, const int* rowk, const int* nrows_dev,
 int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, const int* rowk, const int* nrows_dev,
                  int64_t rows_ub, float* out, bool planes_ready = false, bool raw = false) {
   if (rows_ub <= 0) return SDS_OK;
+  // timing kinds: the independent draft model's kernels are kept apart from the target's
+  const bool is_drafter = &e == &c->drf;
+  const int kd = is_drafter ? SDS_PROF_DRAFT_MODEL : SDS_PROF_DENOISE;
+  const int ks = is_drafter ? SDS_PROF_DRAFT_MODEL : SDS_PROF_SOFTMAX;
   switch (e.den.kind) {
     case SDS_DEN_GMM: {
       if (e.den.means_dtype == SDS_F32 && c->tensor_split && gmm_split_shape(e.den, c->d)) {
@@ -401,7 +407,7 @@ int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, cons
             SDS_LAUNCH(c, SDS_PROF_AUX, launch_transpose_bf16(Ms + i * nc * dd, (int)nc, (int)dd, Mt + i * nc * dd, c->stream));
         }
         if (!planes_ready)   // the draft and init kernels write the two row planes as they write the rows
-          SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_split3(X, (size_t)rows_ub * dd, cap * dd, 2, Xs, c->stream));
+          SDS_LAUNCH(c, ks, launch_split3(X, (size_t)rows_ub * dd, cap * dd, 2, Xs, c->stream));
         static const uint8_t kA[6] = {2, 1, 0, 1, 0, 0}, kB[6] = {0, 1, 2, 0, 1, 0};
         static const uint8_t kLa[3] = {1, 0, 0}, kLb[3] = {0, 1, 0};
         TcGemmArgs g = tc_args(c, e, rowk, nrows_dev, rows_ub);
@@ -409,12 +415,12 @@ int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, cons
         g.tcond = at<double>(c, e.lay.tcond); g.musq = at<double>(c, e.lay.musq); g.logw = e.den.logw_dev;
         g.nseg = 3; g.nplanes = 2; g.a_plane = cap * dd; g.b_plane = nc * dd;
         for (int i = 0; i < 3; ++i) { g.a_idx[i] = kLa[i]; g.b_idx[i] = kLb[i]; }
-        SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiGmmLogits, g, Xs, Ms, c->stream));
+        SDS_LAUNCH(c, kd, launch_gemm_tc(kEpiGmmLogits, g, Xs, Ms, c->stream));
         // rows whose responsibilities need only their first bf16 plane (one-hot rows above all) let
         // the mixing contraction drop the three products with the other planes, tile by tile
         int* flags = at<int>(c, e.lay.flags);
         SDS_CU(c, cudaMemsetAsync(flags, 0, (((size_t)rows_ub + 255) / 256 * 2) * 4, c->stream));
-        SDS_LAUNCH(c, SDS_PROF_DENOISE,
+        SDS_LAUNCH(c, ks,
                    launch_softmax_split3(logits, nrows_dev, (int)rows_ub, (int)nc, (int)dd, X, means,
                                          at<double>(c, e.lay.musq), e.den.logw_dev, at<double>(c, e.lay.tcond), rowk,
                                          cap * nc, Rs, flags, c->stream));
@@ -427,13 +433,13 @@ int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, cons
         m.tile_flags = flags; m.nseg_short = 3;
         m.tile_counts = at<int>(c, c->lay.ctl) + kCtlTilesFull;
         for (int i = 0; i < 3; ++i) { m.a_short[i] = kSa[i]; m.b_short[i] = kSb[i]; }
-        SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiGmmMix, m, Rs, Mt, c->stream));
+        SDS_LAUNCH(c, kd, launch_gemm_tc(kEpiGmmMix, m, Rs, Mt, c->stream));
         return SDS_OK;
       }
       if (e.den.means_dtype == SDS_F32) {
         const int rc = ensure_musq(c, e);
         if (rc != SDS_OK) return rc;
-        SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gmm_f32(gmm_args(c, e), X, rowk, nrows_dev, (int)rows_ub, out, c->stream));
+        SDS_LAUNCH(c, kd, launch_gmm_f32(gmm_args(c, e), X, rowk, nrows_dev, (int)rows_ub, out, c->stream));
         return SDS_OK;
       }
       // large mixture on tensor cores: logits = X M^T, softmax, mix = R M, affine epilogue
@@ -451,12 +457,12 @@ int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, cons
       TcGemmArgs g = tc_args(c, e, rowk, nrows_dev, rows_ub);
       g.N = e.den.ncomp; g.K = c->d; g.out = logits; g.ldo = e.den.ncomp;
       g.tcond = at<double>(c, e.lay.tcond); g.musq = at<double>(c, e.lay.musq); g.logw = e.den.logw_dev;
-      SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiGmmLogits, g, Xb, means, c->stream));
-      SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_softmax_bf16(logits, nrows_dev, (int)rows_ub, e.den.ncomp, R, c->stream));
+      SDS_LAUNCH(c, kd, launch_gemm_tc(kEpiGmmLogits, g, Xb, means, c->stream));
+      SDS_LAUNCH(c, ks, launch_softmax_bf16(logits, nrows_dev, (int)rows_ub, e.den.ncomp, R, c->stream));
       TcGemmArgs m = tc_args(c, e, rowk, nrows_dev, rows_ub);
       m.N = c->d; m.K = e.den.ncomp; m.out = out; m.ldo = c->d;
       m.tcond = at<double>(c, e.lay.tcond); m.xrows = raw ? nullptr : X;
-      SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiGmmMix, m, R, Mt, c->stream));
+      SDS_LAUNCH(c, kd, launch_gemm_tc(kEpiGmmMix, m, R, Mt, c->stream));
       return SDS_OK;
     }
     case SDS_DEN_MLP: {
@@ -471,17 +477,17 @@ int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, cons
         if (l < nl - 1) {
           uint16_t* h = at<uint16_t>(c, (l & 1) ? e.lay.H1 : e.lay.H0);
           g.out = h; g.ldo = g.N; g.temb = static_cast<const uint16_t*>(e.mlp_temb[l]);
-          SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiMlpHidden, g, in, e.mlp_W[l], c->stream));
+          SDS_LAUNCH(c, kd, launch_gemm_tc(kEpiMlpHidden, g, in, e.mlp_W[l], c->stream));
           in = h;
         } else {
           g.out = out; g.ldo = g.N;
-          SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_gemm_tc(kEpiBiasF32, g, in, e.mlp_W[l], c->stream));
+          SDS_LAUNCH(c, kd, launch_gemm_tc(kEpiBiasF32, g, in, e.mlp_W[l], c->stream));
         }
       }
       return SDS_OK;
     }
     case SDS_DEN_PHI4:
-      SDS_LAUNCH(c, SDS_PROF_DENOISE, launch_phi4_grad(X, nrows_dev, (int)rows_ub, e.den.grid_side, e.den.coupling,
+      SDS_LAUNCH(c, kd, launch_phi4_grad(X, nrows_dev, (int)rows_ub, e.den.grid_side, e.den.coupling,
                                                         e.den.periodic, out, c->stream));
       return SDS_OK;
     case SDS_DEN_CALLBACK: {
@@ -809,6 +815,10 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
       c->skipx_now = c->regen_now;
       // where the register-resident verify kernel runs, it also advances its chains and compacts
       c->fusing = c->fuse_advance && (verify_can_advance(A) || c->regen_now);
+      if (w == 0) {                                      // which of these paths the run takes (read back with the control words)
+        c->h_pin[48] = (c->regen_now ? 1 : 0);
+        SDS_CU(c, cudaMemcpyAsync(A.ctl + kCtlPathFlags, c->h_pin + 48, 4, cudaMemcpyHostToDevice, c->stream));
+      }
       rc = sds_draft(c);
       if (rc != SDS_OK) { c->fusing = c->raw_now = c->regen_now = c->skipx_now = false; return rc; }
       rc = sds_verify_window(c);

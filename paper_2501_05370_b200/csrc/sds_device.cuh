@@ -26,6 +26,9 @@ enum Ctl : int {
   kCtlSpare1 = 7,
   kCtlTilesFull = 8,  // mixing-GEMM tiles of the split-precision mixture run with all six products since reset
   kCtlTilesBrief = 9, // ... and with the three products of the first plane only
+  kCtlPositions = 10, // window positions whose accept test the verify kernels evaluated since reset (wraps at 2^31)
+  kCtlPathFlags = 11, // how the last sds_sample_all ran its windows: bit 0 verify drew the drafted states again,
+                      // bit 1 the drafted noise was kept in the workspace between windows (written by the host)
   kCtlWords = 16
 };
 constexpr int kErrNonFinite = 1;

@@ -12,6 +12,7 @@ namespace sds {
 namespace {
 
 constexpr int kGmmWarps = 4;
+constexpr size_t kGmmMaxSmem = 227 * 1024;   // dynamic shared memory one CTA can opt in to
 
 __global__ void k_musq(const float* __restrict__ means, int ncomp, int d, double* __restrict__ musq) {
   const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -26,17 +27,20 @@ __global__ void k_musq(const float* __restrict__ means, int ncomp, int d, double
   if (lane == 0) musq[c] = acc;
 }
 
-// smem layout: [means ncomp*d (optional)] [per-warp logits kGmmWarps*ncomp]
+// smem layout: [means ncomp*d floats (optional)] [per-warp logits kGmmWarps*ncomp doubles]
+// The logits stay in double until the row maximum is taken off: A <x, mu_c> and Bq |mu_c|^2 are large
+// and nearly cancel between components, so a float logit would carry an error of its own size times
+// 2^-24 into the weights.
 template <bool kMeansInSmem>
 __global__ void __launch_bounds__(kGmmWarps * 32) k_gmm_f32(GmmArgs G, const float* __restrict__ X,
                                                             const int* __restrict__ rowk,
                                                             const int* __restrict__ nrows_dev, int rows_host,
                                                             float* __restrict__ out) {
-  extern __shared__ float smem[];
+  extern __shared__ double smem_d[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int nrows = nrows_dev ? min(*nrows_dev, rows_host) : rows_host;
-  float* s_means = smem;
-  float* s_logit = smem + (kMeansInSmem ? (size_t)G.ncomp * G.d : 0) + (size_t)warp * G.ncomp;
+  double* s_logit = smem_d + (size_t)warp * G.ncomp;
+  float* s_means = reinterpret_cast<float*>(smem_d + (size_t)kGmmWarps * G.ncomp);
   if (kMeansInSmem) {
     for (int i = threadIdx.x; i < G.ncomp * G.d; i += blockDim.x) s_means[i] = G.means[i];
     __syncthreads();
@@ -47,30 +51,32 @@ __global__ void __launch_bounds__(kGmmWarps * 32) k_gmm_f32(GmmArgs G, const flo
     const int k = rowk[row];
     const double tA = __ldg(G.tcond + 4 * k + 0), tB = __ldg(G.tcond + 4 * k + 1);
     const float tC = (float)__ldg(G.tcond + 4 * k + 2), tE = (float)__ldg(G.tcond + 4 * k + 3);
-    float mx = -INFINITY;
+    double mx = -INFINITY;
     for (int c = 0; c < G.ncomp; ++c) {
       const float* mu = M + (size_t)c * G.d;
-      float acc = 0.f;
-      for (int i = lane; i < G.d; i += 32) acc = fmaf(x[i], mu[i], acc);
+      double acc = 0.0;
+      for (int i = lane; i < G.d; i += 32) acc = fma((double)x[i], (double)mu[i], acc);
       acc = warp_sum(acc);
-      const float lg = (float)fma(tA, (double)acc, fma(tB, __ldg(G.musq + c), (double)__ldg(G.logw + c)));
+      const double lg = fma(tA, acc, fma(tB, __ldg(G.musq + c), (double)__ldg(G.logw + c)));
       if (lane == 0) s_logit[c] = lg;
-      mx = fmaxf(mx, lg);
+      mx = fmax(mx, lg);
     }
     __syncwarp();
     float den = 0.f;
     for (int c = lane; c < G.ncomp; c += 32) {
-      const float e = expf(s_logit[c] - mx);
-      s_logit[c] = e;
+      const float e = expf((float)(s_logit[c] - mx));
+      s_logit[c] = (double)e;
       den += e;
     }
     den = warp_sum(den);
     __syncwarp();
     const float scale = tC / den;
     for (int i = lane; i < G.d; i += 32) {
-      float acc = 0.f;
-      for (int c = 0; c < G.ncomp; ++c) acc = fmaf(s_logit[c], M[(size_t)c * G.d + i], acc);
-      out[(size_t)row * G.d + i] = fmaf(scale, acc, tE * x[i]);
+      // thousands of signed terms: the mixing sum is kept in double so that its rounding stays below
+      // the float result's own
+      double acc = 0.0;
+      for (int c = 0; c < G.ncomp; ++c) acc = fma(s_logit[c], (double)M[(size_t)c * G.d + i], acc);
+      out[(size_t)row * G.d + i] = fmaf(scale, (float)acc, tE * x[i]);
     }
     __syncwarp();
   }
@@ -386,7 +392,7 @@ cudaError_t launch_gmm_f32(const GmmArgs& G, const float* X, const int* rowk, co
     return cudaGetLastError();
   }
   const size_t means_bytes = (size_t)G.ncomp * G.d * sizeof(float);
-  const size_t logit_bytes = (size_t)kGmmWarps * G.ncomp * sizeof(float);
+  const size_t logit_bytes = (size_t)kGmmWarps * G.ncomp * sizeof(double);
   const bool in_smem = means_bytes + logit_bytes <= 96 * 1024;
   const size_t smem = (in_smem ? means_bytes : 0) + logit_bytes;
   int blocks = (rows_ub + kGmmWarps - 1) / kGmmWarps;
@@ -400,9 +406,23 @@ cudaError_t launch_gmm_f32(const GmmArgs& G, const float* X, const int* rowk, co
     }
     k_gmm_f32<true><<<blocks, kGmmWarps * 32, smem, st>>>(G, X, rowk, nrows_dev, rows_ub, out);
   } else {
+    if (smem > kGmmMaxSmem) return cudaErrorInvalidValue;   // gmm_f32_shape_ok() is the caller's check
+    if (smem > 48 * 1024) {
+      const cudaError_t e =
+          cudaFuncSetAttribute(k_gmm_f32<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+    }
     k_gmm_f32<false><<<blocks, kGmmWarps * 32, smem, st>>>(G, X, rowk, nrows_dev, rows_ub, out);
   }
   return cudaGetLastError();
+}
+
+// Largest mixture the float kernels take: the one-warp-per-row kernel keeps one logit per component and
+// warp in shared memory (227 KB per CTA); the small and the tiled kernel cover their shapes before it.
+bool gmm_f32_shape_ok(int ncomp, int d) {
+  if (ncomp <= 0 || d <= 0) return false;
+  if (ncomp <= kTNC) return true;
+  return (size_t)kGmmWarps * ncomp * sizeof(double) <= kGmmMaxSmem;
 }
 
 }  // namespace sds

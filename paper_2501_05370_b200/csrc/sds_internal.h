@@ -94,6 +94,7 @@ cudaError_t launch_rng_uniforms(uint64_t seed, uint64_t b0, int64_t nb, int k, f
 
 // mixture denoiser, float path (sds_gmm.cu)
 cudaError_t launch_musq(const float* means, int ncomp, int d, double* musq, cudaStream_t st);
+bool gmm_f32_shape_ok(int ncomp, int d);   // whether launch_gmm_f32 has a kernel for this mixture
 cudaError_t launch_gmm_f32(const GmmArgs& G, const float* X, const int* rowk, const int* nrows_dev, int rows_ub,
                            float* out, cudaStream_t st);
 

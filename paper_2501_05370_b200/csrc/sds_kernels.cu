@@ -118,6 +118,7 @@ __global__ void __launch_bounds__(kBlock) k_init(WinArgs A) {
     A.ctl[kCtlTcError] = 0;
     A.ctl[kCtlTilesFull] = 0;
     A.ctl[kCtlTilesBrief] = 0;
+    A.ctl[kCtlPositions] = 0;
   }
   if (b >= A.B) return;
   const uint64_t bg = A.chain_off + (uint64_t)b;
@@ -619,6 +620,7 @@ __global__ void __launch_bounds__(kBlock) k_verify(WinArgs A) {
     if (lane == 0) {
       A.accmask[b] = amask;
       A.jstar[b] = jstar;
+      atomicAdd(A.ctl + kCtlPositions, Lt);
       if (bmask) atomicOr(A.ctl + kCtlError, kErrNonFinite);
       if (TPC > 32) { s_jstar = jstar; s_coef = coef; }
     }
@@ -831,6 +833,7 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t,
     if (lane == 0) {
       A.accmask[b] = amask;
       A.jstar[b] = jstar;
+      atomicAdd(A.ctl + kCtlPositions, done);
       if (frozen) atomicOr(A.ctl + kCtlError, kErrNonFinite);
       if (TPC > 32) { s_jstar = jstar; s_coef = coef; }
     }

@@ -73,6 +73,23 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return false;
 }
 
+// The same wait for a whole warp, with one outcome for all its lanes: lane 0 polls (up to the cap),
+// the result is broadcast, and on success every lane confirms the completed phase itself (one poll,
+// its own acquire) before it touches what the barrier guards. On the give-up path no lane can leave
+// with a different answer than its neighbours, so the aligned tensor-memory loads and warp
+// synchronisations that follow are never reached by part of a warp.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  int ok = 1;
+  if ((threadIdx.x & 31u) == 0u) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+  ok = __shfl_sync(0xffffffffu, ok, 0);
+  if (ok) {
+    bool mine = false;
+    for (uint32_t it = 0; it < 1024u && !mine; ++it) mine = mbar_try_wait(bar, parity);
+    ok = __all_sync(0xffffffffu, mine) ? 1 : 0;
+  }
+  return ok != 0;
+}
+
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int c0, int c1, uint64_t* bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
@@ -92,6 +109,15 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
   uint32_t r;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
   return r;
+}
+// a role that gives up tells its own CTA and, in a pair, the other CTA (whose roles would otherwise
+// each run out their own poll limit before noticing)
+__device__ __forceinline__ void raise_abort(volatile int* abort_flag, bool pair) {
+  *abort_flag = 1;
+  if (pair) {
+    const uint32_t peer = map_to_cta(smem_u32(const_cast<int*>(abort_flag)), cluster_ctarank() ^ 1u);
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(peer), "r"(1u) : "memory");
+  }
 }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
@@ -294,7 +320,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
       }
       if (!ok) {
-        *abort_s = 1;
+        raise_abort(abort_s, PAIR);
         atomicExch(g.err, 1);
       }
     }
@@ -333,7 +359,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (ok) { if (PAIR) umma_commit_pair(tfull_bar + buf); else umma_commit(tfull_bar + buf); }   // accumulator complete
       }
       if (!ok) {
-        *abort_s = 1;
+        raise_abort(abort_s, PAIR);
         atomicExch(g.err, 2);
       }
     }
@@ -395,7 +421,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             }
           }
           if (!waited) {
-            if (!mbar_wait(tfull_bar + buf, bphase, abort_s)) { ok = false; break; }
+            if (!mbar_wait_warp(tfull_bar + buf, bphase, abort_s)) { ok = false; break; }
             tc_fence_after();
             waited = true;
           }
@@ -444,7 +470,7 @@ __global__ void __launch_bounds__(kThreads, 1)
           __syncwarp();
         }
       } else {
-        if (!mbar_wait(tfull_bar + buf, bphase, abort_s)) { ok = false; break; }
+        if (!mbar_wait_warp(tfull_bar + buf, bphase, abort_s)) { ok = false; break; }
         tc_fence_after();
 #pragma unroll 1
         for (int c = 0; c < kCols; c += 32) {
@@ -461,7 +487,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       }
     }
     if (!ok && lane == 0) {
-      *abort_s = 1;
+      raise_abort(abort_s, PAIR);
       atomicExch(g.err, 3);
     }
   }

@@ -4,16 +4,17 @@ from __future__ import annotations
 import numpy as np
 
 from . import binding as sb
+from . import schedules as sc
 
 
 def schedule_for(w):
     """float32 (a, c, sigma) and the mixture conditioning table for workload w (None for non-mixtures)."""
     if w.sampler == "ddpm":
-        a, c, sigma, abar = sb.ddpm_schedule(w.beta())
-        tcond = sb.gmm_tcond_posterior_mean(abar, w.gmm["comp_std"]) if w.denoiser == "gmm" else None
+        a, c, sigma, abar = sc.ddpm_schedule(w.beta())
+        tcond = sc.gmm_tcond_posterior_mean(abar, w.gmm["comp_std"]) if w.denoiser == "gmm" else None
     elif w.sampler == "ula":
-        a, c, sigma = sb.ula_schedule(w.K, w.ula_gamma)
-        tcond = sb.gmm_tcond_grad_energy(w.K, w.gmm["comp_std"]) if w.denoiser == "gmm" else None
+        a, c, sigma = sc.ula_schedule(w.K, w.ula_gamma)
+        tcond = sc.gmm_tcond_grad_energy(w.K, w.gmm["comp_std"]) if w.denoiser == "gmm" else None
     else:
         raise ValueError(w.sampler)
     return a, c, sigma, tcond
@@ -23,9 +24,9 @@ def drafter_for(w, *, gmm=None, mlp=None):
     """Description of an independent draft model for workload w: a (smaller) mixture or MLP."""
     if gmm is not None:
         if w.sampler == "ddpm":
-            tc = sb.gmm_tcond_posterior_mean(sb.ddpm_schedule(w.beta())[3], gmm.comp_std)
+            tc = sc.gmm_tcond_posterior_mean(sc.ddpm_schedule(w.beta())[3], gmm.comp_std)
         else:
-            tc = sb.gmm_tcond_grad_energy(w.K, gmm.comp_std)
+            tc = sc.gmm_tcond_grad_energy(w.K, gmm.comp_std)
         return dict(gmm_means=gmm.means, gmm_logw=gmm.logw, tcond=tc, gmm_bf16=bool(getattr(gmm, "means_bf16", False)))
     if mlp is not None:
         return dict(mlp=mlp)
@@ -36,9 +37,9 @@ def picard_for(w, calls: int):
     """(calls, a_det, c_det) for Sampler(picard=...): the deterministic sampler that goes with the
     workload's schedule (noise-free ancestral step for ddpm, gradient step for Langevin)."""
     if w.sampler == "ddpm":
-        a_det, c_det = sb.ddim_schedule(w.beta())
+        a_det, c_det = sc.ddim_schedule(w.beta())
     else:
-        a_det, c_det, _ = sb.ula_schedule(w.K, w.ula_gamma)
+        a_det, c_det, _ = sc.ula_schedule(w.K, w.ula_gamma)
     return (int(calls), a_det, c_det)
 
 

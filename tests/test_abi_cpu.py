@@ -9,6 +9,7 @@ import pytest
 
 import paper_2501_05370_b200 as sds
 from paper_2501_05370_b200 import binding as sb
+from paper_2501_05370_b200 import schedules as sc
 from oracle import sds_oracle as o
 import workloads as wl
 
@@ -77,7 +78,7 @@ def test_host_side_argument_validation():
 @pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3", "cfg4"])
 def test_ddpm_schedule_helper_matches_oracle(name):
     w = wl.WORKLOADS[name]
-    a, c, s, abar = sb.ddpm_schedule(w.beta())
+    a, c, s, abar = sc.ddpm_schedule(w.beta())
     ao, co, so, abo = o.ddpm_affine(w.beta())
     assert a.dtype == np.float32
     for x, y in ((a, ao), (c, co), (s, so)):
@@ -90,8 +91,8 @@ def test_gmm_conditioning_table_reproduces_oracle_denoiser():
     equals the oracle's definition-level posterior mean / energy gradient."""
     w = wl.WORKLOADS["cfg2"]
     gp = w.gmm_params()
-    a, c, s, abar = sb.ddpm_schedule(w.beta())
-    tc = sb.gmm_tcond_posterior_mean(abar, gp.comp_std).astype(np.float64)
+    a, c, s, abar = sc.ddpm_schedule(w.beta())
+    tc = sc.gmm_tcond_posterior_mean(abar, gp.comp_std).astype(np.float64)
     rng = np.random.default_rng(0)
     mu = gp.means.astype(np.float64)
     for k in (0, 57, 150, 199):
@@ -104,14 +105,14 @@ def test_gmm_conditioning_table_reproduces_oracle_denoiser():
         assert np.allclose(got, want, rtol=2e-5, atol=2e-5)
     w5 = wl.WORKLOADS["cfg5"]
     gp5 = w5.gmm_params(d=32, ncomp=8)
-    tc5 = sb.gmm_tcond_grad_energy(3, gp5.comp_std).astype(np.float64)
+    tc5 = sc.gmm_tcond_grad_energy(3, gp5.comp_std).astype(np.float64)
     x = rng.standard_normal(32) * 4
     mu = gp5.means.astype(np.float64)
     A, Bq, Cc, E = tc5[0]
     lg = gp5.logw + A * (mu @ x) + Bq * np.sum(mu * mu, axis=1)
     r = np.exp(lg - lg.max()); r /= r.sum()
     assert np.allclose(Cc * (r @ mu) + E * x, o.gmm_grad_energy(x, gp5.means, gp5.logw, gp5.comp_std), rtol=1e-6, atol=1e-6)
-    a5, c5, s5 = sb.ula_schedule(3, 1e-3)
+    a5, c5, s5 = sc.ula_schedule(3, 1e-3)
     ao, co, so = o.ula_affine(3, 1e-3)
     assert np.allclose(a5, ao) and np.allclose(c5, co, rtol=1e-7) and np.allclose(s5, so, rtol=1e-7)
 

@@ -7,7 +7,7 @@ import paper_2501_05370_b200 as sds
 from paper_2501_05370_b200 import binding as sb
 from oracle import sds_oracle as o
 import workloads as wl
-from helpers import BAND, ell_close, oracle_setup, rel_l2
+from helpers import BAND, assert_rows_close, ell_close, oracle_setup, rel_l2
 
 pytestmark = pytest.mark.gpu
 
@@ -27,12 +27,8 @@ def test_mlp_denoiser_rows(dims, rows, K):
     k = rng.integers(0, K, size=rows).astype(np.int32)
     out = s.denoise(torch.from_numpy(x).cuda(), torch.from_numpy(k).cuda()).cpu().numpy()
     assert np.all(np.isfinite(out))
-    worst = 0.0
-    for r in range(0, rows, max(1, rows // 60)):
-        worst = max(worst, rel_l2(out[r], den(x[r].astype(np.float64), int(k[r]))))
-    assert worst <= TOL, worst
-    # the last row of the ragged tile as well
-    assert rel_l2(out[rows - 1], den(x[rows - 1].astype(np.float64), int(k[rows - 1]))) <= TOL
+    for r in list(range(0, rows, max(1, rows // 60))) + [rows - 1]:     # the last row of the ragged tile as well
+        assert_rows_close(out[r], den(x[r].astype(np.float64), int(k[r])), TOL, r)
     s.close()
 
 
@@ -50,20 +46,23 @@ def test_large_mixture_denoiser_rows(d, ncomp, rows):
     out = s.denoise(torch.from_numpy(x).cuda(), torch.from_numpy(k).cuda()).cpu().numpy()
     assert np.all(np.isfinite(out))
     for r in range(0, rows, max(1, rows // 50)):
-        assert rel_l2(out[r], den(x[r].astype(np.float64), int(k[r]))) <= TOL, r
+        assert_rows_close(out[r], den(x[r].astype(np.float64), int(k[r])), TOL, r)
     s.close()
 
 
-def _forced_window(s, w, den, seed, off, windows, chains=None):
+def _forced_window(s, w, den, seed, off, windows, chains=None, every_position=None, reset=True):
     """Decisions and log ratios of the verify step replayed by the oracle on the GPU's own arrays
-    (the denoiser outputs are the GPU's; their parity is checked separately at 2e-2)."""
+    (the denoiser outputs are the GPU's; their parity is checked at 2e-2, row norm and element-wise,
+    at the first and last position of every checked chain and at every position of the chains in
+    `every_position`). Returns the number of denoiser rows compared."""
     s.set_option(s.OPT_VERIFY_EARLY_EXIT, 0)      # these checks look at every position of the window
     import math
     a32, c32, s32, _ = sds.schedule_for(w)
     a64, c64, s64 = a32.astype(np.float64), c32.astype(np.float64), s32.astype(np.float64)
     B, L, d, K = s.B, s.L, s.d, s.K
-    band = tests = 0
-    s.reset()
+    band = tests = den_rows = 0
+    if reset:
+        s.reset()
     for _ in range(windows):
         ctl = s.get(sb.GET_CTL)
         na = int(ctl[0])
@@ -77,13 +76,17 @@ def _forced_window(s, w, den, seed, off, windows, chains=None):
         Dq = s.get(sb.GET_DQ)
         ell, logU, accmask, jstar = s.get(sb.GET_ELL), s.get(sb.GET_LOGU), s.get(sb.GET_ACCMASK), s.get(sb.GET_JSTAR)
         X2, T2 = s.get(sb.GET_X), s.get(sb.GET_TAIL)
+        rowk = s.get(sb.GET_ROWK)
         for si, b in enumerate(act):
             if chains is not None and int(b) not in chains:
                 continue
             nb = int(n[b]); Lt = min(L, K - nb); r0 = int(rowoff[si])
             W = np.concatenate([X[r0:r0 + Lt], T[b:b + 1]]).astype(np.float64)
-            for j in (1, Lt):
-                assert rel_l2(Dq[r0 + j - 1], den(W[j - 1], nb + j - 1)) <= TOL
+            assert np.array_equal(rowk[r0:r0 + Lt], nb + np.arange(Lt))
+            full = every_position is not None and int(b) in every_position
+            for j in (range(1, Lt + 1) if full else sorted({1, Lt})):
+                assert_rows_close(Dq[r0 + j - 1], den(W[j - 1], nb + j - 1), TOL, (int(b), j))
+                den_rows += 1
             v = o.verify_window(W, Dq[r0:r0 + Lt], Dc[b], a64, c64, s64, nb, logU[b, :Lt].astype(np.float64))
             amb = np.abs(v["ell"] - logU[b, :Lt]) < BAND
             for j in range(Lt):
@@ -97,9 +100,10 @@ def _forced_window(s, w, den, seed, off, windows, chains=None):
                 assert int(jstar[b]) == v["jstar"]
                 js = int(jstar[b])
                 if js <= Lt:
-                    assert rel_l2(X2[r0 + js] if js < Lt else T2[b], v["Y_reflect"]) <= 1e-5
+                    assert_rows_close(X2[r0 + js] if js < Lt else T2[b], v["Y_reflect"], 1e-5, (int(b), js))
         s.advance()
     assert band <= max(2, 2e-3 * tests)
+    return den_rows
 
 
 def test_mlp_window_forced_and_free_run():
@@ -134,9 +138,14 @@ def test_large_mixture_window_forced_and_free_run():
 
 @pytest.mark.parametrize("name", ["cfg3", "cfg4"])
 def test_full_size_tensor_core_windows_on_sampled_chains(name):
-    """Full benchmark sizes and launch shapes (thousands of GEMM tiles, ragged row counts after the
-    first window); the oracle replays a sample of chains. Then the whole run: every chain ends at
-    n = K with finite state and consistent counters."""
+    """Full benchmark sizes and launch shapes (thousands of GEMM tiles). The oracle replays sixteen
+    chains: the first window (every chain at step 0, full row count), then, after forty more windows,
+    a window in which the chains sit at different steps, some of them so close to the end that their
+    windows are shorter than L and one already finished, so that the row count is no multiple of the
+    tile height and the last tile of every GEMM is ragged; there every position of the sixteen chains
+    is compared with the oracle's denoiser (the first window: every position of four of them).
+    Then the whole run: every chain ends at n = K with finite state and consistent counters."""
+    import torch
     w = wl.WORKLOADS[name]
     if name == "cfg3":
         mp_ = w.mlp_params()
@@ -146,8 +155,27 @@ def test_full_size_tensor_core_windows_on_sampled_chains(name):
         gp = w.gmm_params()
         s = sds.sampler_for(w, gmm=gp)
         den, a, c, sig = oracle_setup(w, gmm=gp)
-    chains = {0, 1, w.B // 2 + 1, w.B - 1}
-    _forced_window(s, w, den, w.sample_seed, 0, 2, chains=chains)
+    rng = np.random.default_rng(11)
+    chains = sorted({0, 1, 2, 3, w.B // 2 + 1, w.B - 2, w.B - 1} | set(int(x) for x in rng.choice(w.B, size=9, replace=False)))
+    chains = chains[:16] if len(chains) > 16 else chains
+    first = _forced_window(s, w, den, w.sample_seed, 0, 1, chains=set(chains), every_position=set(chains[:4]))
+    assert first >= 4 * w.L
+    for _ in range(40):
+        s.draft(); s.verify_window(); s.advance(sync=False)
+    n = s.get(sb.GET_N).copy()
+    assert len(set(n[chains].tolist())) > 1                   # the chains have spread over the steps
+    n[chains[1]] = w.K - 3                                    # a window of three positions
+    n[chains[2]] = w.K                                        # a finished chain: no rows at all
+    n[chains[3]] = w.K - 1                                    # a window of one position
+    n[chains[-1]] = w.K - (w.L - 1)                           # the last chain: one position short of a full window
+    if int(np.minimum(w.L, w.K - n)[n < w.K].sum()) % 128 == 0:
+        n[chains[4]] = w.K - 2
+    s.set_state(n=torch.from_numpy(n).cuda())
+    ctl = s.get(sb.GET_CTL)
+    assert int(ctl[0]) == int(np.sum(n < w.K)) and int(ctl[1]) == int(np.minimum(w.L, w.K - n)[n < w.K].sum())
+    assert int(ctl[1]) % 128 != 0                             # ragged: the row count is no multiple of a tile
+    late = _forced_window(s, w, den, w.sample_seed, 0, 1, chains=set(chains), every_position=set(chains), reset=False)
+    assert late >= 11 * w.L
     out, calls, rows = [x.cpu().numpy() for x in s.sample_all()]
     assert np.all(np.isfinite(out)) and np.array_equal(s.get(sb.GET_N), np.full(w.B, w.K))
     assert np.all(calls >= 1 + -(-w.K // w.L)) and np.all(calls <= 1 + w.K)
