@@ -377,17 +377,28 @@ def kernel_rooflines(w, variant, prof, steps, rows, cw, positions, pk, ctl, traf
             else:
                 per_run = 4.0 * w.gmm["ncomp"] * d * (rows + B)
                 bound = "tensor" if (kind == "denoise" and tensor_mixture(w)) else "alu"
+                if bound == "tensor":
+                    # mixing tiles of blocks whose rows are all one-hot are not computed at all (a copy kernel writes
+                    # those rows): only the contraction work that ran counts as achieved
+                    ran, skipped = int(ctl[8]) + int(ctl[9]), int(ctl[10])
+                    mix_done = ran / max(1, ran + skipped)
+                    per_run *= 0.5 * (1.0 + mix_done)
+                    e["mixing_tiles_skipped_frac"] = 1.0 - mix_done
             if kind == "draft_model":
                 bound, per_run = "alu", 4.0 * max(1, w.gmm["ncomp"] // 2) * d * rows
             peak, unit, src = (tens, "TFLOP/s", pk["source"] + " (sustained bf16 GEMM)") if bound == "tensor" else \
                               (alu_peak, "TFLOP/s", "derived: 148 SMs x 128 fp32 lanes x 2 x max SM clock")
             if bound == "tensor" and split:
                 # float operands as bf16 planes: 3 bf16 products per float product in the logits, 6 in the
-                # mixing (3 for tiles whose responsibilities need only their first plane; the library counts both)
+                # mixing (3 for tiles whose responsibilities need only their first plane; the library counts both),
+                # weighted by the contraction work that ran (the logits always, the mixing where it was not skipped)
                 t_full, t_brief = int(ctl[8]), int(ctl[9])
                 mix = (6.0 * t_full + 3.0 * t_brief) / max(1, t_full + t_brief)
-                peak = tens / ((3.0 + mix) / 2.0)
-                src = pk["source"] + f" (sustained bf16 GEMM / {(3.0 + mix) / 2.0:.2f} bf16 products per float product; {t_brief} of {t_full + t_brief} mixing tiles one-hot)"
+                f_mix = e.get("mixing_tiles_skipped_frac")
+                f_mix = 1.0 if f_mix is None else 1.0 - f_mix
+                products = (3.0 + mix * f_mix) / (1.0 + f_mix)
+                peak = tens / products
+                src = pk["source"] + f" (sustained bf16 GEMM / {products:.2f} bf16 products per float product; {t_brief} of {t_full + t_brief} mixing tiles run on one plane)"
             ach = per_run / (ms / steps * 1e-3) / 1e12
             e.update(bound=bound, achieved=ach, peak=peak, unit=unit, frac=ach / peak, peak_source=src,
                      algorithmic_per_launch=per_run / per_run_launches)
@@ -691,7 +702,7 @@ def run_gpu(args, w):
     value = world * B * K / (ms_per_step * 1e-3)
     e2e_value = world * B * K / (ms_e2e / steps * 1e-3)
     rows_per_step, windows_chains = run_counts(w, args.variant, calls_np, rows_np)
-    positions = float(int(ctl[10]) & 0x7fffffff) if prof.get("verify", (0, 0))[1] > 0 else 0.0   # of the last run
+    positions = float(int(ctl[12]) & 0x7fffffff) if prof.get("verify", (0, 0))[1] > 0 else 0.0   # of the last run
     launch_shape = {"regen": bool(int(ctl[11]) & 1), "noise_cache": bool(int(ctl[11]) & 2)}
     traffic = measured_traffic() if not args.chains else {}
     if args.chains:                                     # a reduced batch: scale the captures to it all the same
@@ -706,6 +717,21 @@ def run_gpu(args, w):
 
     acc_profile = acceptance_by_step(sds, w, dev, args.variant)
     extra = {}
+    if prof.get("verify", (0, 0))[1] > 0 and args.variant == "default" and not args.no_extras:
+        # the streaming kernels with every position of every window evaluated and the drafted rows read back
+        # (options off, outside the timed region): the two-stream reduction of the verify step as such
+        s.set_option(s.OPT_VERIFY_EARLY_EXIT, 0); s.set_option(s.OPT_REGEN_DRAFTS, 0)
+        dev_step()
+        s.profile(True); s.profile_read(reset=True)
+        for _ in range(3):
+            dev_step()
+        prof_all = s.profile_read(reset=True)
+        s.profile(False)
+        ctl_all = s.get(sb.GET_CTL)
+        rl_all = kernel_rooflines(w, args.variant, prof_all, 3, rows_per_step, windows_chains, float(int(ctl_all[12]) & 0x7fffffff),
+                                  pk, ctl_all, {}, {"regen": False})
+        extra["rooflines_every_position"] = [e for e in rl_all if e["kernel"] in ("verify", "draft", "advance")]
+        s.set_option(s.OPT_VERIFY_EARLY_EXIT, 1); s.set_option(s.OPT_REGEN_DRAFTS, 1)
     if w.denoiser == "phi4" and not args.no_extras:
         extra["phi4_energy"] = phi4_energy_statistic(sds, w, dev)
     if args.variant == "independent":

@@ -91,9 +91,11 @@ extern "C" {
 #define SDS_GET_CTL       17    /* int32  [16]        n_active, nrows, windows done, error word, frozen chains, ...;
                                    [8], [9]: mixing-GEMM tiles of the split-precision mixture run with all six
                                    products / with the three of the first plane since sds_reset;
-                                   [10]: window positions whose accept test was evaluated since sds_reset
-                                   (the window kernels; with SDS_OPT_VERIFY_EARLY_EXIT fewer than the rows drafted);
-                                   [11]: how the last sds_sample_all ran its windows (bit 0: SDS_OPT_REGEN_DRAFTS in effect) */
+                                   [10]: mixing-GEMM tiles skipped since sds_reset (SDS_OPT_ONEHOT_ROWS);
+                                   [11]: how the last sds_sample_all ran its windows (bit 0: SDS_OPT_REGEN_DRAFTS in effect,
+                                   bit 2: rows of skipped one-hot blocks read from the means table, see SDS_OPT_ONEHOT_ROWS);
+                                   [12]: window positions whose accept test was evaluated since sds_reset
+                                   (the window kernels; with SDS_OPT_VERIFY_EARLY_EXIT fewer than the rows drafted) */
 #define SDS_GET_ROWK      18    /* int32  [nrows]     transition index of each row */
 #define SDS_GET_DP        19    /* float  [nrows, d]  independent drafter: the draft model's output per drafted row */
 
@@ -260,6 +262,15 @@ int sds_sample_all(sds_ctx* ctx, float* out_dev, int32_t* nfe_calls_dev, int32_t
  * reads only the target outputs, and advances its chains. Same results, bit for bit. SDS_GET_X and
  * SDS_GET_TAIL are then stale after sds_sample_all. */
 #define SDS_OPT_REGEN_DRAFTS 7
+/* SDS_OPT_ONEHOT_ROWS (default 1): mixtures on the tensor cores. The softmax pass stores weights below 2^-40 of
+ * their row as exact zeros (either way). A row left with a single weight is one-hot: its weight is 1 and its
+ * mixing sum is that component's mean. With this option the mixing GEMM skips every block of 256 rows whose
+ * rows are all one-hot, and a copy kernel writes mean rows there instead (sharply peaked posteriors: late
+ * diffusion steps, well separated Langevin modes). The product with an exact one-hot row is the mean itself,
+ * so the results are the same bit for bit; 0 sends every block through the GEMM. Inside sds_sample_all with
+ * SDS_OPT_RAW_ROWS in effect the copy is not made either: the verify and advance kernels read the skipped
+ * blocks' rows from the mixture's means table by component index (SDS_GET_DQ is then stale for those rows). */
+#define SDS_OPT_ONEHOT_ROWS 8
 int sds_set_option(sds_ctx* ctx, int32_t option, int64_t value);
 
 /* Temperature of the accept test (Appendix D, temperature rejection): a draft is accepted iff

@@ -324,6 +324,7 @@ class Sampler:
     OPT_FUSE_ADVANCE = 5
     OPT_RAW_ROWS = 6
     OPT_REGEN_DRAFTS = 7
+    OPT_ONEHOT_ROWS = 8
 
     def set_option(self, option: int, value: int):
         self._chk(self.lib.sds_set_option(self.h, option, value), "sds_set_option")

@@ -52,6 +52,7 @@ struct DenLayout {
   size_t logits, R, Mt;   // large mixture: logits (f32), responsibilities (bf16), transposed means (bf16)
   size_t Xs, Ms;          // float mixture on tensor cores: 3 bf16 planes of the rows / of the means
   size_t flags;           // one int per 128 rows: responsibilities with a non-zero second or third plane
+  size_t amax, hot;       // component of every one-hot row (-1: not one-hot); one int per 256 rows: some row not one-hot
   size_t xb;              // where a bf16 copy of this denoiser's input rows goes when the caller has none
 };
 
@@ -101,7 +102,9 @@ struct sds_ctx {
   bool regen = true;                // sds_sample_all lets the verify kernel draw the drafted states again instead of reading them
   bool fusing = false;              // set around the verify call of the sds_sample_all loop
   bool raw_rows = true;             // sds_sample_all lets the mixing GEMM store accumulators, verify applies C acc + E x
+  bool onehot = true;               // the mixing GEMM skips blocks of rows that are all one-hot; a copy kernel fills them
   bool raw_now = false;             // set around the verify and advance calls of the sds_sample_all loop
+  bool hot_now = false;             // likewise: rows of skipped (all one-hot) blocks are read from the means table, not stored
   bool regen_now = false;           // likewise: verify regenerates the drafted states
   bool skipx_now = false;           // likewise: the draft kernel stores only the bf16 copy of its rows
   // optional per-kernel timing: event pairs recorded around each launch, summed on read
@@ -128,7 +131,7 @@ bool wants_bf16_rows(const sds_denoiser& den) {
 void den_layout(Carve& cv, const sds_denoiser* den, size_t K, int tcond_dim, size_t rows, int32_t d, DenLayout* l) {
   l->tcond = cv.take(K * (size_t)(tcond_dim > 0 ? tcond_dim : 1) * 8);
   l->musq = (den->kind == SDS_DEN_GMM) ? cv.take((size_t)den->ncomp * 8) : kNone;
-  l->H0 = l->H1 = l->logits = l->R = l->Mt = l->Xs = l->Ms = l->flags = kNone;
+  l->H0 = l->H1 = l->logits = l->R = l->Mt = l->Xs = l->Ms = l->flags = l->amax = l->hot = kNone;
   if (gmm_split_shape(*den, d)) {
     l->Xs = cv.take(2 * rows * (size_t)d * 2);
     l->Ms = cv.take(3 * (size_t)den->ncomp * d * 2);
@@ -136,6 +139,8 @@ void den_layout(Carve& cv, const sds_denoiser* den, size_t K, int tcond_dim, siz
     l->R = cv.take(3 * rows * (size_t)den->ncomp * 2);
     l->logits = cv.take(rows * (size_t)den->ncomp * 4);
     l->flags = cv.take(((rows + 255) / 256 * 2) * 4);
+    l->amax = cv.take(rows * 4);
+    l->hot = cv.take(((rows + 255) / 256) * 4);
   }
   if (den->kind == SDS_DEN_MLP) {
     size_t width = 0;
@@ -147,6 +152,8 @@ void den_layout(Carve& cv, const sds_denoiser* den, size_t K, int tcond_dim, siz
     l->logits = cv.take(rows * (size_t)den->ncomp * 4);
     l->R = cv.take(rows * (size_t)den->ncomp * 2);
     l->Mt = cv.take((size_t)d * den->ncomp * 2);
+    l->amax = cv.take(rows * 4);
+    l->hot = cv.take(((rows + 255) / 256) * 4);
   }
 }
 
@@ -263,6 +270,12 @@ WinArgs win_args(sds_ctx* c) {
   A.early_exit = c->early_exit ? 1 : 0;
   A.fuse_advance = c->fusing ? 1 : 0;
   A.raw_ce = c->raw_now ? at<float2>(c, c->lay.ce) : nullptr;
+  if (c->hot_now) {
+    A.hot_amax = at<int>(c, c->tgt.lay.amax);
+    A.hot_flags = at<int>(c, c->tgt.lay.hot);
+    A.hot_means = c->tgt.den.means_dev;
+    A.hot_bf16 = c->tgt.den.means_dtype == SDS_BF16 ? 1 : 0;
+  }
   A.regen = c->regen_now ? 1 : 0;
   A.skip_x = c->skipx_now ? 1 : 0;
   A.seed = c->seed; A.chain_off = (uint64_t)c->chain_off;
@@ -376,7 +389,7 @@ TcGemmArgs tc_args(sds_ctx* c, Engine& e, const int* rowk, const int* nrows_dev,
 // run the target denoiser on dense rows X (and their bf16 copy Xb, NULL = make one); the row count
 // lives on the device (nrows_dev, may be NULL) with a host upper bound for the grids
 int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, const int* rowk, const int* nrows_dev,
-                 int64_t rows_ub, float* out, bool planes_ready = false, bool raw = false) {
+                 int64_t rows_ub, float* out, bool planes_ready = false, bool raw = false, bool indexed = false) {
   if (rows_ub <= 0) return SDS_OK;
   // timing kinds: the independent draft model's kernels are kept apart from the target's
   const bool is_drafter = &e == &c->drf;
@@ -420,10 +433,14 @@ int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, cons
         // the mixing contraction drop the three products with the other planes, tile by tile
         int* flags = at<int>(c, e.lay.flags);
         SDS_CU(c, cudaMemsetAsync(flags, 0, (((size_t)rows_ub + 255) / 256 * 2) * 4, c->stream));
+        // blocks of 256 rows whose rows are all one-hot skip the mixing contraction: their result is a copy of means
+        int* amax = c->onehot ? at<int>(c, e.lay.amax) : nullptr;
+        int* hot = c->onehot ? at<int>(c, e.lay.hot) : nullptr;
+        if (hot) SDS_CU(c, cudaMemsetAsync(hot, 0, (((size_t)rows_ub + 255) / 256) * 4, c->stream));
         SDS_LAUNCH(c, ks,
                    launch_softmax_split3(logits, nrows_dev, (int)rows_ub, (int)nc, (int)dd, X, means,
                                          at<double>(c, e.lay.musq), e.den.logw_dev, at<double>(c, e.lay.tcond), rowk,
-                                         cap * nc, Rs, flags, c->stream));
+                                         cap * nc, Rs, flags, amax, hot, c->stream));
         TcGemmArgs m = tc_args(c, e, rowk, nrows_dev, rows_ub);
         m.N = (int)dd; m.K = (int)nc; m.out = out; m.ldo = (int)dd;
         m.tcond = at<double>(c, e.lay.tcond); m.xrows = raw ? nullptr : X;
@@ -433,7 +450,11 @@ int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, cons
         m.tile_flags = flags; m.nseg_short = 3;
         m.tile_counts = at<int>(c, c->lay.ctl) + kCtlTilesFull;
         for (int i = 0; i < 3; ++i) { m.a_short[i] = kSa[i]; m.b_short[i] = kSb[i]; }
+        m.hot_flags = hot;
         SDS_LAUNCH(c, kd, launch_gemm_tc(kEpiGmmMix, m, Rs, Mt, c->stream));
+        if (hot && !indexed)    // (indexed: the readers of the rows take the skipped blocks' rows from the means themselves)
+          SDS_LAUNCH(c, ks, launch_mix_onehot(means, false, amax, hot, nrows_dev, (int)rows_ub, (int)dd,
+                                              at<double>(c, e.lay.tcond), rowk, raw ? nullptr : X, out, c->stream));
         return SDS_OK;
       }
       if (e.den.means_dtype == SDS_F32) {
@@ -458,11 +479,19 @@ int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, cons
       g.N = e.den.ncomp; g.K = c->d; g.out = logits; g.ldo = e.den.ncomp;
       g.tcond = at<double>(c, e.lay.tcond); g.musq = at<double>(c, e.lay.musq); g.logw = e.den.logw_dev;
       SDS_LAUNCH(c, kd, launch_gemm_tc(kEpiGmmLogits, g, Xb, means, c->stream));
-      SDS_LAUNCH(c, ks, launch_softmax_bf16(logits, nrows_dev, (int)rows_ub, e.den.ncomp, R, c->stream));
+      int* amax = c->onehot ? at<int>(c, e.lay.amax) : nullptr;
+      int* hot = c->onehot ? at<int>(c, e.lay.hot) : nullptr;
+      if (hot) SDS_CU(c, cudaMemsetAsync(hot, 0, (((size_t)rows_ub + 255) / 256) * 4, c->stream));
+      SDS_LAUNCH(c, ks, launch_softmax_bf16(logits, nrows_dev, (int)rows_ub, e.den.ncomp, R, amax, hot, c->stream));
       TcGemmArgs m = tc_args(c, e, rowk, nrows_dev, rows_ub);
       m.N = c->d; m.K = e.den.ncomp; m.out = out; m.ldo = c->d;
       m.tcond = at<double>(c, e.lay.tcond); m.xrows = raw ? nullptr : X;
+      m.hot_flags = hot;
+      m.tile_counts = is_drafter ? nullptr : at<int>(c, c->lay.ctl) + kCtlTilesFull;
       SDS_LAUNCH(c, kd, launch_gemm_tc(kEpiGmmMix, m, R, Mt, c->stream));
+      if (hot && !indexed)   // the skipped blocks: every row is a copy of one mean (with the same affine map as the epilogue's)
+        SDS_LAUNCH(c, ks, launch_mix_onehot(means, true, amax, hot, nrows_dev, (int)rows_ub, c->d,
+                                            at<double>(c, e.lay.tcond), rowk, raw ? nullptr : X, out, c->stream));
       return SDS_OK;
     }
     case SDS_DEN_MLP: {
@@ -745,7 +774,7 @@ int sds_verify_window(sds_ctx* c) {
   // rows drafted by k_draft (the two frozen-output modes) come with their bf16 planes
   const bool planes_ready = A.Xs != nullptr && (c->mode == SDS_FROZEN_PREV || c->mode == SDS_FROZEN_EXACT);
   const int rc = run_denoiser(c, c->tgt, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, (int64_t)c->ub * c->L, A.Dq, planes_ready,
-                              c->raw_now);
+                              c->raw_now, c->hot_now);
   if (rc != SDS_OK) return rc;
   SDS_LAUNCH(c, SDS_PROF_VERIFY, launch_verify(A, c->ub, c->stream));
   c->state = kVerified;
@@ -803,6 +832,9 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
                               (c->tgt.den.means_dtype == SDS_BF16 || (c->tensor_split && gmm_split_shape(c->tgt.den, c->d)));
       c->raw_now = c->raw_rows && tensor_mix && (c->mode == SDS_FROZEN_PREV || c->mode == SDS_FROZEN_EXACT) &&
                    verify_reads_raw_rows(A);
+      // ... and where every row of a block of 256 is one-hot, the block's accumulators are rows of the means table:
+      // nothing is stored for it, verify and advance read the means
+      c->hot_now = c->raw_now && c->onehot;
       // Frozen drafter whose target reads nothing but the bf16 copy of its input rows (the MLP; the bf16 mixture
       // with raw rows): the draft kernel stores only that copy, and verify, which then has no float rows to
       // read, makes the drafted states again from what it holds and advances its chains (it alone knows the
@@ -816,11 +848,11 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
       // where the register-resident verify kernel runs, it also advances its chains and compacts
       c->fusing = c->fuse_advance && (verify_can_advance(A) || c->regen_now);
       if (w == 0) {                                      // which of these paths the run takes (read back with the control words)
-        c->h_pin[48] = (c->regen_now ? 1 : 0);
+        c->h_pin[48] = (c->regen_now ? 1 : 0) | (c->hot_now ? 4 : 0);
         SDS_CU(c, cudaMemcpyAsync(A.ctl + kCtlPathFlags, c->h_pin + 48, 4, cudaMemcpyHostToDevice, c->stream));
       }
       rc = sds_draft(c);
-      if (rc != SDS_OK) { c->fusing = c->raw_now = c->regen_now = c->skipx_now = false; return rc; }
+      if (rc != SDS_OK) { c->fusing = c->raw_now = c->hot_now = c->regen_now = c->skipx_now = false; return rc; }
       rc = sds_verify_window(c);
       const bool fused_adv = c->fusing;
       c->fusing = false;
@@ -828,7 +860,7 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
         if (fused_adv) c->state = kReady;
         else rc = sds_advance(c, nullptr);
       }
-      c->raw_now = c->regen_now = c->skipx_now = false;
+      c->raw_now = c->hot_now = c->regen_now = c->skipx_now = false;
       if (rc != SDS_OK) return rc;
       SDS_CU(c, cudaMemcpyAsync(c->h_pin + 16 + (w & 1) * kCtlWords, A.ctl, kCtlWords * 4, cudaMemcpyDeviceToHost,
                                 c->stream));
@@ -968,6 +1000,7 @@ int sds_set_option(sds_ctx* c, int32_t option, int64_t value) {
     case SDS_OPT_FUSE_ADVANCE: c->fuse_advance = value != 0; return SDS_OK;
     case SDS_OPT_RAW_ROWS: c->raw_rows = value != 0; return SDS_OK;
     case SDS_OPT_REGEN_DRAFTS: c->regen = value != 0; return SDS_OK;
+    case SDS_OPT_ONEHOT_ROWS: c->onehot = value != 0; return SDS_OK;
     default: return SDS_EINVAL;
   }
 }

@@ -26,9 +26,10 @@ enum Ctl : int {
   kCtlSpare1 = 7,
   kCtlTilesFull = 8,  // mixing-GEMM tiles of the split-precision mixture run with all six products since reset
   kCtlTilesBrief = 9, // ... and with the three products of the first plane only
-  kCtlPositions = 10, // window positions whose accept test the verify kernels evaluated since reset (wraps at 2^31)
+  kCtlTilesSkipped = 10, // mixing-GEMM tiles skipped since reset because every row of their block was one-hot
   kCtlPathFlags = 11, // how the last sds_sample_all ran its windows: bit 0 verify drew the drafted states again,
                       // bit 1 the drafted noise was kept in the workspace between windows (written by the host)
+  kCtlPositions = 12, // window positions whose accept test the verify kernels evaluated since reset (wraps at 2^31)
   kCtlWords = 16
 };
 constexpr int kErrNonFinite = 1;
@@ -206,6 +207,16 @@ __device__ __forceinline__ void delta_z_any(bool mean, float wp, float wj, float
 // target output from a stored accumulator (rows kept raw by the mixing contraction): C acc + E x
 __device__ __forceinline__ float4 affine_row4(float cC, float cE, float4 acc, float4 x) {
   return make_float4(fmaf(cC, acc.x, cE * x.x), fmaf(cC, acc.y, cE * x.y), fmaf(cC, acc.z, cE * x.z), fmaf(cC, acc.w, cE * x.w));
+}
+
+// four consecutive elements of a mixture's mean row, float or bf16 table
+__device__ __forceinline__ float4 mean_row4(const void* means, bool bf16, size_t off) {
+  if (bf16) {
+    const uint2 w = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(means) + off));
+    return make_float4(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xffff0000u), __uint_as_float(w.y << 16),
+                       __uint_as_float(w.y & 0xffff0000u));
+  }
+  return __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(means) + off));
 }
 
 // reflected state: m^q + sigma (Z - coef * Delta), coef = 2 (Delta.Z)/|Delta|^2

@@ -15,6 +15,12 @@ struct WinArgs {
   double inv_tau;        // 1 / temperature of the accept test (1 = the exact method)
   const float2* raw_ce;  // non-NULL: Dq holds the mixing contraction's accumulators; the target output of row r
                          // (input X[r], step k = rowk[r]) is fma(C_k, Dq[r], E_k X[r]) with (C_k, E_k) = raw_ce[k]
+  // with raw_ce, rows of blocks the mixing contraction skipped (every row one-hot) are not stored at all: the
+  // accumulator of row r is the mean of component hot_amax[r], read from the mixture's own table
+  const int* hot_amax;   // [B*L] component of every one-hot row (NULL: every row is in Dq)
+  const int* hot_flags;  // [B*L/256] zero = the block of 256 rows was skipped
+  const void* hot_means; // [ncomp, d] float or bf16
+  int hot_bf16;
   int fuse_advance;      // the verify kernel also advances its chain and the last CTA compacts (no advance launch)
   int early_exit;        // verify stops reading a chain's window after the block of positions that holds its first
                          // rejection (d >= 2048: the first position, then pairs; below: fours; large-d kernels only)

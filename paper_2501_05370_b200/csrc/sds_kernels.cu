@@ -119,6 +119,7 @@ __global__ void __launch_bounds__(kBlock) k_init(WinArgs A) {
     A.ctl[kCtlTilesFull] = 0;
     A.ctl[kCtlTilesBrief] = 0;
     A.ctl[kCtlPositions] = 0;
+    A.ctl[kCtlTilesSkipped] = 0;
   }
   if (b >= A.B) return;
   const uint64_t bg = A.chain_off + (uint64_t)b;
@@ -671,6 +672,19 @@ __device__ __forceinline__ float4 redraft4(const WinArgs& A, float4 y, float4 dc
   return y;
 }
 
+// Rows kept raw (the mixing contraction's accumulators): the component whose mean IS row r's accumulator
+// when the row's block of 256 rows was skipped by the contraction (every row one-hot), else -1 (the row is
+// in Dq). Uniform over the threads that share a row.
+__device__ __forceinline__ int raw_row_component(const WinArgs& A, int r) {
+  if (!A.hot_amax) return -1;
+  return (__ldg(A.hot_flags + (r >> 8)) == 0) ? __ldg(A.hot_amax + r) : -1;
+}
+// elements i .. i+3 of row r's accumulator
+__device__ __forceinline__ float4 raw_row4(const WinArgs& A, int r, int comp, int i) {
+  if (comp >= 0) return mean_row4(A.hot_means, A.hot_bf16 != 0, (size_t)comp * A.d + i);
+  return ld4(A.Dq + (size_t)r * A.d + i);
+}
+
 // Register-resident variant for d % 4 == 0 and d <= 4 * EPT * TPC: each thread keeps its slice of
 // the carried output and of the previous drafted state in registers, so every position reads only
 // its own drafted state and target output from memory (8d bytes per verified step), with 2*EPT
@@ -733,13 +747,13 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t,
       const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
       const float inv_s = 1.0f / sk, cs = ck * inv_s;
       const float* wj = (j < Lt) ? A.X + (size_t)(r0 + j) * A.d : A.T + cb;
-      const float* dq = A.Dq + (size_t)(r0 + j - 1) * A.d;
+      const int qcomp = raw_row_component(A, r0 + j - 1);
       float4 vj[REGEN ? 1 : EPT], vq[EPT];
 #pragma unroll
       for (int e = 0; e < EPT; ++e) {
         const int i = (t + e * TPC) * 4;
         if (!REGEN) vj[REGEN ? 0 : e] = (i < A.d) ? ld4(wj + i) : zero4;
-        vq[e] = (i < A.d) ? ld4(dq + i) : zero4;
+        vq[e] = (i < A.d) ? raw_row4(A, r0 + j - 1, qcomp, i) : zero4;
         if (A.Dp && i < A.d) vc[e] = ld4(A.Dp + (size_t)(r0 + j - 1) * A.d + i);   // independent draft model
       }
       if (A.raw_ce) {                    // rows kept raw: the row's input W_{j-1} is in registers already
@@ -851,7 +865,7 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t,
           const int i = (t + e * TPC) * 4;
           if (i < A.d) {
             st4(A.Y + cb + i, REGEN ? vp[e] : ld4(A.T + cb + i));   // REGEN: every block ran, vp holds W_Lt
-            float4 q = ld4(A.Dq + (size_t)(r0 + Lt - 1) * A.d + i);
+            float4 q = raw_row4(A, r0 + Lt - 1, raw_row_component(A, r0 + Lt - 1), i);
             if (A.raw_ce) {
               const float2 ce = __ldg(A.raw_ce + nb + Lt - 1);
               const float4 x = REGEN ? redraft4(A, ld4(snap + i), vc[e], bg, nb, snap_pos, Lt - 1, (uint32_t)(t + e * TPC))
@@ -877,7 +891,7 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t,
   const float inv_s = 1.0f / sk, cs = ck * inv_s;
   const float* wp = A.X + (size_t)(r0 + jstar - 1) * A.d;
   float* wj = (jstar < Lt) ? A.X + (size_t)(r0 + jstar) * A.d : A.T + cb;
-  const float* dq = A.Dq + (size_t)(r0 + jstar - 1) * A.d;
+  const int rcomp = raw_row_component(A, r0 + jstar - 1);
 #pragma unroll
   for (int e = 0; e < EPT; ++e) {
     const int i = (t + e * TPC) * 4;
@@ -888,7 +902,7 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t,
       const float4 w = !REGEN ? ld4(wj + i)
                        : (jstar == done) ? vp[e]
                        : draft_step4(p, vc[e], normal4(A.seed, kStreamDraft, bg, (uint32_t)k, (uint32_t)(t + e * TPC)), ak, ck, sk);
-      float4 q = ld4(dq + i);
+      float4 q = raw_row4(A, r0 + jstar - 1, rcomp, i);
       if (A.raw_ce) {
         const float2 ce = __ldg(A.raw_ce + k);
         q = affine_row4(ce.x, ce.y, q, p);
@@ -942,6 +956,7 @@ __global__ void __launch_bounds__(kBlock) k_advance(WinArgs A) {
       const int adv = min(js, Lt);
       const float* src = (adv < Lt) ? A.X + (size_t)(r0 + adv) * A.d : A.T + cb;
       const float* dsrc = A.Dq + (size_t)(r0 + adv - 1) * A.d;
+      const int dcomp = raw_row_component(A, r0 + adv - 1);
       if (VEC == 4) {
         // four iterations' loads are issued before their stores (eight 128-bit loads in flight)
         for (int i0 = t * 4; i0 < A.d; i0 += TPC * 16) {
@@ -951,7 +966,7 @@ __global__ void __launch_bounds__(kBlock) k_advance(WinArgs A) {
             const int i = i0 + u * TPC * 4;
             if (i < A.d) {
               vy[u] = ld4(src + i);
-              vd[u] = ld4(dsrc + i);
+              vd[u] = raw_row4(A, r0 + adv - 1, dcomp, i);
               if (A.raw_ce) {
                 const float2 ce = __ldg(A.raw_ce + nb + adv - 1);
                 vd[u] = affine_row4(ce.x, ce.y, vd[u], ld4(A.X + (size_t)(r0 + adv - 1) * A.d + i));

@@ -31,15 +31,19 @@ constexpr int kEpiWarps = 8;       // two warps per TMEM lane quarter, each take
 constexpr int kThreads = 64 + 32 * kEpiWarps;   // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..9: epilogue
 constexpr uint32_t kSpinCap = 1u << 22;
 
-template <int BN, bool PAIR> struct TileCfg {
-  static constexpr int kStages = PAIR ? 6 : ((BN == 256) ? 4 : 6);
+template <int BN, bool PAIR, int EPI> struct TileCfg {
+  // the logits epilogue writes whole rows from registers and needs no staging tile: its shared memory
+  // holds one more operand stage instead (the main loop is bound by the bytes in flight)
+  static constexpr bool kStaged = EPI != kEpiGmmLogits;
   static constexpr int kBRows = PAIR ? BN / 2 : BN;                         // rows of B one CTA stages
   static constexpr int kABytes = BM * BK * 2;
   static constexpr int kBBytes = kBRows * BK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kStages = (kStageBytes == 32 * 1024) ? (kStaged ? 6 : 7) : 4;
   static constexpr int kTmemCols = 2 * BN;                                  // two accumulator buffers
-  static constexpr int kEpiStageBytes = kEpiWarps * 32 * 33 * 4;            // one padded 32x32 float tile per epilogue warp
+  static constexpr int kEpiStageBytes = kStaged ? kEpiWarps * 32 * 33 * 4 : 0;   // one padded 32x32 float tile per epilogue warp
   static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/ + kEpiStageBytes;
+  static_assert(kSmemBytes <= 227 * 1024, "shared memory of one CTA");
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -231,12 +235,21 @@ __device__ __forceinline__ bool tile_is_brief(const TcGemmArgs& g, int tm) {
   return f == 0;
 }
 
+// whether tile row `tm` is left to the one-hot gather: every one of its rows has a single non-zero
+// responsibility (hot_flags holds one word per 256 rows, zero = all one-hot), so the product is a copy of
+// one row of B per row and no tensor work is needed
+template <int TM>
+__device__ __forceinline__ bool tile_is_skipped(const TcGemmArgs& g, int tm) {
+  if (!g.hot_flags) return false;
+  return __ldg(g.hot_flags + (TM == 256 ? tm : (tm >> 1))) == 0;
+}
+
 template <int BN, int EPI, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
     k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
               const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB0,
               const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, TcGemmArgs g) {
-  using C = TileCfg<BN, PAIR>;
+  using C = TileCfg<BN, PAIR, EPI>;
   constexpr int TM = PAIR ? 2 * BM : BM;               // rows of one tile (of the pair's tile)
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte aligned operand stages (required by the 128-byte swizzle), barriers behind them
@@ -295,6 +308,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       bool ok = true;
       const uint32_t leader_full0 = PAIR ? map_to_cta(smem_u32(full_bar), 0u) : 0u;
       for (int t = worker; t < total_tiles && ok; t += nworkers) {
+        if (EPI == kEpiGmmMix && tile_is_skipped<TM>(g, t / n_tiles)) continue;
         const int m0 = (t / n_tiles) * TM + (int)rank * BM, n0 = (t % n_tiles) * BN + (int)rank * C::kBRows;
         const bool brief = tile_is_brief<TM>(g, t / n_tiles);
         const int nkb = brief ? kb_seg * g.nseg_short : kblocks;
@@ -332,9 +346,14 @@ __global__ void __launch_bounds__(kThreads, 1)
       uint32_t phase = 0;
       int it = 0;
       bool ok = true;
-      for (int t = worker; t < total_tiles && ok; t += nworkers, ++it) {
+      for (int t = worker; t < total_tiles && ok; t += nworkers) {
+        if (EPI == kEpiGmmMix && tile_is_skipped<TM>(g, t / n_tiles)) {
+          if (g.tile_counts && (t % n_tiles) == 0) atomicAdd(g.tile_counts + 2, n_tiles);
+          continue;
+        }
         const int buf = it & 1;
         const uint32_t bphase = (uint32_t)(it >> 1) & 1u;
+        ++it;
         if (!mbar_wait(tempty_bar + buf, bphase ^ 1u, abort_s)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
@@ -371,9 +390,11 @@ __global__ void __launch_bounds__(kThreads, 1)
     bool ok = true;
     // "drained" goes to the leader's barrier (the MMA issuer of the pair waits there)
     const uint32_t drained0 = (PAIR && rank != 0) ? map_to_cta(smem_u32(tempty_bar), 0u) : 0u;
-    for (int t = worker; t < total_tiles && ok; t += nworkers, ++it) {
+    for (int t = worker; t < total_tiles && ok; t += nworkers) {
+      if (EPI == kEpiGmmMix && tile_is_skipped<TM>(g, t / n_tiles)) continue;
       const int buf = it & 1;
       const uint32_t bphase = (uint32_t)(it >> 1) & 1u;
+      ++it;
       const int m0 = (t / n_tiles) * TM + (int)rank * BM, n0 = (t % n_tiles) * BN + half * kCols;
       const int row = m0 + q * 32 + lane;
       const bool live = row < M;
@@ -515,9 +536,14 @@ __global__ void __launch_bounds__(kThreads, 1)
 // helpers around the GEMMs of the large mixture
 // ------------------------------------------------------------------------------------------
 
-// softmax over ncomp logits per row -> normalised responsibilities in bf16
+// softmax over ncomp logits per row -> normalised responsibilities in bf16. Weights below 2^-40 of
+// the row are dropped (stored as exact zeros; they change no stored bit of the mixing sum's float
+// result). A row left with a single non-zero weight is one-hot: its weight is exactly 1, its mixing sum is
+// a copy of that component's mean. amax[row] gets the component of a one-hot row (-1 otherwise) and
+// hot_flags[row / 256] is raised for every block of 256 rows that holds a row which is not one-hot.
 __global__ void __launch_bounds__(256) k_softmax_bf16(const float* __restrict__ logits, const int* __restrict__ nrows_dev,
-                                                      int rows_host, int ncomp, uint16_t* __restrict__ R) {
+                                                      int rows_host, int ncomp, uint16_t* __restrict__ R,
+                                                      int* __restrict__ amax, int* __restrict__ hot_flags) {
   const int nrows = nrows_dev ? min(*nrows_dev, rows_host) : rows_host;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int row = blockIdx.x * 8 + warp; row < nrows; row += gridDim.x * 8) {
@@ -529,9 +555,67 @@ __global__ void __launch_bounds__(256) k_softmax_bf16(const float* __restrict__ 
     for (int c = lane; c < ncomp; c += 32) den += expf(lg[c] - mx);
     den = warp_sum(den);
     const float inv = 1.0f / den;
+    int nnz = 0, cmax = ncomp;
     for (int c = lane * 2; c < ncomp; c += 64) {
-      const float a = expf(lg[c] - mx) * inv, b = expf(lg[c + 1] - mx) * inv;
+      float a = expf(lg[c] - mx) * inv, b = expf(lg[c + 1] - mx) * inv;
+      if (a < 0x1p-40f) a = 0.f;
+      if (b < 0x1p-40f) b = 0.f;
+      nnz += (a != 0.f) + (b != 0.f);
+      if (lg[c] == mx) cmax = min(cmax, c);
+      if (lg[c + 1] == mx) cmax = min(cmax, c + 1);
       *reinterpret_cast<uint32_t*>(R + (size_t)row * ncomp + c) = pack_bf16x2(a, b);
+    }
+    if (amax) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        nnz += __shfl_xor_sync(0xffffffffu, nnz, o);
+        cmax = min(cmax, __shfl_xor_sync(0xffffffffu, cmax, o));
+      }
+      if (lane == 0) {
+        amax[row] = (nnz == 1) ? cmax : -1;
+        if (nnz != 1 && hot_flags) hot_flags[row >> 8] = 1;
+      }
+    }
+  }
+}
+
+// Rows whose responsibilities are one-hot, in blocks of 256 rows that the mixing GEMM skipped (hot_flags
+// zero): the mixing sum is the component's mean itself. out[row] = means[amax[row]] (raw accumulator
+// form) or C_k means[amax[row]] + E_k x[row] when xrows is given, the same operations as the GEMM's
+// epilogue applies, hence the same bits as the product with an exact one-hot row.
+template <bool BF16>
+__global__ void __launch_bounds__(256) k_mix_onehot(const void* __restrict__ means, const int* __restrict__ amax,
+                                                     const int* __restrict__ hot_flags, const int* __restrict__ nrows_dev,
+                                                     int rows_host, int d, const double* __restrict__ tcond,
+                                                     const int* __restrict__ rowk, const float* __restrict__ xrows,
+                                                     float* __restrict__ out, int rows_per_cta) {
+  const int nrows = nrows_dev ? min(*nrows_dev, rows_host) : rows_host;
+  const int tpr = 256 / rows_per_cta;                       // threads per row
+  const int sub = threadIdx.x / tpr, t = threadIdx.x % tpr;
+  for (int row = blockIdx.x * rows_per_cta + sub; row < nrows; row += gridDim.x * rows_per_cta) {
+    if (__ldg(hot_flags + (row >> 8)) != 0) continue;        // this block went through the GEMM
+    const int c = __ldg(amax + row);
+    if (c < 0) continue;                                     // (cannot happen in a block whose flag is clear)
+    float cC = 1.f, cE = 0.f;
+    if (xrows) {
+      const int k = __ldg(rowk + row);
+      cC = (float)__ldg(tcond + 4 * k + 2);
+      cE = (float)__ldg(tcond + 4 * k + 3);
+    }
+    float* o = out + (size_t)row * d;
+    for (int i = t * 4; i < d; i += tpr * 4) {
+      float4 m;
+      if (BF16) {
+        const uint2 w = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(means) + (size_t)c * d + i));
+        m = make_float4(bf16_lo(w.x), bf16_hi(w.x), bf16_lo(w.y), bf16_hi(w.y));
+      } else {
+        m = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(means) + (size_t)c * d + i));
+      }
+      if (xrows) {
+        const float4 x = ld4(xrows + (size_t)row * d + i);
+        m = make_float4(fmaf(cC, m.x, cE * x.x), fmaf(cC, m.y, cE * x.y), fmaf(cC, m.z, cE * x.z), fmaf(cC, m.w, cE * x.w));
+      }
+      st4(o + i, m);
     }
   }
 }
@@ -603,7 +687,8 @@ __global__ void __launch_bounds__(256)
                      const float* __restrict__ X, const float* __restrict__ means,
                      const double* __restrict__ musq, const float* __restrict__ logw,
                      const double* __restrict__ tcond, const int* __restrict__ rowk, size_t rplane,
-                     uint16_t* __restrict__ R, int* __restrict__ tile_flags) {
+                     uint16_t* __restrict__ R, int* __restrict__ tile_flags, int* __restrict__ amax,
+                     int* __restrict__ hot_flags) {
   constexpr int ncomp = 128 * NQ;
   const int nrows = nrows_dev ? min(*nrows_dev, rows_host) : rows_host;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -666,6 +751,7 @@ __global__ void __launch_bounds__(256)
     den = warp_sum(den);
     const float inv = 1.0f / den;
     uint32_t lower = 0u;                          // any non-zero entry in the second or third plane of this row
+    int nnz = 0, cmax = ncomp;                    // non-zero weights of the row; its largest component
 #pragma unroll
     for (int q = 0; q < NQ; ++q) {
       uint16_t p[3][4];
@@ -673,6 +759,8 @@ __global__ void __launch_bounds__(256)
       for (int u = 0; u < 4; ++u) {
         float r = v[q][u] * inv;
         if (r < 0x1p-40f) r = 0.f;               // below 1e-12 of the row: dropped (keeps one-hot rows exactly one-hot)
+        nnz += (r != 0.f);
+        if (v[q][u] == 1.0f) cmax = min(cmax, 4 * (lane + 32 * q) + u);   // exp(0): the row maximum
         split3(r, p[0][u], p[1][u], p[2][u]);
         lower |= (uint32_t)p[1][u] | (uint32_t)p[2][u];
       }
@@ -683,6 +771,17 @@ __global__ void __launch_bounds__(256)
                                                                     (uint32_t)p[pl][2] | ((uint32_t)p[pl][3] << 16));
     }
     if (tile_flags && __any_sync(0xffffffffu, lower != 0u) && lane == 0) tile_flags[row >> 7] = 1;
+    if (amax) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        nnz += __shfl_xor_sync(0xffffffffu, nnz, o);
+        cmax = min(cmax, __shfl_xor_sync(0xffffffffu, cmax, o));
+      }
+      if (lane == 0) {
+        amax[row] = (nnz == 1) ? cmax : -1;
+        if (nnz != 1 && hot_flags) hot_flags[row >> 8] = 1;
+      }
+    }
   }
 }
 
@@ -727,7 +826,7 @@ bool make_tmap(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t K, uin
 
 template <int BN, int EPI, bool PAIR>
 cudaError_t launch_t(const TcGemmArgs& g, const void* A, const void* B, int grid_tiles_ub, cudaStream_t st) {
-  using C = TileCfg<BN, PAIR>;
+  using C = TileCfg<BN, PAIR, EPI>;
   CUtensorMap tmA[3], tmB[3];
   for (int i = 0; i < 3; ++i) {
     const uint16_t* a = static_cast<const uint16_t*>(A) + (size_t)i * g.a_plane;
@@ -807,11 +906,25 @@ cudaError_t launch_gemm_tc(int epi, const TcGemmArgs& g_in, const void* A_bf16, 
 }
 
 cudaError_t launch_softmax_bf16(const float* logits, const int* nrows_dev, int rows_host, int ncomp, uint16_t* R,
-                                cudaStream_t st) {
+                                int* amax, int* hot_flags, cudaStream_t st) {
   int blocks = (rows_host + 7) / 8;
   if (blocks > 148 * 8) blocks = 148 * 8;
   if (blocks < 1) blocks = 1;
-  k_softmax_bf16<<<blocks, 256, 0, st>>>(logits, nrows_dev, rows_host, ncomp, R);
+  k_softmax_bf16<<<blocks, 256, 0, st>>>(logits, nrows_dev, rows_host, ncomp, R, amax, hot_flags);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_mix_onehot(const void* means, bool means_bf16, const int* amax, const int* hot_flags,
+                              const int* nrows_dev, int rows_host, int d, const double* tcond, const int* rowk,
+                              const float* xrows, float* out, cudaStream_t st) {
+  if (d % 4 != 0) return cudaErrorInvalidValue;
+  // short rows: several rows per CTA so that every thread still has a 128-bit access to make
+  const int rows_per_cta = d >= 4096 ? 1 : (d >= 2048 ? 2 : (d >= 1024 ? 4 : 8));
+  int blocks = (rows_host + rows_per_cta - 1) / rows_per_cta;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  if (means_bf16) k_mix_onehot<true><<<blocks, 256, 0, st>>>(means, amax, hot_flags, nrows_dev, rows_host, d, tcond, rowk, xrows, out, rows_per_cta);
+  else k_mix_onehot<false><<<blocks, 256, 0, st>>>(means, amax, hot_flags, nrows_dev, rows_host, d, tcond, rowk, xrows, out, rows_per_cta);
   return cudaGetLastError();
 }
 
@@ -842,14 +955,14 @@ cudaError_t launch_split3(const float* x, size_t n, size_t plane, int nplanes, u
 cudaError_t launch_softmax_split3(const float* logits, const int* nrows_dev, int rows_host, int ncomp, int d,
                                   const float* X, const float* means, const double* musq, const float* logw,
                                   const double* tcond, const int* rowk, size_t rplane, uint16_t* R, int* tile_flags,
-                                  cudaStream_t st) {
+                                  int* amax, int* hot_flags, cudaStream_t st) {
   int blocks = (rows_host + 7) / 8;
   if (blocks > 148 * 8) blocks = 148 * 8;
   if (blocks < 1) blocks = 1;
 #define SDS_SM3(NQ)                                                                                              \
   case NQ:                                                                                                       \
     k_softmax_split3<NQ><<<blocks, 256, 0, st>>>(logits, nrows_dev, rows_host, d, X, means, musq, logw, tcond,   \
-                                                 rowk, rplane, R, tile_flags);                                   \
+                                                 rowk, rplane, R, tile_flags, amax, hot_flags);                  \
     break;
   switch (ncomp / 128) {
     SDS_SM3(1) SDS_SM3(2) SDS_SM3(3) SDS_SM3(4) SDS_SM3(5) SDS_SM3(6) SDS_SM3(7) SDS_SM3(8)

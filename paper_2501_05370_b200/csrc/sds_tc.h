@@ -40,15 +40,25 @@ struct TcGemmArgs {
   // every row block of a tile means planes 1.. of A are all zero there, and the tile runs the
   // nseg_short segments a_short/b_short instead (the products left out are exact zeros)
   const int* tile_flags;
-  int* tile_counts;      // optional: [0] += tiles run with the full list, [1] += tiles run with the short one
+  // optional (mixing epilogue): one word per 256 rows of A, zero = every row of the block has a single non-zero
+  // entry; tiles of such blocks are skipped altogether (launch_mix_onehot writes their rows)
+  const int* hot_flags;
+  int* tile_counts;      // optional: [0] += tiles run with the full list, [1] += tiles run with the short one,
+                         // [2] += tiles skipped
   int nseg_short;
   uint8_t a_short[8], b_short[8];
 };
 
 bool tc_shape_ok(int N, int K);
 cudaError_t launch_gemm_tc(int epi, const TcGemmArgs& g, const void* A_bf16, const void* B_bf16, cudaStream_t st);
+// amax / hot_flags (both optional): component of every one-hot row (-1 otherwise); one word per 256 rows,
+// zeroed by the caller, raised where a row is not one-hot
 cudaError_t launch_softmax_bf16(const float* logits, const int* nrows_dev, int rows_host, int ncomp, uint16_t* R,
-                                cudaStream_t st);
+                                int* amax, int* hot_flags, cudaStream_t st);
+// rows of the blocks the mixing GEMM skipped: out[row] = means[amax[row]], or C means + E x when xrows is given
+cudaError_t launch_mix_onehot(const void* means, bool means_bf16, const int* amax, const int* hot_flags,
+                              const int* nrows_dev, int rows_host, int d, const double* tcond, const int* rowk,
+                              const float* xrows, float* out, cudaStream_t st);
 cudaError_t launch_transpose_bf16(const uint16_t* M, int ncomp, int d, uint16_t* Mt, cudaStream_t st);
 cudaError_t launch_musq_bf16(const uint16_t* means, int ncomp, int d, double* musq, cudaStream_t st);
 cudaError_t launch_wait_selftest(uint32_t polls, int* status_dev, cudaStream_t st);
@@ -59,7 +69,7 @@ cudaError_t launch_split3(const float* x, size_t n, size_t plane, int nplanes, u
 cudaError_t launch_softmax_split3(const float* logits, const int* nrows_dev, int rows_host, int ncomp, int d,
                                   const float* X, const float* means, const double* musq, const float* logw,
                                   const double* tcond, const int* rowk, size_t rplane, uint16_t* R, int* tile_flags,
-                                  cudaStream_t st);
+                                  int* amax, int* hot_flags, cudaStream_t st);
 cudaError_t launch_f32_to_bf16(const float* x, size_t n, uint16_t* out, cudaStream_t st);
 
 }  // namespace sds
