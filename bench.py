@@ -360,7 +360,7 @@ def kernel_rooflines(w, variant, prof, steps, rows, cw, positions, pk, ctl, traf
     total_ms = sum(v[0] for v in kinds.values())
     bf16_rows = w.denoiser == "mlp" or (w.denoiser == "gmm" and w.gmm.get("means_bf16"))
     split = tensor_mixture(w) and not w.gmm.get("means_bf16")
-    regen, cached = launch_shape.get("regen", False), launch_shape.get("noise_cache", False)
+    regen = launch_shape.get("regen", False)
     out = []
     for kind, (ms, n) in sorted(kinds.items(), key=lambda kv: -kv[1][0]):
         if kind in ("init", "aux"):
@@ -369,36 +369,33 @@ def kernel_rooflines(w, variant, prof, steps, rows, cw, positions, pk, ctl, traf
         avg_s = ms / n * 1e-3
         e = {"kernel": kind, "launches_per_step": per_run_launches, "avg_launch_us": avg_s * 1e6,
              "ms_per_step": ms / steps, "share_of_kernel_time": ms / max(total_ms, 1e-9)}
-        if kind in ("denoise", "fused", "draft_model"):
+        if kind in ("denoise", "fused", "draft_model", "mix"):
             if w.denoiser == "phi4":
                 bound, per_run = "alu", 12.0 * d * (rows + B)
             elif w.denoiser == "mlp":
                 bound, per_run = "tensor", 2.0 * sum(w.mlp_dims[i] * w.mlp_dims[i + 1] for i in range(len(w.mlp_dims) - 1)) * (rows + B)
-            else:
-                per_run = 4.0 * w.gmm["ncomp"] * d * (rows + B)
-                bound = "tensor" if (kind == "denoise" and tensor_mixture(w)) else "alu"
-                if bound == "tensor":
-                    # mixing tiles of blocks whose rows are all one-hot are not computed at all (a copy kernel writes
-                    # those rows): only the contraction work that ran counts as achieved
+            elif tensor_mixture(w) and kind in ("denoise", "mix"):
+                # two contractions of 2 ncomp d flop per row each: "denoise" times the logits GEMM, "mix" the mixing
+                # GEMM, whose tiles are not computed where every row of a block is one-hot (a row of the means table
+                # is read instead): only the contraction work that ran counts as achieved
+                bound, per_run = "tensor", 2.0 * w.gmm["ncomp"] * d * (rows + B)
+                if kind == "mix":
                     ran, skipped = int(ctl[8]) + int(ctl[9]), int(ctl[10])
-                    mix_done = ran / max(1, ran + skipped)
-                    per_run *= 0.5 * (1.0 + mix_done)
-                    e["mixing_tiles_skipped_frac"] = 1.0 - mix_done
+                    per_run *= ran / max(1, ran + skipped)
+                    e["mixing_tiles_skipped_frac"] = skipped / max(1, ran + skipped)
+            else:
+                bound, per_run = "alu", 4.0 * w.gmm["ncomp"] * d * (rows + B)
             if kind == "draft_model":
                 bound, per_run = "alu", 4.0 * max(1, w.gmm["ncomp"] // 2) * d * rows
             peak, unit, src = (tens, "TFLOP/s", pk["source"] + " (sustained bf16 GEMM)") if bound == "tensor" else \
                               (alu_peak, "TFLOP/s", "derived: 148 SMs x 128 fp32 lanes x 2 x max SM clock")
             if bound == "tensor" and split:
-                # float operands as bf16 planes: 3 bf16 products per float product in the logits, 6 in the
-                # mixing (3 for tiles whose responsibilities need only their first plane; the library counts both),
-                # weighted by the contraction work that ran (the logits always, the mixing where it was not skipped)
+                # float operands as bf16 planes: 3 bf16 products per float product in the logits, 6 in the mixing
+                # (3 for tiles whose responsibilities need only their first plane; the library counts both)
                 t_full, t_brief = int(ctl[8]), int(ctl[9])
-                mix = (6.0 * t_full + 3.0 * t_brief) / max(1, t_full + t_brief)
-                f_mix = e.get("mixing_tiles_skipped_frac")
-                f_mix = 1.0 if f_mix is None else 1.0 - f_mix
-                products = (3.0 + mix * f_mix) / (1.0 + f_mix)
+                products = 3.0 if kind == "denoise" else (6.0 * t_full + 3.0 * t_brief) / max(1, t_full + t_brief)
                 peak = tens / products
-                src = pk["source"] + f" (sustained bf16 GEMM / {products:.2f} bf16 products per float product; {t_brief} of {t_full + t_brief} mixing tiles run on one plane)"
+                src = pk["source"] + f" (sustained bf16 GEMM / {products:.2f} bf16 products per float product)"
             ach = per_run / (ms / steps * 1e-3) / 1e12
             e.update(bound=bound, achieved=ach, peak=peak, unit=unit, frac=ach / peak, peak_source=src,
                      algorithmic_per_launch=per_run / per_run_launches)
@@ -406,10 +403,11 @@ def kernel_rooflines(w, variant, prof, steps, rows, cw, positions, pk, ctl, traf
             if kind == "verify":
                 per_run = 8.0 * d * rows                         # two float streams per window position
                 # requested: per evaluated position the target row (and the drafted state unless it is made
-                # again in registers or read from the noise cache), per chain-window the state, the carried
-                # output, the reflected row's inputs again and the two rows the advance step writes
-                per_pos = 4.0 * d if regen else 8.0 * d
-                req = per_pos * positions + (8.0 * d + 4.0 * d + 8.0 * d) * cw
+                # again in registers), per chain-window the state, the carried output, the reflected row's
+                # inputs again and the two rows the advance step writes
+                pos_regen = min(positions, float(int(ctl[13]) & 0x7fffffff))   # positions verified with the states made again
+                req = 8.0 * d * (positions - pos_regen) + 4.0 * d * pos_regen + (8.0 * d + 4.0 * d + 8.0 * d) * cw
+                e["positions_with_states_made_again"] = pos_regen
                 e.update(positions_evaluated_per_step=positions, requested_bytes_per_launch=req / per_run_launches,
                          requested_achieved=req / (ms / steps * 1e-3) / 1e9,
                          requested_frac=req / (ms / steps * 1e-3) / 1e9 / hbm)
@@ -417,10 +415,20 @@ def kernel_rooflines(w, variant, prof, steps, rows, cw, positions, pk, ctl, traf
                 rows_w = 4.0 * d * rows + (2.0 * d * rows if bf16_rows else 0.0) + (4.0 * d * rows if split else 0.0)
                 per_run = 8.0 * d * cw + rows_w
                 # stored by this implementation: the float rows are skipped where nothing reads them
-                moved = 8.0 * d * cw + (2.0 * d * (rows - cw) if (regen and bf16_rows) else rows_w)
+                rows_float = min(rows, float(int(ctl[14]) & 0x7fffffff))       # drafted rows also stored as floats
+                moved = (8.0 * d * cw + rows_w - 4.0 * d * (rows - rows_float)) if bf16_rows else (8.0 * d * cw + rows_w)
                 e.update(requested_bytes_per_launch=moved / per_run_launches,
                          requested_achieved=moved / (ms / steps * 1e-3) / 1e9,
                          requested_frac=moved / (ms / steps * 1e-3) / 1e9 / hbm)
+                # the generator, not memory, bounds this kernel: Philox-4x32-10 takes forty 32 x 32-bit multiplies per
+                # four normals; derived peak: 64 such multiplies per clock and SM (half the 128 fp32 lanes) x 148 SMs
+                drawn = d * (rows - (cw if regen else 0.0))                         # normals per run (about: the last row of a
+                                                                                    # window is not drafted where verify makes it)
+                mult = 10.0 * drawn
+                int_peak = SMS * 64 * pk["sm_max_mhz"] * 1e6
+                e["integer_multiplier"] = {"multiplies_per_launch": mult / per_run_launches,
+                                           "achieved_per_s": mult / (ms / steps * 1e-3), "derived_peak_per_s": int_peak,
+                                           "frac": mult / (ms / steps * 1e-3) / int_peak}
             elif kind == "advance":
                 per_run = 16.0 * d * cw
             elif kind == "softmax":
@@ -703,10 +711,8 @@ def run_gpu(args, w):
     e2e_value = world * B * K / (ms_e2e / steps * 1e-3)
     rows_per_step, windows_chains = run_counts(w, args.variant, calls_np, rows_np)
     positions = float(int(ctl[12]) & 0x7fffffff) if prof.get("verify", (0, 0))[1] > 0 else 0.0   # of the last run
-    launch_shape = {"regen": bool(int(ctl[11]) & 1), "noise_cache": bool(int(ctl[11]) & 2)}
-    traffic = measured_traffic() if not args.chains else {}
-    if args.chains:                                     # a reduced batch: scale the captures to it all the same
-        traffic = measured_traffic()
+    launch_shape = {"regen": bool(int(ctl[11]) & 1), "indexed_one_hot_rows": bool(int(ctl[11]) & 4)}
+    traffic = measured_traffic()                        # captured at a reduced batch, scaled to this one by the chains
     rl = kernel_rooflines(w, args.variant, prof, steps, rows_per_step, windows_chains, positions, pk, ctl, traffic, launch_shape)
     if not rl:
         raise RuntimeError("no kernel of the library ran inside the timed region")

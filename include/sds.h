@@ -95,7 +95,9 @@ extern "C" {
                                    [11]: how the last sds_sample_all ran its windows (bit 0: SDS_OPT_REGEN_DRAFTS in effect,
                                    bit 2: rows of skipped one-hot blocks read from the means table, see SDS_OPT_ONEHOT_ROWS);
                                    [12]: window positions whose accept test was evaluated since sds_reset
-                                   (the window kernels; with SDS_OPT_VERIFY_EARLY_EXIT fewer than the rows drafted) */
+                                   (the window kernels; with SDS_OPT_VERIFY_EARLY_EXIT fewer than the rows drafted);
+                                   [13]: those of them evaluated with the drafted states made again (SDS_OPT_REGEN_DRAFTS);
+                                   [14]: drafted rows stored as floats since sds_reset (the others only as bf16 copies) */
 #define SDS_GET_ROWK      18    /* int32  [nrows]     transition index of each row */
 #define SDS_GET_DP        19    /* float  [nrows, d]  independent drafter: the draft model's output per drafted row */
 
@@ -260,7 +262,11 @@ int sds_sample_all(sds_ctx* ctx, float* out_dev, int32_t* nfe_calls_dev, int32_t
  * function of Y_n, the frozen target output and the chain's noise, which is a function of (seed, chain,
  * step): verify runs the draft recurrence again in registers with the draft kernel's own operations,
  * reads only the target outputs, and advances its chains. Same results, bit for bit. SDS_GET_X and
- * SDS_GET_TAIL are then stale after sds_sample_all. */
+ * SDS_GET_TAIL are then stale after sds_sample_all. With value 1 the choice is made window by window: while
+ * most drafts pass, a window is verified over many positions and reading the drafted rows back is cheaper
+ * than drawing their noise a second time, so the rows are stored and read as without the option; once the
+ * latest finished window needed at most L/4 + 1 positions per chain (known one window late), the rows are
+ * made again. Value 2 makes them again in every window. */
 #define SDS_OPT_REGEN_DRAFTS 7
 /* SDS_OPT_ONEHOT_ROWS (default 1): mixtures on the tensor cores. The softmax pass stores weights below 2^-40 of
  * their row as exact zeros (either way). A row left with a single weight is one-hot: its weight is 1 and its
@@ -335,9 +341,10 @@ int64_t sds_launch_count(const sds_ctx* ctx);
 #define SDS_PROF_ADVANCE  4
 #define SDS_PROF_FUSED    5     /* whole-chain persistent kernel */
 #define SDS_PROF_AUX      6     /* |mu|^2, list rebuild, copies of the initial call */
-#define SDS_PROF_SOFTMAX  7     /* passes between the two GEMMs of a tensor-core mixture (softmax, row conversions) */
+#define SDS_PROF_SOFTMAX  7     /* passes around the two GEMMs of a tensor-core mixture (softmax, row conversions, copies of one-hot rows) */
 #define SDS_PROF_DRAFT_MODEL 8  /* every kernel of the independent draft model (SDS_INDEPENDENT) */
-#define SDS_PROF_KINDS    9
+#define SDS_PROF_MIX      9     /* mixing GEMM of a tensor-core mixture (SDS_PROF_DENOISE then holds its logits GEMM) */
+#define SDS_PROF_KINDS    10
 int sds_profile(sds_ctx* ctx, int32_t enable);
 int sds_profile_read(sds_ctx* ctx, double* ms, int64_t* launches, int32_t reset);
 

@@ -345,7 +345,7 @@ class Sampler:
         self._chk(self.lib.sds_set_projection(self.h, Q.data_ptr(), int(Q.shape[0])), "sds_set_projection")
         self._proj = Q
 
-    PROF_KINDS = ("init", "denoise", "draft", "verify", "advance", "fused", "aux", "softmax", "draft_model")
+    PROF_KINDS = ("init", "denoise", "draft", "verify", "advance", "fused", "aux", "softmax", "draft_model", "mix")
 
     def profile(self, enable: bool):
         self._chk(self.lib.sds_profile(self.h, int(enable)), "sds_profile")

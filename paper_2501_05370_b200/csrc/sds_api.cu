@@ -100,6 +100,7 @@ struct sds_ctx {
   bool early_exit = true;           // verify stops reading a window after the block with the first rejection
   bool fuse_advance = true;         // sds_sample_all lets the verify kernel do the advance step where it can
   bool regen = true;                // sds_sample_all lets the verify kernel draw the drafted states again instead of reading them
+  bool regen_always = false;        // ... in every window (default: only while windows end after a few positions)
   bool fusing = false;              // set around the verify call of the sds_sample_all loop
   bool raw_rows = true;             // sds_sample_all lets the mixing GEMM store accumulators, verify applies C acc + E x
   bool onehot = true;               // the mixing GEMM skips blocks of rows that are all one-hot; a copy kernel fills them
@@ -395,6 +396,7 @@ int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, cons
   const bool is_drafter = &e == &c->drf;
   const int kd = is_drafter ? SDS_PROF_DRAFT_MODEL : SDS_PROF_DENOISE;
   const int ks = is_drafter ? SDS_PROF_DRAFT_MODEL : SDS_PROF_SOFTMAX;
+  const int km = is_drafter ? SDS_PROF_DRAFT_MODEL : SDS_PROF_MIX;
   switch (e.den.kind) {
     case SDS_DEN_GMM: {
       if (e.den.means_dtype == SDS_F32 && c->tensor_split && gmm_split_shape(e.den, c->d)) {
@@ -451,7 +453,7 @@ int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, cons
         m.tile_counts = at<int>(c, c->lay.ctl) + kCtlTilesFull;
         for (int i = 0; i < 3; ++i) { m.a_short[i] = kSa[i]; m.b_short[i] = kSb[i]; }
         m.hot_flags = hot;
-        SDS_LAUNCH(c, kd, launch_gemm_tc(kEpiGmmMix, m, Rs, Mt, c->stream));
+        SDS_LAUNCH(c, km, launch_gemm_tc(kEpiGmmMix, m, Rs, Mt, c->stream));
         if (hot && !indexed)    // (indexed: the readers of the rows take the skipped blocks' rows from the means themselves)
           SDS_LAUNCH(c, ks, launch_mix_onehot(means, false, amax, hot, nrows_dev, (int)rows_ub, (int)dd,
                                               at<double>(c, e.lay.tcond), rowk, raw ? nullptr : X, out, c->stream));
@@ -488,7 +490,7 @@ int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, cons
       m.tcond = at<double>(c, e.lay.tcond); m.xrows = raw ? nullptr : X;
       m.hot_flags = hot;
       m.tile_counts = is_drafter ? nullptr : at<int>(c, c->lay.ctl) + kCtlTilesFull;
-      SDS_LAUNCH(c, kd, launch_gemm_tc(kEpiGmmMix, m, R, Mt, c->stream));
+      SDS_LAUNCH(c, km, launch_gemm_tc(kEpiGmmMix, m, R, Mt, c->stream));
       if (hot && !indexed)   // the skipped blocks: every row is a copy of one mean (with the same affine map as the epilogue's)
         SDS_LAUNCH(c, ks, launch_mix_onehot(means, true, amax, hot, nrows_dev, (int)rows_ub, c->d,
                                             at<double>(c, e.lay.tcond), rowk, raw ? nullptr : X, out, c->stream));
@@ -825,6 +827,11 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
     // Windows are enqueued one ahead of the host's knowledge of the active count: after window w
     // is enqueued the host waits for window w-1's count. A window enqueued with no active chain
     // does nothing on the device.
+    // positions per chain the last known window evaluated (with early exit: up to the first rejection): decides,
+    // window by window, whether verify makes the drafted states again or reads them back
+    double mean_positions = (double)c->L;
+    int64_t pos_seen = 0;
+    int na_before = (int)c->B;
     for (int w = 0;; ++w) {
       // mixtures on the tensor cores: the mixing GEMM stores its accumulators and the verify (and advance)
       // kernels, which hold the rows' inputs anyway, apply C acc + E x: the GEMM's epilogue reads nothing
@@ -843,12 +850,18 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
       const bool bf16_only = A.Xb != nullptr &&
                              (c->tgt.den.kind == SDS_DEN_MLP ||
                               (c->tgt.den.kind == SDS_DEN_GMM && c->tgt.den.means_dtype == SDS_BF16 && c->raw_now));
-      c->regen_now = c->regen && c->fuse_advance && bf16_only && verify_can_regen(A);
+      // Windows in which most drafts pass are verified over many positions, and there reading the drafted rows
+      // back is cheaper than drawing their noise a second time; windows that end after a position or two (the
+      // usual case late in a diffusion chain) gain from the smaller draft stores. The two ways give the same
+      // bits, so the choice follows the positions per chain the latest finished window needed.
+      const bool few_positions = !c->early_exit || mean_positions <= 0.25 * c->L + 1.0;
+      c->regen_now = c->regen && c->fuse_advance && bf16_only && verify_can_regen(A) && (c->regen_always || few_positions);
       c->skipx_now = c->regen_now;
       // where the register-resident verify kernel runs, it also advances its chains and compacts
       c->fusing = c->fuse_advance && (verify_can_advance(A) || c->regen_now);
-      if (w == 0) {                                      // which of these paths the run takes (read back with the control words)
-        c->h_pin[48] = (c->regen_now ? 1 : 0) | (c->hot_now ? 4 : 0);
+      if (w == 0) {                                      // which of these paths the run may take (read back with the control words)
+        const bool may_regen = c->regen && c->fuse_advance && bf16_only && verify_can_regen(A);
+        c->h_pin[48] = (may_regen ? 1 : 0) | (c->hot_now ? 4 : 0);
         SDS_CU(c, cudaMemcpyAsync(A.ctl + kCtlPathFlags, c->h_pin + 48, 4, cudaMemcpyHostToDevice, c->stream));
       }
       rc = sds_draft(c);
@@ -867,8 +880,13 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
       SDS_CU(c, cudaEventRecord(c->ev[w & 1], c->stream));
       if (w >= 1) {
         SDS_CU(c, cudaEventSynchronize(c->ev[(w - 1) & 1]));
-        const int na = c->h_pin[16 + ((w - 1) & 1) * kCtlWords + kCtlNActive];
+        const int32_t* seen = c->h_pin + 16 + ((w - 1) & 1) * kCtlWords;
+        const int na = seen[kCtlNActive];
         if (na == 0) break;
+        const int64_t pos = (int64_t)(uint32_t)seen[kCtlPositions];
+        if (na_before > 0) mean_positions = (double)(pos - pos_seen) / na_before;
+        pos_seen = pos;
+        na_before = na;
         c->ub = na;
       }
       if (w > c->K + 2) break;   // every window advances each active chain by at least one step
@@ -999,7 +1017,7 @@ int sds_set_option(sds_ctx* c, int32_t option, int64_t value) {
     case SDS_OPT_VERIFY_EARLY_EXIT: c->early_exit = value != 0; return SDS_OK;
     case SDS_OPT_FUSE_ADVANCE: c->fuse_advance = value != 0; return SDS_OK;
     case SDS_OPT_RAW_ROWS: c->raw_rows = value != 0; return SDS_OK;
-    case SDS_OPT_REGEN_DRAFTS: c->regen = value != 0; return SDS_OK;
+    case SDS_OPT_REGEN_DRAFTS: c->regen = value != 0; c->regen_always = value == 2; return SDS_OK;
     case SDS_OPT_ONEHOT_ROWS: c->onehot = value != 0; return SDS_OK;
     default: return SDS_EINVAL;
   }

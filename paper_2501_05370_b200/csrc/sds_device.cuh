@@ -30,6 +30,8 @@ enum Ctl : int {
   kCtlPathFlags = 11, // how the last sds_sample_all ran its windows: bit 0 verify drew the drafted states again,
                       // bit 1 the drafted noise was kept in the workspace between windows (written by the host)
   kCtlPositions = 12, // window positions whose accept test the verify kernels evaluated since reset (wraps at 2^31)
+  kCtlPositionsRegen = 13, // ... of which by the verify kernel that makes the drafted states again (no drafted rows read)
+  kCtlRowsFloat = 14, // drafted rows the draft kernel stored as floats since reset (it stores only bf16 copies otherwise)
   kCtlWords = 16
 };
 constexpr int kErrNonFinite = 1;

@@ -119,6 +119,8 @@ __global__ void __launch_bounds__(kBlock) k_init(WinArgs A) {
     A.ctl[kCtlTilesFull] = 0;
     A.ctl[kCtlTilesBrief] = 0;
     A.ctl[kCtlPositions] = 0;
+    A.ctl[kCtlPositionsRegen] = 0;
+    A.ctl[kCtlRowsFloat] = 0;
     A.ctl[kCtlTilesSkipped] = 0;
   }
   if (b >= A.B) return;
@@ -215,6 +217,7 @@ __global__ void __launch_bounds__(kBlock) k_draft(WinArgs A) {
   const uint64_t bg = A.chain_off + (uint64_t)b;
   const size_t cb = (size_t)b * A.d;
   if (t < Lt) A.rowk[r0 + t] = nb + t;            // TPC >= 32 >= Lt
+  if (t == 0 && !A.skip_x) atomicAdd(A.ctl + kCtlRowsFloat, Lt);
   if (VEC == 4) {
     for (int i = t * 4; i < A.d; i += TPC * 4) {
       float4 y = ld4(A.Y + cb + i);
@@ -848,6 +851,7 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t,
       A.accmask[b] = amask;
       A.jstar[b] = jstar;
       atomicAdd(A.ctl + kCtlPositions, done);
+      if (REGEN) atomicAdd(A.ctl + kCtlPositionsRegen, done);
       if (frozen) atomicOr(A.ctl + kCtlError, kErrNonFinite);
       if (TPC > 32) { s_jstar = jstar; s_coef = coef; }
     }

@@ -268,7 +268,7 @@ def test_full_size_runs_agree_bitwise_across_kernel_options(name):
     s = sds.sampler_for(w)
     ref = None
     for fuse, early, pair, whole, raw, regen, hot in [(1, 1, 1, 1, 1, 1, 1), (1, 1, 1, 1, 1, 1, 1), (1, 1, 1, 1, 1, 0, 1), (0, 1, 1, 1, 1, 1, 1),
-                                                     (1, 0, 1, 1, 1, 1, 1), (1, 1, 1, 1, 0, 1, 1), (1, 1, 1, 1, 1, 1, 0), (1, 1, 0, 1, 0, 1, 1),
+                                                     (1, 0, 1, 1, 1, 1, 1), (1, 1, 1, 1, 0, 1, 1), (1, 1, 1, 1, 1, 1, 0), (1, 1, 0, 1, 0, 1, 1), (1, 1, 1, 1, 1, 2, 1),
                                                      (0, 0, 0, 0, 0, 0, 0)]:
         s.set_option(s.OPT_FUSE_ADVANCE, fuse); s.set_option(s.OPT_VERIFY_EARLY_EXIT, early)
         s.set_option(s.OPT_GEMM_PAIR, pair); s.set_option(s.OPT_WHOLE_CHAIN_KERNEL, whole)
@@ -298,11 +298,19 @@ def test_drafted_states_drawn_again_give_the_same_bits(kind, d, L, B):
     else:
         w = wl.WORKLOADS["cfg4"].scaled(d=d, B=B, L=L, K=K)
         s = sds.sampler_for(w, gmm=w.gmm_params(d=d, ncomp=128), seed=81)
+    s.set_option(s.OPT_REGEN_DRAFTS, 2)                   # in every window
     got = [x.cpu().numpy() for x in s.sample_all()]
     assert np.all(np.isfinite(got[0]))
-    windows = int(s.get(sb.GET_CTL)[2])
+    ctl = s.get(sb.GET_CTL)
+    windows = int(ctl[2])
+    assert int(ctl[13]) == int(ctl[12]) > 0 and int(ctl[14]) == 0      # every position verified on states made again, no float rows
+    s.set_option(s.OPT_REGEN_DRAFTS, 1)                   # window by window, from the positions the last window needed
+    mixed = [x.cpu().numpy() for x in s.sample_all()]
+    assert all(np.array_equal(x, y) for x, y in zip(got, mixed))
+    assert int(s.get(sb.GET_CTL)[12]) == int(ctl[12])     # the same positions were evaluated
     s.set_option(s.OPT_REGEN_DRAFTS, 0)
     back = [x.cpu().numpy() for x in s.sample_all()]
+    assert int(s.get(sb.GET_CTL)[13]) == 0
     assert all(np.array_equal(x, y) for x, y in zip(got, back))
     assert windows == int(s.get(sb.GET_CTL)[2])
     s.set_option(s.OPT_FUSE_ADVANCE, 0)
