@@ -27,23 +27,42 @@ namespace {
 constexpr int BM = 128;            // rows per tile = TMEM lanes
 constexpr int BK = 64;             // bf16 elements per K block = one 128-byte swizzle row
 constexpr int UK = 16;             // K per tcgen05.mma of kind::f16
-constexpr int kEpiWarps = 8;       // two warps per TMEM lane quarter, each takes half of the tile's columns
-constexpr int kThreads = 64 + 32 * kEpiWarps;   // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..9: epilogue
+// Epilogue warps: warp w reaches the 32 TMEM lanes of quarter w % 4; the warps of a quarter split the
+// tile's columns. The staged epilogues (activation, bias, affine map, stores turned through shared
+// memory) do about as much work per tile as a main loop over K = 2048 takes, so sixteen warps run them
+// (four per scheduler hide the latencies of the tensor-memory loads, the table loads and the exp/divide
+// chains); the logits epilogue, short next to its long main loop, keeps eight.
+constexpr int epi_warps(int epi) { return epi == kEpiGmmLogits ? 8 : 16; }
+constexpr int gemm_threads(int epi) { return 64 + 32 * epi_warps(epi); }   // warp 0: TMA, warp 1: MMA + TMEM owner, then the epilogue warps
 constexpr uint32_t kSpinCap = 1u << 22;
 
 template <int BN, bool PAIR, int EPI> struct TileCfg {
   // the logits epilogue writes whole rows from registers and needs no staging tile: its shared memory
-  // holds one more operand stage instead (the main loop is bound by the bytes in flight)
+  // holds more operand stages instead (the main loop is bound by the bytes in flight)
   static constexpr bool kStaged = EPI != kEpiGmmLogits;
-  static constexpr int kBRows = PAIR ? BN / 2 : BN;                         // rows of B one CTA stages
+  static constexpr int kEpiWarps = epi_warps(EPI);
+  static constexpr int kThreads = gemm_threads(EPI);
+  // BN = 512 (CTA pairs only): the tile is two sub-tiles of 256 columns, two MMAs per K step into the two
+  // halves of ONE 512-column accumulator (all of tensor memory: no second buffer, the epilogue of a tile is
+  // not overlapped with the next main loop). A is staged once for twice the products, so the operand bytes
+  // per product fall by a quarter: for contractions with a long K and a short epilogue (the logits of the
+  // large mixture), whose main loop is bound by the bytes it can keep in flight.
+  static constexpr int kNSub = BN > 256 ? BN / 256 : 1;                     // MMAs (N <= 256 each) per K step
+  static constexpr int kSubN = BN / kNSub;                                  // columns of one sub-tile
+  static constexpr int kSubBRows = PAIR ? kSubN / 2 : kSubN;                // rows of one sub-tile of B one CTA stages
+  static constexpr int kBRows = kNSub * kSubBRows;                          // rows of B one CTA stages
   static constexpr int kABytes = BM * BK * 2;
-  static constexpr int kBBytes = kBRows * BK * 2;
+  static constexpr int kSubBBytes = kSubBRows * BK * 2;
+  static constexpr int kBBytes = kNSub * kSubBBytes;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kStages = (kStageBytes == 32 * 1024) ? (kStaged ? 6 : 7) : 4;
-  static constexpr int kTmemCols = 2 * BN;                                  // two accumulator buffers
-  static constexpr int kEpiStageBytes = kStaged ? kEpiWarps * 32 * 33 * 4 : 0;   // one padded 32x32 float tile per epilogue warp
-  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/ + kEpiStageBytes;
-  static_assert(kSmemBytes <= 227 * 1024, "shared memory of one CTA");
+  static constexpr int kAccBufs = BN <= 256 ? 2 : 1;                        // accumulator buffers in tensor memory
+  static constexpr int kTmemCols = kAccBufs * BN;
+  static constexpr int kEpiStageBytes = kStaged ? kEpiWarps * 32 * 32 * 4 : 0;   // one swizzled 32x32 float tile per epilogue warp
+  static constexpr int kFixedBytes = 1024 /*align*/ + 256 /*barriers*/ + kEpiStageBytes;
+  static constexpr int kStages = (227 * 1024 - kFixedBytes) / kStageBytes;  // 32 KB stages: 7 unstaged, 5 staged
+  static constexpr int kSmemBytes = kStages * kStageBytes + kFixedBytes;
+  static_assert(kStages >= 3 && kStages <= 8, "operand stages");
+  static_assert(kTmemCols <= 512 && (BN <= 256 || PAIR), "tensor memory holds 512 columns; wide tiles are for pairs");
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -245,7 +264,7 @@ __device__ __forceinline__ bool tile_is_skipped(const TcGemmArgs& g, int tm) {
 }
 
 template <int BN, int EPI, bool PAIR>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(gemm_threads(EPI), 1)
     k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
               const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB0,
               const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, TcGemmArgs g) {
@@ -277,7 +296,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::kStages; ++s) { mbar_init(full_bar + s, 1); mbar_init(empty_bar + s, 1); }
     // the leader's "drained" barriers collect the epilogue warps of both CTAs
-    for (int s = 0; s < 2; ++s) { mbar_init(tfull_bar + s, 1); mbar_init(tempty_bar + s, PAIR ? 2 * kEpiWarps : kEpiWarps); }
+    for (int s = 0; s < 2; ++s) { mbar_init(tfull_bar + s, 1); mbar_init(tempty_bar + s, PAIR ? 2 * C::kEpiWarps : C::kEpiWarps); }
     *abort_s = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -309,7 +328,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       const uint32_t leader_full0 = PAIR ? map_to_cta(smem_u32(full_bar), 0u) : 0u;
       for (int t = worker; t < total_tiles && ok; t += nworkers) {
         if (EPI == kEpiGmmMix && tile_is_skipped<TM>(g, t / n_tiles)) continue;
-        const int m0 = (t / n_tiles) * TM + (int)rank * BM, n0 = (t % n_tiles) * BN + (int)rank * C::kBRows;
+        const int m0 = (t / n_tiles) * TM + (int)rank * BM, n0 = (t % n_tiles) * BN + (int)rank * C::kSubBRows;
         const bool brief = tile_is_brief<TM>(g, t / n_tiles);
         const int nkb = brief ? kb_seg * g.nseg_short : kblocks;
         for (int kb = 0; kb < nkb; ++kb) {
@@ -324,7 +343,9 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (rank == 0) mbar_expect_tx(full_bar + stage, 2u * (uint32_t)C::kStageBytes);
             const uint32_t fb = leader_full0 + (uint32_t)stage * 8u;
             tma_load_2d_pair(sa, ta, kk, m0, fb);
-            tma_load_2d_pair(sa + C::kABytes, tb, kk, n0, fb);
+#pragma unroll
+            for (int sub = 0; sub < C::kNSub; ++sub)      // this CTA's half of every sub-tile of B
+              tma_load_2d_pair(sa + C::kABytes + sub * C::kSubBBytes, tb, kk, n0 + sub * C::kSubN, fb);
           } else {
             mbar_expect_tx(full_bar + stage, (uint32_t)C::kStageBytes);
             tma_load_2d(sa, ta, kk, m0, full_bar + stage);
@@ -341,7 +362,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = make_idesc(TM, BN);
+      constexpr uint32_t idesc = make_idesc(TM, C::kSubN);
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
@@ -351,8 +372,8 @@ __global__ void __launch_bounds__(kThreads, 1)
           if (g.tile_counts && (t % n_tiles) == 0) atomicAdd(g.tile_counts + 2, n_tiles);
           continue;
         }
-        const int buf = it & 1;
-        const uint32_t bphase = (uint32_t)(it >> 1) & 1u;
+        const int buf = C::kAccBufs == 2 ? (it & 1) : 0;
+        const uint32_t bphase = (uint32_t)(C::kAccBufs == 2 ? (it >> 1) : it) & 1u;
         ++it;
         if (!mbar_wait(tempty_bar + buf, bphase ^ 1u, abort_s)) { ok = false; break; }
         tc_fence_after();
@@ -364,12 +385,17 @@ __global__ void __launch_bounds__(kThreads, 1)
           if (!mbar_wait(full_bar + stage, phase, abort_s)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_u32(stages + stage * C::kStageBytes);
-          const uint64_t adesc = make_sdesc(sa), bdesc = make_sdesc(sa + C::kABytes);
+          const uint64_t adesc = make_sdesc(sa);
 #pragma unroll
           for (int k = 0; k < BK / UK; ++k) {
-            // 32 bytes further along K inside the 128-byte swizzle row: +2 in the (>>4) address field
-            if (PAIR) umma_bf16_pair(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb | k) ? 1u : 0u);
-            else umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb | k) ? 1u : 0u);
+#pragma unroll
+            for (int sub = 0; sub < C::kNSub; ++sub) {
+              const uint64_t bdesc = make_sdesc(sa + C::kABytes + sub * C::kSubBBytes);
+              const uint32_t dsub = d_tmem + (uint32_t)(sub * C::kSubN);
+              // 32 bytes further along K inside the 128-byte swizzle row: +2 in the (>>4) address field
+              if (PAIR) umma_bf16_pair(dsub, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb | k) ? 1u : 0u);
+              else umma_bf16(dsub, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb | k) ? 1u : 0u);
+            }
           }
           // frees the stage (in both CTAs of a pair) once these MMAs have read it
           if (PAIR) umma_commit_pair(empty_bar + stage); else umma_commit(empty_bar + stage);
@@ -384,16 +410,16 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
   } else {
     // ---------------- epilogue: warps with (warp & 3) == q reach TMEM lanes 32q .. 32q+31 ----------------
-    const int q = warp & 3, half = (warp - 2) >> 2;
-    constexpr int kCols = BN / 2;                      // columns per epilogue warp
+    const int q = warp & 3, half = (warp - 2) >> 2;    // lane quarter; which share of the columns
+    constexpr int kCols = BN / (C::kEpiWarps / 4);     // columns per epilogue warp
     int it = 0;
     bool ok = true;
     // "drained" goes to the leader's barrier (the MMA issuer of the pair waits there)
     const uint32_t drained0 = (PAIR && rank != 0) ? map_to_cta(smem_u32(tempty_bar), 0u) : 0u;
     for (int t = worker; t < total_tiles && ok; t += nworkers) {
       if (EPI == kEpiGmmMix && tile_is_skipped<TM>(g, t / n_tiles)) continue;
-      const int buf = it & 1;
-      const uint32_t bphase = (uint32_t)(it >> 1) & 1u;
+      const int buf = C::kAccBufs == 2 ? (it & 1) : 0;
+      const uint32_t bphase = (uint32_t)(C::kAccBufs == 2 ? (it >> 1) : it) & 1u;
       ++it;
       const int m0 = (t / n_tiles) * TM + (int)rank * BM, n0 = (t % n_tiles) * BN + half * kCols;
       const int row = m0 + q * 32 + lane;
@@ -406,7 +432,10 @@ __global__ void __launch_bounds__(kThreads, 1)
         // through shared memory instead: eight lanes cover the 32 columns of a row, a warp access
         // covers four rows of 128 contiguous bytes. All eight x loads of a chunk are in flight
         // before the accumulator chunk is read.
-        float* stg = epi_stage + (warp - 2) * (32 * 33);
+        // staging tile of this warp: 32 rows of 128 bytes, the eight 16-byte pieces of row r stored at piece
+        // index p ^ (r & 7), so that both the row-wise writes and the four-rows-at-a-time reads are free of
+        // bank conflicts with 128-bit accesses
+        float4* stg4 = reinterpret_cast<float4*>(epi_stage + (warp - 2) * (32 * 32));
         float rowC = 0.f, rowE = 0.f;
         // xrows == NULL: the caller applies C acc + E x itself where it reads the rows (it holds x there
         // anyway); the accumulator is stored as it is and this epilogue reads nothing
@@ -457,7 +486,9 @@ __global__ void __launch_bounds__(kThreads, 1)
             }
           }
 #pragma unroll
-          for (int j = 0; j < 32; ++j) stg[lane * 33 + j] = __uint_as_float(acc[j]);
+          for (int p8 = 0; p8 < 8; ++p8)
+            stg4[lane * 8 + (p8 ^ (lane & 7))] = make_float4(__uint_as_float(acc[4 * p8]), __uint_as_float(acc[4 * p8 + 1]),
+                                                             __uint_as_float(acc[4 * p8 + 2]), __uint_as_float(acc[4 * p8 + 3]));
           __syncwarp();
           float4 bc = make_float4(0.f, 0.f, 0.f, 0.f);
           if (EPI == kEpiBiasF32 || EPI == kEpiMlpHidden) bc = __ldg(reinterpret_cast<const float4*>(g.bias + col));
@@ -466,7 +497,8 @@ __global__ void __launch_bounds__(kThreads, 1)
             const int rl = 4 * i + rr4;
             const float cC = __shfl_sync(0xffffffffu, rowC, rl), cE = __shfl_sync(0xffffffffu, rowE, rl);
             if (rl < nlive) {
-              const float* sp = stg + rl * 33 + c4;
+              const float4 sv = stg4[rl * 8 + ((lane & 7) ^ (rl & 7))];
+              const float sp[4] = {sv.x, sv.y, sv.z, sv.w};
               if (EPI == kEpiMlpHidden) {                     // h = SiLU(acc + bias + E[k]) as bf16
                 float h0 = sp[0] + bc.x + bf16_lo(tv[i].x), h1 = sp[1] + bc.y + bf16_hi(tv[i].x);
                 float h2 = sp[2] + bc.z + bf16_lo(tv[i].y), h3 = sp[3] + bc.w + bf16_hi(tv[i].y);
@@ -832,7 +864,7 @@ cudaError_t launch_t(const TcGemmArgs& g, const void* A, const void* B, int grid
     const uint16_t* a = static_cast<const uint16_t*>(A) + (size_t)i * g.a_plane;
     const uint16_t* b = static_cast<const uint16_t*>(B) + (size_t)i * g.b_plane;
     if (!make_tmap(&tmA[i], g.nplanes > i ? a : A, (uint64_t)g.rows_cap, (uint64_t)g.K, BM)) return cudaErrorInvalidValue;
-    if (!make_tmap(&tmB[i], g.nplanes > i ? b : B, (uint64_t)g.N, (uint64_t)g.K, C::kBRows)) return cudaErrorInvalidValue;
+    if (!make_tmap(&tmB[i], g.nplanes > i ? b : B, (uint64_t)g.N, (uint64_t)g.K, C::kSubBRows)) return cudaErrorInvalidValue;
   }
   cudaError_t e = cudaFuncSetAttribute(k_gemm_tc<BN, EPI, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
   if (e != cudaSuccess) return e;
@@ -845,7 +877,7 @@ cudaError_t launch_t(const TcGemmArgs& g, const void* A, const void* B, int grid
     if (pairs < 1) pairs = 1;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(2 * pairs);
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(C::kThreads);
     cfg.dynamicSmemBytes = C::kSmemBytes;
     cfg.stream = st;
     cudaLaunchAttribute attr{};
@@ -867,7 +899,7 @@ cudaError_t launch_t(const TcGemmArgs& g, const void* A, const void* B, int grid
   }
   int grid = grid_tiles_ub < sms ? grid_tiles_ub : sms;
   if (grid < 1) grid = 1;
-  k_gemm_tc<BN, EPI, PAIR><<<grid, kThreads, C::kSmemBytes, st>>>(tmA[0], tmA[1], tmA[2], tmB[0], tmB[1], tmB[2], g);
+  k_gemm_tc<BN, EPI, PAIR><<<grid, C::kThreads, C::kSmemBytes, st>>>(tmA[0], tmA[1], tmA[2], tmB[0], tmB[1], tmB[2], g);
   return cudaGetLastError();
 }
 
@@ -894,6 +926,11 @@ cudaError_t launch_gemm_tc(int epi, const TcGemmArgs& g_in, const void* A_bf16, 
       tiles = ((g.rows_host + BM - 1) / BM) * (g.N / 256);                                 \
     }                                                                                      \
     return wide ? launch_t<256, E, false>(g, A_bf16, B_bf16, tiles, st) : launch_t<128, E, false>(g, A_bf16, B_bf16, tiles, st);
+  // long contractions with the short logits epilogue: tiles of 256 x 512 on one accumulator (see TileCfg)
+  if (epi == kEpiGmmLogits && pair && (g.N % 512) == 0 && g.K >= 4096 && g.nseg == 1) {
+    const cudaError_t e_ = launch_t<512, kEpiGmmLogits, true>(g, A_bf16, B_bf16, m_tiles * (g.N / 512), st);
+    if (e_ != cudaErrorLaunchOutOfResources) return e_;
+  }
   switch (epi) {
     SDS_TC_CASE(kEpiMlpHidden)
     SDS_TC_CASE(kEpiBiasF32)

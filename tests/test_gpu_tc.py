@@ -34,7 +34,8 @@ def test_mlp_denoiser_rows(dims, rows, K):
     s.close()
 
 
-@pytest.mark.parametrize("d,ncomp,rows", [(256, 128, 200), (384, 256, 77), (1024, 384, 260)])
+@pytest.mark.parametrize("d,ncomp,rows", [(256, 128, 200), (384, 256, 77), (1024, 384, 260),
+                                          (4096, 512, 300), (4096, 1024, 515)])   # long K, N % 512 == 0: 256 x 512 logits tiles
 def test_large_mixture_denoiser_rows(d, ncomp, rows):
     import torch
     w = wl.WORKLOADS["cfg4"].scaled(d=d, B=rows, L=1, K=50)
