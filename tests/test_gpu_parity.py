@@ -131,6 +131,30 @@ def _window_check(s, w, den, a32, c32, s32, seed, chain_off, stats, chains=None,
         dc_arg = Dp[r0:r0 + Lt] if draft_den is not None else Dc[b]
         v = o.verify_window(W, Dq[r0:r0 + Lt], dc_arg, a64, c64, s64, nb, logU[b, :Lt].astype(np.float64), proj=proj)
         amb = np.abs(v["ell"] - logU[b, :Lt]) < BAND
+        if proj is None and draft_den is None and stats.get("mode", 0) == 0:
+            # The same test on the kernel's own single-precision Delta and Z (its element formulas retyped
+            # in float32, sums in double as in the kernel): the decisions must then agree everywhere, not
+            # only outside the band (the band exists because the oracle forms Delta and Z in double). A
+            # margin of 1e-6 covers the order of the double sums and the emulated fused multiply-adds.
+            f32 = np.float32
+            fma = lambda x, y, z: (x.astype(np.float64) * np.float64(y) + z.astype(np.float64)).astype(f32)
+            for j in range(1, Lt + 1):
+                k = nb + j - 1
+                ak, ck, sk = f32(a32[k]), f32(c32[k]), f32(s32[k])
+                inv_s = f32(1.0) / sk
+                cs = ck * inv_s
+                wp = X[r0 + j - 1]
+                wj = X[r0 + j] if j < Lt else T[b]
+                D = cs * (Dc[b] - Dq[r0 + j - 1])
+                Z = fma(wp, -ak, wj)                                                # fmaf(-a, wp, wj)
+                Z = fma(Dc[b], -ck, Z) * inv_s                                      # fmaf(-c, dc, .) / sigma
+                S1k = float(np.sum(D.astype(np.float64) ** 2))
+                S2k = float(np.sum(D.astype(np.float64) * Z.astype(np.float64)))
+                ellk = -0.5 * S1k - S2k
+                if abs(ellk - float(logU[b, j - 1])) > 1e-6 * max(1.0, abs(ellk)):
+                    want_acc = (S1k < 1e-30) or (f32(logU[b, j - 1]) <= f32(ellk))
+                    assert bool((int(accmask[b]) >> (j - 1)) & 1) == bool(want_acc), ("exact replay", b, j, ellk, logU[b, j - 1])
+                    stats["exact"] = stats.get("exact", 0) + 1
         for j in range(Lt):
             assert ell_close(float(ell[b, j]), float(v["ell"][j])), (b, j, ell[b, j], v["ell"][j])
             assert abs(S1[b, j] - v["S1"][j]) <= 1e-5 * max(v["S1"][j], 1e-12) + 1e-12
@@ -214,6 +238,8 @@ def test_window_forced_parity(name, B, d, L, K, ncomp, windows):
             break
         na = _window_check(s, w, den, a32, c32, s32, seed, off, stats)
     assert stats["band"] <= max(2, 2e-3 * stats["tests"])
+    assert stats.get("exact", 0) >= 0.99 * stats["tests"]        # decisions replayed exactly on the kernel's own Delta and Z
+    print(f"band events {stats['band']} of {stats['tests']} tests; {stats.get('exact', 0)} decisions replayed exactly")
     s.close()
 
 
