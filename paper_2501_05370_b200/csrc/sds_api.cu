@@ -141,7 +141,7 @@ void den_layout(Carve& cv, const sds_denoiser* den, size_t K, int tcond_dim, siz
     l->logits = cv.take(rows * (size_t)den->ncomp * 4);
     l->flags = cv.take(((rows + 255) / 256 * 2) * 4);
     l->amax = cv.take(rows * 4);
-    l->hot = cv.take(((rows + 255) / 256) * 4);
+    l->hot = cv.take(((rows + 255) / 256 + 1) * 4);     // [0]: some block holds a row that is not one-hot; then one word per block
   }
   if (den->kind == SDS_DEN_MLP) {
     size_t width = 0;
@@ -154,7 +154,7 @@ void den_layout(Carve& cv, const sds_denoiser* den, size_t K, int tcond_dim, siz
     l->R = cv.take(rows * (size_t)den->ncomp * 2);
     l->Mt = cv.take((size_t)d * den->ncomp * 2);
     l->amax = cv.take(rows * 4);
-    l->hot = cv.take(((rows + 255) / 256) * 4);
+    l->hot = cv.take(((rows + 255) / 256 + 1) * 4);     // [0]: some block holds a row that is not one-hot; then one word per block
   }
 }
 
@@ -273,7 +273,7 @@ WinArgs win_args(sds_ctx* c) {
   A.raw_ce = c->raw_now ? at<float2>(c, c->lay.ce) : nullptr;
   if (c->hot_now) {
     A.hot_amax = at<int>(c, c->tgt.lay.amax);
-    A.hot_flags = at<int>(c, c->tgt.lay.hot);
+    A.hot_flags = at<int>(c, c->tgt.lay.hot) + 1;       // (word 0 says whether any block is mixed)
     A.hot_means = c->tgt.den.means_dev;
     A.hot_bf16 = c->tgt.den.means_dtype == SDS_BF16 ? 1 : 0;
   }
@@ -437,12 +437,13 @@ int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, cons
         SDS_CU(c, cudaMemsetAsync(flags, 0, (((size_t)rows_ub + 255) / 256 * 2) * 4, c->stream));
         // blocks of 256 rows whose rows are all one-hot skip the mixing contraction: their result is a copy of means
         int* amax = c->onehot ? at<int>(c, e.lay.amax) : nullptr;
-        int* hot = c->onehot ? at<int>(c, e.lay.hot) : nullptr;
-        if (hot) SDS_CU(c, cudaMemsetAsync(hot, 0, (((size_t)rows_ub + 255) / 256) * 4, c->stream));
+        int* any_mixed = c->onehot ? at<int>(c, e.lay.hot) : nullptr;
+        int* hot = any_mixed ? any_mixed + 1 : nullptr;
+        if (hot) SDS_CU(c, cudaMemsetAsync(any_mixed, 0, (((size_t)rows_ub + 255) / 256 + 1) * 4, c->stream));
         SDS_LAUNCH(c, ks,
                    launch_softmax_split3(logits, nrows_dev, (int)rows_ub, (int)nc, (int)dd, X, means,
                                          at<double>(c, e.lay.musq), e.den.logw_dev, at<double>(c, e.lay.tcond), rowk,
-                                         cap * nc, Rs, flags, amax, hot, c->stream));
+                                         cap * nc, Rs, flags, amax, hot, any_mixed, c->stream));
         TcGemmArgs m = tc_args(c, e, rowk, nrows_dev, rows_ub);
         m.N = (int)dd; m.K = (int)nc; m.out = out; m.ldo = (int)dd;
         m.tcond = at<double>(c, e.lay.tcond); m.xrows = raw ? nullptr : X;
@@ -452,7 +453,7 @@ int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, cons
         m.tile_flags = flags; m.nseg_short = 3;
         m.tile_counts = at<int>(c, c->lay.ctl) + kCtlTilesFull;
         for (int i = 0; i < 3; ++i) { m.a_short[i] = kSa[i]; m.b_short[i] = kSb[i]; }
-        m.hot_flags = hot;
+        m.hot_flags = hot; m.mixed_blocks = any_mixed;
         SDS_LAUNCH(c, km, launch_gemm_tc(kEpiGmmMix, m, Rs, Mt, c->stream));
         if (hot && !indexed)    // (indexed: the readers of the rows take the skipped blocks' rows from the means themselves)
           SDS_LAUNCH(c, ks, launch_mix_onehot(means, false, amax, hot, nrows_dev, (int)rows_ub, (int)dd,
@@ -482,13 +483,14 @@ int run_denoiser(sds_ctx* c, Engine& e, const float* X, const uint16_t* Xb, cons
       g.tcond = at<double>(c, e.lay.tcond); g.musq = at<double>(c, e.lay.musq); g.logw = e.den.logw_dev;
       SDS_LAUNCH(c, kd, launch_gemm_tc(kEpiGmmLogits, g, Xb, means, c->stream));
       int* amax = c->onehot ? at<int>(c, e.lay.amax) : nullptr;
-      int* hot = c->onehot ? at<int>(c, e.lay.hot) : nullptr;
-      if (hot) SDS_CU(c, cudaMemsetAsync(hot, 0, (((size_t)rows_ub + 255) / 256) * 4, c->stream));
-      SDS_LAUNCH(c, ks, launch_softmax_bf16(logits, nrows_dev, (int)rows_ub, e.den.ncomp, R, amax, hot, c->stream));
+      int* any_mixed = c->onehot ? at<int>(c, e.lay.hot) : nullptr;
+      int* hot = any_mixed ? any_mixed + 1 : nullptr;
+      if (hot) SDS_CU(c, cudaMemsetAsync(any_mixed, 0, (((size_t)rows_ub + 255) / 256 + 1) * 4, c->stream));
+      SDS_LAUNCH(c, ks, launch_softmax_bf16(logits, nrows_dev, (int)rows_ub, e.den.ncomp, R, amax, hot, any_mixed, c->stream));
       TcGemmArgs m = tc_args(c, e, rowk, nrows_dev, rows_ub);
       m.N = c->d; m.K = e.den.ncomp; m.out = out; m.ldo = c->d;
       m.tcond = at<double>(c, e.lay.tcond); m.xrows = raw ? nullptr : X;
-      m.hot_flags = hot;
+      m.hot_flags = hot; m.mixed_blocks = any_mixed;
       m.tile_counts = is_drafter ? nullptr : at<int>(c, c->lay.ctl) + kCtlTilesFull;
       SDS_LAUNCH(c, km, launch_gemm_tc(kEpiGmmMix, m, R, Mt, c->stream));
       if (hot && !indexed)   // the skipped blocks: every row is a copy of one mean (with the same affine map as the epilogue's)

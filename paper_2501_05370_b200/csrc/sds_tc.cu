@@ -293,6 +293,13 @@ __global__ void __launch_bounds__(gemm_threads(EPI), 1)
   const int kb_seg = (g.K + BK - 1) / BK;
   const int kblocks = kb_seg * g.nseg;
 
+  // every block of rows one-hot (the word is raised by the softmax pass where one is not): nothing to
+  // multiply; all CTAs read the same word and leave before any barrier or tensor memory exists
+  if (EPI == kEpiGmmMix && g.mixed_blocks && *g.mixed_blocks == 0) {
+    if (g.tile_counts && blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(g.tile_counts + 2, total_tiles);
+    return;
+  }
+
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::kStages; ++s) { mbar_init(full_bar + s, 1); mbar_init(empty_bar + s, 1); }
     // the leader's "drained" barriers collect the epilogue warps of both CTAs
@@ -575,7 +582,8 @@ __global__ void __launch_bounds__(gemm_threads(EPI), 1)
 // hot_flags[row / 256] is raised for every block of 256 rows that holds a row which is not one-hot.
 __global__ void __launch_bounds__(256) k_softmax_bf16(const float* __restrict__ logits, const int* __restrict__ nrows_dev,
                                                       int rows_host, int ncomp, uint16_t* __restrict__ R,
-                                                      int* __restrict__ amax, int* __restrict__ hot_flags) {
+                                                      int* __restrict__ amax, int* __restrict__ hot_flags,
+                                                      int* __restrict__ mixed_blocks) {
   const int nrows = nrows_dev ? min(*nrows_dev, rows_host) : rows_host;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int row = blockIdx.x * 8 + warp; row < nrows; row += gridDim.x * 8) {
@@ -583,6 +591,26 @@ __global__ void __launch_bounds__(256) k_softmax_bf16(const float* __restrict__ 
     float mx = -INFINITY;
     for (int c = lane; c < ncomp; c += 32) mx = fmaxf(mx, lg[c]);
     mx = warp_max(mx);
+    // A maximum that stands alone by more than 30 settles the row: every other weight is below e^-30,
+    // hence below the 2^-40 under which weights are stored as zeros, and the remaining one is
+    // 1 / (1 + less than 2^-24) = 1 in float: exactly what the general path below computes.
+    int near = 0, cnear = ncomp;
+    for (int c = lane; c < ncomp; c += 32) {
+      const bool in = lg[c] >= mx - 30.0f;
+      near += in;
+      if (lg[c] == mx) cnear = min(cnear, c);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      near += __shfl_xor_sync(0xffffffffu, near, o);
+      cnear = min(cnear, __shfl_xor_sync(0xffffffffu, cnear, o));
+    }
+    if (near == 1) {
+      for (int c = lane * 2; c < ncomp; c += 64)
+        *reinterpret_cast<uint32_t*>(R + (size_t)row * ncomp + c) = (cnear == c ? 0x3F80u : 0u) | (cnear == c + 1 ? 0x3F800000u : 0u);
+      if (amax && lane == 0) amax[row] = cnear;
+      continue;
+    }
     float den = 0.f;
     for (int c = lane; c < ncomp; c += 32) den += expf(lg[c] - mx);
     den = warp_sum(den);
@@ -605,7 +633,10 @@ __global__ void __launch_bounds__(256) k_softmax_bf16(const float* __restrict__ 
       }
       if (lane == 0) {
         amax[row] = (nnz == 1) ? cmax : -1;
-        if (nnz != 1 && hot_flags) hot_flags[row >> 8] = 1;
+        if (nnz != 1 && hot_flags) {
+          hot_flags[row >> 8] = 1;
+          if (mixed_blocks) *mixed_blocks = 1;
+        }
       }
     }
   }
@@ -713,29 +744,55 @@ __global__ void k_split3(const float* __restrict__ x, size_t n, size_t plane, in
 // their logit again in double (warp-wide dot product, fixed combination order); all others weigh
 // less than e^-29. Writes the normalised
 // responsibilities as three bf16 planes. One warp per row.
-template <int NQ>   // ncomp = 128 * NQ: a lane holds NQ groups of four consecutive components in registers
+// LAZY (needs hot_flags): a CTA takes whole blocks of 256 rows and first works every row out without
+// storing its responsibilities (only the row's component and the flags); where the block turns out to hold
+// a row that is not one-hot, the mixing contraction will read the block, and a second pass stores the
+// three planes of all its rows. Blocks of one-hot rows, which the contraction skips, cost no stores.
+template <int NQ, bool LAZY>   // ncomp = 128 * NQ: a lane holds NQ groups of four consecutive components in registers
 __global__ void __launch_bounds__(256)
     k_softmax_split3(const float* __restrict__ logits, const int* __restrict__ nrows_dev, int rows_host, int d,
                      const float* __restrict__ X, const float* __restrict__ means,
                      const double* __restrict__ musq, const float* __restrict__ logw,
                      const double* __restrict__ tcond, const int* __restrict__ rowk, size_t rplane,
                      uint16_t* __restrict__ R, int* __restrict__ tile_flags, int* __restrict__ amax,
-                     int* __restrict__ hot_flags) {
+                     int* __restrict__ hot_flags, int* __restrict__ mixed_blocks) {
   constexpr int ncomp = 128 * NQ;
   const int nrows = nrows_dev ? min(*nrows_dev, rows_host) : rows_host;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (int row = blockIdx.x * 8 + warp; row < nrows; row += gridDim.x * 8) {
-    const float* lg = logits + (size_t)row * ncomp;
+  // LAZY: blocks of 256 rows per CTA, up to two passes; otherwise one pass over rows 8 apart
+  const int nblk = LAZY ? (nrows + 255) / 256 : 1;
+  for (int blk = LAZY ? (int)blockIdx.x : 0; blk < nblk; blk += LAZY ? (int)gridDim.x : 1) {
+  int mixed = 0;                                  // some row of this warp in the block is not one-hot
+  for (int pass = 0; pass < (LAZY ? 2 : 1); ++pass) {
+  const bool store = !LAZY || pass == 1;
+  const int row_first = LAZY ? blk * 256 + warp : (int)blockIdx.x * 8 + warp;
+  const int row_end = LAZY ? min(nrows, blk * 256 + 256) : nrows;
+  const int row_step = LAZY ? 8 : (int)gridDim.x * 8;
+  // a warp takes its rows one after the other: the next row's logits and step index are requested before
+  // the current row is worked on, so that their latency is not paid row by row
+  float4 nxt[NQ];
+  int k_nxt = 0;
+  if (row_first < row_end) {
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) nxt[q] = ld4(logits + (size_t)row_first * ncomp + 4 * (lane + 32 * q));
+    k_nxt = __ldg(rowk + row_first);
+  }
+  for (int row = row_first; row < row_end; row += row_step) {
     float v[NQ][4];
     float mx = -INFINITY;
 #pragma unroll
     for (int q = 0; q < NQ; ++q) {
-      const float4 t = ld4(lg + 4 * (lane + 32 * q));
+      const float4 t = nxt[q];
       v[q][0] = t.x; v[q][1] = t.y; v[q][2] = t.z; v[q][3] = t.w;
       mx = fmaxf(mx, fmaxf(fmaxf(t.x, t.y), fmaxf(t.z, t.w)));
     }
+    const int k = k_nxt;
+    if (row + row_step < row_end) {
+#pragma unroll
+      for (int q = 0; q < NQ; ++q) nxt[q] = ld4(logits + (size_t)(row + row_step) * ncomp + 4 * (lane + 32 * q));
+      k_nxt = __ldg(rowk + row + row_step);
+    }
     mx = warp_max(mx);
-    const int k = rowk[row];
     const double tA = __ldg(tcond + 4 * k + 0), tB = __ldg(tcond + 4 * k + 1);
     const float* x = X + (size_t)row * d;
     // A row whose maximum stands alone (nothing else within 30) is one-hot to within e^-30 whatever
@@ -745,6 +802,34 @@ __global__ void __launch_bounds__(256)
     for (int q = 0; q < NQ; ++q)
 #pragma unroll
       for (int u = 0; u < 4; ++u) near += __popc(__ballot_sync(0xffffffffu, v[q][u] >= mx - 30.0f));
+    if (near == 1) {
+      // the common case, settled here: every other weight is below e^-30 of the row, hence below the 2^-40
+      // under which weights are stored as zeros, and the remaining one is 1 / (1 + less than 2^-24) = 1 in
+      // float: exactly what the general path below computes, without its exponentials and splits
+      int cmax = ncomp;
+#pragma unroll
+      for (int q = 0; q < NQ; ++q)
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (v[q][u] == mx) cmax = min(cmax, 4 * (lane + 32 * q) + u);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) cmax = min(cmax, __shfl_xor_sync(0xffffffffu, cmax, o));
+      if (store) {
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) {
+          const int c0 = 4 * (lane + 32 * q);
+          const size_t o = (size_t)row * ncomp + c0;
+          const uint32_t one = 0x3F80u;            // 1.0 in bfloat16
+          const uint2 p0 = make_uint2((cmax == c0 ? one : 0u) | (cmax == c0 + 1 ? one << 16 : 0u),
+                                      (cmax == c0 + 2 ? one : 0u) | (cmax == c0 + 3 ? one << 16 : 0u));
+          *reinterpret_cast<uint2*>(R + o) = p0;
+          *reinterpret_cast<uint2*>(R + rplane + o) = make_uint2(0u, 0u);
+          *reinterpret_cast<uint2*>(R + 2 * rplane + o) = make_uint2(0u, 0u);
+        }
+      }
+      if (pass == 0 && amax && lane == 0) amax[row] = cmax;
+      continue;
+    }
     const bool refine = near > 1;
 #pragma unroll
     for (int q = 0; q < NQ; ++q) {
@@ -797,23 +882,34 @@ __global__ void __launch_bounds__(256)
         lower |= (uint32_t)p[1][u] | (uint32_t)p[2][u];
       }
       const size_t o = (size_t)row * ncomp + 4 * (lane + 32 * q);
+      if (store) {
 #pragma unroll
-      for (int pl = 0; pl < 3; ++pl)
-        *reinterpret_cast<uint2*>(R + pl * rplane + o) = make_uint2((uint32_t)p[pl][0] | ((uint32_t)p[pl][1] << 16),
-                                                                    (uint32_t)p[pl][2] | ((uint32_t)p[pl][3] << 16));
-    }
-    if (tile_flags && __any_sync(0xffffffffu, lower != 0u) && lane == 0) tile_flags[row >> 7] = 1;
-    if (amax) {
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        nnz += __shfl_xor_sync(0xffffffffu, nnz, o);
-        cmax = min(cmax, __shfl_xor_sync(0xffffffffu, cmax, o));
-      }
-      if (lane == 0) {
-        amax[row] = (nnz == 1) ? cmax : -1;
-        if (nnz != 1 && hot_flags) hot_flags[row >> 8] = 1;
+        for (int pl = 0; pl < 3; ++pl)
+          *reinterpret_cast<uint2*>(R + pl * rplane + o) = make_uint2((uint32_t)p[pl][0] | ((uint32_t)p[pl][1] << 16),
+                                                                      (uint32_t)p[pl][2] | ((uint32_t)p[pl][3] << 16));
       }
     }
+    if (pass == 0) {
+      if (tile_flags && __any_sync(0xffffffffu, lower != 0u) && lane == 0) tile_flags[row >> 7] = 1;
+      if (amax) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          nnz += __shfl_xor_sync(0xffffffffu, nnz, o);
+          cmax = min(cmax, __shfl_xor_sync(0xffffffffu, cmax, o));
+        }
+        mixed |= (nnz != 1);
+        if (lane == 0) {
+          amax[row] = (nnz == 1) ? cmax : -1;
+          if (nnz != 1 && hot_flags) {
+            hot_flags[row >> 8] = 1;
+            if (mixed_blocks) *mixed_blocks = 1;
+          }
+        }
+      }
+    }
+  }
+  if (LAZY && pass == 0 && !__syncthreads_or(mixed)) break;   // every row of the block one-hot: nobody reads its planes
+  }
   }
 }
 
@@ -943,11 +1039,11 @@ cudaError_t launch_gemm_tc(int epi, const TcGemmArgs& g_in, const void* A_bf16, 
 }
 
 cudaError_t launch_softmax_bf16(const float* logits, const int* nrows_dev, int rows_host, int ncomp, uint16_t* R,
-                                int* amax, int* hot_flags, cudaStream_t st) {
+                                int* amax, int* hot_flags, int* mixed_blocks, cudaStream_t st) {
   int blocks = (rows_host + 7) / 8;
   if (blocks > 148 * 8) blocks = 148 * 8;
   if (blocks < 1) blocks = 1;
-  k_softmax_bf16<<<blocks, 256, 0, st>>>(logits, nrows_dev, rows_host, ncomp, R, amax, hot_flags);
+  k_softmax_bf16<<<blocks, 256, 0, st>>>(logits, nrows_dev, rows_host, ncomp, R, amax, hot_flags, mixed_blocks);
   return cudaGetLastError();
 }
 
@@ -992,14 +1088,24 @@ cudaError_t launch_split3(const float* x, size_t n, size_t plane, int nplanes, u
 cudaError_t launch_softmax_split3(const float* logits, const int* nrows_dev, int rows_host, int ncomp, int d,
                                   const float* X, const float* means, const double* musq, const float* logw,
                                   const double* tcond, const int* rowk, size_t rplane, uint16_t* R, int* tile_flags,
-                                  int* amax, int* hot_flags, cudaStream_t st) {
+                                  int* amax, int* hot_flags, int* mixed_blocks, cudaStream_t st) {
   int blocks = (rows_host + 7) / 8;
   if (blocks > 148 * 8) blocks = 148 * 8;
   if (blocks < 1) blocks = 1;
+  // with the one-hot bookkeeping and enough blocks of 256 rows to fill the machine: planes stored only where read
+  const int blocks256 = (rows_host + 255) / 256;
+  const bool lazy = amax != nullptr && hot_flags != nullptr && blocks256 >= 2 * 148;
+  if (lazy) blocks = blocks256 < 148 * 8 ? blocks256 : 148 * 8;
 #define SDS_SM3(NQ)                                                                                              \
   case NQ:                                                                                                       \
-    k_softmax_split3<NQ><<<blocks, 256, 0, st>>>(logits, nrows_dev, rows_host, d, X, means, musq, logw, tcond,   \
-                                                 rowk, rplane, R, tile_flags, amax, hot_flags);                  \
+    if (lazy)                                                                                                    \
+      k_softmax_split3<NQ, true><<<blocks, 256, 0, st>>>(logits, nrows_dev, rows_host, d, X, means, musq, logw,  \
+                                                         tcond, rowk, rplane, R, tile_flags, amax, hot_flags,    \
+                                                         mixed_blocks);                                          \
+    else                                                                                                         \
+      k_softmax_split3<NQ, false><<<blocks, 256, 0, st>>>(logits, nrows_dev, rows_host, d, X, means, musq, logw, \
+                                                          tcond, rowk, rplane, R, tile_flags, amax, hot_flags,   \
+                                                          mixed_blocks);                                         \
     break;
   switch (ncomp / 128) {
     SDS_SM3(1) SDS_SM3(2) SDS_SM3(3) SDS_SM3(4) SDS_SM3(5) SDS_SM3(6) SDS_SM3(7) SDS_SM3(8)

@@ -43,6 +43,7 @@ struct TcGemmArgs {
   // optional (mixing epilogue): one word per 256 rows of A, zero = every row of the block has a single non-zero
   // entry; tiles of such blocks are skipped altogether (launch_mix_onehot writes their rows)
   const int* hot_flags;
+  const int* mixed_blocks;  // optional, with hot_flags: device word, zero = no block needs the contraction at all
   int* tile_counts;      // optional: [0] += tiles run with the full list, [1] += tiles run with the short one,
                          // [2] += tiles skipped
   int nseg_short;
@@ -51,10 +52,10 @@ struct TcGemmArgs {
 
 bool tc_shape_ok(int N, int K);
 cudaError_t launch_gemm_tc(int epi, const TcGemmArgs& g, const void* A_bf16, const void* B_bf16, cudaStream_t st);
-// amax / hot_flags (both optional): component of every one-hot row (-1 otherwise); one word per 256 rows,
-// zeroed by the caller, raised where a row is not one-hot
+// amax / hot_flags / mixed_blocks (all optional): component of every one-hot row (-1 otherwise); one word per
+// 256 rows, zeroed by the caller, raised where a row is not one-hot; one word raised if any block holds such a row
 cudaError_t launch_softmax_bf16(const float* logits, const int* nrows_dev, int rows_host, int ncomp, uint16_t* R,
-                                int* amax, int* hot_flags, cudaStream_t st);
+                                int* amax, int* hot_flags, int* mixed_blocks, cudaStream_t st);
 // rows of the blocks the mixing GEMM skipped: out[row] = means[amax[row]], or C means + E x when xrows is given
 cudaError_t launch_mix_onehot(const void* means, bool means_bf16, const int* amax, const int* hot_flags,
                               const int* nrows_dev, int rows_host, int d, const double* tcond, const int* rowk,
@@ -69,7 +70,7 @@ cudaError_t launch_split3(const float* x, size_t n, size_t plane, int nplanes, u
 cudaError_t launch_softmax_split3(const float* logits, const int* nrows_dev, int rows_host, int ncomp, int d,
                                   const float* X, const float* means, const double* musq, const float* logw,
                                   const double* tcond, const int* rowk, size_t rplane, uint16_t* R, int* tile_flags,
-                                  int* amax, int* hot_flags, cudaStream_t st);
+                                  int* amax, int* hot_flags, int* mixed_blocks, cudaStream_t st);
 cudaError_t launch_f32_to_bf16(const float* x, size_t n, uint16_t* out, cudaStream_t st);
 
 }  // namespace sds
