@@ -420,15 +420,20 @@ def kernel_rooflines(w, variant, prof, steps, rows, cw, positions, pk, ctl, traf
                 e.update(requested_bytes_per_launch=moved / per_run_launches,
                          requested_achieved=moved / (ms / steps * 1e-3) / 1e9,
                          requested_frac=moved / (ms / steps * 1e-3) / 1e9 / hbm)
-                # the generator, not memory, bounds this kernel: Philox-4x32-10 takes forty 32 x 32-bit multiplies per
-                # four normals; derived peak: 64 such multiplies per clock and SM (half the 128 fp32 lanes) x 148 SMs
+                # the generator, not memory, bounds this kernel. Philox-4x32-10 takes twenty high-half and twenty
+                # low-half 32 x 32-bit multiplies per four normals; measured unit rates on this part: 32 high-half
+                # and 128 low-half multiplies per clock and SM, so one block keeps an SM's multiplier busy for
+                # 20/32 + 20/128 = 0.78 clocks; and the kernel issues 32 instructions per lane and normal (profiler),
+                # 128 lanes per clock and SM: one clock per block. The slower of the two bounds the kernel.
                 drawn = d * (rows - (cw if regen else 0.0))                         # normals per run (about: the last row of a
                                                                                     # window is not drafted where verify makes it)
-                mult = 10.0 * drawn
-                int_peak = SMS * 64 * pk["sm_max_mhz"] * 1e6
-                e["integer_multiplier"] = {"multiplies_per_launch": mult / per_run_launches,
-                                           "achieved_per_s": mult / (ms / steps * 1e-3), "derived_peak_per_s": int_peak,
-                                           "frac": mult / (ms / steps * 1e-3) / int_peak}
+                sm_hz = SMS * pk["sm_max_mhz"] * 1e6
+                mult_bound = 4.0 * sm_hz / (20.0 / 32.0 + 20.0 / 128.0)
+                issue_bound = 4.0 * sm_hz / (4.0 * 32.0 / 128.0)
+                rate = drawn / (ms / steps * 1e-3)
+                e["generator"] = {"normals_per_launch": drawn / per_run_launches, "achieved_normals_per_s": rate,
+                                  "multiplier_bound_normals_per_s": mult_bound, "issue_bound_normals_per_s": issue_bound,
+                                  "frac_of_multiplier_bound": rate / mult_bound, "frac_of_issue_bound": rate / issue_bound}
             elif kind == "advance":
                 per_run = 16.0 * d * cw
             elif kind == "softmax":
