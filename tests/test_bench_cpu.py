@@ -74,3 +74,29 @@ def test_lattice_energy_conventions():
     pairs = (0.5 + 0.25) ** 2 + 0.5 ** 2 + 0.25 ** 2
     site = (0.25 - 1) ** 2 + (0.0625 - 1) ** 2 + 2.0
     assert abs(once[0] - (1.5 * pairs + site)) < 1e-12 and abs(twice[0] - (3.0 * pairs + site)) < 1e-12
+
+
+def test_bench_started_without_a_launcher_becomes_n_ranks(monkeypatch):
+    """`python bench.py --gpus 4` with no launcher around it re-executes itself as four ranks through
+    sharding.launch_ranks (one per GPU, loopback rendezvous) and exits with the launcher's code; under a
+    launcher (WORLD_SIZE and RANK set) it does not launch again."""
+    import sys
+    from paper_2501_05370_b200 import sharding
+    calls = []
+    monkeypatch.setattr(sharding, "launch_ranks", lambda n, script, argv, **kw: calls.append((n, script, list(argv))) or 7)
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "4", "--steps", "2"])
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    monkeypatch.delenv("RANK", raising=False)
+    try:
+        bench.main()
+        raise AssertionError("bench.main() should have exited with the launcher's code")
+    except SystemExit as e:
+        assert e.code == 7
+    assert calls == [(4, os.path.abspath(bench.__file__), ["--gpus", "4", "--steps", "2"])]
+    # inside a rank: no second launch (run_gpu is reached instead)
+    reached = []
+    monkeypatch.setattr(bench, "run_gpu", lambda args, w: reached.append((args.gpus, w.name)))
+    monkeypatch.setenv("WORLD_SIZE", "4")
+    monkeypatch.setenv("RANK", "1")
+    bench.main()
+    assert reached == [(4, "cfg4")] and len(calls) == 1
