@@ -779,7 +779,7 @@ def test_early_exit_run_matches_oracle():
 
 @pytest.mark.gpu
 @pytest.mark.parametrize("d,L,B,mode", [(64, 8, 70, 0), (1024, 12, 40, 0), (2048, 7, 9, 0), (3072, 8, 24, 1), (3072, 8, 24, 0), (4096, 16, 12, 0), (8192, 6, 5, 0),
-                          (16384, 5, 6, 0)])
+                          (16384, 5, 6, 0), (12292, 5, 6, 0), (5000, 6, 5, 0)])
 def test_sample_all_with_fused_advance_equals_the_stepwise_calls(d, L, B, mode):
     """sds_sample_all (verify kernel advancing its chains, early exit on) against an explicit
     draft / verify / advance loop, and against the same run with the advance kernel: same bits.

@@ -286,7 +286,7 @@ def test_full_size_runs_agree_bitwise_across_kernel_options(name):
 
 @pytest.mark.parametrize("kind,d,L,B", [("gmm", 512, 9, 21), ("gmm", 1536, 7, 13), ("mlp", 3072, 8, 10), ("gmm", 4096, 6, 9),
                                          ("mlp", 8192, 5, 5), ("gmm", 16384, 6, 4), ("gmm", 512, 1, 5), ("gmm", 1024, 2, 7),
-                                         ("gmm", 2048, 32, 3)])
+                                         ("gmm", 2048, 32, 3), ("gmm", 12416, 5, 5), ("gmm", 6272, 4, 5)])
 def test_drafted_states_drawn_again_give_the_same_bits(kind, d, L, B):
     """Targets that read only the bf16 rows (the MLP, the bf16 mixture): inside sds_sample_all the draft
     kernel stores only those rows and verify runs the draft recurrence again from Y_n, the carried
