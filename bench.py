@@ -622,6 +622,8 @@ def run_gpu(args, w):
     s = gpu_sampler(sds, w, args.variant, chain_id_offset=sharding.weak_offset(rank, w.B), device=dev)
     if args.variant == "independent":
         s.set_option(s.OPT_WHOLE_CHAIN_KERNEL, 0)      # the cost ratio is about the draft-model and target kernels
+    if args.staged:
+        s.set_option(s.OPT_STAGED_WINDOWS, s.STAGED_ADAPTIVE if args.staged == "adaptive" else int(args.staged))
     B, d, K = w.B, w.d, w.K
     out = torch.empty((B, d), dtype=torch.float32, device=dev)
     calls = torch.empty((B,), dtype=torch.int32, device=dev)
@@ -793,6 +795,8 @@ def main():
     ap.add_argument("--chains", type=int, default=0, help="chains per GPU (default: the workload's own B)")
     ap.add_argument("--variant", default="default", choices=VARIANTS,
                     help="another drafter or accept test on the same workload (default: the workload's own)")
+    ap.add_argument("--staged", default="", help="evaluate every window in stages: a stage length, or 'adaptive' "
+                    "(same samples; default: whole windows, as the paper states the method)")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the per-workload table and the lattice energy statistic (profiler captures)")
     args = ap.parse_args()

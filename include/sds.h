@@ -89,6 +89,7 @@ extern "C" {
 #define SDS_GET_NFE_CALLS 15    /* int32  [B]         sequential batched target calls the chain took part in */
 #define SDS_GET_NFE_ROWS  16    /* int32  [B]         target rows evaluated for the chain */
 #define SDS_GET_CTL       17    /* int32  [16]        n_active, nrows, windows done, error word, frozen chains, ...;
+                                   [7]: chain-stages in which every position was accepted (SDS_OPT_STAGED_WINDOWS);
                                    [8], [9]: mixing-GEMM tiles of the split-precision mixture run with all six
                                    products / with the three of the first plane since sds_reset;
                                    [10]: mixing-GEMM tiles skipped since sds_reset (SDS_OPT_ONEHOT_ROWS);
@@ -277,6 +278,20 @@ int sds_sample_all(sds_ctx* ctx, float* out_dev, int32_t* nfe_calls_dev, int32_t
  * SDS_OPT_RAW_ROWS in effect the copy is not made either: the verify and advance kernels read the skipped
  * blocks' rows from the mixture's means table by component index (SDS_GET_DQ is then stale for those rows). */
 #define SDS_OPT_ONEHOT_ROWS 8
+/* SDS_OPT_STAGED_WINDOWS (default 0 = off): inside sds_sample_all, for SDS_FROZEN_PREV without a projection, every
+ * launch drafts, evaluates and verifies at most `stage` positions of each chain's window. A chain whose stage
+ * accepted all its positions continues with the REST OF THE SAME WINDOW in the next launch: its carried output
+ * stays frozen, the draws are keyed by chain and step as always, and the accept tests run in the same order, so
+ * the samples (and every accept decision) are those of whole windows of L positions, bit for bit. What changes
+ * is the work: rows after a rejection are never drafted nor given to the target, at the price of one more
+ * sequential target call for each stage a chain passes. The paper evaluates the target on all L drafted states
+ * in one batched pass (Algorithm 4); this is that window evaluated lazily, for batches in which the rows of a
+ * pass are not free. nfe_calls counts the launches a chain took part in, nfe_rows the rows evaluated for it,
+ * both as they really were. Values: 1..32 a fixed stage length; SDS_STAGED_ADAPTIVE: the length starts at L,
+ * doubles when more than half of the chain-stages of the latest finished launch passed, halves (down to 1)
+ * when fewer than an eighth did. Control word [7] counts the chain-stages that passed since reset. */
+#define SDS_OPT_STAGED_WINDOWS 9
+#define SDS_STAGED_ADAPTIVE 255
 int sds_set_option(sds_ctx* ctx, int32_t option, int64_t value);
 
 /* Temperature of the accept test (Appendix D, temperature rejection): a draft is accepted iff

@@ -325,6 +325,8 @@ class Sampler:
     OPT_RAW_ROWS = 6
     OPT_REGEN_DRAFTS = 7
     OPT_ONEHOT_ROWS = 8
+    OPT_STAGED_WINDOWS = 9
+    STAGED_ADAPTIVE = 255
 
     def set_option(self, option: int, value: int):
         self._chk(self.lib.sds_set_option(self.h, option, value), "sds_set_option")

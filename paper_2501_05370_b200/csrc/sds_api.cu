@@ -38,6 +38,7 @@ struct Layout {
   size_t Y, Dc, T, X, Dq, Xb;
   size_t n, act, rowoff, rowk, ctl;
   size_t S1, S2, ell, logU, accmask, jstar, nfe_calls, nfe_rows;
+  size_t rem;             // staged windows: positions left in a chain's window
   size_t Gk;
   size_t Gx, Gb, Pb, Dp;  // independent drafter: gathered rows (f32, bf16), its outputs per call and per row
   size_t ce;              // (C_k, E_k) of the target mixture as floats, for rows kept raw
@@ -108,6 +109,9 @@ struct sds_ctx {
   bool hot_now = false;             // likewise: rows of skipped (all one-hot) blocks are read from the means table, not stored
   bool regen_now = false;           // likewise: verify regenerates the drafted states
   bool skipx_now = false;           // likewise: the draft kernel stores only the bf16 copy of its rows
+  int staged = 0;                   // SDS_OPT_STAGED_WINDOWS: 0 off, 1..L fixed stage length, SDS_STAGED_ADAPTIVE
+  bool staged_now = false;          // set for the whole of a staged sds_sample_all
+  int cap_now = 0, cap_next = 0;    // stage length of the window being enqueued, and of the one after it
   // optional per-kernel timing: event pairs recorded around each launch, summed on read
   bool prof_on = false;
   std::vector<cudaEvent_t> prof_ev[SDS_PROF_KINDS];
@@ -185,6 +189,7 @@ void make_layout(const sds_schedule* sch, const sds_denoiser* den, const sds_den
   l.jstar = cv.take((size_t)B * 4);
   l.nfe_calls = cv.take((size_t)B * 4);
   l.nfe_rows = cv.take((size_t)B * 4);
+  l.rem = cv.take((size_t)B * 4);
   den_layout(cv, den, K, sch->tcond_dim, rows, d, tl);
   tl->xb = l.Xb;
   l.Gx = l.Gb = l.Pb = l.Dp = l.Gk = kNone;
@@ -279,6 +284,10 @@ WinArgs win_args(sds_ctx* c) {
   }
   A.regen = c->regen_now ? 1 : 0;
   A.skip_x = c->skipx_now ? 1 : 0;
+  A.staged = c->staged_now ? 1 : 0;
+  A.cap = c->cap_now;
+  A.cap_next = c->cap_next;
+  A.rem = at<int>(c, c->lay.rem);
   A.seed = c->seed; A.chain_off = (uint64_t)c->chain_off;
   A.a = at<float>(c, c->lay.a); A.c = at<float>(c, c->lay.c); A.sigma = at<float>(c, c->lay.sigma);
   A.Y = at<float>(c, c->lay.Y); A.Dc = at<float>(c, c->lay.Dc); A.T = at<float>(c, c->lay.T);
@@ -777,7 +786,9 @@ int sds_verify_window(sds_ctx* c) {
   WinArgs A = win_args(c);
   // rows drafted by k_draft (the two frozen-output modes) come with their bf16 planes
   const bool planes_ready = A.Xs != nullptr && (c->mode == SDS_FROZEN_PREV || c->mode == SDS_FROZEN_EXACT);
-  const int rc = run_denoiser(c, c->tgt, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, (int64_t)c->ub * c->L, A.Dq, planes_ready,
+  // (the host's bound on the rows: a staged window has at most cap rows per chain)
+  const int64_t rows_ub = (int64_t)c->ub * (c->staged_now ? std::min(c->cap_now, c->L) : c->L);
+  const int rc = run_denoiser(c, c->tgt, A.X, A.Xb, A.rowk, A.ctl + kCtlNRows, rows_ub, A.Dq, planes_ready,
                               c->raw_now, c->hot_now);
   if (rc != SDS_OK) return rc;
   SDS_LAUNCH(c, SDS_PROF_VERIFY, launch_verify(A, c->ub, c->stream));
@@ -824,6 +835,20 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
     c->ub = 0;
     c->state = kReady;
   } else {
+    // Staged windows: a launch drafts and verifies at most `cap` positions of every chain's window; a chain whose
+    // stage accepted everything goes on with the rest of its window in the next launch, its carried output still
+    // frozen, so the samples are those of whole windows, bit for bit, while the rows that follow a rejection are
+    // never drafted nor given to the target. The stage length follows the share of chain-stages that passed.
+    struct StageGuard {
+      sds_ctx* c;
+      ~StageGuard() { c->staged_now = false; }
+    } stage_guard{c};
+    const bool adaptive = c->staged == SDS_STAGED_ADAPTIVE;
+    c->staged_now = c->staged != 0 && c->mode == SDS_FROZEN_PREV && !c->Q;
+    c->cap_now = c->cap_next = (c->staged_now && !adaptive) ? std::min(c->staged, c->L) : c->L;
+    int cap_hist[2] = {c->cap_now, c->cap_now};
+    int cap_policy = c->cap_next;                        // the stage length the next enqueued scan will be given
+    int64_t passed_seen = 0;
     rc = sds_reset(c);
     if (rc != SDS_OK) return rc;
     // Windows are enqueued one ahead of the host's knowledge of the active count: after window w
@@ -861,6 +886,9 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
       c->skipx_now = c->regen_now;
       // where the register-resident verify kernel runs, it also advances its chains and compacts
       c->fusing = c->fuse_advance && (verify_can_advance(A) || c->regen_now);
+      c->cap_now = c->cap_next;                          // what the last scan sized this window's rows for
+      c->cap_next = cap_policy;                          // what this window's scan sizes the next window's rows for
+      cap_hist[w & 1] = c->cap_now;
       if (w == 0) {                                      // which of these paths the run may take (read back with the control words)
         const bool may_regen = c->regen && c->fuse_advance && bf16_only && verify_can_regen(A);
         c->h_pin[48] = (may_regen ? 1 : 0) | (c->hot_now ? 4 : 0);
@@ -888,6 +916,15 @@ int sds_sample_all(sds_ctx* c, float* out_dev, int32_t* nfe_calls_dev, int32_t* 
         const int64_t pos = (int64_t)(uint32_t)seen[kCtlPositions];
         if (na_before > 0) mean_positions = (double)(pos - pos_seen) / na_before;
         pos_seen = pos;
+        if (c->staged_now && adaptive && na_before > 0) {
+          // window w-1 ran with cap_hist[(w-1)&1]; the scan of window w is enqueued already, so the new length
+          // reaches window w+2
+          const double pass = (double)((int64_t)(uint32_t)seen[kCtlStagePassed] - passed_seen) / na_before;
+          const int used = cap_hist[(w - 1) & 1];
+          if (pass > 0.5) cap_policy = std::min(c->L, std::max(cap_policy, 2 * used));
+          else if (pass < 0.125) cap_policy = std::max(1, std::min(cap_policy, used / 2));
+        }
+        passed_seen = (int64_t)(uint32_t)seen[kCtlStagePassed];
         na_before = na;
         c->ub = na;
       }
@@ -974,6 +1011,7 @@ int sds_set_state(sds_ctx* c, const float* Y_dev, const int32_t* n_dev, const fl
   if (Dc_dev) SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.Dc, Dc_dev, Bd, cudaMemcpyDeviceToDevice, c->stream));
   if (n_dev)
     SDS_CU(c, cudaMemcpyAsync(c->ws + c->lay.n, n_dev, (size_t)c->B * 4, cudaMemcpyDeviceToDevice, c->stream));
+  SDS_CU(c, cudaMemsetAsync(c->ws + c->lay.rem, 0, (size_t)c->B * 4, c->stream));   // no window is under way
   SDS_LAUNCH(c, SDS_PROF_AUX, launch_compact(win_args(c), c->stream));
   c->ub = (int)c->B;
   return SDS_OK;
@@ -1021,6 +1059,10 @@ int sds_set_option(sds_ctx* c, int32_t option, int64_t value) {
     case SDS_OPT_RAW_ROWS: c->raw_rows = value != 0; return SDS_OK;
     case SDS_OPT_REGEN_DRAFTS: c->regen = value != 0; c->regen_always = value == 2; return SDS_OK;
     case SDS_OPT_ONEHOT_ROWS: c->onehot = value != 0; return SDS_OK;
+    case SDS_OPT_STAGED_WINDOWS:
+      if (value < 0 || (value > 32 && value != SDS_STAGED_ADAPTIVE)) return SDS_EINVAL;
+      c->staged = (int)value;
+      return SDS_OK;
     default: return SDS_EINVAL;
   }
 }

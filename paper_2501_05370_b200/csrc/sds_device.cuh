@@ -23,7 +23,7 @@ enum Ctl : int {
   kCtlFrozen = 4,     // chains frozen because of a non-finite log ratio
   kCtlDone = 5,       // block-completion counter of the advance kernel
   kCtlTcError = 6,    // set by a tensor-core kernel whose bounded wait gave up
-  kCtlSpare1 = 7,
+  kCtlStagePassed = 7, // staged windows: chain-stages since reset in which every position was accepted
   kCtlTilesFull = 8,  // mixing-GEMM tiles of the split-precision mixture run with all six products since reset
   kCtlTilesBrief = 9, // ... and with the three products of the first plane only
   kCtlTilesSkipped = 10, // mixing-GEMM tiles skipped since reset because every row of their block was one-hot

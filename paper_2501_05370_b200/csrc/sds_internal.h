@@ -27,6 +27,9 @@ struct WinArgs {
   int regen;             // verify draws the drafted states again from Y_n, the carried output and the noise instead of
                          // reading them (needs fuse_advance; see verify_can_regen)
   int skip_x;            // the draft kernel stores only the bf16 copies of its rows (nothing reads the float rows)
+  int staged;            // windows are evaluated in stages of at most `cap` positions (see window_len)
+  int cap, cap_next;     // stage length of this launch, and of the next one (the active-list scan sizes its rows)
+  int* rem;              // [B] positions left in a window whose stage accepted everything, else 0
   uint64_t seed;
   uint64_t chain_off;
   const float* a;        // [K]

@@ -19,7 +19,23 @@ struct Group {
   __device__ static int lane() { return threadIdx.x % TPC; }
 };
 
-__device__ __forceinline__ int window_len(const WinArgs& A, int nb) { return min(A.L, A.K - nb); }
+// Positions left in chain b's window: a window of L positions (fewer at the end of the chain), or
+// what remains of one that is being evaluated in stages.
+__device__ __forceinline__ int window_left(const WinArgs& A, int b, int nb) {
+  if (A.staged) {
+    const int r = __ldcg(A.rem + b);
+    if (r > 0) return r;
+  }
+  return min(A.L, A.K - nb);
+}
+// Positions of chain b this launch drafts and verifies: the window, or (staged windows) its next `cap`
+// positions. A stage that accepts all its positions leaves the carried output frozen and the rest of the
+// window to the next launch, so the draws, the tests and their order are those of the whole window.
+__device__ __forceinline__ int window_len(const WinArgs& A, int b, int nb, int cap) {
+  const int left = window_left(A, b, nb);
+  return A.staged ? min(left, cap) : left;
+}
+__device__ __forceinline__ int window_len(const WinArgs& A, int b, int nb) { return window_len(A, b, nb, A.cap); }
 
 // ---------------------------------------------------------------------------------------
 // compaction: dense ascending list of chains with n < K and their first rows (one CTA)
@@ -35,7 +51,7 @@ __device__ void compact_scan(const WinArgs& A) {
   int cnt = 0, rows = 0;
   for (int b = b0; b < b1; ++b) {
     const int nb = __ldcg(A.n + b);
-    if (nb < A.K) { cnt += 1; rows += min(A.L, A.K - nb); }
+    if (nb < A.K) { cnt += 1; rows += window_len(A, b, nb, A.cap_next); }
   }
   int c = cnt, r = rows;                  // inclusive warp scans
 #pragma unroll
@@ -57,7 +73,7 @@ __device__ void compact_scan(const WinArgs& A) {
       A.act[pos] = b;
       A.rowoff[pos] = row;
       pos += 1;
-      row += min(A.L, A.K - nb);
+      row += window_len(A, b, nb, A.cap_next);
     }
   }
   if (tid == 0) {
@@ -151,6 +167,7 @@ __global__ void __launch_bounds__(kBlock) k_init(WinArgs A) {
     A.nfe_rows[b] = first;
     A.accmask[b] = 0u;
     A.jstar[b] = 0;
+    A.rem[b] = 0;
   }
 }
 
@@ -213,7 +230,7 @@ __global__ void __launch_bounds__(kBlock) k_draft(WinArgs A) {
   const int s = G::slot(), t = G::lane();
   if (s >= A.ctl[kCtlNActive]) return;
   const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
-  const int Lt = window_len(A, nb);
+  const int Lt = window_len(A, b, nb);
   const uint64_t bg = A.chain_off + (uint64_t)b;
   const size_t cb = (size_t)b * A.d;
   if (t < Lt) A.rowk[r0 + t] = nb + t;            // TPC >= 32 >= Lt
@@ -268,7 +285,7 @@ __global__ void __launch_bounds__(kBlock) k_gather_pos(WinArgs A, int j) {
   const int s = G::slot(), t = G::lane();
   if (s >= A.ctl[kCtlNActive]) return;
   const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
-  const int Lt = window_len(A, nb);
+  const int Lt = window_len(A, b, nb);
   const int jj = min(j, Lt);
   const float* src = (j == 1) ? A.Y + (size_t)b * A.d : A.X + (size_t)(r0 + jj - 1) * A.d;
   const size_t go = (size_t)s * A.d, x0 = (size_t)r0 * A.d;
@@ -305,7 +322,7 @@ __global__ void __launch_bounds__(kBlock) k_draft_pos(WinArgs A, int j) {
   const int s = G::slot(), t = G::lane();
   if (s >= A.ctl[kCtlNActive]) return;
   const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
-  const int Lt = window_len(A, nb);
+  const int Lt = window_len(A, b, nb);
   if (j > Lt) return;
   const int k = nb + j - 1;
   const uint64_t bg = A.chain_off + (uint64_t)b;
@@ -359,7 +376,7 @@ __global__ void __launch_bounds__(kBlock) k_picard_start(WinArgs A) {
   const int s = G::slot(), t = G::lane();
   if (s >= A.ctl[kCtlNActive]) return;
   const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
-  const int Lt = window_len(A, nb);
+  const int Lt = window_len(A, b, nb);
   const size_t cb = (size_t)b * A.d;
   if (t < Lt) A.rowk[r0 + t] = nb + t;
   if (VEC == 4) {
@@ -391,7 +408,7 @@ __global__ void __launch_bounds__(kBlock) k_picard_step(WinArgs A) {
   const int s = G::slot(), t = G::lane();
   if (s >= A.ctl[kCtlNActive]) return;
   const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
-  const int Lt = window_len(A, nb);
+  const int Lt = window_len(A, b, nb);
   if (VEC == 4) {
     for (int i = t * 4; i < A.d; i += TPC * 4) {
       float4 f = ld4(A.X + (size_t)r0 * A.d + i);                 // previous iterate's F_j
@@ -424,7 +441,7 @@ __global__ void __launch_bounds__(kBlock) k_picard_draft(WinArgs A) {
   const int s = G::slot(), t = G::lane();
   if (s >= A.ctl[kCtlNActive]) return;
   const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
-  const int Lt = window_len(A, nb);
+  const int Lt = window_len(A, b, nb);
   const uint64_t bg = A.chain_off + (uint64_t)b;
   const size_t cb = (size_t)b * A.d;
   if (VEC == 4) {
@@ -476,7 +493,7 @@ __global__ void __launch_bounds__(kBlock) k_project(WinArgs A) {
   const int s = blockIdx.x, j = blockIdx.y + 1;
   if (s >= A.ctl[kCtlNActive]) return;
   const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
-  const int Lt = window_len(A, nb);
+  const int Lt = window_len(A, b, nb);
   if (j > Lt) return;
   const int d = A.d, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const size_t cb = (size_t)b * d;
@@ -535,7 +552,7 @@ __global__ void __launch_bounds__(kBlock) k_verify(WinArgs A) {
   const int lane = threadIdx.x & 31, warp = t >> 5;
   if (s >= A.ctl[kCtlNActive]) return;              // uniform per group (a warp, or the whole CTA)
   const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
-  const int Lt = window_len(A, nb);
+  const int Lt = window_len(A, b, nb);
   const uint64_t bg = A.chain_off + (uint64_t)b;
   const size_t cb = (size_t)b * A.d;
 
@@ -708,7 +725,9 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t,
   const int lane = threadIdx.x & 31, warp = t >> 5;
   const bool fa = A.fuse_advance != 0;                 // also do this chain's part of the advance step
   const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
-  const int Lt = window_len(A, nb);
+  const int left = window_left(A, b, nb);
+  const int Lt = A.staged ? min(left, A.cap) : left;
+  const bool more = Lt < left;                           // staged window: positions remain after this launch's
   const uint64_t bg = A.chain_off + (uint64_t)b;
   const size_t cb = (size_t)b * A.d;
   const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -869,6 +888,7 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t,
           const int i = (t + e * TPC) * 4;
           if (i < A.d) {
             st4(A.Y + cb + i, REGEN ? vp[e] : ld4(A.T + cb + i));   // REGEN: every block ran, vp holds W_Lt
+            if (more) continue;                                     // the window goes on: the carried output stays frozen
             float4 q = raw_row4(A, r0 + Lt - 1, raw_row_component(A, r0 + Lt - 1), i);
             if (A.raw_ce) {
               const float2 ce = __ldg(A.raw_ce + nb + Lt - 1);
@@ -881,10 +901,15 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t,
         }
         if (t == 0) {
           A.n[b] = nb + Lt;
+          if (A.staged) {
+            A.rem[b] = left - Lt;
+            atomicAdd(A.ctl + kCtlStagePassed, 1);
+          }
           count_window(A, b, Lt);
         }
       } else if (t == 0) {                               // non-finite log ratio: stop this chain
         A.n[b] = A.K;
+        if (A.staged) A.rem[b] = 0;
         atomicAdd(A.ctl + kCtlFrozen, 1);
       }
     }
@@ -927,6 +952,7 @@ __device__ __forceinline__ void verify_reg_chain(const WinArgs& A, int s, int t,
   }
   if (fa && t == 0) {
     A.n[b] = nb + jstar;
+    if (A.staged) A.rem[b] = 0;                          // a rejection ends the window
     count_window(A, b, Lt);
   }
 }
@@ -953,8 +979,10 @@ __global__ void __launch_bounds__(kBlock) k_advance(WinArgs A) {
   const int n_active = A.ctl[kCtlNActive];
   if (s < n_active) {
     const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
-    const int Lt = window_len(A, nb);
+    const int left = window_left(A, b, nb);
+    const int Lt = A.staged ? min(left, A.cap) : left;
     const int js = A.jstar[b];
+    const bool more = js > Lt && Lt < left;              // staged window, every position of this stage accepted
     const size_t cb = (size_t)b * A.d;
     if (js >= 1) {
       const int adv = min(js, Lt);
@@ -970,6 +998,7 @@ __global__ void __launch_bounds__(kBlock) k_advance(WinArgs A) {
             const int i = i0 + u * TPC * 4;
             if (i < A.d) {
               vy[u] = ld4(src + i);
+              if (more) continue;                        // the carried output stays frozen for the rest of the window
               vd[u] = raw_row4(A, r0 + adv - 1, dcomp, i);
               if (A.raw_ce) {
                 const float2 ce = __ldg(A.raw_ce + nb + adv - 1);
@@ -980,21 +1009,29 @@ __global__ void __launch_bounds__(kBlock) k_advance(WinArgs A) {
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
             const int i = i0 + u * TPC * 4;
-            if (i < A.d) { st4(A.Y + cb + i, vy[u]); st4(A.Dc + cb + i, vd[u]); }
+            if (i < A.d) {
+              st4(A.Y + cb + i, vy[u]);
+              if (!more) st4(A.Dc + cb + i, vd[u]);
+            }
           }
         }
       } else {
         for (int i = t; i < A.d; i += TPC) {
           A.Y[cb + i] = src[i];
-          A.Dc[cb + i] = dsrc[i];
+          if (!more) A.Dc[cb + i] = dsrc[i];
         }
       }
       if (t == 0) {
         A.n[b] = nb + adv;
+        if (A.staged) {
+          A.rem[b] = more ? left - Lt : 0;
+          if (js > Lt) atomicAdd(A.ctl + kCtlStagePassed, 1);
+        }
         count_window(A, b, Lt);
       }
     } else if (t == 0) {                              // non-finite log ratio: stop this chain
       A.n[b] = A.K;
+      if (A.staged) A.rem[b] = 0;
       atomicAdd(A.ctl + kCtlFrozen, 1);
     }
   }

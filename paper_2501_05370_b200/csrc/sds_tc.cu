@@ -1009,8 +1009,13 @@ cudaError_t launch_gemm_tc(int epi, const TcGemmArgs& g_in, const void* A_bf16, 
   if (g.nseg > 8 || g.nplanes < 1 || g.nplanes > 3) return cudaErrorInvalidValue;
   if (!tc_shape_ok(g.N, g.K) || g.rows_cap <= 0 || g.rows_host > g.rows_cap) return cudaErrorInvalidValue;
   if (g.rows_host <= 0) return cudaSuccess;
-  const bool wide = (g.N % 256) == 0;
-  const bool pair = wide && g.pair != 0;
+  // Few rows (a staged window late in a chain): the largest tile shape that still gives every SM, or SM pair, a
+  // tile; below that the smallest one. A tile's main loop is as long as K whatever its shape, so with fewer
+  // tiles than SMs the time is one tile's time and smaller tiles are shorter ones.
+  const int64_t units = ((int64_t)g.rows_host + BM - 1) / BM * (g.N / 128);   // 128 x 128 blocks of the output
+  const bool few = units < 2 * 148;
+  const bool wide = (g.N % 256) == 0 && !(few && units < 148);
+  const bool pair = wide && g.pair != 0 && !few;
   const int tm = pair ? 2 * BM : BM;
   const int m_tiles = (g.rows_host + tm - 1) / tm;
   int tiles = m_tiles * (g.N / (wide ? 256 : 128));
@@ -1023,7 +1028,7 @@ cudaError_t launch_gemm_tc(int epi, const TcGemmArgs& g_in, const void* A_bf16, 
     }                                                                                      \
     return wide ? launch_t<256, E, false>(g, A_bf16, B_bf16, tiles, st) : launch_t<128, E, false>(g, A_bf16, B_bf16, tiles, st);
   // long contractions with the short logits epilogue: tiles of 256 x 512 on one accumulator (see TileCfg)
-  if (epi == kEpiGmmLogits && pair && (g.N % 512) == 0 && g.K >= 4096 && g.nseg == 1) {
+  if (epi == kEpiGmmLogits && pair && (g.N % 512) == 0 && g.K >= 4096 && g.nseg == 1 && units >= 4 * 148) {
     const cudaError_t e_ = launch_t<512, kEpiGmmLogits, true>(g, A_bf16, B_bf16, m_tiles * (g.N / 512), st);
     if (e_ != cudaErrorLaunchOutOfResources) return e_;
   }

@@ -868,3 +868,41 @@ def test_sequential_target_calls_fall_with_the_window_size(d):
     assert calls[0] == 1 + 200
     assert all(a > b for a, b in zip(calls, calls[1:])), calls
     assert calls[-1] < 0.6 * 200
+
+
+# ----------------------------------------------------------------------------------------
+# staged windows: the same window evaluated a few positions per launch
+# ----------------------------------------------------------------------------------------
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("d,L,B", [(64, 8, 70), (1000, 12, 20), (1027, 5, 9), (3072, 8, 24), (16384, 16, 6)])
+def test_staged_windows_give_the_samples_of_whole_windows(d, L, B):
+    """Algorithm 4 evaluated lazily: every launch takes at most `stage` positions of each chain's window and a
+    chain that passed its stage goes on with the rest of the SAME window (carried output frozen). Final states
+    bit for bit those of whole windows, for every stage length, with the advance step inside verify or in its own
+    kernel; only the work differs: never more target rows, never fewer sequential calls."""
+    w = wl.WORKLOADS["cfg2"].scaled(B=B, d=d, K=3 * L + 7, L=L)
+    gp = w.gmm_params(d=d, ncomp=8)
+    s = sds.sampler_for(w, gmm=gp, seed=91)
+    s.set_option(s.OPT_WHOLE_CHAIN_KERNEL, 0)
+    ref = [x.cpu().numpy() for x in s.sample_all()]
+    assert int(s.get(sb.GET_CTL)[7]) == 0
+    assert np.all(np.isfinite(ref[0]))
+    for fuse in (1, 0):
+        s.set_option(s.OPT_FUSE_ADVANCE, fuse)
+        for stage in (1, 2, 3, L - 1, L, s.STAGED_ADAPTIVE):
+            s.set_option(s.OPT_STAGED_WINDOWS, stage)
+            got = [x.cpu().numpy() for x in s.sample_all()]
+            assert np.array_equal(got[0], ref[0]), (fuse, stage)
+            assert np.all(got[2] <= ref[2]) and np.all(got[1] >= ref[1]), (fuse, stage)
+            if stage == L:
+                assert np.array_equal(got[1], ref[1]) and np.array_equal(got[2], ref[2])
+            if stage == 1:                                 # one row per launch: a call per step, no row wasted
+                assert np.array_equal(got[2], got[1]) and np.all(got[1] == w.K + 1)
+            assert np.array_equal(s.get(sb.GET_N), np.full(B, w.K))
+    s.set_option(s.OPT_STAGED_WINDOWS, 0)
+    s.set_option(s.OPT_FUSE_ADVANCE, 1)
+    again = [x.cpu().numpy() for x in s.sample_all()]
+    assert all(np.array_equal(x, y) for x, y in zip(again, ref))
+    s.close()

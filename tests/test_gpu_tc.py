@@ -330,3 +330,28 @@ def test_drafted_states_drawn_again_give_the_same_bits(kind, d, L, B):
     if kind == "gmm" and L >= 5:                          # (the random network's drafts are rejected at once)
         assert len(set(adv[adv > 0].tolist())) >= 3       # the windows did end at several different positions
     s.close()
+
+
+@pytest.mark.parametrize("kind,d,L,B", [("gmm", 1536, 7, 13), ("mlp", 3072, 8, 10), ("gmm", 16384, 6, 4), ("gmm", 2048, 32, 3)])
+def test_staged_windows_on_the_tensor_core_targets(kind, d, L, B):
+    """Staged windows with the bf16 targets: states drafted again or read back, one-hot rows read from the means
+    table, every stage length: the final states of whole windows, bit for bit."""
+    K = 3 * L + 4
+    if kind == "mlp":
+        w = wl.WORKLOADS["cfg3"].scaled(d=d, B=B, L=L, K=K, mlp_dims=[d, 256, d])
+        s = sds.sampler_for(w, mlp=w.mlp_params(), seed=83)
+    else:
+        w = wl.WORKLOADS["cfg4"].scaled(d=d, B=B, L=L, K=K)
+        s = sds.sampler_for(w, gmm=w.gmm_params(d=d, ncomp=128), seed=83)
+    ref = [x.cpu().numpy() for x in s.sample_all()]
+    assert np.all(np.isfinite(ref[0]))
+    for regen in (1, 2, 0):
+        s.set_option(s.OPT_REGEN_DRAFTS, regen)
+        for stage in (1, 2, 3, L, s.STAGED_ADAPTIVE):
+            s.set_option(s.OPT_STAGED_WINDOWS, stage)
+            got = [x.cpu().numpy() for x in s.sample_all()]
+            assert np.array_equal(got[0], ref[0]), (regen, stage)
+            assert np.all(got[2] <= ref[2]) and np.all(got[1] >= ref[1]), (regen, stage)
+            if stage == L:
+                assert np.array_equal(got[1], ref[1]) and np.array_equal(got[2], ref[2])
+    s.close()
