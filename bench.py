@@ -492,6 +492,28 @@ def acceptance_by_step(sds, w, dev, variant: str = "default", chains: int = 64, 
             "rate": [round(float(a / t), 4) if t > 0 else None for a, t in zip(accepted, tested)]}
 
 
+def staged_run(s, w, out, calls, rows, ref_out, steps: int):
+    """ms per run and counters of sds_sample_all with SDS_OPT_STAGED_WINDOWS adaptive on an existing sampler; the
+    final states must equal ref_out (the whole-window run's) bit for bit."""
+    import torch
+    st = torch.cuda.current_stream()
+    s.set_option(s.OPT_STAGED_WINDOWS, s.STAGED_ADAPTIVE)
+    for _ in range(2):
+        s.sample_all(out, calls, rows)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(st)
+    for _ in range(steps):
+        s.sample_all(out, calls, rows)
+    e1.record(st)
+    e1.synchronize()
+    s.set_option(s.OPT_STAGED_WINDOWS, 0)
+    ms = e0.elapsed_time(e1) / steps
+    c, r = calls.cpu().numpy().astype(np.int64), rows.cpu().numpy().astype(np.int64)
+    return {"ms_per_run": ms, "chain_steps_per_s": w.B * w.K / (ms * 1e-3), "mean_target_calls": float(c.mean()),
+            "mean_target_rows": float(r.mean()), "same_samples": bool(torch.equal(out, ref_out)), "steps_timed": steps,
+            "stage": "adaptive"}
+
+
 def quick_config(sds, name, dev, steps: int = 5, warmup: int = 2):
     """ms per run, chain-steps/s and the counters of another workload, in the same process."""
     import torch
@@ -512,12 +534,15 @@ def quick_config(sds, name, dev, steps: int = 5, warmup: int = 2):
     ms = e0.elapsed_time(e1) / steps
     c, r = calls.cpu().numpy().astype(np.int64), rows.cpu().numpy().astype(np.int64)
     rws, cw = run_counts(w, "default", c, r)
+    res = {"B": w.B, "d": w.d, "L": w.L, "K": w.K, "ms_per_run": ms, "chain_steps_per_s": w.B * w.K / (ms * 1e-3),
+           "mean_target_calls": float(c.mean()), "mean_target_rows": float(r.mean()),
+           "mean_advance": float(w.K * w.B / max(cw, 1.0)), "steps_timed": steps}
+    if name in ("cfg3", "cfg4", "cfg5"):                   # (cfg1, cfg2 run as one whole-chain launch)
+        res["staged_windows"] = staged_run(s, w, out, calls, rows, out.clone(), steps)
     s.close()
     del out
     torch.cuda.empty_cache()
-    return {"B": w.B, "d": w.d, "L": w.L, "K": w.K, "ms_per_run": ms, "chain_steps_per_s": w.B * w.K / (ms * 1e-3),
-            "mean_target_calls": float(c.mean()), "mean_target_rows": float(r.mean()),
-            "mean_advance": float(w.K * w.B / max(cw, 1.0)), "steps_timed": steps}
+    return res
 
 
 def phi4_energies(x, side, beta):
@@ -745,6 +770,11 @@ def run_gpu(args, w):
                                   pk, ctl_all, {}, {"regen": False})
         extra["rooflines_every_position"] = [e for e in rl_all if e["kernel"] in ("verify", "draft", "advance")]
         s.set_option(s.OPT_VERIFY_EARLY_EXIT, 1); s.set_option(s.OPT_REGEN_DRAFTS, 1)
+    if prof.get("verify", (0, 0))[1] > 0 and args.variant == "default" and not args.no_extras and not args.staged:
+        # the same run with every window evaluated in stages (same samples, checked here against the timed run's):
+        # reported beside the headline, which stays on whole windows as the paper states the method
+        ref_out = out.clone()
+        extra["staged_windows"] = staged_run(s, w, out, calls, rows, ref_out, min(steps, 5))
     if w.denoiser == "phi4" and not args.no_extras:
         extra["phi4_energy"] = phi4_energy_statistic(sds, w, dev)
     if args.variant == "independent":
