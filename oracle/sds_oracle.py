@@ -471,7 +471,7 @@ def picard_trajectory(denoise, a_det, c_det, Y, D_c, n, Lt, iters):
 
 
 def speculative_chain(denoise, a, c, sigma, L, seed, b, d, mode=FROZEN_PREV, Y0=None,
-                      record=False, decide_f32=True, draft_denoise=None, tau=1.0, proj=None, picard=None):
+                      record=False, decide_f32=True, draft_denoise=None, tau=1.0, proj=None, picard=None, stage=None):
     """Algorithm 4 for chain b with the frozen-target drafter, or (mode INDEPENDENT) with the draft
     model draft_denoise(x, k): m^p_k(y) = a_k y + c_k D^p(y, k) evaluated at every drafted state.
 
@@ -483,9 +483,18 @@ def speculative_chain(denoise, a, c, sigma, L, seed, b, d, mode=FROZEN_PREV, Y0=
     output is already known; the verify call evaluates positions 2..Lt. The carried output (start
     of the next window's Picard sequence) follows the FROZEN_PREV rule.
 
+    stage (FROZEN_PREV only; None = the algorithm as printed): the window of Algorithm 4 evaluated lazily, at
+    most `stage` positions per target call. The accept tests of a window use only the window's frozen output,
+    the drafted states and the draws keyed by (chain, step), so a window whose first `stage` positions were all
+    accepted can draft, evaluate and test its next positions afterwards with the same frozen output: the same
+    states and decisions as the one batched call, fewer rows evaluated after a rejection (nfe_rows), one more
+    sequential call for each stage passed (nfe_calls). `adv` then lists the advance of each call.
+
     denoise(x, k) -> D; transition means are a_k y + c_k D, std sigma_k.
     Returns dict(Y, nfe_calls, nfe_rows, adv (list), windows (list of per-window records if record)).
     """
+    if stage is not None and (mode != FROZEN_PREV or stage < 1):
+        raise ValueError("staged evaluation is defined for the carried-output drafter")
     K = len(a)
     Y = normals(seed, STREAM_INIT, b, 0, d) if Y0 is None else np.asarray(Y0, dtype=np.float64).copy()
     n = 0
@@ -498,8 +507,13 @@ def speculative_chain(denoise, a, c, sigma, L, seed, b, d, mode=FROZEN_PREV, Y0=
         nfe_rows += 1
     advs = []
     windows = []
+    left = 0                               # staged evaluation: positions of the current window not yet tested
     while n < K:
         Lt = min(L, K - n)
+        if stage is not None:
+            if left == 0:
+                left = Lt                  # a new window
+            Lt = min(left, stage)
         W = np.empty((Lt + 1, d))
         W[0] = Y
         Dq = np.empty((Lt, d))
@@ -554,7 +568,11 @@ def speculative_chain(denoise, a, c, sigma, L, seed, b, d, mode=FROZEN_PREV, Y0=
             windows.append(dict(n=n, W=W.copy(), Dq=Dq.copy(), D_c=(Dp if mode == INDEPENDENT else D_c).copy(),
                                 logU=logU, xi=xi, M_p=None if Mp is None else Mp.copy(), **v))
         Y = W[adv].copy()
-        D_c = Dq[adv - 1].copy()
+        if stage is not None and v["jstar"] > Lt and Lt < left:
+            left -= Lt                     # every position of the stage accepted: the window goes on, output frozen
+        else:
+            left = 0
+            D_c = Dq[adv - 1].copy()
         n += adv
         advs.append(adv)
     return dict(Y=Y, nfe_calls=nfe_calls, nfe_rows=nfe_rows, adv=advs, windows=windows)

@@ -906,3 +906,24 @@ def test_staged_windows_give_the_samples_of_whole_windows(d, L, B):
     again = [x.cpu().numpy() for x in s.sample_all()]
     assert all(np.array_equal(x, y) for x, y in zip(again, ref))
     s.close()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("stage", [1, 3, 5])
+def test_staged_free_run_against_the_oracle_counters(stage):
+    """A fixed stage length, chain by chain against the oracle's lazily evaluated windows: final state, sequential
+    target calls and target rows (a chain that differs must show a rounding-band event in the oracle's record)."""
+    w = wl.WORKLOADS["cfg2"].scaled(B=48, K=60)
+    gp = w.gmm_params()
+    s = sds.sampler_for(w, gmm=gp, seed=w.sample_seed)
+    s.set_option(s.OPT_WHOLE_CHAIN_KERNEL, 0)
+    s.set_option(s.OPT_STAGED_WINDOWS, stage)
+    out, calls, rows = [x.cpu().numpy() for x in s.sample_all()]
+    assert int(s.get(sb.GET_CTL)[7]) > 0 or stage >= w.L
+    den, a, c, sig = oracle_setup(w, gmm=gp)
+    bad = 0
+    for b in range(0, w.B, 3):
+        r = o.speculative_chain(den, a, c, sig, w.L, w.sample_seed, b, w.d, record=True, stage=stage)
+        bad += not chain_matches_or_band(r, calls[b], rows[b], out[b])
+    assert bad <= 1
+    s.close()

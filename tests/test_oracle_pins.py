@@ -812,3 +812,34 @@ def test_picard_drafter_keeps_the_target_law():
         se = math.sqrt(S[:, i].var() / N + P[:, i].var() / N)
         assert abs(S[:, i].mean() - P[:, i].mean()) < 4 * se
     assert _mmd_perm_pvalue(S, P, np.random.default_rng(3)) > 0.01
+
+
+def test_staged_evaluation_of_a_window_changes_no_state_and_no_decision():
+    """Algorithm 4 with its window evaluated a few positions per target call: the final state and the sequence of
+    accepted steps are those of the one batched call, exactly (fp64, same operations); only the counters move:
+    never more rows, never fewer calls; stage >= L is the algorithm as printed; stage 1 is one row per step."""
+    d, K, L = 6, 60, 7
+    rng = np.random.default_rng(11)
+    means = rng.normal(0, 2.0, size=(5, d))
+    logw = np.log(np.full(5, 0.2))
+    beta = np.linspace(1e-4, 0.05, K)
+    a, c, sig, abar = o.ddpm_affine(beta)
+    den = lambda x, k: o.gmm_posterior_mean(x, abar[k], means, logw, 0.4)
+    for b in range(6):
+        ref = o.speculative_chain(den, a, c, sig, L, 123, b, d, record=True)
+        steps_ref = np.cumsum(ref["adv"])
+        for stage in (1, 2, 3, L - 1, L, L + 5):
+            r = o.speculative_chain(den, a, c, sig, L, 123, b, d, stage=stage, record=True)
+            assert np.array_equal(r["Y"], ref["Y"]), (b, stage)
+            assert r["nfe_rows"] <= ref["nfe_rows"] and r["nfe_calls"] >= ref["nfe_calls"]
+            # every state the whole-window run passed through is passed through by the staged run
+            assert set(steps_ref.tolist()) <= set(np.cumsum(r["adv"]).tolist())
+            if stage >= L:
+                assert r["nfe_rows"] == ref["nfe_rows"] and r["nfe_calls"] == ref["nfe_calls"] and r["adv"] == ref["adv"]
+            if stage == 1:
+                assert r["nfe_calls"] == K + 1 and r["nfe_rows"] == K + 1
+        # rows saved are exactly the positions behind a rejection that the batched call evaluated for nothing
+        r2 = o.speculative_chain(den, a, c, sig, L, 123, b, d, stage=2)
+        assert r2["nfe_rows"] < ref["nfe_rows"]
+    with pytest.raises(ValueError):
+        o.speculative_chain(den, a, c, sig, L, 123, 0, d, mode=o.FROZEN_EXACT, stage=2)
