@@ -124,3 +124,24 @@ def test_sampler_refuses_to_run_without_cuda():
     w = wl.WORKLOADS["cfg1"]
     with pytest.raises(RuntimeError):
         sds.sampler_for(w)
+
+
+def test_binding_constants_equal_the_header_macros():
+    """Every SDS_OPT_* / SDS_GET_* / SDS_PROF_* macro and status code the binding names has the header's value."""
+    txt = open(os.path.join(ROOT, "include", "sds.h")).read()
+    macros = {m.group(1): int(m.group(2), 0) for m in re.finditer(r"#define\s+(SDS_[A-Z0-9_]+)\s+\(?(-?\d+)\)?", txt)}
+    assert macros["SDS_OPT_STAGED_WINDOWS"] == sb.Sampler.OPT_STAGED_WINDOWS
+    assert macros["SDS_STAGED_ADAPTIVE"] == sb.Sampler.STAGED_ADAPTIVE
+    checked = 0
+    for name, val in macros.items():
+        if name.startswith("SDS_OPT_"):
+            assert getattr(sb.Sampler, name[4:]) == val, name
+            checked += 1
+        elif name.startswith("SDS_GET_") and hasattr(sb, name[4:]):
+            assert getattr(sb, name[4:]) == val, name
+            checked += 1
+        elif hasattr(sb, name):
+            assert getattr(sb, name) == val, name
+            checked += 1
+    assert checked >= 25
+    assert len(sb.Sampler.PROF_KINDS) == macros["SDS_PROF_KINDS"]
