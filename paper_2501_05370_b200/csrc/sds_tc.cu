@@ -1009,13 +1009,14 @@ cudaError_t launch_gemm_tc(int epi, const TcGemmArgs& g_in, const void* A_bf16, 
   if (g.nseg > 8 || g.nplanes < 1 || g.nplanes > 3) return cudaErrorInvalidValue;
   if (!tc_shape_ok(g.N, g.K) || g.rows_cap <= 0 || g.rows_host > g.rows_cap) return cudaErrorInvalidValue;
   if (g.rows_host <= 0) return cudaSuccess;
-  // Few rows (a staged window late in a chain): the largest tile shape that still gives every SM, or SM pair, a
-  // tile; below that the smallest one. A tile's main loop is as long as K whatever its shape, so with fewer
-  // tiles than SMs the time is one tile's time and smaller tiles are shorter ones.
+  // Few rows (a staged window late in a chain): with fewer tiles than SMs a launch takes one tile's time, which
+  // follows the operand bytes a CTA stages per K step: 32 KB for a 128 x 128 tile and for a CTA's half of a
+  // 256 x 256 pair tile, 48 KB for a 128 x 256 tile or a half of a 256 x 512 one. Up to one 128 x 128 block per SM
+  // the small tile puts every block on an SM of its own; above that the pair tile needs half the waves.
   const int64_t units = ((int64_t)g.rows_host + BM - 1) / BM * (g.N / 128);   // 128 x 128 blocks of the output
-  const bool few = units < 2 * 148;
-  const bool wide = (g.N % 256) == 0 && !(few && units < 148);
-  const bool pair = wide && g.pair != 0 && !few;
+  const bool few = units <= 148;
+  const bool wide = (g.N % 256) == 0 && !few;
+  const bool pair = wide && g.pair != 0;
   const int tm = pair ? 2 * BM : BM;
   const int m_tiles = (g.rows_host + tm - 1) / tm;
   int tiles = m_tiles * (g.N / (wide ? 256 : 128));
