@@ -355,3 +355,20 @@ def test_staged_windows_on_the_tensor_core_targets(kind, d, L, B):
             if stage == L:
                 assert np.array_equal(got[1], ref[1]) and np.array_equal(got[2], ref[2])
     s.close()
+
+
+@pytest.mark.parametrize("name", ["cfg3", "cfg4"])
+def test_full_size_staged_run_gives_the_samples_of_whole_windows(name):
+    """The bench configurations at full size, stage length chosen by the library: final states bit for bit those
+    of whole windows, fewer target rows, and the counters add up (every chain took K steps)."""
+    import torch
+    w = wl.WORKLOADS[name]
+    s = sds.sampler_for(w, **({"mlp": w.mlp_params()} if w.denoiser == "mlp" else {"gmm": w.gmm_params()}), seed=w.sample_seed)
+    ref = [x.clone() for x in s.sample_all()]
+    s.set_option(s.OPT_STAGED_WINDOWS, s.STAGED_ADAPTIVE)
+    got = s.sample_all()
+    assert torch.equal(got[0], ref[0])
+    assert int(got[2].sum()) < int(ref[2].sum()) and int(got[1].sum()) >= int(ref[1].sum())
+    assert np.array_equal(s.get(sb.GET_N), np.full(w.B, w.K))
+    assert int(s.get(sb.GET_CTL)[7]) > 0
+    s.close()
