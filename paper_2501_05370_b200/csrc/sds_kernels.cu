@@ -968,6 +968,197 @@ __global__ void __launch_bounds__(TPC > kBlock ? TPC : kBlock) k_verify_reg(WinA
   if (A.fuse_advance) window_tail(A, n_active);
 }
 
+// Rows read back, every position of the window evaluated, the advance step included: the kernel for windows in
+// which most drafts pass (long rows, one chain per CTA of TPC threads). One sweep over the positions with no
+// barrier and no decision in between (the accept tests of all positions are taken together afterwards), and
+// nothing but the carried output, the previous state and one position's pieces live in it: a bare kernel with
+// these loads and this arithmetic streams at 6.7 TB/s on this part, which the general kernel, with its blocks of
+// positions and the registers its other cases need, does not reach. Same per-thread order of the elements, same
+// shuffle tree and same order of the warps' sums as verify_reg_chain: same bits.
+template <int TPC, int EPT>
+__global__ void __launch_bounds__(TPC) k_verify_all(WinArgs A) {
+  constexpr int kWarps = TPC / 32;
+  __shared__ double s_red[2 * kMaxL * kWarps];
+  __shared__ int s_jstar;
+  __shared__ float s_coef;
+  const int s = blockIdx.x, t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  const int n_active = A.ctl[kCtlNActive];
+  if (s >= n_active) {
+    window_tail(A, n_active);
+    return;
+  }
+  const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
+  const int left = window_left(A, b, nb);
+  const int Lt = A.staged ? min(left, A.cap) : left;
+  const bool more = Lt < left;                             // staged window: positions remain after this launch's
+  const uint64_t bg = A.chain_off + (uint64_t)b;
+  const size_t cb = (size_t)b * A.d;
+  const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+  // which rows are rows of the means table (one-hot rows of skipped blocks): lane j-1 looks up position j
+  int comp_lane = -1;
+  if (lane < Lt) comp_lane = raw_row_component(A, r0 + lane);
+  {
+    float4 vc[EPT], vp[EPT];
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) {
+      const int i = (t + e * TPC) * 4;
+      vc[e] = (i < A.d) ? ld4(A.Dc + cb + i) : zero4;
+      vp[e] = (i < A.d) ? ld4(A.X + (size_t)r0 * A.d + i) : zero4;   // W_0 = Y_n
+    }
+    for (int j = 1; j <= Lt; ++j) {
+      const int k = nb + j - 1;
+      const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
+      const float inv_s = 1.0f / sk, cs = ck * inv_s;
+      const float* wj = (j < Lt) ? A.X + (size_t)(r0 + j) * A.d : A.T + cb;
+      const int qcomp = __shfl_sync(0xffffffffu, comp_lane, j - 1);
+      float4 vj[EPT], vq[EPT];
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) {
+        const int i = (t + e * TPC) * 4;
+        vj[e] = (i < A.d) ? ld4(wj + i) : zero4;
+        vq[e] = (i < A.d) ? raw_row4(A, r0 + j - 1, qcomp, i) : zero4;
+      }
+      if (A.raw_ce) {
+        const float2 ce = __ldg(A.raw_ce + k);
+#pragma unroll
+        for (int e = 0; e < EPT; ++e) vq[e] = affine_row4(ce.x, ce.y, vq[e], vp[e]);
+      }
+      double p1 = 0.0, p2 = 0.0;
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) {
+        const float4 w = vj[e];
+        if ((t + e * TPC) * 4 < A.d) {
+          float D, Z;
+          delta_z(vp[e].x, w.x, vq[e].x, vc[e].x, ak, ck, cs, inv_s, D, Z);
+          p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+          delta_z(vp[e].y, w.y, vq[e].y, vc[e].y, ak, ck, cs, inv_s, D, Z);
+          p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+          delta_z(vp[e].z, w.z, vq[e].z, vc[e].z, ak, ck, cs, inv_s, D, Z);
+          p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+          delta_z(vp[e].w, w.w, vq[e].w, vc[e].w, ak, ck, cs, inv_s, D, Z);
+          p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+        }
+        vp[e] = w;
+      }
+      p1 = warp_sum(p1);
+      p2 = warp_sum(p2);
+      if (lane == 0) {
+        s_red[(j - 1) * kWarps + warp] = p1;
+        s_red[kMaxL * kWarps + (j - 1) * kWarps + warp] = p2;
+      }
+    }
+  }
+  __syncthreads();
+  if (warp == 0) {                                         // the accept tests of all positions, one per lane
+    double myS1 = 0.0, myS2 = 0.0;
+    bool acc = true, bad = false;
+    const bool mine = lane < Lt;
+    if (mine) {
+      for (int w = 0; w < kWarps; ++w) {
+        myS1 += s_red[lane * kWarps + w];
+        myS2 += s_red[kMaxL * kWarps + lane * kWarps + w];
+      }
+      const float U = uniform01(A.seed, bg, (uint32_t)(nb + lane));
+      const float lu = logf(U);
+      const float ellf = (float)((-0.5 * myS1 - myS2) * A.inv_tau);
+      acc = (myS1 < 1e-30) || (lu <= ellf);
+      bad = !isfinite(ellf);
+      const size_t o = (size_t)b * A.L + lane;
+      A.S1[o] = myS1;
+      A.S2[o] = myS2;
+      A.ell[o] = ellf;
+      A.logU[o] = lu;
+    }
+    const uint32_t vmask = (Lt >= 32) ? 0xffffffffu : ((1u << Lt) - 1u);
+    const uint32_t am = __ballot_sync(0xffffffffu, acc) & vmask;
+    const uint32_t bm = __ballot_sync(0xffffffffu, bad) & vmask;
+    const uint32_t rej = ~am & vmask;
+    int jstar = Lt + 1;
+    float coef = 0.f;
+    if (rej) {
+      jstar = __ffs(rej);
+      coef = __shfl_sync(0xffffffffu, (float)(2.0 * myS2 / myS1), jstar - 1);
+    }
+    if (bm) jstar = -1;                                    // non-finite log ratio
+    if (lane == 0) {
+      A.accmask[b] = am;
+      A.jstar[b] = jstar;
+      atomicAdd(A.ctl + kCtlPositions, Lt);
+      if (bm) atomicOr(A.ctl + kCtlError, kErrNonFinite);
+      s_jstar = jstar;
+      s_coef = coef;
+    }
+  }
+  __syncthreads();
+  const int jstar = s_jstar;
+  const float coef = s_coef;
+  if (jstar < 1 || jstar > Lt) {
+    if (jstar >= 1) {                                      // every draft accepted: the window's last state and output carry on
+      const int qc = more ? -1 : __shfl_sync(0xffffffffu, comp_lane, Lt - 1);
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) {
+        const int i = (t + e * TPC) * 4;
+        if (i < A.d) {
+          st4(A.Y + cb + i, ld4(A.T + cb + i));
+          if (more) continue;                              // the window goes on: the carried output stays frozen
+          float4 q = raw_row4(A, r0 + Lt - 1, qc, i);
+          if (A.raw_ce) {
+            const float2 ce = __ldg(A.raw_ce + nb + Lt - 1);
+            q = affine_row4(ce.x, ce.y, q, ld4(A.X + (size_t)(r0 + Lt - 1) * A.d + i));
+          }
+          st4(A.Dc + cb + i, q);
+        }
+      }
+      if (t == 0) {
+        A.n[b] = nb + Lt;
+        if (A.staged) {
+          A.rem[b] = left - Lt;
+          atomicAdd(A.ctl + kCtlStagePassed, 1);
+        }
+        count_window(A, b, Lt);
+      }
+    } else if (t == 0) {                                   // non-finite log ratio: stop this chain
+      A.n[b] = A.K;
+      if (A.staged) A.rem[b] = 0;
+      atomicAdd(A.ctl + kCtlFrozen, 1);
+    }
+  } else {
+    const int k = nb + jstar - 1;
+    const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
+    const float inv_s = 1.0f / sk, cs = ck * inv_s;
+    const float* wp = A.X + (size_t)(r0 + jstar - 1) * A.d;
+    float* wj = (jstar < Lt) ? A.X + (size_t)(r0 + jstar) * A.d : A.T + cb;
+    const int rcomp = __shfl_sync(0xffffffffu, comp_lane, jstar - 1);
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) {
+      const int i = (t + e * TPC) * 4;
+      if (i < A.d) {
+        const float4 p = ld4(wp + i), w = ld4(wj + i), c4 = ld4(A.Dc + cb + i);
+        float4 q = raw_row4(A, r0 + jstar - 1, rcomp, i);
+        if (A.raw_ce) {
+          const float2 ce = __ldg(A.raw_ce + k);
+          q = affine_row4(ce.x, ce.y, q, p);
+        }
+        float4 o;
+        float D, Z;
+        delta_z(p.x, w.x, q.x, c4.x, ak, ck, cs, inv_s, D, Z); o.x = reflect_elem(p.x, q.x, Z, D, ak, ck, sk, coef);
+        delta_z(p.y, w.y, q.y, c4.y, ak, ck, cs, inv_s, D, Z); o.y = reflect_elem(p.y, q.y, Z, D, ak, ck, sk, coef);
+        delta_z(p.z, w.z, q.z, c4.z, ak, ck, cs, inv_s, D, Z); o.z = reflect_elem(p.z, q.z, Z, D, ak, ck, sk, coef);
+        delta_z(p.w, w.w, q.w, c4.w, ak, ck, cs, inv_s, D, Z); o.w = reflect_elem(p.w, q.w, Z, D, ak, ck, sk, coef);
+        st4(wj + i, o);
+        st4(A.Y + cb + i, o);                              // the reflected state is the next state; its target row carries on
+        st4(A.Dc + cb + i, q);
+      }
+    }
+    if (t == 0) {
+      A.n[b] = nb + jstar;
+      if (A.staged) A.rem[b] = 0;                          // a rejection ends the window
+      count_window(A, b, Lt);
+    }
+  }
+  window_tail(A, n_active);
+}
+
 // ---------------------------------------------------------------------------------------
 // C1 advance: Y <- W_adv, carried output <- target row adv, n += adv, counters; the CTA that
 // finishes last rebuilds the active list
@@ -1134,6 +1325,13 @@ cudaError_t launch_picard_draft(const WinArgs& A, int ub, cudaStream_t st) {
 template <int TPC, int EPT>
 cudaError_t launch_verify_reg(const WinArgs& A, int chains, cudaStream_t st) {
   if (!A.regen) {
+    if constexpr (TPC >= 1024) {
+      // every position evaluated and the advance step inside: the one-sweep kernel
+      if (!A.early_exit && A.fuse_advance && !A.Dp) {
+        k_verify_all<TPC, EPT><<<chains, TPC, 0, st>>>(A);
+        return cudaGetLastError();
+      }
+    }
     k_verify_reg<TPC, EPT, false><<<chains, TPC, 0, st>>>(A);
     return cudaGetLastError();
   }
