@@ -1159,6 +1159,148 @@ __global__ void __launch_bounds__(TPC) k_verify_all(WinArgs A) {
   window_tail(A, n_active);
 }
 
+// A stage of ONE position per chain (staged windows late in a chain), drafted state made again, advance included:
+// everything a chain needs stays in registers (state, carried output, the drafted state, the target row), there
+// is no block structure, no copy of the front state and nothing to draw twice. Same element order, shuffle tree
+// and order of the warps' sums as verify_reg_chain, and its formulas for the test and the reflection: same bits.
+template <int TPC, int EPT>
+__global__ void __launch_bounds__(TPC) k_verify_one(WinArgs A) {
+  constexpr int kWarps = TPC / 32;
+  __shared__ double s_red[2 * kWarps];
+  __shared__ int s_acc;
+  __shared__ float s_coef;
+  const int s = blockIdx.x, t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  const int n_active = A.ctl[kCtlNActive];
+  if (s >= n_active) {
+    window_tail(A, n_active);
+    return;
+  }
+  const int b = A.act[s], r0 = A.rowoff[s], nb = A.n[b];
+  const int left = window_left(A, b, nb);                  // (the stage itself is one position: cap == 1)
+  const bool more = 1 < left;
+  const uint64_t bg = A.chain_off + (uint64_t)b;
+  const size_t cb = (size_t)b * A.d;
+  const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+  const int k = nb;
+  const float ak = __ldg(A.a + k), ck = __ldg(A.c + k), sk = __ldg(A.sigma + k);
+  const float inv_s = 1.0f / sk, cs = ck * inv_s;
+  const int qcomp = raw_row_component(A, r0);
+  // (1024 threads of four slots each: the target row does not fit beside the other three arrays in 64 registers;
+  // the tail reads it a second time, from L2)
+  constexpr bool KEEPQ = !(TPC >= 1024 && EPT >= 4);
+  float4 vc[EPT], vp[EPT], vw[EPT], vq[EPT];
+  auto target_row = [&](int e) -> float4 {
+    const int i = (t + e * TPC) * 4;
+    float4 q = (i < A.d) ? raw_row4(A, r0, qcomp, i) : zero4;
+    if (A.raw_ce) {
+      const float2 ce = __ldg(A.raw_ce + k);
+      q = affine_row4(ce.x, ce.y, q, vp[e]);
+    }
+    return q;
+  };
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) {
+    const int i = (t + e * TPC) * 4;
+    vc[e] = (i < A.d) ? ld4(A.Dc + cb + i) : zero4;
+    vp[e] = (i < A.d) ? ld4(A.Y + cb + i) : zero4;          // W_0 = Y_n
+  }
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) vq[e] = target_row(e);
+  double p1 = 0.0, p2 = 0.0;
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) {
+    const float4 w = draft_step4(vp[e], vc[e], normal4(A.seed, kStreamDraft, bg, (uint32_t)k, (uint32_t)(t + e * TPC)), ak, ck, sk);
+    if ((t + e * TPC) * 4 < A.d) {
+      float D, Z;
+      delta_z(vp[e].x, w.x, vq[e].x, vc[e].x, ak, ck, cs, inv_s, D, Z);
+      p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+      delta_z(vp[e].y, w.y, vq[e].y, vc[e].y, ak, ck, cs, inv_s, D, Z);
+      p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+      delta_z(vp[e].z, w.z, vq[e].z, vc[e].z, ak, ck, cs, inv_s, D, Z);
+      p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+      delta_z(vp[e].w, w.w, vq[e].w, vc[e].w, ak, ck, cs, inv_s, D, Z);
+      p1 = fma((double)D, (double)D, p1); p2 = fma((double)D, (double)Z, p2);
+    }
+    vw[e] = w;
+  }
+  p1 = warp_sum(p1);
+  p2 = warp_sum(p2);
+  if (lane == 0) {
+    s_red[warp] = p1;
+    s_red[kWarps + warp] = p2;
+  }
+  __syncthreads();
+  if (t == 0) {
+    double myS1 = 0.0, myS2 = 0.0;
+    for (int w = 0; w < kWarps; ++w) {
+      myS1 += s_red[w];
+      myS2 += s_red[kWarps + w];
+    }
+    const float lu = logf(uniform01(A.seed, bg, (uint32_t)nb));
+    const float ellf = (float)((-0.5 * myS1 - myS2) * A.inv_tau);
+    const bool acc = (myS1 < 1e-30) || (lu <= ellf);
+    const bool bad = !isfinite(ellf);
+    const size_t o = (size_t)b * A.L;
+    A.S1[o] = myS1;
+    A.S2[o] = myS2;
+    A.ell[o] = ellf;
+    A.logU[o] = lu;
+    const int jstar = bad ? -1 : (acc ? 2 : 1);
+    A.accmask[b] = acc ? 1u : 0u;
+    A.jstar[b] = jstar;
+    atomicAdd(A.ctl + kCtlPositions, 1);
+    atomicAdd(A.ctl + kCtlPositionsRegen, 1);
+    if (bad) atomicOr(A.ctl + kCtlError, kErrNonFinite);
+    s_acc = jstar;
+    s_coef = acc ? 0.f : (float)(2.0 * myS2 / myS1);
+  }
+  __syncthreads();
+  const int jstar = s_acc;
+  const float coef = s_coef;
+  if (jstar == 2) {                                        // accepted: the drafted state is the next state
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) {
+      const int i = (t + e * TPC) * 4;
+      if (i < A.d) {
+        st4(A.Y + cb + i, vw[e]);
+        if (!more) st4(A.Dc + cb + i, KEEPQ ? vq[e] : target_row(e));   // the window ends here: its target row carries on
+      }
+    }
+    if (t == 0) {
+      A.n[b] = nb + 1;
+      A.rem[b] = left - 1;
+      atomicAdd(A.ctl + kCtlStagePassed, 1);
+      count_window(A, b, 1);
+    }
+  } else if (jstar == 1) {                                 // rejected: the reflected state, and the window ends
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) {
+      const int i = (t + e * TPC) * 4;
+      if (i < A.d) {
+        const float4 p = vp[e], w = vw[e], q = KEEPQ ? vq[e] : target_row(e), c4 = vc[e];
+        float4 o;
+        float D, Z;
+        delta_z(p.x, w.x, q.x, c4.x, ak, ck, cs, inv_s, D, Z); o.x = reflect_elem(p.x, q.x, Z, D, ak, ck, sk, coef);
+        delta_z(p.y, w.y, q.y, c4.y, ak, ck, cs, inv_s, D, Z); o.y = reflect_elem(p.y, q.y, Z, D, ak, ck, sk, coef);
+        delta_z(p.z, w.z, q.z, c4.z, ak, ck, cs, inv_s, D, Z); o.z = reflect_elem(p.z, q.z, Z, D, ak, ck, sk, coef);
+        delta_z(p.w, w.w, q.w, c4.w, ak, ck, cs, inv_s, D, Z); o.w = reflect_elem(p.w, q.w, Z, D, ak, ck, sk, coef);
+        st4(A.Y + cb + i, o);
+        st4(A.Dc + cb + i, q);
+      }
+    }
+    if (t == 0) {
+      A.n[b] = nb + 1;
+      A.rem[b] = 0;
+      count_window(A, b, 1);
+    }
+  } else if (t == 0) {                                     // non-finite log ratio: stop this chain
+    A.n[b] = A.K;
+    A.rem[b] = 0;
+    atomicAdd(A.ctl + kCtlFrozen, 1);
+  }
+  window_tail(A, n_active);
+}
+
 // ---------------------------------------------------------------------------------------
 // C1 advance: Y <- W_adv, carried output <- target row adv, n += adv, counters; the CTA that
 // finishes last rebuilds the active list
@@ -1336,6 +1478,10 @@ cudaError_t launch_verify_reg(const WinArgs& A, int chains, cudaStream_t st) {
     return cudaGetLastError();
   }
   if (!A.fuse_advance) return cudaErrorInvalidValue;     // the regenerated states exist only in this kernel: it must advance
+  if (A.staged && A.cap == 1) {                          // every chain's stage is one position
+    k_verify_one<TPC, EPT><<<chains, TPC, 0, st>>>(A);
+    return cudaGetLastError();
+  }
   const size_t smem = (size_t)A.d * sizeof(float);
   if (smem + 2 * kMaxL * (TPC / 32) * sizeof(double) + 64 > 48 * 1024) {   // the kernel's own shared arrays count too
     const cudaError_t e = cudaFuncSetAttribute(k_verify_reg<TPC, EPT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
